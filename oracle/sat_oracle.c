@@ -1,0 +1,364 @@
+/*
+ * CPU oracle for the SAT (staleness-alleviated training) partition-parallel GCN step.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the plain, slow, obviously-correct statement
+ * of what the hot path computes; the tests, the smoke check and the benchmark's CPU
+ * baseline leg are its only users.  It shares no code with the CUDA library and the
+ * CUDA library never calls it.
+ *
+ * Conventions
+ *   - every sum is accumulated in double precision in the order the formula is
+ *     written (row by row, neighbour by neighbour, k ascending);
+ *   - inputs that the method stores as fp32 (features, cached embeddings, weights,
+ *     gradients handed from layer to layer) are read as fp32; results are rounded to
+ *     fp32 only where the method itself stores them (layer outputs, cache entries,
+ *     predictor state and output, gradients);
+ *   - `omp parallel for` appears only over independent output rows / columns, so the
+ *     summation order of every output element is fixed.
+ *
+ * Notation follows the paper: P = propagation matrix of GCN (Appendix, Preliminaries),
+ * P = P_in + P_out per partition, H_in / H_out(halo) in- and out-of-subgraph
+ * embeddings (Eq. "matrix form forward"), D = G o sigma'(Z), G_W, G_H (Appendix,
+ * backward equations), S / C = LSTM hidden state / memory cell and
+ * dH = GCN(S, A) (Section "Embedding Predictor").
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-1  Propagation matrix of GCN with self-loops (Appendix, Preliminaries: "P is the
+ * propagation matrix following the definition of GCN"):
+ *     P = D~^{-1/2} (A + I) D~^{-1/2},   d~_v = deg(v) + 1,
+ *     p_vu = 1 / sqrt(d~_v d~_u)  for u in N(v) or u == v.
+ * `dtil` holds the integers d~_v.
+ * ---------------------------------------------------------------------------------- */
+static inline double p_entry(int32_t dt_v, int32_t dt_u)
+{
+    return 1.0 / sqrt((double)dt_v * (double)dt_u);
+}
+
+void orc_degrees(int32_t n, const int64_t *rowptr, int32_t *dtil, float *dinv)
+{
+    for (int32_t v = 0; v < n; ++v) {
+        dtil[v] = (int32_t)(rowptr[v + 1] - rowptr[v]) + 1;
+        dinv[v] = (float)(1.0 / sqrt((double)dtil[v]));
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-6  Layer forward for partition m (Appendix, forward of SAT; Eq. "sat forward"):
+ *     AGG = P_in H_in + P_out H_halo            (one pass over the local CSR)
+ *     Z   = AGG W + b
+ *     H   = ReLU(Z)  (act = 1)   or   H = Z  (act = 0)
+ * Local CSR: rows = inner nodes of m, columns are local ids: c < n_in is inner node c,
+ * c >= n_in is halo node c - n_in; the self-loop is an explicit entry.
+ * rows_sel (may be NULL = all rows) restricts the computation to a sample of rows;
+ * outputs are always addressed by the full row id.
+ * AGG and Z are kept in double (the method never exposes them); H is the fp32 layer
+ * output.
+ * ---------------------------------------------------------------------------------- */
+void orc_layer_fwd(int32_t n_sel, const int32_t *rows_sel,
+                   int32_t n_in, const int64_t *lrowptr, const int32_t *lcol,
+                   const int32_t *inner_gid, const int32_t *halo_gid, const int32_t *dtil,
+                   int32_t d_in, int32_t d_out,
+                   const float *H_in, int64_t ld_in, const float *H_halo, int64_t ld_halo,
+                   const float *W, const float *bias, int32_t act,
+                   double *AGG /* [n_in x d_in] */, double *Z /* [n_in x d_out] */,
+                   float *H /* [n_in x ld_h] */, int64_t ld_h)
+{
+    int32_t count = rows_sel ? n_sel : n_in;
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int32_t i = 0; i < count; ++i) {
+        int32_t v = rows_sel ? rows_sel[i] : i;
+        double *agg = AGG + (int64_t)v * d_in;
+        for (int32_t k = 0; k < d_in; ++k) agg[k] = 0.0;
+        int32_t dt_v = dtil[inner_gid[v]];
+        for (int64_t e = lrowptr[v]; e < lrowptr[v + 1]; ++e) {
+            int32_t c = lcol[e];
+            const float *src;
+            int32_t dt_u;
+            if (c < n_in) {
+                src = H_in + (int64_t)c * ld_in;
+                dt_u = dtil[inner_gid[c]];
+            } else {
+                src = H_halo + (int64_t)(c - n_in) * ld_halo;
+                dt_u = dtil[halo_gid[c - n_in]];
+            }
+            double p = p_entry(dt_v, dt_u);
+            for (int32_t k = 0; k < d_in; ++k) agg[k] += p * (double)src[k];
+        }
+        double *z = Z + (int64_t)v * d_out;
+        for (int32_t j = 0; j < d_out; ++j) z[j] = 0.0;
+        for (int32_t k = 0; k < d_in; ++k) {
+            double a = agg[k];
+            const float *wrow = W + (int64_t)k * d_out;
+            for (int32_t j = 0; j < d_out; ++j) z[j] += a * (double)wrow[j];
+        }
+        float *h = H + (int64_t)v * ld_h;
+        for (int32_t j = 0; j < d_out; ++j) {
+            if (bias) z[j] += (double)bias[j];
+            double o = (act == 1 && !(z[j] > 0.0)) ? 0.0 : z[j];
+            h[j] = (float)o;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-9  Layer backward for partition m (Appendix, backward equations):
+ *     D     = G_out o [Z > 0]         (hidden layer; mask supplied as bytes)   or  D = G_out
+ *     G_W  += AGG^T D                  (G_W = (P H)^T D)
+ *     G_b  += column sums of D
+ *     G_AGG = D W^T
+ *     G_in  = P_in^T  G_AGG            (G_H = P^T D W^T restricted to inner columns: the
+ *                                       predicted halo embeddings are constants)
+ *     G_halo= P_out^T G_AGG            (optional; the part a gradient exchange would need)
+ * P^T is applied as a scatter over the same local CSR, row by row, so the order of
+ * additions into every output element is the row order.
+ * ---------------------------------------------------------------------------------- */
+void orc_layer_bwd(int32_t n_in, int32_t n_halo, const int64_t *lrowptr, const int32_t *lcol,
+                   const int32_t *inner_gid, const int32_t *halo_gid, const int32_t *dtil,
+                   int32_t d_in, int32_t d_out,
+                   const float *G_out, int64_t ld_g, const uint8_t *mask /* [n_in x d_out] or NULL */,
+                   const double *AGG, const float *W,
+                   double *G_W /* [d_in x d_out], += */, double *G_b /* [d_out], += */,
+                   float *G_in /* [n_in x ld_gin] or NULL */, int64_t ld_gin,
+                   float *G_halo /* [n_halo x ld_gh] or NULL */, int64_t ld_gh)
+{
+    double *D = (double *)malloc(sizeof(double) * (size_t)n_in * d_out);
+    double *GA = (double *)malloc(sizeof(double) * (size_t)n_in * d_in);
+#pragma omp parallel for
+    for (int32_t v = 0; v < n_in; ++v)
+        for (int32_t j = 0; j < d_out; ++j) {
+            double g = (double)G_out[(int64_t)v * ld_g + j];
+            if (mask && !mask[(int64_t)v * d_out + j]) g = 0.0;
+            D[(int64_t)v * d_out + j] = g;
+        }
+    /* G_W[k][j] += sum_v AGG[v][k] D[v][j], v ascending */
+#pragma omp parallel for
+    for (int32_t k = 0; k < d_in; ++k) {
+        double *gw = G_W + (int64_t)k * d_out;
+        for (int32_t v = 0; v < n_in; ++v) {
+            double a = AGG[(int64_t)v * d_in + k];
+            const double *drow = D + (int64_t)v * d_out;
+            for (int32_t j = 0; j < d_out; ++j) gw[j] += a * drow[j];
+        }
+    }
+#pragma omp parallel for
+    for (int32_t j = 0; j < d_out; ++j) {
+        double s = 0.0;
+        for (int32_t v = 0; v < n_in; ++v) s += D[(int64_t)v * d_out + j];
+        G_b[j] += s;
+    }
+    /* G_AGG[v][k] = sum_j D[v][j] W[k][j] */
+#pragma omp parallel for
+    for (int32_t v = 0; v < n_in; ++v)
+        for (int32_t k = 0; k < d_in; ++k) {
+            double s = 0.0;
+            const float *wrow = W + (int64_t)k * d_out;
+            const double *drow = D + (int64_t)v * d_out;
+            for (int32_t j = 0; j < d_out; ++j) s += drow[j] * (double)wrow[j];
+            GA[(int64_t)v * d_in + k] = s;
+        }
+    if (G_in || G_halo) {
+        int32_t n_tot = n_in + n_halo;
+        double *T = (double *)calloc((size_t)n_tot * d_in, sizeof(double));
+        /* scatter form of P^T: each thread owns a disjoint range of feature columns */
+#pragma omp parallel
+        {
+            int nt = 1, id = 0;
+#ifdef _OPENMP
+            nt = omp_get_num_threads();
+            id = omp_get_thread_num();
+#endif
+            int32_t k0 = (int32_t)((int64_t)d_in * id / nt), k1 = (int32_t)((int64_t)d_in * (id + 1) / nt);
+            if (k1 > k0)
+                for (int32_t v = 0; v < n_in; ++v) {
+                    int32_t dt_v = dtil[inner_gid[v]];
+                    const double *ga = GA + (int64_t)v * d_in;
+                    for (int64_t e = lrowptr[v]; e < lrowptr[v + 1]; ++e) {
+                        int32_t c = lcol[e];
+                        int32_t dt_u = c < n_in ? dtil[inner_gid[c]] : dtil[halo_gid[c - n_in]];
+                        double p = p_entry(dt_v, dt_u);
+                        double *t = T + (int64_t)c * d_in;
+                        for (int32_t k = k0; k < k1; ++k) t[k] += p * ga[k];
+                    }
+                }
+        }
+        if (G_in)
+            for (int32_t u = 0; u < n_in; ++u)
+                for (int32_t k = 0; k < d_in; ++k) G_in[(int64_t)u * ld_gin + k] = (float)T[(int64_t)u * d_in + k];
+        if (G_halo)
+            for (int32_t u = 0; u < n_halo; ++u)
+                for (int32_t k = 0; k < d_in; ++k)
+                    G_halo[(int64_t)u * ld_gh + k] = (float)T[(int64_t)(n_in + u) * d_in + k];
+        free(T);
+    }
+    free(D);
+    free(GA);
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-4  LSTM over the cached snapshots (Section "Embedding Predictor": the recurrent
+ * part of the RNN-GNN predictor iterates over epochs t-tau .. t-1).
+ * For every cached node (slot) w:  s = c = 0; for the k snapshots, oldest first:
+ *     a = x W_x + s U_h + b           (4h wide, gate order i, f, g, o)
+ *     i = sigm(a_i) f = sigm(a_f) g = tanh(a_g) o = sigm(a_o)
+ *     c = f o c + i o g ;  s = o o tanh(c)
+ * S_w = final s, stored fp32 (zeros when k == 0).
+ * snaps[t] is snapshot t (oldest = 0), each [n_slots x ld].
+ * ---------------------------------------------------------------------------------- */
+static inline double sigm(double x) { return 1.0 / (1.0 + exp(-x)); }
+
+void orc_lstm(int32_t n_sel, const int32_t *slots_sel, int32_t n_slots, int32_t k,
+              const float *const *snaps, int64_t ld, int32_t d, int32_t h,
+              const float *Wx /* [d x 4h] */, const float *Uh /* [h x 4h] */, const float *b /* [4h] */,
+              float *S /* [n_slots x h] */)
+{
+    int32_t count = slots_sel ? n_sel : n_slots;
+#pragma omp parallel
+    {
+        double *a = (double *)malloc(sizeof(double) * 4 * (size_t)h);
+        double *s = (double *)malloc(sizeof(double) * (size_t)h);
+        double *c = (double *)malloc(sizeof(double) * (size_t)h);
+#pragma omp for schedule(dynamic, 16)
+        for (int32_t idx = 0; idx < count; ++idx) {
+            int32_t w = slots_sel ? slots_sel[idx] : idx;
+            for (int32_t j = 0; j < h; ++j) s[j] = c[j] = 0.0;
+            for (int32_t t = 0; t < k; ++t) {
+                const float *x = snaps[t] + (int64_t)w * ld;
+                for (int32_t j = 0; j < 4 * h; ++j) a[j] = 0.0;
+                for (int32_t q = 0; q < d; ++q) {
+                    double xv = (double)x[q];
+                    const float *wr = Wx + (int64_t)q * 4 * h;
+                    for (int32_t j = 0; j < 4 * h; ++j) a[j] += xv * (double)wr[j];
+                }
+                for (int32_t q = 0; q < h; ++q) {
+                    double sv = s[q];
+                    const float *ur = Uh + (int64_t)q * 4 * h;
+                    for (int32_t j = 0; j < 4 * h; ++j) a[j] += sv * (double)ur[j];
+                }
+                for (int32_t j = 0; j < 4 * h; ++j) a[j] += (double)b[j];
+                for (int32_t j = 0; j < h; ++j) {
+                    double gi = sigm(a[j]), gf = sigm(a[h + j]), gg = tanh(a[2 * h + j]), go = sigm(a[3 * h + j]);
+                    c[j] = gf * c[j] + gi * gg;
+                    s[j] = go * tanh(c[j]);
+                }
+            }
+            for (int32_t j = 0; j < h; ++j) S[(int64_t)w * h + j] = (float)s[j];
+        }
+        free(a);
+        free(s);
+        free(c);
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-5  Graph convolution on the final LSTM state plus skip connection, for the halo
+ * rows of partition m (Section "Embedding Predictor": dH = GCN(S, A) on the 1-hop
+ * extended subgraph; the prediction corrects the newest cached embedding):
+ *     a_u   = p_uu S_u + sum_{v in N(u) cap V_m} p_uv S_v
+ *     dH_u  = a_u W_g + b_g
+ *     Hhat_u= Htilde_u(newest) + dH_u
+ * Halo-row CSR: row j = halo node j of m, columns = local inner ids of its neighbours
+ * inside m.  `newest` may be NULL (no committed snapshot: Htilde = 0).
+ * ---------------------------------------------------------------------------------- */
+void orc_predict_halo(int32_t n_sel, const int32_t *rows_sel,
+                      int32_t n_halo, const int64_t *hrow_ptr, const int32_t *hrow_col,
+                      const int32_t *inner_gid, const int32_t *halo_gid, const int32_t *slot,
+                      const int32_t *dtil, int32_t h, int32_t d,
+                      const float *S /* [n_slots x h] */, const float *newest, int64_t ld_new,
+                      const float *Wg /* [h x d] */, const float *bg /* [d] */,
+                      float *out /* [n_halo x ld_out] */, int64_t ld_out)
+{
+    int32_t count = rows_sel ? n_sel : n_halo;
+#pragma omp parallel
+    {
+        double *a = (double *)malloc(sizeof(double) * (size_t)h);
+#pragma omp for schedule(dynamic, 16)
+        for (int32_t idx = 0; idx < count; ++idx) {
+            int32_t j = rows_sel ? rows_sel[idx] : idx;
+            int32_t u = halo_gid[j];
+            int32_t dt_u = dtil[u];
+            const float *su = S + (int64_t)slot[u] * h;
+            double puu = p_entry(dt_u, dt_u);
+            for (int32_t q = 0; q < h; ++q) a[q] = puu * (double)su[q];
+            for (int64_t e = hrow_ptr[j]; e < hrow_ptr[j + 1]; ++e) {
+                int32_t v = inner_gid[hrow_col[e]];
+                double p = p_entry(dt_u, dtil[v]);
+                const float *sv = S + (int64_t)slot[v] * h;
+                for (int32_t q = 0; q < h; ++q) a[q] += p * (double)sv[q];
+            }
+            for (int32_t c = 0; c < d; ++c) {
+                double acc = 0.0;
+                for (int32_t q = 0; q < h; ++q) acc += a[q] * (double)Wg[(int64_t)q * d + c];
+                acc += (double)bg[c];
+                if (newest) acc += (double)newest[(int64_t)slot[u] * ld_new + c];
+                out[(int64_t)j * ld_out + c] = (float)acc;
+            }
+        }
+        free(a);
+    }
+}
+
+/* ------------------------------------------------------------------------------------
+ * O-8  Loss and its gradient with respect to the logits (Eq. "global loss" /
+ * Eq. "local loss": L = sum_m w_m (1/|V_m|) sum_{v in V_m} Loss(h_v, y_v); with
+ * w_m = |V_m| / N every node carries weight 1/N).
+ *   softmax cross-entropy:  Loss_v = -log softmax(z_v)[y_v];  dLoss/dz = softmax(z) - onehot(y)
+ *   sigmoid BCE (multi-label): Loss_v = (1/C) sum_c [softplus(z_c) - y_c z_c];
+ *                              dLoss/dz_c = (sigm(z_c) - y_c) / C
+ * Returns the sum over the given rows of scale * Loss_v; G = scale * dLoss/dz (fp32).
+ * ---------------------------------------------------------------------------------- */
+double orc_loss_ce(int32_t n, int32_t n_classes, const float *Z, int64_t ld_z, const int32_t *y,
+                   double scale, float *G, int64_t ld_g)
+{
+    double total = 0.0;
+    for (int32_t v = 0; v < n; ++v) {
+        const float *z = Z + (int64_t)v * ld_z;
+        double mx = (double)z[0];
+        for (int32_t c = 1; c < n_classes; ++c)
+            if ((double)z[c] > mx) mx = (double)z[c];
+        double se = 0.0;
+        for (int32_t c = 0; c < n_classes; ++c) se += exp((double)z[c] - mx);
+        double lse = mx + log(se);
+        total += scale * (lse - (double)z[y[v]]);
+        if (G)
+            for (int32_t c = 0; c < n_classes; ++c) {
+                double pr = exp((double)z[c] - lse);
+                G[(int64_t)v * ld_g + c] = (float)(scale * (pr - (c == y[v] ? 1.0 : 0.0)));
+            }
+    }
+    return total;
+}
+
+double orc_loss_bce(int32_t n, int32_t n_labels, const float *Z, int64_t ld_z, const uint8_t *Y,
+                    double scale, float *G, int64_t ld_g)
+{
+    double total = 0.0;
+    for (int32_t v = 0; v < n; ++v) {
+        const float *z = Z + (int64_t)v * ld_z;
+        double acc = 0.0;
+        for (int32_t c = 0; c < n_labels; ++c) {
+            double x = (double)z[c], yv = (double)Y[(int64_t)v * n_labels + c];
+            double sp = (x > 0.0 ? x : 0.0) + log1p(exp(-fabs(x))); /* softplus */
+            acc += sp - yv * x;
+            if (G) G[(int64_t)v * ld_g + c] = (float)(scale * (sigm(x) - yv) / (double)n_labels);
+        }
+        total += scale * acc / (double)n_labels;
+    }
+    return total;
+}

@@ -1,0 +1,368 @@
+"""CPU oracle of the SAT partition-parallel GCN epoch.  TEST INFRASTRUCTURE ONLY.
+
+The integer structures (partition lists, halo sets, cache slots) are written out from
+their definitions with numpy; the floating-point steps call the plain C loops of
+sat_oracle.c (double accumulation, formula order).  Nothing here is shared with, or
+imported by, the CUDA library.
+
+Paper passages followed (section / equation names of arXiv 2308.13466):
+  partition, non-overlapping subgraphs            Preliminaries, "Distributed Training for GNNs"
+  in- / out-of-subgraph neighbours                Eq. "mini-batch", Eq. "matrix form forward"
+  1-hop extended subgraph G-bar_m                 Section "Embedding Predictor", temporal graphs
+  halo set  U_{v in V_m} N(v) \\ V_m               Eq. "communication complexity"
+  historical embeddings, sliding window tau       Section "Problem Formulation"; Eq. "problem formulation"
+  predictor = LSTM + GCN, skip connection         Section "Embedding Predictor"
+  pull / forward / push / loss / gradients        Algorithm 1
+  layer forward / backward formulas               Appendix (forward and backward of SAT)
+"""
+from __future__ import annotations
+
+import ctypes as C
+from dataclasses import dataclass, field
+
+import numpy as np
+
+from .build import build_oracle
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build_oracle())
+        _lib.orc_loss_ce.restype = C.c_double
+        _lib.orc_loss_bce.restype = C.c_double
+        _lib.orc_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def _p(a, ctype=C.c_void_p):
+    if a is None:
+        return None
+    return a.ctypes.data_as(ctype)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+# --------------------------------------------------------------------------------------
+# O-1  degrees of A + I and D~^{-1/2}
+# --------------------------------------------------------------------------------------
+def degrees(rowptr: np.ndarray):
+    n = rowptr.shape[0] - 1
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    dtil = np.empty(n, dtype=np.int32)
+    dinv = np.empty(n, dtype=np.float32)
+    lib().orc_degrees(C.c_int32(n), _p(rowptr), _p(dtil), _p(dinv))
+    return dtil, dinv
+
+
+# --------------------------------------------------------------------------------------
+# O-2  partition structures
+# --------------------------------------------------------------------------------------
+def contig_blocks(n: int, M: int) -> np.ndarray:
+    """Contiguous id blocks: part[v] = floor(v * M / n)."""
+    return (np.arange(n, dtype=np.int64) * M // n).astype(np.int32)
+
+
+@dataclass
+class Partitioning:
+    n: int
+    M: int
+    part: np.ndarray
+    slot: np.ndarray                       # int32 [n]: rank in C (sorted union of all halo sets) or -1
+    n_slots: int
+    inner_gid: list = field(default_factory=list)   # I_m, ascending global ids
+    halo_gid: list = field(default_factory=list)    # B_m, ascending global ids
+    loc_rowptr: list = field(default_factory=list)  # local CSR over rows I_m, int64
+    loc_col: list = field(default_factory=list)     # local column ids (inner < n_m <= halo), ascending per row
+    hrow_ptr: list = field(default_factory=list)    # halo-row CSR (rows B_m), int64
+    hrow_col: list = field(default_factory=list)    # local inner ids of the neighbours inside m, ascending
+    halo_slot: list = field(default_factory=list)   # slot[B_m]
+    push_local: list = field(default_factory=list)  # local ids of inner nodes that are in C, ascending
+    push_slot: list = field(default_factory=list)   # their slots
+
+
+def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: int) -> Partitioning:
+    """All per-partition lists, from their definitions.
+
+    I_m = {v : part[v] = m};  B_m = sorted unique { u not in V_m : exists v in V_m, (v,u) in E };
+    local CSR: rows I_m, entries N(v) + {v}, columns renamed to local ids (inner: rank in
+    I_m; halo: n_m + rank in B_m) and sorted ascending; halo-row CSR: for u in B_m the
+    neighbours of u inside V_m (the transpose of the halo block); C = sorted union of the
+    B_m, slot = rank in C; push list = inner nodes of m that are in C.
+    """
+    n = rowptr.shape[0] - 1
+    part = np.ascontiguousarray(part, dtype=np.int32)
+    deg = np.diff(rowptr)
+    P = Partitioning(n=n, M=M, part=part, slot=None, n_slots=0)
+    in_any_halo = np.zeros(n, dtype=bool)
+    per = []
+    for m in range(M):
+        inner = np.nonzero(part == m)[0].astype(np.int64)
+        n_m = inner.shape[0]
+        loc_of = np.full(n, -1, dtype=np.int64)
+        loc_of[inner] = np.arange(n_m)
+        d_m = deg[inner]
+        src = np.repeat(np.arange(n_m, dtype=np.int64), d_m)
+        # positions of the rows of I_m inside the global col array
+        starts = np.repeat(rowptr[inner] - np.concatenate([[0], np.cumsum(d_m)[:-1]]), d_m)
+        dst = col[starts + np.arange(src.shape[0], dtype=np.int64)].astype(np.int64)
+        outside = part[dst] != m
+        halo = np.unique(dst[outside])
+        in_any_halo[halo] = True
+        # add the self-loop of every inner row
+        src2 = np.concatenate([src, np.arange(n_m, dtype=np.int64)])
+        dst2 = np.concatenate([dst, inner])
+        out2 = np.concatenate([outside, np.zeros(n_m, dtype=bool)])
+        lid = np.where(out2, n_m + np.searchsorted(halo, dst2), loc_of[dst2])
+        order = np.lexsort((lid, src2))
+        loc_col = lid[order].astype(np.int32)
+        loc_rowptr = np.zeros(n_m + 1, dtype=np.int64)
+        np.cumsum(np.bincount(src2, minlength=n_m), out=loc_rowptr[1:])
+        # halo-row CSR = cut edges regrouped by halo node
+        hs = np.searchsorted(halo, dst[outside])
+        hv = src[outside]
+        o2 = np.lexsort((hv, hs))
+        hrow_col = hv[o2].astype(np.int32)
+        hrow_ptr = np.zeros(halo.shape[0] + 1, dtype=np.int64)
+        np.cumsum(np.bincount(hs, minlength=halo.shape[0]), out=hrow_ptr[1:])
+        per.append((inner.astype(np.int32), halo.astype(np.int32), loc_rowptr, loc_col, hrow_ptr, hrow_col))
+    Cset = np.nonzero(in_any_halo)[0]
+    slot = np.full(n, -1, dtype=np.int32)
+    slot[Cset] = np.arange(Cset.shape[0], dtype=np.int32)
+    P.slot, P.n_slots = slot, int(Cset.shape[0])
+    for inner, halo, lrp, lc, hp, hc in per:
+        P.inner_gid.append(inner)
+        P.halo_gid.append(halo)
+        P.loc_rowptr.append(lrp)
+        P.loc_col.append(lc)
+        P.hrow_ptr.append(hp)
+        P.hrow_col.append(hc)
+        P.halo_slot.append(slot[halo])
+        pl = np.nonzero(slot[inner] >= 0)[0].astype(np.int32)
+        P.push_local.append(pl)
+        P.push_slot.append(slot[inner[pl]])
+    return P
+
+
+# --------------------------------------------------------------------------------------
+# O-3  historical-embedding cache: ring of tau readable snapshots + 1 write buffer
+# --------------------------------------------------------------------------------------
+class CacheRing:
+    """Per cached layer l (embeddings H^(l), l = 1..L-1) a ring of tau+1 buffers over the
+    |C| boundary nodes.  Reads during an epoch see only committed snapshots (at most the
+    tau newest); pushes of the running epoch go to the write buffer, which becomes the
+    newest snapshot at commit.  Initially everything is zero and no snapshot is valid."""
+
+    def __init__(self, n_slots: int, widths, tau: int):
+        self.tau = tau
+        self.n_slots = n_slots
+        self.widths = list(widths)
+        self.buf = [np.zeros((tau + 1, n_slots, w), dtype=np.float32) for w in widths]
+        self.write_idx = 0
+        self.n_valid = 0
+
+    def snapshots(self, layer: int):
+        """Valid snapshots of cached layer `layer` (1-based), oldest first."""
+        k = min(self.n_valid, self.tau)
+        idx = [(self.write_idx - 1 - a) % (self.tau + 1) for a in range(k - 1, -1, -1)]
+        return [self.buf[layer - 1][i] for i in idx]
+
+    def newest(self, layer: int):
+        s = self.snapshots(layer)
+        return s[-1] if s else None
+
+    def push(self, layer: int, slots: np.ndarray, rows: np.ndarray):
+        self.buf[layer - 1][self.write_idx][slots] = rows
+
+    def commit(self):
+        self.write_idx = (self.write_idx + 1) % (self.tau + 1)
+        self.n_valid = min(self.n_valid + 1, self.tau)
+
+
+# --------------------------------------------------------------------------------------
+# O-4 / O-5  predictor
+# --------------------------------------------------------------------------------------
+def lstm_state(snaps, d: int, h: int, Wx, Uh, b, n_slots: int, slots_sel=None) -> np.ndarray:
+    """Final LSTM hidden state S [n_slots, h] over the snapshots (oldest first)."""
+    k = len(snaps)
+    S = np.zeros((n_slots, h), dtype=np.float32)
+    if k == 0:
+        return S
+    snaps = [_f32(s) for s in snaps]
+    ld = snaps[0].shape[1]
+    arr = (C.c_void_p * k)(*[s.ctypes.data for s in snaps])
+    Wx, Uh, b = _f32(Wx), _f32(Uh), _f32(b)
+    sel = None if slots_sel is None else np.ascontiguousarray(slots_sel, dtype=np.int32)
+    lib().orc_lstm(C.c_int32(0 if sel is None else sel.shape[0]), _p(sel), C.c_int32(n_slots), C.c_int32(k),
+                   arr, C.c_int64(ld), C.c_int32(d), C.c_int32(h), _p(Wx), _p(Uh), _p(b), _p(S))
+    return S
+
+
+def predict_halo(P: Partitioning, m: int, dtil, S, newest, Wg, bg, rows_sel=None) -> np.ndarray:
+    """Predicted halo embeddings of partition m: newest snapshot + GCN(S) (skip connection)."""
+    h, d = Wg.shape
+    nh = P.halo_gid[m].shape[0]
+    out = np.zeros((nh, d), dtype=np.float32)
+    sel = None if rows_sel is None else np.ascontiguousarray(rows_sel, dtype=np.int32)
+    S = _f32(S)
+    newest = None if newest is None else _f32(newest)
+    Wg, bg = _f32(Wg), _f32(bg)
+    lib().orc_predict_halo(C.c_int32(0 if sel is None else sel.shape[0]), _p(sel),
+                           C.c_int32(nh), _p(P.hrow_ptr[m]), _p(P.hrow_col[m]),
+                           _p(P.inner_gid[m]), _p(P.halo_gid[m]), _p(P.slot), _p(dtil),
+                           C.c_int32(h), C.c_int32(d), _p(S), _p(newest),
+                           C.c_int64(0 if newest is None else newest.shape[1]),
+                           _p(Wg), _p(bg), _p(out), C.c_int64(d))
+    return out
+
+
+def historical_halo(P: Partitioning, m: int, newest, d: int) -> np.ndarray:
+    """Identity predictor: the plain historical embedding (newest snapshot, zeros if none)."""
+    nh = P.halo_gid[m].shape[0]
+    if newest is None:
+        return np.zeros((nh, d), dtype=np.float32)
+    return np.ascontiguousarray(newest[P.halo_slot[m]], dtype=np.float32)
+
+
+# --------------------------------------------------------------------------------------
+# O-6  layer forward,  O-9  layer backward,  O-8  loss
+# --------------------------------------------------------------------------------------
+def layer_fwd(P: Partitioning, m: int, dtil, H_in, H_halo, W, bias, act: int, rows_sel=None):
+    """Returns (AGG float64 [n_m, d_in], Z float64 [n_m, d_out], H fp32 [n_m, d_out])."""
+    n_in = P.inner_gid[m].shape[0]
+    d_in, d_out = W.shape
+    H_in, H_halo, W = _f32(H_in), _f32(H_halo), _f32(W)
+    bias = None if bias is None else _f32(bias)
+    if H_halo.shape[0] == 0:
+        H_halo = np.zeros((1, d_in), dtype=np.float32)
+    AGG = np.zeros((n_in, d_in), dtype=np.float64)
+    Z = np.zeros((n_in, d_out), dtype=np.float64)
+    H = np.zeros((n_in, d_out), dtype=np.float32)
+    sel = None if rows_sel is None else np.ascontiguousarray(rows_sel, dtype=np.int32)
+    lib().orc_layer_fwd(C.c_int32(0 if sel is None else sel.shape[0]), _p(sel),
+                        C.c_int32(n_in), _p(P.loc_rowptr[m]), _p(P.loc_col[m]),
+                        _p(P.inner_gid[m]), _p(P.halo_gid[m]), _p(dtil),
+                        C.c_int32(d_in), C.c_int32(d_out),
+                        _p(H_in), C.c_int64(H_in.shape[1]), _p(H_halo), C.c_int64(H_halo.shape[1]),
+                        _p(W), _p(bias), C.c_int32(act), _p(AGG), _p(Z), _p(H), C.c_int64(d_out))
+    return AGG, Z, H
+
+
+def layer_bwd(P: Partitioning, m: int, dtil, G_out, mask, AGG, W, G_W, G_b, want_in=True, want_halo=False):
+    """Accumulates into G_W, G_b (float64); returns (G_in fp32 or None, G_halo fp32 or None)."""
+    n_in = P.inner_gid[m].shape[0]
+    n_halo = P.halo_gid[m].shape[0]
+    d_in, d_out = W.shape
+    G_out, W = _f32(G_out), _f32(W)
+    AGG = np.ascontiguousarray(AGG, dtype=np.float64)
+    mask = None if mask is None else np.ascontiguousarray(mask, dtype=np.uint8)
+    G_in = np.zeros((n_in, d_in), dtype=np.float32) if want_in else None
+    G_halo = np.zeros((n_halo, d_in), dtype=np.float32) if want_halo else None
+    lib().orc_layer_bwd(C.c_int32(n_in), C.c_int32(n_halo), _p(P.loc_rowptr[m]), _p(P.loc_col[m]),
+                        _p(P.inner_gid[m]), _p(P.halo_gid[m]), _p(dtil),
+                        C.c_int32(d_in), C.c_int32(d_out), _p(G_out), C.c_int64(G_out.shape[1]), _p(mask),
+                        _p(AGG), _p(W), _p(G_W), _p(G_b), _p(G_in), C.c_int64(d_in), _p(G_halo), C.c_int64(d_in))
+    return G_in, G_halo
+
+
+def loss_grad(kind: str, Z, labels, scale: float):
+    """(scaled loss sum over the rows, G = scale * dLoss/dZ fp32)."""
+    Z = _f32(Z)
+    n, c = Z.shape
+    G = np.zeros((n, c), dtype=np.float32)
+    if kind == "ce":
+        y = np.ascontiguousarray(labels, dtype=np.int32)
+        val = lib().orc_loss_ce(C.c_int32(n), C.c_int32(c), _p(Z), C.c_int64(c), _p(y), C.c_double(scale), _p(G), C.c_int64(c))
+    else:
+        Y = np.ascontiguousarray(labels, dtype=np.uint8)
+        val = lib().orc_loss_bce(C.c_int32(n), C.c_int32(c), _p(Z), C.c_int64(c), _p(Y), C.c_double(scale), _p(G), C.c_int64(c))
+    return float(val), G
+
+
+# --------------------------------------------------------------------------------------
+# O-10  one SAT epoch over all partitions (Algorithm 1, lines of the epoch loop)
+# --------------------------------------------------------------------------------------
+@dataclass
+class EpochResult:
+    loss: float
+    G_W: list
+    G_b: list
+    per_part: list      # per partition: dict(H=[H^(1..L)], halo=[Hhat inputs of layers 1..L], G_in=[...], Z=[...], AGG=[...])
+    S: list             # per cached layer: LSTM state table or None (identity predictor)
+
+
+def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, loss_kind: str,
+              order=None, keep: bool = True, want_halo_grad: bool = False, parts=None) -> EpochResult:
+    """pull (predict) -> forward -> push, per layer; loss; backward; commit the ring.
+
+    pred: list (one entry per cached layer) of dict(Wx, Uh, b, Wg, bg) or None for the
+    identity predictor (plain historical embeddings).  `parts` restricts the epoch to a
+    subset of partitions (then the ring is not committed)."""
+    L = len(W)
+    n = P.n
+    ms = list(range(P.M)) if parts is None else list(parts)
+    if order is not None:
+        ms = list(order)
+    # LSTM state table: depends only on committed snapshots, one per cached layer
+    S = []
+    for l in range(1, L):
+        pr = pred[l - 1] if pred is not None else None
+        if pr is None:
+            S.append(None)
+        else:
+            h, d = pr["Wg"].shape
+            S.append(lstm_state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots))
+    G_W = [np.zeros(w.shape, dtype=np.float64) for w in W]
+    G_b = [np.zeros(w.shape[1], dtype=np.float64) for w in W]
+    total_loss = 0.0
+    per_part = [None] * P.M
+    for m in ms:
+        inner, halo = P.inner_gid[m], P.halo_gid[m]
+        H_in = _f32(X[inner])
+        rec = dict(H=[], halo=[], G_in=[], Z=[], AGG=[], G_halo=[])
+        for l in range(1, L + 1):
+            if l == 1:
+                H_halo = _f32(X[halo])                      # raw features are exact
+            else:
+                pr = pred[l - 2] if pred is not None else None
+                if pr is None:
+                    H_halo = historical_halo(P, m, cache.newest(l - 1), W[l - 1].shape[0])
+                else:
+                    H_halo = predict_halo(P, m, dtil, S[l - 2], cache.newest(l - 1), pr["Wg"], pr["bg"])
+            AGG, Z, H = layer_fwd(P, m, dtil, H_in, H_halo, W[l - 1], b[l - 1], 1 if l < L else 0)
+            if l < L:
+                cache.push(l, P.push_slot[m], H[P.push_local[m]])
+            rec["halo"].append(H_halo)
+            rec["AGG"].append(AGG)
+            rec["Z"].append(Z)
+            rec["H"].append(H)
+            H_in = H
+        lab = labels[inner]
+        val, G = loss_grad(loss_kind, rec["H"][-1], lab, 1.0 / n)
+        total_loss += val
+        rec["G_L"] = G
+        g_ins = [None] * L
+        g_halos = [None] * L
+        for l in range(L, 0, -1):
+            mask = None if l == L else (rec["Z"][l - 1] > 0.0).astype(np.uint8)
+            G_in, G_halo = layer_bwd(P, m, dtil, G, mask, rec["AGG"][l - 1], W[l - 1], G_W[l - 1], G_b[l - 1],
+                                     want_in=(l > 1), want_halo=want_halo_grad)
+            g_ins[l - 1] = G_in
+            g_halos[l - 1] = G_halo
+            G = G_in
+        rec["G_in"] = g_ins
+        rec["G_halo"] = g_halos
+        if not keep:
+            rec["AGG"] = rec["Z"] = None
+        per_part[m] = rec
+    if parts is None:
+        cache.commit()
+    return EpochResult(loss=total_loss, G_W=G_W, G_b=G_b, per_part=per_part, S=S)
