@@ -1,0 +1,268 @@
+/*
+ * sat_b200 — C ABI of the SAT (staleness-alleviated training, arXiv 2308.13466) hot path
+ * for one NVIDIA B200 (sm_100a).
+ *
+ * The library holds M graph partitions of one graph on one GPU and runs, per partition
+ * or for all partitions at once, the GCN layer step of historical-value training:
+ * pull predicted out-of-subgraph ("halo") embeddings from the historical-embedding cache
+ * (Algorithm 1, "Pull"), run the local layer forward (Eq. "sat forward"; Appendix,
+ * forward of SAT), push the fresh boundary embeddings (Algorithm 1, "Push"), and run the
+ * local backward (Appendix, backward equations).
+ *
+ * General rules
+ *   - Plain C types only.  Every pointer argument says HOST or DEVICE.  Device tensors
+ *     are caller-owned (allocated by the caller, e.g. through PyTorch), are never
+ *     retained after the call, and must be 16-byte aligned with a leading dimension
+ *     (`ld`, in floats) that is a multiple of 4 and >= the row width.
+ *   - All floating tensors are fp32, row-major.
+ *   - All work is enqueued on the stream given to sat_create (borrowed, not owned) and
+ *     is asynchronous; argument and state errors are reported synchronously and leave
+ *     the outputs untouched.
+ *   - Every function returns a sat_status (0 = ok, < 0 = error) and never throws,
+ *     aborts, traps or blocks indefinitely.  sat_last_error() gives a message.
+ *   - `part` selects a partition m in [0, M) or SAT_ALL_PARTS (-1): all partitions in one
+ *     launch, operands being the per-partition tensors concatenated in partition order
+ *     (inner rows: N rows; halo rows: sum_m b_m rows).  Results are identical to the M
+ *     per-partition calls.
+ *   - Layer index convention: GNN layer l in 1..L consumes H^(l-1) and produces H^(l);
+ *     cached layer l in 1..L-1 stores H^(l); sat_predict(layer = l) yields the halo input
+ *     of GNN layer l+1.
+ */
+#ifndef SAT_B200_H
+#define SAT_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sat_ctx sat_ctx; /* opaque; owns only library-internal device / host memory */
+typedef int32_t sat_status;
+
+enum {
+    SAT_OK = 0,
+    SAT_EINVAL = -1, /* bad argument: null pointer, shape, alignment, index out of range   */
+    SAT_ESTATE = -2, /* call order: e.g. sat_partition before sat_graph_load                */
+    SAT_ENOMEM = -3, /* device or host allocation failed                                    */
+    SAT_ECUDA = -4,  /* CUDA runtime error (sticky for the context)                         */
+    SAT_EDATA = -5   /* malformed graph: rowptr not monotone, column out of range, columns   */
+                     /* unsorted or duplicated, self-loop stored, or graph not symmetric     */
+};
+
+enum { SAT_HOST = 0, SAT_DEVICE = 1 };                   /* where an index array lives           */
+enum { SAT_ALL_PARTS = -1 };
+enum { SAT_PART_GIVEN = 0, SAT_PART_CONTIG_BLOCKS = 1 }; /* sat_partition methods                */
+enum { SAT_ACT_NONE = 0, SAT_ACT_RELU = 1 };
+enum { SAT_LOSS_SOFTMAX_CE = 0, SAT_LOSS_SIGMOID_BCE = 1 };
+enum { SAT_ROWS_INNER = 0, SAT_ROWS_HALO = 1 };          /* sat_gather_rows                      */
+enum { SAT_CACHE_ZERO = 0, SAT_CACHE_COPY = 1 };         /* sat_cache_init                       */
+
+/* ---------------------------------------------------------------------------------------
+ * Context
+ * ------------------------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device`.  `cuda_stream` is a cudaStream_t (may be 0 for
+ * the default stream); it is borrowed for the lifetime of the context. */
+sat_status sat_create(sat_ctx **ctx, int device, void *cuda_stream);
+sat_status sat_destroy(sat_ctx *ctx);
+/* Message of the most recent error on this context (valid until the next call). */
+const char *sat_last_error(const sat_ctx *ctx);
+/* Waits for the stream and returns SAT_ECUDA if any enqueued work failed. */
+sat_status sat_sync_status(sat_ctx *ctx);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_graph_load — the input graph G(V, E) (Preliminaries) and GCN's propagation matrix
+ * P = D~^{-1/2} (A + I) D~^{-1/2}, d~_v = deg(v) + 1 (Appendix, Preliminaries: "P is the
+ * propagation matrix following the definition of GCN").
+ *
+ *   n        number of nodes
+ *   nnz      number of stored directed edges (both directions of every undirected edge;
+ *            self-loops must NOT be stored — the library adds I itself)
+ *   rowptr   int64 [n+1], col int32 [nnz]; HOST or DEVICE as `ptr_space` says; columns
+ *            sorted ascending and unique inside a row.  The graph must be symmetric.
+ * The arrays are copied; the caller may free them after the call.  The graph is validated
+ * on the device (SAT_EDATA on failure; this call synchronises the stream).  Computes
+ * dinv[v] = (deg(v)+1)^{-1/2}; P is never stored: p_vu = dinv[v] * dinv[u].
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_graph_load(sat_ctx *ctx, int32_t n, int64_t nnz, const int64_t *rowptr, const int32_t *col,
+                          int ptr_space);
+/* Copies dinv (fp32 [n]) to HOST memory. */
+sat_status sat_graph_dinv(sat_ctx *ctx, float *dinv_host);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_partition — split G into M non-overlapping subgraphs G_m(V_m, E_m) (Algorithm 1,
+ * "Partitioning the raw graph"; Preliminaries, "Distributed Training for GNNs") and build,
+ * per partition, the 1-hop extended subgraph of Section "Embedding Predictor":
+ *   I_m  inner nodes, ascending global id
+ *   B_m  halo nodes = sorted unique  U_{v in V_m} N(v) \ V_m   (Eq. "communication
+ *        complexity", second term)
+ *   local CSR over rows I_m with entries N(v) + {v}; local column id = rank in I_m for an
+ *        inner node, n_m + rank in B_m for a halo node; columns ascending (P_in | P_out of
+ *        the Appendix: P = P_in + P_out)
+ *   halo-row CSR: for u in B_m its neighbours inside V_m as local inner ids, ascending
+ *        (= P_out^T)
+ *   C = sorted union of all B_m = the nodes the cache stores; slot[v] = rank of v in C or -1
+ *   push list of m: local ids (ascending) and slots of the inner nodes of m that are in C.
+ * Methods: SAT_PART_GIVEN uses part_of_node (int32 [n], values in [0, M), HOST or DEVICE
+ * per `ptr_space`); SAT_PART_CONTIG_BLOCKS ignores it and uses part[v] = floor(v*M/n)
+ * (the paper partitions with METIS, which is a third-party tool and not part of this
+ * library: pass its output through SAT_PART_GIVEN).
+ * All structures are integer and are built on the device; this call synchronises.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const int32_t *part_of_node, int ptr_space);
+
+/* Sizes of partition m (any output pointer may be NULL).  m = SAT_ALL_PARTS gives totals:
+ * n, sum_m b_m, nnz(A+I), |C|, number of cut-edge entries. */
+sat_status sat_part_sizes(sat_ctx *ctx, int32_t m, int32_t *n_inner, int32_t *n_halo, int64_t *nnz_local,
+                          int32_t *n_push, int64_t *nnz_hrow);
+/* Copies the lists of partition m to HOST arrays sized by sat_part_sizes (any may be NULL):
+ * inner_gid [n_inner], halo_gid [n_halo], halo_slot [n_halo], push_local [n_push],
+ * push_slot [n_push], loc_rowptr int64 [n_inner+1] (starting at 0), loc_col [nnz_local],
+ * hrow_ptr int64 [n_halo+1] (starting at 0), hrow_col [nnz_hrow]. */
+sat_status sat_part_lists(sat_ctx *ctx, int32_t m, int32_t *inner_gid, int32_t *halo_gid, int32_t *halo_slot,
+                          int32_t *push_local, int32_t *push_slot, int64_t *loc_rowptr, int32_t *loc_col,
+                          int64_t *hrow_ptr, int32_t *hrow_col);
+/* Copies part[] (int32 [n], may be NULL) and slot[] (int32 [n], may be NULL) to HOST memory
+ * and returns |C|. */
+sat_status sat_slot_map(sat_ctx *ctx, int32_t *part_host, int32_t *slot_host, int32_t *n_slots);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_gather_rows — out[i, :] = x[gid(i), :] for the inner (SAT_ROWS_INNER) or halo
+ * (SAT_ROWS_HALO) nodes of `part`, x being a DEVICE matrix over all n nodes in global id
+ * order.  With SAT_ROWS_HALO on the raw features this is the layer-1 pull: H_halo^(0) =
+ * X[B_m] (out-of-subgraph term of Eq. "mini-batch" with h^(0) = x).
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_gather_rows(sat_ctx *ctx, int32_t part, int which, const float *x, int32_t ld_x, int32_t d,
+                           float *out, int32_t ld_out);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_cache_init — the offline memory of historical embeddings (Section "Problem
+ * Formulation": H~_out) as a ring, per cached layer, of tau readable snapshots plus one
+ * write buffer over the |C| boundary nodes; tau is the sliding window of Eq. "problem
+ * formulation".  width[i] is the embedding width of cached layer i+1.
+ * mode SAT_CACHE_ZERO: all zeros, no valid snapshot.  SAT_CACHE_COPY: init[i] (DEVICE,
+ * [|C| x width[i]], ld = width rounded up to 4) becomes the single valid snapshot of layer
+ * i+1.  Memory: sum_i (tau+1) * |C| * ld_i * 4 bytes, owned by the context.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, const int32_t *width, int32_t tau, int mode,
+                          const float *const *init);
+
+/* Predictor parameters g_omega (Section "Embedding Predictor": LSTM + GCN), all DEVICE,
+ * dense row-major without padding: Wx [d x 4h], Uh [h x 4h], b [4h] (gate order i, f, g, o),
+ * Wg [h x d], bg [d].  d = width of the cached layer. */
+typedef struct sat_pred_params {
+    const float *Wx, *Uh, *b, *Wg, *bg;
+    int32_t h;
+} sat_pred_params;
+
+/* ---------------------------------------------------------------------------------------
+ * sat_predict — predicted out-of-subgraph embeddings Hhat_out^(l, m) = g_omega over the
+ * temporal graph of the last min(n_valid, tau) cached snapshots (Eq. "sat forward",
+ * Eq. "problem formulation", Section "Embedding Predictor"):
+ *   LSTM over the snapshots (oldest first, zero initial state) for every cached node -> S;
+ *   for halo node u of partition m:  a_u = p_uu S_u + sum_{v in N(u), v in V_m} p_uv S_v,
+ *   Hhat_u = H~_u(newest snapshot) + a_u Wg + bg     (graph convolution + skip connection).
+ * params == NULL is the identity predictor: Hhat_u = H~_u(newest) (plain historical
+ * embeddings).  With no valid snapshot H~ = 0 and S = 0.
+ *   reuse_state  0: run the LSTM now (for all |C| cached nodes; the table S is kept in the
+ *                context per cached layer);  1: reuse the table of the previous call for
+ *                this layer (caller guarantees parameters and ring are unchanged;
+ *                SAT_ESTATE if there is none since the last commit).
+ *   halo_out     DEVICE [b_m x ld_out] (part = SAT_ALL_PARTS: [sum_m b_m x ld_out]).
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, const sat_pred_params *params, int reuse_state,
+                       float *halo_out, int32_t ld_out);
+/* Copies the LSTM state table S of cached layer `layer` (fp32 [|C| x h]) to HOST memory. */
+sat_status sat_predict_state(sat_ctx *ctx, int32_t layer, float *S_host, int32_t h);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_layer_fwd — local GCN layer forward (Appendix, forward of SAT):
+ *     AGG = P_in h_in + P_out h_halo ;  Z = AGG W + bias ;  h_out = ReLU(Z) or Z.
+ *   h_in   DEVICE [n_m x ld_in]   in-subgraph embeddings H_in^(l-1, m), rows in I_m order
+ *   h_halo DEVICE [b_m x ld_halo] out-of-subgraph embeddings (raw features for layer 1,
+ *          sat_predict output otherwise); may be NULL when b_m = 0
+ *   W      DEVICE [d_in x d_out] dense row-major;  bias DEVICE [d_out] or NULL
+ *   h_out  DEVICE [n_m x ld_out]
+ * What the backward needs (AGG and the sign of Z) is kept inside the context per layer,
+ * for the rows of `part`; a later sat_layer_fwd of the same (part, layer) overwrites it.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in, int32_t d_out,
+                         const float *h_in, int32_t ld_in, const float *h_halo, int32_t ld_halo,
+                         const float *W, const float *bias, int act, float *h_out, int32_t ld_out);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_layer_bwd — local backward of the same layer (Appendix, backward equations):
+ *     D = g_out o [Z > 0] (ReLU layer) or g_out ;  g_W (+)= AGG^T D ;  g_b (+)= 1^T D ;
+ *     G_AGG = D W^T ;  g_in = P_in^T G_AGG ;  g_halo = P_out^T G_AGG.
+ * The predicted halo embeddings are constants of the epoch (Section "Optimization
+ * Algorithm"), so g_halo is an optional by-product and is not propagated.
+ *   g_out  DEVICE [n_m x ld_g]  gradient w.r.t. this layer's output h_out
+ *   g_W    DEVICE [d_in x d_out] dense; g_b DEVICE [d_out] or NULL
+ *   accumulate  0: overwrite g_W / g_b; 1: add to them (summing partitions gives the
+ *               gradient of the global loss, Eq. "global loss")
+ *   g_in   DEVICE [n_m x ld_gin] or NULL (layer 1);  g_halo DEVICE [b_m x ld_gh] or NULL
+ * Requires the matching sat_layer_fwd to have run (SAT_ESTATE otherwise).  Results are
+ * bit-reproducible from run to run (no floating-point atomics).
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g,
+                         const float *W, float *g_W, float *g_b, int accumulate,
+                         float *g_in, int32_t ld_gin, float *g_halo, int32_t ld_gh);
+
+/* ---------------------------------------------------------------------------------------
+ * sat_cache_update — push (Algorithm 1, "Push computed embeddings to the server"): rows of
+ * h_out (DEVICE [n_m x ld], the output of GNN layer `layer` < L) that belong to boundary
+ * nodes are written into the write buffer of cached layer `layer`.  Invisible to
+ * sat_predict until sat_cache_commit.  Every boundary node must be pushed once per epoch
+ * (rows not pushed keep whatever the buffer held tau+1 epochs earlier).
+ * sat_cache_commit — end of epoch: the write buffer becomes the newest snapshot, the oldest
+ * one is dropped, n_valid = min(n_valid + 1, tau); LSTM state tables are invalidated.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer, const float *h_out, int32_t ld);
+sat_status sat_cache_commit(sat_ctx *ctx);
+/* Ring bookkeeping: index of the write buffer in [0, tau] and number of valid snapshots. */
+sat_status sat_cache_state(sat_ctx *ctx, int32_t *write_idx, int32_t *n_valid);
+/* Copies snapshot `age` (0 = newest committed, ..., n_valid-1 = oldest; -1 = the write
+ * buffer) of cached layer `layer` to HOST memory as dense [|C| x width]. */
+sat_status sat_cache_read(sat_ctx *ctx, int32_t layer, int32_t age, float *out_host);
+/* Checkpoint / resume of the whole ring of one cached layer: raw [(tau+1) x |C| x width]
+ * HOST array in buffer-index order, plus write_idx / n_valid via sat_cache_state and
+ * sat_cache_set_state. */
+sat_status sat_cache_export(sat_ctx *ctx, int32_t layer, float *out_host);
+sat_status sat_cache_import(sat_ctx *ctx, int32_t layer, const float *in_host);
+sat_status sat_cache_set_state(sat_ctx *ctx, int32_t write_idx, int32_t n_valid);
+
+/* ---------------------------------------------------------------------------------------
+ * Auxiliary steps of the epoch (Algorithm 1, "Local GNN update" / "Global GNN update").
+ * sat_loss_grad — local loss (Eq. "local loss") weighted by w_m = |V_m| / N (Eq. "global
+ * loss"), i.e. every node carries weight 1/N:  *loss_sum (DEVICE double, += ) receives
+ * sum_v Loss_v / N over the rows of `part`; g = (1/N) dLoss_v/dz (DEVICE [n_m x ld_g]).
+ *   SAT_LOSS_SOFTMAX_CE:  labels int32 [n_m] DEVICE;  Loss_v = -log softmax(z_v)[y_v]
+ *   SAT_LOSS_SIGMOID_BCE: labels uint8 [n_m x n_classes] DEVICE;
+ *                         Loss_v = (1/C) sum_c softplus(z_c) - y_c z_c
+ * sat_sgd_step — w <- w - lr * g over `count` floats (the parameter step on the summed
+ * gradient; all partitions share theta within an epoch, so AGG is the identity here).
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_t n_classes, const float *z, int32_t ld_z,
+                         const void *labels, double *loss_sum, float *g, int32_t ld_g);
+sat_status sat_sgd_step(sat_ctx *ctx, int64_t count, float *w, const float *g, float lr);
+
+/* Number of kernels this context has launched since creation (all entry points). */
+sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
+
+/* Optional device timing per kernel family, with CUDA events on the context's stream (measurement aid; the
+ * paper has no counterpart).  sat_profile_enable(1) clears the records and starts bracketing every family's
+ * launches with an event pair; sat_profile_enable(0) stops.  sat_profile_read waits for the stream and returns,
+ * for family f in [0, sat_profile_families()), its name, number of bracketed calls, total milliseconds and the
+ * algorithmic bytes / flops those calls moved / performed (each operand read once, each result written once). */
+enum { SAT_PROF_SPMM_FWD = 0, SAT_PROF_SPMM_BWD, SAT_PROF_SPMM_HROW, SAT_PROF_GEMM_NN, SAT_PROF_GEMM_NT,
+       SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS };
+int32_t sat_profile_families(void);
+sat_status sat_profile_enable(sat_ctx *ctx, int enable);
+sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int64_t *calls, double *ms, double *bytes,
+                            double *flops);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAT_B200_H */

@@ -300,12 +300,14 @@ class EpochResult:
 
 
 def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, loss_kind: str,
-              order=None, keep: bool = True, want_halo_grad: bool = False, parts=None) -> EpochResult:
+              order=None, keep: bool = True, want_halo_grad: bool = False, parts=None, masks=None) -> EpochResult:
     """pull (predict) -> forward -> push, per layer; loss; backward; commit the ring.
 
     pred: list (one entry per cached layer) of dict(Wx, Uh, b, Wg, bg) or None for the
     identity predictor (plain historical embeddings).  `parts` restricts the epoch to a
-    subset of partitions (then the ring is not committed)."""
+    subset of partitions (then the ring is not committed).  `masks[m][l-1]`, when given,
+    replaces [Z^(l) > 0] in the backward of partition m (the derivative of ReLU where Z is
+    zero up to rounding is a tie: either sign decision is a correct result)."""
     L = len(W)
     n = P.n
     ms = list(range(P.M)) if parts is None else list(parts)
@@ -353,6 +355,8 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
         g_halos = [None] * L
         for l in range(L, 0, -1):
             mask = None if l == L else (rec["Z"][l - 1] > 0.0).astype(np.uint8)
+            if mask is not None and masks is not None and masks[m] is not None and masks[m][l - 1] is not None:
+                mask = np.ascontiguousarray(masks[m][l - 1], dtype=np.uint8)
             G_in, G_halo = layer_bwd(P, m, dtil, G, mask, rec["AGG"][l - 1], W[l - 1], G_W[l - 1], G_b[l - 1],
                                      want_in=(l > 1), want_halo=want_halo_grad)
             g_ins[l - 1] = G_in

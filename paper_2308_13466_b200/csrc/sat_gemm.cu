@@ -1,0 +1,281 @@
+// Dense contractions of the sat_b200 library on the CUDA cores (fp32 FMA, fp32 accumulate):
+// the general-shape path used for every size the tensor-core path does not take.
+//   NN: C = A B (+bias, ReLU, sign mask, gathered residual)          layer transform, predictor output
+//   NT: C = (A o mask) B^T                                            input gradient  D W^T
+//   TN: C (+)= A^T (B o mask), colsum (+)= 1^T (B o mask), split-K    weight / bias gradient
+#include "sat_internal.h"
+
+#define BM 64
+#define BN 64
+#define BK 16
+#define TN_ROWS_PER_SPLIT 4096
+
+__device__ __forceinline__ bool mask_bit(const uint32_t *mask, int64_t row, int32_t mask_words, int32_t c)
+{
+    return (mask[row * mask_words + (c >> 5)] >> (c & 31)) & 1u;
+}
+
+// 256 threads, thread (ty, tx) = (t / 16, t % 16) owns rows ty*4.., cols tx*4.. of the 64x64 tile
+#define INNER_PRODUCT()                                              \
+    _Pragma("unroll") for (int kk = 0; kk < BK; ++kk) {             \
+        float a[4], b[4];                                            \
+        _Pragma("unroll") for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i]; \
+        _Pragma("unroll") for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j]; \
+        _Pragma("unroll") for (int i = 0; i < 4; ++i)                \
+            _Pragma("unroll") for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]); \
+    }
+
+__global__ void __launch_bounds__(256)
+k_gemm_nn(int64_t m, int32_t n, int32_t k1, const float *__restrict__ A, int64_t lda, const float *__restrict__ B, int64_t ldb,
+          int32_t k2, const float *__restrict__ A2, int64_t lda2, const float *__restrict__ B2, int64_t ldb2,
+          float *__restrict__ C, int64_t ldc, const float *__restrict__ bias, int relu, uint32_t *__restrict__ mask_out,
+          int32_t mask_words, const float *__restrict__ resid, const int32_t *__restrict__ resid_idx, int64_t ld_resid)
+{
+    // the contraction runs over the virtual concatenation [A | A2] [B ; B2] (k2 may be 0)
+    const int32_t k = k1 + k2;
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+    const int64_t row0 = (int64_t)blockIdx.x * BM;
+    const int32_t col0 = blockIdx.y * BN;
+    float acc[4][4] = {};
+    for (int32_t k0 = 0; k0 < k; k0 += BK) {
+        {   // A tile: thread loads 4 consecutive k of one row
+            const int r = t >> 2, kq = (t & 3) * 4;
+            const int64_t gr = row0 + r;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gk = k0 + kq + q;
+                float x = 0.f;
+                if (gr < m && gk < k) x = gk < k1 ? A[gr * lda + gk] : A2[gr * lda2 + (gk - k1)];
+                As[kq + q][r] = x;
+            }
+        }
+        {   // B tile: thread loads 4 consecutive n of one k
+            const int kk = t >> 4, nq = (t & 15) * 4;
+            const int32_t gk = k0 + kk;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gn = col0 + nq + q;
+                float x = 0.f;
+                if (gk < k && gn < n) x = gk < k1 ? B[(int64_t)gk * ldb + gn] : B2[(int64_t)(gk - k1) * ldb2 + gn];
+                Bs[kk][nq + q] = x;
+            }
+        }
+        __syncthreads();
+        INNER_PRODUCT();
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t gr = row0 + ty * 4 + i;
+        uint32_t nib = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int32_t gn = col0 + tx * 4 + j;
+            if (gr < m && gn < n) {
+                float z = acc[i][j] + (bias ? bias[gn] : 0.f);
+                if (resid) z += resid[(int64_t)resid_idx[gr] * ld_resid + gn];
+                if (z > 0.f) nib |= 1u << j;
+                if (relu && !(z > 0.f)) z = 0.f;
+                C[gr * ldc + gn] = z;
+            }
+        }
+        if (mask_out) {
+            // 8 threads (tx & 7) share one 32-bit word of the row
+            uint32_t wbits = nib << (4 * (tx & 7));
+            wbits |= __shfl_xor_sync(0xffffffffu, wbits, 1);
+            wbits |= __shfl_xor_sync(0xffffffffu, wbits, 2);
+            wbits |= __shfl_xor_sync(0xffffffffu, wbits, 4);
+            const int32_t word = (col0 >> 5) + (tx >> 3);
+            if ((tx & 7) == 0 && gr < m && word < mask_words) mask_out[gr * mask_words + word] = wbits;
+        }
+    }
+}
+
+sat_status sat_gemm_nn(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *B, int32_t ldb,
+                       float *C, int32_t ldc, const GemmEpilogue &ep)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_GEMM_NN, 4.0 * ((double)m * (k + n) + (double)k * n), 2.0 * (double)m * n * k);
+    dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN));
+    k_gemm_nn<<<grid, 256, 0, ctx->stream>>>(m, n, k, A, lda, B, ldb, 0, nullptr, 0, nullptr, 0, C, ldc, ep.bias, ep.relu, ep.mask_out,
+                                             ep.mask_words, ep.resid, ep.resid_idx, ep.ld_resid);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+sat_status sat_gemm_nn_dual(sat_ctx *ctx, int64_t m, int32_t n, int32_t k1, const float *A1, int32_t lda1, const float *B1, int32_t ldb1,
+                            int32_t k2, const float *A2, int32_t lda2, const float *B2, int32_t ldb2, const float *bias, float *C,
+                            int32_t ldc)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_GEMM_NN, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
+    dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN));
+    k_gemm_nn<<<grid, 256, 0, ctx->stream>>>(m, n, k1, A1, lda1, B1, ldb1, k2, A2, lda2, B2, ldb2, C, ldc, bias, 0, nullptr, 0, nullptr,
+                                             nullptr, 0);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+__global__ void __launch_bounds__(256)
+k_gemm_nt(int64_t m, int32_t n, int32_t k, const float *__restrict__ A, int64_t lda, const uint32_t *__restrict__ mask,
+          int32_t mask_words, const float *__restrict__ B, int64_t ldb, float *__restrict__ C, int64_t ldc)
+{
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+    const int64_t row0 = (int64_t)blockIdx.x * BM;
+    const int32_t col0 = blockIdx.y * BN;
+    float acc[4][4] = {};
+    for (int32_t k0 = 0; k0 < k; k0 += BK) {
+        const int r = t >> 2, kq = (t & 3) * 4;
+        {
+            const int64_t gr = row0 + r;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gk = k0 + kq + q;
+                float x = 0.f;
+                if (gr < m && gk < k) {
+                    x = A[gr * lda + gk];
+                    if (mask && !mask_bit(mask, gr, mask_words, gk)) x = 0.f;
+                }
+                As[kq + q][r] = x;
+            }
+        }
+        {   // B^T tile: B is [n x k]; thread loads 4 consecutive k of one n
+            const int32_t gn = col0 + r;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gk = k0 + kq + q;
+                Bs[kq + q][r] = (gn < n && gk < k) ? B[(int64_t)gn * ldb + gk] : 0.f;
+            }
+        }
+        __syncthreads();
+        INNER_PRODUCT();
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t gr = row0 + ty * 4 + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int32_t gn = col0 + tx * 4 + j;
+            if (gr < m && gn < n) C[gr * ldc + gn] = acc[i][j];
+        }
+    }
+}
+
+sat_status sat_gemm_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const uint32_t *mask,
+                       int32_t mask_words, const float *B, int32_t ldb, float *C, int32_t ldc)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_GEMM_NT, 4.0 * ((double)m * (k + n) + (double)k * n), 2.0 * (double)m * n * k);
+    dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN));
+    k_gemm_nt<<<grid, 256, 0, ctx->stream>>>(m, n, k, A, lda, mask, mask_words, B, ldb, C, ldc);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+// split-K over the row dimension: block (x, y, z) computes the [64 x 64] tile (x, y) of A^T (B o mask)
+// over rows [z * rows_per_split, ...), and the blocks with x == 0 also the column sums of (B o mask).
+__global__ void __launch_bounds__(256)
+k_gemm_tn(int64_t rows, int64_t rows_per_split, int32_t m, int32_t n, const float *__restrict__ A, int64_t lda,
+          const float *__restrict__ B, int64_t ldb, const uint32_t *__restrict__ mask, int32_t mask_words,
+          float *__restrict__ part_C /* [splits x m x n] */, float *__restrict__ part_cs /* [splits x n] or null */)
+{
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+    const int32_t m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
+    const int64_t r_begin = (int64_t)blockIdx.z * rows_per_split;
+    const int64_t r_end = (r_begin + rows_per_split < rows) ? r_begin + rows_per_split : rows;
+    float acc[4][4] = {};
+    float cs[4] = {0.f, 0.f, 0.f, 0.f};
+    const bool want_cs = part_cs != nullptr && blockIdx.x == 0;
+    for (int64_t r0 = r_begin; r0 < r_end; r0 += BK) {
+        {   // A^T tile: As[kk][i] = A[r0 + kk][m0 + i]; thread loads 4 consecutive m of one row
+            const int kk = t >> 4, iq = (t & 15) * 4;
+            const int64_t gr = r0 + kk;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gm = m0 + iq + q;
+                As[kk][iq + q] = (gr < r_end && gm < m) ? A[gr * lda + gm] : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int32_t gn = n0 + iq + q;
+                float x = 0.f;
+                if (gr < r_end && gn < n) {
+                    x = B[gr * ldb + gn];
+                    if (mask && !mask_bit(mask, gr, mask_words, gn)) x = 0.f;
+                }
+                Bs[kk][iq + q] = x;
+            }
+        }
+        __syncthreads();
+        INNER_PRODUCT();
+        if (want_cs && ty == 0) {
+#pragma unroll
+            for (int kk = 0; kk < BK; ++kk)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) cs[j] += Bs[kk][tx * 4 + j];
+        }
+        __syncthreads();
+    }
+    float *pc = part_C + (int64_t)blockIdx.z * m * n;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int32_t gm = m0 + ty * 4 + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int32_t gn = n0 + tx * 4 + j;
+            if (gm < m && gn < n) pc[(int64_t)gm * n + gn] = acc[i][j];
+        }
+    }
+    if (want_cs && ty == 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int32_t gn = n0 + tx * 4 + j;
+            if (gn < n) part_cs[(int64_t)blockIdx.z * n + gn] = cs[j];
+        }
+    }
+}
+
+// out[i] (+)= sum_z part[z][i], z ascending (fixed order: reproducible)
+__global__ void k_splitk_reduce(const float *__restrict__ part, int64_t count, int32_t splits, int accumulate, float *__restrict__ out,
+                                int32_t ncols, int64_t ld_out)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    float s = 0.f;
+    for (int z = 0; z < splits; ++z) s += part[(int64_t)z * count + i];
+    const int64_t r = i / ncols, c = i - r * ncols;
+    float *o = out + r * ld_out + c;
+    *o = accumulate ? *o + s : s;
+}
+
+sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
+                       const uint32_t *mask, int32_t mask_words, float *C, int32_t ldc, float *colsum, int accumulate)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_GEMM_TN, 4.0 * ((double)rows * (m + n) + (double)m * n), 2.0 * (double)rows * m * n);
+    int64_t splits = cdiv64(rows > 0 ? rows : 1, TN_ROWS_PER_SPLIT);
+    if (splits > 1024) splits = 1024;
+    int64_t rows_per_split = cdiv64(cdiv64(rows > 0 ? rows : 1, splits), BK) * BK;
+    splits = cdiv64(rows > 0 ? rows : 1, rows_per_split);
+    const size_t bytes = (size_t)splits * ((size_t)m * n + n) * sizeof(float);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_splitk, bytes));
+    float *part_C = (float *)ctx->buf_splitk.p;
+    float *part_cs = colsum ? part_C + (size_t)splits * m * n : nullptr;
+    dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN), (unsigned)splits);
+    k_gemm_tn<<<grid, 256, 0, ctx->stream>>>(rows, rows_per_split, m, n, A, lda, B, ldb, mask, mask_words, part_C, part_cs);
+    SAT_LAUNCHED(ctx);
+    k_splitk_reduce<<<(unsigned)cdiv64((int64_t)m * n, 256), 256, 0, ctx->stream>>>(part_C, (int64_t)m * n, (int32_t)splits, accumulate, C, n, ldc);
+    SAT_LAUNCHED(ctx);
+    if (colsum) {
+        k_splitk_reduce<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(part_cs, n, (int32_t)splits, accumulate, colsum, n, n);
+        SAT_LAUNCHED(ctx);
+    }
+    return SAT_OK;
+}

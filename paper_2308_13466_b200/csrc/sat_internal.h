@@ -1,0 +1,216 @@
+// Internal declarations of the sat_b200 library (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <vector>
+
+#include "../../include/sat_b200.h"
+
+#define SAT_MAX_LAYERS 16
+#define SAT_MAX_PARTS 4096
+#define SAT_SPMM_CHUNK 256 /* edges per SpMM work item */
+
+// A growable device buffer owned by the context.
+struct DevBuf {
+    void *p = nullptr;
+    size_t bytes = 0;
+};
+
+struct LayerState {
+    float *agg = nullptr;      // [N x ld_in]  saved aggregation (rows in partition-major order)
+    uint32_t *mask = nullptr;  // [N x mask_words] bit j of word w: Z[row][32w + j] > 0
+    int32_t d_in = 0, d_out = 0, ld_in = 0, mask_words = 0;
+    int act = 0;
+    std::vector<uint8_t> valid;  // per partition: forward state present
+};
+
+struct CacheLayer {
+    float *buf = nullptr;  // [(tau+1) x n_slots x ld]
+    int32_t width = 0, ld = 0;
+    float *S = nullptr;  // LSTM state table [n_slots x h]
+    int32_t S_h = 0;
+    bool S_valid = false;
+};
+
+// kernel families for the optional per-family device timing (sat_profile_*)
+enum {
+    SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_COUNT
+};
+
+struct ProfRec {
+    int family;
+    cudaEvent_t a, b;
+    double bytes, flops;
+};
+
+struct sat_ctx {
+    bool prof_on = false;
+    std::vector<ProfRec> prof;
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    char err[512] = {0};
+    bool cuda_failed = false;
+    int64_t launches = 0;
+    int *d_flag = nullptr;  // device status word used by validation kernels
+    int *h_flag = nullptr;  // pinned host mirror
+
+    // ---- graph ----
+    bool graph_ok = false;
+    int32_t n = 0;
+    int64_t nnz = 0;  // stored directed edges (no self-loops)
+    int64_t *rowptr = nullptr;
+    int32_t *col = nullptr;
+    float *dinv = nullptr;
+
+    // ---- partition ----
+    bool part_ok = false;
+    int32_t M = 0;
+    int32_t *part = nullptr;      // [n]
+    int32_t *perm = nullptr;      // [n]   inner global ids, partition-major (= concatenated I_m)
+    int32_t *pos = nullptr;       // [n]   inverse of perm
+    int32_t *halo_gid = nullptr;  // [nb]  concatenated B_m
+    int32_t *halo_slot = nullptr; // [nb]
+    int32_t *slot = nullptr;      // [n]
+    int32_t n_slots = 0;
+    int64_t nb = 0;               // sum_m b_m
+    int32_t *push_row = nullptr;  // [n_slots] partition-major row index of every boundary node
+    int32_t *push_slot = nullptr; // [n_slots]
+    int64_t *lrowptr = nullptr;   // [n+1] local CSR, rows partition-major
+    int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
+    int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
+    float *dinv_enc = nullptr;    // [n + nb] dinv of the node behind each encoded column
+    int64_t *hrow_ptr = nullptr;  // [nb+1] halo-row CSR
+    int32_t *hrow_pos = nullptr;  // [nnz_cut] partition-major row of the inner neighbour
+    int32_t *hrow_slot = nullptr; // [nnz_cut] its cache slot
+    int64_t nnz_cut = 0;
+    // SpMM work items (rows cut into chunks of SAT_SPMM_CHUNK edges)
+    int32_t *first_item = nullptr; // [n+1]
+    int32_t *item_row = nullptr;   // [n_items]
+    int32_t *item_mslot = nullptr; // [n_items] index of the partial-sum row for items of multi-chunk rows, else -1
+    int32_t *mrows = nullptr;      // [n_mrows] rows with more than one chunk
+    int32_t n_items = 0, n_mrows = 0, n_mitems = 0;
+    std::vector<int32_t> h_inner_off, h_push_off, h_item_off, h_mrow_off, h_mitem_off;
+    std::vector<int64_t> h_halo_off, h_lnnz_off, h_hrow_off;
+
+    // ---- cache ----
+    bool cache_ok = false;
+    int32_t n_cached = 0, tau = 0, write_idx = 0, n_valid = 0;
+    CacheLayer cache[SAT_MAX_LAYERS];
+
+    // ---- layers ----
+    LayerState layers[SAT_MAX_LAYERS + 1];
+
+    // ---- scratch ----
+    DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc;
+};
+
+sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
+sat_status sat_check_cuda(sat_ctx *ctx, cudaError_t e, const char *what);
+sat_status sat_ensure(sat_ctx *ctx, DevBuf &b, size_t bytes);
+void sat_free_buf(DevBuf &b);
+
+#define SAT_CUDA(ctx, call)                                          \
+    do {                                                             \
+        cudaError_t e__ = (call);                                    \
+        if (e__ != cudaSuccess) return sat_check_cuda(ctx, e__, #call); \
+    } while (0)
+
+#define SAT_TRY(expr)                   \
+    do {                                \
+        sat_status s__ = (expr);        \
+        if (s__ != SAT_OK) return s__;  \
+    } while (0)
+
+// Counts the launch and checks the launch error.
+#define SAT_LAUNCHED(ctx)                                                     \
+    do {                                                                      \
+        (ctx)->launches++;                                                    \
+        cudaError_t e__ = cudaGetLastError();                                 \
+        if (e__ != cudaSuccess) return sat_check_cuda(ctx, e__, "kernel launch"); \
+    } while (0)
+
+// Brackets the launches of one kernel family with CUDA events on the context's stream when profiling is on.
+struct ProfScope {
+    sat_ctx *ctx;
+    ProfRec rec;
+    bool on;
+    ProfScope(sat_ctx *c, int family, double bytes, double flops) : ctx(c), on(c->prof_on)
+    {
+        if (!on) return;
+        rec.family = family;
+        rec.bytes = bytes;
+        rec.flops = flops;
+        if (cudaEventCreate(&rec.a) != cudaSuccess || cudaEventCreate(&rec.b) != cudaSuccess) {
+            on = false;
+            return;
+        }
+        cudaEventRecord(rec.a, ctx->stream);
+    }
+    ~ProfScope()
+    {
+        if (!on) return;
+        cudaEventRecord(rec.b, ctx->stream);
+        ctx->prof.push_back(rec);
+    }
+};
+
+static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static inline int32_t round_up4(int32_t x) { return (x + 3) & ~3; }
+
+// ---- device-side helpers implemented in the .cu files ----
+// exclusive scan: out[i] = sum_{j<i} in[j], i = 0..count (count+1 outputs), int64 results
+sat_status sat_scan_i32(sat_ctx *ctx, const int32_t *in, int64_t count, int64_t *out);
+
+// row range / bases of a partition selector
+struct PartView {
+    int32_t row0, n_rows;     // partition-major rows
+    int64_t halo0, n_halo;    // halo positions
+    int32_t item0, n_items;   // SpMM work items
+    int32_t mrow0, n_mrows;   // multi-chunk rows
+    int32_t mitem0, n_mitems; // partial-sum rows
+    int32_t push0, n_push;
+    int64_t lnnz;             // local non-zeros (entries of A + I) of the selected rows
+};
+sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
+
+// SpMM family (sat_spmm.cu)
+//   out[row] = dinv[row] * sum_e dinv[col_e] * src(col_e), over all entries of the row (inner_only = 0)
+//   or over its inner prefix (inner_only = 1).  `in_base` / `halo_base` are the virtual bases of the
+//   partition-major inner matrix and of the concatenated halo matrix (already offset for a single
+//   partition); `out_base` likewise.
+sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
+                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out);
+//   halo-row products: out[j] = sum_{e in hrow(j)} dinv[halo j] dinv[inner e] * src[pos_e]   (+ self term if self_src)
+sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src,
+                         int by_slot, const float *self_src, float *out_base, int32_t ld_out);
+sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d, const float *src, int32_t ld_src,
+                      float *out, int32_t ld_out);
+sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d,
+                       const float *src_base, int32_t ld_src, float *dst, int32_t ld_dst);
+
+// GEMM family (sat_gemm.cu)
+// C[m x n] = A[m x k] B[k x n] (+ bias) with optional ReLU, sign-mask output, row-gathered residual add.
+struct GemmEpilogue {
+    const float *bias = nullptr;       // [n]
+    int relu = 0;
+    uint32_t *mask_out = nullptr;      // [m x mask_words] bit = (z > 0)
+    int32_t mask_words = 0;
+    const float *resid = nullptr;      // C += resid[resid_idx[i]] (row gather), ld_resid
+    const int32_t *resid_idx = nullptr;
+    int32_t ld_resid = 0;
+};
+sat_status sat_gemm_nn(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *B,
+                       int32_t ldb, float *C, int32_t ldc, const GemmEpilogue &ep);
+// C[m x n] = (A o mask)[m x k] B^T, B stored [n x k] row-major (ldb); mask may be null
+sat_status sat_gemm_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const uint32_t *mask,
+                       int32_t mask_words, const float *B, int32_t ldb, float *C, int32_t ldc);
+// C[m x n] (+)= A^T (B o mask): A [rows x m] (lda), B [rows x n] (ldb); colsum[n] (+)= 1^T (B o mask) if non-null.
+sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B,
+                       int32_t ldb, const uint32_t *mask, int32_t mask_words, float *C, int32_t ldc, float *colsum,
+                       int accumulate);

@@ -1,0 +1,474 @@
+// Entry points of the per-epoch steps: halo pull, predictor, layer forward / backward,
+// cache push / commit, loss seed and parameter step.
+#include "sat_internal.h"
+
+#define CHECK_CTX(ctx)                                                                             \
+    do {                                                                                           \
+        if (!(ctx)) return SAT_EINVAL;                                                             \
+        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
+        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
+    } while (0)
+
+static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+static bool ok_ld(int32_t ld, int32_t d) { return ld >= d && (ld & 3) == 0; }
+
+template <typename T>
+static sat_status dev_realloc(sat_ctx *ctx, T **p, int64_t count)
+{
+    if (*p) {
+        SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        cudaFree(*p);
+        *p = nullptr;
+    }
+    SAT_CUDA(ctx, cudaMalloc((void **)p, (size_t)(count > 0 ? count : 1) * sizeof(T)));
+    return SAT_OK;
+}
+
+// =====================================================================================
+// sat_gather_rows
+// =====================================================================================
+extern "C" sat_status sat_gather_rows(sat_ctx *ctx, int32_t part, int which, const float *x, int32_t ld_x, int32_t d, float *out,
+                                      int32_t ld_out)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (which != SAT_ROWS_INNER && which != SAT_ROWS_HALO) return sat_fail(ctx, SAT_EINVAL, "sat_gather_rows: bad row selector");
+    const int64_t count = which == SAT_ROWS_INNER ? v.n_rows : v.n_halo;
+    if (count == 0) return SAT_OK;
+    if (!x || !out || d <= 0 || !ok_ld(ld_x, d) || !ok_ld(ld_out, d) || !aligned16(x) || !aligned16(out))
+        return sat_fail(ctx, SAT_EINVAL, "sat_gather_rows: null / misaligned tensor or bad leading dimension");
+    const int32_t *idx = which == SAT_ROWS_INNER ? ctx->perm + v.row0 : ctx->halo_gid + v.halo0;
+    return sat_gather(ctx, idx, count, d, x, ld_x, out, ld_out);
+}
+
+// =====================================================================================
+// cache ring
+// =====================================================================================
+extern "C" sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, const int32_t *width, int32_t tau, int mode,
+                                     const float *const *init)
+{
+    CHECK_CTX(ctx);
+    if (!ctx->part_ok) return sat_fail(ctx, SAT_ESTATE, "sat_cache_init: call sat_partition first");
+    if (n_cached_layers < 0 || n_cached_layers > SAT_MAX_LAYERS || tau < 1 || (n_cached_layers > 0 && !width))
+        return sat_fail(ctx, SAT_EINVAL, "sat_cache_init: bad layer count / tau");
+    if (mode != SAT_CACHE_ZERO && mode != SAT_CACHE_COPY) return sat_fail(ctx, SAT_EINVAL, "sat_cache_init: bad mode");
+    if (mode == SAT_CACHE_COPY && !init) return sat_fail(ctx, SAT_EINVAL, "sat_cache_init: SAT_CACHE_COPY needs init");
+    for (int i = 0; i < n_cached_layers; ++i)
+        if (width[i] <= 0 || (mode == SAT_CACHE_COPY && (!init[i] || !aligned16(init[i]))))
+            return sat_fail(ctx, SAT_EINVAL, "sat_cache_init: bad width or init pointer for layer %d", i + 1);
+    for (int i = 0; i < SAT_MAX_LAYERS; ++i) {
+        if (ctx->cache[i].buf) cudaFree(ctx->cache[i].buf);
+        if (ctx->cache[i].S) cudaFree(ctx->cache[i].S);
+        ctx->cache[i] = CacheLayer();
+    }
+    ctx->cache_ok = false;
+    for (int i = 0; i < n_cached_layers; ++i) {
+        CacheLayer &c = ctx->cache[i];
+        c.width = width[i];
+        c.ld = round_up4(width[i]);
+        const size_t bytes = (size_t)(tau + 1) * (size_t)ctx->n_slots * c.ld * sizeof(float);
+        SAT_CUDA(ctx, cudaMalloc((void **)&c.buf, bytes ? bytes : 16));
+        SAT_CUDA(ctx, cudaMemsetAsync(c.buf, 0, bytes, ctx->stream));
+        if (mode == SAT_CACHE_COPY && ctx->n_slots > 0)
+            SAT_CUDA(ctx, cudaMemcpyAsync(c.buf, init[i], (size_t)ctx->n_slots * c.ld * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+    }
+    ctx->n_cached = n_cached_layers;
+    ctx->tau = tau;
+    ctx->write_idx = mode == SAT_CACHE_COPY ? 1 : 0;
+    ctx->n_valid = mode == SAT_CACHE_COPY ? 1 : 0;
+    ctx->cache_ok = true;
+    return SAT_OK;
+}
+
+static sat_status cache_layer(sat_ctx *ctx, int32_t layer, CacheLayer **c, const char *who)
+{
+    if (!ctx->cache_ok) return sat_fail(ctx, SAT_ESTATE, "%s: call sat_cache_init first", who);
+    if (layer < 1 || layer > ctx->n_cached) return sat_fail(ctx, SAT_EINVAL, "%s: cached layer %d out of range [1, %d]", who, layer, ctx->n_cached);
+    *c = &ctx->cache[layer - 1];
+    return SAT_OK;
+}
+
+// buffer index of the snapshot of a given age (0 = newest committed)
+static int32_t ring_index(const sat_ctx *ctx, int32_t age) { return ((ctx->write_idx - 1 - age) % (ctx->tau + 1) + (ctx->tau + 1)) % (ctx->tau + 1); }
+static float *ring_buf(const sat_ctx *ctx, const CacheLayer *c, int32_t idx) { return c->buf + (size_t)idx * ctx->n_slots * c->ld; }
+
+extern "C" sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer, const float *h_out, int32_t ld)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_cache_update"));
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (v.n_push == 0) return SAT_OK;
+    if (!h_out || !ok_ld(ld, c->width) || !aligned16(h_out)) return sat_fail(ctx, SAT_EINVAL, "sat_cache_update: null / misaligned h_out or bad ld");
+    const float *src_base = h_out - (int64_t)v.row0 * ld;
+    return sat_scatter(ctx, ctx->push_row + v.push0, ctx->push_slot + v.push0, v.n_push, c->width, src_base, ld,
+                       ring_buf(ctx, c, ctx->write_idx), c->ld);
+}
+
+extern "C" sat_status sat_cache_commit(sat_ctx *ctx)
+{
+    CHECK_CTX(ctx);
+    if (!ctx->cache_ok) return sat_fail(ctx, SAT_ESTATE, "sat_cache_commit: call sat_cache_init first");
+    ctx->write_idx = (ctx->write_idx + 1) % (ctx->tau + 1);
+    ctx->n_valid = ctx->n_valid + 1 < ctx->tau ? ctx->n_valid + 1 : ctx->tau;
+    for (int i = 0; i < ctx->n_cached; ++i) ctx->cache[i].S_valid = false;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_cache_state(sat_ctx *ctx, int32_t *write_idx, int32_t *n_valid)
+{
+    if (!ctx) return SAT_EINVAL;
+    if (!ctx->cache_ok) return sat_fail(ctx, SAT_ESTATE, "sat_cache_state: call sat_cache_init first");
+    if (write_idx) *write_idx = ctx->write_idx;
+    if (n_valid) *n_valid = ctx->n_valid;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_cache_set_state(sat_ctx *ctx, int32_t write_idx, int32_t n_valid)
+{
+    if (!ctx) return SAT_EINVAL;
+    if (!ctx->cache_ok) return sat_fail(ctx, SAT_ESTATE, "sat_cache_set_state: call sat_cache_init first");
+    if (write_idx < 0 || write_idx > ctx->tau || n_valid < 0 || n_valid > ctx->tau) return sat_fail(ctx, SAT_EINVAL, "sat_cache_set_state: out of range");
+    ctx->write_idx = write_idx;
+    ctx->n_valid = n_valid;
+    for (int i = 0; i < ctx->n_cached; ++i) ctx->cache[i].S_valid = false;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_cache_read(sat_ctx *ctx, int32_t layer, int32_t age, float *out_host)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_cache_read"));
+    if (!out_host || age < -1 || age >= ctx->n_valid) return sat_fail(ctx, SAT_EINVAL, "sat_cache_read: null output or age outside [-1, n_valid)");
+    if (ctx->n_slots == 0) return SAT_OK;
+    const int32_t idx = age < 0 ? ctx->write_idx : ring_index(ctx, age);
+    SAT_CUDA(ctx, cudaMemcpy2DAsync(out_host, (size_t)c->width * 4, ring_buf(ctx, c, idx), (size_t)c->ld * 4, (size_t)c->width * 4,
+                                    (size_t)ctx->n_slots, cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_cache_export(sat_ctx *ctx, int32_t layer, float *out_host)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_cache_export"));
+    if (!out_host) return sat_fail(ctx, SAT_EINVAL, "sat_cache_export: null output");
+    const size_t rows = (size_t)(ctx->tau + 1) * ctx->n_slots;
+    if (rows == 0) return SAT_OK;
+    SAT_CUDA(ctx, cudaMemcpy2DAsync(out_host, (size_t)c->width * 4, c->buf, (size_t)c->ld * 4, (size_t)c->width * 4, rows,
+                                    cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_cache_import(sat_ctx *ctx, int32_t layer, const float *in_host)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_cache_import"));
+    if (!in_host) return sat_fail(ctx, SAT_EINVAL, "sat_cache_import: null input");
+    const size_t rows = (size_t)(ctx->tau + 1) * ctx->n_slots;
+    c->S_valid = false;
+    if (rows == 0) return SAT_OK;
+    SAT_CUDA(ctx, cudaMemcpy2DAsync(c->buf, (size_t)c->ld * 4, in_host, (size_t)c->width * 4, (size_t)c->width * 4, rows,
+                                    cudaMemcpyHostToDevice, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+// =====================================================================================
+// sat_predict
+// =====================================================================================
+// a = x Wx (+ s Uh) + b computed by the dense path into `gates` [rows x 4h] (gate blocks i | f | g | o);
+// this kernel applies the cell:  c = f c + i g ; s = o tanh(c).
+__global__ void k_lstm_cell(const float *__restrict__ gates, int64_t rows, int32_t h, int first, float *__restrict__ c, float *__restrict__ s)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * h) return;
+    const int64_t r = t / h;
+    const int j = (int)(t - r * h);
+    const float *a = gates + r * 4 * (int64_t)h;
+    const float gi = 1.f / (1.f + expf(-a[j]));
+    const float gf = 1.f / (1.f + expf(-a[h + j]));
+    const float gg = tanhf(a[2 * h + j]);
+    const float go = 1.f / (1.f + expf(-a[3 * h + j]));
+    const float cp = first ? 0.f : c[t];
+    const float cn = gf * cp + gi * gg;
+    c[t] = cn;
+    s[t] = go * tanhf(cn);
+}
+
+// dual-operand NN product (defined in sat_gemm.cu): C = [A1 | A2] [B1 ; B2] + bias
+sat_status sat_gemm_nn_dual(sat_ctx *ctx, int64_t m, int32_t n, int32_t k1, const float *A1, int32_t lda1, const float *B1, int32_t ldb1,
+                            int32_t k2, const float *A2, int32_t lda2, const float *B2, int32_t ldb2, const float *bias, float *C,
+                            int32_t ldc);
+
+static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p)
+{
+    const int32_t h = p->h, d = c->width;
+    const int64_t rows = ctx->n_slots;
+    if (!c->S || c->S_h != h) {
+        SAT_TRY(dev_realloc(ctx, &c->S, rows * h));
+        c->S_h = h;
+    }
+    const int32_t k = ctx->n_valid < ctx->tau ? ctx->n_valid : ctx->tau;
+    if (k == 0 || rows == 0) {
+        SAT_CUDA(ctx, cudaMemsetAsync(c->S, 0, (size_t)(rows > 0 ? rows : 1) * h * sizeof(float), ctx->stream));
+        c->S_valid = true;
+        return SAT_OK;
+    }
+    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_w, (size_t)rows * 4 * h * sizeof(float)));
+    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_c, (size_t)rows * h * sizeof(float)));
+    float *gates = (float *)ctx->buf_lstm_w.p;
+    float *cell = (float *)ctx->buf_lstm_c.p;
+    for (int32_t t = 0; t < k; ++t) {
+        const float *x = ring_buf(ctx, c, ring_index(ctx, k - 1 - t));  // oldest first
+        SAT_TRY(sat_gemm_nn_dual(ctx, rows, 4 * h, d, x, c->ld, p->Wx, 4 * h, t == 0 ? 0 : h, c->S, h, p->Uh, 4 * h, p->b, gates, 4 * h));
+        {
+            ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 7.0, 0.0);
+            k_lstm_cell<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(gates, rows, h, t == 0, cell, c->S);
+            SAT_LAUNCHED(ctx);
+        }
+    }
+    c->S_valid = true;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, const sat_pred_params *params, int reuse_state,
+                                  float *halo_out, int32_t ld_out)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_predict"));
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    const int32_t d = c->width;
+    if (v.n_halo > 0 && (!halo_out || !ok_ld(ld_out, d) || !aligned16(halo_out)))
+        return sat_fail(ctx, SAT_EINVAL, "sat_predict: null / misaligned halo_out or bad ld_out");
+    const float *newest = ctx->n_valid > 0 ? ring_buf(ctx, c, ring_index(ctx, 0)) : nullptr;
+    if (!params) {  // identity predictor: plain historical embeddings
+        if (v.n_halo == 0) return SAT_OK;
+        if (!newest) {
+            SAT_CUDA(ctx, cudaMemset2DAsync(halo_out, (size_t)ld_out * 4, 0, (size_t)d * 4, (size_t)v.n_halo, ctx->stream));
+            return SAT_OK;
+        }
+        return sat_gather(ctx, ctx->halo_slot + v.halo0, v.n_halo, d, newest, c->ld, halo_out, ld_out);
+    }
+    if (params->h <= 0 || !params->Wx || !params->Uh || !params->b || !params->Wg || !params->bg)
+        return sat_fail(ctx, SAT_EINVAL, "sat_predict: incomplete predictor parameters");
+    if (reuse_state) {
+        if (!c->S_valid || c->S_h != params->h) return sat_fail(ctx, SAT_ESTATE, "sat_predict: no LSTM state table to reuse for layer %d", layer);
+    } else {
+        SAT_TRY(run_lstm(ctx, c, params));
+    }
+    if (v.n_halo == 0) return SAT_OK;
+    const int32_t h = params->h;
+    const int32_t ld_a = round_up4(h);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_pred_a, (size_t)v.n_halo * ld_a * sizeof(float)));
+    float *a = (float *)ctx->buf_pred_a.p;
+    // graph convolution on the LSTM state: a_u = p_uu S_u + sum_{v in N(u) cap V_m} p_uv S_v
+    // (h is a multiple of 4 or the S rows are not 16-byte aligned: the S table uses ld = h, so require h % 4 == 0)
+    if (h & 3) return sat_fail(ctx, SAT_EINVAL, "sat_predict: predictor width h must be a multiple of 4");
+    SAT_TRY(sat_spmm_hrow(ctx, v, h, c->S, h, 1, c->S, a - v.halo0 * ld_a, ld_a));
+    GemmEpilogue ep;
+    ep.bias = params->bg;
+    if (newest) {
+        ep.resid = newest;
+        ep.resid_idx = ctx->halo_slot + v.halo0;
+        ep.ld_resid = c->ld;
+    }
+    return sat_gemm_nn(ctx, v.n_halo, d, h, a, ld_a, params->Wg, d, halo_out, ld_out, ep);
+}
+
+extern "C" sat_status sat_predict_state(sat_ctx *ctx, int32_t layer, float *S_host, int32_t h)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_predict_state"));
+    if (!S_host) return sat_fail(ctx, SAT_EINVAL, "sat_predict_state: null output");
+    if (!c->S_valid || c->S_h != h) return sat_fail(ctx, SAT_ESTATE, "sat_predict_state: no state table of width %d for layer %d", h, layer);
+    SAT_CUDA(ctx, cudaMemcpyAsync(S_host, c->S, (size_t)ctx->n_slots * h * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+// =====================================================================================
+// sat_layer_fwd / sat_layer_bwd
+// =====================================================================================
+extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in, int32_t d_out, const float *h_in,
+                                    int32_t ld_in, const float *h_halo, int32_t ld_halo, const float *W, const float *bias, int act,
+                                    float *h_out, int32_t ld_out)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    if (d_in <= 0 || d_out <= 0 || !W || (act != SAT_ACT_NONE && act != SAT_ACT_RELU)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: bad dims / W / act");
+    if (v.n_rows > 0 && (!h_in || !h_out || !ok_ld(ld_in, d_in) || !ok_ld(ld_out, d_out) || !aligned16(h_in) || !aligned16(h_out)))
+        return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: null / misaligned h_in / h_out or bad leading dimension");
+    if (v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo)))
+        return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: null / misaligned h_halo or bad ld_halo");
+    LayerState &L = ctx->layers[layer];
+    const int32_t ld_agg = round_up4(d_in), words = (d_out + 31) / 32;
+    if (!L.agg || L.d_in != d_in || L.d_out != d_out) {
+        SAT_TRY(dev_realloc(ctx, &L.agg, (int64_t)ctx->n * ld_agg));
+        SAT_TRY(dev_realloc(ctx, &L.mask, (int64_t)ctx->n * words));
+        L.d_in = d_in;
+        L.d_out = d_out;
+        L.ld_in = ld_agg;
+        L.mask_words = words;
+        L.valid.assign(ctx->M, 0);
+    }
+    L.act = act;
+    if (v.n_rows == 0) return SAT_OK;
+    const float *in_base = h_in - (int64_t)v.row0 * ld_in;
+    const float *halo_base = h_halo ? h_halo - v.halo0 * (int64_t)ld_halo : nullptr;
+    SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg));
+    GemmEpilogue ep;
+    ep.bias = bias;
+    ep.relu = act == SAT_ACT_RELU;
+    if (act == SAT_ACT_RELU) {
+        ep.mask_out = L.mask + (int64_t)v.row0 * words;
+        ep.mask_words = words;
+    }
+    SAT_TRY(sat_gemm_nn(ctx, v.n_rows, d_out, d_in, L.agg + (int64_t)v.row0 * ld_agg, ld_agg, W, d_out, h_out, ld_out, ep));
+    if (part == SAT_ALL_PARTS) L.valid.assign(ctx->M, 1);
+    else L.valid[part] = 1;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g, const float *W,
+                                    float *g_W, float *g_b, int accumulate, float *g_in, int32_t ld_gin, float *g_halo, int32_t ld_gh)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    LayerState &L = ctx->layers[layer];
+    if (!L.agg) return sat_fail(ctx, SAT_ESTATE, "sat_layer_bwd: sat_layer_fwd has not run for layer %d", layer);
+    for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m)
+        if (!L.valid[m]) return sat_fail(ctx, SAT_ESTATE, "sat_layer_bwd: sat_layer_fwd has not run for partition %d of layer %d", m, layer);
+    const int32_t d_in = L.d_in, d_out = L.d_out;
+    if (!W || !g_W) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: null W / g_W");
+    if (v.n_rows > 0 && (!g_out || !ok_ld(ld_g, d_out) || !aligned16(g_out))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: null / misaligned g_out or bad ld_g");
+    if (g_in && v.n_rows > 0 && (!ok_ld(ld_gin, d_in) || !aligned16(g_in))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_in or bad ld_gin");
+    if (g_halo && v.n_halo > 0 && (!ok_ld(ld_gh, d_in) || !aligned16(g_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_halo or bad ld_gh");
+    const uint32_t *mask = L.act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * L.mask_words : nullptr;
+    // G_W (+)= AGG^T D, G_b (+)= 1^T D   with D = g_out o [Z > 0]
+    SAT_TRY(sat_gemm_tn(ctx, v.n_rows, d_in, d_out, L.agg + (int64_t)v.row0 * L.ld_in, L.ld_in, g_out, ld_g, mask, L.mask_words, g_W, d_out,
+                        g_b, accumulate));
+    if ((!g_in && !g_halo) || v.n_rows == 0) return SAT_OK;
+    // G_AGG = D W^T
+    const int32_t ld_ga = round_up4(d_in);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_gagg, (size_t)v.n_rows * ld_ga * sizeof(float)));
+    float *gagg = (float *)ctx->buf_gagg.p;
+    SAT_TRY(sat_gemm_nt(ctx, v.n_rows, d_in, d_out, g_out, ld_g, mask, L.mask_words, W, d_out, gagg, ld_ga));
+    const float *ga_base = gagg - (int64_t)v.row0 * ld_ga;
+    // G_in = P_in^T G_AGG: the inner block of P is symmetric, so P_in^T = P_in (inner prefix of every local row)
+    if (g_in) SAT_TRY(sat_spmm(ctx, v, 1, d_in, ga_base, ld_ga, nullptr, 0, g_in - (int64_t)v.row0 * ld_gin, ld_gin));
+    // G_halo = P_out^T G_AGG over the halo-row CSR
+    if (g_halo) SAT_TRY(sat_spmm_hrow(ctx, v, d_in, ga_base, ld_ga, 0, nullptr, g_halo - v.halo0 * (int64_t)ld_gh, ld_gh));
+    return SAT_OK;
+}
+
+// =====================================================================================
+// loss seed, parameter step
+// =====================================================================================
+// one warp per row
+__global__ void k_loss_ce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const int32_t *__restrict__ y, float scale,
+                          float *__restrict__ g, int64_t ld_g, float *__restrict__ row_loss)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const float *zr = z + r * ld_z;
+    float mx = -INFINITY;
+    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float se = 0.f;
+    for (int c = lane; c < C; c += 32) se += expf(zr[c] - mx);
+    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+    const float lse = mx + logf(se);
+    const int32_t yr = y[r];
+    for (int c = lane; c < C; c += 32) g[r * ld_g + c] = scale * (expf(zr[c] - lse) - (c == yr ? 1.f : 0.f));
+    if (lane == 0) row_loss[r] = scale * (lse - zr[yr]);
+}
+
+__global__ void k_loss_bce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const uint8_t *__restrict__ y, float scale,
+                           float *__restrict__ g, int64_t ld_g, float *__restrict__ row_loss)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const float *zr = z + r * ld_z;
+    const float inv_c = 1.f / (float)C;
+    float acc = 0.f;
+    for (int c = lane; c < C; c += 32) {
+        const float x = zr[c], yv = (float)y[r * C + c];
+        acc += fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))) - yv * x;
+        g[r * ld_g + c] = scale * inv_c * (1.f / (1.f + expf(-x)) - yv);
+    }
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) row_loss[r] = scale * inv_c * acc;
+}
+
+// single block, fixed order: *total += sum(row_loss)
+__global__ void k_loss_sum(const float *__restrict__ row_loss, int64_t rows, double *total)
+{
+    __shared__ double red[256];
+    double s = 0.0;
+    for (int64_t i = threadIdx.x; i < rows; i += 256) s += (double)row_loss[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *total += red[0];
+}
+
+extern "C" sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_t n_classes, const float *z, int32_t ld_z,
+                                    const void *labels, double *loss_sum, float *g, int32_t ld_g)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (kind != SAT_LOSS_SOFTMAX_CE && kind != SAT_LOSS_SIGMOID_BCE) return sat_fail(ctx, SAT_EINVAL, "sat_loss_grad: unknown loss");
+    if (v.n_rows == 0) return SAT_OK;
+    if (n_classes <= 0 || !z || !labels || !g || ld_z < n_classes || ld_g < n_classes) return sat_fail(ctx, SAT_EINVAL, "sat_loss_grad: null tensor or bad shape");
+    SAT_TRY(sat_ensure(ctx, ctx->buf_misc, (size_t)v.n_rows * sizeof(float)));
+    float *row_loss = (float *)ctx->buf_misc.p;
+    const float scale = 1.0f / (float)ctx->n;
+    ProfScope prof(ctx, SATK_LOSS, 8.0 * (double)v.n_rows * n_classes, 0.0);
+    const unsigned blocks = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
+    if (kind == SAT_LOSS_SOFTMAX_CE)
+        k_loss_ce<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, (const int32_t *)labels, scale, g, ld_g, row_loss);
+    else
+        k_loss_bce<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, (const uint8_t *)labels, scale, g, ld_g, row_loss);
+    SAT_LAUNCHED(ctx);
+    if (loss_sum) {
+        k_loss_sum<<<1, 256, 0, ctx->stream>>>(row_loss, v.n_rows, loss_sum);
+        SAT_LAUNCHED(ctx);
+    }
+    return SAT_OK;
+}
+
+__global__ void k_sgd(int64_t count, float *__restrict__ w, const float *__restrict__ g, float lr)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) w[i] = w[i] - lr * g[i];
+}
+
+extern "C" sat_status sat_sgd_step(sat_ctx *ctx, int64_t count, float *w, const float *g, float lr)
+{
+    CHECK_CTX(ctx);
+    if (count < 0 || (count > 0 && (!w || !g))) return sat_fail(ctx, SAT_EINVAL, "sat_sgd_step: null tensor");
+    if (count == 0) return SAT_OK;
+    k_sgd<<<(unsigned)cdiv64(count, 256), 256, 0, ctx->stream>>>(count, w, g, lr);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}

@@ -1,0 +1,299 @@
+// CSR SpMM kernels of the sat_b200 library (aggregation with the propagation matrix P),
+// row gather and row scatter.  All of them are bandwidth-bound: every feature row is moved
+// with 128-bit loads, one group of lanes per work item, warp shuffles broadcast the column
+// ids, and nothing is accumulated with floating-point atomics (results are reproducible).
+#include "sat_internal.h"
+
+__device__ __forceinline__ float4 ld4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ void fma4(float4 &a, float w, const float4 &x)
+{
+    a.x = fmaf(w, x.x, a.x);
+    a.y = fmaf(w, x.y, a.y);
+    a.z = fmaf(w, x.z, a.z);
+    a.w = fmaf(w, x.w, a.w);
+}
+
+template <int G>
+__device__ __forceinline__ unsigned group_mask(int lane_in_warp)
+{
+    return G == 32 ? 0xffffffffu : (((1u << (G & 31)) - 1u) << (lane_in_warp & ~(G - 1)));
+}
+
+// -------------------------------------------------------------------------------------
+// One group of G lanes per work item (a row, or a chunk of SAT_SPMM_CHUNK entries of a
+// long row).  Lane l owns float4 columns l, l+G, ..., l+(NV-1)G of the feature row.
+//   single-chunk rows write  out[row] = dinv[row] * sum_e dinv[col_e] * src[col_e]
+//   chunks of long rows write their un-scaled partial sum to `partial`; k_spmm_fixup adds
+//   them in chunk order.
+// -------------------------------------------------------------------------------------
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ inner_cnt, const int32_t *__restrict__ lenc,
+             const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
+             const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0, int inner_only, int32_t n,
+             int32_t d4, const float *__restrict__ in_base, int64_t ld_in, const float *__restrict__ halo_base, int64_t ld_halo,
+             float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial)
+{
+    const int lane = threadIdx.x & (G - 1);
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    if (gid >= n_items) return;
+    const unsigned mask = group_mask<G>(threadIdx.x & 31);
+    const int col0 = blockIdx.y * (G * NV);  // first float4 column of this block column
+    const int32_t item = item0 + (int32_t)gid;
+    const int32_t row = item_row[item];
+    const int32_t k = item - first_item[row];
+    const int64_t rb = lrowptr[row];
+    const int64_t re = inner_only ? rb + inner_cnt[row] : lrowptr[row + 1];
+    const int64_t e0 = rb + (int64_t)k * SAT_SPMM_CHUNK;
+    const int64_t e1 = (e0 + SAT_SPMM_CHUNK < re) ? e0 + SAT_SPMM_CHUNK : re;
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t eb = e0; eb < e1; eb += G) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float w = 0.f;
+        if (e < e1) {
+            c = __ldg(lenc + e);
+            w = __ldg(dinv_enc + c);
+        }
+        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t cj = __shfl_sync(mask, c, j, G);
+            const float wj = __shfl_sync(mask, w, j, G);
+            const float *src = cj < n ? in_base + (int64_t)cj * ld_in : halo_base + (int64_t)(cj - n) * ld_halo;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
+            }
+        }
+    }
+    const int32_t ms = item_mslot[item];
+    if (ms < 0) {
+        const float s = __ldg(dinv_enc + row);
+        float *o = out_base + (int64_t)row * ld_out;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(s * acc[v].x, s * acc[v].y, s * acc[v].z, s * acc[v].w);
+        }
+    } else {
+        float *o = partial + (int64_t)(ms - mitem0) * (4 * (int64_t)d4);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = acc[v];
+        }
+    }
+}
+
+// rows cut into several chunks: add the partial sums in chunk order, scale, store
+__global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, int32_t n_mrows, const int32_t *__restrict__ first_item,
+                             const int32_t *__restrict__ item_mslot, int32_t mitem0, const float *__restrict__ dinv_enc, int32_t d4,
+                             const float *__restrict__ partial, float *__restrict__ out_base, int64_t ld_out)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= n_mrows) return;
+    const int32_t row = mrows[mrow0 + i];
+    const int32_t it0 = first_item[row], it1 = first_item[row + 1];
+    const int32_t ms0 = item_mslot[it0] - mitem0;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int32_t q = 0; q < it1 - it0; ++q) {
+        const float4 x = *reinterpret_cast<const float4 *>(partial + ((int64_t)(ms0 + q) * d4 + c) * 4);
+        a.x += x.x;
+        a.y += x.y;
+        a.z += x.z;
+        a.w += x.w;
+    }
+    const float s = dinv_enc[row];
+    *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c) = make_float4(s * a.x, s * a.y, s * a.z, s * a.w);
+}
+
+template <int G, int NV>
+static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d4, const float *in_base, int32_t ld_in,
+                         const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial)
+{
+    dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
+    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->dinv_enc, ctx->item_row,
+                                                        ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
+                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial);
+}
+
+sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
+                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out)
+{
+    if (v.n_items == 0) return SAT_OK;
+    const int32_t d4 = (d + 3) / 4;
+    // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once
+    const double n_src = inner_only ? (double)v.n_rows : (double)v.n_rows + (double)v.n_halo;
+    const double n_ent = (double)v.lnnz;  // the backward uses the inner prefix of every row; counted in full here
+    ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
+                   4.0 * n_ent + 12.0 * v.n_rows + 4.0 * n_src + 4.0 * d * (n_src + v.n_rows), 2.0 * n_ent * d);
+    float *partial = nullptr;
+    if (v.n_mitems > 0) {
+        SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * d4 * 16));
+        partial = (float *)ctx->buf_partial.p;
+    }
+#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial
+    if (d4 <= 4) launch_items<4, 1>(ARGS);
+    else if (d4 <= 8) launch_items<8, 1>(ARGS);
+    else if (d4 <= 16) launch_items<16, 1>(ARGS);
+    else if (d4 <= 32) launch_items<32, 1>(ARGS);
+    else if (d4 <= 64) launch_items<32, 2>(ARGS);
+    else if (d4 <= 96) launch_items<32, 3>(ARGS);
+    else if (d4 <= 128) launch_items<32, 4>(ARGS);
+    else if (d4 <= 160) launch_items<32, 5>(ARGS);
+    else if (d4 <= 192) launch_items<32, 6>(ARGS);
+    else launch_items<32, 8>(ARGS);
+#undef ARGS
+    SAT_LAUNCHED(ctx);
+    if (v.n_mrows > 0) {
+        k_spmm_fixup<<<(unsigned)cdiv64((int64_t)v.n_mrows * d4, 256), 256, 0, ctx->stream>>>(
+            ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, ctx->dinv_enc, d4, partial, out_base, ld_out);
+        SAT_LAUNCHED(ctx);
+    }
+    return SAT_OK;
+}
+
+// -------------------------------------------------------------------------------------
+// Halo-row products (rows = halo entries of the partition, columns = their neighbours
+// inside the partition):
+//   out[j] = dinv[u_j] * ( [self] dinv[u_j] * self_src[halo_slot_j] + sum_e dinv[v_e] * src[idx_e] )
+// idx_e is the partition-major row of v_e (by_slot = 0) or its cache slot (by_slot = 1).
+// Used for the predictor's graph convolution on the LSTM state (self term, by slot) and for
+// the optional halo gradient P_out^T G_AGG (no self term, by row).
+// -------------------------------------------------------------------------------------
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
+            const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
+            int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
+            float *__restrict__ out_base, int64_t ld_out)
+{
+    const int lane = threadIdx.x & (G - 1);
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    if (gid >= n_halo) return;
+    const unsigned mask = group_mask<G>(threadIdx.x & 31);
+    const int col0 = blockIdx.y * (G * NV);
+    const int64_t j = halo0 + gid;
+    const float du = __ldg(dinv_enc + n + j);
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (self_src) {
+        const float *src = self_src + (int64_t)halo_slot[j] * ld_src;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
+        }
+    }
+    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+    for (int64_t eb = e0; eb < e1; eb += G) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float w = 0.f;
+        if (e < e1) {
+            const int32_t p = __ldg(hrow_pos + e);
+            w = __ldg(dinv_enc + p);
+            c = by_slot ? __ldg(hrow_slot + e) : p;
+        }
+        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
+#pragma unroll 4
+        for (int q = 0; q < cnt; ++q) {
+            const int32_t cj = __shfl_sync(mask, c, q, G);
+            const float wj = __shfl_sync(mask, w, q, G);
+            const float *src = src_base + (int64_t)cj * ld_src;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
+            }
+        }
+    }
+    float *o = out_base + j * ld_out;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int idx = col0 + lane + v * G;
+        if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(du * acc[v].x, du * acc[v].y, du * acc[v].z, du * acc[v].w);
+    }
+}
+
+template <int G, int NV>
+static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4, const float *src_base, int32_t ld_src,
+                        const float *self_src, float *out_base, int32_t ld_out)
+{
+    dim3 grid((unsigned)cdiv64(v.n_halo * G, 256), (unsigned)cdiv64(d4, G * NV));
+    k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->halo_slot, ctx->dinv_enc, ctx->n,
+                                                       v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out);
+}
+
+sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src, int by_slot,
+                         const float *self_src, float *out_base, int32_t ld_out)
+{
+    if (v.n_halo == 0) return SAT_OK;
+    const int32_t d4 = (d + 3) / 4;
+    ProfScope prof(ctx, SATK_SPMM_HROW, 0.0, 0.0);
+#define ARGS ctx, v, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out
+    if (d4 <= 4) launch_hrow<4, 1>(ARGS);
+    else if (d4 <= 8) launch_hrow<8, 1>(ARGS);
+    else if (d4 <= 16) launch_hrow<16, 1>(ARGS);
+    else if (d4 <= 32) launch_hrow<32, 1>(ARGS);
+    else if (d4 <= 64) launch_hrow<32, 2>(ARGS);
+    else if (d4 <= 128) launch_hrow<32, 4>(ARGS);
+    else launch_hrow<32, 8>(ARGS);
+#undef ARGS
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+// -------------------------------------------------------------------------------------
+// row gather / scatter (pull of raw features, push into the cache, identity predictor)
+// -------------------------------------------------------------------------------------
+__global__ void k_gather_rows(const int32_t *__restrict__ idx, int64_t count, int32_t d4, const float *__restrict__ src, int64_t ld_src,
+                              float *__restrict__ out, int64_t ld_out)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= count) return;
+    const float4 x = ld4(src + (int64_t)idx[i] * ld_src + 4 * c);
+    *reinterpret_cast<float4 *>(out + i * ld_out + 4 * c) = x;
+}
+
+sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d, const float *src, int32_t ld_src, float *out,
+                      int32_t ld_out)
+{
+    if (count == 0) return SAT_OK;
+    const int32_t d4 = (d + 3) / 4;
+    ProfScope prof(ctx, SATK_GATHER, (8.0 * d + 4.0) * (double)count, 0.0);
+    k_gather_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(idx, count, d4, src, ld_src, out, ld_out);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+__global__ void k_scatter_rows(const int32_t *__restrict__ src_row, const int32_t *__restrict__ dst_row, int64_t count, int32_t d4,
+                               const float *__restrict__ src_base, int64_t ld_src, float *__restrict__ dst, int64_t ld_dst)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= count) return;
+    const float4 x = ld4(src_base + (int64_t)src_row[i] * ld_src + 4 * c);
+    *reinterpret_cast<float4 *>(dst + (int64_t)dst_row[i] * ld_dst + 4 * c) = x;
+}
+
+sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
+                       int32_t ld_src, float *dst, int32_t ld_dst)
+{
+    if (count == 0) return SAT_OK;
+    const int32_t d4 = (d + 3) / 4;
+    ProfScope prof(ctx, SATK_SCATTER, (8.0 * d + 8.0) * (double)count, 0.0);
+    k_scatter_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(src_row, dst_row, count, d4, src_base, ld_src, dst, ld_dst);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}

@@ -1,0 +1,126 @@
+"""One SAT epoch as a sequence of library calls (Algorithm 1 of the paper, epoch body).
+
+This module only owns device buffers (torch tensors) and strings the C entry points
+together in the order of Algorithm 1:  for every layer: pull (predict) -> forward ->
+push;  then loss, backward, commit.  It contains no arithmetic of its own.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+
+
+def _pad4(d: int) -> int:
+    return (d + 3) & ~3
+
+
+def _buf(rows: int, d: int, device) -> torch.Tensor:
+    """[rows, d] view of a zero-initialised buffer whose row stride is a multiple of 4 floats."""
+    full = torch.zeros((max(rows, 1), _pad4(d)), dtype=torch.float32, device=device)
+    return full[:rows, :d]
+
+
+class SatEpoch:
+    """Holds a context, the partitioned graph, the cache ring and the activation / gradient buffers
+    of a GCN with layer widths `dims`, and runs epochs either with one launch set for all
+    partitions (`step`) or partition by partition (`step_per_partition`)."""
+
+    def __init__(self, rowptr, col, M: int, dims, tau: int, loss: str, part_given=None, device: int = 0):
+        self.device = torch.device("cuda", device)
+        torch.cuda.set_device(self.device)
+        self.stream = torch.cuda.current_stream(self.device)
+        self.ctx = B.sat_create(device, self.stream.cuda_stream)
+        self.n = int(rowptr.shape[0] - 1)
+        self.M, self.dims, self.tau, self.loss = M, list(dims), tau, loss
+        self.L = len(dims) - 1
+        B.sat_graph_load(self.ctx, rowptr, col)
+        if part_given is None:
+            B.sat_partition(self.ctx, M, B.SAT_PART_CONTIG_BLOCKS)
+        else:
+            B.sat_partition(self.ctx, M, B.SAT_PART_GIVEN, part_given)
+        self.sizes = [B.sat_part_sizes(self.ctx, m) for m in range(M)]
+        tot = B.sat_part_sizes(self.ctx, B.SAT_ALL_PARTS)
+        self.nb, self.nnz, self.n_slots = tot[1], tot[2], tot[3]
+        self.inner_off = np.concatenate([[0], np.cumsum([s[0] for s in self.sizes])]).astype(np.int64)
+        self.halo_off = np.concatenate([[0], np.cumsum([s[1] for s in self.sizes])]).astype(np.int64)
+        B.sat_cache_init(self.ctx, self.dims[1:-1], tau)
+        dev = self.device
+        self.H = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # H[l], l = 1..L (partition-major rows)
+        self.G = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # gradient w.r.t. H[l]
+        self.halo = _buf(self.nb, max(self.dims[:-1]), dev)                       # halo input of the running layer
+        self.X_in = _buf(self.n, self.dims[0], dev)
+        self.gW = [torch.zeros((self.dims[l], self.dims[l + 1]), dtype=torch.float32, device=dev) for l in range(self.L)]
+        self.gb = [torch.zeros(self.dims[l + 1], dtype=torch.float32, device=dev) for l in range(self.L)]
+        self.loss_sum = torch.zeros(1, dtype=torch.float64, device=dev)
+        self.X = None
+        self.labels = None
+
+    def close(self):
+        if self.ctx is not None:
+            B.sat_destroy(self.ctx)
+            self.ctx = None
+
+    # ---- inputs -------------------------------------------------------------------
+    def set_inputs(self, X: torch.Tensor, labels_perm: torch.Tensor):
+        """X: [n, d0] CUDA features in global id order (row stride multiple of 4);
+        labels_perm: labels in partition-major row order (int32 [n] or uint8 [n, C])."""
+        self.X = X
+        self.labels = labels_perm
+        B.sat_gather_rows(self.ctx, B.SAT_ALL_PARTS, B.SAT_ROWS_INNER, X, self.X_in)
+
+    def halo_view(self, d: int, m: int = B.SAT_ALL_PARTS):
+        if m == B.SAT_ALL_PARTS:
+            return self.halo[:, :d]
+        return self.halo[self.halo_off[m]:self.halo_off[m + 1], :d]
+
+    def rows(self, t: torch.Tensor, m: int):
+        if m == B.SAT_ALL_PARTS:
+            return t
+        return t[self.inner_off[m]:self.inner_off[m + 1]]
+
+    # ---- one epoch ----------------------------------------------------------------
+    def _forward_backward(self, m: int, W, b, pred, accumulate: int, reuse_state: int):
+        ctx, L = self.ctx, self.L
+        h_in = self.rows(self.X_in, m)
+        for l in range(1, L + 1):
+            d_in = self.dims[l - 1]
+            hv = self.halo_view(d_in, m)
+            if l == 1:
+                B.sat_gather_rows(ctx, m, B.SAT_ROWS_HALO, self.X, hv)                 # pull raw features
+            else:
+                B.sat_predict(ctx, l - 1, m, pred[l - 2] if pred is not None else None, reuse_state, hv)  # pull predicted
+            h_out = self.rows(self.H[l], m)
+            B.sat_layer_fwd(ctx, m, l, h_in, hv, W[l - 1], b[l - 1], B.SAT_ACT_RELU if l < L else B.SAT_ACT_NONE, h_out)
+            if l < L:
+                B.sat_cache_update(ctx, m, l, h_out)                                    # push
+            h_in = h_out
+        kind = B.SAT_LOSS_SOFTMAX_CE if self.loss == "ce" else B.SAT_LOSS_SIGMOID_BCE
+        g = self.rows(self.G[L], m)
+        B.sat_loss_grad(ctx, m, kind, self.rows(self.H[L], m), self.rows(self.labels, m), self.loss_sum, g)
+        for l in range(L, 0, -1):
+            g_in = self.rows(self.G[l - 1], m) if l > 1 else None
+            B.sat_layer_bwd(ctx, m, l, g, W[l - 1], self.gW[l - 1], self.gb[l - 1], accumulate, g_in, None)
+            g = g_in
+
+    def step(self, W, b, pred, lr: float | None = None):
+        """All partitions per launch.  W, b: lists of CUDA tensors; pred: list of sat_pred_params or None."""
+        self.loss_sum.zero_()
+        self._forward_backward(B.SAT_ALL_PARTS, W, b, pred, 0, 0)
+        B.sat_cache_commit(self.ctx)
+        if lr is not None:
+            for l in range(self.L):
+                B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
+                B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
+
+    def step_per_partition(self, W, b, pred, order=None, lr: float | None = None):
+        """Same epoch, one partition at a time (the LSTM state table is computed by the first call of every layer)."""
+        self.loss_sum.zero_()
+        for i, m in enumerate(order if order is not None else range(self.M)):
+            self._forward_backward(m, W, b, pred, 0 if i == 0 else 1, 0 if i == 0 else 1)
+        B.sat_cache_commit(self.ctx)
+        if lr is not None:
+            for l in range(self.L):
+                B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
+                B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
