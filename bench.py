@@ -1,0 +1,343 @@
+#!/usr/bin/env python
+"""Benchmark of the SAT epoch step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload medium]
+
+A step is one steady-state SAT epoch over all partitions of the workload: layer-1 halo
+pull, predictor (LSTM over the cached snapshots + graph convolution + skip) for every
+cached layer, every layer forward (SpMM + transform), cache push, loss seed, every layer
+backward, ring commit and the SGD step.  metric = edges/s = nnz(A + I) / epoch time.
+Prints ONE JSON line on rank 0.
+
+--impl reference times the CPU oracle (as it stands) on the host cores instead, on a
+bounded sample of the same workload per step.
+With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica of the
+workload (the path of this build does not shard across GPUs; there is no collective on
+the data path); the value is the aggregate over ranks, timed as the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel on the benchmark
+# workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
+NCU_TRAFFIC_BYTES = {}
+
+FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), bf16=float(p["bf16_tflops_sustained"]), source="measured")
+    return dict(hbm=6650.0, bf16=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        for ln in self.lines:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    power_w_max=max(power) if power else None, samples=len(sm), reasons=sorted(reasons))
+
+
+# ------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline of the default run, and the whole of --impl reference)
+# ------------------------------------------------------------------------------------------
+class OracleSample:
+    """The oracle on a bounded sample of the workload: `k` partitions per step (all their layers, forward and
+    backward, plus the LSTM for the cached nodes they read), from a full ring (tau snapshots of synthetic
+    non-negative embeddings — the work does not depend on the values)."""
+
+    def __init__(self, wl):
+        from oracle import sat_ref as orc
+        self.orc, self.wl = orc, wl
+        part = wl.part_given if wl.part_given is not None else orc.contig_blocks(wl.n, wl.M)
+        self.dtil, _ = orc.degrees(wl.rowptr)
+        self.P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+        self.cache = orc.CacheRing(self.P.n_slots, wl.dims[1:-1], wl.tau)
+        rng = np.random.default_rng(0)
+        for buf in self.cache.buf:
+            buf[:] = np.abs(rng.standard_normal(buf.shape, dtype=np.float32))
+        self.cache.n_valid = wl.tau
+        self.cores = orc.num_threads()
+
+    def run(self, parts):
+        wl = self.wl
+        t0 = time.perf_counter()
+        self.orc.run_epoch(self.P, self.dtil, self.cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=True, parts=parts)
+        dt = time.perf_counter() - t0
+        edges = sum(int(self.P.loc_rowptr[m][-1]) for m in parts)
+        return edges, dt
+
+
+def run_reference(args, wl):
+    """--impl reference: the oracle, one partition per step (rotating), W warm-up steps then K timed steps."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample(wl)
+    for i in range(args.warmup):
+        smp.run([i % wl.M])
+    edges, secs = 0, 0.0
+    for i in range(args.steps):
+        e, t = smp.run([(args.warmup + i) % wl.M])
+        edges += e
+        secs += t
+    value = edges / secs
+    sample = (f"per step: 1 of {wl.M} partitions (rotating) of the {wl.name} workload, all layers fwd+bwd+predictor "
+              f"incl. the LSTM for the cached nodes that partition reads; ring full (tau={wl.tau})")
+    line = dict(impl="reference", metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s",
+                n_gpus=0, steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * secs / max(args.steps, 1), higher_is_better=True,
+                scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=workload_config(wl),
+                cpu_baseline=dict(value=value, unit="edges/s", cores=smp.cores, kind="oracle", sample=sample),
+                e2e=dict(value=value, unit="edges/s", h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(wl):
+    return dict(workload=f"{wl.name}: {wl.n} nodes, nnz(A+I)={wl.nnz}, GCN {'-'.join(map(str, wl.dims))}, "
+                         f"{wl.M} partitions (contiguous id blocks after BFS relabel), predictor history {wl.tau}, h={wl.pred[0]['h'] if wl.pred else 0}",
+                nodes=wl.n, nnz=wl.nnz, partitions=wl.M, tau=wl.tau,
+                l2="working set per epoch (activations, saved aggregations, ring) far exceeds the 126 MB L2; no flush")
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args, wl):
+    import torch
+    import paper_2308_13466_b200.binding as B
+    from paper_2308_13466_b200.epoch import SatEpoch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU implementation")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def up(a):
+        return torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+
+    def pad2d(a):
+        full = torch.zeros((a.shape[0], (a.shape[1] + 3) & ~3), dtype=torch.float32, device=dev)
+        v = full[:, :a.shape[1]]
+        v.copy_(torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)))
+        return v
+
+    ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss, part_given=wl.part_given, device=local)
+    perm = np.empty(wl.n, dtype=np.int64)
+    off = 0
+    for m in range(wl.M):
+        lst = B.sat_part_lists(ep.ctx, m)["inner_gid"]
+        perm[off:off + lst.shape[0]] = lst
+        off += lst.shape[0]
+    X_dev = pad2d(wl.X)
+    labels_perm = np.ascontiguousarray(wl.labels[perm])
+    ep.set_inputs(X_dev, up(labels_perm))
+    W = [up(w) for w in wl.W]
+    b = [up(x) for x in wl.b]
+    preds = [B.make_pred_params(up(p["Wx"]), up(p["Uh"]), up(p["b"]), up(p["Wg"]), up(p["bg"]), int(p["h"])) for p in wl.pred]
+    lr = 0.01
+
+    # fill the ring with real embeddings (tau + 1 epochs), then W warm-up steps
+    for _ in range(wl.tau + 1):
+        ep.step(W, b, preds, lr)
+    for _ in range(max(args.warmup, 0)):
+        ep.step(W, b, preds, lr)
+    stream = torch.cuda.current_stream(dev)
+
+    # ---- device-resident timing ----
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    B.sat_profile_enable(ep.ctx, True)
+    launches0 = B.sat_launch_count(ep.ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        ep.step(W, b, preds, lr)
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = B.sat_launch_count(ep.ctx) - launches0
+    prof = B.sat_profile_read(ep.ctx)
+    B.sat_profile_enable(ep.ctx, False)
+    clocks = sampler.stop()
+    loss = float(ep.loss_sum.item())
+
+    # ---- end to end: host buffers in, host results out, every step ----
+    hX = torch.from_numpy(np.ascontiguousarray(wl.X)).pin_memory()
+    hlab = torch.from_numpy(labels_perm).pin_memory()
+    hW = [torch.from_numpy(w.copy()).pin_memory() for w in wl.W]
+    hb = [torch.from_numpy(x.copy()).pin_memory() for x in wl.b]
+    h_loss = torch.zeros(1, dtype=torch.float64).pin_memory()
+    h_gW = [torch.zeros(w.shape, dtype=torch.float32).pin_memory() for w in wl.W]
+    lab_dev = ep.labels
+    e2e_steps = max(3, min(args.steps, 10))
+    h2d = hX.numel() * 4 + hlab.numel() * hlab.element_size() + sum(w.numel() * 4 for w in hW) + sum(x.numel() * 4 for x in hb)
+    d2h = 8 + sum(g.numel() * 4 for g in h_gW)
+
+    def e2e_step():
+        X_dev.copy_(hX, non_blocking=True)
+        lab_dev.copy_(hlab, non_blocking=True)
+        for d_, h_ in zip(W, hW):
+            d_.copy_(h_, non_blocking=True)
+        for d_, h_ in zip(b, hb):
+            d_.copy_(h_, non_blocking=True)
+        ep.set_inputs(X_dev, lab_dev)
+        ep.step(W, b, preds, None)
+        h_loss.copy_(ep.loss_sum, non_blocking=True)
+        for h_, d_ in zip(h_gW, ep.gW):
+            h_.copy_(d_, non_blocking=True)
+        stream.synchronize()
+
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- max over ranks ----
+    if dist is not None:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+    ms_per_step = ms / args.steps
+    value = world * wl.nnz / (ms_per_step * 1e-3)
+    e2e_value = world * wl.nnz * e2e_steps / e2e_s
+
+    if rank == 0:
+        peaks = measured_peaks()
+        fam = max(prof, key=lambda k: prof[k]["ms"])
+        rec = prof[fam]
+        per_launch_ms = rec["ms"] / max(rec["calls"], 1)
+        if fam.startswith("gemm"):
+            tfl = rec["flops"] / (rec["ms"] * 1e-3) / 1e12
+            roofline = dict(kernel=fam, bound="alu", achieved=tfl, peak=FP32_ALU_PEAK_TFLOPS, unit="TFLOP/s",
+                            frac=tfl / FP32_ALU_PEAK_TFLOPS, traffic=NCU_TRAFFIC_BYTES.get(fam),
+                            peak_source="derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz")
+        else:
+            gbs = rec["bytes"] / (rec["ms"] * 1e-3) / 1e9
+            roofline = dict(kernel=fam, bound="hbm", achieved=gbs, peak=peaks["hbm"], unit="GB/s", frac=gbs / peaks["hbm"],
+                            traffic=NCU_TRAFFIC_BYTES.get(fam), peak_source=f"{peaks['source']} HBM copy bandwidth")
+        roofline.update(launches=rec["calls"], ms_per_launch=per_launch_ms, share_of_step=rec["ms"] / ms)
+        families = {k: dict(calls=v["calls"], ms_per_step=v["ms"] / args.steps,
+                            gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else 0.0,
+                            tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else 0.0)
+                    for k, v in prof.items() if v["calls"]}
+        cpu = None
+        if world == 1 and not args.no_cpu_baseline:
+            smp = OracleSample(wl)
+            k = max(1, wl.M // 2)
+            edges, secs = smp.run(list(range(k)))
+            cpu = dict(value=edges / secs, unit="edges/s", cores=smp.cores, kind="oracle", seconds=secs,
+                       sample=f"partitions 0..{k - 1} of {wl.M} of the {wl.name} workload (all layers fwd+bwd+predictor, "
+                              f"LSTM for the cached nodes they read), ring full; {edges} edges")
+        line = dict(metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s", n_gpus=world,
+                    steps=args.steps, warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
+                    vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
+                    e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps),
+                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, kernel_families=families,
+                    loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
+                    multi_gpu="replicas only" if world > 1 else None)
+        print(json.dumps(line), flush=True)
+    ep.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="medium")
+    ap.add_argument("--shrink", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from sat_synth import make_workload
+    if args.impl == "reference" and int(os.environ.get("RANK", "0")) != 0:
+        return
+    wl = make_workload(args.workload, shrink=args.shrink)
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        import __graft_entry__
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            from paper_2308_13466_b200.build import build
+            build()
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

@@ -297,6 +297,7 @@ class EpochResult:
     G_b: list
     per_part: list      # per partition: dict(H=[H^(1..L)], halo=[Hhat inputs of layers 1..L], G_in=[...], Z=[...], AGG=[...])
     S: list             # per cached layer: LSTM state table or None (identity predictor)
+    S_slots: object = None  # slots for which S was computed (None = all)
 
 
 def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, loss_kind: str,
@@ -315,13 +316,18 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
         ms = list(order)
     # LSTM state table: depends only on committed snapshots, one per cached layer
     S = []
+    sel = None
+    if parts is not None:
+        # only the cached nodes these partitions read: their halo nodes and the halo nodes' neighbours inside them
+        need = [P.halo_slot[m] for m in ms] + [P.slot[P.inner_gid[m][P.hrow_col[m]]] for m in ms]
+        sel = np.unique(np.concatenate(need)) if need else np.empty(0, dtype=np.int32)
     for l in range(1, L):
         pr = pred[l - 1] if pred is not None else None
         if pr is None:
             S.append(None)
         else:
             h, d = pr["Wg"].shape
-            S.append(lstm_state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots))
+            S.append(lstm_state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots, slots_sel=sel))
     G_W = [np.zeros(w.shape, dtype=np.float64) for w in W]
     G_b = [np.zeros(w.shape[1], dtype=np.float64) for w in W]
     total_loss = 0.0
@@ -369,4 +375,4 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
         per_part[m] = rec
     if parts is None:
         cache.commit()
-    return EpochResult(loss=total_loss, G_W=G_W, G_b=G_b, per_part=per_part, S=S)
+    return EpochResult(loss=total_loss, G_W=G_W, G_b=G_b, per_part=per_part, S=S, S_slots=sel)

@@ -57,7 +57,7 @@ EXPORTS = [
     "sat_part_sizes", "sat_part_lists", "sat_slot_map", "sat_gather_rows", "sat_cache_init", "sat_predict",
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
-    "sat_launch_count",
+    "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
 ]
 
 
@@ -276,3 +276,23 @@ def sat_launch_count(ctx) -> int:
     c = C.c_int64()
     _check(ctx, _lib.sat_launch_count(ctx, C.byref(c)))
     return c.value
+
+
+def sat_profile_families() -> int:
+    return int(_lib.sat_profile_families())
+
+
+def sat_profile_enable(ctx, enable: bool):
+    _check(ctx, _lib.sat_profile_enable(ctx, C.c_int(1 if enable else 0)))
+
+
+def sat_profile_read(ctx) -> dict:
+    """{family name: dict(calls, ms, bytes, flops)} of the calls bracketed since sat_profile_enable(True)."""
+    out = {}
+    for f in range(sat_profile_families()):
+        name = C.c_char_p()
+        calls = C.c_int64()
+        ms, by, fl = C.c_double(), C.c_double(), C.c_double()
+        _check(ctx, _lib.sat_profile_read(ctx, C.c_int32(f), C.byref(name), C.byref(calls), C.byref(ms), C.byref(by), C.byref(fl)))
+        out[name.value.decode()] = dict(calls=calls.value, ms=ms.value, bytes=by.value, flops=fl.value)
+    return out
