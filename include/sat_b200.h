@@ -247,6 +247,21 @@ sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_t n_classes
                          const void *labels, double *loss_sum, float *g, int32_t ld_g);
 sat_status sat_sgd_step(sat_ctx *ctx, int64_t count, float *w, const float *g, float lr);
 
+/* ---------------------------------------------------------------------------------------
+ * The dense contractions of the layer step on caller tensors (all DEVICE fp32; the paper has no counterpart:
+ * they are the matrix products inside the forward / backward formulas of the Appendix, exposed so that the
+ * kernels can be exercised and measured in isolation).  Same kernels and same path selection as inside
+ * sat_layer_fwd / sat_layer_bwd / sat_predict.
+ *   sat_dense_nn: C[m x n] = A[m x k] W[k x n] + bias        (W dense row-major, bias [n] or NULL)
+ *   sat_dense_nt: C[m x n] = A[m x k] W[n x k]^T
+ *   sat_dense_tn: C[m x n] = A[rows x m]^T B[rows x n]        (C dense row-major)
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_dense_nn(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W, const float *bias,
+                        float *C, int32_t ldc);
+sat_status sat_dense_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W, float *C, int32_t ldc);
+sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
+                        float *C);
+
 /* Number of kernels this context has launched since creation (all entry points). */
 sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
 
@@ -256,7 +271,7 @@ sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
  * for family f in [0, sat_profile_families()), its name, number of bracketed calls, total milliseconds and the
  * algorithmic bytes / flops those calls moved / performed (each operand read once, each result written once). */
 enum { SAT_PROF_SPMM_FWD = 0, SAT_PROF_SPMM_BWD, SAT_PROF_SPMM_HROW, SAT_PROF_GEMM_NN, SAT_PROF_GEMM_NT,
-       SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS };
+       SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS, SAT_PROF_MASK };
 int32_t sat_profile_families(void);
 sat_status sat_profile_enable(sat_ctx *ctx, int enable);
 sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int64_t *calls, double *ms, double *bytes,

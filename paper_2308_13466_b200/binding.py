@@ -57,7 +57,7 @@ EXPORTS = [
     "sat_part_sizes", "sat_part_lists", "sat_slot_map", "sat_gather_rows", "sat_cache_init", "sat_predict",
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
-    "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
+    "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
 ]
 
 
@@ -270,6 +270,27 @@ def sat_loss_grad(ctx, part: int, kind: int, z, labels, loss_sum, g):
 def sat_sgd_step(ctx, w, g, lr: float):
     assert w.is_contiguous() and g.is_contiguous() and w.numel() == g.numel()
     _check(ctx, _lib.sat_sgd_step(ctx, C.c_int64(w.numel()), _dev(w), _dev(g), C.c_float(lr)))
+
+
+def sat_dense_nn(ctx, A, W, bias, out):
+    """out[m, n] = A[m, k] W[k, n] + bias"""
+    assert W.is_contiguous()
+    _check(ctx, _lib.sat_dense_nn(ctx, C.c_int64(A.shape[0]), C.c_int32(W.shape[1]), C.c_int32(W.shape[0]), _dev(A), C.c_int32(_ld(A)),
+                                  _dev(W), _dev(bias), _dev(out), C.c_int32(_ld(out))))
+
+
+def sat_dense_nt(ctx, A, W, out):
+    """out[m, n] = A[m, k] W[n, k]^T"""
+    assert W.is_contiguous()
+    _check(ctx, _lib.sat_dense_nt(ctx, C.c_int64(A.shape[0]), C.c_int32(W.shape[0]), C.c_int32(W.shape[1]), _dev(A), C.c_int32(_ld(A)),
+                                  _dev(W), _dev(out), C.c_int32(_ld(out))))
+
+
+def sat_dense_tn(ctx, A, Bm, out):
+    """out[m, n] = A[rows, m]^T Bm[rows, n]  (out dense)"""
+    assert out.is_contiguous()
+    _check(ctx, _lib.sat_dense_tn(ctx, C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A), C.c_int32(_ld(A)),
+                                  _dev(Bm), C.c_int32(_ld(Bm)), _dev(out)))
 
 
 def sat_launch_count(ctx) -> int:

@@ -93,12 +93,12 @@ extern "C" sat_status sat_create(sat_ctx **out, int device, void *cuda_stream)
     if (!ctx) return SAT_ENOMEM;
     ctx->device = device;
     ctx->stream = (cudaStream_t)cuda_stream;
-    if (cudaMalloc((void **)&ctx->d_flag, sizeof(int)) != cudaSuccess ||
+    if (cudaMalloc((void **)&ctx->d_flag, 2 * sizeof(int)) != cudaSuccess ||
         cudaMallocHost((void **)&ctx->h_flag, sizeof(int)) != cudaSuccess) {
         delete ctx;
         return SAT_ENOMEM;
     }
-    cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), ctx->stream);
+    cudaMemsetAsync(ctx->d_flag, 0, 2 * sizeof(int), ctx->stream);  // [0] validation flags, [1] kernel wait time-outs
     *out = ctx;
     return SAT_OK;
 }
@@ -167,6 +167,10 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_lstm_w);
     sat_free_buf(ctx->buf_pred_a);
     sat_free_buf(ctx->buf_misc);
+    sat_free_buf(ctx->buf_colsum);
+    sat_free_buf(ctx->buf_dmask);
+    sat_free_buf(ctx->buf_wsplit);
+    sat_free_buf(ctx->buf_wsplit2);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;
@@ -180,6 +184,12 @@ extern "C" sat_status sat_sync_status(sat_ctx *ctx)
     if (!ctx) return SAT_EINVAL;
     SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     if (ctx->cuda_failed) return SAT_ECUDA;
+    SAT_CUDA(ctx, cudaMemcpyAsync(ctx->h_flag, ctx->d_flag + 1, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (*ctx->h_flag) {
+        ctx->cuda_failed = true;
+        return sat_fail(ctx, SAT_ECUDA, "a tensor-core kernel gave up waiting on a barrier (status %d)", *ctx->h_flag);
+    }
     return SAT_OK;
 }
 
@@ -194,7 +204,7 @@ extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
 // per-family device timing
 // =====================================================================================
 static const char *k_family_names[SATK_COUNT] = {"spmm_fwd", "spmm_bwd", "spmm_hrow", "gemm_nn", "gemm_nt", "gemm_tn",
-                                                 "lstm_cell", "gather", "scatter", "loss"};
+                                                 "lstm_cell", "gather", "scatter", "loss", "mask"};
 
 static void prof_clear(sat_ctx *ctx)
 {

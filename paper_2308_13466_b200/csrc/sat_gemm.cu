@@ -255,6 +255,15 @@ __global__ void k_splitk_reduce(const float *__restrict__ part, int64_t count, i
     *o = accumulate ? *o + s : s;
 }
 
+sat_status sat_splitk_reduce(sat_ctx *ctx, const float *part, int64_t count, int32_t splits, int accumulate, float *out, int32_t ncols,
+                             int32_t ld_out)
+{
+    if (count == 0) return SAT_OK;
+    k_splitk_reduce<<<(unsigned)cdiv64(count, 256), 256, 0, ctx->stream>>>(part, count, splits, accumulate, out, ncols, ld_out);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
 sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
                        const uint32_t *mask, int32_t mask_words, float *C, int32_t ldc, float *colsum, int accumulate)
 {

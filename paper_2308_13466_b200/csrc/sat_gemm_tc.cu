@@ -1,0 +1,652 @@
+// Dense contractions on the 5th-generation tensor cores (tcgen05.mma kind::tf32, accumulators in TMEM,
+// operands staged in shared memory by TMA) with fp32-level accuracy from a two-term TF32 split:
+//     x = hi + lo,  hi = tf32(x), lo = tf32(x - hi)            (|x - hi - lo| <= 2^-22 |x|)
+//     A B ~= Ah Bh + Ah Bl + Al Bh                              (three MMAs per k-step, fp32 accumulate)
+// Activations stay plain fp32 in global memory: TMA brings the fp32 tile into shared memory and the
+// converter warps round it to TF32 in place and write the residual tile next to it (element-wise, so the
+// swizzled layout never has to be decoded).  Weights are pre-split once per call into two fp32 planes.
+//
+//   k_gemm_tc_k   C[M x N] = A[M x K] B[N x K]^T   both operands K-major, 64-byte swizzle, BLOCK_K = 16
+//                 (layer transform, LSTM gates with two A operands, predictor output, input gradient)
+//   k_gemm_tc_mn  C[M x N] = A[R x M]^T B[R x N]   both operands MN-major, 128-byte swizzle with 32-byte atoms, split over R
+//                 (weight gradient)
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = converters during the
+// main loop, then epilogue (one TMEM lane quadrant each).  Every mbarrier wait is bounded; a timeout raises a
+// status word and lets the CTA drain (TMEM is freed, the kernel returns).
+#include <cuda.h>
+
+#include "sat_internal.h"
+
+#define TC_BM 128
+#define TC_BK 16          /* fp32 elements per k-block: 64-byte rows */
+#define TC_THREADS 192
+#define TC_WAIT_LIMIT (1u << 22)
+
+// =====================================================================================
+// PTX wrappers
+// =====================================================================================
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// bounded wait: returns false (and raises *dead) when the limit is hit or another thread already gave up
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status)
+{
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < TC_WAIT_LIMIT; ++it) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t"
+            ".reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t"
+            "}"
+            : "=r"(ok)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (ok) return true;
+        if (*dead) return false;
+    }
+    *dead = 1;
+    atomicOr(status, 1);
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                     smem_u32(smem_dst)),
+                 "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t"
+        "}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t *r)
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, %18, "
+        "%19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), sm_100 version, swizzle mode
+__device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout_type)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)layout_type << 61;
+    return d;
+}
+
+// instruction descriptor for kind::tf32 (TF32 operands in 32-bit containers, fp32 accumulation)
+__host__ __device__ inline uint32_t make_idesc(int n, int a_mn_major, int b_mn_major)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;   // D format: f32
+    d |= 2u << 7;   // A format: tf32
+    d |= 2u << 10;  // B format: tf32
+    d |= (uint32_t)a_mn_major << 15;
+    d |= (uint32_t)b_mn_major << 16;
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(TC_BM >> 4) << 24;
+    return d;
+}
+
+// =====================================================================================
+// TF32 split of a shared-memory tile, element-wise: hi = tf32(x) in place, lo = tf32(x - hi) at the same offset
+// =====================================================================================
+__device__ __forceinline__ float tf32_round(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);  // round half away from zero to 10 mantissa bits
+}
+__device__ __forceinline__ void split_tile(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
+{
+    for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += (uint32_t)nthreads * 16) {
+        float4 x = *reinterpret_cast<float4 *>(hi_tile + off);
+        float4 h, l;
+        h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
+        h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
+        h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
+        h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
+        *reinterpret_cast<float4 *>(hi_tile + off) = h;
+        *reinterpret_cast<float4 *>(lo_tile + off) = l;
+    }
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// make generic-proxy shared-memory writes visible to the tensor-core (async) proxy
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// =====================================================================================
+// K-major kernel
+// =====================================================================================
+struct TcEpilogue {
+    float *C;
+    int64_t ldc;
+    const float *bias;
+    int relu;
+    uint32_t *mask_out;
+    int32_t mask_words;
+    const float *resid;  // C += resid[resid_idx[row]]  (row gather)
+    const int32_t *resid_idx;
+    int64_t ld_resid;
+};
+
+struct TcShared {
+    uint64_t full[4];   // TMA bytes of the stage have landed
+    uint64_t conv[4];   // the converter threads have split the stage
+    uint64_t empty[4];  // the MMAs reading the stage have completed
+    uint64_t accum;     // all MMAs of the tile have completed
+    uint32_t tmem_base;
+    int dead;
+};
+
+#define TC_CONV_THREADS 128
+
+__global__ void __launch_bounds__(TC_THREADS, 2)
+k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB_hi,
+            const __grid_constant__ CUtensorMap mapB_lo, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t stages,
+            int32_t tmem_cols, TcEpilogue ep, int *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t a_bytes = TC_BM * TC_BK * 4;  // one plane of the A tile: 128 rows x 64 B
+    const uint32_t b_bytes = (uint32_t)bn * TC_BK * 4;
+    const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // [A hi | A lo | B hi | B lo]
+    TcShared *sh = (TcShared *)(smem + (size_t)stages * stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.x * TC_BM;
+    const int32_t n0 = blockIdx.y * bn;
+    const int32_t nkb = nkb1 + nkb2;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&sh->full[s], 1);
+            mbar_init(&sh->conv[s], TC_CONV_THREADS);
+            mbar_init(&sh->empty[s], 1);
+        }
+        mbar_init(&sh->accum, 1);
+        sh->dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"((uint32_t)tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+    volatile int *dead = &sh->dead;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int32_t kb = 0; kb < nkb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) break;
+                uint8_t *st = smem + (size_t)s * stage_bytes;
+                mbar_expect_tx(&sh->full[s], a_bytes + 2 * b_bytes);
+                if (kb < nkb1) tma_load_2d(st, &mapA, &sh->full[s], kb * TC_BK, (int32_t)m0);
+                else tma_load_2d(st, &mapA2, &sh->full[s], (kb - nkb1) * TC_BK, (int32_t)m0);
+                tma_load_2d(st + 2 * a_bytes, &mapB_hi, &sh->full[s], kb * TC_BK, n0);
+                tma_load_2d(st + 2 * a_bytes + b_bytes, &mapB_lo, &sh->full[s], kb * TC_BK, n0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(bn, 0, 0);
+            for (int32_t kb = 0; kb < nkb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait(&sh->full[s], ph, dead, status)) break;
+                if (!mbar_wait(&sh->conv[s], ph, dead, status)) break;
+                tc_fence_after();
+                const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+#pragma unroll
+                for (int ks = 0; ks < TC_BK / 8; ++ks) {
+                    // K-major, 64-byte swizzle: rows 64 B apart, 8-row groups 512 B apart; a k-step (8 values) is 32 B inside the row
+                    const uint64_t a_hi = make_desc(st + ks * 32, 16, 512, 4);
+                    const uint64_t a_lo = make_desc(st + a_bytes + ks * 32, 16, 512, 4);
+                    const uint64_t b_hi = make_desc(st + 2 * a_bytes + ks * 32, 16, 512, 4);
+                    const uint64_t b_lo = make_desc(st + 2 * a_bytes + b_bytes + ks * 32, 16, 512, 4);
+                    tc_mma(tmem, a_hi, b_hi, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                    tc_mma(tmem, a_hi, b_lo, idesc, 1u);
+                    tc_mma(tmem, a_lo, b_hi, idesc, 1u);
+                }
+                tc_commit(&sh->empty[s]);  // the stage is free once these MMAs have read it
+            }
+            tc_commit(&sh->accum);
+        }
+    } else {
+        // ---- converters: split every A tile into TF32 hi (in place) and lo ----
+        const int ctid = threadIdx.x - 64;
+        bool alive = true;
+        for (int32_t kb = 0; kb < nkb && alive; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            alive = mbar_wait(&sh->full[s], ph, dead, status);
+            if (!alive) break;
+            uint8_t *st = smem + (size_t)s * stage_bytes;
+            split_tile(st, st + a_bytes, a_bytes, ctid, TC_CONV_THREADS);
+            fence_async_smem();
+            mbar_arrive(&sh->conv[s]);
+        }
+        // ---- epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 = rows of the tile ----
+        const int q = warp & 3;
+        const int64_t row = m0 + q * 32 + lane;
+        const bool ok = alive && mbar_wait(&sh->accum, 0, dead, status);
+        tc_fence_after();
+        if (ok) {
+            const bool row_ok = row < M;
+            const float *rrow = nullptr;
+            if (row_ok && ep.resid_idx) rrow = ep.resid + (int64_t)ep.resid_idx[row] * ep.ld_resid;
+            const bool vec = ((ep.ldc & 3) == 0) && ((((uintptr_t)ep.C) & 15u) == 0);
+            for (int c0 = 0; c0 < bn; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                if (!row_ok) continue;
+                uint32_t bits = 0;
+                float *crow = ep.C + row * ep.ldc;
+#pragma unroll
+                for (int j4 = 0; j4 < 32; j4 += 4) {
+                    float z4[4];
+#pragma unroll
+                    for (int jj = 0; jj < 4; ++jj) {
+                        const int j = j4 + jj;
+                        const int32_t col = n0 + c0 + j;
+                        float z = __uint_as_float(r[j]);
+                        if (col < N) {
+                            if (ep.bias) z += __ldg(ep.bias + col);
+                            if (rrow) z += __ldg(rrow + col);
+                            if (z > 0.f) bits |= 1u << j;
+                            if (ep.relu && !(z > 0.f)) z = 0.f;
+                        }
+                        z4[jj] = z;
+                    }
+                    const int32_t colb = n0 + c0 + j4;
+                    if (vec && colb + 3 < N) {
+                        *reinterpret_cast<float4 *>(crow + colb) = make_float4(z4[0], z4[1], z4[2], z4[3]);
+                    } else {
+#pragma unroll
+                        for (int jj = 0; jj < 4; ++jj)
+                            if (colb + jj < N) crow[colb + jj] = z4[jj];
+                    }
+                }
+                if (ep.mask_out) {
+                    const int32_t word = (n0 + c0) >> 5;
+                    if (word < ep.mask_words) ep.mask_out[row * ep.mask_words + word] = bits;
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
+    }
+}
+
+// =====================================================================================
+// MN-major kernel (weight gradient): block (x, y, z) = tile (x, y) of A^T B over rows [z * rps, (z + 1) * rps)
+// =====================================================================================
+__global__ void __launch_bounds__(TC_THREADS, 2)
+k_gemm_tc_mn(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB, int32_t Mdim, int32_t N, int64_t rps,
+             int32_t bn, int32_t stages, int32_t tmem_cols, float *part_C, int *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t blk_bytes = TC_BK * 128;                // one 32-column block of a k-block: 16 rows x 128 B
+    const int n_blks_b = (bn + 31) / 32;
+    const uint32_t a_bytes = (TC_BM / 32) * blk_bytes;     // one plane of A: 128 columns
+    const uint32_t b_bytes = (uint32_t)n_blks_b * blk_bytes;
+    const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // [A hi | A lo | B hi | B lo]
+    TcShared *sh = (TcShared *)(smem + (size_t)stages * stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int32_t m0 = blockIdx.x * TC_BM;
+    const int32_t n0 = blockIdx.y * bn;
+    const int64_t r0 = (int64_t)blockIdx.z * rps;
+    const int32_t nkb = (int32_t)(rps / TC_BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&sh->full[s], 1);
+            mbar_init(&sh->conv[s], TC_CONV_THREADS);
+            mbar_init(&sh->empty[s], 1);
+        }
+        mbar_init(&sh->accum, 1);
+        sh->dead = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"((uint32_t)tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sh->tmem_base;
+    volatile int *dead = &sh->dead;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int32_t kb = 0; kb < nkb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) break;
+                uint8_t *st = smem + (size_t)s * stage_bytes;
+                const int32_t r = (int32_t)(r0 + (int64_t)kb * TC_BK);
+                mbar_expect_tx(&sh->full[s], a_bytes + b_bytes);
+                for (int bl = 0; bl < TC_BM / 32; ++bl) tma_load_2d(st + bl * blk_bytes, &mapA, &sh->full[s], m0 + bl * 32, r);
+                for (int bl = 0; bl < n_blks_b; ++bl) tma_load_2d(st + 2 * a_bytes + bl * blk_bytes, &mapB, &sh->full[s], n0 + bl * 32, r);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = make_idesc(bn, 1, 1);
+            for (int32_t kb = 0; kb < nkb; ++kb) {
+                const int s = kb % stages;
+                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+                if (!mbar_wait(&sh->full[s], ph, dead, status)) break;
+                if (!mbar_wait(&sh->conv[s], ph, dead, status)) break;
+                tc_fence_after();
+                const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+#pragma unroll
+                for (int ks = 0; ks < TC_BK / 8; ++ks) {
+                    // MN-major 32-bit operands use the 128-byte swizzle with 32-byte atoms (the only layout the tensor core
+                    // accepts for them): 32-column blocks blk_bytes apart (leading offset), groups of 4 k-rows 512 B apart
+                    // (stride offset); a k-step is 8 rows = 1024 B
+                    const uint32_t koff = ks * 1024;
+                    const uint64_t a_hi = make_desc(st + koff, blk_bytes, 512, 1);
+                    const uint64_t a_lo = make_desc(st + a_bytes + koff, blk_bytes, 512, 1);
+                    const uint64_t b_hi = make_desc(st + 2 * a_bytes + koff, blk_bytes, 512, 1);
+                    const uint64_t b_lo = make_desc(st + 2 * a_bytes + b_bytes + koff, blk_bytes, 512, 1);
+                    tc_mma(tmem, a_hi, b_hi, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                    tc_mma(tmem, a_hi, b_lo, idesc, 1u);
+                    tc_mma(tmem, a_lo, b_hi, idesc, 1u);
+                }
+                tc_commit(&sh->empty[s]);
+            }
+            tc_commit(&sh->accum);
+        }
+    } else {
+        const int ctid = threadIdx.x - 64;
+        bool alive = true;
+        for (int32_t kb = 0; kb < nkb && alive; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            alive = mbar_wait(&sh->full[s], ph, dead, status);
+            if (!alive) break;
+            uint8_t *st = smem + (size_t)s * stage_bytes;
+            split_tile(st, st + a_bytes, a_bytes, ctid, TC_CONV_THREADS);
+            split_tile(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TC_CONV_THREADS);
+            fence_async_smem();
+            mbar_arrive(&sh->conv[s]);
+        }
+        const int q = warp & 3;
+        const int32_t row = m0 + q * 32 + lane;
+        const bool ok = alive && mbar_wait(&sh->accum, 0, dead, status);
+        tc_fence_after();
+        if (ok) {
+            float *pc = part_C + (int64_t)blockIdx.z * Mdim * N;
+            for (int c0 = 0; c0 < bn; c0 += 32) {
+                uint32_t r[32];
+                tc_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                if (row >= Mdim) continue;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const int32_t col = n0 + c0 + j;
+                    if (col < N) pc[(int64_t)row * N + col] = __uint_as_float(r[j]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
+    }
+}
+
+// =====================================================================================
+// element-wise helpers
+// =====================================================================================
+// D = src o mask (written only when `dst` is non-null) and per-block column sums of it for the bias gradient
+#define MASK_ROWS_PER_BLOCK 64
+__global__ void k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t rows, int32_t d, const uint32_t *__restrict__ mask,
+                            int32_t mask_words, float *__restrict__ dst, int64_t ld_dst, float *__restrict__ colsum_part)
+{
+    const int64_t r0 = (int64_t)blockIdx.x * MASK_ROWS_PER_BLOCK;
+    const int64_t r1 = (r0 + MASK_ROWS_PER_BLOCK < rows) ? r0 + MASK_ROWS_PER_BLOCK : rows;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+        float s = 0.f;
+        for (int64_t r = r0; r < r1; ++r) {
+            float x = src[r * ld + c];
+            if (mask && !((mask[r * mask_words + (c >> 5)] >> (c & 31)) & 1u)) x = 0.f;
+            if (dst) dst[r * ld_dst + c] = x;
+            s += x;
+        }
+        if (colsum_part) colsum_part[(int64_t)blockIdx.x * d + c] = s;
+    }
+}
+
+// B operand planes [n_pad x k_pad] (K-major, fp32 containers holding TF32 hi / lo) from fp32 weights.
+//   transpose = 1: W is [K x N] row-major (ldw) -> B[n][k] = W[k][n]          (C = A W)
+//   transpose = 0: W is [N x K] row-major (ldw) -> B[n][k] = W[n][k]          (C = A W^T)
+// A second source W2 (same orientation, k2 rows) continues along K at column offset k1_pad.
+__global__ void k_split_weights(const float *__restrict__ W, int64_t ldw, int32_t k1, int32_t k1_pad, const float *__restrict__ W2,
+                                int64_t ldw2, int32_t k2, int32_t n, int32_t n_pad, int32_t k_pad, int transpose,
+                                float *__restrict__ hi, float *__restrict__ lo)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (int64_t)n_pad * k_pad) return;
+    const int32_t nn = (int32_t)(i / k_pad), kk = (int32_t)(i - (int64_t)nn * k_pad);
+    float x = 0.f;
+    if (nn < n) {
+        if (kk < k1) x = transpose ? W[(int64_t)kk * ldw + nn] : W[(int64_t)nn * ldw + kk];
+        else if (kk >= k1_pad && kk - k1_pad < k2) x = transpose ? W2[(int64_t)(kk - k1_pad) * ldw2 + nn] : W2[(int64_t)nn * ldw2 + (kk - k1_pad)];
+    }
+    const float h = tf32_round(x);
+    hi[i] = h;
+    lo[i] = tf32_round(x - h);
+}
+
+// =====================================================================================
+// host side
+// =====================================================================================
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                    const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static PFN_encodeTiled get_encode()
+{
+    static PFN_encodeTiled fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+            fn = (PFN_encodeTiled)p;
+    }
+    return fn;
+}
+
+// 2-D fp32 tensor map: `inner` contiguous elements per row, `outer` rows `ld` elements apart
+static sat_status make_map(sat_ctx *ctx, CUtensorMap *map, const void *base, int64_t inner, int64_t outer, int64_t ld, int box_inner,
+                           int box_outer, CUtensorMapSwizzle swz)
+{
+    PFN_encodeTiled enc = get_encode();
+    if (!enc) return sat_fail(ctx, SAT_ECUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t gdim[2] = {(cuuint64_t)(inner > 0 ? inner : 1), (cuuint64_t)(outer > 0 ? outer : 1)};
+    cuuint64_t gstr[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void *>(base), gdim, gstr, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return sat_fail(ctx, SAT_EINVAL, "cuTensorMapEncodeTiled failed (%d): base %p inner %lld outer %lld ld %lld", (int)r, base,
+                                           (long long)inner, (long long)outer, (long long)ld);
+    return SAT_OK;
+}
+
+static int tmem_cols_for(int bn) { return bn <= 32 ? 32 : bn <= 64 ? 64 : bn <= 128 ? 128 : 256; }
+static int tile_n_for(int n) { return n >= 256 ? 256 : (n + 31) / 32 * 32; }
+
+bool sat_use_tc(int32_t n, int32_t k)
+{
+    static int no_tc = -1;
+    if (no_tc < 0) {
+        const char *e = getenv("SAT_NO_TC");
+        no_tc = (e && e[0] == '1') ? 1 : 0;
+    }
+    return !no_tc && k >= 16 && n >= 16;
+}
+
+sat_status sat_mask_rows(sat_ctx *ctx, const float *src, int32_t ld, int64_t rows, int32_t d, const uint32_t *mask, int32_t mask_words,
+                         float *dst, int32_t ld_dst, float *colsum, int accumulate)
+{
+    if (rows == 0 || d == 0) return SAT_OK;
+    if (!dst && !colsum) return SAT_OK;
+    ProfScope prof(ctx, SATK_SPLIT, (dst ? 8.0 : 4.0) * (double)rows * d, 0.0);
+    const int64_t blocks = cdiv64(rows, MASK_ROWS_PER_BLOCK);
+    float *part = nullptr;
+    if (colsum) {
+        SAT_TRY(sat_ensure(ctx, ctx->buf_colsum, (size_t)blocks * d * sizeof(float)));
+        part = (float *)ctx->buf_colsum.p;
+    }
+    k_mask_rows<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld, rows, d, mask, mask_words, dst, ld_dst, part);
+    SAT_LAUNCHED(ctx);
+    if (colsum) SAT_TRY(sat_splitk_reduce(ctx, part, d, (int32_t)blocks, accumulate, colsum, d, d));
+    return SAT_OK;
+}
+
+sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1, const float *W2, int32_t ldw2, int32_t k2, int32_t n,
+                          int transpose, DevBuf &buf, TcWeights *out)
+{
+    const int32_t k1_pad = W2 ? (k1 + TC_BK - 1) / TC_BK * TC_BK : k1;
+    const int32_t k_tot = k1_pad + (W2 ? k2 : 0);
+    const int32_t k_pad = (k_tot + TC_BK - 1) / TC_BK * TC_BK;
+    const int32_t bn = tile_n_for(n);
+    const int32_t n_pad = (n + bn - 1) / bn * bn;
+    const size_t plane = ((size_t)n_pad * k_pad * sizeof(float) + 255) & ~(size_t)255;
+    SAT_TRY(sat_ensure(ctx, buf, 2 * plane));
+    out->hi = (float *)buf.p;
+    out->lo = (float *)((uint8_t *)buf.p + plane);
+    out->ld = k_pad;
+    out->n_pad = n_pad;
+    k_split_weights<<<(unsigned)cdiv64((int64_t)n_pad * k_pad, 256), 256, 0, ctx->stream>>>(W, ldw, k1, k1_pad, W2, ldw2, k2, n, n_pad, k_pad,
+                                                                                          transpose, out->hi, out->lo);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+static bool g_attr_k = false, g_attr_mn = false;
+#define TC_SMEM_BUDGET (100 * 1024)
+
+// C[m x n] = [A | A2] B^T with B = pre-split weight planes [n_pad x k_pad]
+sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
+                       const TcWeights &Bw, const TcEpilogueHost &eh, int family)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    const int32_t nkb1 = (k1 + TC_BK - 1) / TC_BK, nkb2 = A2 ? (k2 + TC_BK - 1) / TC_BK : 0;
+    const int32_t bn = tile_n_for(n);
+    const uint32_t stage_bytes = 2 * (TC_BM * TC_BK * 4) + 2 * (uint32_t)bn * TC_BK * 4;
+    int stages = (int)(TC_SMEM_BUDGET / stage_bytes);
+    if (stages > 4) stages = 4;
+    if (stages < 2) stages = 2;
+    const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
+    ProfScope prof(ctx, family, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
+    CUtensorMap mA, mA2, mB_hi, mB_lo;
+    SAT_TRY(make_map(ctx, &mA, A, k1, m, lda, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
+    if (A2) SAT_TRY(make_map(ctx, &mA2, A2, k2, m, lda2, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
+    else mA2 = mA;
+    SAT_TRY(make_map(ctx, &mB_hi, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
+    SAT_TRY(make_map(ctx, &mB_lo, Bw.lo, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
+    if (!g_attr_k) {
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        g_attr_k = true;
+    }
+    TcEpilogue ep;
+    ep.C = eh.C;
+    ep.ldc = eh.ldc;
+    ep.bias = eh.bias;
+    ep.relu = eh.relu;
+    ep.mask_out = eh.mask_out;
+    ep.mask_words = eh.mask_words;
+    ep.resid = eh.resid;
+    ep.resid_idx = eh.resid_idx;
+    ep.ld_resid = eh.ld_resid;
+    dim3 grid((unsigned)cdiv64(m, TC_BM), (unsigned)cdiv64(n, bn));
+    k_gemm_tc_k<<<grid, TC_THREADS, smem, ctx->stream>>>(mA, mA2, mB_hi, mB_lo, m, n, nkb1, nkb2, bn, stages, tmem_cols_for(bn), ep,
+                                                          ctx->d_flag + 1);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+// C[m x n] (+)= A^T B over `rows` rows: A fp32 [rows x m] (lda), B fp32 [rows x n] (ldb)
+sat_status sat_gemm_tc_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb, float *C,
+                          int32_t ldc, int accumulate)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_GEMM_TN, 4.0 * ((double)rows * (m + n) + (double)m * n), 2.0 * (double)rows * m * n);
+    const int32_t bn = tile_n_for(n);
+    const int n_blks_b = (bn + 31) / 32;
+    const uint32_t stage_bytes = 2 * ((TC_BM / 32) * TC_BK * 128) + 2 * (uint32_t)n_blks_b * TC_BK * 128;
+    int stages = (int)(TC_SMEM_BUDGET / stage_bytes);
+    if (stages > 4) stages = 4;
+    if (stages < 2) stages = 2;
+    const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
+    const int64_t tiles = cdiv64(m, TC_BM) * cdiv64(n, bn);
+    int64_t splits = (2 * 148 + tiles - 1) / tiles;
+    const int64_t max_splits = cdiv64(rows > 0 ? rows : 1, 8 * TC_BK);
+    if (splits > max_splits) splits = max_splits;
+    if (splits < 1) splits = 1;
+    const int64_t rps = cdiv64(cdiv64(rows > 0 ? rows : 1, splits), TC_BK) * TC_BK;
+    splits = cdiv64(rows > 0 ? rows : 1, rps);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_splitk, (size_t)splits * m * n * sizeof(float)));
+    float *part = (float *)ctx->buf_splitk.p;
+    CUtensorMap mA, mB;
+    SAT_TRY(make_map(ctx, &mA, A, m, rows, lda, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B));
+    SAT_TRY(make_map(ctx, &mB, B, n, rows, ldb, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B));
+    if (!g_attr_mn) {
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_mn, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        g_attr_mn = true;
+    }
+    dim3 grid((unsigned)cdiv64(m, TC_BM), (unsigned)cdiv64(n, bn), (unsigned)splits);
+    k_gemm_tc_mn<<<grid, TC_THREADS, smem, ctx->stream>>>(mA, mB, m, n, rps, bn, stages, tmem_cols_for(bn), part, ctx->d_flag + 1);
+    SAT_LAUNCHED(ctx);
+    return sat_splitk_reduce(ctx, part, (int64_t)m * n, (int32_t)splits, accumulate, C, n, ldc);
+}

@@ -40,7 +40,7 @@ struct CacheLayer {
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
-    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_COUNT
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_COUNT
 };
 
 struct ProfRec {
@@ -107,7 +107,8 @@ struct sat_ctx {
     LayerState layers[SAT_MAX_LAYERS + 1];
 
     // ---- scratch ----
-    DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc;
+    DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
+        buf_wsplit, buf_wsplit2;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
@@ -214,3 +215,38 @@ sat_status sat_gemm_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const floa
 sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B,
                        int32_t ldb, const uint32_t *mask, int32_t mask_words, float *C, int32_t ldc, float *colsum,
                        int accumulate);
+
+// out[r][c] (+)= sum_z part[z][r * ncols + c], z ascending (fixed order: reproducible)
+sat_status sat_splitk_reduce(sat_ctx *ctx, const float *part, int64_t count, int32_t splits, int accumulate, float *out, int32_t ncols,
+                             int32_t ld_out);
+
+// GEMM family on the tensor cores (sat_gemm_tc.cu): TF32 two-term split, fp32 operands in global memory
+struct TcWeights {         // weight operand as two fp32 planes [n_pad x ld] holding the TF32 hi / lo terms, K-major
+    float *hi = nullptr, *lo = nullptr;
+    int32_t ld = 0, n_pad = 0;
+};
+struct TcEpilogueHost {
+    float *C = nullptr;
+    int32_t ldc = 0;
+    const float *bias = nullptr;
+    int relu = 0;
+    uint32_t *mask_out = nullptr;
+    int32_t mask_words = 0;
+    const float *resid = nullptr;      // C += resid[resid_idx[i]] (row gather)
+    const int32_t *resid_idx = nullptr;
+    int32_t ld_resid = 0;
+};
+// tensor-core path on / off for a contraction with n outputs and k terms (SAT_NO_TC=1 in the environment forces the CUDA cores)
+bool sat_use_tc(int32_t n, int32_t k);
+// dst = src o mask (skipped when dst is null) and colsum (+)= 1^T (src o mask) (skipped when colsum is null)
+sat_status sat_mask_rows(sat_ctx *ctx, const float *src, int32_t ld, int64_t rows, int32_t d, const uint32_t *mask, int32_t mask_words,
+                         float *dst, int32_t ld_dst, float *colsum, int accumulate);
+// weight planes in `buf`; transpose = 1 for W given as [K x N], 0 for [N x K]; optional second source continuing along K
+sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1, const float *W2, int32_t ldw2, int32_t k2, int32_t n,
+                          int transpose, DevBuf &buf, TcWeights *out);
+// C[m x n] = [A | A2] B^T (+ epilogue)
+sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
+                       const TcWeights &Bw, const TcEpilogueHost &eh, int family);
+// C[m x n] (+)= A^T B over `rows` rows
+sat_status sat_gemm_tc_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb, float *C,
+                          int32_t ldc, int accumulate);

@@ -1,5 +1,7 @@
 // Entry points of the per-epoch steps: halo pull, predictor, layer forward / backward,
 // cache push / commit, loss seed and parameter step.
+#include <cstdlib>
+
 #include "sat_internal.h"
 
 #define CHECK_CTX(ctx)                                                                             \
@@ -225,9 +227,24 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
     SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_c, (size_t)rows * h * sizeof(float)));
     float *gates = (float *)ctx->buf_lstm_w.p;
     float *cell = (float *)ctx->buf_lstm_c.p;
+    const bool tc = sat_use_tc(4 * h, d);
+    TcWeights W1, W2;   // weight planes for the first step (x only) and the later steps ([x | s])
+    if (tc) {
+        SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &W1));
+        if (k > 1) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit2, &W2));
+    }
     for (int32_t t = 0; t < k; ++t) {
         const float *x = ring_buf(ctx, c, ring_index(ctx, k - 1 - t));  // oldest first
-        SAT_TRY(sat_gemm_nn_dual(ctx, rows, 4 * h, d, x, c->ld, p->Wx, 4 * h, t == 0 ? 0 : h, c->S, h, p->Uh, 4 * h, p->b, gates, 4 * h));
+        if (tc) {
+            TcEpilogueHost eh;
+            eh.C = gates;
+            eh.ldc = 4 * h;
+            eh.bias = p->b;
+            if (t == 0) SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, x, c->ld, d, nullptr, 0, 0, W1, eh, SATK_GEMM_NN));
+            else SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, x, c->ld, d, c->S, h, h, W2, eh, SATK_GEMM_NN));
+        } else {
+            SAT_TRY(sat_gemm_nn_dual(ctx, rows, 4 * h, d, x, c->ld, p->Wx, 4 * h, t == 0 ? 0 : h, c->S, h, p->Uh, 4 * h, p->b, gates, 4 * h));
+        }
         {
             ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 7.0, 0.0);
             k_lstm_cell<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(gates, rows, h, t == 0, cell, c->S);
@@ -274,6 +291,20 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
     // (h is a multiple of 4 or the S rows are not 16-byte aligned: the S table uses ld = h, so require h % 4 == 0)
     if (h & 3) return sat_fail(ctx, SAT_EINVAL, "sat_predict: predictor width h must be a multiple of 4");
     SAT_TRY(sat_spmm_hrow(ctx, v, h, c->S, h, 1, c->S, a - v.halo0 * ld_a, ld_a));
+    if (sat_use_tc(d, h)) {
+        TcWeights Wg;
+        SAT_TRY(sat_tc_weights(ctx, params->Wg, d, h, nullptr, 0, 0, d, 1, ctx->buf_wsplit, &Wg));
+        TcEpilogueHost eh;
+        eh.C = halo_out;
+        eh.ldc = ld_out;
+        eh.bias = params->bg;
+        if (newest) {
+            eh.resid = newest;
+            eh.resid_idx = ctx->halo_slot + v.halo0;
+            eh.ld_resid = c->ld;
+        }
+        return sat_gemm_tc(ctx, v.n_halo, d, a, ld_a, h, nullptr, 0, 0, Wg, eh, SATK_GEMM_NN);
+    }
     GemmEpilogue ep;
     ep.bias = params->bg;
     if (newest) {
@@ -328,14 +359,27 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     const float *in_base = h_in - (int64_t)v.row0 * ld_in;
     const float *halo_base = h_halo ? h_halo - v.halo0 * (int64_t)ld_halo : nullptr;
     SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg));
-    GemmEpilogue ep;
-    ep.bias = bias;
-    ep.relu = act == SAT_ACT_RELU;
-    if (act == SAT_ACT_RELU) {
-        ep.mask_out = L.mask + (int64_t)v.row0 * words;
+    uint32_t *mask_out = act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * words : nullptr;
+    const float *agg = L.agg + (int64_t)v.row0 * ld_agg;
+    if (sat_use_tc(d_out, d_in)) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, d_out, d_in, nullptr, 0, 0, d_out, 1, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = h_out;
+        eh.ldc = ld_out;
+        eh.bias = bias;
+        eh.relu = act == SAT_ACT_RELU;
+        eh.mask_out = mask_out;
+        eh.mask_words = words;
+        SAT_TRY(sat_gemm_tc(ctx, v.n_rows, d_out, agg, ld_agg, d_in, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+    } else {
+        GemmEpilogue ep;
+        ep.bias = bias;
+        ep.relu = act == SAT_ACT_RELU;
+        ep.mask_out = mask_out;
         ep.mask_words = words;
+        SAT_TRY(sat_gemm_nn(ctx, v.n_rows, d_out, d_in, agg, ld_agg, W, d_out, h_out, ld_out, ep));
     }
-    SAT_TRY(sat_gemm_nn(ctx, v.n_rows, d_out, d_in, L.agg + (int64_t)v.row0 * ld_agg, ld_agg, W, d_out, h_out, ld_out, ep));
     if (part == SAT_ALL_PARTS) L.valid.assign(ctx->M, 1);
     else L.valid[part] = 1;
     return SAT_OK;
@@ -358,21 +402,98 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     if (g_in && v.n_rows > 0 && (!ok_ld(ld_gin, d_in) || !aligned16(g_in))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_in or bad ld_gin");
     if (g_halo && v.n_halo > 0 && (!ok_ld(ld_gh, d_in) || !aligned16(g_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_halo or bad ld_gh");
     const uint32_t *mask = L.act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * L.mask_words : nullptr;
-    // G_W (+)= AGG^T D, G_b (+)= 1^T D   with D = g_out o [Z > 0]
-    SAT_TRY(sat_gemm_tn(ctx, v.n_rows, d_in, d_out, L.agg + (int64_t)v.row0 * L.ld_in, L.ld_in, g_out, ld_g, mask, L.mask_words, g_W, d_out,
-                        g_b, accumulate));
-    if ((!g_in && !g_halo) || v.n_rows == 0) return SAT_OK;
+    const float *agg = L.agg + (int64_t)v.row0 * L.ld_in;
+    const bool want_dx = (g_in || g_halo) && v.n_rows > 0;
+    const bool tc_w = sat_use_tc(d_out, d_in) && v.n_rows >= 256;   // weight gradient on the tensor cores
+    // input gradient on the tensor cores, except when the halo gradient is wanted: that output sums thousands of signed
+    // cut-edge terms, and the truncating fp32 accumulation of the tensor cores would be amplified by the cancellation
+    const bool tc_x = want_dx && !g_halo && sat_use_tc(d_in, d_out);
+    const float *D = g_out;  // D = g_out o [Z > 0]: materialised once for the tensor-core contractions
+    int32_t ld_d = ld_g;
+    if (tc_w || tc_x) {
+        float *dm = nullptr;
+        if (mask) {
+            ld_d = round_up4(d_out);
+            SAT_TRY(sat_ensure(ctx, ctx->buf_dmask, (size_t)v.n_rows * ld_d * sizeof(float)));
+            dm = (float *)ctx->buf_dmask.p;
+            D = dm;
+        }
+        SAT_TRY(sat_mask_rows(ctx, g_out, ld_g, v.n_rows, d_out, mask, L.mask_words, dm, ld_d, tc_w ? g_b : nullptr, accumulate));
+    }
+    // G_W (+)= AGG^T D, G_b (+)= 1^T D
+    if (tc_w) SAT_TRY(sat_gemm_tc_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
+    else SAT_TRY(sat_gemm_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, g_out, ld_g, mask, L.mask_words, g_W, d_out, g_b, accumulate));
+    if (!want_dx) return SAT_OK;
     // G_AGG = D W^T
     const int32_t ld_ga = round_up4(d_in);
     SAT_TRY(sat_ensure(ctx, ctx->buf_gagg, (size_t)v.n_rows * ld_ga * sizeof(float)));
     float *gagg = (float *)ctx->buf_gagg.p;
-    SAT_TRY(sat_gemm_nt(ctx, v.n_rows, d_in, d_out, g_out, ld_g, mask, L.mask_words, W, d_out, gagg, ld_ga));
+    if (tc_x) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, d_out, d_out, nullptr, 0, 0, d_in, 0, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = gagg;
+        eh.ldc = ld_ga;
+        SAT_TRY(sat_gemm_tc(ctx, v.n_rows, d_in, D, ld_d, d_out, nullptr, 0, 0, Wp, eh, SATK_GEMM_NT));
+    } else {
+        SAT_TRY(sat_gemm_nt(ctx, v.n_rows, d_in, d_out, g_out, ld_g, mask, L.mask_words, W, d_out, gagg, ld_ga));
+    }
     const float *ga_base = gagg - (int64_t)v.row0 * ld_ga;
     // G_in = P_in^T G_AGG: the inner block of P is symmetric, so P_in^T = P_in (inner prefix of every local row)
     if (g_in) SAT_TRY(sat_spmm(ctx, v, 1, d_in, ga_base, ld_ga, nullptr, 0, g_in - (int64_t)v.row0 * ld_gin, ld_gin));
     // G_halo = P_out^T G_AGG over the halo-row CSR
     if (g_halo) SAT_TRY(sat_spmm_hrow(ctx, v, d_in, ga_base, ld_ga, 0, nullptr, g_halo - v.halo0 * (int64_t)ld_gh, ld_gh));
     return SAT_OK;
+}
+
+// =====================================================================================
+// dense contractions on caller tensors
+// =====================================================================================
+extern "C" sat_status sat_dense_nn(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W,
+                                   const float *bias, float *C, int32_t ldc)
+{
+    CHECK_CTX(ctx);
+    if (m < 0 || n <= 0 || k <= 0 || !A || !W || !C || !ok_ld(lda, k) || !ok_ld(ldc, n) || !aligned16(A) || !aligned16(C))
+        return sat_fail(ctx, SAT_EINVAL, "sat_dense_nn: null / misaligned tensor or bad shape");
+    if (sat_use_tc(n, k)) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, n, k, nullptr, 0, 0, n, 1, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = C;
+        eh.ldc = ldc;
+        eh.bias = bias;
+        return sat_gemm_tc(ctx, m, n, A, lda, k, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN);
+    }
+    GemmEpilogue ep;
+    ep.bias = bias;
+    return sat_gemm_nn(ctx, m, n, k, A, lda, W, n, C, ldc, ep);
+}
+
+extern "C" sat_status sat_dense_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W, float *C,
+                                   int32_t ldc)
+{
+    CHECK_CTX(ctx);
+    if (m < 0 || n <= 0 || k <= 0 || !A || !W || !C || !ok_ld(lda, k) || !ok_ld(ldc, n) || !aligned16(A) || !aligned16(C))
+        return sat_fail(ctx, SAT_EINVAL, "sat_dense_nt: null / misaligned tensor or bad shape");
+    if (sat_use_tc(n, k)) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, k, k, nullptr, 0, 0, n, 0, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = C;
+        eh.ldc = ldc;
+        return sat_gemm_tc(ctx, m, n, A, lda, k, nullptr, 0, 0, Wp, eh, SATK_GEMM_NT);
+    }
+    return sat_gemm_nt(ctx, m, n, k, A, lda, nullptr, 0, W, k, C, ldc);
+}
+
+extern "C" sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B,
+                                   int32_t ldb, float *C)
+{
+    CHECK_CTX(ctx);
+    if (rows < 0 || n <= 0 || m <= 0 || !A || !B || !C || !ok_ld(lda, m) || !ok_ld(ldb, n) || !aligned16(A) || !aligned16(B))
+        return sat_fail(ctx, SAT_EINVAL, "sat_dense_tn: null / misaligned tensor or bad shape");
+    if (sat_use_tc(n, m) && rows >= 256) return sat_gemm_tc_tn(ctx, rows, m, n, A, lda, B, ldb, C, n, 0);
+    return sat_gemm_tn(ctx, rows, m, n, A, lda, B, ldb, nullptr, 0, C, n, nullptr, 0);
 }
 
 // =====================================================================================
