@@ -171,6 +171,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_dmask);
     sat_free_buf(ctx->buf_wsplit);
     sat_free_buf(ctx->buf_wsplit2);
+    sat_free_buf(ctx->buf_bias);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;

@@ -64,6 +64,20 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
                  "l"((uint64_t)map), "r"(smem_u32(bar)), "r"(x), "r"(y)
                  : "memory");
 }
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap *map, const void *smem_src, int32_t x, int32_t y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"((uint64_t)map), "r"(smem_u32(smem_src)),
+                 "r"(x), "r"(y)
+                 : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// waits until at most `N` of this thread's bulk stores still read their shared-memory source
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t *bar)
@@ -128,17 +142,32 @@ __device__ __forceinline__ float tf32_round(float x)
 {
     return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);  // round half away from zero to 10 mantissa bits
 }
+__device__ __forceinline__ void split4(const float4 &x, float4 &h, float4 &l)
+{
+    h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
+    h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
+    h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
+    h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
+}
+// two 16-byte chunks per thread and iteration, loads first (the loop is latency-bound otherwise)
 __device__ __forceinline__ void split_tile(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
 {
-    for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += (uint32_t)nthreads * 16) {
-        float4 x = *reinterpret_cast<float4 *>(hi_tile + off);
-        float4 h, l;
-        h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
-        h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
-        h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
-        h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
-        *reinterpret_cast<float4 *>(hi_tile + off) = h;
-        *reinterpret_cast<float4 *>(lo_tile + off) = l;
+    const uint32_t step = (uint32_t)nthreads * 16;
+    for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += 2 * step) {
+        const uint32_t off2 = off + step;
+        const bool two = off2 < bytes;
+        const float4 x1 = *reinterpret_cast<float4 *>(hi_tile + off);
+        float4 x2 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (two) x2 = *reinterpret_cast<float4 *>(hi_tile + off2);
+        float4 h1, l1, h2, l2;
+        split4(x1, h1, l1);
+        split4(x2, h2, l2);
+        *reinterpret_cast<float4 *>(hi_tile + off) = h1;
+        *reinterpret_cast<float4 *>(lo_tile + off) = l1;
+        if (two) {
+            *reinterpret_cast<float4 *>(hi_tile + off2) = h2;
+            *reinterpret_cast<float4 *>(lo_tile + off2) = l2;
+        }
     }
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
@@ -164,45 +193,56 @@ struct TcEpilogue {
 };
 
 struct TcShared {
-    uint64_t full[4];   // TMA bytes of the stage have landed
-    uint64_t conv[4];   // the converter threads have split the stage
-    uint64_t empty[4];  // the MMAs reading the stage have completed
-    uint64_t accum;     // all MMAs of the tile have completed
+    uint64_t full[4];       // TMA bytes of the stage have landed
+    uint64_t conv[4];       // the converter threads have split the stage
+    uint64_t empty[4];      // the MMAs reading the stage have completed
+    uint64_t accum;         // (MN-major kernel) all MMAs of the tile have completed
+    uint64_t acc_full[2];   // (K-major kernel) accumulator buffer holds a finished tile
+    uint64_t acc_empty[2];  // (K-major kernel) accumulator buffer has been drained by the epilogue
     uint32_t tmem_base;
     int dead;
 };
 
 #define TC_CONV_THREADS 128
+#define TC_EPI_THREADS 128
+#define TCK_CONV_THREADS 256
+#define TCK_THREADS 448   /* warp 0 TMA, warp 1 MMA, warps 2-9 converters, warps 10-13 epilogue */
+#define TCK_STAGES 4
+#define TCK_OUT_BYTES (4 * 2 * 4096)  /* per epilogue warp two 32 x 32 fp32 staging tiles for the TMA stores */
 
-__global__ void __launch_bounds__(TC_THREADS, 2)
-k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB_hi,
-            const __grid_constant__ CUtensorMap mapB_lo, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t stages,
-            int32_t tmem_cols, TcEpilogue ep, int *status)
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of TCK_STAGES k-blocks
+// and the two TMEM accumulator buffers let the TMA loads, the TF32 split, the MMAs and the epilogue of consecutive tiles
+// overlap.  A and B arrive as raw fp32 tiles; the converters round them to TF32 in place and write the residual tiles.
+__global__ void __launch_bounds__(TCK_THREADS, 1)
+k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB,
+            const __grid_constant__ CUtensorMap mapC, int use_tma_store, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t n_tiles_n, int64_t n_tiles, TcEpilogue ep, int *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t a_bytes = TC_BM * TC_BK * 4;  // one plane of the A tile: 128 rows x 64 B
     const uint32_t b_bytes = (uint32_t)bn * TC_BK * 4;
     const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // [A hi | A lo | B hi | B lo]
-    TcShared *sh = (TcShared *)(smem + (size_t)stages * stage_bytes);
+    uint8_t *out_stage = smem + (size_t)TCK_STAGES * stage_bytes;
+    TcShared *sh = (TcShared *)(out_stage + TCK_OUT_BYTES);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * TC_BM;
-    const int32_t n0 = blockIdx.y * bn;
     const int32_t nkb = nkb1 + nkb2;
+    const uint32_t acc_cols = 256;  // column stride between the two accumulator buffers
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
+        for (int s = 0; s < TCK_STAGES; ++s) {
             mbar_init(&sh->full[s], 1);
-            mbar_init(&sh->conv[s], TC_CONV_THREADS);
+            mbar_init(&sh->conv[s], TCK_CONV_THREADS);
             mbar_init(&sh->empty[s], 1);
         }
-        mbar_init(&sh->accum, 1);
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sh->acc_full[i], 1);
+            mbar_init(&sh->acc_empty[i], TC_EPI_THREADS);
+        }
         sh->dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"((uint32_t)tmem_cols)
-                     : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -212,111 +252,160 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     volatile int *dead = &sh->dead;
 
     if (warp == 0) {
+        // ---------------- TMA producer ----------------
         if (lane == 0) {
-            for (int32_t kb = 0; kb < nkb; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-                if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) break;
-                uint8_t *st = smem + (size_t)s * stage_bytes;
-                mbar_expect_tx(&sh->full[s], a_bytes + 2 * b_bytes);
-                if (kb < nkb1) tma_load_2d(st, &mapA, &sh->full[s], kb * TC_BK, (int32_t)m0);
-                else tma_load_2d(st, &mapA2, &sh->full[s], (kb - nkb1) * TC_BK, (int32_t)m0);
-                tma_load_2d(st + 2 * a_bytes, &mapB_hi, &sh->full[s], kb * TC_BK, n0);
-                tma_load_2d(st + 2 * a_bytes + b_bytes, &mapB_lo, &sh->full[s], kb * TC_BK, n0);
+            uint32_t it = 0;
+            for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+                const int32_t m0 = (int32_t)(t / n_tiles_n) * TC_BM;
+                const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
+                for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % TCK_STAGES;
+                    const uint32_t ph = (it / TCK_STAGES) & 1u;
+                    if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) goto done;
+                    uint8_t *st = smem + (size_t)s * stage_bytes;
+                    mbar_expect_tx(&sh->full[s], a_bytes + b_bytes);
+                    if (kb < nkb1) tma_load_2d(st, &mapA, &sh->full[s], kb * TC_BK, m0);
+                    else tma_load_2d(st, &mapA2, &sh->full[s], (kb - nkb1) * TC_BK, m0);
+                    tma_load_2d(st + 2 * a_bytes, &mapB, &sh->full[s], kb * TC_BK, n0);
+                }
             }
         }
     } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = make_idesc(bn, 0, 0);
-            for (int32_t kb = 0; kb < nkb; ++kb) {
-                const int s = kb % stages;
-                const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-                if (!mbar_wait(&sh->full[s], ph, dead, status)) break;
-                if (!mbar_wait(&sh->conv[s], ph, dead, status)) break;
+            uint32_t it = 0, lt = 0;
+            for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1u;
+                if (!mbar_wait(&sh->acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, dead, status)) goto done;
                 tc_fence_after();
-                const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                const uint32_t acc = tmem + buf * acc_cols;
+                for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
+                    const int s = it % TCK_STAGES;
+                    const uint32_t ph = (it / TCK_STAGES) & 1u;
+                    if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
+                    if (!mbar_wait(&sh->conv[s], ph, dead, status)) goto done;
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
 #pragma unroll
-                for (int ks = 0; ks < TC_BK / 8; ++ks) {
-                    // K-major, 64-byte swizzle: rows 64 B apart, 8-row groups 512 B apart; a k-step (8 values) is 32 B inside the row
-                    const uint64_t a_hi = make_desc(st + ks * 32, 16, 512, 4);
-                    const uint64_t a_lo = make_desc(st + a_bytes + ks * 32, 16, 512, 4);
-                    const uint64_t b_hi = make_desc(st + 2 * a_bytes + ks * 32, 16, 512, 4);
-                    const uint64_t b_lo = make_desc(st + 2 * a_bytes + b_bytes + ks * 32, 16, 512, 4);
-                    tc_mma(tmem, a_hi, b_hi, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
-                    tc_mma(tmem, a_hi, b_lo, idesc, 1u);
-                    tc_mma(tmem, a_lo, b_hi, idesc, 1u);
+                    for (int ks = 0; ks < TC_BK / 8; ++ks) {
+                        // K-major, 64-byte swizzle: rows 64 B apart, 8-row groups 512 B apart; a k-step (8 values) is 32 B inside the row
+                        const uint64_t a_hi = make_desc(st + ks * 32, 16, 512, 4);
+                        const uint64_t a_lo = make_desc(st + a_bytes + ks * 32, 16, 512, 4);
+                        const uint64_t b_hi = make_desc(st + 2 * a_bytes + ks * 32, 16, 512, 4);
+                        const uint64_t b_lo = make_desc(st + 2 * a_bytes + b_bytes + ks * 32, 16, 512, 4);
+                        tc_mma(acc, a_hi, b_hi, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
+                        tc_mma(acc, a_hi, b_lo, idesc, 1u);
+                        tc_mma(acc, a_lo, b_hi, idesc, 1u);
+                    }
+                    tc_commit(&sh->empty[s]);  // the stage is free once these MMAs have read it
                 }
-                tc_commit(&sh->empty[s]);  // the stage is free once these MMAs have read it
+                tc_commit(&sh->acc_full[buf]);
             }
-            tc_commit(&sh->accum);
+        }
+    } else if (warp < 10) {
+        // ---------------- converters: TF32 split of the A and B tiles of every k-block ----------------
+        const int ctid = threadIdx.x - 64;
+        uint32_t it = 0;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+            for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
+                const int s = it % TCK_STAGES;
+                const uint32_t ph = (it / TCK_STAGES) & 1u;
+                if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
+                uint8_t *st = smem + (size_t)s * stage_bytes;
+                split_tile(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
+                split_tile(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_THREADS);
+                fence_async_smem();
+                mbar_arrive(&sh->conv[s]);
+            }
         }
     } else {
-        // ---- converters: split every A tile into TF32 hi (in place) and lo ----
-        const int ctid = threadIdx.x - 64;
-        bool alive = true;
-        for (int32_t kb = 0; kb < nkb && alive; ++kb) {
-            const int s = kb % stages;
-            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-            alive = mbar_wait(&sh->full[s], ph, dead, status);
-            if (!alive) break;
-            uint8_t *st = smem + (size_t)s * stage_bytes;
-            split_tile(st, st + a_bytes, a_bytes, ctid, TC_CONV_THREADS);
-            fence_async_smem();
-            mbar_arrive(&sh->conv[s]);
-        }
-        // ---- epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 = rows of the tile ----
+        // ---------------- epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 = rows of the tile ----------------
         const int q = warp & 3;
-        const int64_t row = m0 + q * 32 + lane;
-        const bool ok = alive && mbar_wait(&sh->accum, 0, dead, status);
-        tc_fence_after();
-        if (ok) {
+        uint8_t *obuf = out_stage + (warp - 10) * 8192;
+        uint32_t ob = 0;
+        const bool vec = ((ep.ldc & 3) == 0) && ((((uintptr_t)ep.C) & 15u) == 0);
+        uint32_t lt = 0;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
+            const int64_t m0 = (t / n_tiles_n) * TC_BM;
+            const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
+            const uint32_t buf = lt & 1u;
+            if (!mbar_wait(&sh->acc_full[buf], (lt >> 1) & 1u, dead, status)) goto done;
+            tc_fence_after();
+            const int64_t row = m0 + q * 32 + lane;
             const bool row_ok = row < M;
             const float *rrow = nullptr;
             if (row_ok && ep.resid_idx) rrow = ep.resid + (int64_t)ep.resid_idx[row] * ep.ld_resid;
-            const bool vec = ((ep.ldc & 3) == 0) && ((((uintptr_t)ep.C) & 15u) == 0);
+            float *crow = ep.C + row * ep.ldc;
             for (int c0 = 0; c0 < bn; c0 += 32) {
                 uint32_t r[32];
-                tc_ld32(tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                if (!row_ok) continue;
+                tc_ld32(tmem + buf * acc_cols + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                 uint32_t bits = 0;
-                float *crow = ep.C + row * ep.ldc;
+                if (row_ok) {
+                    // bias is padded with zeros to the tile width and the accumulators of padded columns are exactly zero,
+                    // so no column predicate is needed (the stores clip)
+                    float bq[32];
+                    if (ep.bias) {
 #pragma unroll
-                for (int j4 = 0; j4 < 32; j4 += 4) {
-                    float z4[4];
-#pragma unroll
-                    for (int jj = 0; jj < 4; ++jj) {
-                        const int j = j4 + jj;
-                        const int32_t col = n0 + c0 + j;
-                        float z = __uint_as_float(r[j]);
-                        if (col < N) {
-                            if (ep.bias) z += __ldg(ep.bias + col);
-                            if (rrow) z += __ldg(rrow + col);
-                            if (z > 0.f) bits |= 1u << j;
-                            if (ep.relu && !(z > 0.f)) z = 0.f;
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 bv = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + j);
+                            bq[4 * j] = bv.x; bq[4 * j + 1] = bv.y; bq[4 * j + 2] = bv.z; bq[4 * j + 3] = bv.w;
                         }
-                        z4[jj] = z;
-                    }
-                    const int32_t colb = n0 + c0 + j4;
-                    if (vec && colb + 3 < N) {
-                        *reinterpret_cast<float4 *>(crow + colb) = make_float4(z4[0], z4[1], z4[2], z4[3]);
                     } else {
 #pragma unroll
-                        for (int jj = 0; jj < 4; ++jj)
-                            if (colb + jj < N) crow[colb + jj] = z4[jj];
+                        for (int j = 0; j < 32; ++j) bq[j] = 0.f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float z = __uint_as_float(r[j]) + bq[j];
+                        if (rrow && n0 + c0 + j < N) z += __ldg(rrow + n0 + c0 + j);
+                        bits |= (z > 0.f ? 1u : 0u) << j;
+                        if (ep.relu) z = fmaxf(z, 0.f);
+                        r[j] = __float_as_uint(z);
                     }
                 }
-                if (ep.mask_out) {
+                if (use_tma_store) {
+                    // stage the 32 x 32 block (128-byte swizzle: 16-byte chunk j of row r sits at chunk j ^ (r & 7)) and
+                    // let the TMA write it as whole 128-byte row segments; rows / columns past the matrix are clipped
+                    if (lane == 0) tma_store_wait_read<1>();  // the buffer used two blocks ago has been read
+                    __syncwarp();
+                    uint8_t *dst = obuf + ob * 4096 + lane * 128;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4 *>(dst + ((j ^ (lane & 7)) << 4)) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) tma_store_2d(&mapC, obuf + ob * 4096, n0 + c0, (int32_t)(m0 + q * 32));
+                    ob ^= 1u;
+                } else if (row_ok) {
+#pragma unroll
+                    for (int j4 = 0; j4 < 32; j4 += 4) {
+                        const int32_t colb = n0 + c0 + j4;
+                        if (vec && colb + 3 < N) {
+                            *reinterpret_cast<uint4 *>(crow + colb) = make_uint4(r[j4], r[j4 + 1], r[j4 + 2], r[j4 + 3]);
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+                                if (colb + jj < N) crow[colb + jj] = __uint_as_float(r[j4 + jj]);
+                        }
+                    }
+                }
+                if (ep.mask_out && row_ok) {
                     const int32_t word = (n0 + c0) >> 5;
                     if (word < ep.mask_words) ep.mask_out[row * ep.mask_words + word] = bits;
                 }
             }
+            tc_fence_before();
+            mbar_arrive(&sh->acc_empty[buf]);  // the accumulator buffer may be overwritten by the tile after next
         }
+        if (use_tma_store && lane == 0) tma_store_wait_all();
     }
+done:
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)tmem_cols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
 }
 
@@ -465,7 +554,7 @@ __global__ void k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t r
     }
 }
 
-// B operand planes [n_pad x k_pad] (K-major, fp32 containers holding TF32 hi / lo) from fp32 weights.
+// B operand [n_pad x k_pad] (K-major fp32, zero padded) from fp32 weights; the TF32 split happens in the GEMM kernel.
 //   transpose = 1: W is [K x N] row-major (ldw) -> B[n][k] = W[k][n]          (C = A W)
 //   transpose = 0: W is [N x K] row-major (ldw) -> B[n][k] = W[n][k]          (C = A W^T)
 // A second source W2 (same orientation, k2 rows) continues along K at column offset k1_pad.
@@ -481,9 +570,8 @@ __global__ void k_split_weights(const float *__restrict__ W, int64_t ldw, int32_
         if (kk < k1) x = transpose ? W[(int64_t)kk * ldw + nn] : W[(int64_t)nn * ldw + kk];
         else if (kk >= k1_pad && kk - k1_pad < k2) x = transpose ? W2[(int64_t)(kk - k1_pad) * ldw2 + nn] : W2[(int64_t)nn * ldw2 + (kk - k1_pad)];
     }
-    const float h = tf32_round(x);
-    hi[i] = h;
-    lo[i] = tf32_round(x - h);
+    hi[i] = x;
+    (void)lo;
 }
 
 // =====================================================================================
@@ -562,9 +650,9 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
     const int32_t bn = tile_n_for(n);
     const int32_t n_pad = (n + bn - 1) / bn * bn;
     const size_t plane = ((size_t)n_pad * k_pad * sizeof(float) + 255) & ~(size_t)255;
-    SAT_TRY(sat_ensure(ctx, buf, 2 * plane));
+    SAT_TRY(sat_ensure(ctx, buf, plane));
     out->hi = (float *)buf.p;
-    out->lo = (float *)((uint8_t *)buf.p + plane);
+    out->lo = nullptr;
     out->ld = k_pad;
     out->n_pad = n_pad;
     k_split_weights<<<(unsigned)cdiv64((int64_t)n_pad * k_pad, 256), 256, 0, ctx->stream>>>(W, ldw, k1, k1_pad, W2, ldw2, k2, n, n_pad, k_pad,
@@ -576,7 +664,7 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
 static bool g_attr_k = false, g_attr_mn = false;
 #define TC_SMEM_BUDGET (100 * 1024)
 
-// C[m x n] = [A | A2] B^T with B = pre-split weight planes [n_pad x k_pad]
+// C[m x n] = [A | A2] B^T with B = packed weights [n_pad x k_pad]
 sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
                        const TcWeights &Bw, const TcEpilogueHost &eh, int family)
 {
@@ -584,34 +672,43 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     const int32_t nkb1 = (k1 + TC_BK - 1) / TC_BK, nkb2 = A2 ? (k2 + TC_BK - 1) / TC_BK : 0;
     const int32_t bn = tile_n_for(n);
     const uint32_t stage_bytes = 2 * (TC_BM * TC_BK * 4) + 2 * (uint32_t)bn * TC_BK * 4;
-    int stages = (int)(TC_SMEM_BUDGET / stage_bytes);
-    if (stages > 4) stages = 4;
-    if (stages < 2) stages = 2;
-    const size_t smem = (size_t)stages * stage_bytes + sizeof(TcShared) + 1024;
+    const size_t smem = (size_t)TCK_STAGES * stage_bytes + TCK_OUT_BYTES + sizeof(TcShared) + 1024;
     ProfScope prof(ctx, family, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
-    CUtensorMap mA, mA2, mB_hi, mB_lo;
+    CUtensorMap mA, mA2, mB, mC;
+    const int use_tma_store = ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
+    if (use_tma_store) SAT_TRY(make_map(ctx, &mC, eh.C, n, m, eh.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B));
+    else memset(&mC, 0, sizeof(mC));
     SAT_TRY(make_map(ctx, &mA, A, k1, m, lda, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
     if (A2) SAT_TRY(make_map(ctx, &mA2, A2, k2, m, lda2, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
     else mA2 = mA;
-    SAT_TRY(make_map(ctx, &mB_hi, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
-    SAT_TRY(make_map(ctx, &mB_lo, Bw.lo, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
+    SAT_TRY(make_map(ctx, &mB, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
     if (!g_attr_k) {
-        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         g_attr_k = true;
     }
     TcEpilogue ep;
     ep.C = eh.C;
     ep.ldc = eh.ldc;
-    ep.bias = eh.bias;
+    ep.bias = nullptr;
+    if (eh.bias) {  // zero-padded copy so that the epilogue can read whole 128-bit vectors
+        const size_t padded = (size_t)cdiv64(n, bn) * bn;
+        SAT_TRY(sat_ensure(ctx, ctx->buf_bias, padded * sizeof(float)));
+        SAT_CUDA(ctx, cudaMemsetAsync(ctx->buf_bias.p, 0, padded * sizeof(float), ctx->stream));
+        SAT_CUDA(ctx, cudaMemcpyAsync(ctx->buf_bias.p, eh.bias, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+        ep.bias = (const float *)ctx->buf_bias.p;
+    }
     ep.relu = eh.relu;
     ep.mask_out = eh.mask_out;
     ep.mask_words = eh.mask_words;
     ep.resid = eh.resid;
     ep.resid_idx = eh.resid_idx;
     ep.ld_resid = eh.ld_resid;
-    dim3 grid((unsigned)cdiv64(m, TC_BM), (unsigned)cdiv64(n, bn));
-    k_gemm_tc_k<<<grid, TC_THREADS, smem, ctx->stream>>>(mA, mA2, mB_hi, mB_lo, m, n, nkb1, nkb2, bn, stages, tmem_cols_for(bn), ep,
-                                                          ctx->d_flag + 1);
+    const int32_t n_tiles_n = (int32_t)cdiv64(n, bn);
+    const int64_t n_tiles = cdiv64(m, TC_BM) * n_tiles_n;
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+    const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
+    k_gemm_tc_k<<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }

@@ -108,7 +108,7 @@ struct sat_ctx {
 
     // ---- scratch ----
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2;
+        buf_wsplit, buf_wsplit2, buf_bias;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
