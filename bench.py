@@ -35,7 +35,10 @@ if ROOT not in sys.path:
 # workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
 NCU_TRAFFIC_BYTES = {}
 
-FP32_ALU_PEAK_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12   # 148 SMs x 128 FMA lanes x 2 flop x max SM clock
+# The contractions run on the tensor cores in TF32 (two-term split: three TF32 MMAs per product term).  The box's
+# measured tensor peak is a bf16 figure; TF32 is taken as measured bf16 x the nominal ratio 1.1 / 2.25 PFLOP/s.
+TF32_OVER_BF16 = 1.1 / 2.25
+TF32_MMAS_PER_TERM = 3
 
 
 def measured_peaks():
@@ -281,10 +284,12 @@ def run_ours(args, wl):
         rec = prof[fam]
         per_launch_ms = rec["ms"] / max(rec["calls"], 1)
         if fam.startswith("gemm"):
-            tfl = rec["flops"] / (rec["ms"] * 1e-3) / 1e12
-            roofline = dict(kernel=fam, bound="alu", achieved=tfl, peak=FP32_ALU_PEAK_TFLOPS, unit="TFLOP/s",
-                            frac=tfl / FP32_ALU_PEAK_TFLOPS, traffic=NCU_TRAFFIC_BYTES.get(fam),
-                            peak_source="derived: 148 SMs x 128 fp32 FMA lanes x 2 x 1.965 GHz")
+            tfl = TF32_MMAS_PER_TERM * rec["flops"] / (rec["ms"] * 1e-3) / 1e12
+            peak = peaks["bf16"] * TF32_OVER_BF16
+            roofline = dict(kernel=fam, bound="tensor", achieved=tfl, peak=peak, unit="TFLOP/s", frac=tfl / peak,
+                            traffic=NCU_TRAFFIC_BYTES.get(fam),
+                            achieved_note="TF32 tensor flops issued = 3 x the algorithmic 2mnk (two-term TF32 split)",
+                            peak_source=f"{peaks['source']} sustained bf16 {peaks['bf16']:.0f} TFLOP/s x nominal TF32/bf16 ratio {TF32_OVER_BF16:.3f}")
         else:
             gbs = rec["bytes"] / (rec["ms"] * 1e-3) / 1e9
             roofline = dict(kernel=fam, bound="hbm", achieved=gbs, peak=peaks["hbm"], unit="GB/s", frac=gbs / peaks["hbm"],

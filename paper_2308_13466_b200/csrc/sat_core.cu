@@ -120,6 +120,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->hrow_ptr);
     dev_free(&ctx->hrow_pos);
     dev_free(&ctx->hrow_slot);
+    dev_free(&ctx->hlong);
     dev_free(&ctx->first_item);
     dev_free(&ctx->item_row);
     dev_free(&ctx->item_mslot);
@@ -695,6 +696,18 @@ __global__ void k_hrow(const int64_t *__restrict__ rowptr, const int32_t *__rest
     if (lane == 0 && !hrow_ptr) cnt[j] = run;
 }
 
+__global__ void k_hlong_flag(const int64_t *__restrict__ hrow_ptr, int64_t nb, int32_t *__restrict__ flag)
+{
+    int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < nb) flag[j] = (hrow_ptr[j + 1] - hrow_ptr[j]) > SAT_HROW_LONG ? 1 : 0;
+}
+
+__global__ void k_hlong_fill(const int32_t *__restrict__ flag, const int64_t *__restrict__ off, int64_t nb, int32_t *__restrict__ out)
+{
+    int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j < nb && flag[j]) out[off[j]] = (int32_t)j;
+}
+
 __global__ void k_chunks(const int64_t *__restrict__ lrowptr, int32_t n, int32_t *__restrict__ nch)
 {
     int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -936,6 +949,39 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
         P_TRY(rc);
     }
 
+    // ---- long halo rows (hubs adjacent to many nodes of one partition) get their own list ----
+    {
+        int32_t *t_hf = nullptr;
+        int64_t *t_ho = nullptr;
+        P_TRY(dev_alloc(ctx, &t_hf, ctx->nb + 1));
+        rc = dev_alloc(ctx, &t_ho, ctx->nb + 2);
+        if (rc == SAT_OK) {
+            k_hlong_flag<<<GRID1(ctx->nb)>>>(ctx->hrow_ptr, ctx->nb, t_hf);
+            ctx->launches++;
+            rc = sat_scan_i32(ctx, t_hf, ctx->nb, t_ho);
+        }
+        int64_t n_hl = 0;
+        std::vector<int64_t> off_h((size_t)M + 1, 0);
+        if (rc == SAT_OK) rc = copy_i64(ctx, t_ho + ctx->nb, &n_hl);
+        for (int m = 0; m <= M && rc == SAT_OK; ++m) rc = copy_i64(ctx, t_ho + ctx->h_halo_off[m], &off_h[m]);
+        cudaError_t e = cudaStreamSynchronize(st);
+        if (rc == SAT_OK && e == cudaSuccess) {
+            ctx->n_hlong = (int32_t)n_hl;
+            ctx->h_hlong_off.assign(M + 1, 0);
+            for (int m = 0; m <= M; ++m) ctx->h_hlong_off[m] = (int32_t)off_h[m];
+            rc = dev_alloc(ctx, &ctx->hlong, ctx->n_hlong);
+        }
+        if (rc == SAT_OK && e == cudaSuccess) {
+            k_hlong_fill<<<GRID1(ctx->nb)>>>(t_hf, t_ho, ctx->nb, ctx->hlong);
+            ctx->launches++;
+            e = cudaStreamSynchronize(st);
+        }
+        dev_free(&t_hf);
+        dev_free(&t_ho);
+        if (e != cudaSuccess) P_TRY(sat_check_cuda(ctx, e, "long halo rows"));
+        P_TRY(rc);
+    }
+
     // ---- SpMM work items ----
     P_TRY(dev_alloc(ctx, &t_item_off, (int64_t)n + 2));
     P_TRY(dev_alloc(ctx, &ctx->first_item, (int64_t)n + 1));
@@ -1013,6 +1059,8 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v)
     v->push0 = ctx->h_push_off[a];
     v->n_push = ctx->h_push_off[b] - v->push0;
     v->lnnz = ctx->h_lnnz_off[b] - ctx->h_lnnz_off[a];
+    v->hlong0 = ctx->h_hlong_off[a];
+    v->n_hlong = ctx->h_hlong_off[b] - v->hlong0;
     return SAT_OK;
 }
 

@@ -242,24 +242,43 @@ k_gemm_tn(int64_t rows, int64_t rows_per_split, int32_t m, int32_t n, const floa
     }
 }
 
-// out[i] (+)= sum_z part[z][i], z ascending (fixed order: reproducible)
-__global__ void k_splitk_reduce(const float *__restrict__ part, int64_t count, int32_t splits, int accumulate, float *__restrict__ out,
-                                int32_t ncols, int64_t ld_out)
+// out[i] (+)= sum_z part[z][i]: eight lanes take the splits round-robin (four independent loads in flight each), their sums
+// are added in lane order (fixed order: reproducible)
+__global__ void __launch_bounds__(256)
+k_splitk_reduce(const float *__restrict__ part, int64_t count, int32_t splits, int accumulate, float *__restrict__ out,
+                int32_t ncols, int64_t ld_out)
 {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= count) return;
-    float s = 0.f;
-    for (int z = 0; z < splits; ++z) s += part[(int64_t)z * count + i];
-    const int64_t r = i / ncols, c = i - r * ncols;
-    float *o = out + r * ld_out + c;
-    *o = accumulate ? *o + s : s;
+    __shared__ float red[8][32];
+    const int o = threadIdx.x & 31, zl = threadIdx.x >> 5;
+    const int64_t i = (int64_t)blockIdx.x * 32 + o;
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+    if (i < count) {
+        int z = zl;
+        for (; z + 24 < splits; z += 32) {
+            s0 += part[(int64_t)z * count + i];
+            s1 += part[(int64_t)(z + 8) * count + i];
+            s2 += part[(int64_t)(z + 16) * count + i];
+            s3 += part[(int64_t)(z + 24) * count + i];
+        }
+        for (; z < splits; z += 8) s0 += part[(int64_t)z * count + i];
+    }
+    red[zl][o] = (s0 + s1) + (s2 + s3);
+    __syncthreads();
+    if (zl == 0 && i < count) {
+        float s = red[0][o];
+#pragma unroll
+        for (int g = 1; g < 8; ++g) s += red[g][o];
+        const int64_t r = i / ncols, c = i - r * ncols;
+        float *dst = out + r * ld_out + c;
+        *dst = accumulate ? *dst + s : s;
+    }
 }
 
 sat_status sat_splitk_reduce(sat_ctx *ctx, const float *part, int64_t count, int32_t splits, int accumulate, float *out, int32_t ncols,
                              int32_t ld_out)
 {
     if (count == 0) return SAT_OK;
-    k_splitk_reduce<<<(unsigned)cdiv64(count, 256), 256, 0, ctx->stream>>>(part, count, splits, accumulate, out, ncols, ld_out);
+    k_splitk_reduce<<<(unsigned)cdiv64(count, 32), 256, 0, ctx->stream>>>(part, count, splits, accumulate, out, ncols, ld_out);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
@@ -280,11 +299,7 @@ sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const f
     dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN), (unsigned)splits);
     k_gemm_tn<<<grid, 256, 0, ctx->stream>>>(rows, rows_per_split, m, n, A, lda, B, ldb, mask, mask_words, part_C, part_cs);
     SAT_LAUNCHED(ctx);
-    k_splitk_reduce<<<(unsigned)cdiv64((int64_t)m * n, 256), 256, 0, ctx->stream>>>(part_C, (int64_t)m * n, (int32_t)splits, accumulate, C, n, ldc);
-    SAT_LAUNCHED(ctx);
-    if (colsum) {
-        k_splitk_reduce<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(part_cs, n, (int32_t)splits, accumulate, colsum, n, n);
-        SAT_LAUNCHED(ctx);
-    }
+    SAT_TRY(sat_splitk_reduce(ctx, part_C, (int64_t)m * n, (int32_t)splits, accumulate, C, n, ldc));
+    if (colsum) SAT_TRY(sat_splitk_reduce(ctx, part_cs, n, (int32_t)splits, accumulate, colsum, n, n));
     return SAT_OK;
 }

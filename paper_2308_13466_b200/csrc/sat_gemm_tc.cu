@@ -190,7 +190,20 @@ struct TcEpilogue {
     const float *resid;  // C += resid[resid_idx[row]]  (row gather)
     const int32_t *resid_idx;
     int64_t ld_resid;
+    int32_t lstm_h;      // > 0: fused LSTM cell, C = hidden state [M x lstm_h], lstm_c = cell state
+    int lstm_first;
+    float *lstm_c;
 };
+
+// logistic and tanh from the hardware exponential (ex2.approx) and reciprocal: absolute error of a few 1e-7, which is
+// what matters for gate values in [0, 1] / [-1, 1]; an order of magnitude cheaper than the libm versions, so that the
+// four epilogue warps keep up with the main loop
+__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
+__device__ __forceinline__ float tanh_fast(float x)
+{
+    const float e = __expf(-2.f * fabsf(x));
+    return copysignf(__fdividef(1.f - e, 1.f + e), x);
+}
 
 struct TcShared {
     uint64_t full[4];       // TMA bytes of the stage have landed
@@ -340,6 +353,54 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             for (int c0 = 0; c0 < bn; c0 += 32) {
                 uint32_t r[32];
                 tc_ld32(tmem + buf * acc_cols + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                if (ep.lstm_h > 0) {
+                    // packed columns 4 j .. 4 j + 3 are the (i, f, g, o) pre-activations of hidden unit j
+                    if (row_ok) {
+                        const int32_t j0 = (n0 + c0) >> 2;
+                        float sv[8], cv[8], cprev[8];
+                        const bool full = j0 + 7 < ep.lstm_h && (ep.lstm_h & 3) == 0;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) cprev[u] = 0.f;
+                        if (!ep.lstm_first) {
+                            if (full) {
+                                const float4 c0v = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
+                                const float4 c1v = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0 + 4);
+                                cprev[0] = c0v.x; cprev[1] = c0v.y; cprev[2] = c0v.z; cprev[3] = c0v.w;
+                                cprev[4] = c1v.x; cprev[5] = c1v.y; cprev[6] = c1v.z; cprev[7] = c1v.w;
+                            } else {
+#pragma unroll
+                                for (int u = 0; u < 8; ++u)
+                                    if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[row * ep.lstm_h + j0 + u];
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const float4 bv = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + u);
+                            const float gi = sigmoid_fast(__uint_as_float(r[4 * u]) + bv.x);
+                            const float gf = sigmoid_fast(__uint_as_float(r[4 * u + 1]) + bv.y);
+                            const float gg = tanh_fast(__uint_as_float(r[4 * u + 2]) + bv.z);
+                            const float go = sigmoid_fast(__uint_as_float(r[4 * u + 3]) + bv.w);
+                            cv[u] = gf * cprev[u] + gi * gg;
+                            sv[u] = go * tanh_fast(cv[u]);
+                        }
+                        if (full) {
+                            float4 *cd = reinterpret_cast<float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
+                            float4 *sd = reinterpret_cast<float4 *>(ep.C + row * ep.ldc + j0);
+                            cd[0] = make_float4(cv[0], cv[1], cv[2], cv[3]);
+                            cd[1] = make_float4(cv[4], cv[5], cv[6], cv[7]);
+                            sd[0] = make_float4(sv[0], sv[1], sv[2], sv[3]);
+                            sd[1] = make_float4(sv[4], sv[5], sv[6], sv[7]);
+                        } else {
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if (j0 + u < ep.lstm_h) {
+                                    ep.lstm_c[row * ep.lstm_h + j0 + u] = cv[u];
+                                    ep.C[row * ep.ldc + j0 + u] = sv[u];
+                                }
+                        }
+                    }
+                    continue;
+                }
                 uint32_t bits = 0;
                 if (row_ok) {
                     // bias is padded with zeros to the tile width and the accumulators of padded columns are exactly zero,
@@ -535,23 +596,69 @@ k_gemm_tc_mn(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ C
 // =====================================================================================
 // element-wise helpers
 // =====================================================================================
-// D = src o mask (written only when `dst` is non-null) and per-block column sums of it for the bias gradient
-#define MASK_ROWS_PER_BLOCK 64
-__global__ void k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t rows, int32_t d, const uint32_t *__restrict__ mask,
-                            int32_t mask_words, float *__restrict__ dst, int64_t ld_dst, float *__restrict__ colsum_part)
+// D = src o mask (written only when `dst` is non-null) and per-block column sums of it for the bias gradient.
+// A block covers MASK_ROWS_PER_BLOCK rows; TPR threads (a power of two >= d / 4) walk one row with 128-bit accesses,
+// 256 / TPR rows per pass; each thread keeps the running sum of its four columns, the row groups are added through
+// shared memory in fixed order.
+#define MASK_ROWS_PER_BLOCK 512
+__global__ void __launch_bounds__(256)
+k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t rows, int32_t d, int32_t tpr, const uint32_t *__restrict__ mask,
+            int32_t mask_words, float *__restrict__ dst, int64_t ld_dst, float *__restrict__ colsum_part)
 {
+    __shared__ float4 red[256];
+    const int c4 = threadIdx.x % tpr, rg = threadIdx.x / tpr, n_rg = 256 / tpr;
     const int64_t r0 = (int64_t)blockIdx.x * MASK_ROWS_PER_BLOCK;
     const int64_t r1 = (r0 + MASK_ROWS_PER_BLOCK < rows) ? r0 + MASK_ROWS_PER_BLOCK : rows;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float s = 0.f;
-        for (int64_t r = r0; r < r1; ++r) {
-            float x = src[r * ld + c];
-            if (mask && !((mask[r * mask_words + (c >> 5)] >> (c & 31)) & 1u)) x = 0.f;
-            if (dst) dst[r * ld_dst + c] = x;
-            s += x;
+    const int d4 = (d + 3) / 4;
+    for (int cb = 0; cb < d4; cb += tpr) {  // column blocks (one unless d > 1024)
+        const int c = cb + c4;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < d4) {
+            for (int64_t r = r0 + rg; r < r1; r += n_rg) {
+                float4 x = __ldg(reinterpret_cast<const float4 *>(src + r * ld) + c);
+                if (mask) {
+                    const uint32_t w = mask[r * mask_words + (c >> 3)] >> ((c & 7) * 4);
+                    if (!(w & 1u)) x.x = 0.f;
+                    if (!(w & 2u)) x.y = 0.f;
+                    if (!(w & 4u)) x.z = 0.f;
+                    if (!(w & 8u)) x.w = 0.f;
+                }
+                if (4 * c + 3 >= d) {  // ragged tail: keep the padding columns out of the sums
+                    if (4 * c + 1 >= d) x.y = 0.f;
+                    if (4 * c + 2 >= d) x.z = 0.f;
+                    x.w = 0.f;
+                }
+                if (dst) *(reinterpret_cast<float4 *>(dst + r * ld_dst) + c) = x;
+                s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
+            }
         }
-        if (colsum_part) colsum_part[(int64_t)blockIdx.x * d + c] = s;
+        if (colsum_part) {
+            red[threadIdx.x] = s;
+            __syncthreads();
+            if (rg == 0 && c < d4) {
+                float4 t = red[c4];
+                for (int g = 1; g < n_rg; ++g) {
+                    const float4 y = red[g * tpr + c4];
+                    t.x += y.x; t.y += y.y; t.z += y.z; t.w += y.w;
+                }
+                float *o = colsum_part + (int64_t)blockIdx.x * d + 4 * c;
+                o[0] = t.x;
+                if (4 * c + 1 < d) o[1] = t.y;
+                if (4 * c + 2 < d) o[2] = t.z;
+                if (4 * c + 3 < d) o[3] = t.w;
+            }
+            __syncthreads();
+        }
     }
+}
+
+// zero-padded bias for the tile width (optionally with the same gate interleave as the weights)
+__global__ void k_pack_bias(const float *__restrict__ bias, int32_t n, int32_t n_pad, int32_t gate_h, float *__restrict__ out)
+{
+    const int32_t np = blockIdx.x * blockDim.x + threadIdx.x;
+    if (np >= n_pad) return;
+    const int32_t nn = gate_h > 0 ? (np & 3) * gate_h + (np >> 2) : np;
+    out[np] = np < n ? bias[nn] : 0.f;
 }
 
 // B operand [n_pad x k_pad] (K-major fp32, zero padded) from fp32 weights; the TF32 split happens in the GEMM kernel.
@@ -559,14 +666,15 @@ __global__ void k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t r
 //   transpose = 0: W is [N x K] row-major (ldw) -> B[n][k] = W[n][k]          (C = A W^T)
 // A second source W2 (same orientation, k2 rows) continues along K at column offset k1_pad.
 __global__ void k_split_weights(const float *__restrict__ W, int64_t ldw, int32_t k1, int32_t k1_pad, const float *__restrict__ W2,
-                                int64_t ldw2, int32_t k2, int32_t n, int32_t n_pad, int32_t k_pad, int transpose,
+                                int64_t ldw2, int32_t k2, int32_t n, int32_t n_pad, int32_t k_pad, int transpose, int32_t gate_h,
                                 float *__restrict__ hi, float *__restrict__ lo)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (int64_t)n_pad * k_pad) return;
-    const int32_t nn = (int32_t)(i / k_pad), kk = (int32_t)(i - (int64_t)nn * k_pad);
+    const int32_t np = (int32_t)(i / k_pad), kk = (int32_t)(i - (int64_t)np * k_pad);
+    const int32_t nn = gate_h > 0 ? (np & 3) * gate_h + (np >> 2) : np;  // packed row -> logical column
     float x = 0.f;
-    if (nn < n) {
+    if (np < n) {
         if (kk < k1) x = transpose ? W[(int64_t)kk * ldw + nn] : W[(int64_t)nn * ldw + kk];
         else if (kk >= k1_pad && kk - k1_pad < k2) x = transpose ? W2[(int64_t)(kk - k1_pad) * ldw2 + nn] : W2[(int64_t)nn * ldw2 + (kk - k1_pad)];
     }
@@ -635,14 +743,16 @@ sat_status sat_mask_rows(sat_ctx *ctx, const float *src, int32_t ld, int64_t row
         SAT_TRY(sat_ensure(ctx, ctx->buf_colsum, (size_t)blocks * d * sizeof(float)));
         part = (float *)ctx->buf_colsum.p;
     }
-    k_mask_rows<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld, rows, d, mask, mask_words, dst, ld_dst, part);
+    int tpr = 1;
+    while (tpr < (d + 3) / 4 && tpr < 256) tpr <<= 1;
+    k_mask_rows<<<(unsigned)blocks, 256, 0, ctx->stream>>>(src, ld, rows, d, tpr, mask, mask_words, dst, ld_dst, part);
     SAT_LAUNCHED(ctx);
     if (colsum) SAT_TRY(sat_splitk_reduce(ctx, part, d, (int32_t)blocks, accumulate, colsum, d, d));
     return SAT_OK;
 }
 
 sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1, const float *W2, int32_t ldw2, int32_t k2, int32_t n,
-                          int transpose, DevBuf &buf, TcWeights *out)
+                          int transpose, DevBuf &buf, TcWeights *out, int32_t gate_h)
 {
     const int32_t k1_pad = W2 ? (k1 + TC_BK - 1) / TC_BK * TC_BK : k1;
     const int32_t k_tot = k1_pad + (W2 ? k2 : 0);
@@ -656,7 +766,7 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
     out->ld = k_pad;
     out->n_pad = n_pad;
     k_split_weights<<<(unsigned)cdiv64((int64_t)n_pad * k_pad, 256), 256, 0, ctx->stream>>>(W, ldw, k1, k1_pad, W2, ldw2, k2, n, n_pad, k_pad,
-                                                                                          transpose, out->hi, out->lo);
+                                                                                          transpose, gate_h, out->hi, out->lo);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
@@ -675,7 +785,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     const size_t smem = (size_t)TCK_STAGES * stage_bytes + TCK_OUT_BYTES + sizeof(TcShared) + 1024;
     ProfScope prof(ctx, family, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
     CUtensorMap mA, mA2, mB, mC;
-    const int use_tma_store = ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
+    const int use_tma_store = eh.lstm_h == 0 && ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
     if (use_tma_store) SAT_TRY(make_map(ctx, &mC, eh.C, n, m, eh.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B));
     else memset(&mC, 0, sizeof(mC));
     SAT_TRY(make_map(ctx, &mA, A, k1, m, lda, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
@@ -693,10 +803,14 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     if (eh.bias) {  // zero-padded copy so that the epilogue can read whole 128-bit vectors
         const size_t padded = (size_t)cdiv64(n, bn) * bn;
         SAT_TRY(sat_ensure(ctx, ctx->buf_bias, padded * sizeof(float)));
-        SAT_CUDA(ctx, cudaMemsetAsync(ctx->buf_bias.p, 0, padded * sizeof(float), ctx->stream));
-        SAT_CUDA(ctx, cudaMemcpyAsync(ctx->buf_bias.p, eh.bias, (size_t)n * sizeof(float), cudaMemcpyDeviceToDevice, ctx->stream));
+        k_pack_bias<<<(unsigned)cdiv64(padded, 256), 256, 0, ctx->stream>>>(eh.bias, n, (int32_t)padded, eh.lstm_h, (float *)ctx->buf_bias.p);
+        SAT_LAUNCHED(ctx);
         ep.bias = (const float *)ctx->buf_bias.p;
     }
+    ep.lstm_h = eh.lstm_h;
+    ep.lstm_first = eh.lstm_first;
+    ep.lstm_c = eh.lstm_c;
+    if (eh.lstm_h > 0 && (!eh.bias || !eh.lstm_c || n != 4 * eh.lstm_h)) return sat_fail(ctx, SAT_EINVAL, "fused LSTM epilogue needs bias, cell state and n = 4h");
     ep.relu = eh.relu;
     ep.mask_out = eh.mask_out;
     ep.mask_words = eh.mask_words;

@@ -14,6 +14,7 @@
 #define SAT_MAX_LAYERS 16
 #define SAT_MAX_PARTS 4096
 #define SAT_SPMM_CHUNK 256 /* edges per SpMM work item */
+#define SAT_HROW_LONG 256  /* halo rows with more entries than this get a whole thread block */
 
 // A growable device buffer owned by the context.
 struct DevBuf {
@@ -89,6 +90,9 @@ struct sat_ctx {
     int32_t *hrow_pos = nullptr;  // [nnz_cut] partition-major row of the inner neighbour
     int32_t *hrow_slot = nullptr; // [nnz_cut] its cache slot
     int64_t nnz_cut = 0;
+    int32_t *hlong = nullptr;     // [n_hlong] halo positions of the halo rows longer than SAT_HROW_LONG
+    int32_t n_hlong = 0;
+    std::vector<int32_t> h_hlong_off;
     // SpMM work items (rows cut into chunks of SAT_SPMM_CHUNK edges)
     int32_t *first_item = nullptr; // [n+1]
     int32_t *item_row = nullptr;   // [n_items]
@@ -176,6 +180,7 @@ struct PartView {
     int32_t mrow0, n_mrows;   // multi-chunk rows
     int32_t mitem0, n_mitems; // partial-sum rows
     int32_t push0, n_push;
+    int32_t hlong0, n_hlong;  // long halo rows
     int64_t lnnz;             // local non-zeros (entries of A + I) of the selected rows
 };
 sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
@@ -235,6 +240,11 @@ struct TcEpilogueHost {
     const float *resid = nullptr;      // C += resid[resid_idx[i]] (row gather)
     const int32_t *resid_idx = nullptr;
     int32_t ld_resid = 0;
+    // fused LSTM cell (the weights must have been packed with gate interleave): the n = 4h outputs of a row are the gate
+    // pre-activations; the epilogue applies c = f c + i g, s = o tanh(c) and writes s to C [m x h] and c to lstm_c [m x h]
+    int32_t lstm_h = 0;
+    int lstm_first = 0;                // first step: previous cell state is zero
+    float *lstm_c = nullptr;
 };
 // tensor-core path on / off for a contraction with n outputs and k terms (SAT_NO_TC=1 in the environment forces the CUDA cores)
 bool sat_use_tc(int32_t n, int32_t k);
@@ -242,8 +252,10 @@ bool sat_use_tc(int32_t n, int32_t k);
 sat_status sat_mask_rows(sat_ctx *ctx, const float *src, int32_t ld, int64_t rows, int32_t d, const uint32_t *mask, int32_t mask_words,
                          float *dst, int32_t ld_dst, float *colsum, int accumulate);
 // weight planes in `buf`; transpose = 1 for W given as [K x N], 0 for [N x K]; optional second source continuing along K
+// gate_h > 0: the n = 4 gate_h columns (gate blocks i | f | g | o) are interleaved so that packed column 4 j + gate is gate `gate`
+// of hidden unit j (what the fused LSTM epilogue expects)
 sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1, const float *W2, int32_t ldw2, int32_t k2, int32_t n,
-                          int transpose, DevBuf &buf, TcWeights *out);
+                          int transpose, DevBuf &buf, TcWeights *out, int32_t gate_h = 0);
 // C[m x n] = [A | A2] B^T (+ epilogue)
 sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
                        const TcWeights &Bw, const TcEpilogueHost &eh, int family);

@@ -223,29 +223,40 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
         c->S_valid = true;
         return SAT_OK;
     }
-    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_w, (size_t)rows * 4 * h * sizeof(float)));
+    if (!(sat_use_tc(4 * h, d) && 4 * h <= 256)) SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_w, (size_t)rows * 4 * h * sizeof(float)));
     SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_c, (size_t)rows * h * sizeof(float)));
     float *gates = (float *)ctx->buf_lstm_w.p;
     float *cell = (float *)ctx->buf_lstm_c.p;
     const bool tc = sat_use_tc(4 * h, d);
-    TcWeights W1, W2;   // weight planes for the first step (x only) and the later steps ([x | s])
+    // the cell update can be fused into the epilogue (s and c updated in place) when one tile spans all 4h gate columns:
+    // then a tile reads only its own rows of s, and does so before its epilogue overwrites them
+    const bool fused = tc && 4 * h <= 256;
+    TcWeights W1, W2;   // packed weights for the first step (x only) and the later steps ([x | s])
     if (tc) {
-        SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &W1));
-        if (k > 1) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit2, &W2));
+        SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &W1, fused ? h : 0));
+        if (k > 1) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit2, &W2, fused ? h : 0));
     }
     for (int32_t t = 0; t < k; ++t) {
         const float *x = ring_buf(ctx, c, ring_index(ctx, k - 1 - t));  // oldest first
         if (tc) {
             TcEpilogueHost eh;
-            eh.C = gates;
-            eh.ldc = 4 * h;
             eh.bias = p->b;
+            if (fused) {
+                eh.C = c->S;
+                eh.ldc = h;
+                eh.lstm_h = h;
+                eh.lstm_first = t == 0;
+                eh.lstm_c = cell;
+            } else {
+                eh.C = gates;
+                eh.ldc = 4 * h;
+            }
             if (t == 0) SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, x, c->ld, d, nullptr, 0, 0, W1, eh, SATK_GEMM_NN));
             else SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, x, c->ld, d, c->S, h, h, W2, eh, SATK_GEMM_NN));
         } else {
             SAT_TRY(sat_gemm_nn_dual(ctx, rows, 4 * h, d, x, c->ld, p->Wx, 4 * h, t == 0 ? 0 : h, c->S, h, p->Uh, 4 * h, p->b, gates, 4 * h));
         }
-        {
+        if (!fused) {
             ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 7.0, 0.0);
             k_lstm_cell<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(gates, rows, h, t == 0, cell, c->S);
             SAT_LAUNCHED(ctx);

@@ -193,6 +193,7 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
         }
     }
     const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+    if (e1 - e0 > SAT_HROW_LONG) return;  // handled by k_spmm_hrow_long
     for (int64_t eb = e0; eb < e1; eb += G) {
         const int64_t e = eb + lane;
         int32_t c = 0;
@@ -223,6 +224,55 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
     }
 }
 
+// One thread block per long halo row: the 256 / G lane groups take the entries round-robin, their partial sums are added
+// in group order through shared memory (fixed order: reproducible), group 0 adds the self term and stores.
+template <int G, int NV>
+__global__ void __launch_bounds__(256)
+k_spmm_hrow_long(const int32_t *__restrict__ hlong, int32_t hlong0, const int64_t *__restrict__ hrow_ptr,
+                 const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot, const int32_t *__restrict__ halo_slot,
+                 const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src,
+                 const float *__restrict__ self_src, float *__restrict__ out_base, int64_t ld_out)
+{
+    constexpr int NG = 256 / G;
+    __shared__ float4 red[NG][G * NV];
+    const int lane = threadIdx.x & (G - 1), grp = threadIdx.x / G;
+    const int col0 = blockIdx.y * (G * NV);
+    const int64_t j = hlong[hlong0 + blockIdx.x];
+    const float du = __ldg(dinv_enc + n + j);
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+    for (int64_t e = e0 + grp; e < e1; e += NG) {
+        const int32_t p = __ldg(hrow_pos + e);
+        const float w = __ldg(dinv_enc + p);
+        const int32_t c = by_slot ? __ldg(hrow_slot + e) : p;
+        const float *src = src_base + (int64_t)c * ld_src;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) fma4(acc[v], w, ld4(src + 4 * idx));
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) red[grp][lane + v * G] = acc[v];
+    __syncthreads();
+    if (grp == 0) {
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx >= d4) continue;
+            float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (self_src) fma4(a, du, ld4(self_src + (int64_t)halo_slot[j] * ld_src + 4 * idx));
+            for (int g = 0; g < NG; ++g) {
+                const float4 x = red[g][lane + v * G];
+                a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
+            }
+            *reinterpret_cast<float4 *>(out_base + j * ld_out + 4 * idx) = make_float4(du * a.x, du * a.y, du * a.z, du * a.w);
+        }
+    }
+}
+
 template <int G, int NV>
 static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4, const float *src_base, int32_t ld_src,
                         const float *self_src, float *out_base, int32_t ld_out)
@@ -230,6 +280,13 @@ static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4
     dim3 grid((unsigned)cdiv64(v.n_halo * G, 256), (unsigned)cdiv64(d4, G * NV));
     k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->halo_slot, ctx->dinv_enc, ctx->n,
                                                        v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out);
+    if (v.n_hlong > 0) {
+        dim3 grid2((unsigned)v.n_hlong, (unsigned)cdiv64(d4, G * NV));
+        k_spmm_hrow_long<G, NV><<<grid2, 256, 0, ctx->stream>>>(ctx->hlong, v.hlong0, ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot,
+                                                                 ctx->halo_slot, ctx->dinv_enc, ctx->n, by_slot, d4, src_base, ld_src,
+                                                                 self_src, out_base, ld_out);
+        ctx->launches++;
+    }
 }
 
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src, int by_slot,
