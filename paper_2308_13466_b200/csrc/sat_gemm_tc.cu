@@ -416,10 +416,20 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #pragma unroll
                         for (int j = 0; j < 32; ++j) bq[j] = 0.f;
                     }
+                    if (rrow) {
+                        // gathered residual row: 128-bit loads (rows are padded to a multiple of 4 floats)
+                        const int32_t n4 = (N + 3) & ~3;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            if (n0 + c0 + 4 * j < n4) {
+                                const float4 rv = __ldg(reinterpret_cast<const float4 *>(rrow + n0 + c0) + j);
+                                bq[4 * j] += rv.x; bq[4 * j + 1] += rv.y; bq[4 * j + 2] += rv.z; bq[4 * j + 3] += rv.w;
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         float z = __uint_as_float(r[j]) + bq[j];
-                        if (rrow && n0 + c0 + j < N) z += __ldg(rrow + n0 + c0 + j);
                         bits |= (z > 0.f ? 1u : 0u) << j;
                         if (ep.relu) z = fmaxf(z, 0.f);
                         r[j] = __float_as_uint(z);
