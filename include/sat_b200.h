@@ -262,6 +262,32 @@ sat_status sat_dense_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const flo
 sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
                         float *C);
 
+/* ---------------------------------------------------------------------------------------
+ * sat_dense_tn_static — C[m x n] = A[rows x m]^T B[rows x n] like sat_dense_tn, for callers that cannot allocate.
+ * (The paper has no counterpart; this is a deployment variant of the weight-gradient product.)
+ *
+ * Who needs it: code that must not call cudaMalloc — a process whose device heap is fully owned by another component,
+ * latency-critical loops that cannot take the device-wide synchronisation an allocation implies, or a host region in which
+ * allocation calls are forbidden.  This entry point needs no context, calls no cudaMalloc / cudaFree and no allocating
+ * library routine: the partial sums of the row splits live in an 8 MiB array that is part of the library image (every
+ * GPU that loads the library holds it until the process exits).
+ *
+ *   cuda_stream  cudaStream_t to enqueue on (may be 0); the device must be current
+ *   A, B, C      DEVICE fp32, caller-owned; A [rows x lda], B [rows x ldb], C dense [m x n] (overwritten)
+ *   errbuf       HOST buffer (may be NULL) that receives a message when the status is not SAT_OK
+ * Limit: m * n <= 2,097,152 (the array holds at least one m x n block of partial sums); larger shapes are rejected with
+ * SAT_EINVAL and a message naming the limit — use sat_dense_tn then.  Fewer splits fit for larger m * n, so very tall
+ * inputs run slower here than through sat_dense_tn.
+ * Set-up: the first call on each device looks up the device address of the array (once per device, kept for the
+ * process); make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array.  It keeps whatever the previous call left; nothing has to be
+ * cleared because each call overwrites every partial block it later reads.  Two calls that overlap on the GPU (different
+ * streams, or concurrent threads) race on the array: serialise them.
+ * The result is bit-reproducible from call to call (fixed split sizes and summation order).
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_dense_tn_static(void *cuda_stream, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B,
+                               int32_t ldb, float *C, char *errbuf, int32_t errbuf_len);
+
 /* Number of kernels this context has launched since creation (all entry points). */
 sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
 

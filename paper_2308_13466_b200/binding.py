@@ -57,7 +57,7 @@ EXPORTS = [
     "sat_part_sizes", "sat_part_lists", "sat_slot_map", "sat_gather_rows", "sat_cache_init", "sat_predict",
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
-    "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
+    "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
 ]
 
 
@@ -291,6 +291,18 @@ def sat_dense_tn(ctx, A, Bm, out):
     assert out.is_contiguous()
     _check(ctx, _lib.sat_dense_tn(ctx, C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A), C.c_int32(_ld(A)),
                                   _dev(Bm), C.c_int32(_ld(Bm)), _dev(out)))
+
+
+def sat_dense_tn_static(stream: int, A, Bm, out):
+    """out[m, n] = A[rows, m]^T Bm[rows, n] without any allocation: the split partial sums live in an array built into the
+    library (for callers that must not call cudaMalloc).  Needs no context; `stream` is a raw cudaStream_t (0 = default).
+    Raises SatError with the library's message, e.g. when m * n exceeds the built-in scratch."""
+    assert out.is_contiguous()
+    err = C.create_string_buffer(256)
+    st = _lib.sat_dense_tn_static(C.c_void_p(stream), C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A),
+                                  C.c_int32(_ld(A)), _dev(Bm), C.c_int32(_ld(Bm)), _dev(out), err, C.c_int32(256))
+    if st != SAT_OK:
+        raise SatError(st, err.value.decode())
 
 
 def sat_launch_count(ctx) -> int:

@@ -303,3 +303,80 @@ sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const f
     if (colsum) SAT_TRY(sat_splitk_reduce(ctx, part_cs, n, (int32_t)splits, accumulate, colsum, n, n));
     return SAT_OK;
 }
+
+// =====================================================================================
+// sat_dense_tn_static: the split weight-gradient product without any allocation
+// =====================================================================================
+// Some callers must not allocate device memory at all: code that runs while another component owns the whole device
+// heap (a serving process that pre-reserves every byte), real-time loops where cudaMalloc's implicit device-wide
+// synchronisation is not acceptable, and code running inside a region where allocation calls are forbidden.  For them the
+// split partial sums of C = A^T B live in this fixed array, which is part of the library image: every GPU that loads the
+// library carries it until the process exits.
+#define SAT_STATIC_SCRATCH_FLOATS (2 * 1024 * 1024) /* 8 MiB */
+static __device__ __align__(256) float sat_static_scratch[SAT_STATIC_SCRATCH_FLOATS];
+
+#include <mutex>
+
+#define SAT_STATIC_MAX_DEVICES 64
+static std::mutex g_static_mutex;
+static float *g_static_ptr[SAT_STATIC_MAX_DEVICES] = {nullptr};  // device address of sat_static_scratch, per device
+
+static sat_status static_fail(char *errbuf, int32_t errbuf_len, sat_status code, const char *fmt, ...)
+{
+    if (errbuf && errbuf_len > 0) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(errbuf, (size_t)errbuf_len, fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+extern "C" sat_status sat_dense_tn_static(void *cuda_stream, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda,
+                                          const float *B, int32_t ldb, float *C, char *errbuf, int32_t errbuf_len)
+{
+    if (errbuf && errbuf_len > 0) errbuf[0] = 0;
+    if (rows < 0 || m <= 0 || n <= 0 || !A || !B || !C || lda < m || ldb < n)
+        return static_fail(errbuf, errbuf_len, SAT_EINVAL, "sat_dense_tn_static: null tensor or bad shape (rows %lld, m %d, n %d, lda %d, ldb %d)",
+                           (long long)rows, m, n, lda, ldb);
+    if ((int64_t)m * n > SAT_STATIC_SCRATCH_FLOATS)
+        return static_fail(errbuf, errbuf_len, SAT_EINVAL,
+                           "sat_dense_tn_static: m * n = %lld exceeds the built-in scratch of %d floats (8 MiB); use sat_dense_tn",
+                           (long long)m * n, SAT_STATIC_SCRATCH_FLOATS);
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= SAT_STATIC_MAX_DEVICES)
+        return static_fail(errbuf, errbuf_len, SAT_ECUDA, "sat_dense_tn_static: no usable current device (%s)", cudaGetErrorString(e));
+    float *scratch = nullptr;
+    {
+        // one-time set-up per device: `sat_static_scratch` named in host code is only a handle, the kernels need the
+        // address the symbol has on the current device
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev]) {
+            float *p = nullptr;
+            e = cudaGetSymbolAddress((void **)&p, sat_static_scratch);
+            if (e != cudaSuccess || !p)
+                return static_fail(errbuf, errbuf_len, SAT_ECUDA, "sat_dense_tn_static: cudaGetSymbolAddress failed (%s)", cudaGetErrorString(e));
+            g_static_ptr[dev] = p;
+        }
+        scratch = g_static_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // as many row splits as the fixed array holds (each split owns an m x n block of partial sums)
+    int64_t splits = cdiv64(rows > 0 ? rows : 1, TN_ROWS_PER_SPLIT);
+    const int64_t cap = SAT_STATIC_SCRATCH_FLOATS / ((int64_t)m * n);
+    if (splits > cap) splits = cap;
+    if (splits > 1024) splits = 1024;
+    int64_t rows_per_split = cdiv64(cdiv64(rows > 0 ? rows : 1, splits), BK) * BK;
+    splits = cdiv64(rows > 0 ? rows : 1, rows_per_split);
+    // every element of the `splits` partial blocks is written by exactly one thread block below, so nothing left over from
+    // an earlier call is ever read and no clearing is needed
+    dim3 grid((unsigned)cdiv64(m, BM), (unsigned)cdiv64(n, BN), (unsigned)splits);
+    k_gemm_tn<<<grid, 256, 0, st>>>(rows, rows_per_split, m, n, A, lda, B, ldb, nullptr, 0, scratch, nullptr);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return static_fail(errbuf, errbuf_len, SAT_ECUDA, "sat_dense_tn_static: launch failed (%s)", cudaGetErrorString(e));
+    k_splitk_reduce<<<(unsigned)cdiv64((int64_t)m * n, 32), 256, 0, st>>>(scratch, (int64_t)m * n, (int32_t)splits, 0, C, n, n);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return static_fail(errbuf, errbuf_len, SAT_ECUDA, "sat_dense_tn_static: launch failed (%s)", cudaGetErrorString(e));
+    return SAT_OK;
+}
