@@ -89,7 +89,7 @@ class Partitioning:
     push_slot: list = field(default_factory=list)   # their slots
 
 
-def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: int) -> Partitioning:
+def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: int, only_parts=None) -> Partitioning:
     """All per-partition lists, from their definitions.
 
     I_m = {v : part[v] = m};  B_m = sorted unique { u not in V_m : exists v in V_m, (v,u) in E };
@@ -97,14 +97,27 @@ def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: in
     I_m; halo: n_m + rank in B_m) and sorted ascending; halo-row CSR: for u in B_m the
     neighbours of u inside V_m (the transpose of the halo block); C = sorted union of the
     B_m, slot = rank in C; push list = inner nodes of m that are in C.
+    `only_parts` builds the per-partition lists of a subset only (the others stay None); C and
+    slot[] are always global: u is in some B_m exactly when an edge (v, u) has part[v] != part[u].
     """
     n = rowptr.shape[0] - 1
     part = np.ascontiguousarray(part, dtype=np.int32)
     deg = np.diff(rowptr)
     P = Partitioning(n=n, M=M, part=part, slot=None, n_slots=0)
     in_any_halo = np.zeros(n, dtype=bool)
+    step = 1 << 24                                    # union of all halo sets, edge chunk by edge chunk
+    row_of = np.repeat(np.arange(n, dtype=np.int32), deg)
+    for e0 in range(0, col.shape[0], step):
+        c = col[e0:e0 + step]
+        cut = part[row_of[e0:e0 + step]] != part[c]
+        in_any_halo[c[cut]] = True
+    del row_of
     per = []
+    todo = list(range(M)) if only_parts is None else list(only_parts)
     for m in range(M):
+        if m not in todo:
+            per.append(None)
+            continue
         inner = np.nonzero(part == m)[0].astype(np.int64)
         n_m = inner.shape[0]
         loc_of = np.full(n, -1, dtype=np.int64)
@@ -116,7 +129,6 @@ def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: in
         dst = col[starts + np.arange(src.shape[0], dtype=np.int64)].astype(np.int64)
         outside = part[dst] != m
         halo = np.unique(dst[outside])
-        in_any_halo[halo] = True
         # add the self-loop of every inner row
         src2 = np.concatenate([src, np.arange(n_m, dtype=np.int64)])
         dst2 = np.concatenate([dst, inner])
@@ -138,7 +150,12 @@ def build_partition(rowptr: np.ndarray, col: np.ndarray, part: np.ndarray, M: in
     slot = np.full(n, -1, dtype=np.int32)
     slot[Cset] = np.arange(Cset.shape[0], dtype=np.int32)
     P.slot, P.n_slots = slot, int(Cset.shape[0])
-    for inner, halo, lrp, lc, hp, hc in per:
+    for item in per:
+        if item is None:
+            for lst in (P.inner_gid, P.halo_gid, P.loc_rowptr, P.loc_col, P.hrow_ptr, P.hrow_col, P.halo_slot, P.push_local, P.push_slot):
+                lst.append(None)
+            continue
+        inner, halo, lrp, lc, hp, hc = item
         P.inner_gid.append(inner)
         P.halo_gid.append(halo)
         P.loc_rowptr.append(lrp)

@@ -84,9 +84,8 @@ def rmat_graph(seed: int, scale: int, n: int, probs=(0.57, 0.19, 0.19, 0.05), *,
     Exactly one of:
       n_samples            accept this many directed samples (endpoint >= n rejected),
                            then drop self-loops and duplicates;
-      n_unique_undirected  keep sampling in rounds until this many distinct unordered
-                           pairs exist; the last round contributes its new pairs in
-                           sample order until the target is met.
+      n_unique_undirected  keep sampling in rounds until at least this many distinct unordered
+                           pairs exist; a surplus is dropped uniformly at random (seeded).
     attach_isolated: every node left without an edge gets one edge to a node drawn from
     the R-MAT row marginal, so the graph has no isolated node (the citation /
     co-purchase graphs this stands in for have none).
@@ -117,19 +116,20 @@ def rmat_graph(seed: int, scale: int, n: int, probs=(0.57, 0.19, 0.19, 0.05), *,
         keys = np.unique(lo * n + hi)
     else:
         keys = np.empty(0, dtype=np.int64)
-        round_size = int(min(max(n_unique_undirected // 2, 1 << 16), 1 << 24))
         while keys.shape[0] < n_unique_undirected:
-            r, c = draw(round_size)
-            keep = r != c
-            k = np.minimum(r[keep], c[keep]) * n + np.maximum(r[keep], c[keep])
-            uk, first = np.unique(k, return_index=True)
-            fresh = ~np.isin(uk, keys, assume_unique=True)
-            uk, first = uk[fresh], first[fresh]
-            need = n_unique_undirected - keys.shape[0]
-            if uk.shape[0] > need:
-                order = np.argsort(first, kind="stable")[:need]
-                uk = uk[order]
-            keys = np.union1d(keys, uk)
+            want = int((n_unique_undirected - keys.shape[0]) * 1.5) + (1 << 16)
+            parts = [keys]
+            while want > 0:                       # bounded chunks keep the temporaries small
+                chunk = min(want, 1 << 25)
+                r, c = draw(chunk)
+                keep = r != c
+                parts.append(np.minimum(r[keep], c[keep]) * n + np.maximum(r[keep], c[keep]))
+                want -= chunk
+            keys = np.unique(np.concatenate(parts))
+        if keys.shape[0] > n_unique_undirected:   # drop the surplus uniformly at random (seeded)
+            pick = rng.choice(keys.shape[0], size=n_unique_undirected, replace=False)
+            pick.sort()
+            keys = keys[pick]
     lo = keys // n
     hi = keys - lo * n
 

@@ -58,3 +58,31 @@ def pred_to_device(pred_list, B):
                                       dev(p["b"].astype(np.float32)), dev(p["Wg"].astype(np.float32)),
                                       dev(p["bg"].astype(np.float32)), h))
     return out
+
+
+TIE = 1e-4  # a hidden pre-activation with |Z| <= TIE * rms(Z) is below the tolerance of Z itself: its ReLU mask bit is a tie
+
+
+def relu_tie_masks(res, P, H_gpu, inner_off, L):
+    """Compares the oracle's ReLU masks [Z > 0] with the CUDA path's (H > 0) for every partition and hidden layer.
+
+    Where |Z| is at rounding level the two sides may decide the sign differently and both are correct; anywhere else a
+    disagreement is an error (asserted).  Returns (masks, differs): masks[m][l-1] = the CUDA path's decision (uint8) to hand
+    to the oracle's backward, differs = whether any tie was decided differently."""
+    masks, differs = [None] * P.M, False
+    for m in range(P.M):
+        if res.per_part[m] is None:
+            continue
+        masks[m] = []
+        r0 = int(inner_off[m])
+        for l in range(1, L):
+            Z = res.per_part[m]["Z"][l - 1]
+            theirs = H_gpu[l][r0:r0 + Z.shape[0]] > 0
+            diff = (Z > 0) != theirs
+            if diff.any():
+                rms = float(np.sqrt(np.mean(Z * Z)))
+                assert np.all(np.abs(Z[diff]) <= TIE * rms), f"ReLU mask disagreement away from zero (partition {m}, layer {l})"
+                differs = True
+            masks[m].append(theirs.astype(np.uint8))
+        masks[m].append(None)
+    return masks, differs

@@ -8,7 +8,7 @@ import pytest
 
 from oracle import sat_ref as orc
 from sat_synth import make_workload
-from tests.gpu_util import assert_close, dev, dev2d, pred_to_device
+from tests.gpu_util import assert_close, dev, dev2d, pred_to_device, relu_tie_masks
 
 pytestmark = pytest.mark.gpu
 
@@ -54,21 +54,8 @@ def test_epochs_from_synchronised_state(B, name, shrink):
             torch.cuda.synchronize()
             # ReLU ties: where |Z| is at rounding level the two sides may decide the sign differently; both are
             # correct, so the oracle's backward is redone with the CUDA path's decision on exactly those entries.
-            masks, redo = [None] * P.M, False
-            for m in range(P.M):
-                masks[m] = []
-                r0 = int(ep.inner_off[m])
-                for l in range(1, wl.L):
-                    Z = res.per_part[m]["Z"][l - 1]
-                    mine = Z > 0
-                    theirs = ep.H[l][r0:r0 + Z.shape[0]].cpu().numpy() > 0
-                    diff = mine != theirs
-                    if diff.any():
-                        rms = float(np.sqrt(np.mean(Z * Z)))
-                        assert np.all(np.abs(Z[diff]) <= 1e-5 * rms), f"epoch {t}: mask disagreement away from zero"
-                        redo = True
-                    masks[m].append(theirs.astype(np.uint8))
-                masks[m].append(None)
+            H_gpu = [None] + [ep.H[l].cpu().numpy() for l in range(1, wl.L + 1)]
+            masks, redo = relu_tie_masks(res, P, H_gpu, ep.inner_off, wl.L)
             if redo:
                 cache = before
                 res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, W, b, wl.pred, wl.loss, masks=masks)
