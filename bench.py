@@ -224,7 +224,7 @@ def run_ours(args, wl):
     ep.set_inputs(X_dev, up(labels_perm))
     W = [up(w) for w in wl.W]
     b = [up(x) for x in wl.b]
-    preds = [B.make_pred_params(up(p["Wx"]), up(p["Uh"]), up(p["b"]), up(p["Wg"]), up(p["bg"]), int(p["h"])) for p in wl.pred]
+    preds = [B.make_pred_params(up(p["Wx"]), up(p["Uh"]), up(p["b"]), up(p["Wg"]), up(p["bg"]), int(p["h"]), 1) for p in wl.pred]  # version 1: the predictor is not updated during the run
     lr = 0.01
 
     # fill the ring with real embeddings (tau + 1 epochs), then W warm-up steps

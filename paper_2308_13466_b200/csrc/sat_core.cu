@@ -133,6 +133,7 @@ static void free_cache(sat_ctx *ctx)
     for (int i = 0; i < SAT_MAX_LAYERS; ++i) {
         dev_free(&ctx->cache[i].buf);
         dev_free(&ctx->cache[i].S);
+        dev_free(&ctx->cache[i].proj);
         ctx->cache[i] = CacheLayer();
     }
     ctx->cache_ok = false;

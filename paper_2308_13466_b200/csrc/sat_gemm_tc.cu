@@ -2,17 +2,18 @@
 // operands staged in shared memory by TMA) with fp32-level accuracy from a two-term TF32 split:
 //     x = hi + lo,  hi = tf32(x), lo = tf32(x - hi)            (|x - hi - lo| <= 2^-22 |x|)
 //     A B ~= Ah Bh + Ah Bl + Al Bh                              (three MMAs per k-step, fp32 accumulate)
-// Activations stay plain fp32 in global memory: TMA brings the fp32 tile into shared memory and the
-// converter warps round it to TF32 in place and write the residual tile next to it (element-wise, so the
-// swizzled layout never has to be decoded).  Weights are pre-split once per call into two fp32 planes.
+// Activations and weights stay plain fp32 in global memory: TMA brings the fp32 tiles into shared memory and the
+// converter warps round them to TF32 in place and write the residual tiles next to them (element-wise, so the
+// swizzled layout never has to be decoded).  Weights are repacked once per call into the K-major operand layout.
 //
-//   k_gemm_tc_k   C[M x N] = A[M x K] B[N x K]^T   both operands K-major, 64-byte swizzle, BLOCK_K = 16
-//                 (layer transform, LSTM gates with two A operands, predictor output, input gradient)
+//   k_gemm_tc_k   C[M x N] = A[M x K] B[N x K]^T   both operands K-major, 64-byte swizzle, BLOCK_K = 16, persistent
+//                 (layer transform, LSTM gates with two A operands or a cached projection, predictor output, input gradient)
 //   k_gemm_tc_mn  C[M x N] = A[R x M]^T B[R x N]   both operands MN-major, 128-byte swizzle with 32-byte atoms, split over R
 //                 (weight gradient)
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..5 = converters during the
-// main loop, then epilogue (one TMEM lane quadrant each).  Every mbarrier wait is bounded; a timeout raises a
-// status word and lets the CTA drain (TMEM is freed, the kernel returns).
+// Warp roles of k_gemm_tc_k: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..7 = converters,
+// warps 8..15 = epilogue (two per TMEM lane quadrant).  k_gemm_tc_mn: warps 0 / 1 as above, warps 2..5 convert during the
+// main loop and then run the epilogue.  Every mbarrier wait is bounded; a timeout raises a status word and lets the CTA
+// drain (TMEM is freed, the kernel returns).
 #include <cuda.h>
 
 #include "sat_internal.h"
@@ -56,6 +57,16 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     *dead = 1;
     atomicOr(status, 1);
     return false;
+}
+// whole-warp wait: lane 0 polls, then every lane observes the completed phase itself (one immediate try_wait each), so
+// that a waiting warp issues one poll per round instead of 32
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *dead, int *status, int lane)
+{
+    int ok = 1;
+    if (lane == 0) ok = mbar_wait(bar, parity, dead, status) ? 1 : 0;
+    ok = __shfl_sync(0xffffffffu, ok, 0);
+    if (!ok) return false;
+    return mbar_wait(bar, parity, dead, status);
 }
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, uint64_t *bar, int32_t x, int32_t y)
 {
@@ -193,6 +204,8 @@ struct TcEpilogue {
     int32_t lstm_h;      // > 0: fused LSTM cell, C = hidden state [M x lstm_h], lstm_c = cell state
     int lstm_first;
     float *lstm_c;
+    const float *addend; // [M x ld_addend] added to the gate pre-activations (cached input projection), or null
+    int64_t ld_addend;
 };
 
 // logistic and tanh from the hardware exponential (ex2.approx) and reciprocal: absolute error of a few 1e-7, which is
@@ -218,14 +231,24 @@ struct TcShared {
 
 #define TC_CONV_THREADS 128
 #define TC_EPI_THREADS 128
-#define TCK_CONV_THREADS 256
-#define TCK_THREADS 448   /* warp 0 TMA, warp 1 MMA, warps 2-9 converters, warps 10-13 epilogue */
+#define TCK_CONV_WARPS 6
+#define TCK_CONV_THREADS (TCK_CONV_WARPS * 32)
+#define TCK_EPI_WARPS 8
+#define TCK_EPI_THREADS (TCK_EPI_WARPS * 32)
+#define TCK_EPI_WARP0 (2 + TCK_CONV_WARPS)
+#define TCK_THREADS (64 + TCK_CONV_THREADS + TCK_EPI_THREADS) /* warp 0 TMA, warp 1 MMA, then the converter warps, then the epilogue warps: 512 threads, 128 registers each */
 #define TCK_STAGES 4
-#define TCK_OUT_BYTES (4 * 2 * 4096)  /* per epilogue warp two 32 x 32 fp32 staging tiles for the TMA stores */
+#define TCK_OUT_BYTES (TCK_EPI_WARPS * 4096)  /* per epilogue warp one 32 x 32 fp32 staging tile for the TMA stores */
+
+enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2 };
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of TCK_STAGES k-blocks
 // and the two TMEM accumulator buffers let the TMA loads, the TF32 split, the MMAs and the epilogue of consecutive tiles
 // overlap.  A and B arrive as raw fp32 tiles; the converters round them to TF32 in place and write the residual tiles.
+// The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell) and runs on eight
+// warps, two per TMEM lane quadrant taking alternate 32-column chunks: with one warp per scheduler the epilogue was bound
+// by instruction issue and load latency (9 - 14 us per 128 x 256 tile, longer than the main loop of a K = 256 tile).
+template <int EPI>
 __global__ void __launch_bounds__(TCK_THREADS, 1)
 k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB,
             const __grid_constant__ CUtensorMap mapC, int use_tma_store, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t n_tiles_n, int64_t n_tiles, TcEpilogue ep, int *status)
@@ -249,7 +272,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh->acc_full[i], 1);
-            mbar_init(&sh->acc_empty[i], TC_EPI_THREADS);
+            mbar_init(&sh->acc_empty[i], TCK_EPI_THREADS);
         }
         sh->dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -316,7 +339,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 tc_commit(&sh->acc_full[buf]);
             }
         }
-    } else if (warp < 10) {
+    } else if (warp < TCK_EPI_WARP0) {
         // ---------------- converters: TF32 split of the A and B tiles of every k-block ----------------
         const int ctid = threadIdx.x - 64;
         uint32_t it = 0;
@@ -324,7 +347,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
                 const int s = it % TCK_STAGES;
                 const uint32_t ph = (it / TCK_STAGES) & 1u;
-                if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
+                if (!mbar_wait_warp(&sh->full[s], ph, dead, status, lane)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 split_tile(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
                 split_tile(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_THREADS);
@@ -333,53 +356,87 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             }
         }
     } else {
-        // ---------------- epilogue: warp w owns TMEM lanes 32 (w % 4) .. +31 = rows of the tile ----------------
+        // ---------------- epilogue ----------------
+        // warp w reads TMEM lanes 32 (w % 4) .. +31 = rows of the tile, one row per thread; the two warps of a lane quadrant
+        // take alternate 32-column chunks.  Per-row side operands (gathered residual row, cached projection, previous cell
+        // state) are latency-bound loads: they are issued one chunk ahead, the first chunk's before the accumulator is ready.
+        const int e = warp - TCK_EPI_WARP0;
         const int q = warp & 3;
-        uint8_t *obuf = out_stage + (warp - 10) * 8192;
-        uint32_t ob = 0;
+        const int c_first = 32 * (e >> 2);
+        uint8_t *obuf = out_stage + e * 4096;
         const bool vec = ((ep.ldc & 3) == 0) && ((((uintptr_t)ep.C) & 15u) == 0);
+        const int32_t n4 = (N + 3) & ~3;
+        const bool lstm_full = EPI == EPI_LSTM && (ep.lstm_h & 3) == 0;
+        const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
         uint32_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
             const int64_t m0 = (t / n_tiles_n) * TC_BM;
             const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
             const uint32_t buf = lt & 1u;
-            if (!mbar_wait(&sh->acc_full[buf], (lt >> 1) & 1u, dead, status)) goto done;
-            tc_fence_after();
             const int64_t row = m0 + q * 32 + lane;
             const bool row_ok = row < M;
-            const float *rrow = nullptr;
-            if (row_ok && ep.resid_idx) rrow = ep.resid + (int64_t)ep.resid_idx[row] * ep.ld_resid;
             float *crow = ep.C + row * ep.ldc;
-            for (int c0 = 0; c0 < bn; c0 += 32) {
+            const float *srow = nullptr;  // this thread's row of the side operand, at column n0
+            if (row_ok) {
+                if (EPI == EPI_RESID) srow = ep.resid + (int64_t)ep.resid_idx[row] * ep.ld_resid + n0;  // rows padded to 4 floats
+                if (EPI == EPI_LSTM && ep.addend) srow = ep.addend + row * ep.ld_addend + n0;
+            }
+            const int32_t side_lim = (EPI == EPI_RESID ? n4 : N) - n0;
+            float4 side[8], cside[2];
+            auto load_side = [&](int c0) {
+                if (EPI != EPI_PLAIN) {
+#pragma unroll
+                    for (int u = 0; u < 8; ++u)
+                        side[u] = (srow && c0 + 4 * u < side_lim) ? __ldg(reinterpret_cast<const float4 *>(srow + c0) + u) : zero4;
+                }
+                if (EPI == EPI_LSTM) {
+                    cside[0] = cside[1] = zero4;
+                    const int32_t j0 = (n0 + c0) >> 2;
+                    if (row_ok && lstm_full && !ep.lstm_first && j0 + 7 < ep.lstm_h) {
+                        cside[0] = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
+                        cside[1] = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0 + 4);
+                    }
+                }
+            };
+            if (c_first < bn) load_side(c_first);
+            if (!mbar_wait_warp(&sh->acc_full[buf], (lt >> 1) & 1u, dead, status, lane)) goto done;
+            tc_fence_after();
+            for (int c0 = c_first; c0 < bn; c0 += 64) {
                 uint32_t r[32];
                 tc_ld32(tmem + buf * acc_cols + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                if (ep.lstm_h > 0) {
+                if (EPI == EPI_LSTM) {
                     // packed columns 4 j .. 4 j + 3 are the (i, f, g, o) pre-activations of hidden unit j
                     if (row_ok) {
                         const int32_t j0 = (n0 + c0) >> 2;
-                        float sv[8], cv[8], cprev[8];
-                        const bool full = j0 + 7 < ep.lstm_h && (ep.lstm_h & 3) == 0;
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) cprev[u] = 0.f;
-                        if (!ep.lstm_first) {
-                            if (full) {
-                                const float4 c0v = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
-                                const float4 c1v = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0 + 4);
-                                cprev[0] = c0v.x; cprev[1] = c0v.y; cprev[2] = c0v.z; cprev[3] = c0v.w;
-                                cprev[4] = c1v.x; cprev[5] = c1v.y; cprev[6] = c1v.z; cprev[7] = c1v.w;
-                            } else {
-#pragma unroll
-                                for (int u = 0; u < 8; ++u)
-                                    if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[row * ep.lstm_h + j0 + u];
-                            }
-                        }
+                        const bool full = lstm_full && j0 + 7 < ep.lstm_h;
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
-                            const float4 bv = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + u);
-                            const float gi = sigmoid_fast(__uint_as_float(r[4 * u]) + bv.x);
-                            const float gf = sigmoid_fast(__uint_as_float(r[4 * u + 1]) + bv.y);
-                            const float gg = tanh_fast(__uint_as_float(r[4 * u + 2]) + bv.z);
-                            const float go = sigmoid_fast(__uint_as_float(r[4 * u + 3]) + bv.w);
+                            float4 b4 = side[u];
+                            if (ep.bias) {
+                                const float4 bb = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + u);
+                                b4.x += bb.x; b4.y += bb.y; b4.z += bb.z; b4.w += bb.w;
+                            }
+                            r[4 * u] = __float_as_uint(__uint_as_float(r[4 * u]) + b4.x);
+                            r[4 * u + 1] = __float_as_uint(__uint_as_float(r[4 * u + 1]) + b4.y);
+                            r[4 * u + 2] = __float_as_uint(__uint_as_float(r[4 * u + 2]) + b4.z);
+                            r[4 * u + 3] = __float_as_uint(__uint_as_float(r[4 * u + 3]) + b4.w);
+                        }
+                        float cprev[8];
+                        cprev[0] = cside[0].x; cprev[1] = cside[0].y; cprev[2] = cside[0].z; cprev[3] = cside[0].w;
+                        cprev[4] = cside[1].x; cprev[5] = cside[1].y; cprev[6] = cside[1].z; cprev[7] = cside[1].w;
+                        if (!ep.lstm_first && !full) {
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[row * ep.lstm_h + j0 + u];
+                        }
+                        if (c0 + 64 < bn) load_side(c0 + 64);
+                        float sv[8], cv[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            const float gi = sigmoid_fast(__uint_as_float(r[4 * u]));
+                            const float gf = sigmoid_fast(__uint_as_float(r[4 * u + 1]));
+                            const float gg = tanh_fast(__uint_as_float(r[4 * u + 2]));
+                            const float go = sigmoid_fast(__uint_as_float(r[4 * u + 3]));
                             cv[u] = gf * cprev[u] + gi * gg;
                             sv[u] = go * tanh_fast(cv[u]);
                         }
@@ -405,49 +462,40 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 if (row_ok) {
                     // bias is padded with zeros to the tile width and the accumulators of padded columns are exactly zero,
                     // so no column predicate is needed (the stores clip)
-                    float bq[32];
-                    if (ep.bias) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 bv = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + j);
-                            bq[4 * j] = bv.x; bq[4 * j + 1] = bv.y; bq[4 * j + 2] = bv.z; bq[4 * j + 3] = bv.w;
+                    for (int j = 0; j < 8; ++j) {
+                        float4 b4 = EPI == EPI_RESID ? side[j] : zero4;
+                        if (ep.bias) {
+                            const float4 bb = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + j);
+                            b4.x += bb.x; b4.y += bb.y; b4.z += bb.z; b4.w += bb.w;
                         }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) bq[j] = 0.f;
+                        r[4 * j] = __float_as_uint(__uint_as_float(r[4 * j]) + b4.x);
+                        r[4 * j + 1] = __float_as_uint(__uint_as_float(r[4 * j + 1]) + b4.y);
+                        r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + b4.z);
+                        r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + b4.w);
                     }
-                    if (rrow) {
-                        // gathered residual row: 128-bit loads (rows are padded to a multiple of 4 floats)
-                        const int32_t n4 = (N + 3) & ~3;
+                    if (EPI == EPI_RESID && c0 + 64 < bn) load_side(c0 + 64);
+                    if (EPI == EPI_PLAIN && ep.mask_out) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            if (n0 + c0 + 4 * j < n4) {
-                                const float4 rv = __ldg(reinterpret_cast<const float4 *>(rrow + n0 + c0) + j);
-                                bq[4 * j] += rv.x; bq[4 * j + 1] += rv.y; bq[4 * j + 2] += rv.z; bq[4 * j + 3] += rv.w;
-                            }
-                        }
+                        for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
                     }
+                    if (ep.relu) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float z = __uint_as_float(r[j]) + bq[j];
-                        bits |= (z > 0.f ? 1u : 0u) << j;
-                        if (ep.relu) z = fmaxf(z, 0.f);
-                        r[j] = __float_as_uint(z);
+                        for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(fmaxf(__uint_as_float(r[j]), 0.f));
                     }
                 }
                 if (use_tma_store) {
                     // stage the 32 x 32 block (128-byte swizzle: 16-byte chunk j of row r sits at chunk j ^ (r & 7)) and
                     // let the TMA write it as whole 128-byte row segments; rows / columns past the matrix are clipped
-                    if (lane == 0) tma_store_wait_read<1>();  // the buffer used two blocks ago has been read
+                    if (lane == 0) tma_store_wait_read<0>();  // the previous block has left the staging tile
                     __syncwarp();
-                    uint8_t *dst = obuf + ob * 4096 + lane * 128;
+                    uint8_t *dst = obuf + lane * 128;
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
                         *reinterpret_cast<uint4 *>(dst + ((j ^ (lane & 7)) << 4)) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
                     fence_async_smem();
                     __syncwarp();
-                    if (lane == 0) tma_store_2d(&mapC, obuf + ob * 4096, n0 + c0, (int32_t)(m0 + q * 32));
-                    ob ^= 1u;
+                    if (lane == 0) tma_store_2d(&mapC, obuf, n0 + c0, (int32_t)(m0 + q * 32));
                 } else if (row_ok) {
 #pragma unroll
                     for (int j4 = 0; j4 < 32; j4 += 4) {
@@ -461,7 +509,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         }
                     }
                 }
-                if (ep.mask_out && row_ok) {
+                if (EPI == EPI_PLAIN && ep.mask_out && row_ok) {
                     const int32_t word = (n0 + c0) >> 5;
                     if (word < ep.mask_words) ep.mask_out[row * ep.mask_words + word] = bits;
                 }
@@ -803,7 +851,9 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     else mA2 = mA;
     SAT_TRY(make_map(ctx, &mB, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
     if (!g_attr_k) {
-        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_LSTM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
         g_attr_k = true;
     }
     TcEpilogue ep;
@@ -813,14 +863,20 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     if (eh.bias) {  // zero-padded copy so that the epilogue can read whole 128-bit vectors
         const size_t padded = (size_t)cdiv64(n, bn) * bn;
         SAT_TRY(sat_ensure(ctx, ctx->buf_bias, padded * sizeof(float)));
-        k_pack_bias<<<(unsigned)cdiv64(padded, 256), 256, 0, ctx->stream>>>(eh.bias, n, (int32_t)padded, eh.lstm_h, (float *)ctx->buf_bias.p);
+        k_pack_bias<<<(unsigned)cdiv64(padded, 256), 256, 0, ctx->stream>>>(eh.bias, n, (int32_t)padded, eh.lstm_h > 0 ? eh.lstm_h : eh.pack_gate_h,
+                                                                            (float *)ctx->buf_bias.p);
         SAT_LAUNCHED(ctx);
         ep.bias = (const float *)ctx->buf_bias.p;
     }
     ep.lstm_h = eh.lstm_h;
     ep.lstm_first = eh.lstm_first;
     ep.lstm_c = eh.lstm_c;
-    if (eh.lstm_h > 0 && (!eh.bias || !eh.lstm_c || n != 4 * eh.lstm_h)) return sat_fail(ctx, SAT_EINVAL, "fused LSTM epilogue needs bias, cell state and n = 4h");
+    ep.addend = eh.addend;
+    ep.ld_addend = eh.ld_addend;
+    if (eh.lstm_h > 0 && ((!eh.bias && !eh.addend) || !eh.lstm_c || n != 4 * eh.lstm_h || (eh.addend && (eh.ld_addend & 3))))
+        return sat_fail(ctx, SAT_EINVAL, "fused LSTM epilogue needs bias or addend, cell state and n = 4h");
+    if (eh.resid_idx && (eh.mask_out || eh.lstm_h > 0))
+        return sat_fail(ctx, SAT_EINVAL, "gathered-residual epilogue cannot be combined with a mask output or the LSTM cell");
     ep.relu = eh.relu;
     ep.mask_out = eh.mask_out;
     ep.mask_words = eh.mask_words;
@@ -832,7 +888,12 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
-    k_gemm_tc_k<<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
+    if (ep.lstm_h > 0)
+        k_gemm_tc_k<EPI_LSTM><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
+    else if (ep.resid_idx)
+        k_gemm_tc_k<EPI_RESID><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
+    else
+        k_gemm_tc_k<EPI_PLAIN><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }

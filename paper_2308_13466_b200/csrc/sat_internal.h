@@ -36,6 +36,11 @@ struct CacheLayer {
     float *S = nullptr;  // LSTM state table [n_slots x h]
     int32_t S_h = 0;
     bool S_valid = false;
+    // input projections x Wx + b of the ring buffers (gate-interleaved columns), reused while the caller's parameter
+    // version stays the same: [(tau+1) x n_slots x 4 proj_h]; proj_tag[i] = version the projection of buffer i was made with
+    float *proj = nullptr;
+    int32_t proj_h = 0;
+    std::vector<uint64_t> proj_tag;
 };
 
 // kernel families for the optional per-family device timing (sat_profile_*)
@@ -245,6 +250,9 @@ struct TcEpilogueHost {
     int32_t lstm_h = 0;
     int lstm_first = 0;                // first step: previous cell state is zero
     float *lstm_c = nullptr;
+    const float *addend = nullptr;     // dense [m x ld_addend], added to the accumulators before the LSTM cell (row-aligned)
+    int32_t ld_addend = 0;
+    int32_t pack_gate_h = 0;           // > 0: the bias is interleaved like weights packed with gate_h (without the LSTM epilogue)
 };
 // tensor-core path on / off for a contraction with n outputs and k terms (SAT_NO_TC=1 in the environment forces the CUDA cores)
 bool sat_use_tc(int32_t n, int32_t k);

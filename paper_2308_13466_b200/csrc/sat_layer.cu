@@ -62,6 +62,7 @@ extern "C" sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, cons
     for (int i = 0; i < SAT_MAX_LAYERS; ++i) {
         if (ctx->cache[i].buf) cudaFree(ctx->cache[i].buf);
         if (ctx->cache[i].S) cudaFree(ctx->cache[i].S);
+        if (ctx->cache[i].proj) cudaFree(ctx->cache[i].proj);
         ctx->cache[i] = CacheLayer();
     }
     ctx->cache_ok = false;
@@ -104,6 +105,7 @@ extern "C" sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer
     SAT_TRY(sat_part_view(ctx, part, &v));
     if (v.n_push == 0) return SAT_OK;
     if (!h_out || !ok_ld(ld, c->width) || !aligned16(h_out)) return sat_fail(ctx, SAT_EINVAL, "sat_cache_update: null / misaligned h_out or bad ld");
+    if (!c->proj_tag.empty()) c->proj_tag[ctx->write_idx] = 0;  // the buffer changes: its cached input projection is stale
     const float *src_base = h_out - (int64_t)v.row0 * ld;
     return sat_scatter(ctx, ctx->push_row + v.push0, ctx->push_slot + v.push0, v.n_push, c->width, src_base, ld,
                        ring_buf(ctx, c, ctx->write_idx), c->ld);
@@ -135,7 +137,10 @@ extern "C" sat_status sat_cache_set_state(sat_ctx *ctx, int32_t write_idx, int32
     if (write_idx < 0 || write_idx > ctx->tau || n_valid < 0 || n_valid > ctx->tau) return sat_fail(ctx, SAT_EINVAL, "sat_cache_set_state: out of range");
     ctx->write_idx = write_idx;
     ctx->n_valid = n_valid;
-    for (int i = 0; i < ctx->n_cached; ++i) ctx->cache[i].S_valid = false;
+    for (int i = 0; i < ctx->n_cached; ++i) {
+        ctx->cache[i].S_valid = false;
+        ctx->cache[i].proj_tag.assign(ctx->cache[i].proj_tag.size(), 0);
+    }
     return SAT_OK;
 }
 
@@ -175,6 +180,7 @@ extern "C" sat_status sat_cache_import(sat_ctx *ctx, int32_t layer, const float 
     if (!in_host) return sat_fail(ctx, SAT_EINVAL, "sat_cache_import: null input");
     const size_t rows = (size_t)(ctx->tau + 1) * ctx->n_slots;
     c->S_valid = false;
+    c->proj_tag.assign(c->proj_tag.size(), 0);
     if (rows == 0) return SAT_OK;
     SAT_CUDA(ctx, cudaMemcpy2DAsync(c->buf, (size_t)c->ld * 4, in_host, (size_t)c->width * 4, (size_t)c->width * 4, rows,
                                     cudaMemcpyHostToDevice, ctx->stream));
@@ -209,6 +215,72 @@ sat_status sat_gemm_nn_dual(sat_ctx *ctx, int64_t m, int32_t n, int32_t k1, cons
                             int32_t k2, const float *A2, int32_t lda2, const float *B2, int32_t ldb2, const float *bias, float *C,
                             int32_t ldc);
 
+// first LSTM step from a cached input projection (gate-interleaved columns 4 j + gate): previous state is zero
+__global__ void k_lstm_cell_first(const float *__restrict__ proj, int64_t rows, int32_t h, float *__restrict__ c, float *__restrict__ s)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * h) return;
+    const float4 a = __ldg(reinterpret_cast<const float4 *>(proj) + t);  // (i, f, g, o) of unit t % h of row t / h
+    const float gi = 1.f / (1.f + expf(-a.x));
+    const float gg = tanhf(a.z);
+    const float go = 1.f / (1.f + expf(-a.w));
+    const float cn = gi * gg;
+    c[t] = cn;
+    s[t] = go * tanhf(cn);
+}
+
+// LSTM with cached input projections (parameter version promised by the caller): only ring buffers whose projection is
+// missing or was made with another version are projected; the recurrence then contracts over h only.
+static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p, int32_t k, float *cell)
+{
+    const int32_t h = p->h, d = c->width;
+    const int64_t rows = ctx->n_slots;
+    const int64_t plane = rows * 4 * h;
+    if (!c->proj || c->proj_h != h) {
+        SAT_TRY(dev_realloc(ctx, &c->proj, (int64_t)(ctx->tau + 1) * plane));
+        c->proj_h = h;
+        c->proj_tag.assign(ctx->tau + 1, 0);
+    }
+    TcWeights Wp;
+    bool packed = false;
+    for (int32_t t = 0; t < k; ++t) {
+        const int32_t idx = ring_index(ctx, k - 1 - t);
+        if (c->proj_tag[idx] == p->version) continue;
+        if (!packed) {
+            SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
+            packed = true;
+        }
+        TcEpilogueHost eh;
+        eh.C = c->proj + (int64_t)idx * plane;
+        eh.ldc = 4 * h;
+        eh.bias = p->b;
+        eh.pack_gate_h = h;
+        SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+        c->proj_tag[idx] = p->version;
+    }
+    TcWeights Up;
+    if (k > 1) SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit2, &Up, h));
+    for (int32_t t = 0; t < k; ++t) {
+        const float *pr = c->proj + (int64_t)ring_index(ctx, k - 1 - t) * plane;  // oldest first
+        if (t == 0) {
+            ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 6.0, 0.0);
+            k_lstm_cell_first<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(pr, rows, h, cell, c->S);
+            SAT_LAUNCHED(ctx);
+        } else {
+            TcEpilogueHost eh;
+            eh.C = c->S;
+            eh.ldc = h;
+            eh.lstm_h = h;
+            eh.lstm_c = cell;
+            eh.addend = pr;
+            eh.ld_addend = 4 * h;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_NN));
+        }
+    }
+    c->S_valid = true;
+    return SAT_OK;
+}
+
 static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p)
 {
     const int32_t h = p->h, d = c->width;
@@ -231,6 +303,7 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
     // the cell update can be fused into the epilogue (s and c updated in place) when one tile spans all 4h gate columns:
     // then a tile reads only its own rows of s, and does so before its epilogue overwrites them
     const bool fused = tc && 4 * h <= 256;
+    if (fused && p->version != 0 && sat_use_tc(4 * h, h)) return run_lstm_cached(ctx, c, p, k, cell);
     TcWeights W1, W2;   // packed weights for the first step (x only) and the later steps ([x | s])
     if (tc) {
         SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &W1, fused ? h : 0));

@@ -49,14 +49,14 @@ def dev(a: np.ndarray, device="cuda"):
     return torch.from_numpy(np.ascontiguousarray(a)).to(device)
 
 
-def pred_to_device(pred_list, B):
+def pred_to_device(pred_list, B, version: int = 0):
     """Oracle-side predictor dicts -> list of sat_pred_params (device copies kept alive by the structs)."""
     out = []
     for p in pred_list:
         h = int(p["Wg"].shape[0])
         out.append(B.make_pred_params(dev(p["Wx"].astype(np.float32)), dev(p["Uh"].astype(np.float32)),
                                       dev(p["b"].astype(np.float32)), dev(p["Wg"].astype(np.float32)),
-                                      dev(p["bg"].astype(np.float32)), h))
+                                      dev(p["bg"].astype(np.float32)), h, version))
     return out
 
 

@@ -142,3 +142,48 @@ def test_cache_checkpoint_resume(B):
             assert np.array_equal(a, b_)
     finally:
         ep2.close()
+
+
+def test_cached_input_projections_over_a_wrapping_ring(B):
+    """Predictor parameters with a version promise: the library keeps x Wx + b per cached snapshot and projects only new
+    snapshots.  Free-running epochs (no re-synchronisation, fixed weights) until the ring has wrapped twice; the LSTM state,
+    the layer outputs and the ring must still match the oracle running the same epochs, and the versioned and unversioned
+    paths must agree."""
+    import torch
+    wl = make_workload("medium", shrink=16)
+    Wd = [dev(w) for w in wl.W]
+    bd = [dev(x) for x in wl.b]
+    n_epochs = 2 * (wl.tau + 1) + 1
+    outs = {}
+    for version in (0, 9):
+        preds = pred_to_device(wl.pred, B, version)
+        ep, P, dtil, perm = _setup(B, wl)
+        try:
+            for _ in range(n_epochs):
+                ep.step(Wd, bd, preds)
+            torch.cuda.synchronize()
+            # the LSTM state of the ring as the next epoch would see it (the commit dropped the one the epochs used)
+            S = []
+            for l in range(1, wl.L):
+                halo0 = torch.empty((P.halo_gid[0].shape[0], wl.dims[l]), dtype=torch.float32, device="cuda")
+                B.sat_predict(ep.ctx, l, 0, preds[l - 1], 0, halo0)
+                S.append(B.sat_predict_state(ep.ctx, l, P.n_slots, wl.pred[l - 1]["h"]))
+            outs[version] = dict(H=[h.cpu().numpy().copy() for h in ep.H[1:]], S=S,
+                                 ring=[B.sat_cache_export(ep.ctx, l, wl.tau, P.n_slots, wl.dims[l]) for l in range(1, wl.L)],
+                                 state=B.sat_cache_state(ep.ctx))
+        finally:
+            ep.close()
+    cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
+    for _ in range(n_epochs):
+        res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=False)
+    for version in (0, 9):
+        o = outs[version]
+        assert o["state"] == (cache.write_idx, cache.n_valid)
+        for l in range(1, wl.L):
+            pr = wl.pred[l - 1]
+            S_want = orc.lstm_state(cache.snapshots(l), wl.dims[l], pr["h"], pr["Wx"], pr["Uh"], pr["b"], P.n_slots)
+            assert_close(o["S"][l - 1], S_want, f"version {version}: LSTM state of layer {l} after {n_epochs} epochs")
+            newest = (cache.write_idx - 1) % (wl.tau + 1)
+            assert_close(o["ring"][l - 1][newest], cache.buf[l - 1][newest], f"version {version}: newest snapshot of layer {l}")
+        for l in range(1, wl.L + 1):
+            assert_close(o["H"][l - 1], _gather_H(res, P, l), f"version {version}: H^{l} after {n_epochs} epochs")
