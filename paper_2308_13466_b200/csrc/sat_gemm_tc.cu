@@ -36,7 +36,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-// bounded wait: returns false (and raises *dead) when the limit is hit or another thread already gave up
+// bounded wait: returns false (and raises *dead) when the limit is hit or another thread already gave up.
+// SLEEP_NS > 0 backs off between polls: a spinning warp otherwise takes issue slots from the warps doing the work
+// (the epilogue shares its schedulers with the waiting converter warps).
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *dead, int *status)
 {
     const uint32_t addr = smem_u32(bar);
@@ -53,6 +56,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
             : "memory");
         if (ok) return true;
         if (*dead) return false;
+        if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     }
     *dead = 1;
     atomicOr(status, 1);
@@ -63,7 +67,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *dead, int *status, int lane)
 {
     int ok = 1;
-    if (lane == 0) ok = mbar_wait(bar, parity, dead, status) ? 1 : 0;
+    if (lane == 0) ok = mbar_wait<64>(bar, parity, dead, status) ? 1 : 0;
     ok = __shfl_sync(0xffffffffu, ok, 0);
     if (!ok) return false;
     return mbar_wait(bar, parity, dead, status);
@@ -147,38 +151,28 @@ __host__ __device__ inline uint32_t make_idesc(int n, int a_mn_major, int b_mn_m
 }
 
 // =====================================================================================
-// TF32 split of a shared-memory tile, element-wise: hi = tf32(x) in place, lo = tf32(x - hi) at the same offset
+// TF32 split of a shared-memory tile, element-wise.  The tensor core reads an fp32 container as TF32 by ignoring the low
+// 13 mantissa bits, so the raw tile already is the "hi" operand (hi = x with those bits cleared); only the residual
+// lo = x - hi (exact in fp32, again truncated by the tensor core when read) has to be written, at the same offset of the
+// second tile.  |x - hi - tf32(lo)| < 2^-20 |x|.
 // =====================================================================================
-__device__ __forceinline__ float tf32_round(float x)
+__device__ __forceinline__ float tf32_residual(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ float4 residual4(const float4 &x)
 {
-    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);  // round half away from zero to 10 mantissa bits
-}
-__device__ __forceinline__ void split4(const float4 &x, float4 &h, float4 &l)
-{
-    h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
-    h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
-    h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
-    h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
+    return make_float4(tf32_residual(x.x), tf32_residual(x.y), tf32_residual(x.z), tf32_residual(x.w));
 }
 // two 16-byte chunks per thread and iteration, loads first (the loop is latency-bound otherwise)
-__device__ __forceinline__ void split_tile(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
+__device__ __forceinline__ void split_tile(const uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
 {
     const uint32_t step = (uint32_t)nthreads * 16;
     for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += 2 * step) {
         const uint32_t off2 = off + step;
         const bool two = off2 < bytes;
-        const float4 x1 = *reinterpret_cast<float4 *>(hi_tile + off);
+        const float4 x1 = *reinterpret_cast<const float4 *>(hi_tile + off);
         float4 x2 = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (two) x2 = *reinterpret_cast<float4 *>(hi_tile + off2);
-        float4 h1, l1, h2, l2;
-        split4(x1, h1, l1);
-        split4(x2, h2, l2);
-        *reinterpret_cast<float4 *>(hi_tile + off) = h1;
-        *reinterpret_cast<float4 *>(lo_tile + off) = l1;
-        if (two) {
-            *reinterpret_cast<float4 *>(hi_tile + off2) = h2;
-            *reinterpret_cast<float4 *>(lo_tile + off2) = l2;
-        }
+        if (two) x2 = *reinterpret_cast<const float4 *>(hi_tile + off2);
+        *reinterpret_cast<float4 *>(lo_tile + off) = residual4(x1);
+        if (two) *reinterpret_cast<float4 *>(lo_tile + off2) = residual4(x2);
     }
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
@@ -237,12 +231,28 @@ struct TcShared {
 #define TCK_EPI_THREADS (TCK_EPI_WARPS * 32)
 #define TCK_EPI_WARP0 (2 + TCK_CONV_WARPS)
 #define TCK_THREADS (64 + TCK_CONV_THREADS + TCK_EPI_THREADS) /* warp 0 TMA, warp 1 MMA, then the converter warps, then the epilogue warps: 512 threads, 128 registers each */
-#define TCK_STAGES 4
 #define TCK_OUT_BYTES (TCK_EPI_WARPS * 4096)  /* per epilogue warp one 32 x 32 fp32 staging tile for the TMA stores */
 
-enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2 };
+// Epilogue variants.  The ones with a per-row side operand streamed from global memory (gathered residual rows, cached
+// LSTM input projection) keep a ring of 32 x 32 side tiles per epilogue warp in shared memory, filled by cp.async several
+// chunks ahead: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
+// small K (the predictor width), so they give up main-loop stages for the ring.
+enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3 };
+template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, out_bytes = TCK_OUT_BYTES; };
+template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 3, out_bytes = TCK_OUT_BYTES; };
+template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, out_bytes = 0; };
+template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 4, out_bytes = 0; };
 
-// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of TCK_STAGES k-blocks
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, bool valid)
+{
+    // src-size 0 writes 16 zero bytes without reading the source
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(valid ? 16u : 0u) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of k-block stages
 // and the two TMEM accumulator buffers let the TMA loads, the TF32 split, the MMAs and the epilogue of consecutive tiles
 // overlap.  A and B arrive as raw fp32 tiles; the converters round them to TF32 in place and write the residual tiles.
 // The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell) and runs on eight
@@ -258,14 +268,17 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     const uint32_t a_bytes = TC_BM * TC_BK * 4;  // one plane of the A tile: 128 rows x 64 B
     const uint32_t b_bytes = (uint32_t)bn * TC_BK * 4;
     const uint32_t stage_bytes = 2 * a_bytes + 2 * b_bytes;  // [A hi | A lo | B hi | B lo]
-    uint8_t *out_stage = smem + (size_t)TCK_STAGES * stage_bytes;
-    TcShared *sh = (TcShared *)(out_stage + TCK_OUT_BYTES);
+    constexpr int STAGES = TckCfg<EPI>::stages;
+    constexpr int RING = TckCfg<EPI>::ring;
+    uint8_t *out_stage = smem + (size_t)STAGES * stage_bytes;
+    uint8_t *ring_base = out_stage + TckCfg<EPI>::out_bytes;
+    TcShared *sh = (TcShared *)(ring_base + (size_t)TCK_EPI_WARPS * RING * 4096);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int32_t nkb = nkb1 + nkb2;
     const uint32_t acc_cols = 256;  // column stride between the two accumulator buffers
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < TCK_STAGES; ++s) {
+        for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sh->full[s], 1);
             mbar_init(&sh->conv[s], TCK_CONV_THREADS);
             mbar_init(&sh->empty[s], 1);
@@ -295,8 +308,8 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const int32_t m0 = (int32_t)(t / n_tiles_n) * TC_BM;
                 const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
                 for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % TCK_STAGES;
-                    const uint32_t ph = (it / TCK_STAGES) & 1u;
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) goto done;
                     uint8_t *st = smem + (size_t)s * stage_bytes;
                     mbar_expect_tx(&sh->full[s], a_bytes + b_bytes);
@@ -317,8 +330,8 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 tc_fence_after();
                 const uint32_t acc = tmem + buf * acc_cols;
                 for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
-                    const int s = it % TCK_STAGES;
-                    const uint32_t ph = (it / TCK_STAGES) & 1u;
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
                     if (!mbar_wait(&sh->conv[s], ph, dead, status)) goto done;
                     tc_fence_after();
@@ -345,8 +358,8 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         uint32_t it = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
             for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
-                const int s = it % TCK_STAGES;
-                const uint32_t ph = (it / TCK_STAGES) & 1u;
+                const int s = it % STAGES;
+                const uint32_t ph = (it / STAGES) & 1u;
                 if (!mbar_wait_warp(&sh->full[s], ph, dead, status, lane)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 split_tile(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
@@ -358,16 +371,82 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     } else {
         // ---------------- epilogue ----------------
         // warp w reads TMEM lanes 32 (w % 4) .. +31 = rows of the tile, one row per thread; the two warps of a lane quadrant
-        // take alternate 32-column chunks.  Per-row side operands (gathered residual row, cached projection, previous cell
-        // state) are latency-bound loads: they are issued one chunk ahead, the first chunk's before the accumulator is ready.
+        // take alternate 32-column chunks.
+        constexpr bool LSTM = EPI == EPI_LSTM || EPI == EPI_LSTM_ADD;
         const int e = warp - TCK_EPI_WARP0;
         const int q = warp & 3;
         const int c_first = 32 * (e >> 2);
         uint8_t *obuf = out_stage + e * 4096;
         const bool vec = ((ep.ldc & 3) == 0) && ((((uintptr_t)ep.C) & 15u) == 0);
         const int32_t n4 = (N + 3) & ~3;
-        const bool lstm_full = EPI == EPI_LSTM && (ep.lstm_h & 3) == 0;
+        const bool lstm_full = LSTM && (ep.lstm_h & 3) == 0;
         const float4 zero4 = make_float4(0.f, 0.f, 0.f, 0.f);
+
+        // Side-operand ring (RING slots of 32 rows x 128 B, 128-byte swizzle like the store staging tile), private to the
+        // warp: cp.async group counting plus __syncwarp is all the synchronisation needed.  The prefetch cursor (pf_*)
+        // walks this warp's (tile, chunk) sequence RING chunks ahead of the consumer.
+        uint8_t *ring = ring_base + (size_t)e * RING * 4096;
+        int64_t pf_t = blockIdx.x;
+        int pf_c = c_first;
+        const float *pf_srow = nullptr;
+        int32_t pf_lim = 0;
+        int32_t pf_idx_next = -1;   // (gathered residual) row index for the tile after the cursor's, fetched a tile early
+        uint32_t pf_slot = 0, rd_slot = 0;
+        auto pf_enter_tile = [&](int32_t idx_now) {
+            // called when the cursor enters tile pf_t; idx_now = gathered row index for this thread's row, or -1
+            pf_srow = nullptr;
+            if (pf_t < n_tiles) {
+                const int64_t prow = (pf_t / n_tiles_n) * TC_BM + q * 32 + lane;
+                const int32_t pn0 = (int32_t)(pf_t % n_tiles_n) * bn;
+                if (EPI == EPI_RESID) {
+                    if (prow < M && idx_now >= 0) pf_srow = ep.resid + (int64_t)idx_now * ep.ld_resid + pn0;  // rows padded to 4 floats
+                    pf_lim = n4 - pn0;
+                    const int64_t nt = pf_t + gridDim.x;
+                    const int64_t nrow = (nt / n_tiles_n) * TC_BM + q * 32 + lane;
+                    pf_idx_next = (nt < n_tiles && nrow < M) ? __ldg(ep.resid_idx + nrow) : -1;
+                } else {
+                    if (prow < M) pf_srow = ep.addend + prow * ep.ld_addend + pn0;
+                    pf_lim = N - pn0;
+                }
+            }
+        };
+        auto pf_issue = [&]() {
+            // one group per call (possibly empty), so that the consumer's wait count is uniform.  Lane L copies 16-byte
+            // piece (L & 7) of rows (L >> 3) + 4 i: an instruction touches 4 rows (4 cache lines) instead of 32, which
+            // matters because the load/store unit handles one line per cycle.
+            if (pf_t < n_tiles && pf_c < bn) {
+                uint8_t *slot = ring + pf_slot * 4096;
+                const float *base = EPI == EPI_RESID ? ep.resid : ep.addend;
+                const int piece = lane & 7;
+                const bool col_ok = pf_c + 4 * piece < pf_lim;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int rr = (lane >> 3) + 4 * i;
+                    const float *rowp = reinterpret_cast<const float *>(__shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)pf_srow, rr));
+                    const bool valid = rowp != nullptr && col_ok;
+                    cp_async16(slot + rr * 128 + ((piece ^ (rr & 7)) << 4), (valid ? rowp : base) + pf_c + 4 * piece, valid);
+                }
+                pf_c += 64;
+                if (pf_c >= bn) {
+                    pf_c = c_first;
+                    pf_t += gridDim.x;
+                    pf_enter_tile(pf_idx_next);
+                }
+            }
+            cp_async_commit();
+            pf_slot = pf_slot + 1 == RING ? 0 : pf_slot + 1;
+        };
+        if (RING > 0 && c_first < bn) {
+            int32_t idx0 = -1;
+            if (EPI == EPI_RESID && pf_t < n_tiles) {
+                const int64_t prow = (pf_t / n_tiles_n) * TC_BM + q * 32 + lane;
+                if (prow < M) idx0 = __ldg(ep.resid_idx + prow);
+            }
+            pf_enter_tile(idx0);
+#pragma unroll
+            for (int i = 0; i < RING; ++i) pf_issue();
+        }
+
         uint32_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
             const int64_t m0 = (t / n_tiles_n) * TC_BM;
@@ -376,20 +455,10 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             const int64_t row = m0 + q * 32 + lane;
             const bool row_ok = row < M;
             float *crow = ep.C + row * ep.ldc;
-            const float *srow = nullptr;  // this thread's row of the side operand, at column n0
-            if (row_ok) {
-                if (EPI == EPI_RESID) srow = ep.resid + (int64_t)ep.resid_idx[row] * ep.ld_resid + n0;  // rows padded to 4 floats
-                if (EPI == EPI_LSTM && ep.addend) srow = ep.addend + row * ep.ld_addend + n0;
-            }
-            const int32_t side_lim = (EPI == EPI_RESID ? n4 : N) - n0;
             float4 side[8], cside[2];
-            auto load_side = [&](int c0) {
-                if (EPI != EPI_PLAIN) {
-#pragma unroll
-                    for (int u = 0; u < 8; ++u)
-                        side[u] = (srow && c0 + 4 * u < side_lim) ? __ldg(reinterpret_cast<const float4 *>(srow + c0) + u) : zero4;
-                }
-                if (EPI == EPI_LSTM) {
+            // previous cell state of the next chunk, fetched one chunk ahead (two 128-bit loads per thread)
+            auto load_cell = [&](int c0) {
+                if (LSTM) {
                     cside[0] = cside[1] = zero4;
                     const int32_t j0 = (n0 + c0) >> 2;
                     if (row_ok && lstm_full && !ep.lstm_first && j0 + 7 < ep.lstm_h) {
@@ -398,20 +467,30 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     }
                 }
             };
-            if (c_first < bn) load_side(c_first);
+            if (c_first < bn) load_cell(c_first);
             if (!mbar_wait_warp(&sh->acc_full[buf], (lt >> 1) & 1u, dead, status, lane)) goto done;
             tc_fence_after();
             for (int c0 = c_first; c0 < bn; c0 += 64) {
                 uint32_t r[32];
                 tc_ld32(tmem + buf * acc_cols + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                if (EPI == EPI_LSTM) {
+                if (RING > 0) {
+                    cp_async_wait<(RING > 0 ? RING - 1 : 0)>();  // every lane's copies of the oldest chunk in the ring have landed ...
+                    __syncwarp();                                // ... and are visible to the lane that owns the row
+                    const uint8_t *src = ring + rd_slot * 4096 + lane * 128;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) side[u] = *reinterpret_cast<const float4 *>(src + ((u ^ (lane & 7)) << 4));
+                    rd_slot = rd_slot + 1 == RING ? 0 : rd_slot + 1;
+                    __syncwarp();  // all lanes have read the slot: refill it with the chunk RING steps ahead
+                    pf_issue();
+                }
+                if (LSTM) {
                     // packed columns 4 j .. 4 j + 3 are the (i, f, g, o) pre-activations of hidden unit j
                     if (row_ok) {
                         const int32_t j0 = (n0 + c0) >> 2;
                         const bool full = lstm_full && j0 + 7 < ep.lstm_h;
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
-                            float4 b4 = side[u];
+                            float4 b4 = EPI == EPI_LSTM_ADD ? side[u] : zero4;
                             if (ep.bias) {
                                 const float4 bb = __ldg(reinterpret_cast<const float4 *>(ep.bias + n0 + c0) + u);
                                 b4.x += bb.x; b4.y += bb.y; b4.z += bb.z; b4.w += bb.w;
@@ -429,7 +508,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                             for (int u = 0; u < 8; ++u)
                                 if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[row * ep.lstm_h + j0 + u];
                         }
-                        if (c0 + 64 < bn) load_side(c0 + 64);
+                        if (c0 + 64 < bn) load_cell(c0 + 64);
                         float sv[8], cv[8];
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
@@ -474,7 +553,6 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + b4.z);
                         r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + b4.w);
                     }
-                    if (EPI == EPI_RESID && c0 + 64 < bn) load_side(c0 + 64);
                     if (EPI == EPI_PLAIN && ep.mask_out) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
@@ -518,6 +596,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             mbar_arrive(&sh->acc_empty[buf]);  // the accumulator buffer may be overwritten by the tile after next
         }
         if (use_tma_store && lane == 0) tma_store_wait_all();
+        if (RING > 0) cp_async_wait<0>();
     }
 done:
     tc_fence_before();
@@ -829,8 +908,35 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
     return SAT_OK;
 }
 
-static bool g_attr_k = false, g_attr_mn = false;
+static bool g_attr_mn = false;
 #define TC_SMEM_BUDGET (100 * 1024)
+
+struct TckLaunch {
+    CUtensorMap mA, mA2, mB, mC;
+    int use_tma_store;
+    int64_t m;
+    int32_t n, nkb1, nkb2, bn, n_tiles_n;
+    int64_t n_tiles;
+    unsigned grid;
+    uint32_t stage_bytes;
+};
+
+template <int EPI>
+static sat_status launch_tck(sat_ctx *ctx, const TckLaunch &L, const TcEpilogue &ep)
+{
+    static bool attr_set = false;
+    const size_t smem = (size_t)TckCfg<EPI>::stages * L.stage_bytes + TckCfg<EPI>::out_bytes + (size_t)TCK_EPI_WARPS * TckCfg<EPI>::ring * 4096 +
+                        sizeof(TcShared) + 1024;
+    if (smem > 227 * 1024) return sat_fail(ctx, SAT_EINVAL, "tensor-core GEMM: shared-memory layout of %zu bytes does not fit", smem);
+    if (!attr_set) {
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    k_gemm_tc_k<EPI><<<L.grid, TCK_THREADS, smem, ctx->stream>>>(L.mA, L.mA2, L.mB, L.mC, L.use_tma_store, L.m, L.n, L.nkb1, L.nkb2, L.bn, L.n_tiles_n,
+                                                                L.n_tiles, ep, ctx->d_flag + 1);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
 
 // C[m x n] = [A | A2] B^T with B = packed weights [n_pad x k_pad]
 sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
@@ -840,7 +946,6 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     const int32_t nkb1 = (k1 + TC_BK - 1) / TC_BK, nkb2 = A2 ? (k2 + TC_BK - 1) / TC_BK : 0;
     const int32_t bn = tile_n_for(n);
     const uint32_t stage_bytes = 2 * (TC_BM * TC_BK * 4) + 2 * (uint32_t)bn * TC_BK * 4;
-    const size_t smem = (size_t)TCK_STAGES * stage_bytes + TCK_OUT_BYTES + sizeof(TcShared) + 1024;
     ProfScope prof(ctx, family, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
     CUtensorMap mA, mA2, mB, mC;
     const int use_tma_store = eh.lstm_h == 0 && ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
@@ -850,12 +955,6 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     if (A2) SAT_TRY(make_map(ctx, &mA2, A2, k2, m, lda2, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
     else mA2 = mA;
     SAT_TRY(make_map(ctx, &mB, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
-    if (!g_attr_k) {
-        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_RESID>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI_LSTM>, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024));
-        g_attr_k = true;
-    }
     TcEpilogue ep;
     ep.C = eh.C;
     ep.ldc = eh.ldc;
@@ -888,14 +987,15 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     int sms = 148;
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
-    if (ep.lstm_h > 0)
-        k_gemm_tc_k<EPI_LSTM><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
-    else if (ep.resid_idx)
-        k_gemm_tc_k<EPI_RESID><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
-    else
-        k_gemm_tc_k<EPI_PLAIN><<<grid, TCK_THREADS, smem, ctx->stream>>>(mA, mA2, mB, mC, use_tma_store, m, n, nkb1, nkb2, bn, n_tiles_n, n_tiles, ep, ctx->d_flag + 1);
-    SAT_LAUNCHED(ctx);
-    return SAT_OK;
+    TckLaunch L;
+    L.mA = mA; L.mA2 = mA2; L.mB = mB; L.mC = mC;
+    L.use_tma_store = use_tma_store;
+    L.m = m; L.n = n; L.nkb1 = nkb1; L.nkb2 = nkb2; L.bn = bn; L.n_tiles_n = n_tiles_n; L.n_tiles = n_tiles;
+    L.grid = grid;
+    L.stage_bytes = stage_bytes;
+    if (ep.lstm_h > 0) return ep.addend ? launch_tck<EPI_LSTM_ADD>(ctx, L, ep) : launch_tck<EPI_LSTM>(ctx, L, ep);
+    if (ep.resid_idx) return launch_tck<EPI_RESID>(ctx, L, ep);
+    return launch_tck<EPI_PLAIN>(ctx, L, ep);
 }
 
 // C[m x n] (+)= A^T B over `rows` rows: A fp32 [rows x m] (lda), B fp32 [rows x n] (ldb)
