@@ -584,49 +584,121 @@ extern "C" sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_
 // loss seed, parameter step
 // =====================================================================================
 // one warp per row
-__global__ void k_loss_ce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const int32_t *__restrict__ y, float scale,
-                          float *__restrict__ g, int64_t ld_g, float *__restrict__ row_loss)
-{
-    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (r >= rows) return;
-    const float *zr = z + r * ld_z;
-    float mx = -INFINITY;
-    for (int c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
-    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float se = 0.f;
-    for (int c = lane; c < C; c += 32) se += expf(zr[c] - mx);
-    for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
-    const float lse = mx + logf(se);
-    const int32_t yr = y[r];
-    for (int c = lane; c < C; c += 32) g[r * ld_g + c] = scale * (expf(zr[c] - lse) - (c == yr ? 1.f : 0.f));
-    if (lane == 0) row_loss[r] = scale * (lse - zr[yr]);
-}
+// Loss kernels: one warp per row, LOSS_ROWS_PER_BLOCK consecutive rows per block (each warp walks its share in order).
+// The row losses are summed in double per warp, the warps of a block in fixed order, and k_loss_sum adds the block
+// partials in fixed order: the total does not depend on scheduling.
+#define LOSS_ROWS_PER_BLOCK 256
 
-__global__ void k_loss_bce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const uint8_t *__restrict__ y, float scale,
-                           float *__restrict__ g, int64_t ld_g, float *__restrict__ row_loss)
+__device__ __forceinline__ void loss_block_partial(double warp_sum, double *__restrict__ block_partial)
 {
-    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (r >= rows) return;
-    const float *zr = z + r * ld_z;
-    const float inv_c = 1.f / (float)C;
-    float acc = 0.f;
-    for (int c = lane; c < C; c += 32) {
-        const float x = zr[c], yv = (float)y[r * C + c];
-        acc += fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))) - yv * x;
-        g[r * ld_g + c] = scale * inv_c * (1.f / (1.f + expf(-x)) - yv);
+    __shared__ double red[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) red[warp] = warp_sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double s = 0.0;
+        for (int w = 0; w < 8; ++w) s += red[w];
+        block_partial[blockIdx.x] = s;
     }
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) row_loss[r] = scale * inv_c * acc;
 }
 
-// single block, fixed order: *total += sum(row_loss)
-__global__ void k_loss_sum(const float *__restrict__ row_loss, int64_t rows, double *total)
+// softmax cross-entropy: the row (up to 32 CPL classes) is held in registers, one exponential per class
+template <int CPL>
+__global__ void __launch_bounds__(256)
+k_loss_ce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const int32_t *__restrict__ y, float scale,
+          float *__restrict__ g, int64_t ld_g, double *__restrict__ block_partial)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t r0 = (int64_t)blockIdx.x * LOSS_ROWS_PER_BLOCK;
+    double acc = 0.0;
+    for (int i = warp; i < LOSS_ROWS_PER_BLOCK; i += 8) {
+        const int64_t r = r0 + i;
+        if (r >= rows) break;
+        const float *zr = z + r * ld_z;
+        float v[CPL];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+            const int c = lane + 32 * j;
+            v[j] = c < C ? zr[c] : -INFINITY;
+            mx = fmaxf(mx, v[j]);
+        }
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+            v[j] = lane + 32 * j < C ? expf(v[j] - mx) : 0.f;
+            se += v[j];
+        }
+        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float inv = 1.f / se;
+        const int32_t yr = y[r];
+#pragma unroll
+        for (int j = 0; j < CPL; ++j) {
+            const int c = lane + 32 * j;
+            if (c < C) g[r * ld_g + c] = scale * (v[j] * inv - (c == yr ? 1.f : 0.f));
+        }
+        if (lane == 0) acc += (double)(scale * (mx + logf(se) - zr[yr]));
+    }
+    loss_block_partial(acc, block_partial);
+}
+
+// any number of classes: three passes over the row
+__global__ void __launch_bounds__(256)
+k_loss_ce_wide(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const int32_t *__restrict__ y, float scale,
+               float *__restrict__ g, int64_t ld_g, double *__restrict__ block_partial)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t r0 = (int64_t)blockIdx.x * LOSS_ROWS_PER_BLOCK;
+    double acc = 0.0;
+    for (int i = warp; i < LOSS_ROWS_PER_BLOCK; i += 8) {
+        const int64_t r = r0 + i;
+        if (r >= rows) break;
+        const float *zr = z + r * ld_z;
+        float mx = -INFINITY;
+        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, zr[c]);
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float se = 0.f;
+        for (int c = lane; c < C; c += 32) se += expf(zr[c] - mx);
+        for (int o = 16; o > 0; o >>= 1) se += __shfl_xor_sync(0xffffffffu, se, o);
+        const float inv = 1.f / se;
+        const int32_t yr = y[r];
+        for (int c = lane; c < C; c += 32) g[r * ld_g + c] = scale * (expf(zr[c] - mx) * inv - (c == yr ? 1.f : 0.f));
+        if (lane == 0) acc += (double)(scale * (mx + logf(se) - zr[yr]));
+    }
+    loss_block_partial(acc, block_partial);
+}
+
+__global__ void __launch_bounds__(256)
+k_loss_bce(int64_t rows, int32_t C, const float *__restrict__ z, int64_t ld_z, const uint8_t *__restrict__ y, float scale,
+           float *__restrict__ g, int64_t ld_g, double *__restrict__ block_partial)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t r0 = (int64_t)blockIdx.x * LOSS_ROWS_PER_BLOCK;
+    const float inv_c = 1.f / (float)C;
+    double acc = 0.0;
+    for (int i = warp; i < LOSS_ROWS_PER_BLOCK; i += 8) {
+        const int64_t r = r0 + i;
+        if (r >= rows) break;
+        const float *zr = z + r * ld_z;
+        float a = 0.f;
+        for (int c = lane; c < C; c += 32) {
+            const float x = zr[c], yv = (float)y[r * C + c];
+            a += fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))) - yv * x;
+            g[r * ld_g + c] = scale * inv_c * (1.f / (1.f + expf(-x)) - yv);
+        }
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) acc += (double)(scale * inv_c * a);
+    }
+    loss_block_partial(acc, block_partial);
+}
+
+// single block, fixed order: *total += sum(block_partial)
+__global__ void k_loss_sum(const double *__restrict__ block_partial, int64_t count, double *total)
 {
     __shared__ double red[256];
     double s = 0.0;
-    for (int64_t i = threadIdx.x; i < rows; i += 256) s += (double)row_loss[i];
+    for (int64_t i = threadIdx.x; i < count; i += 256) s += block_partial[i];
     red[threadIdx.x] = s;
     __syncthreads();
     for (int o = 128; o > 0; o >>= 1) {
@@ -645,18 +717,23 @@ extern "C" sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_
     if (kind != SAT_LOSS_SOFTMAX_CE && kind != SAT_LOSS_SIGMOID_BCE) return sat_fail(ctx, SAT_EINVAL, "sat_loss_grad: unknown loss");
     if (v.n_rows == 0) return SAT_OK;
     if (n_classes <= 0 || !z || !labels || !g || ld_z < n_classes || ld_g < n_classes) return sat_fail(ctx, SAT_EINVAL, "sat_loss_grad: null tensor or bad shape");
-    SAT_TRY(sat_ensure(ctx, ctx->buf_misc, (size_t)v.n_rows * sizeof(float)));
-    float *row_loss = (float *)ctx->buf_misc.p;
+    const unsigned blocks = (unsigned)cdiv64(v.n_rows, LOSS_ROWS_PER_BLOCK);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_misc, (size_t)blocks * sizeof(double)));
+    double *block_partial = (double *)ctx->buf_misc.p;
     const float scale = 1.0f / (float)ctx->n;
     ProfScope prof(ctx, SATK_LOSS, 8.0 * (double)v.n_rows * n_classes, 0.0);
-    const unsigned blocks = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
-    if (kind == SAT_LOSS_SOFTMAX_CE)
-        k_loss_ce<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, (const int32_t *)labels, scale, g, ld_g, row_loss);
-    else
-        k_loss_bce<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, (const uint8_t *)labels, scale, g, ld_g, row_loss);
+    if (kind == SAT_LOSS_SOFTMAX_CE) {
+        const int32_t *yl = (const int32_t *)labels;
+        if (n_classes <= 32) k_loss_ce<1><<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, yl, scale, g, ld_g, block_partial);
+        else if (n_classes <= 64) k_loss_ce<2><<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, yl, scale, g, ld_g, block_partial);
+        else if (n_classes <= 128) k_loss_ce<4><<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, yl, scale, g, ld_g, block_partial);
+        else k_loss_ce_wide<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, yl, scale, g, ld_g, block_partial);
+    } else {
+        k_loss_bce<<<blocks, 256, 0, ctx->stream>>>(v.n_rows, n_classes, z, ld_z, (const uint8_t *)labels, scale, g, ld_g, block_partial);
+    }
     SAT_LAUNCHED(ctx);
     if (loss_sum) {
-        k_loss_sum<<<1, 256, 0, ctx->stream>>>(row_loss, v.n_rows, loss_sum);
+        k_loss_sum<<<1, 256, 0, ctx->stream>>>(block_partial, (int64_t)blocks, loss_sum);
         SAT_LAUNCHED(ctx);
     }
     return SAT_OK;

@@ -167,77 +167,20 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
 // Used for the predictor's graph convolution on the LSTM state (self term, by slot) and for
 // the optional halo gradient P_out^T G_AGG (no self term, by row).
 // -------------------------------------------------------------------------------------
-template <int G, int NV>
-__global__ void __launch_bounds__(256)
-k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
-            const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
-            int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
-            float *__restrict__ out_base, int64_t ld_out)
-{
-    const int lane = threadIdx.x & (G - 1);
-    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
-    if (gid >= n_halo) return;
-    const unsigned mask = group_mask<G>(threadIdx.x & 31);
-    const int col0 = blockIdx.y * (G * NV);
-    const int64_t j = halo0 + gid;
-    const float du = __ldg(dinv_enc + n + j);
-    float4 acc[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (self_src) {
-        const float *src = self_src + (int64_t)halo_slot[j] * ld_src;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int idx = col0 + lane + v * G;
-            if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
-        }
-    }
-    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
-    if (e1 - e0 > SAT_HROW_LONG) return;  // handled by k_spmm_hrow_long
-    for (int64_t eb = e0; eb < e1; eb += G) {
-        const int64_t e = eb + lane;
-        int32_t c = 0;
-        float w = 0.f;
-        if (e < e1) {
-            const int32_t p = __ldg(hrow_pos + e);
-            w = __ldg(dinv_enc + p);
-            c = by_slot ? __ldg(hrow_slot + e) : p;
-        }
-        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
-#pragma unroll 4
-        for (int q = 0; q < cnt; ++q) {
-            const int32_t cj = __shfl_sync(mask, c, q, G);
-            const float wj = __shfl_sync(mask, w, q, G);
-            const float *src = src_base + (int64_t)cj * ld_src;
-#pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                const int idx = col0 + lane + v * G;
-                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
-            }
-        }
-    }
-    float *o = out_base + j * ld_out;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int idx = col0 + lane + v * G;
-        if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(du * acc[v].x, du * acc[v].y, du * acc[v].z, du * acc[v].w);
-    }
-}
-
-// One thread block per long halo row: the 256 / G lane groups take the entries round-robin, their partial sums are added
+// One thread block per long halo row (the first blocks of the grid, so that they start first and the short rows fill the
+// other SMs meanwhile): the 256 / G lane groups take the entries round-robin, their partial sums are added
 // in group order through shared memory (fixed order: reproducible), group 0 adds the self term and stores.
 template <int G, int NV>
-__global__ void __launch_bounds__(256)
-k_spmm_hrow_long(const int32_t *__restrict__ hlong, int32_t hlong0, const int64_t *__restrict__ hrow_ptr,
-                 const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot, const int32_t *__restrict__ halo_slot,
-                 const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src,
-                 const float *__restrict__ self_src, float *__restrict__ out_base, int64_t ld_out)
+__device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos,
+                                                const int32_t *__restrict__ hrow_slot, const int32_t *__restrict__ halo_slot,
+                                                const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4,
+                                                const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
+                                                float *__restrict__ out_base, int64_t ld_out)
 {
     constexpr int NG = 256 / G;
     __shared__ float4 red[NG][G * NV];
     const int lane = threadIdx.x & (G - 1), grp = threadIdx.x / G;
     const int col0 = blockIdx.y * (G * NV);
-    const int64_t j = hlong[hlong0 + blockIdx.x];
     const float du = __ldg(dinv_enc + n + j);
     float4 acc[NV];
 #pragma unroll
@@ -274,19 +217,75 @@ k_spmm_hrow_long(const int32_t *__restrict__ hlong, int32_t hlong0, const int64_
 }
 
 template <int G, int NV>
+__global__ void __launch_bounds__(256)
+k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
+            const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
+            int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
+            float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong)
+{
+    if ((int32_t)blockIdx.x < n_hlong) {
+        hrow_long_block<G, NV>(hlong[hlong0 + blockIdx.x], hrow_ptr, hrow_pos, hrow_slot, halo_slot, dinv_enc, n, by_slot, d4, src_base, ld_src,
+                               self_src, out_base, ld_out);
+        return;
+    }
+    const int lane = threadIdx.x & (G - 1);
+    const int64_t gid = ((int64_t)(blockIdx.x - n_hlong) * blockDim.x + threadIdx.x) / G;
+    if (gid >= n_halo) return;
+    const unsigned mask = group_mask<G>(threadIdx.x & 31);
+    const int col0 = blockIdx.y * (G * NV);
+    const int64_t j = halo0 + gid;
+    const float du = __ldg(dinv_enc + n + j);
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (self_src) {
+        const float *src = self_src + (int64_t)halo_slot[j] * ld_src;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
+        }
+    }
+    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+    if (e1 - e0 > SAT_HROW_LONG) return;  // handled by a block of its own (hrow_long_block)
+    for (int64_t eb = e0; eb < e1; eb += G) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float w = 0.f;
+        if (e < e1) {
+            const int32_t p = __ldg(hrow_pos + e);
+            w = __ldg(dinv_enc + p);
+            c = by_slot ? __ldg(hrow_slot + e) : p;
+        }
+        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
+#pragma unroll 4
+        for (int q = 0; q < cnt; ++q) {
+            const int32_t cj = __shfl_sync(mask, c, q, G);
+            const float wj = __shfl_sync(mask, w, q, G);
+            const float *src = src_base + (int64_t)cj * ld_src;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
+            }
+        }
+    }
+    float *o = out_base + j * ld_out;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int idx = col0 + lane + v * G;
+        if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(du * acc[v].x, du * acc[v].y, du * acc[v].z, du * acc[v].w);
+    }
+}
+
+template <int G, int NV>
 static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4, const float *src_base, int32_t ld_src,
                         const float *self_src, float *out_base, int32_t ld_out)
 {
-    dim3 grid((unsigned)cdiv64(v.n_halo * G, 256), (unsigned)cdiv64(d4, G * NV));
+    dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hlong), (unsigned)cdiv64(d4, G * NV));
     k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->halo_slot, ctx->dinv_enc, ctx->n,
-                                                       v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out);
-    if (v.n_hlong > 0) {
-        dim3 grid2((unsigned)v.n_hlong, (unsigned)cdiv64(d4, G * NV));
-        k_spmm_hrow_long<G, NV><<<grid2, 256, 0, ctx->stream>>>(ctx->hlong, v.hlong0, ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot,
-                                                                 ctx->halo_slot, ctx->dinv_enc, ctx->n, by_slot, d4, src_base, ld_src,
-                                                                 self_src, out_base, ld_out);
-        ctx->launches++;
-    }
+                                                       v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out,
+                                                       ctx->hlong, (int32_t)v.hlong0, (int32_t)v.n_hlong);
 }
 
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src, int by_slot,
