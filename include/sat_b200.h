@@ -206,12 +206,21 @@ sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in
  * Algorithm"), so g_halo is an optional by-product and is not propagated.
  *   g_out  DEVICE [n_m x ld_g]  gradient w.r.t. this layer's output h_out
  *   g_W    DEVICE [d_in x d_out] dense; g_b DEVICE [d_out] or NULL
- *   accumulate  0: overwrite g_W / g_b; 1: add to them (summing partitions gives the
- *               gradient of the global loss, Eq. "global loss")
+ *   accumulate  bit set of SAT_BWD_* flags (0 and 1 keep their plain meaning):
+ *               SAT_BWD_ACCUMULATE (1)   add to g_W / g_b instead of overwriting them (summing partitions gives the
+ *                                        gradient of the global loss, Eq. "global loss")
+ *               SAT_BWD_MASK_G_IN (2)    write g_in already multiplied by the ReLU mask that sat_layer_fwd recorded for
+ *                                        layer - 1 on these rows, i.e. g_in = D of layer - 1 instead of the gradient w.r.t.
+ *                                        h_in (no-op when layer - 1 has no ReLU or has not run): saves the separate
+ *                                        masking pass over the activations' gradient
+ *               SAT_BWD_G_OUT_MASKED (4) g_out is such a pre-masked gradient (D of this layer): the mask is not applied again
  *   g_in   DEVICE [n_m x ld_gin] or NULL (layer 1);  g_halo DEVICE [b_m x ld_gh] or NULL
  * Requires the matching sat_layer_fwd to have run (SAT_ESTATE otherwise).  Results are
  * bit-reproducible from run to run (no floating-point atomics).
  * ------------------------------------------------------------------------------------- */
+#define SAT_BWD_ACCUMULATE 1
+#define SAT_BWD_MASK_G_IN 2
+#define SAT_BWD_G_OUT_MASKED 4
 sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g,
                          const float *W, float *g_W, float *g_b, int accumulate,
                          float *g_in, int32_t ld_gin, float *g_halo, int32_t ld_gh);

@@ -21,6 +21,7 @@ SAT_ALL_PARTS = -1
 SAT_PART_GIVEN, SAT_PART_CONTIG_BLOCKS = 0, 1
 SAT_ACT_NONE, SAT_ACT_RELU = 0, 1
 SAT_LOSS_SOFTMAX_CE, SAT_LOSS_SIGMOID_BCE = 0, 1
+SAT_BWD_ACCUMULATE, SAT_BWD_MASK_G_IN, SAT_BWD_G_OUT_MASKED = 1, 2, 4
 SAT_ROWS_INNER, SAT_ROWS_HALO = 0, 1
 SAT_CACHE_ZERO, SAT_CACHE_COPY = 0, 1
 

@@ -737,7 +737,7 @@ k_gemm_tc_mn(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ C
 // A block covers MASK_ROWS_PER_BLOCK rows; TPR threads (a power of two >= d / 4) walk one row with 128-bit accesses,
 // 256 / TPR rows per pass; each thread keeps the running sum of its four columns, the row groups are added through
 // shared memory in fixed order.
-#define MASK_ROWS_PER_BLOCK 512
+#define MASK_ROWS_PER_BLOCK 256
 __global__ void __launch_bounds__(256)
 k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t rows, int32_t d, int32_t tpr, const uint32_t *__restrict__ mask,
             int32_t mask_words, float *__restrict__ dst, int64_t ld_dst, float *__restrict__ colsum_part)
@@ -751,22 +751,36 @@ k_mask_rows(const float *__restrict__ src, int64_t ld, int64_t rows, int32_t d, 
         const int c = cb + c4;
         float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c < d4) {
-            for (int64_t r = r0 + rg; r < r1; r += n_rg) {
-                float4 x = __ldg(reinterpret_cast<const float4 *>(src + r * ld) + c);
-                if (mask) {
-                    const uint32_t w = mask[r * mask_words + (c >> 3)] >> ((c & 7) * 4);
-                    if (!(w & 1u)) x.x = 0.f;
-                    if (!(w & 2u)) x.y = 0.f;
-                    if (!(w & 4u)) x.z = 0.f;
-                    if (!(w & 8u)) x.w = 0.f;
+            // four rows in flight per thread (the loop is latency-bound otherwise); the sums are taken in row order
+            for (int64_t r = r0 + rg; r < r1; r += 4 * n_rg) {
+                float4 x[4];
+                uint32_t w[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int64_t rr = r + (int64_t)u * n_rg;
+                    x[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    w[u] = 0xFu;
+                    if (rr < r1) {
+                        x[u] = __ldg(reinterpret_cast<const float4 *>(src + rr * ld) + c);
+                        if (mask) w[u] = __ldg(mask + rr * mask_words + (c >> 3)) >> ((c & 7) * 4);
+                    }
                 }
-                if (4 * c + 3 >= d) {  // ragged tail: keep the padding columns out of the sums
-                    if (4 * c + 1 >= d) x.y = 0.f;
-                    if (4 * c + 2 >= d) x.z = 0.f;
-                    x.w = 0.f;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int64_t rr = r + (int64_t)u * n_rg;
+                    if (rr >= r1) break;
+                    if (!(w[u] & 1u)) x[u].x = 0.f;
+                    if (!(w[u] & 2u)) x[u].y = 0.f;
+                    if (!(w[u] & 4u)) x[u].z = 0.f;
+                    if (!(w[u] & 8u)) x[u].w = 0.f;
+                    if (4 * c + 3 >= d) {  // ragged tail: keep the padding columns out of the sums
+                        if (4 * c + 1 >= d) x[u].y = 0.f;
+                        if (4 * c + 2 >= d) x[u].z = 0.f;
+                        x[u].w = 0.f;
+                    }
+                    if (dst) *(reinterpret_cast<float4 *>(dst + rr * ld_dst) + c) = x[u];
+                    s.x += x[u].x; s.y += x[u].y; s.z += x[u].z; s.w += x[u].w;
                 }
-                if (dst) *(reinterpret_cast<float4 *>(dst + r * ld_dst) + c) = x;
-                s.x += x.x; s.y += x.y; s.z += x.z; s.w += x.w;
             }
         }
         if (colsum_part) {

@@ -195,8 +195,10 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
 //   or over its inner prefix (inner_only = 1).  `in_base` / `halo_base` are the virtual bases of the
 //   partition-major inner matrix and of the concatenated halo matrix (already offset for a single
 //   partition); `out_base` likewise.
+// omask (or null): bit mask [rows x omask_words] indexed like out_base; output components whose bit is 0 are written as 0
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
-                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out);
+                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask = nullptr,
+                    int32_t omask_words = 0);
 //   halo-row products: out[j] = sum_{e in hrow(j)} dinv[halo j] dinv[inner e] * src[pos_e]   (+ self term if self_src)
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src,
                          int by_slot, const float *self_src, float *out_base, int32_t ld_out);

@@ -485,7 +485,22 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     if (v.n_rows > 0 && (!g_out || !ok_ld(ld_g, d_out) || !aligned16(g_out))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: null / misaligned g_out or bad ld_g");
     if (g_in && v.n_rows > 0 && (!ok_ld(ld_gin, d_in) || !aligned16(g_in))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_in or bad ld_gin");
     if (g_halo && v.n_halo > 0 && (!ok_ld(ld_gh, d_in) || !aligned16(g_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_halo or bad ld_gh");
-    const uint32_t *mask = L.act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * L.mask_words : nullptr;
+    const int flags = accumulate;
+    accumulate = flags & SAT_BWD_ACCUMULATE;
+    if (flags & ~(SAT_BWD_ACCUMULATE | SAT_BWD_MASK_G_IN | SAT_BWD_G_OUT_MASKED)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: unknown flag bits");
+    const uint32_t *mask = (L.act == SAT_ACT_RELU && !(flags & SAT_BWD_G_OUT_MASKED)) ? L.mask + (int64_t)v.row0 * L.mask_words : nullptr;
+    // ReLU mask of the layer below, applied to g_in on request (indexed by partition-major row like g_in)
+    const uint32_t *mask_in = nullptr;
+    int32_t mask_in_words = 0;
+    if ((flags & SAT_BWD_MASK_G_IN) && layer > 1) {
+        LayerState &Lp = ctx->layers[layer - 1];
+        bool ok = Lp.agg && Lp.act == SAT_ACT_RELU && Lp.mask && Lp.d_out == L.d_in;
+        for (int m = (part == SAT_ALL_PARTS ? 0 : part); ok && m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m) ok = Lp.valid[m];
+        if (ok) {
+            mask_in = Lp.mask;
+            mask_in_words = Lp.mask_words;
+        }
+    }
     const float *agg = L.agg + (int64_t)v.row0 * L.ld_in;
     const bool want_dx = (g_in || g_halo) && v.n_rows > 0;
     const bool tc_w = sat_use_tc(d_out, d_in) && v.n_rows >= 256;   // weight gradient on the tensor cores
@@ -524,7 +539,7 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     }
     const float *ga_base = gagg - (int64_t)v.row0 * ld_ga;
     // G_in = P_in^T G_AGG: the inner block of P is symmetric, so P_in^T = P_in (inner prefix of every local row)
-    if (g_in) SAT_TRY(sat_spmm(ctx, v, 1, d_in, ga_base, ld_ga, nullptr, 0, g_in - (int64_t)v.row0 * ld_gin, ld_gin));
+    if (g_in) SAT_TRY(sat_spmm(ctx, v, 1, d_in, ga_base, ld_ga, nullptr, 0, g_in - (int64_t)v.row0 * ld_gin, ld_gin, mask_in, mask_in_words));
     // G_halo = P_out^T G_AGG over the halo-row CSR
     if (g_halo) SAT_TRY(sat_spmm_hrow(ctx, v, d_in, ga_base, ld_ga, 0, nullptr, g_halo - v.halo0 * (int64_t)ld_gh, ld_gh));
     return SAT_OK;

@@ -13,6 +13,16 @@ __device__ __forceinline__ void fma4(float4 &a, float w, const float4 &x)
     a.w = fmaf(w, x.w, a.w);
 }
 
+// zero the components of float4 column `idx` of a row whose bits in the row's bit mask (word_base = row * words) are 0
+__device__ __forceinline__ void mask4(float4 &r, const uint32_t *__restrict__ omask, int64_t word_base, int idx)
+{
+    const uint32_t m = __ldg(omask + word_base + (idx >> 3)) >> ((idx & 7) * 4);
+    if (!(m & 1u)) r.x = 0.f;
+    if (!(m & 2u)) r.y = 0.f;
+    if (!(m & 4u)) r.z = 0.f;
+    if (!(m & 8u)) r.w = 0.f;
+}
+
 template <int G>
 __device__ __forceinline__ unsigned group_mask(int lane_in_warp)
 {
@@ -32,7 +42,7 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
              const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
              const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0, int inner_only, int32_t n,
              int32_t d4, const float *__restrict__ in_base, int64_t ld_in, const float *__restrict__ halo_base, int64_t ld_halo,
-             float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial)
+             float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial, const uint32_t *__restrict__ omask, int32_t omask_words)
 {
     const int lane = threadIdx.x & (G - 1);
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
@@ -77,7 +87,11 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int idx = col0 + lane + v * G;
-            if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(s * acc[v].x, s * acc[v].y, s * acc[v].z, s * acc[v].w);
+            if (idx < d4) {
+                float4 r = make_float4(s * acc[v].x, s * acc[v].y, s * acc[v].z, s * acc[v].w);
+                if (omask) mask4(r, omask, (int64_t)row * omask_words, idx);
+                *reinterpret_cast<float4 *>(o + 4 * idx) = r;
+            }
         }
     } else {
         float *o = partial + (int64_t)(ms - mitem0) * (4 * (int64_t)d4);
@@ -92,7 +106,8 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
 // rows cut into several chunks: add the partial sums in chunk order, scale, store
 __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, int32_t n_mrows, const int32_t *__restrict__ first_item,
                              const int32_t *__restrict__ item_mslot, int32_t mitem0, const float *__restrict__ dinv_enc, int32_t d4,
-                             const float *__restrict__ partial, float *__restrict__ out_base, int64_t ld_out)
+                             const float *__restrict__ partial, float *__restrict__ out_base, int64_t ld_out,
+                             const uint32_t *__restrict__ omask, int32_t omask_words)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / d4;
@@ -110,21 +125,24 @@ __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, i
         a.w += x.w;
     }
     const float s = dinv_enc[row];
-    *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c) = make_float4(s * a.x, s * a.y, s * a.z, s * a.w);
+    float4 r = make_float4(s * a.x, s * a.y, s * a.z, s * a.w);
+    if (omask) mask4(r, omask, (int64_t)row * omask_words, c);
+    *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c) = r;
 }
 
 template <int G, int NV>
 static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d4, const float *in_base, int32_t ld_in,
-                         const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial)
+                         const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial, const uint32_t *omask,
+                         int32_t omask_words)
 {
     dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
     k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->dinv_enc, ctx->item_row,
                                                         ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
-                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial);
+                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words);
 }
 
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
-                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out)
+                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask, int32_t omask_words)
 {
     if (v.n_items == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
@@ -138,7 +156,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
         SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * d4 * 16));
         partial = (float *)ctx->buf_partial.p;
     }
-#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial
+#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words
     if (d4 <= 4) launch_items<4, 1>(ARGS);
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);
@@ -153,7 +171,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     SAT_LAUNCHED(ctx);
     if (v.n_mrows > 0) {
         k_spmm_fixup<<<(unsigned)cdiv64((int64_t)v.n_mrows * d4, 256), 256, 0, ctx->stream>>>(
-            ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, ctx->dinv_enc, d4, partial, out_base, ld_out);
+            ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, ctx->dinv_enc, d4, partial, out_base, ld_out, omask, omask_words);
         SAT_LAUNCHED(ctx);
     }
     return SAT_OK;

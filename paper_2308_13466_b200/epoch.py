@@ -101,7 +101,9 @@ class SatEpoch:
         B.sat_loss_grad(ctx, m, kind, self.rows(self.H[L], m), self.rows(self.labels, m), self.loss_sum, g)
         for l in range(L, 0, -1):
             g_in = self.rows(self.G[l - 1], m) if l > 1 else None
-            B.sat_layer_bwd(ctx, m, l, g, W[l - 1], self.gW[l - 1], self.gb[l - 1], accumulate, g_in, None)
+            # the gradient handed down is written already multiplied by the ReLU mask of the layer below (no separate pass)
+            flags = accumulate | (B.SAT_BWD_MASK_G_IN if l > 1 else 0) | (B.SAT_BWD_G_OUT_MASKED if l < L else 0)
+            B.sat_layer_bwd(ctx, m, l, g, W[l - 1], self.gW[l - 1], self.gb[l - 1], flags, g_in, None)
             g = g_in
 
     def step(self, W, b, pred, lr: float | None = None):

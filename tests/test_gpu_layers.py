@@ -139,6 +139,21 @@ def _check_calls(B, case: Case, parts, check_halo_grad=True):
             note("G_in", assert_close(g_in.cpu().numpy(), gin_o, f"G_in l={l} m={m}"))
             if check_halo_grad and b_m:
                 note("G_halo", assert_close(g_halo.cpu().numpy(), ghalo_o, f"G_halo l={l} m={m}"))
+            # fused masking: g_in written as D of the layer below; a pre-masked g_out is not masked again
+            gW_plain, gb_plain, gin_plain = gW.cpu().numpy().copy(), gb.cpu().numpy().copy(), g_in.cpu().numpy().copy()
+            if l > 1:
+                g_in2 = empty2d(n_m, wl.dims[l - 1])
+                g_halo2 = empty2d(b_m, wl.dims[l - 1]) if check_halo_grad else None   # same contraction path as the plain call
+                B.sat_layer_bwd(ctx, m, l, dev2d(G_out), Wd[l - 1], gW, gb, B.SAT_BWD_MASK_G_IN, g_in2, g_halo2)
+                assert np.array_equal(g_in2.cpu().numpy(), np.where(gpu_masks[l - 1], gin_plain, 0.0).astype(np.float32)), \
+                    f"g_in with the mask of layer {l - 1} fused, m={m}"
+            if l < L:
+                B.sat_layer_bwd(ctx, m, l, dev2d(np.where(gpu_masks[l], G_out, 0.0).astype(np.float32)), Wd[l - 1], gW, gb,
+                                B.SAT_BWD_G_OUT_MASKED, g_in, None)
+                assert np.array_equal(gW.cpu().numpy(), gW_plain) and np.array_equal(gb.cpu().numpy(), gb_plain), \
+                    f"pre-masked g_out, l={l} m={m}"
+                # (the input gradient may take the tensor-core path here: no halo gradient is asked for)
+                assert_close(g_in.cpu().numpy(), gin_o, f"G_in from a pre-masked g_out, l={l} m={m}")
             # accumulate = 1 adds to what is there
             B.sat_layer_bwd(ctx, m, l, dev2d(G_out), Wd[l - 1], gW, gb, 1, None, None)
             note("G_W2", assert_close(gW.cpu().numpy(), 2 * GW, f"accumulated G_W l={l} m={m}"))
