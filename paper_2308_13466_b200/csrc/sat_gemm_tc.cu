@@ -151,18 +151,32 @@ __host__ __device__ inline uint32_t make_idesc(int n, int a_mn_major, int b_mn_m
 }
 
 // =====================================================================================
-// TF32 split of a shared-memory tile, element-wise.  The tensor core reads an fp32 container as TF32 by ignoring the low
-// 13 mantissa bits, so the raw tile already is the "hi" operand (hi = x with those bits cleared); only the residual
-// lo = x - hi (exact in fp32, again truncated by the tensor core when read) has to be written, at the same offset of the
-// second tile.  |x - hi - tf32(lo)| < 2^-20 |x|.
+// TF32 split of a shared-memory tile, element-wise (the swizzled layout never has to be decoded).
+//
+// The tensor core reads an fp32 container as TF32 by ignoring the low 13 mantissa bits.  split_tile_residual uses that:
+// the raw tile already is the "hi" operand (hi = x with those bits cleared) and only lo = tf32_rn(x - hi) is written, to
+// the second tile (x - hi is exact; rounding lo to nearest keeps the representation error |x - hi - lo| <= 2^-21 |x|
+// free of bias).  split_tile_round rounds hi to nearest as well and rewrites the raw tile in place: hi and lo are then
+// symmetric around x, which matters for the weight gradient (a small difference of ~1e5 signed terms per element).
 // =====================================================================================
-__device__ __forceinline__ float tf32_residual(float x) { return x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u); }
+__device__ __forceinline__ float tf32_round(float x)
+{
+    return __uint_as_float((__float_as_uint(x) + 0x1000u) & 0xFFFFE000u);  // round half away from zero to 10 mantissa bits
+}
+__device__ __forceinline__ float tf32_residual(float x) { return tf32_round(x - __uint_as_float(__float_as_uint(x) & 0xFFFFE000u)); }
 __device__ __forceinline__ float4 residual4(const float4 &x)
 {
     return make_float4(tf32_residual(x.x), tf32_residual(x.y), tf32_residual(x.z), tf32_residual(x.w));
 }
-// two 16-byte chunks per thread and iteration, loads first (the loop is latency-bound otherwise)
-__device__ __forceinline__ void split_tile(const uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
+__device__ __forceinline__ void split4(const float4 &x, float4 &h, float4 &l)
+{
+    h.x = tf32_round(x.x); l.x = tf32_round(x.x - h.x);
+    h.y = tf32_round(x.y); l.y = tf32_round(x.y - h.y);
+    h.z = tf32_round(x.z); l.z = tf32_round(x.z - h.z);
+    h.w = tf32_round(x.w); l.w = tf32_round(x.w - h.w);
+}
+// two 16-byte chunks per thread and iteration, loads first (the loops are latency-bound otherwise)
+__device__ __forceinline__ void split_tile_residual(const uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
 {
     const uint32_t step = (uint32_t)nthreads * 16;
     for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += 2 * step) {
@@ -173,6 +187,26 @@ __device__ __forceinline__ void split_tile(const uint8_t *hi_tile, uint8_t *lo_t
         if (two) x2 = *reinterpret_cast<const float4 *>(hi_tile + off2);
         *reinterpret_cast<float4 *>(lo_tile + off) = residual4(x1);
         if (two) *reinterpret_cast<float4 *>(lo_tile + off2) = residual4(x2);
+    }
+}
+__device__ __forceinline__ void split_tile_round(uint8_t *hi_tile, uint8_t *lo_tile, uint32_t bytes, int tid, int nthreads)
+{
+    const uint32_t step = (uint32_t)nthreads * 16;
+    for (uint32_t off = (uint32_t)tid * 16; off < bytes; off += 2 * step) {
+        const uint32_t off2 = off + step;
+        const bool two = off2 < bytes;
+        const float4 x1 = *reinterpret_cast<float4 *>(hi_tile + off);
+        float4 x2 = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (two) x2 = *reinterpret_cast<float4 *>(hi_tile + off2);
+        float4 h1, l1, h2, l2;
+        split4(x1, h1, l1);
+        split4(x2, h2, l2);
+        *reinterpret_cast<float4 *>(hi_tile + off) = h1;
+        *reinterpret_cast<float4 *>(lo_tile + off) = l1;
+        if (two) {
+            *reinterpret_cast<float4 *>(hi_tile + off2) = h2;
+            *reinterpret_cast<float4 *>(lo_tile + off2) = l2;
+        }
     }
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar)
@@ -197,7 +231,7 @@ struct TcEpilogue {
     int64_t ld_resid;
     int32_t lstm_h;      // > 0: fused LSTM cell, C = hidden state [M x lstm_h], lstm_c = cell state
     int lstm_first;
-    float *lstm_c;
+    float *lstm_c;       // cell state in the blocked layout of sat_cell_offset
     const float *addend; // [M x ld_addend] added to the gate pre-activations (cached input projection), or null
     int64_t ld_addend;
 };
@@ -362,8 +396,8 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const uint32_t ph = (it / STAGES) & 1u;
                 if (!mbar_wait_warp(&sh->full[s], ph, dead, status, lane)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
-                split_tile(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
-                split_tile(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_THREADS);
+                split_tile_residual(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
+                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_THREADS);
                 fence_async_smem();
                 mbar_arrive(&sh->conv[s]);
             }
@@ -462,8 +496,9 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     cside[0] = cside[1] = zero4;
                     const int32_t j0 = (n0 + c0) >> 2;
                     if (row_ok && lstm_full && !ep.lstm_first && j0 + 7 < ep.lstm_h) {
-                        cside[0] = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
-                        cside[1] = *reinterpret_cast<const float4 *>(ep.lstm_c + row * ep.lstm_h + j0 + 4);
+                        const float *cp = ep.lstm_c + sat_cell_offset(row, j0, ep.lstm_h);
+                        cside[0] = *reinterpret_cast<const float4 *>(cp);
+                        cside[1] = *reinterpret_cast<const float4 *>(cp + 4);
                     }
                 }
             };
@@ -506,7 +541,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         if (!ep.lstm_first && !full) {
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
-                                if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[row * ep.lstm_h + j0 + u];
+                                if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[sat_cell_offset(row, j0 + u, ep.lstm_h)];
                         }
                         if (c0 + 64 < bn) load_cell(c0 + 64);
                         float sv[8], cv[8];
@@ -520,7 +555,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                             sv[u] = go * tanh_fast(cv[u]);
                         }
                         if (full) {
-                            float4 *cd = reinterpret_cast<float4 *>(ep.lstm_c + row * ep.lstm_h + j0);
+                            float4 *cd = reinterpret_cast<float4 *>(ep.lstm_c + sat_cell_offset(row, j0, ep.lstm_h));
                             float4 *sd = reinterpret_cast<float4 *>(ep.C + row * ep.ldc + j0);
                             cd[0] = make_float4(cv[0], cv[1], cv[2], cv[3]);
                             cd[1] = make_float4(cv[4], cv[5], cv[6], cv[7]);
@@ -530,7 +565,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 #pragma unroll
                             for (int u = 0; u < 8; ++u)
                                 if (j0 + u < ep.lstm_h) {
-                                    ep.lstm_c[row * ep.lstm_h + j0 + u] = cv[u];
+                                    ep.lstm_c[sat_cell_offset(row, j0 + u, ep.lstm_h)] = cv[u];
                                     ep.C[row * ep.ldc + j0 + u] = sv[u];
                                 }
                         }
@@ -699,8 +734,8 @@ k_gemm_tc_mn(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ C
             alive = mbar_wait(&sh->full[s], ph, dead, status);
             if (!alive) break;
             uint8_t *st = smem + (size_t)s * stage_bytes;
-            split_tile(st, st + a_bytes, a_bytes, ctid, TC_CONV_THREADS);
-            split_tile(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TC_CONV_THREADS);
+            split_tile_round(st, st + a_bytes, a_bytes, ctid, TC_CONV_THREADS);
+            split_tile_round(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TC_CONV_THREADS);
             fence_async_smem();
             mbar_arrive(&sh->conv[s]);
         }

@@ -233,6 +233,15 @@ sat_status sat_splitk_reduce(sat_ctx *ctx, const float *part, int64_t count, int
                              int32_t ld_out);
 
 // GEMM family on the tensor cores (sat_gemm_tc.cu): TF32 two-term split, fp32 operands in global memory
+// Cell state of the fused LSTM (internal scratch, never exposed): blocks of [32 rows x 8 units] = 1 KB, block index
+// (row / 32) * ceil(h / 8) + unit / 8.  A warp of the GEMM epilogue (one row per lane, 8 units per chunk) then reads and
+// writes one contiguous KB instead of 32 separate cache lines.
+__host__ __device__ inline int64_t sat_cell_offset(int64_t row, int32_t j, int32_t h)
+{
+    return (((row >> 5) * ((h + 7) >> 3) + (j >> 3)) << 8) + ((row & 31) << 3) + (j & 7);
+}
+inline size_t sat_cell_floats(int64_t rows, int32_t h) { return (size_t)((rows + 31) / 32) * ((h + 7) / 8) * 256; }
+
 struct TcWeights {         // weight operand as two fp32 planes [n_pad x ld] holding the TF32 hi / lo terms, K-major
     float *hi = nullptr, *lo = nullptr;
     int32_t ld = 0, n_pad = 0;

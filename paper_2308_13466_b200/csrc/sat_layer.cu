@@ -225,7 +225,7 @@ __global__ void k_lstm_cell_first(const float *__restrict__ proj, int64_t rows, 
     const float gg = tanhf(a.z);
     const float go = 1.f / (1.f + expf(-a.w));
     const float cn = gi * gg;
-    c[t] = cn;
+    c[sat_cell_offset(t / h, (int32_t)(t % h), h)] = cn;
     s[t] = go * tanhf(cn);
 }
 
@@ -296,7 +296,7 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
         return SAT_OK;
     }
     if (!(sat_use_tc(4 * h, d) && 4 * h <= 256)) SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_w, (size_t)rows * 4 * h * sizeof(float)));
-    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_c, (size_t)rows * h * sizeof(float)));
+    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_c, sat_cell_floats(rows, h) * sizeof(float)));
     float *gates = (float *)ctx->buf_lstm_w.p;
     float *cell = (float *)ctx->buf_lstm_c.p;
     const bool tc = sat_use_tc(4 * h, d);
