@@ -305,6 +305,126 @@ sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const f
 }
 
 // =====================================================================================
+// Weight gradient with a narrow output (n <= 64: the classifier layer), fp32 FMA with round-to-nearest.
+// C = A^T B sums ~1e5 signed terms per element that cancel to a few 1e-3 of their magnitude (softmax gradients sum to
+// zero); the tensor-core contraction, whose accumulation truncates, was measured at 1e-4 relative error there against
+// 2e-5 for this kernel, which at this width costs about the same.
+//   block (x, y): rows [x * rows_per_block, ...), columns m = y * 256 + thread of A; NT accumulators per thread; B rows are
+//   staged in shared memory and broadcast; partial sums per row block, added in block order by k_splitk_reduce.
+// =====================================================================================
+#define TNN_STAGE 32
+__device__ __forceinline__ void tnn_cp16(void *smem_dst, const void *gsrc, bool valid)
+{
+    // src-size 0 writes 16 zero bytes without reading the source
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc),
+                 "r"(valid ? 16u : 0u)
+                 : "memory");
+}
+// two stages of [TNN_STAGE x 256] of A and [TNN_STAGE x NT] of B, filled by cp.async while the previous stage is consumed
+template <int NT>
+__global__ void __launch_bounds__(256)
+k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, const float *__restrict__ A, int64_t lda,
+                 const float *__restrict__ B, int64_t ldb, float *__restrict__ part)
+{
+    extern __shared__ __align__(16) float tnn_smem[];
+    constexpr int STAGE_FLOATS = TNN_STAGE * 256 + TNN_STAGE * NT;
+    const int32_t m0 = blockIdx.y * 256;
+    const int32_t col = m0 + threadIdx.x;
+    const int32_t m4 = (m + 3) & ~3, n4 = (n + 3) & ~3;
+    const int64_t r_begin = (int64_t)blockIdx.x * rows_per_block;
+    const int64_t r_end = r_begin + rows_per_block < rows ? r_begin + rows_per_block : rows;
+    auto load_stage = [&](int s, int64_t r0) {
+        float *As = tnn_smem + s * STAGE_FLOATS, *Bs = As + TNN_STAGE * 256;
+#pragma unroll
+        for (int k = 0; k < TNN_STAGE * 64 / 256; ++k) {
+            const int i = threadIdx.x + 256 * k, rr = i >> 6, c4 = i & 63;
+            const bool ok = r0 + rr < r_end && m0 + 4 * c4 < m4;
+            tnn_cp16(As + rr * 256 + 4 * c4, ok ? A + (r0 + rr) * lda + m0 + 4 * c4 : A, ok);
+        }
+        for (int i = threadIdx.x; i < TNN_STAGE * (NT / 4); i += 256) {
+            const int rr = i / (NT / 4), j4 = i - rr * (NT / 4);
+            const bool ok = r0 + rr < r_end && 4 * j4 < n4;
+            tnn_cp16(Bs + rr * NT + 4 * j4, ok ? B + (r0 + rr) * ldb + 4 * j4 : B, ok);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    float acc[NT];
+#pragma unroll
+    for (int j = 0; j < NT; ++j) acc[j] = 0.f;
+    int s = 0;
+    load_stage(0, r_begin);
+    for (int64_t r0 = r_begin; r0 < r_end; r0 += TNN_STAGE, s ^= 1) {
+        if (r0 + TNN_STAGE < r_end) {
+            load_stage(s ^ 1, r0 + TNN_STAGE);
+            asm volatile("cp.async.wait_group 1;" ::: "memory");
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();
+        const float *As = tnn_smem + s * STAGE_FLOATS, *Bs = As + TNN_STAGE * 256;
+#pragma unroll 4
+        for (int rr = 0; rr < TNN_STAGE; ++rr) {
+            const float a = As[rr * 256 + threadIdx.x];
+#pragma unroll
+            for (int j4 = 0; j4 < NT; j4 += 4) {
+                const float4 b = *reinterpret_cast<const float4 *>(Bs + rr * NT + j4);
+                acc[j4] = fmaf(a, b.x, acc[j4]);
+                acc[j4 + 1] = fmaf(a, b.y, acc[j4 + 1]);
+                acc[j4 + 2] = fmaf(a, b.z, acc[j4 + 2]);
+                acc[j4 + 3] = fmaf(a, b.w, acc[j4 + 3]);
+            }
+        }
+        __syncthreads();  // the stage is refilled two iterations later
+    }
+    if (col < m) {
+        float *o = part + ((int64_t)blockIdx.x * m + col) * n;
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+            if (j < n) o[j] = acc[j];
+    }
+}
+
+template <int NT>
+static sat_status launch_tn_narrow(sat_ctx *ctx, dim3 grid, int64_t rows, int64_t rpb, int32_t m, int32_t n, const float *A, int32_t lda,
+                                   const float *B, int32_t ldb, float *part)
+{
+    static bool attr_set = false;
+    const size_t smem = 2 * (size_t)(TNN_STAGE * 256 + TNN_STAGE * NT) * sizeof(float);
+    if (!attr_set) {
+        SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tn_narrow<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set = true;
+    }
+    k_gemm_tn_narrow<NT><<<grid, 256, smem, ctx->stream>>>(rows, rpb, m, n, A, lda, B, ldb, part);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+// C[m x n] (+)= A^T B over `rows` rows for n <= 64 (B already masked)
+sat_status sat_gemm_tn_narrow(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
+                              float *C, int32_t ldc, int accumulate)
+{
+    if (m == 0 || n == 0) return SAT_OK;
+    if (n > 64 || (lda & 3) || (ldb & 3) || (((uintptr_t)A | (uintptr_t)B) & 15u))
+        return sat_fail(ctx, SAT_EINVAL, "sat_gemm_tn_narrow: n must be <= 64, operands 16-byte aligned with leading dimensions in multiples of 4");
+    ProfScope prof(ctx, SATK_GEMM_TN, 4.0 * ((double)rows * (m + n) + (double)m * n), 2.0 * (double)rows * m * n);
+    // two CTAs fit on an SM (80 KB of shared memory each): one full wave of row blocks
+    int sms = 148;
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
+    const int64_t want = (2 * (int64_t)sms) / cdiv64(m, 256) > 0 ? (2 * (int64_t)sms) / cdiv64(m, 256) : 1;
+    int64_t rpb = cdiv64(cdiv64(rows > 0 ? rows : 1, want), TNN_STAGE) * TNN_STAGE;
+    if (rpb < 4 * TNN_STAGE) rpb = 4 * TNN_STAGE;
+    const int64_t blocks = cdiv64(rows > 0 ? rows : 1, rpb);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_splitk, (size_t)blocks * m * n * sizeof(float)));
+    float *part = (float *)ctx->buf_splitk.p;
+    dim3 grid((unsigned)blocks, (unsigned)cdiv64(m, 256));
+    if (n <= 16) SAT_TRY(launch_tn_narrow<16>(ctx, grid, rows, rpb, m, n, A, lda, B, ldb, part));
+    else if (n <= 32) SAT_TRY(launch_tn_narrow<32>(ctx, grid, rows, rpb, m, n, A, lda, B, ldb, part));
+    else if (n <= 48) SAT_TRY(launch_tn_narrow<48>(ctx, grid, rows, rpb, m, n, A, lda, B, ldb, part));
+    else SAT_TRY(launch_tn_narrow<64>(ctx, grid, rows, rpb, m, n, A, lda, B, ldb, part));
+    return sat_splitk_reduce(ctx, part, (int64_t)m * n, (int32_t)blocks, accumulate, C, n, ldc);
+}
+
+// =====================================================================================
 // sat_dense_tn_static: the split weight-gradient product without any allocation
 // =====================================================================================
 // Some callers must not allocate device memory at all: code that runs while another component owns the whole device

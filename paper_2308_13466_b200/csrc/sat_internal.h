@@ -229,6 +229,8 @@ sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const f
                        int accumulate);
 
 // out[r][c] (+)= sum_z part[z][r * ncols + c], z ascending (fixed order: reproducible)
+sat_status sat_gemm_tn_narrow(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb,
+                              float *C, int32_t ldc, int accumulate);
 sat_status sat_splitk_reduce(sat_ctx *ctx, const float *part, int64_t count, int32_t splits, int accumulate, float *out, int32_t ncols,
                              int32_t ld_out);
 

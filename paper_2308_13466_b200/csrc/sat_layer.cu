@@ -520,7 +520,8 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
         SAT_TRY(sat_mask_rows(ctx, g_out, ld_g, v.n_rows, d_out, mask, L.mask_words, dm, ld_d, tc_w ? g_b : nullptr, accumulate));
     }
     // G_W (+)= AGG^T D, G_b (+)= 1^T D
-    if (tc_w) SAT_TRY(sat_gemm_tc_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
+    if (tc_w && d_out <= 64) SAT_TRY(sat_gemm_tn_narrow(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
+    else if (tc_w) SAT_TRY(sat_gemm_tc_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
     else SAT_TRY(sat_gemm_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, g_out, ld_g, mask, L.mask_words, g_W, d_out, g_b, accumulate));
     if (!want_dx) return SAT_OK;
     // G_AGG = D W^T
