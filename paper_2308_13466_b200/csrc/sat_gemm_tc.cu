@@ -261,6 +261,11 @@ struct TcShared {
 #define TC_EPI_THREADS 128
 #define TCK_CONV_WARPS 6
 #define TCK_CONV_THREADS (TCK_CONV_WARPS * 32)
+/* The converter warps work in two groups on alternate k-blocks, so two stages are being split at any time.  Every stage
+ * count is even, hence a stage is always handled by the same group and each group meets the phases of its stages in
+ * order (a parity wait must never be more than one phase ahead of its barrier). */
+#define TCK_CONV_GROUPS 2
+#define TCK_CONV_GROUP_THREADS (TCK_CONV_THREADS / TCK_CONV_GROUPS)
 #define TCK_EPI_WARPS 8
 #define TCK_EPI_THREADS (TCK_EPI_WARPS * 32)
 #define TCK_EPI_WARP0 (2 + TCK_CONV_WARPS)
@@ -276,6 +281,9 @@ template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, ou
 template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 3, out_bytes = TCK_OUT_BYTES; };
 template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, out_bytes = 0; };
 template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 4, out_bytes = 0; };
+static_assert(TckCfg<EPI_PLAIN>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_RESID>::stages % TCK_CONV_GROUPS == 0 &&
+                  TckCfg<EPI_LSTM>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_LSTM_ADD>::stages % TCK_CONV_GROUPS == 0,
+              "a stage must always be split by the same converter group");
 
 __device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, bool valid)
 {
@@ -314,7 +322,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sh->full[s], 1);
-            mbar_init(&sh->conv[s], TCK_CONV_THREADS);
+            mbar_init(&sh->conv[s], TCK_CONV_GROUP_THREADS);
             mbar_init(&sh->empty[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
@@ -388,16 +396,18 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         }
     } else if (warp < TCK_EPI_WARP0) {
         // ---------------- converters: TF32 split of the A and B tiles of every k-block ----------------
-        const int ctid = threadIdx.x - 64;
+        const int grp = (threadIdx.x - 64) / TCK_CONV_GROUP_THREADS;
+        const int ctid = (threadIdx.x - 64) % TCK_CONV_GROUP_THREADS;
         uint32_t it = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
             for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
+                if ((int)(it % TCK_CONV_GROUPS) != grp) continue;
                 const int s = it % STAGES;
                 const uint32_t ph = (it / STAGES) & 1u;
                 if (!mbar_wait_warp(&sh->full[s], ph, dead, status, lane)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
-                split_tile_residual(st, st + a_bytes, a_bytes, ctid, TCK_CONV_THREADS);
-                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_THREADS);
+                split_tile_residual(st, st + a_bytes, a_bytes, ctid, TCK_CONV_GROUP_THREADS);
+                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_GROUP_THREADS);
                 fence_async_smem();
                 mbar_arrive(&sh->conv[s]);
             }
