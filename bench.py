@@ -35,7 +35,7 @@ if ROOT not in sys.path:
 # workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
 # gemm_nn: 300 MB = the 256-wide layer transform and the LSTM gate contraction alike (profiles/k_gemm_tc_k_medium.md);
 # spmm_fwd: 684 MB = the d = 256 launch (profiles/k_spmm_items_medium.md).
-NCU_TRAFFIC_BYTES = {"gemm_nn": 300.0e6, "spmm_fwd": 683.6e6}
+NCU_TRAFFIC_BYTES = {"gemm_nn": 300.0e6, "spmm_fwd": 683.6e6, "gemm_side": None}
 
 # The contractions run on the tensor cores in TF32 (two-term split: three TF32 MMAs per product term).  The box's
 # measured tensor peak is a bf16 figure; TF32 is taken as measured bf16 x the nominal ratio 1.1 / 2.25 PFLOP/s.
@@ -298,7 +298,7 @@ def run_ours(args, wl):
         fam = max(prof, key=lambda k: prof[k]["ms"])
         rec = prof[fam]
         per_launch_ms = rec["ms"] / max(rec["calls"], 1)
-        if fam.startswith("gemm"):
+        if fam.startswith("gemm") and fam != "gemm_side":   # gemm_side: K = h contractions with a streamed side operand (HBM-bound)
             tfl = TF32_MMAS_PER_TERM * rec["flops"] / (rec["ms"] * 1e-3) / 1e12
             peak = peaks["bf16"] * TF32_OVER_BF16
             roofline = dict(kernel=fam, bound="tensor", achieved=tfl, peak=peak, unit="TFLOP/s", frac=tfl / peak,

@@ -207,7 +207,7 @@ extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
 // per-family device timing
 // =====================================================================================
 static const char *k_family_names[SATK_COUNT] = {"spmm_fwd", "spmm_bwd", "spmm_hrow", "gemm_nn", "gemm_nt", "gemm_tn",
-                                                 "lstm_cell", "gather", "scatter", "loss", "mask"};
+                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side"};
 
 static void prof_clear(sat_ctx *ctx)
 {

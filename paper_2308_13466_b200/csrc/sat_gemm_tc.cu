@@ -1005,7 +1005,12 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     const int32_t nkb1 = (k1 + TC_BK - 1) / TC_BK, nkb2 = A2 ? (k2 + TC_BK - 1) / TC_BK : 0;
     const int32_t bn = tile_n_for(n);
     const uint32_t stage_bytes = 2 * (TC_BM * TC_BK * 4) + 2 * (uint32_t)bn * TC_BK * 4;
-    ProfScope prof(ctx, family, 4.0 * ((double)m * (k1 + k2 + n) + (double)(k1 + k2) * n), 2.0 * (double)m * n * (k1 + k2));
+    // algorithmic bytes: operands once, results once.  Plain: A, B, C.  Gathered residual: + the residual rows.  LSTM cell:
+    // the output is the hidden state [m x h] plus the cell state read and written, and the cached projection if it is added.
+    double alg_bytes = 4.0 * ((double)m * (k1 + k2) + (double)(k1 + k2) * n);
+    if (eh.lstm_h > 0) alg_bytes += 4.0 * (double)m * eh.lstm_h * (eh.lstm_first ? 2.0 : 3.0) + (eh.addend ? 4.0 * (double)m * n : 0.0);
+    else alg_bytes += 4.0 * (double)m * n * (eh.resid_idx ? 2.0 : 1.0);
+    ProfScope prof(ctx, family, alg_bytes, 2.0 * (double)m * n * (k1 + k2));
     CUtensorMap mA, mA2, mB, mC;
     const int use_tma_store = eh.lstm_h == 0 && ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
     if (use_tma_store) SAT_TRY(make_map(ctx, &mC, eh.C, n, m, eh.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B));

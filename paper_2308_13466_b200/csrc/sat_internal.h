@@ -46,7 +46,7 @@ struct CacheLayer {
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
-    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_COUNT
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_COUNT
 };
 
 struct ProfRec {

@@ -274,7 +274,7 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
             eh.lstm_c = cell;
             eh.addend = pr;
             eh.ld_addend = 4 * h;
-            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_NN));
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
         }
     }
     c->S_valid = true;
@@ -387,7 +387,7 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
             eh.resid_idx = ctx->halo_slot + v.halo0;
             eh.ld_resid = c->ld;
         }
-        return sat_gemm_tc(ctx, v.n_halo, d, a, ld_a, h, nullptr, 0, 0, Wg, eh, SATK_GEMM_NN);
+        return sat_gemm_tc(ctx, v.n_halo, d, a, ld_a, h, nullptr, 0, 0, Wg, eh, SATK_GEMM_SIDE);
     }
     GemmEpilogue ep;
     ep.bias = params->bg;
