@@ -374,7 +374,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
+                    // the converters arrive on conv[s] only after they have seen full[s] (the TMA bytes) themselves
                     if (!mbar_wait(&sh->conv[s], ph, dead, status)) goto done;
                     tc_fence_after();
                     const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
@@ -404,7 +404,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 if ((int)(it % TCK_CONV_GROUPS) != grp) continue;
                 const int s = it % STAGES;
                 const uint32_t ph = (it / STAGES) & 1u;
-                if (!mbar_wait_warp(&sh->full[s], ph, dead, status, lane)) goto done;
+                if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 split_tile_residual(st, st + a_bytes, a_bytes, ctid, TCK_CONV_GROUP_THREADS);
                 split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_GROUP_THREADS);
