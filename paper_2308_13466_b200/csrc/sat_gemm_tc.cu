@@ -236,15 +236,25 @@ struct TcEpilogue {
     int64_t ld_addend;
 };
 
-// logistic and tanh from the hardware exponential (ex2.approx) and reciprocal: absolute error of a few 1e-7, which is
-// what matters for gate values in [0, 1] / [-1, 1]; an order of magnitude cheaper than the libm versions, so that the
-// four epilogue warps keep up with the main loop
-__device__ __forceinline__ float sigmoid_fast(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
-__device__ __forceinline__ float tanh_fast(float x)
+// logistic and tanh from the hardware base-2 exponential and reciprocal (ex2.approx / rcp.approx, flush-to-zero forms:
+// one instruction each): absolute error of a few 1e-7, which is what matters for gate values in [0, 1] / [-1, 1].  Four and
+// five instructions per value; the LSTM epilogue is bound by instruction issue, so the libm versions (and even __expf /
+// __fdividef, which carry range handling) cost more than the memory traffic of the step.
+__device__ __forceinline__ float ex2_fast(float x)
 {
-    const float e = __expf(-2.f * fabsf(x));
-    return copysignf(__fdividef(1.f - e, 1.f + e), x);
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float sigmoid_fast(float x) { return rcp_fast(1.f + ex2_fast(-1.4426950408889634f * x)); }
+// tanh x = 1 - 2 / (1 + e^{2x}); saturates correctly (e -> inf gives 1, e -> 0 gives -1)
+__device__ __forceinline__ float tanh_fast(float x) { return fmaf(-2.f, rcp_fast(1.f + ex2_fast(2.8853900817779268f * x)), 1.f); }
 
 struct TcShared {
     uint64_t full[4];       // TMA bytes of the stage have landed
@@ -365,6 +375,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = make_idesc(bn, 0, 0);
+            const uint64_t desc0 = make_desc(smem_u32(smem), 16, 512, 4);
             uint32_t it = 0, lt = 0;
             for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
                 const uint32_t buf = lt & 1u;
@@ -377,14 +388,15 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     // the converters arrive on conv[s] only after they have seen full[s] (the TMA bytes) themselves
                     if (!mbar_wait(&sh->conv[s], ph, dead, status)) goto done;
                     tc_fence_after();
-                    const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
+                    // K-major, 64-byte swizzle: rows 64 B apart, 8-row groups 512 B apart; a k-step (8 values) is 32 B inside the
+                    // row.  Only the 14-bit start-address field (bytes >> 4) differs between the descriptors of a stage.
+                    const uint64_t a_hi0 = desc0 + (uint64_t)(((uint32_t)s * stage_bytes) >> 4);
 #pragma unroll
                     for (int ks = 0; ks < TC_BK / 8; ++ks) {
-                        // K-major, 64-byte swizzle: rows 64 B apart, 8-row groups 512 B apart; a k-step (8 values) is 32 B inside the row
-                        const uint64_t a_hi = make_desc(st + ks * 32, 16, 512, 4);
-                        const uint64_t a_lo = make_desc(st + a_bytes + ks * 32, 16, 512, 4);
-                        const uint64_t b_hi = make_desc(st + 2 * a_bytes + ks * 32, 16, 512, 4);
-                        const uint64_t b_lo = make_desc(st + 2 * a_bytes + b_bytes + ks * 32, 16, 512, 4);
+                        const uint64_t a_hi = a_hi0 + (uint64_t)(ks * 2);
+                        const uint64_t a_lo = a_hi + (a_bytes >> 4);
+                        const uint64_t b_hi = a_hi + (2 * a_bytes >> 4);
+                        const uint64_t b_lo = b_hi + (b_bytes >> 4);
                         tc_mma(acc, a_hi, b_hi, idesc, (kb > 0 || ks > 0) ? 1u : 0u);
                         tc_mma(acc, a_hi, b_lo, idesc, 1u);
                         tc_mma(acc, a_lo, b_hi, idesc, 1u);
