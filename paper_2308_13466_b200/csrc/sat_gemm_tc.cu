@@ -475,12 +475,24 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const float *base = EPI == EPI_RESID ? ep.resid : ep.addend;
                 const int piece = lane & 7;
                 const bool col_ok = pf_c + 4 * piece < pf_lim;
+                if (EPI == EPI_RESID) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int rr = (lane >> 3) + 4 * i;
-                    const float *rowp = reinterpret_cast<const float *>(__shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)pf_srow, rr));
-                    const bool valid = rowp != nullptr && col_ok;
-                    cp_async16(slot + rr * 128 + ((piece ^ (rr & 7)) << 4), (valid ? rowp : base) + pf_c + 4 * piece, valid);
+                    for (int i = 0; i < 8; ++i) {  // gathered rows: the row pointer lives in the lane that owns the row
+                        const int rr = (lane >> 3) + 4 * i;
+                        const float *rowp = reinterpret_cast<const float *>(__shfl_sync(0xffffffffu, (unsigned long long)(uintptr_t)pf_srow, rr));
+                        const bool valid = rowp != nullptr && col_ok;
+                        cp_async16(slot + rr * 128 + ((piece ^ (rr & 7)) << 4), (valid ? rowp : base) + pf_c + 4 * piece, valid);
+                    }
+                } else {
+                    // dense side operand: rows of the tile are ld_addend apart
+                    const int64_t prow0 = (pf_t / n_tiles_n) * TC_BM + q * 32 + (lane >> 3);
+                    const float *p0 = base + prow0 * ep.ld_addend + (int32_t)(pf_t % n_tiles_n) * bn + pf_c + 4 * piece;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr = (lane >> 3) + 4 * i;
+                        const bool valid = prow0 + 4 * i < M && col_ok;
+                        cp_async16(slot + rr * 128 + ((piece ^ (rr & 7)) << 4), valid ? p0 + (int64_t)(4 * i) * ep.ld_addend : base, valid);
+                    }
                 }
                 pf_c += 64;
                 if (pf_c >= bn) {
