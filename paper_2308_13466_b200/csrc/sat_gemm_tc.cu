@@ -11,7 +11,7 @@
 //   k_gemm_tc_mn  C[M x N] = A[R x M]^T B[R x N]   both operands MN-major, 128-byte swizzle with 32-byte atoms, split over R
 //                 (weight gradient)
 // Warp roles of k_gemm_tc_k: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..7 = converters,
-// warps 8..15 = epilogue (two per TMEM lane quadrant).  k_gemm_tc_mn: warps 0 / 1 as above, warps 2..5 convert during the
+// warps 8..15 = epilogue (two per TMEM lane quadrant); the K = h variants with a side operand use 2 + 12 instead.  k_gemm_tc_mn: warps 0 / 1 as above, warps 2..5 convert during the
 // main loop and then run the epilogue.  Every mbarrier wait is bounded; a timeout raises a status word and lets the CTA
 // drain (TMEM is freed, the kernel returns).
 #include <cuda.h>
@@ -269,28 +269,24 @@ struct TcShared {
 
 #define TC_CONV_THREADS 128
 #define TC_EPI_THREADS 128
-#define TCK_CONV_WARPS 6
-#define TCK_CONV_THREADS (TCK_CONV_WARPS * 32)
-/* The converter warps work in two groups on alternate k-blocks, so two stages are being split at any time.  Every stage
+/* 512 threads, 128 registers each: warp 0 TMA, warp 1 MMA, then the converter warps, then the epilogue warps.  The split
+ * between converters and epilogue depends on the epilogue variant (TckCfg): the K = h variants with a side operand have
+ * four k-blocks per tile and an epilogue bound by instruction issue, so they run 2 + 12 instead of 6 + 8.
+ * The converter warps work in two groups on alternate k-blocks, so two stages are being split at any time.  Every stage
  * count is even, hence a stage is always handled by the same group and each group meets the phases of its stages in
  * order (a parity wait must never be more than one phase ahead of its barrier). */
+#define TCK_THREADS 512
 #define TCK_CONV_GROUPS 2
-#define TCK_CONV_GROUP_THREADS (TCK_CONV_THREADS / TCK_CONV_GROUPS)
-#define TCK_EPI_WARPS 8
-#define TCK_EPI_THREADS (TCK_EPI_WARPS * 32)
-#define TCK_EPI_WARP0 (2 + TCK_CONV_WARPS)
-#define TCK_THREADS (64 + TCK_CONV_THREADS + TCK_EPI_THREADS) /* warp 0 TMA, warp 1 MMA, then the converter warps, then the epilogue warps: 512 threads, 128 registers each */
-#define TCK_OUT_BYTES (TCK_EPI_WARPS * 4096)  /* per epilogue warp one 32 x 32 fp32 staging tile for the TMA stores */
 
 // Epilogue variants.  The ones with a per-row side operand streamed from global memory (gathered residual rows, cached
-// LSTM input projection) keep a ring of 32 x 32 side tiles per epilogue warp in shared memory, filled by cp.async several
-// chunks ahead: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
+// LSTM input projection) keep a ring of 32 x 32 side tiles per epilogue warp in shared memory, filled by cp.async ahead of
+// the consumer: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
 // small K (the predictor width), so they give up main-loop stages for the ring.
 enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3 };
-template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, out_bytes = TCK_OUT_BYTES; };
-template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 3, out_bytes = TCK_OUT_BYTES; };
-template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, out_bytes = 0; };
-template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 4, out_bytes = 0; };
+template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
+template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 2, conv_warps = 2, epi_warps = 12, out_bytes = 0; };
 static_assert(TckCfg<EPI_PLAIN>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_RESID>::stages % TCK_CONV_GROUPS == 0 &&
                   TckCfg<EPI_LSTM>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_LSTM_ADD>::stages % TCK_CONV_GROUPS == 0,
               "a stage must always be split by the same converter group");
@@ -307,8 +303,8 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of k-block stages
 // and the two TMEM accumulator buffers let the TMA loads, the TF32 split, the MMAs and the epilogue of consecutive tiles
 // overlap.  A and B arrive as raw fp32 tiles; the converters round them to TF32 in place and write the residual tiles.
-// The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell) and runs on eight
-// warps, two per TMEM lane quadrant taking alternate 32-column chunks: with one warp per scheduler the epilogue was bound
+// The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell) and runs on eight or
+// twelve warps, two or three per TMEM lane quadrant taking 32-column chunks in turn: with one warp per scheduler the epilogue was bound
 // by instruction issue and load latency (9 - 14 us per 128 x 256 tile, longer than the main loop of a K = 256 tile).
 template <int EPI>
 __global__ void __launch_bounds__(TCK_THREADS, 1)
@@ -324,7 +320,11 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     constexpr int RING = TckCfg<EPI>::ring;
     uint8_t *out_stage = smem + (size_t)STAGES * stage_bytes;
     uint8_t *ring_base = out_stage + TckCfg<EPI>::out_bytes;
-    TcShared *sh = (TcShared *)(ring_base + (size_t)TCK_EPI_WARPS * RING * 4096);
+    constexpr int CONV_THREADS = TckCfg<EPI>::conv_warps * 32, CONV_GROUP_THREADS = CONV_THREADS / TCK_CONV_GROUPS;
+    constexpr int EPI_WARPS = TckCfg<EPI>::epi_warps, EPI_WARP0 = 2 + TckCfg<EPI>::conv_warps;
+    constexpr int CHUNK_STEP = 32 * (EPI_WARPS / 4);  // the EPI_WARPS / 4 warps of a TMEM lane quadrant take 32-column chunks in turn
+    static_assert(64 + CONV_THREADS + EPI_WARPS * 32 == TCK_THREADS && EPI_WARP0 % 4 == 0 && EPI_WARPS % 4 == 0, "warp roles");
+    TcShared *sh = (TcShared *)(ring_base + (size_t)EPI_WARPS * RING * 4096);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int32_t nkb = nkb1 + nkb2;
     const uint32_t acc_cols = 256;  // column stride between the two accumulator buffers
@@ -332,12 +332,12 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&sh->full[s], 1);
-            mbar_init(&sh->conv[s], TCK_CONV_GROUP_THREADS);
+            mbar_init(&sh->conv[s], CONV_GROUP_THREADS);
             mbar_init(&sh->empty[s], 1);
         }
         for (int i = 0; i < 2; ++i) {
             mbar_init(&sh->acc_full[i], 1);
-            mbar_init(&sh->acc_empty[i], TCK_EPI_THREADS);
+            mbar_init(&sh->acc_empty[i], EPI_WARPS * 32);
         }
         sh->dead = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -406,10 +406,10 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 tc_commit(&sh->acc_full[buf]);
             }
         }
-    } else if (warp < TCK_EPI_WARP0) {
+    } else if (warp < EPI_WARP0) {
         // ---------------- converters: TF32 split of the A and B tiles of every k-block ----------------
-        const int grp = (threadIdx.x - 64) / TCK_CONV_GROUP_THREADS;
-        const int ctid = (threadIdx.x - 64) % TCK_CONV_GROUP_THREADS;
+        const int grp = (threadIdx.x - 64) / CONV_GROUP_THREADS;
+        const int ctid = (threadIdx.x - 64) % CONV_GROUP_THREADS;
         uint32_t it = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
             for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
@@ -418,18 +418,18 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 const uint32_t ph = (it / STAGES) & 1u;
                 if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
-                split_tile_residual(st, st + a_bytes, a_bytes, ctid, TCK_CONV_GROUP_THREADS);
-                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, TCK_CONV_GROUP_THREADS);
+                split_tile_residual(st, st + a_bytes, a_bytes, ctid, CONV_GROUP_THREADS);
+                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, CONV_GROUP_THREADS);
                 fence_async_smem();
                 mbar_arrive(&sh->conv[s]);
             }
         }
     } else {
         // ---------------- epilogue ----------------
-        // warp w reads TMEM lanes 32 (w % 4) .. +31 = rows of the tile, one row per thread; the two warps of a lane quadrant
+        // warp w reads TMEM lanes 32 (w % 4) .. +31 = rows of the tile, one row per thread; the warps of a lane quadrant
         // take alternate 32-column chunks.
         constexpr bool LSTM = EPI == EPI_LSTM || EPI == EPI_LSTM_ADD;
-        const int e = warp - TCK_EPI_WARP0;
+        const int e = warp - EPI_WARP0;
         const int q = warp & 3;
         const int c_first = 32 * (e >> 2);
         uint8_t *obuf = out_stage + e * 4096;
@@ -494,7 +494,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         cp_async16(slot + rr * 128 + ((piece ^ (rr & 7)) << 4), valid ? p0 + (int64_t)(4 * i) * ep.ld_addend : base, valid);
                     }
                 }
-                pf_c += 64;
+                pf_c += CHUNK_STEP;
                 if (pf_c >= bn) {
                     pf_c = c_first;
                     pf_t += gridDim.x;
@@ -539,7 +539,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             if (c_first < bn) load_cell(c_first);
             if (!mbar_wait_warp(&sh->acc_full[buf], (lt >> 1) & 1u, dead, status, lane)) goto done;
             tc_fence_after();
-            for (int c0 = c_first; c0 < bn; c0 += 64) {
+            for (int c0 = c_first; c0 < bn; c0 += CHUNK_STEP) {
                 uint32_t r[32];
                 tc_ld32(tmem + buf * acc_cols + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                 if (RING > 0) {
@@ -577,7 +577,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                             for (int u = 0; u < 8; ++u)
                                 if (j0 + u < ep.lstm_h) cprev[u] = ep.lstm_c[sat_cell_offset(row, j0 + u, ep.lstm_h)];
                         }
-                        if (c0 + 64 < bn) load_cell(c0 + 64);
+                        if (c0 + CHUNK_STEP < bn) load_cell(c0 + CHUNK_STEP);
                         float sv[8], cv[8];
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
@@ -1008,7 +1008,7 @@ template <int EPI>
 static sat_status launch_tck(sat_ctx *ctx, const TckLaunch &L, const TcEpilogue &ep)
 {
     static bool attr_set = false;
-    const size_t smem = (size_t)TckCfg<EPI>::stages * L.stage_bytes + TckCfg<EPI>::out_bytes + (size_t)TCK_EPI_WARPS * TckCfg<EPI>::ring * 4096 +
+    const size_t smem = (size_t)TckCfg<EPI>::stages * L.stage_bytes + TckCfg<EPI>::out_bytes + (size_t)TckCfg<EPI>::epi_warps * TckCfg<EPI>::ring * 4096 +
                         sizeof(TcShared) + 1024;
     if (smem > 227 * 1024) return sat_fail(ctx, SAT_EINVAL, "tensor-core GEMM: shared-memory layout of %zu bytes does not fit", smem);
     if (!attr_set) {
