@@ -14,6 +14,8 @@ every value is drawn from the seeded generators of this package.
               100 -> 256 -> 256 -> 47, 32 partitions, history 4
   multilabel  717,000 nodes, 7 M distinct undirected edges, 300 -> 512 -> 512 -> 512 -> 100,
               100 independent Bernoulli(0.1) labels, 16 partitions, history 8
+  odd         (parity tests only) 6,000-node R-MAT graph, 50 -> 72 -> 40 -> 7, 3 partitions, history 3,
+              predictor width 24, non-zero biases everywhere: widths that are no multiple of a tile, a k-block or 8
 
 R-MAT graphs use (a, b, c, d) = (0.57, 0.19, 0.19, 0.05), get a seeded id permutation,
 and are then relabelled in BFS order so that contiguous id blocks are the partitions.
@@ -40,6 +42,8 @@ WORKLOADS = {
                   dims=[100, 256, 256, 47], M=32, tau=4, h=64, loss="ce"),
     "multilabel": dict(kind="rmat", scale=20, n=717_000, n_unique=7_000_000,
                        dims=[300, 512, 512, 512, 100], M=16, tau=8, h=64, loss="bce"),
+    "odd": dict(kind="rmat", scale=13, n=6_000, n_samples=40_000,
+                dims=[50, 72, 40, 7], M=3, tau=3, h=24, loss="ce", bias=0.1),
 }
 
 
@@ -73,8 +77,18 @@ class Workload:
         return int(self.col.shape[0]) + self.n
 
 
-def make_workload(name: str, seed: int = 0, shrink: int = 1, with_dense: bool = True) -> Workload:
+def _bias(seed: int, d: int, tag: str, scale: float) -> np.ndarray:
+    """Zeros (the benchmark workloads) or seeded values in (-scale sqrt(6/(1+d)), +...) x sqrt(1+d): order `scale`."""
+    if scale == 0.0:
+        return np.zeros(d, dtype=np.float32)
+    u = glorot_uniform(seed, 1, d, tag).reshape(d)          # uniform in +-sqrt(6 / (1 + d))
+    return (u * (scale / np.sqrt(6.0 / (1 + d)))).astype(np.float32)
+
+
+def make_workload(name: str, seed: int = 0, shrink: int = 1, with_dense: bool = True, **overrides) -> Workload:
+    """`overrides` replace entries of the workload's configuration (e.g. h=20, bias=0.05)."""
     cfg = dict(WORKLOADS[name])
+    cfg.update(overrides)
     part_given = None
     if cfg["kind"] == "sbm":
         n = cfg["n"] // shrink
@@ -113,15 +127,15 @@ def make_workload(name: str, seed: int = 0, shrink: int = 1, with_dense: bool = 
             wl.labels = bernoulli_labels(seed, n, dims[-1], 0.1)
     for l in range(1, L + 1):
         wl.W.append(glorot_uniform(seed, dims[l - 1], dims[l], f"W{l}"))
-        wl.b.append(np.zeros(dims[l], dtype=np.float32))
+        wl.b.append(_bias(seed, dims[l], f"b{l}", cfg.get("bias", 0.0)))
     for l in range(1, L):  # cached layers store H^(l), width dims[l]
         d, h = dims[l], min(cfg["h"], dims[l])
         wl.pred.append(dict(
             Wx=glorot_uniform(seed, d, 4 * h, f"pred{l}.Wx"),
             Uh=glorot_uniform(seed, h, 4 * h, f"pred{l}.Uh"),
-            b=np.zeros(4 * h, dtype=np.float32),
+            b=_bias(seed, 4 * h, f"pred{l}.b", cfg.get("bias", 0.0)),
             Wg=glorot_uniform(seed, h, d, f"pred{l}.Wg"),
-            bg=np.zeros(d, dtype=np.float32),
+            bg=_bias(seed, d, f"pred{l}.bg", cfg.get("bias", 0.0)),
             h=h,
         ))
     return wl

@@ -35,16 +35,20 @@ def _gather_H(res, P, l):
     return np.concatenate([res.per_part[m]["H"][l - 1] for m in range(P.M)])
 
 
-@pytest.mark.parametrize("name,shrink", [("tiny", 1), ("medium", 16)])
-def test_epochs_from_synchronised_state(B, name, shrink):
+@pytest.mark.parametrize("name,shrink,over,version", [
+    ("tiny", 1, {}, 0), ("medium", 16, {}, 0),
+    # widths that are no multiple of a tile / k-block / 8, non-zero biases in the layers and the predictor; with and
+    # without cached input projections (the oracle keeps no such state)
+    ("odd", 1, {}, 0), ("odd", 1, {}, 3), ("odd", 1, {"h": 20}, 0), ("odd", 1, {"h": 20}, 3), ("odd", 1, {"h": 32}, 3)])
+def test_epochs_from_synchronised_state(B, name, shrink, over, version):
     import torch
-    wl = make_workload(name, shrink=shrink)
+    wl = make_workload(name, shrink=shrink, **over)
     ep, P, dtil, perm = _setup(B, wl)
     try:
         cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
         W = [w.copy() for w in wl.W]
         b = [x.copy() for x in wl.b]
-        preds = pred_to_device(wl.pred, B)
+        preds = pred_to_device(wl.pred, B, version)
         for t in range(1, wl.tau + 3):
             Wd = [dev(w) for w in W]
             bd = [dev(x) for x in b]

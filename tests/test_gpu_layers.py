@@ -269,6 +269,7 @@ def test_five_node_predictor_numbers(B, five_node):
     ("dense", 64, [0, 9]),
     ("large", 128, [3, 31]),
     ("multilabel", 32, [1, 15]),
+    ("odd", 1, [0, 2]),       # 50 -> 72 -> 40 -> 7, predictor width 24, non-zero biases
 ])
 def test_shrunk_workloads_every_call(B, name, shrink, parts):
     """The four R-MAT workloads at reduced node count, full widths (602 / 300 / 100-wide ragged rows, 41 / 47 / 100
