@@ -242,12 +242,16 @@ def run_ours(args, wl):
     B.sat_profile_enable(ep.ctx, True)
     launches0 = B.sat_launch_count(ep.ctx)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     e0.record(stream)
-    for _ in range(args.steps):
+    marks[0].record(stream)
+    for i in range(args.steps):
         ep.step(W, b, preds, lr)
+        marks[i + 1].record(stream)
     e1.record(stream)
     barrier()
     ms = e0.elapsed_time(e1)
+    step_ms = [marks[i].elapsed_time(marks[i + 1]) for i in range(args.steps)]
     launches = B.sat_launch_count(ep.ctx) - launches0
     prof = B.sat_profile_read(ep.ctx)
     B.sat_profile_enable(ep.ctx, False)
@@ -351,12 +355,20 @@ def run_ours(args, wl):
             cpu = dict(value=edges / secs, unit="edges/s", cores=smp.cores, kind="oracle", seconds=secs,
                        sample=f"partitions 0..{k - 1} of {wl.M} of the {wl.name} workload (all layers fwd+bwd+predictor, "
                               f"LSTM for the cached nodes they read), ring full; {edges} edges")
+        # whole-epoch view: algorithmic bytes of every kernel family over the epoch time, against the HBM copy rate; the
+        # SpMM families also as the gather rate they sustain from L2 (entries x row bytes / time), which is what bounds them
+        alg_bytes = sum(v["bytes"] for v in prof.values()) / args.steps
+        epoch = dict(ms_median=float(np.median(step_ms)), ms_min=float(min(step_ms)),
+                     edge_passes_per_s=world * wl.nnz * 2 * wl.L / (ms_per_step * 1e-3),
+                     algorithmic_bytes=alg_bytes, hbm_frac=alg_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm"],
+                     spmm_gather_gbs={k: (prof[k]["flops"] / 2.0 * 4.0) / (prof[k]["ms"] * 1e-3) / 1e9
+                                      for k in ("spmm_fwd", "spmm_bwd") if prof.get(k, {}).get("ms", 0) > 0})
         line = dict(metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s", n_gpus=world,
                     steps=args.steps, warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
                     e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                              loss=e2e_loss, pipelined="inputs of step i+1 copied on a second stream while step i computes"),
-                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, kernel_families=families,
+                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, kernel_families=families,
                     loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
                     multi_gpu="replicas only" if world > 1 else None)
         print(json.dumps(line), flush=True)

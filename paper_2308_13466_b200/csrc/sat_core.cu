@@ -1060,6 +1060,7 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v)
     v->push0 = ctx->h_push_off[a];
     v->n_push = ctx->h_push_off[b] - v->push0;
     v->lnnz = ctx->h_lnnz_off[b] - ctx->h_lnnz_off[a];
+    v->hnnz = ctx->h_hrow_off.empty() ? 0 : ctx->h_hrow_off[b] - ctx->h_hrow_off[a];
     v->hlong0 = ctx->h_hlong_off[a];
     v->n_hlong = ctx->h_hlong_off[b] - v->hlong0;
     return SAT_OK;

@@ -187,6 +187,7 @@ struct PartView {
     int32_t push0, n_push;
     int32_t hlong0, n_hlong;  // long halo rows
     int64_t lnnz;             // local non-zeros (entries of A + I) of the selected rows
+    int64_t hnnz;             // of which entries with a halo column (= entries of the halo-row CSR)
 };
 sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
 

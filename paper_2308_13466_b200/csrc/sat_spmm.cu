@@ -148,7 +148,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     const int32_t d4 = (d + 3) / 4;
     // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once
     const double n_src = inner_only ? (double)v.n_rows : (double)v.n_rows + (double)v.n_halo;
-    const double n_ent = (double)v.lnnz;  // the backward uses the inner prefix of every row; counted in full here
+    const double n_ent = (double)(inner_only ? v.lnnz - v.hnnz : v.lnnz);  // the backward reads the inner prefix of every row
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
                    4.0 * n_ent + 12.0 * v.n_rows + 4.0 * n_src + 4.0 * d * (n_src + v.n_rows), 2.0 * n_ent * d);
     float *partial = nullptr;

@@ -37,6 +37,7 @@ def _gather_H(res, P, l):
 
 @pytest.mark.parametrize("name,shrink,over,version", [
     ("tiny", 1, {}, 0), ("medium", 16, {}, 0),
+    ("medium", 16, {"h": 256}, 0),     # wide predictor: 4h = 1024 gate columns, cell update as a kernel of its own
     # widths that are no multiple of a tile / k-block / 8, non-zero biases in the layers and the predictor; with and
     # without cached input projections (the oracle keeps no such state)
     ("odd", 1, {}, 0), ("odd", 1, {}, 3), ("odd", 1, {"h": 20}, 0), ("odd", 1, {"h": 20}, 3), ("odd", 1, {"h": 32}, 3)])
