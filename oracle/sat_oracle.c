@@ -362,3 +362,92 @@ double orc_loss_bce(int32_t n, int32_t n_labels, const float *Z, int64_t ld_z, c
     }
     return total;
 }
+
+/* ------------------------------------------------------------------------------------------
+ * Lossy storage of historical embeddings (Supplement, "Data Compression for Historical Embedding
+ * Storage"): the encoded-polyline scheme applied to every row of an embedding matrix.
+ *   q_j = round-half-away-from-zero(x_j * 10^p)   (the product of an fp32 value and 10^p, p <= 7, is exact in fp64)
+ *   e_0 = q_0,  e_j = q_j - q_{j-1}               (delta against the previous element of the row)
+ *   v   = e << 1, bitwise inverted when e < 0     (sign folded into bit 0)
+ *   5-bit groups of v, least significant first; every group but the last gets bit 0x20; each + 63 -> one ASCII byte
+ * Rows are independent; row r occupies bytes [offset[r], offset[r+1]).
+ * Decoding reverses the steps; x_hat_j = (float)((double)q_j / 10^p).
+ * ------------------------------------------------------------------------------------------ */
+static double pow10_int(int32_t p)
+{
+    double s = 1.0;
+    for (int32_t i = 0; i < p; ++i) s *= 10.0;
+    return s;
+}
+
+static int64_t codec_quantise(float x, double scale) { return (int64_t)llround((double)x * scale); }
+
+static int32_t codec_put(int64_t e, uint8_t *out) /* writes the bytes of one signed integer, returns their number */
+{
+    uint64_t v = (uint64_t)e << 1;
+    if (e < 0) v = ~v;
+    int32_t n = 0;
+    while (v >= 0x20) {
+        if (out) out[n] = (uint8_t)((0x20 | (v & 0x1f)) + 63);
+        ++n;
+        v >>= 5;
+    }
+    if (out) out[n] = (uint8_t)(v + 63);
+    return n + 1;
+}
+
+/* bytes per row into row_bytes[rows] */
+void orc_codec_row_bytes(int64_t rows, int32_t d, const float *X, int64_t ld, int32_t p, int32_t *row_bytes)
+{
+    const double scale = pow10_int(p);
+    for (int64_t r = 0; r < rows; ++r) {
+        int64_t prev = 0;
+        int32_t total = 0;
+        for (int32_t j = 0; j < d; ++j) {
+            const int64_t q = codec_quantise(X[r * ld + j], scale);
+            total += codec_put(q - prev, (uint8_t *)0);
+            prev = q;
+        }
+        row_bytes[r] = total;
+    }
+}
+
+/* offsets[rows + 1] must hold the exclusive prefix sums of the row sizes */
+void orc_codec_encode(int64_t rows, int32_t d, const float *X, int64_t ld, int32_t p, const int64_t *offsets, uint8_t *out)
+{
+    const double scale = pow10_int(p);
+    for (int64_t r = 0; r < rows; ++r) {
+        int64_t prev = 0;
+        uint8_t *o = out + offsets[r];
+        for (int32_t j = 0; j < d; ++j) {
+            const int64_t q = codec_quantise(X[r * ld + j], scale);
+            o += codec_put(q - prev, o);
+            prev = q;
+        }
+    }
+}
+
+/* returns 0, or 1 + the index of the first malformed row (wrong number of values, or a value that does not end) */
+int64_t orc_codec_decode(int64_t rows, int32_t d, const uint8_t *in, const int64_t *offsets, int32_t p, float *X, int64_t ld)
+{
+    const double scale = pow10_int(p);
+    for (int64_t r = 0; r < rows; ++r) {
+        int64_t pos = offsets[r], end = offsets[r + 1], q = 0;
+        for (int32_t j = 0; j < d; ++j) {
+            uint64_t v = 0;
+            int shift = 0;
+            for (;;) {
+                if (pos >= end) return r + 1;
+                const uint32_t c = (uint32_t)in[pos++] - 63u;
+                v |= (uint64_t)(c & 0x1f) << shift;
+                shift += 5;
+                if (c < 0x20) break;
+            }
+            const int64_t e = (v & 1) ? ~(int64_t)(v >> 1) : (int64_t)(v >> 1);
+            q += e;
+            X[r * ld + j] = (float)((double)q / scale);
+        }
+        if (pos != end) return r + 1;
+    }
+    return 0;
+}

@@ -393,3 +393,33 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
     if parts is None:
         cache.commit()
     return EpochResult(loss=total_loss, G_W=G_W, G_b=G_b, per_part=per_part, S=S, S_slots=sel)
+
+
+# ------------------------------------------------------------------------------------------
+# Lossy storage of historical embeddings (Supplement, "Data Compression for Historical Embedding Storage")
+# ------------------------------------------------------------------------------------------
+def codec_encode(X: np.ndarray, precision: int):
+    """Polyline-style encoding of every row of X (fp32 [rows, d]) at `precision` decimal places.
+    Returns (bytes uint8 [total], offsets int64 [rows + 1])."""
+    X = _f32(X)
+    rows, d = X.shape
+    sizes = np.zeros(rows, dtype=np.int32)
+    lib().orc_codec_row_bytes(C.c_int64(rows), C.c_int32(d), _p(X), C.c_int64(X.strides[0] // 4), C.c_int32(precision), _p(sizes))
+    offsets = np.zeros(rows + 1, dtype=np.int64)
+    np.cumsum(sizes, out=offsets[1:])
+    out = np.zeros(int(offsets[-1]), dtype=np.uint8)
+    lib().orc_codec_encode(C.c_int64(rows), C.c_int32(d), _p(X), C.c_int64(X.strides[0] // 4), C.c_int32(precision), _p(offsets), _p(out))
+    return out, offsets
+
+
+def codec_decode(data: np.ndarray, offsets: np.ndarray, d: int, precision: int) -> np.ndarray:
+    """Inverse of codec_encode: fp32 [rows, d]; raises on a malformed row."""
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    offsets = np.ascontiguousarray(offsets, dtype=np.int64)
+    rows = offsets.shape[0] - 1
+    X = np.zeros((rows, d), dtype=np.float32)
+    lib().orc_codec_decode.restype = C.c_int64
+    bad = lib().orc_codec_decode(C.c_int64(rows), C.c_int32(d), _p(data), _p(offsets), C.c_int32(precision), _p(X), C.c_int64(d))
+    if bad:
+        raise ValueError(f"codec_decode: malformed row {bad - 1}")
+    return X
