@@ -304,6 +304,34 @@ sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const 
 sat_status sat_dense_tn_static(void *cuda_stream, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B,
                                int32_t ldb, float *C, char *errbuf, int32_t errbuf_len);
 
+/* ---------------------------------------------------------------------------------------
+ * Embedding codec — lossy storage of historical embeddings (Supplement, "Data Compression for
+ * Historical Embedding Storage": the encoded-polyline scheme at a configurable decimal precision).
+ * Every row of an fp32 matrix is one delta-coded sequence:
+ *     q_j = round-half-away-from-zero(x_j * 10^p)      (evaluated in fp64, where the product is exact for p <= 7)
+ *     e_0 = q_0, e_j = q_j - q_{j-1};  v = e << 1, bitwise inverted when e < 0
+ *     5-bit groups of v, least significant first, bit 0x20 on every group but the last, each + 63 -> one ASCII byte
+ * Row r occupies bytes [row_offsets[r], row_offsets[r+1]).  Decoding: x_j = (float)((double)q_j / 10^p).
+ * The paper fixes neither the rounding of ties nor what the deltas run over; this is the reading taken here.
+ *
+ *   sat_codec_plan    sizes: writes row_offsets (DEVICE int64 [rows + 1], exclusive prefix sums of the row sizes) and
+ *                     returns the total in *total_bytes (HOST); synchronises the context's stream
+ *   sat_codec_encode  writes the bytes (DEVICE uint8, capacity >= the planned total) for the same x / precision
+ *   sat_codec_decode  inverse; rows whose bytes do not hold exactly d values raise the device status word
+ *                     (sat_sync_status returns SAT_EDATA) and are left partly written
+ *   sat_cache_requantise  stores the committed snapshot `age` (0 = newest) of cached layer `layer` the way a compressed
+ *                     ring would hold it: encode + decode in place (context scratch); *bytes (HOST, nullable) = size
+ *                     of the encoded snapshot.  Cached input projections of that snapshot are dropped.
+ * x: DEVICE [rows x ld] fp32, ld >= d; precision in 0..7.  SAT_EINVAL on bad arguments.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
+                          int64_t *row_offsets, int64_t *total_bytes);
+sat_status sat_codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
+                            const int64_t *row_offsets, uint8_t *out, int64_t out_capacity);
+sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d,
+                            int32_t precision, float *x, int32_t ld);
+sat_status sat_cache_requantise(sat_ctx *ctx, int32_t layer, int32_t age, int32_t precision, int64_t *bytes);
+
 /* Number of kernels this context has launched since creation (all entry points). */
 sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
 

@@ -59,6 +59,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise",
 ]
 
 
@@ -293,6 +294,33 @@ def sat_dense_tn(ctx, A, Bm, out):
     assert out.is_contiguous()
     _check(ctx, _lib.sat_dense_tn(ctx, C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A), C.c_int32(_ld(A)),
                                   _dev(Bm), C.c_int32(_ld(Bm)), _dev(out)))
+
+
+def sat_codec_plan(ctx, x, precision: int, row_offsets):
+    """Sizes of the encoded rows of x (CUDA fp32 [rows, d]): fills row_offsets (CUDA int64 [rows + 1]), returns the total."""
+    total = C.c_int64(0)
+    _check(ctx, _lib.sat_codec_plan(ctx, _dev(x), C.c_int32(_ld(x)), C.c_int64(x.shape[0]), C.c_int32(x.shape[1]), C.c_int32(precision),
+                                    _dev(row_offsets), C.byref(total)))
+    return int(total.value)
+
+
+def sat_codec_encode(ctx, x, precision: int, row_offsets, out):
+    """Writes the encoded rows of x into out (CUDA uint8, at least the planned total)."""
+    _check(ctx, _lib.sat_codec_encode(ctx, _dev(x), C.c_int32(_ld(x)), C.c_int64(x.shape[0]), C.c_int32(x.shape[1]), C.c_int32(precision),
+                                      _dev(row_offsets), _dev(out), C.c_int64(out.numel())))
+
+
+def sat_codec_decode(ctx, data, row_offsets, precision: int, x):
+    """Decodes rows into x (CUDA fp32 [rows, d]); malformed rows surface as SAT_EDATA from sat_sync_status."""
+    _check(ctx, _lib.sat_codec_decode(ctx, _dev(data), _dev(row_offsets), C.c_int64(x.shape[0]), C.c_int32(x.shape[1]), C.c_int32(precision),
+                                      _dev(x), C.c_int32(_ld(x))))
+
+
+def sat_cache_requantise(ctx, layer: int, age: int, precision: int) -> int:
+    """Replaces committed snapshot `age` of cached layer `layer` by its encode + decode image; returns the encoded size."""
+    total = C.c_int64(0)
+    _check(ctx, _lib.sat_cache_requantise(ctx, C.c_int32(layer), C.c_int32(age), C.c_int32(precision), C.byref(total)))
+    return int(total.value)
 
 
 def sat_dense_tn_static(stream: int, A, Bm, out):

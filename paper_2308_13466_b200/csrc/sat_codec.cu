@@ -1,0 +1,228 @@
+// Lossy storage of historical embeddings (Supplement, "Data Compression for Historical Embedding Storage"): the
+// encoded-polyline scheme applied to every row of an fp32 matrix.
+//   q_j = round-half-away-from-zero(x_j * 10^p)   (fp64: the product of an fp32 value and 10^p, p <= 7, is exact)
+//   e_0 = q_0, e_j = q_j - q_{j-1};  v = e << 1, bitwise inverted when e < 0
+//   5-bit groups of v, least significant first, bit 0x20 on all but the last, each + 63 -> one byte
+// One warp per row in all three kernels.  The code length of an element depends only on x_j and x_{j-1}, so sizes and
+// bytes are produced element-parallel (warp prefix sums give the byte positions); decoding finds the value boundaries of
+// 32 bytes at a time with a ballot (a byte below 0x20 after the -63 ends a value), lets the lane holding the last byte of
+// a value assemble it, and turns the deltas into values with a 64-bit warp prefix sum.  Integer and byte work: HBM-bound.
+#include "sat_internal.h"
+
+#define CODEC_MAX_GROUPS 13  /* 64 bits / 5 */
+
+__device__ __forceinline__ int64_t codec_quantise(float x, double scale) { return llround((double)x * scale); }
+__device__ __forceinline__ uint64_t codec_fold(int64_t e)
+{
+    const uint64_t v = (uint64_t)e << 1;
+    return e < 0 ? ~v : v;
+}
+__device__ __forceinline__ int codec_len(uint64_t v) { return v == 0 ? 1 : (64 - __clzll((long long)v) + 4) / 5; }
+
+// folded delta of this lane's element against its predecessor: the predecessor's quantised value comes from the lane
+// below, or, for lane 0, from the last element of the previous group of 32 (`carry`, updated here)
+__device__ __forceinline__ uint64_t codec_symbol(int64_t q, int lane, int64_t &carry)
+{
+    const int64_t up = __shfl_up_sync(0xffffffffu, q, 1);
+    const int64_t prev = lane == 0 ? carry : up;
+    carry = __shfl_sync(0xffffffffu, q, 31);
+    return codec_fold(q - prev);
+}
+
+__global__ void __launch_bounds__(256)
+k_codec_sizes(const float *__restrict__ x, int64_t ld, int64_t rows, int32_t d, double scale, int32_t *__restrict__ row_bytes)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const float *row = x + r * ld;
+    int32_t total = 0;
+    int64_t carry = 0;
+    for (int32_t j0 = 0; j0 < d; j0 += 32) {
+        const int32_t j = j0 + lane;
+        const int64_t q = j < d ? codec_quantise(row[j], scale) : 0;
+        const uint64_t v = codec_symbol(q, lane, carry);
+        if (j < d) total += codec_len(v);
+    }
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
+    if (lane == 0) row_bytes[r] = total;
+}
+
+__global__ void __launch_bounds__(256)
+k_codec_encode(const float *__restrict__ x, int64_t ld, int64_t rows, int32_t d, double scale, const int64_t *__restrict__ offsets,
+               uint8_t *__restrict__ out)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const float *row = x + r * ld;
+    int64_t run = offsets[r];
+    int64_t carry = 0;
+    for (int32_t j0 = 0; j0 < d; j0 += 32) {
+        const int32_t j = j0 + lane;
+        const int64_t q = j < d ? codec_quantise(row[j], scale) : 0;
+        const uint64_t v = codec_symbol(q, lane, carry);
+        const int len = j < d ? codec_len(v) : 0;
+        int incl = len;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        uint8_t *dst = out + run + (incl - len);
+        for (int k = 0; k < len; ++k) {
+            const uint32_t g = (uint32_t)(v >> (5 * k)) & 0x1fu;
+            dst[k] = (uint8_t)((k + 1 < len ? 0x20u : 0u) + g + 63u);
+        }
+        run += __shfl_sync(0xffffffffu, incl, 31);
+    }
+}
+
+// status bit 2: a row does not hold exactly d well-formed values
+__global__ void __launch_bounds__(256)
+k_codec_decode(const uint8_t *__restrict__ in, const int64_t *__restrict__ offsets, int64_t rows, int32_t d, double scale,
+               float *__restrict__ x, int64_t ld, int *__restrict__ status)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    const int64_t b0 = offsets[r], b1 = offsets[r + 1];
+    float *row = x + r * ld;
+    int64_t q_run = 0;
+    int32_t elem_base = 0;
+    bool bad = b1 < b0;
+    for (int64_t pos = b0; pos < b1; pos += 32) {
+        const int64_t p = pos + lane;
+        const bool valid = p < b1;
+        const uint32_t c = valid ? (uint32_t)in[p] - 63u : 0xffu;
+        if (valid && c > 63u) bad = true;  // outside the alphabet
+        const bool term = valid && c < 0x20u;
+        const unsigned tm = __ballot_sync(0xffffffffu, term);
+        int64_t e = 0;
+        if (term) {
+            int64_t s = p;  // first byte of the value that ends at p
+            while (s > b0 && p - s < CODEC_MAX_GROUPS) {
+                if ((uint32_t)in[s - 1] - 63u < 0x20u) break;
+                --s;
+            }
+            if (s > b0 && (uint32_t)in[s - 1] - 63u >= 0x20u) bad = true;  // more groups than a 64-bit value has
+            uint64_t v = 0;
+            for (int64_t t = s; t <= p; ++t) v |= (uint64_t)(((uint32_t)in[t] - 63u) & 0x1fu) << (5 * (int)(t - s));
+            e = (v & 1) ? ~(int64_t)(v >> 1) : (int64_t)(v >> 1);
+        }
+        int64_t incl = e;
+        for (int o = 1; o < 32; o <<= 1) {
+            const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (term) {
+            const int32_t elem = elem_base + __popc(tm & ((1u << lane) - 1u));
+            if (elem < d) row[elem] = (float)((double)(q_run + incl) / scale);
+            else bad = true;
+        }
+        q_run += __shfl_sync(0xffffffffu, incl, 31);
+        elem_base += __popc(tm);
+        if (pos + 32 >= b1 && lane == (int)(b1 - 1 - pos) && !term) bad = true;  // the last value never ends
+    }
+    if (elem_base != d) bad = true;
+    if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, 2);
+}
+
+static double codec_scale(int32_t precision)
+{
+    double s = 1.0;
+    for (int32_t i = 0; i < precision; ++i) s *= 10.0;
+    return s;
+}
+
+static sat_status codec_check(sat_ctx *ctx, const char *who, const void *x, int32_t ld, int64_t rows, int32_t d, int32_t precision)
+{
+    if (rows < 0 || d <= 0 || ld < d || precision < 0 || precision > 7 || (rows > 0 && !x))
+        return sat_fail(ctx, SAT_EINVAL, "%s: null tensor, bad shape or precision outside 0..7", who);
+    return SAT_OK;
+}
+
+static sat_status codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision, int64_t *row_offsets,
+                             int64_t *total_bytes)
+{
+    SAT_TRY(sat_ensure(ctx, ctx->buf_codec_sizes, (size_t)(rows > 0 ? rows : 1) * sizeof(int32_t)));
+    int32_t *sizes = (int32_t *)ctx->buf_codec_sizes.p;
+    if (rows > 0) {
+        ProfScope prof(ctx, SATK_CODEC, 4.0 * (double)rows * d + 12.0 * (double)rows, 0.0);
+        k_codec_sizes<<<(unsigned)cdiv64(rows * 32, 256), 256, 0, ctx->stream>>>(x, ld, rows, d, codec_scale(precision), sizes);
+        SAT_LAUNCHED(ctx);
+    }
+    SAT_TRY(sat_scan_i32(ctx, sizes, rows, row_offsets));
+    if (total_bytes) {
+        SAT_CUDA(ctx, cudaMemcpyAsync(total_bytes, row_offsets + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+        SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
+                                     int64_t *row_offsets, int64_t *total_bytes)
+{
+    if (!ctx) return SAT_EINVAL;
+    SAT_TRY(codec_check(ctx, "sat_codec_plan", x, ld, rows, d, precision));
+    if (!row_offsets || !total_bytes) return sat_fail(ctx, SAT_EINVAL, "sat_codec_plan: null row_offsets / total_bytes");
+    return codec_plan(ctx, x, ld, rows, d, precision, row_offsets, total_bytes);
+}
+
+static sat_status codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
+                               const int64_t *row_offsets, uint8_t *out, int64_t total)
+{
+    if (rows == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_CODEC, 4.0 * (double)rows * d + 8.0 * (double)rows + (double)total, 0.0);
+    k_codec_encode<<<(unsigned)cdiv64(rows * 32, 256), 256, 0, ctx->stream>>>(x, ld, rows, d, codec_scale(precision), row_offsets, out);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
+                                       const int64_t *row_offsets, uint8_t *out, int64_t out_capacity)
+{
+    if (!ctx) return SAT_EINVAL;
+    SAT_TRY(codec_check(ctx, "sat_codec_encode", x, ld, rows, d, precision));
+    if (!row_offsets || out_capacity < 0 || (rows > 0 && !out)) return sat_fail(ctx, SAT_EINVAL, "sat_codec_encode: null row_offsets / out");
+    int64_t total = 0;
+    SAT_CUDA(ctx, cudaMemcpyAsync(&total, row_offsets + rows, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (total > out_capacity)
+        return sat_fail(ctx, SAT_EINVAL, "sat_codec_encode: the rows need %lld bytes, the output holds %lld", (long long)total, (long long)out_capacity);
+    return codec_encode(ctx, x, ld, rows, d, precision, row_offsets, out, total);
+}
+
+static sat_status codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d, int32_t precision,
+                               float *x, int32_t ld, double bytes_in)
+{
+    if (rows == 0) return SAT_OK;
+    ProfScope prof(ctx, SATK_CODEC, 4.0 * (double)rows * d + 8.0 * (double)rows + bytes_in, 0.0);
+    k_codec_decode<<<(unsigned)cdiv64(rows * 32, 256), 256, 0, ctx->stream>>>(in, row_offsets, rows, d, codec_scale(precision), x, ld,
+                                                                             ctx->d_flag + 1);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d,
+                                       int32_t precision, float *x, int32_t ld)
+{
+    if (!ctx) return SAT_EINVAL;
+    SAT_TRY(codec_check(ctx, "sat_codec_decode", x, ld, rows, d, precision));
+    if (!row_offsets || (rows > 0 && !in)) return sat_fail(ctx, SAT_EINVAL, "sat_codec_decode: null row_offsets / in");
+    return codec_decode(ctx, in, row_offsets, rows, d, precision, x, ld, 0.0);
+}
+
+// encode + decode of one matrix in place through context scratch (what a compressed ring would hand back)
+sat_status sat_codec_roundtrip(sat_ctx *ctx, float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision, int64_t *bytes)
+{
+    SAT_TRY(sat_ensure(ctx, ctx->buf_codec_off, (size_t)(rows + 1) * sizeof(int64_t)));
+    int64_t *offsets = (int64_t *)ctx->buf_codec_off.p;
+    int64_t total = 0;
+    SAT_TRY(codec_plan(ctx, x, ld, rows, d, precision, offsets, &total));
+    SAT_TRY(sat_ensure(ctx, ctx->buf_codec_bytes, (size_t)(total > 0 ? total : 1)));
+    uint8_t *data = (uint8_t *)ctx->buf_codec_bytes.p;
+    SAT_TRY(codec_encode(ctx, x, ld, rows, d, precision, offsets, data, total));
+    SAT_TRY(codec_decode(ctx, data, offsets, rows, d, precision, x, ld, (double)total));
+    if (bytes) *bytes = total;
+    return SAT_OK;
+}

@@ -165,6 +165,9 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_gagg);
     sat_free_buf(ctx->buf_splitk);
     sat_free_buf(ctx->buf_lstm_c);
+    sat_free_buf(ctx->buf_codec_sizes);
+    sat_free_buf(ctx->buf_codec_off);
+    sat_free_buf(ctx->buf_codec_bytes);
     sat_free_buf(ctx->buf_lstm_s);
     sat_free_buf(ctx->buf_lstm_w);
     sat_free_buf(ctx->buf_pred_a);
@@ -189,9 +192,13 @@ extern "C" sat_status sat_sync_status(sat_ctx *ctx)
     if (ctx->cuda_failed) return SAT_ECUDA;
     SAT_CUDA(ctx, cudaMemcpyAsync(ctx->h_flag, ctx->d_flag + 1, sizeof(int), cudaMemcpyDeviceToHost, ctx->stream));
     SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
-    if (*ctx->h_flag) {
+    if (*ctx->h_flag & 1) {
         ctx->cuda_failed = true;
         return sat_fail(ctx, SAT_ECUDA, "a tensor-core kernel gave up waiting on a barrier (status %d)", *ctx->h_flag);
+    }
+    if (*ctx->h_flag & 2) {  // malformed codec input: reported once, the context stays usable
+        SAT_CUDA(ctx, cudaMemsetAsync(ctx->d_flag + 1, 0, sizeof(int), ctx->stream));
+        return sat_fail(ctx, SAT_EDATA, "sat_codec_decode: a row does not hold exactly d well-formed values");
     }
     return SAT_OK;
 }
@@ -207,7 +214,7 @@ extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
 // per-family device timing
 // =====================================================================================
 static const char *k_family_names[SATK_COUNT] = {"spmm_fwd", "spmm_bwd", "spmm_hrow", "gemm_nn", "gemm_nt", "gemm_tn",
-                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side"};
+                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side", "codec"};
 
 static void prof_clear(sat_ctx *ctx)
 {

@@ -46,7 +46,7 @@ struct CacheLayer {
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
-    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_COUNT
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_CODEC, SATK_COUNT
 };
 
 struct ProfRec {
@@ -116,6 +116,7 @@ struct sat_ctx {
     LayerState layers[SAT_MAX_LAYERS + 1];
 
     // ---- scratch ----
+    DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
         buf_wsplit, buf_wsplit2, buf_bias;
 };
@@ -176,6 +177,9 @@ static inline int32_t round_up4(int32_t x) { return (x + 3) & ~3; }
 // ---- device-side helpers implemented in the .cu files ----
 // exclusive scan: out[i] = sum_{j<i} in[j], i = 0..count (count+1 outputs), int64 results
 sat_status sat_scan_i32(sat_ctx *ctx, const int32_t *in, int64_t count, int64_t *out);
+
+// embedding codec (sat_codec.cu): encode + decode of one matrix in place; *bytes (host, nullable) = encoded size
+sat_status sat_codec_roundtrip(sat_ctx *ctx, float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision, int64_t *bytes);
 
 // row range / bases of a partition selector
 struct PartView {

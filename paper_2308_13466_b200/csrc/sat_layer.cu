@@ -121,6 +121,21 @@ extern "C" sat_status sat_cache_commit(sat_ctx *ctx)
     return SAT_OK;
 }
 
+extern "C" sat_status sat_cache_requantise(sat_ctx *ctx, int32_t layer, int32_t age, int32_t precision, int64_t *bytes)
+{
+    CHECK_CTX(ctx);
+    CacheLayer *c;
+    SAT_TRY(cache_layer(ctx, layer, &c, "sat_cache_requantise"));
+    if (age < 0 || age >= (ctx->n_valid < ctx->tau ? ctx->n_valid : ctx->tau))
+        return sat_fail(ctx, SAT_EINVAL, "sat_cache_requantise: age %d outside the %d committed snapshots", age, ctx->n_valid < ctx->tau ? ctx->n_valid : ctx->tau);
+    if (precision < 0 || precision > 7) return sat_fail(ctx, SAT_EINVAL, "sat_cache_requantise: precision outside 0..7");
+    const int32_t idx = ring_index(ctx, age);
+    SAT_TRY(sat_codec_roundtrip(ctx, ring_buf(ctx, c, idx), c->ld, ctx->n_slots, c->width, precision, bytes));
+    if (!c->proj_tag.empty()) c->proj_tag[idx] = 0;  // the cached projection was made from the unquantised snapshot
+    c->S_valid = false;
+    return SAT_OK;
+}
+
 extern "C" sat_status sat_cache_state(sat_ctx *ctx, int32_t *write_idx, int32_t *n_valid)
 {
     if (!ctx) return SAT_EINVAL;
