@@ -4,9 +4,9 @@
 //   e_0 = q_0, e_j = q_j - q_{j-1};  v = e << 1, bitwise inverted when e < 0
 //   5-bit groups of v, least significant first, bit 0x20 on all but the last, each + 63 -> one byte
 // One warp per row in all three kernels.  The code length of an element depends only on x_j and x_{j-1}, so sizes and
-// bytes are produced element-parallel (warp prefix sums give the byte positions); decoding finds the value boundaries of
-// 32 bytes at a time with a ballot (a byte below 0x20 after the -63 ends a value), lets the lane holding the last byte of
-// a value assemble it, and turns the deltas into values with a 64-bit warp prefix sum.  Integer and byte work: HBM-bound.
+// bytes are produced element-parallel (warp prefix sums give the byte positions); decoding takes 128 bytes at a time (a
+// byte below 0x20 after the -63 ends a value), lets the lane holding the last byte of a value assemble it, and turns the
+// deltas into values with a 64-bit warp prefix sum.  Integer and byte work: HBM-bound.
 #include "sat_internal.h"
 
 #define CODEC_MAX_GROUPS 13  /* 64 bits / 5 */
@@ -77,7 +77,11 @@ k_codec_encode(const float *__restrict__ x, int64_t ld, int64_t rows, int32_t d,
     }
 }
 
-// status bit 2: a row does not hold exactly d well-formed values
+// status bit 2: a row does not hold exactly d well-formed values.
+// 128 bytes per iteration, four consecutive bytes per lane.  A byte below 0x20 (after the -63) ends a value; the lane that
+// holds the last byte of a value assembles it (walking back over at most 12 continuation bytes, usually its own), the
+// lanes' delta sums go through one 64-bit warp prefix sum per window, and the element index of a value is the number of
+// terminators before it (one 32-bit prefix sum per window).
 __global__ void __launch_bounds__(256)
 k_codec_decode(const uint8_t *__restrict__ in, const int64_t *__restrict__ offsets, int64_t rows, int32_t d, double scale,
                float *__restrict__ x, int64_t ld, int *__restrict__ status)
@@ -90,39 +94,71 @@ k_codec_decode(const uint8_t *__restrict__ in, const int64_t *__restrict__ offse
     int64_t q_run = 0;
     int32_t elem_base = 0;
     bool bad = b1 < b0;
-    for (int64_t pos = b0; pos < b1; pos += 32) {
-        const int64_t p = pos + lane;
-        const bool valid = p < b1;
-        const uint32_t c = valid ? (uint32_t)in[p] - 63u : 0xffu;
-        if (valid && c > 63u) bad = true;  // outside the alphabet
-        const bool term = valid && c < 0x20u;
-        const unsigned tm = __ballot_sync(0xffffffffu, term);
-        int64_t e = 0;
-        if (term) {
-            int64_t s = p;  // first byte of the value that ends at p
-            while (s > b0 && p - s < CODEC_MAX_GROUPS) {
-                if ((uint32_t)in[s - 1] - 63u < 0x20u) break;
-                --s;
+    for (int64_t pos = b0; pos < b1; pos += 128) {
+        const int64_t p0 = pos + 4 * lane;
+        uint32_t c[4];
+        int n_term = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            c[k] = p0 + k < b1 ? (uint32_t)in[p0 + k] - 63u : 0xffu;
+            if (p0 + k < b1 && c[k] > 63u) bad = true;  // outside the alphabet
+            if (c[k] < 0x20u) ++n_term;
+        }
+        // values that end in this lane's bytes
+        int64_t e[4];
+        int64_t lane_sum = 0;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            e[k] = 0;
+            if (c[k] < 0x20u) {
+                uint64_t v = c[k] & 0x1fu;
+                int groups = 1;
+                // continuation bytes before it: first this lane's own, then earlier bytes of the row
+                int kk = k - 1;
+                int64_t s = p0 + k;  // first byte of the value found so far
+                while (groups < CODEC_MAX_GROUPS) {
+                    uint32_t cc;
+                    if (kk >= 0) cc = c[kk];
+                    else if (s > b0) cc = (uint32_t)in[s - 1] - 63u;
+                    else break;
+                    if (cc < 0x20u) break;
+                    v = (v << 5) | (cc & 0x1fu);
+                    --kk;
+                    --s;
+                    ++groups;
+                }
+                if (groups == CODEC_MAX_GROUPS && s > b0 && (uint32_t)in[s - 1] - 63u >= 0x20u) bad = true;  // longer than 64 bits
+                e[k] = (v & 1) ? ~(int64_t)(v >> 1) : (int64_t)(v >> 1);
+                lane_sum += e[k];
             }
-            if (s > b0 && (uint32_t)in[s - 1] - 63u >= 0x20u) bad = true;  // more groups than a 64-bit value has
-            uint64_t v = 0;
-            for (int64_t t = s; t <= p; ++t) v |= (uint64_t)(((uint32_t)in[t] - 63u) & 0x1fu) << (5 * (int)(t - s));
-            e = (v & 1) ? ~(int64_t)(v >> 1) : (int64_t)(v >> 1);
         }
-        int64_t incl = e;
+        // exclusive prefixes over the lanes: element index and running quantised value
+        int cnt_incl = n_term;
+        int64_t sum_incl = lane_sum;
         for (int o = 1; o < 32; o <<= 1) {
-            const int64_t up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+            const int cu = __shfl_up_sync(0xffffffffu, cnt_incl, o);
+            const int64_t su = __shfl_up_sync(0xffffffffu, sum_incl, o);
+            if (lane >= o) {
+                cnt_incl += cu;
+                sum_incl += su;
+            }
         }
-        if (term) {
-            const int32_t elem = elem_base + __popc(tm & ((1u << lane) - 1u));
-            if (elem < d) row[elem] = (float)((double)(q_run + incl) / scale);
-            else bad = true;
+        int32_t elem = elem_base + cnt_incl - n_term;
+        int64_t q = q_run + sum_incl - lane_sum;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            if (c[k] < 0x20u) {
+                q += e[k];
+                if (elem < d) row[elem] = (float)((double)q / scale);
+                else bad = true;
+                ++elem;
+            }
         }
-        q_run += __shfl_sync(0xffffffffu, incl, 31);
-        elem_base += __popc(tm);
-        if (pos + 32 >= b1 && lane == (int)(b1 - 1 - pos) && !term) bad = true;  // the last value never ends
+        q_run += __shfl_sync(0xffffffffu, sum_incl, 31);
+        elem_base += __shfl_sync(0xffffffffu, cnt_incl, 31);
     }
+    // the last byte of the row must end a value, and the row must hold exactly d values
+    if (lane == 0 && b1 > b0 && (uint32_t)in[b1 - 1] - 63u >= 0x20u) bad = true;
     if (elem_base != d) bad = true;
     if (__any_sync(0xffffffffu, bad) && lane == 0) atomicOr(status, 2);
 }
