@@ -1,19 +1,20 @@
 // Dense contractions on the 5th-generation tensor cores (tcgen05.mma kind::tf32, accumulators in TMEM,
 // operands staged in shared memory by TMA) with fp32-level accuracy from a two-term TF32 split:
-//     x = hi + lo,  hi = tf32(x), lo = tf32(x - hi)            (|x - hi - lo| <= 2^-22 |x|)
+//     x = hi + lo                                               (|x - hi - lo| <= 2^-21 |x|)
 //     A B ~= Ah Bh + Ah Bl + Al Bh                              (three MMAs per k-step, fp32 accumulate)
 // Activations and weights stay plain fp32 in global memory: TMA brings the fp32 tiles into shared memory and the
-// converter warps round them to TF32 in place and write the residual tiles next to them (element-wise, so the
-// swizzled layout never has to be decoded).  Weights are repacked once per call into the K-major operand layout.
+// converter warps write the residual tiles next to them, element-wise, so the swizzled layout never has to be decoded
+// (see "TF32 split of a shared-memory tile" below for the two variants).  Weights are repacked once per call into the
+// K-major operand layout.
 //
 //   k_gemm_tc_k   C[M x N] = A[M x K] B[N x K]^T   both operands K-major, 64-byte swizzle, BLOCK_K = 16, persistent
 //                 (layer transform, LSTM gates with two A operands or a cached projection, predictor output, input gradient)
 //   k_gemm_tc_mn  C[M x N] = A[R x M]^T B[R x N]   both operands MN-major, 128-byte swizzle with 32-byte atoms, split over R
 //                 (weight gradient)
-// Warp roles of k_gemm_tc_k: warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, warps 2..7 = converters,
-// warps 8..15 = epilogue (two per TMEM lane quadrant); the K = h variants with a side operand use 2 + 12 instead.  k_gemm_tc_mn: warps 0 / 1 as above, warps 2..5 convert during the
-// main loop and then run the epilogue.  Every mbarrier wait is bounded; a timeout raises a status word and lets the CTA
-// drain (TMEM is freed, the kernel returns).
+// Warp roles of k_gemm_tc_k (512 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer, then 6 converter and
+// 8 epilogue warps (two per TMEM lane quadrant), or 2 + 12 for the K = h variants with a side operand.  k_gemm_tc_mn:
+// warps 0 / 1 as above, warps 2..5 convert during the main loop and then run the epilogue.  Every mbarrier wait is
+// bounded; a timeout raises a status word and lets the CTA drain (TMEM is freed, the kernel returns).
 #include <cuda.h>
 
 #include "sat_internal.h"
@@ -302,10 +303,11 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 // Persistent: each CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  The shared-memory ring of k-block stages
 // and the two TMEM accumulator buffers let the TMA loads, the TF32 split, the MMAs and the epilogue of consecutive tiles
-// overlap.  A and B arrive as raw fp32 tiles; the converters round them to TF32 in place and write the residual tiles.
-// The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell) and runs on eight or
-// twelve warps, two or three per TMEM lane quadrant taking 32-column chunks in turn: with one warp per scheduler the epilogue was bound
-// by instruction issue and load latency (9 - 14 us per 128 x 256 tile, longer than the main loop of a K = 256 tile).
+// overlap.  A and B arrive as raw fp32 tiles, which the tensor core reads as the hi operands; the converters write the
+// residual tiles.  The epilogue is a template parameter (plain bias / ReLU / mask, gathered residual, fused LSTM cell)
+// and runs on eight or twelve warps, two or three per TMEM lane quadrant taking 32-column chunks in turn: with one warp
+// per scheduler the epilogue was bound by instruction issue and load latency (9 - 14 us per 128 x 256 tile, longer than
+// the main loop of a K = 256 tile).
 template <int EPI>
 __global__ void __launch_bounds__(TCK_THREADS, 1)
 k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB,
