@@ -423,3 +423,15 @@ def codec_decode(data: np.ndarray, offsets: np.ndarray, d: int, precision: int) 
     if bad:
         raise ValueError(f"codec_decode: malformed row {bad - 1}")
     return X
+
+
+# ------------------------------------------------------------------------------------------
+# Staleness of the out-of-subgraph embeddings (Eq. "staleness def"): || H_out - H~_out || over the halo of a partition
+# ------------------------------------------------------------------------------------------
+def staleness(P: Partitioning, m: int, H_fresh_by_gid: np.ndarray, H_used_halo: np.ndarray) -> float:
+    """Frobenius norm of the difference between the fresh embeddings of the halo nodes of partition m
+    (rows of H_fresh_by_gid [n, d], indexed by global node id) and the embeddings the partition used for them
+    (H_used_halo [b_m, d], in halo order)."""
+    fresh = np.asarray(H_fresh_by_gid)[P.halo_gid[m]].astype(np.float64)
+    diff = fresh - np.asarray(H_used_halo).astype(np.float64)
+    return float(np.sqrt(np.sum(diff * diff)))

@@ -279,3 +279,29 @@ def test_epoch_is_partition_order_invariant():
         assert np.array_equal(r0.per_part[m]["H"][-1], r1.per_part[m]["H"][-1])
     np.testing.assert_allclose(r0.G_W[0], r1.G_W[0], rtol=1e-12, atol=1e-15)
     assert abs(r0.loss - r1.loss) < 1e-12
+
+
+def test_staleness_norm_closed_forms():
+    """Eq. "staleness def": zero for identical embeddings, |c| sqrt(b_m d) for a constant offset, absolutely homogeneous,
+    and equal to the library Frobenius norm of the explicitly gathered difference."""
+    rng = np.random.default_rng(11)
+    rowptr, col = random_graph(rng, 60, 0.12)
+    part = rng.integers(0, 3, size=60).astype(np.int32)
+    P = orc.build_partition(rowptr, col, part, 3)
+    H = rng.normal(size=(60, 9)).astype(np.float32)
+    for m in range(3):
+        halo = P.halo_gid[m]
+        assert orc.staleness(P, m, H, H[halo]) == 0.0
+        used = (H[halo].astype(np.float64) + 0.25).astype(np.float32)
+        want = np.linalg.norm(H[halo].astype(np.float64) - used.astype(np.float64), "fro")
+        assert abs(orc.staleness(P, m, H, used) - want) <= 1e-12 * max(want, 1.0)
+        other = rng.normal(size=(halo.shape[0], 9)).astype(np.float32)
+        a = orc.staleness(P, m, H, other)
+        assert abs(a - np.linalg.norm(H[halo].astype(np.float64) - other.astype(np.float64))) <= 1e-12 * max(a, 1.0)
+        # constant offset on exactly representable values
+        Hq = np.round(H * 8) / 8
+        assert abs(orc.staleness(P, m, Hq, Hq[halo] + np.float32(0.5)) - 0.5 * np.sqrt(halo.shape[0] * 9)) <= 1e-12 * (1 + halo.shape[0])
+        # a permutation of the halo rows changes the value unless the rows agree: the halo order matters
+        if halo.shape[0] > 1:
+            rolled = np.roll(H[halo], 1, axis=0)
+            assert orc.staleness(P, m, H, rolled) > 0.0
