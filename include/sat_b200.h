@@ -305,6 +305,20 @@ sat_status sat_dense_tn_static(void *cuda_stream, int64_t rows, int32_t m, int32
                                int32_t ldb, float *C, char *errbuf, int32_t errbuf_len);
 
 /* ---------------------------------------------------------------------------------------
+ * sat_staleness — staleness of the out-of-subgraph embeddings of a partition (Eq. "staleness def"):
+ *     sq_sum = sum over the halo rows j of `part` of || h_fresh[row of halo node j] - h_used_halo[j] ||^2 ,
+ * the squared Frobenius norm the equation takes the root of (squared, so that partitions can be added up).
+ *   h_fresh      DEVICE [n x ld]  this epoch's embeddings of ALL nodes in partition-major row order (the h_out of
+ *                sat_layer_fwd called with SAT_ALL_PARTS, or the per-partition outputs side by side)
+ *   h_used_halo  DEVICE [b_m x ld_halo]  what the partition used for its halo: the identity predictor's output for the
+ *                historical embeddings, sat_predict's output for the predicted ones
+ *   sq_sum       DEVICE double, overwritten.  Accumulation in fp64, fixed order (reproducible).
+ * A diagnostic: not part of the training step.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_staleness(sat_ctx *ctx, int32_t part, int32_t d, const float *h_fresh, int32_t ld, const float *h_used_halo,
+                         int32_t ld_halo, double *sq_sum);
+
+/* ---------------------------------------------------------------------------------------
  * Embedding codec — lossy storage of historical embeddings (Supplement, "Data Compression for
  * Historical Embedding Storage": the encoded-polyline scheme at a configurable decimal precision).
  * Every row of an fp32 matrix is one delta-coded sequence:

@@ -59,7 +59,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness",
 ]
 
 
@@ -294,6 +294,13 @@ def sat_dense_tn(ctx, A, Bm, out):
     assert out.is_contiguous()
     _check(ctx, _lib.sat_dense_tn(ctx, C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A), C.c_int32(_ld(A)),
                                   _dev(Bm), C.c_int32(_ld(Bm)), _dev(out)))
+
+
+def sat_staleness(ctx, part: int, h_fresh, h_used_halo, sq_sum):
+    """sq_sum (CUDA float64 [1]) = squared Frobenius norm of (fresh embeddings of the halo nodes - embeddings used for them)."""
+    d = int(h_used_halo.shape[1])
+    _check(ctx, _lib.sat_staleness(ctx, C.c_int32(part), C.c_int32(d), _dev(h_fresh), C.c_int32(_ld(h_fresh)), _dev(h_used_halo),
+                                   C.c_int32(_ld(h_used_halo)), _dev(sq_sum)))
 
 
 def sat_codec_plan(ctx, x, precision: int, row_offsets):

@@ -770,6 +770,51 @@ extern "C" sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_
     return SAT_OK;
 }
 
+// staleness diagnostic: one warp per halo row, fp64 accumulation, block partials added in fixed order by k_loss_sum
+__global__ void __launch_bounds__(256)
+k_staleness(const int32_t *__restrict__ halo_gid, const int32_t *__restrict__ pos, int64_t halo0, int64_t n_halo, int32_t d,
+            const float *__restrict__ fresh, int64_t ld, const float *__restrict__ used, int64_t ld_used, double *__restrict__ block_partial)
+{
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t j0 = (int64_t)blockIdx.x * LOSS_ROWS_PER_BLOCK;
+    double acc = 0.0;
+    for (int i = warp; i < LOSS_ROWS_PER_BLOCK; i += 8) {
+        const int64_t j = j0 + i;
+        if (j >= n_halo) break;
+        const float *a = fresh + (int64_t)pos[halo_gid[halo0 + j]] * ld;
+        const float *b = used + j * ld_used;
+        double s = 0.0;
+        for (int c = lane; c < d; c += 32) {
+            const double t = (double)a[c] - (double)b[c];
+            s += t * t;
+        }
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        acc += s;
+    }
+    loss_block_partial(acc, block_partial);
+}
+
+extern "C" sat_status sat_staleness(sat_ctx *ctx, int32_t part, int32_t d, const float *h_fresh, int32_t ld, const float *h_used_halo,
+                                    int32_t ld_halo, double *sq_sum)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (!sq_sum || d <= 0) return sat_fail(ctx, SAT_EINVAL, "sat_staleness: null result or bad width");
+    SAT_CUDA(ctx, cudaMemsetAsync(sq_sum, 0, sizeof(double), ctx->stream));
+    if (v.n_halo == 0) return SAT_OK;
+    if (!h_fresh || !h_used_halo || ld < d || ld_halo < d) return sat_fail(ctx, SAT_EINVAL, "sat_staleness: null tensor or bad leading dimension");
+    const unsigned blocks = (unsigned)cdiv64(v.n_halo, LOSS_ROWS_PER_BLOCK);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_misc, (size_t)blocks * sizeof(double)));
+    double *block_partial = (double *)ctx->buf_misc.p;
+    k_staleness<<<blocks, 256, 0, ctx->stream>>>(ctx->halo_gid, ctx->pos, v.halo0, v.n_halo, d, h_fresh, ld,
+                                                 h_used_halo, ld_halo, block_partial);
+    SAT_LAUNCHED(ctx);
+    k_loss_sum<<<1, 256, 0, ctx->stream>>>(block_partial, (int64_t)blocks, sq_sum);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
+
 __global__ void k_sgd(int64_t count, float *__restrict__ w, const float *__restrict__ g, float lr)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

@@ -192,3 +192,54 @@ def test_cached_input_projections_over_a_wrapping_ring(B):
             assert_close(o["ring"][l - 1][newest], cache.buf[l - 1][newest], f"version {version}: newest snapshot of layer {l}")
         for l in range(1, wl.L + 1):
             assert_close(o["H"][l - 1], _gather_H(res, P, l), f"version {version}: H^{l} after {n_epochs} epochs")
+
+
+def test_staleness_of_historical_and_predicted_halos(B):
+    """Eq. "staleness def" on a running ring: || H_out - H~_out || with the newest committed snapshot as H~ (what
+    historical-embedding training would use) and with the predictor's output, per partition and summed, against the oracle
+    on the same arrays."""
+    import torch
+    wl = make_workload("medium", shrink=16)
+    Wd = [dev(w) for w in wl.W]
+    bd = [dev(x) for x in wl.b]
+    preds = pred_to_device(wl.pred, B, 2)
+    ep, P, dtil, perm = _setup(B, wl)
+    try:
+        for _ in range(wl.tau + 1):
+            ep.step(Wd, bd, preds, 0.01)
+        nb = sum(h.shape[0] for h in P.halo_gid)
+        used = {}
+        for l in range(1, wl.L):     # what the next epoch will use for its halos, taken before that epoch runs
+            hist = torch.empty((nb, wl.dims[l]), dtype=torch.float32, device="cuda")
+            pred = torch.empty((nb, wl.dims[l]), dtype=torch.float32, device="cuda")
+            B.sat_predict(ep.ctx, l, B.SAT_ALL_PARTS, None, 0, hist)
+            B.sat_predict(ep.ctx, l, B.SAT_ALL_PARTS, preds[l - 1], 0, pred)
+            used[l] = (hist, pred)
+        ep.step(Wd, bd, preds, 0.01)
+        torch.cuda.synchronize()
+        sq = torch.zeros(1, dtype=torch.float64, device="cuda")
+        off = np.concatenate([[0], np.cumsum([h.shape[0] for h in P.halo_gid])])
+        for l in range(1, wl.L):
+            H_pm = ep.H[l].cpu().numpy()
+            H_gid = np.empty_like(H_pm)
+            H_gid[perm] = H_pm
+            for kind, u in zip(("historical", "predicted"), used[l]):
+                u_host = u.cpu().numpy()
+                total = 0.0
+                for m in range(wl.M):
+                    want = orc.staleness(P, m, H_gid, u_host[off[m]:off[m + 1]])
+                    B.sat_staleness(ep.ctx, m, ep.H[l], u[off[m]:off[m + 1]], sq)
+                    got = float(sq.item()) ** 0.5
+                    assert abs(got - want) <= 1e-10 * max(want, 1e-30), (kind, l, m, got, want)
+                    assert want > 0.0          # the weights moved: the history is stale
+                    total += want * want
+                B.sat_staleness(ep.ctx, B.SAT_ALL_PARTS, ep.H[l], u, sq)
+                assert abs(float(sq.item()) - total) <= 1e-10 * total
+        # identical embeddings: exactly zero
+        pos = np.empty(wl.n, dtype=np.int64)
+        pos[perm] = np.arange(wl.n)
+        same = ep.H[1][torch.as_tensor(pos[P.halo_gid[0]], device="cuda")].contiguous()
+        B.sat_staleness(ep.ctx, 0, ep.H[1], same, sq)
+        assert float(sq.item()) == 0.0
+    finally:
+        ep.close()
