@@ -284,10 +284,10 @@ struct TcShared {
 // the consumer: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
 // small K (the predictor width), so they give up main-loop stages for the ring.
 enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3 };
-template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
-template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
-template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
-template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 2, conv_warps = 2, epi_warps = 12, out_bytes = 0; };
+template <int EPI> struct TckCfg { static constexpr bool b_presplit = false; static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_RESID> { static constexpr bool b_presplit = true; static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_LSTM> { static constexpr bool b_presplit = false; static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
+template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr bool b_presplit = true; static constexpr int stages = 2, ring = 2, conv_warps = 2, epi_warps = 12, out_bytes = 0; };
 static_assert(TckCfg<EPI_PLAIN>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_RESID>::stages % TCK_CONV_GROUPS == 0 &&
                   TckCfg<EPI_LSTM>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_LSTM_ADD>::stages % TCK_CONV_GROUPS == 0,
               "a stage must always be split by the same converter group");
@@ -311,7 +311,7 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 template <int EPI>
 __global__ void __launch_bounds__(TCK_THREADS, 1)
 k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapA2, const __grid_constant__ CUtensorMap mapB,
-            const __grid_constant__ CUtensorMap mapC, int use_tma_store, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t n_tiles_n, int64_t n_tiles, TcEpilogue ep, int *status)
+            const __grid_constant__ CUtensorMap mapBlo, const __grid_constant__ CUtensorMap mapC, int use_tma_store, int64_t M, int32_t N, int32_t nkb1, int32_t nkb2, int32_t bn, int32_t n_tiles_n, int64_t n_tiles, TcEpilogue ep, int *status)
 {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -366,10 +366,13 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) goto done;
                     uint8_t *st = smem + (size_t)s * stage_bytes;
-                    mbar_expect_tx(&sh->full[s], a_bytes + b_bytes);
+                    mbar_expect_tx(&sh->full[s], a_bytes + (TckCfg<EPI>::b_presplit ? 2 * b_bytes : b_bytes));
                     if (kb < nkb1) tma_load_2d(st, &mapA, &sh->full[s], kb * TC_BK, m0);
                     else tma_load_2d(st, &mapA2, &sh->full[s], (kb - nkb1) * TC_BK, m0);
                     tma_load_2d(st + 2 * a_bytes, &mapB, &sh->full[s], kb * TC_BK, n0);
+                    // the K = h variants read the residual plane of the weights from global memory as well: B is the same
+                    // for every tile there, and splitting it again per tile costs the two converter warps more than A does
+                    if (TckCfg<EPI>::b_presplit) tma_load_2d(st + 2 * a_bytes + b_bytes, &mapBlo, &sh->full[s], kb * TC_BK, n0);
                 }
             }
         }
@@ -421,7 +424,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 split_tile_residual(st, st + a_bytes, a_bytes, ctid, CONV_GROUP_THREADS);
-                split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, CONV_GROUP_THREADS);
+                if (!TckCfg<EPI>::b_presplit) split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, CONV_GROUP_THREADS);
                 fence_async_smem();
                 mbar_arrive(&sh->conv[s]);
             }
@@ -901,7 +904,7 @@ __global__ void k_split_weights(const float *__restrict__ W, int64_t ldw, int32_
         else if (kk >= k1_pad && kk - k1_pad < k2) x = transpose ? W2[(int64_t)(kk - k1_pad) * ldw2 + nn] : W2[(int64_t)nn * ldw2 + (kk - k1_pad)];
     }
     hi[i] = x;
-    (void)lo;
+    lo[i] = tf32_residual(x);  // second plane: read by the variants that do not split B in the kernel
 }
 
 // =====================================================================================
@@ -982,9 +985,9 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
     const int32_t bn = tile_n_for(n);
     const int32_t n_pad = (n + bn - 1) / bn * bn;
     const size_t plane = ((size_t)n_pad * k_pad * sizeof(float) + 255) & ~(size_t)255;
-    SAT_TRY(sat_ensure(ctx, buf, plane));
+    SAT_TRY(sat_ensure(ctx, buf, 2 * plane));
     out->hi = (float *)buf.p;
-    out->lo = nullptr;
+    out->lo = (float *)((char *)buf.p + plane);
     out->ld = k_pad;
     out->n_pad = n_pad;
     k_split_weights<<<(unsigned)cdiv64((int64_t)n_pad * k_pad, 256), 256, 0, ctx->stream>>>(W, ldw, k1, k1_pad, W2, ldw2, k2, n, n_pad, k_pad,
@@ -997,7 +1000,7 @@ static bool g_attr_mn = false;
 #define TC_SMEM_BUDGET (100 * 1024)
 
 struct TckLaunch {
-    CUtensorMap mA, mA2, mB, mC;
+    CUtensorMap mA, mA2, mB, mBlo, mC;
     int use_tma_store;
     int64_t m;
     int32_t n, nkb1, nkb2, bn, n_tiles_n;
@@ -1017,7 +1020,7 @@ static sat_status launch_tck(sat_ctx *ctx, const TckLaunch &L, const TcEpilogue 
         SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
-    k_gemm_tc_k<EPI><<<L.grid, TCK_THREADS, smem, ctx->stream>>>(L.mA, L.mA2, L.mB, L.mC, L.use_tma_store, L.m, L.n, L.nkb1, L.nkb2, L.bn, L.n_tiles_n,
+    k_gemm_tc_k<EPI><<<L.grid, TCK_THREADS, smem, ctx->stream>>>(L.mA, L.mA2, L.mB, L.mBlo, L.mC, L.use_tma_store, L.m, L.n, L.nkb1, L.nkb2, L.bn, L.n_tiles_n,
                                                                 L.n_tiles, ep, ctx->d_flag + 1);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
@@ -1037,7 +1040,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     if (eh.lstm_h > 0) alg_bytes += 4.0 * (double)m * eh.lstm_h * (eh.lstm_first ? 2.0 : 3.0) + (eh.addend ? 4.0 * (double)m * n : 0.0);
     else alg_bytes += 4.0 * (double)m * n * (eh.resid_idx ? 2.0 : 1.0);
     ProfScope prof(ctx, family, alg_bytes, 2.0 * (double)m * n * (k1 + k2));
-    CUtensorMap mA, mA2, mB, mC;
+    CUtensorMap mA, mA2, mB, mBlo, mC;
     const int use_tma_store = eh.lstm_h == 0 && ((eh.ldc & 3) == 0) && ((((uintptr_t)eh.C) & 15u) == 0);
     if (use_tma_store) SAT_TRY(make_map(ctx, &mC, eh.C, n, m, eh.ldc, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B));
     else memset(&mC, 0, sizeof(mC));
@@ -1045,6 +1048,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     if (A2) SAT_TRY(make_map(ctx, &mA2, A2, k2, m, lda2, TC_BK, TC_BM, CU_TENSOR_MAP_SWIZZLE_64B));
     else mA2 = mA;
     SAT_TRY(make_map(ctx, &mB, Bw.hi, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
+    SAT_TRY(make_map(ctx, &mBlo, Bw.lo, Bw.ld, Bw.n_pad, Bw.ld, TC_BK, bn, CU_TENSOR_MAP_SWIZZLE_64B));
     TcEpilogue ep;
     ep.C = eh.C;
     ep.ldc = eh.ldc;
@@ -1078,7 +1082,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->device);
     const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
     TckLaunch L;
-    L.mA = mA; L.mA2 = mA2; L.mB = mB; L.mC = mC;
+    L.mA = mA; L.mA2 = mA2; L.mB = mB; L.mBlo = mBlo; L.mC = mC;
     L.use_tma_store = use_tma_store;
     L.m = m; L.n = n; L.nkb1 = nkb1; L.nkb2 = nkb2; L.bn = bn; L.n_tiles_n = n_tiles_n; L.n_tiles = n_tiles;
     L.grid = grid;
