@@ -278,16 +278,20 @@ struct TcShared {
  * order (a parity wait must never be more than one phase ahead of its barrier). */
 #define TCK_THREADS 512
 #define TCK_CONV_GROUPS 2
+/* The weights' residual plane is made once by k_split_weights and fetched by TMA next to the raw plane: B is the same for
+ * every row tile, and splitting its tile again per k-block cost the converters twice what the A tile costs (measured:
+ * K = 256 transform 132 -> 118 us, K = 64 LSTM step 98 -> 85 us) for 16 KB more L2 -> SM traffic per k-block. */
+#define TCK_B_PRESPLIT 1
 
 // Epilogue variants.  The ones with a per-row side operand streamed from global memory (gathered residual rows, cached
 // LSTM input projection) keep a ring of 32 x 32 side tiles per epilogue warp in shared memory, filled by cp.async ahead of
 // the consumer: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
 // small K (the predictor width), so they give up main-loop stages for the ring.
 enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3 };
-template <int EPI> struct TckCfg { static constexpr bool b_presplit = false; static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
-template <> struct TckCfg<EPI_RESID> { static constexpr bool b_presplit = true; static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
-template <> struct TckCfg<EPI_LSTM> { static constexpr bool b_presplit = false; static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
-template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr bool b_presplit = true; static constexpr int stages = 2, ring = 2, conv_warps = 2, epi_warps = 12, out_bytes = 0; };
+template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
+template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
+template <> struct TckCfg<EPI_LSTM_ADD> { static constexpr int stages = 2, ring = 2, conv_warps = 2, epi_warps = 12, out_bytes = 0; };
 static_assert(TckCfg<EPI_PLAIN>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_RESID>::stages % TCK_CONV_GROUPS == 0 &&
                   TckCfg<EPI_LSTM>::stages % TCK_CONV_GROUPS == 0 && TckCfg<EPI_LSTM_ADD>::stages % TCK_CONV_GROUPS == 0,
               "a stage must always be split by the same converter group");
@@ -366,13 +370,11 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(&sh->empty[s], ph ^ 1u, dead, status)) goto done;
                     uint8_t *st = smem + (size_t)s * stage_bytes;
-                    mbar_expect_tx(&sh->full[s], a_bytes + (TckCfg<EPI>::b_presplit ? 2 * b_bytes : b_bytes));
+                    mbar_expect_tx(&sh->full[s], a_bytes + (TCK_B_PRESPLIT ? 2 * b_bytes : b_bytes));
                     if (kb < nkb1) tma_load_2d(st, &mapA, &sh->full[s], kb * TC_BK, m0);
                     else tma_load_2d(st, &mapA2, &sh->full[s], (kb - nkb1) * TC_BK, m0);
                     tma_load_2d(st + 2 * a_bytes, &mapB, &sh->full[s], kb * TC_BK, n0);
-                    // the K = h variants read the residual plane of the weights from global memory as well: B is the same
-                    // for every tile there, and splitting it again per tile costs the two converter warps more than A does
-                    if (TckCfg<EPI>::b_presplit) tma_load_2d(st + 2 * a_bytes + b_bytes, &mapBlo, &sh->full[s], kb * TC_BK, n0);
+                    if (TCK_B_PRESPLIT) tma_load_2d(st + 2 * a_bytes + b_bytes, &mapBlo, &sh->full[s], kb * TC_BK, n0);
                 }
             }
         }
@@ -424,7 +426,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                 if (!mbar_wait(&sh->full[s], ph, dead, status)) goto done;
                 uint8_t *st = smem + (size_t)s * stage_bytes;
                 split_tile_residual(st, st + a_bytes, a_bytes, ctid, CONV_GROUP_THREADS);
-                if (!TckCfg<EPI>::b_presplit) split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, CONV_GROUP_THREADS);
+                if (!TCK_B_PRESPLIT) split_tile_residual(st + 2 * a_bytes, st + 2 * a_bytes + b_bytes, b_bytes, ctid, CONV_GROUP_THREADS);
                 fence_async_smem();
                 mbar_arrive(&sh->conv[s]);
             }
