@@ -744,7 +744,7 @@ k_gemm_tc_mn(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ C
             for (int32_t kb = 0; kb < nkb; ++kb) {
                 const int s = kb % stages;
                 const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-                if (!mbar_wait(&sh->full[s], ph, dead, status)) break;
+                // the converters arrive on conv[s] only after they have seen full[s] (the TMA bytes) themselves
                 if (!mbar_wait(&sh->conv[s], ph, dead, status)) break;
                 tc_fence_after();
                 const uint32_t st = smem_u32(smem + (size_t)s * stage_bytes);
