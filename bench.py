@@ -35,7 +35,7 @@ if ROOT not in sys.path:
 # workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
 # gemm_nn: 302 MB = the 256-wide layer transform; gemm_side: 304 MB = the LSTM recurrence step (profiles/k_gemm_tc_k_medium.md);
 # spmm_fwd: 684 MB = the d = 256 launch (profiles/k_spmm_items_medium.md).
-NCU_TRAFFIC_BYTES = {"gemm_nn": 302.3e6, "spmm_fwd": 683.6e6, "gemm_side": 304.6e6}
+NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 683.6e6, "gemm_side": 304.4e6}
 
 # The contractions run on the tensor cores in TF32 (two-term split: three TF32 MMAs per product term).  The box's
 # measured tensor peak is a bf16 figure; TF32 is taken as measured bf16 x the nominal ratio 1.1 / 2.25 PFLOP/s.
