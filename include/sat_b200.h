@@ -68,7 +68,9 @@ sat_status sat_create(sat_ctx **ctx, int device, void *cuda_stream);
 sat_status sat_destroy(sat_ctx *ctx);
 /* Message of the most recent error on this context (valid until the next call). */
 const char *sat_last_error(const sat_ctx *ctx);
-/* Waits for the stream and returns SAT_ECUDA if any enqueued work failed. */
+/* Waits for the stream and reads the device status word: SAT_ECUDA if any enqueued work failed or a tensor-core kernel
+ * gave up waiting on one of its (bounded) barrier waits (sticky: the context is unusable afterwards); SAT_EDATA if
+ * sat_codec_decode met a malformed row (reported once, the context stays usable). */
 sat_status sat_sync_status(sat_ctx *ctx);
 
 /* ---------------------------------------------------------------------------------------
