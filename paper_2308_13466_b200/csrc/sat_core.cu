@@ -120,6 +120,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->hrow_ptr);
     dev_free(&ctx->hrow_pos);
     dev_free(&ctx->hrow_slot);
+    dev_free(&ctx->hrow_w);
     dev_free(&ctx->hlong);
     dev_free(&ctx->first_item);
     dev_free(&ctx->item_row);
@@ -679,7 +680,8 @@ __device__ __forceinline__ int32_t find_part(const int64_t *off, int32_t M, int6
 __global__ void k_hrow(const int64_t *__restrict__ rowptr, const int32_t *__restrict__ col, const int32_t *__restrict__ part,
                        const int32_t *__restrict__ pos, const int32_t *__restrict__ slot, const int32_t *__restrict__ halo_gid,
                        const int64_t *__restrict__ halo_off, int32_t M, int64_t nb, int32_t *__restrict__ cnt,
-                       const int64_t *__restrict__ hrow_ptr, int32_t *__restrict__ hrow_pos, int32_t *__restrict__ hrow_slot)
+                       const int64_t *__restrict__ hrow_ptr, int32_t *__restrict__ hrow_pos, int32_t *__restrict__ hrow_slot,
+                       const float *__restrict__ dinv, float *__restrict__ hrow_w)
 {
     int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     int lane = threadIdx.x & 31;
@@ -698,6 +700,7 @@ __global__ void k_hrow(const int64_t *__restrict__ rowptr, const int32_t *__rest
             int k = run + __popc(bi & ((1u << lane) - 1u));
             hrow_pos[o + k] = pos[v];
             hrow_slot[o + k] = slot[v];
+            hrow_w[o + k] = dinv[v];
         }
         run += __popc(bi);
     }
@@ -934,7 +937,7 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
         if (e == cudaSuccess && rc == SAT_OK) rc = dev_alloc(ctx, &ctx->hrow_ptr, ctx->nb + 1);
         if (e == cudaSuccess && rc == SAT_OK) {
             k_hrow<<<GRIDW(ctx->nb)>>>(ctx->rowptr, ctx->col, ctx->part, ctx->pos, ctx->slot, ctx->halo_gid, d_halo_off, M, ctx->nb,
-                                       t_hcnt, nullptr, nullptr, nullptr);
+                                       t_hcnt, nullptr, nullptr, nullptr, nullptr, nullptr);
             ctx->launches++;
             rc = sat_scan_i32(ctx, t_hcnt, ctx->nb, ctx->hrow_ptr);
         }
@@ -942,9 +945,10 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
         if (e == cudaSuccess && rc == SAT_OK) e = cudaStreamSynchronize(st);
         if (e == cudaSuccess && rc == SAT_OK) rc = dev_alloc(ctx, &ctx->hrow_pos, ctx->nnz_cut);
         if (e == cudaSuccess && rc == SAT_OK) rc = dev_alloc(ctx, &ctx->hrow_slot, ctx->nnz_cut);
+        if (e == cudaSuccess && rc == SAT_OK) rc = dev_alloc(ctx, &ctx->hrow_w, ctx->nnz_cut);
         if (e == cudaSuccess && rc == SAT_OK) {
             k_hrow<<<GRIDW(ctx->nb)>>>(ctx->rowptr, ctx->col, ctx->part, ctx->pos, ctx->slot, ctx->halo_gid, d_halo_off, M, ctx->nb,
-                                       nullptr, ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot);
+                                       nullptr, ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->dinv, ctx->hrow_w);
             ctx->launches++;
             e = cudaGetLastError();
         }

@@ -94,6 +94,7 @@ struct sat_ctx {
     int64_t *hrow_ptr = nullptr;  // [nb+1] halo-row CSR
     int32_t *hrow_pos = nullptr;  // [nnz_cut] partition-major row of the inner neighbour
     int32_t *hrow_slot = nullptr; // [nnz_cut] its cache slot
+    float *hrow_w = nullptr;      // [nnz_cut] its dinv (the entry's weight up to the row's own dinv)
     int64_t nnz_cut = 0;
     int32_t *hlong = nullptr;     // [n_hlong] halo positions of the halo rows longer than SAT_HROW_LONG
     int32_t n_hlong = 0;

@@ -190,7 +190,8 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
 // in group order through shared memory (fixed order: reproducible), group 0 adds the self term and stores.
 template <int G, int NV>
 __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos,
-                                                const int32_t *__restrict__ hrow_slot, const int32_t *__restrict__ halo_slot,
+                                                const int32_t *__restrict__ hrow_slot, const float *__restrict__ hrow_w,
+                                                const int32_t *__restrict__ halo_slot,
                                                 const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4,
                                                 const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
                                                 float *__restrict__ out_base, int64_t ld_out)
@@ -205,9 +206,8 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
     for (int64_t e = e0 + grp; e < e1; e += NG) {
-        const int32_t p = __ldg(hrow_pos + e);
-        const float w = __ldg(dinv_enc + p);
-        const int32_t c = by_slot ? __ldg(hrow_slot + e) : p;
+        const float w = __ldg(hrow_w + e);
+        const int32_t c = by_slot ? __ldg(hrow_slot + e) : __ldg(hrow_pos + e);
         const float *src = src_base + (int64_t)c * ld_src;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
@@ -237,19 +237,18 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
-            const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
+            const float *__restrict__ hrow_w, const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
             int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
             float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong)
 {
     if ((int32_t)blockIdx.x < n_hlong) {
-        hrow_long_block<G, NV>(hlong[hlong0 + blockIdx.x], hrow_ptr, hrow_pos, hrow_slot, halo_slot, dinv_enc, n, by_slot, d4, src_base, ld_src,
+        hrow_long_block<G, NV>(hlong[hlong0 + blockIdx.x], hrow_ptr, hrow_pos, hrow_slot, hrow_w, halo_slot, dinv_enc, n, by_slot, d4, src_base, ld_src,
                                self_src, out_base, ld_out);
         return;
     }
     const int lane = threadIdx.x & (G - 1);
     const int64_t gid = ((int64_t)(blockIdx.x - n_hlong) * blockDim.x + threadIdx.x) / G;
     if (gid >= n_halo) return;
-    const unsigned mask = group_mask<G>(threadIdx.x & 31);
     const int col0 = blockIdx.y * (G * NV);
     const int64_t j = halo0 + gid;
     const float du = __ldg(dinv_enc + n + j);
@@ -266,26 +265,29 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
     }
     const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
     if (e1 - e0 > SAT_HROW_LONG) return;  // handled by a block of its own (hrow_long_block)
-    for (int64_t eb = e0; eb < e1; eb += G) {
-        const int64_t e = eb + lane;
-        int32_t c = 0;
-        float w = 0.f;
-        if (e < e1) {
-            const int32_t p = __ldg(hrow_pos + e);
-            w = __ldg(dinv_enc + p);
-            c = by_slot ? __ldg(hrow_slot + e) : p;
-        }
-        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
-#pragma unroll 4
-        for (int q = 0; q < cnt; ++q) {
-            const int32_t cj = __shfl_sync(mask, c, q, G);
-            const float wj = __shfl_sync(mask, w, q, G);
-            const float *src = src_base + (int64_t)cj * ld_src;
+    // Halo rows are short (a handful of cut edges): every lane reads the entry's column and weight itself (one broadcast
+    // transaction per group) instead of sharing them through shuffles, four entries in flight; entries in order, so the
+    // sum has the same order as the long-row path's per-group partial sums.
+    const int32_t *__restrict__ ecol = by_slot ? hrow_slot : hrow_pos;
+    for (int64_t e = e0; e < e1; e += 4) {
+        int32_t c[4];
+        float w[4];
 #pragma unroll
-            for (int v = 0; v < NV; ++v) {
-                const int idx = col0 + lane + v * G;
-                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
-            }
+        for (int u = 0; u < 4; ++u) {
+            const bool ok = e + u < e1;
+            c[u] = ok ? __ldg(ecol + e + u) : -1;
+            w[u] = ok ? __ldg(hrow_w + e + u) : 0.f;
+        }
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx >= d4) continue;
+            float4 x[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) x[u] = c[u] >= 0 ? ld4(src_base + (int64_t)c[u] * ld_src + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (c[u] >= 0) fma4(acc[v], w[u], x[u]);
         }
     }
     float *o = out_base + j * ld_out;
@@ -301,7 +303,7 @@ static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4
                         const float *self_src, float *out_base, int32_t ld_out)
 {
     dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hlong), (unsigned)cdiv64(d4, G * NV));
-    k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->halo_slot, ctx->dinv_enc, ctx->n,
+    k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->hrow_w, ctx->halo_slot, ctx->dinv_enc, ctx->n,
                                                        v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out,
                                                        ctx->hlong, (int32_t)v.hlong0, (int32_t)v.n_hlong);
 }
