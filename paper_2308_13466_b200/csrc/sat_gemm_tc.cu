@@ -237,26 +237,6 @@ struct TcEpilogue {
     int64_t ld_addend;
 };
 
-// logistic and tanh from the hardware base-2 exponential and reciprocal (ex2.approx / rcp.approx, flush-to-zero forms:
-// one instruction each): absolute error of a few 1e-7, which is what matters for gate values in [0, 1] / [-1, 1].  Four and
-// five instructions per value; the LSTM epilogue is bound by instruction issue, so the libm versions (and even __expf /
-// __fdividef, which carry range handling) cost more than the memory traffic of the step.
-__device__ __forceinline__ float ex2_fast(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float rcp_fast(float x)
-{
-    float y;
-    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ float sigmoid_fast(float x) { return rcp_fast(1.f + ex2_fast(-1.4426950408889634f * x)); }
-// tanh x = 1 - 2 / (1 + e^{2x}); saturates correctly (e -> inf gives 1, e -> 0 gives -1)
-__device__ __forceinline__ float tanh_fast(float x) { return fmaf(-2.f, rcp_fast(1.f + ex2_fast(2.8853900817779268f * x)), 1.f); }
-
 struct TcShared {
     uint64_t full[4];       // TMA bytes of the stage have landed
     uint64_t conv[4];       // the converter threads have split the stage

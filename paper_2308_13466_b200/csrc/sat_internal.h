@@ -250,6 +250,28 @@ __host__ __device__ inline int64_t sat_cell_offset(int64_t row, int32_t j, int32
 }
 inline size_t sat_cell_floats(int64_t rows, int32_t h) { return (size_t)((rows + 31) / 32) * ((h + 7) / 8) * 256; }
 
+#ifdef __CUDACC__
+// logistic and tanh from the hardware base-2 exponential and reciprocal (ex2.approx / rcp.approx, flush-to-zero forms:
+// one instruction each): absolute error of a few 1e-7, which is what matters for gate values in [0, 1] / [-1, 1].  Four and
+// five instructions per value; the LSTM epilogue is bound by instruction issue, so the libm versions (and even __expf /
+// __fdividef, which carry range handling) cost more than the memory traffic of the step.
+__device__ __forceinline__ float ex2_fast(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_fast(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float sigmoid_fast(float x) { return rcp_fast(1.f + ex2_fast(-1.4426950408889634f * x)); }
+// tanh x = 1 - 2 / (1 + e^{2x}); saturates correctly (e -> inf gives 1, e -> 0 gives -1)
+__device__ __forceinline__ float tanh_fast(float x) { return fmaf(-2.f, rcp_fast(1.f + ex2_fast(2.8853900817779268f * x)), 1.f); }
+#endif
+
 struct TcWeights {         // weight operand as two fp32 planes [n_pad x ld] holding the TF32 hi / lo terms, K-major
     float *hi = nullptr, *lo = nullptr;
     int32_t ld = 0, n_pad = 0;

@@ -236,12 +236,12 @@ __global__ void k_lstm_cell_first(const float *__restrict__ proj, int64_t rows, 
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= rows * h) return;
     const float4 a = __ldg(reinterpret_cast<const float4 *>(proj) + t);  // (i, f, g, o) of unit t % h of row t / h
-    const float gi = 1.f / (1.f + expf(-a.x));
-    const float gg = tanhf(a.z);
-    const float go = 1.f / (1.f + expf(-a.w));
+    const float gi = sigmoid_fast(a.x);   // same gate arithmetic as the fused cell of the later steps
+    const float gg = tanh_fast(a.z);
+    const float go = sigmoid_fast(a.w);
     const float cn = gi * gg;
     c[sat_cell_offset(t / h, (int32_t)(t % h), h)] = cn;
-    s[t] = go * tanhf(cn);
+    s[t] = go * tanh_fast(cn);
 }
 
 // LSTM with cached input projections (parameter version promised by the caller): only ring buffers whose projection is
