@@ -309,7 +309,7 @@ sat_status sat_gemm_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const f
 // C = A^T B sums ~1e5 signed terms per element that cancel to a few 1e-3 of their magnitude (softmax gradients sum to
 // zero); the tensor-core contraction, whose accumulation truncates, was measured at 1e-4 relative error there against
 // 2e-5 for this kernel, which at this width costs about the same.
-//   block (x, y): rows [x * rows_per_block, ...), columns m = y * 256 + thread of A; NT accumulators per thread; B rows are
+//   block (x, y): rows [x * rows_per_block, ...), columns y * 256 .. + 255 of A, two per thread; B rows are
 //   staged in shared memory and broadcast; partial sums per row block, added in block order by k_splitk_reduce.
 // =====================================================================================
 #define TNN_STAGE 32
@@ -320,37 +320,39 @@ __device__ __forceinline__ void tnn_cp16(void *smem_dst, const void *gsrc, bool 
                  "r"(valid ? 16u : 0u)
                  : "memory");
 }
-// two stages of [TNN_STAGE x 256] of A and [TNN_STAGE x NT] of B, filled by cp.async while the previous stage is consumed
+// two stages of [TNN_STAGE x 256] of A and [TNN_STAGE x NT] of B, filled by cp.async while the previous stage is consumed;
+// 128 threads, each owning columns t and t + 128 of the block's 256 columns of A (2 NT accumulators: two FMAs per
+// broadcast shared-memory load of B)
 template <int NT>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(128)
 k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, const float *__restrict__ A, int64_t lda,
                  const float *__restrict__ B, int64_t ldb, float *__restrict__ part)
 {
     extern __shared__ __align__(16) float tnn_smem[];
     constexpr int STAGE_FLOATS = TNN_STAGE * 256 + TNN_STAGE * NT;
     const int32_t m0 = blockIdx.y * 256;
-    const int32_t col = m0 + threadIdx.x;
+    const int32_t col0 = m0 + threadIdx.x, col1 = col0 + 128;
     const int32_t m4 = (m + 3) & ~3, n4 = (n + 3) & ~3;
     const int64_t r_begin = (int64_t)blockIdx.x * rows_per_block;
     const int64_t r_end = r_begin + rows_per_block < rows ? r_begin + rows_per_block : rows;
     auto load_stage = [&](int s, int64_t r0) {
         float *As = tnn_smem + s * STAGE_FLOATS, *Bs = As + TNN_STAGE * 256;
 #pragma unroll
-        for (int k = 0; k < TNN_STAGE * 64 / 256; ++k) {
-            const int i = threadIdx.x + 256 * k, rr = i >> 6, c4 = i & 63;
+        for (int k = 0; k < TNN_STAGE * 64 / 128; ++k) {
+            const int i = threadIdx.x + 128 * k, rr = i >> 6, c4 = i & 63;
             const bool ok = r0 + rr < r_end && m0 + 4 * c4 < m4;
             tnn_cp16(As + rr * 256 + 4 * c4, ok ? A + (r0 + rr) * lda + m0 + 4 * c4 : A, ok);
         }
-        for (int i = threadIdx.x; i < TNN_STAGE * (NT / 4); i += 256) {
+        for (int i = threadIdx.x; i < TNN_STAGE * (NT / 4); i += 128) {
             const int rr = i / (NT / 4), j4 = i - rr * (NT / 4);
             const bool ok = r0 + rr < r_end && 4 * j4 < n4;
             tnn_cp16(Bs + rr * NT + 4 * j4, ok ? B + (r0 + rr) * ldb + 4 * j4 : B, ok);
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    float acc[NT];
+    float acc0[NT], acc1[NT];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) acc[j] = 0.f;
+    for (int j = 0; j < NT; ++j) acc0[j] = acc1[j] = 0.f;
     int s = 0;
     load_stage(0, r_begin);
     for (int64_t r0 = r_begin; r0 < r_end; r0 += TNN_STAGE, s ^= 1) {
@@ -362,25 +364,35 @@ k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, con
         }
         __syncthreads();
         const float *As = tnn_smem + s * STAGE_FLOATS, *Bs = As + TNN_STAGE * 256;
-#pragma unroll 4
+#pragma unroll 2
         for (int rr = 0; rr < TNN_STAGE; ++rr) {
-            const float a = As[rr * 256 + threadIdx.x];
+            const float a0 = As[rr * 256 + threadIdx.x], a1 = As[rr * 256 + 128 + threadIdx.x];
 #pragma unroll
             for (int j4 = 0; j4 < NT; j4 += 4) {
                 const float4 b = *reinterpret_cast<const float4 *>(Bs + rr * NT + j4);
-                acc[j4] = fmaf(a, b.x, acc[j4]);
-                acc[j4 + 1] = fmaf(a, b.y, acc[j4 + 1]);
-                acc[j4 + 2] = fmaf(a, b.z, acc[j4 + 2]);
-                acc[j4 + 3] = fmaf(a, b.w, acc[j4 + 3]);
+                acc0[j4] = fmaf(a0, b.x, acc0[j4]);
+                acc0[j4 + 1] = fmaf(a0, b.y, acc0[j4 + 1]);
+                acc0[j4 + 2] = fmaf(a0, b.z, acc0[j4 + 2]);
+                acc0[j4 + 3] = fmaf(a0, b.w, acc0[j4 + 3]);
+                acc1[j4] = fmaf(a1, b.x, acc1[j4]);
+                acc1[j4 + 1] = fmaf(a1, b.y, acc1[j4 + 1]);
+                acc1[j4 + 2] = fmaf(a1, b.z, acc1[j4 + 2]);
+                acc1[j4 + 3] = fmaf(a1, b.w, acc1[j4 + 3]);
             }
         }
         __syncthreads();  // the stage is refilled two iterations later
     }
-    if (col < m) {
-        float *o = part + ((int64_t)blockIdx.x * m + col) * n;
+    if (col0 < m) {
+        float *o = part + ((int64_t)blockIdx.x * m + col0) * n;
 #pragma unroll
         for (int j = 0; j < NT; ++j)
-            if (j < n) o[j] = acc[j];
+            if (j < n) o[j] = acc0[j];
+    }
+    if (col1 < m) {
+        float *o = part + ((int64_t)blockIdx.x * m + col1) * n;
+#pragma unroll
+        for (int j = 0; j < NT; ++j)
+            if (j < n) o[j] = acc1[j];
     }
 }
 
@@ -394,7 +406,7 @@ static sat_status launch_tn_narrow(sat_ctx *ctx, dim3 grid, int64_t rows, int64_
         SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tn_narrow<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         attr_set = true;
     }
-    k_gemm_tn_narrow<NT><<<grid, 256, smem, ctx->stream>>>(rows, rpb, m, n, A, lda, B, ldb, part);
+    k_gemm_tn_narrow<NT><<<grid, 128, smem, ctx->stream>>>(rows, rpb, m, n, A, lda, B, ldb, part);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
