@@ -37,6 +37,9 @@ if ROOT not in sys.path:
 # spmm_fwd: 684 MB = the d = 256 launch (profiles/k_spmm_items_medium.md).
 NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 683.6e6, "gemm_side": 304.4e6}
 
+# L2 -> SM streaming rate measured on this box with a TMA-only kernel (operand tiles resident in L2), in GB/s
+L2_STREAM_GBS = 9700.0
+
 # The contractions run on the tensor cores in TF32 (two-term split: three TF32 MMAs per product term).  The box's
 # measured tensor peak is a bf16 figure; TF32 is taken as measured bf16 x the nominal ratio 1.1 / 2.25 PFLOP/s.
 TF32_OVER_BF16 = 1.1 / 2.25
@@ -360,6 +363,12 @@ def run_ours(args, wl):
             roofline = dict(kernel=fam, bound="hbm", achieved=gbs, peak=peaks["hbm"], unit="GB/s", frac=gbs / peaks["hbm"],
                             traffic=NCU_TRAFFIC_BYTES.get(fam), peak_source=f"{peaks['source']} HBM copy bandwidth")
         roofline.update(launches=rec["calls"], ms_per_launch=per_launch_ms, share_of_step=rec["ms"] / ms)
+        if fam.startswith("spmm") and rec["flops"] > 0:
+            # the SpMM reads every neighbour row once per edge: that stream comes out of L2, not HBM (hit rate 63 % in the ncu
+            # capture), and its rate, not the HBM fraction above, is what bounds the kernel
+            gather = rec["flops"] / 2.0 * 4.0 / (rec["ms"] * 1e-3) / 1e9
+            roofline["l2_gather"] = dict(achieved=gather, unit="GB/s", reference=L2_STREAM_GBS, frac=gather / L2_STREAM_GBS,
+                                         reference_source="L2 -> SM rate of a pure TMA streaming kernel on this box (DESIGN.md section 8)")
         families = {k: dict(calls=v["calls"], ms_per_step=v["ms"] / args.steps,
                             gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else 0.0,
                             tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else 0.0)
