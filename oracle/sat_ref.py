@@ -435,3 +435,98 @@ def staleness(P: Partitioning, m: int, H_fresh_by_gid: np.ndarray, H_used_halo: 
     fresh = np.asarray(H_fresh_by_gid)[P.halo_gid[m]].astype(np.float64)
     diff = fresh - np.asarray(H_used_halo).astype(np.float64)
     return float(np.sqrt(np.sum(diff * diff)))
+
+
+# ------------------------------------------------------------------------------------------
+# O-12  embedding-predictor objective and its gradient (Eq. "predictor loss", Eq. "mini-batch training",
+#       Algorithm 1 "Embedding predictor update"); fp64 numpy, written out step by step
+# ------------------------------------------------------------------------------------------
+def _logistic(x):
+    return 1.0 / (1.0 + np.exp(-x))
+
+
+def pred_halo_weights(P: Partitioning, m: int, dtil):
+    """Entries of the predictor's graph convolution for the halo rows of partition m as three arrays
+    (halo row j, cache slot, weight p): the self term p_uu and p_uv for the neighbours v of u inside V_m."""
+    dt = np.asarray(dtil, dtype=np.float64)
+    halo = P.halo_gid[m]
+    nh = halo.shape[0]
+    counts = np.diff(P.hrow_ptr[m]).astype(np.int64)
+    rows_nb = np.repeat(np.arange(nh, dtype=np.int64), counts)
+    v = P.inner_gid[m][P.hrow_col[m]]
+    p_nb = 1.0 / np.sqrt(dt[halo[rows_nb]] * dt[v])
+    rows = np.concatenate([np.arange(nh, dtype=np.int64), rows_nb])
+    slots = np.concatenate([P.slot[halo], P.slot[v]]).astype(np.int64)
+    p = np.concatenate([1.0 / dt[halo], p_nb])
+    return rows, slots, p
+
+
+def pred_loss_grad(P: Partitioning, dtil, snaps, target, Wx, Uh, b, Wg, bg, row_weight=None):
+    """Objective of the embedding predictor of one cached layer and its gradient.
+
+    snaps: the valid snapshots [n_slots x d], oldest first (the temporal graph of the last tau epochs);
+    target: [n_slots x d] the embeddings pushed in the running epoch (what the prediction should have been).
+    Prediction for halo node u of partition m (Section "Embedding Predictor"): LSTM over the snapshots -> final
+    hidden state S; a_u = p_uu S_u + sum_{v in N(u) cap V_m} p_uv S_v; Hhat_u = newest_u + a_u Wg + bg.
+    Loss (Eq. "predictor loss" with the squared Euclidean norm, Eq. "mini-batch training" for the weights):
+        L = (1/M) sum_m sum_{u in B_m} w_u^(m) * 1/2 |Hhat_u - target_u|^2,
+    w_u^(m) = 1/b_m by default; row_weight[m] (length b_m) replaces it (1/|batch| on a sampled batch, 0 elsewhere).
+    Returns (L, dict(Wx, Uh, b, Wg, bg)) in float64."""
+    Wx, Uh, b, Wg, bg = (np.asarray(a, dtype=np.float64) for a in (Wx, Uh, b, Wg, bg))
+    h, d = Wg.shape
+    ns = P.n_slots
+    k = len(snaps)
+    X = [np.asarray(s, dtype=np.float64)[:, :d] for s in snaps]
+    T = np.asarray(target, dtype=np.float64)[:, :d]
+    # ---- LSTM over the snapshots, every cached node a sequence of length k, zero initial state ----
+    hs = [np.zeros((ns, h))]
+    cs = [np.zeros((ns, h))]
+    gates = []
+    for t in range(k):
+        z = X[t] @ Wx + hs[-1] @ Uh + b
+        gi, gf = _logistic(z[:, :h]), _logistic(z[:, h:2 * h])
+        gg, go = np.tanh(z[:, 2 * h:3 * h]), _logistic(z[:, 3 * h:])
+        c = gf * cs[-1] + gi * gg
+        gates.append((gi, gf, gg, go))
+        cs.append(c)
+        hs.append(go * np.tanh(c))
+    S = hs[-1]
+    newest = X[-1] if k > 0 else np.zeros((ns, d))
+    # ---- graph convolution on S, skip connection, loss ----
+    loss = 0.0
+    G = dict(Wx=np.zeros_like(Wx), Uh=np.zeros_like(Uh), b=np.zeros_like(b), Wg=np.zeros_like(Wg), bg=np.zeros_like(bg))
+    G_S = np.zeros((ns, h))
+    for m in range(P.M):
+        nh = P.halo_gid[m].shape[0]
+        if nh == 0:
+            continue
+        rows, slots, p = pred_halo_weights(P, m, dtil)
+        a = np.zeros((nh, h))
+        np.add.at(a, rows, p[:, None] * S[slots])
+        hs_m = P.halo_slot[m].astype(np.int64)
+        pred = newest[hs_m] + a @ Wg + bg
+        w = np.full(nh, 1.0 / nh) if row_weight is None or row_weight[m] is None else np.asarray(row_weight[m], dtype=np.float64)
+        diff = pred - T[hs_m]
+        loss += float(np.sum(w * 0.5 * np.sum(diff * diff, axis=1))) / P.M
+        E = diff * (w / P.M)[:, None]                  # dL / dHhat
+        G["bg"] += E.sum(axis=0)
+        G["Wg"] += a.T @ E
+        G_a = E @ Wg.T
+        np.add.at(G_S, slots, p[:, None] * G_a[rows])  # transpose of the graph convolution
+    # ---- back-propagation through time ----
+    dh = G_S
+    dc = np.zeros((ns, h))
+    for t in range(k - 1, -1, -1):
+        gi, gf, gg, go = gates[t]
+        tc = np.tanh(cs[t + 1])
+        dc = dc + dh * go * (1.0 - tc * tc)
+        dz = np.concatenate([dc * gg * gi * (1.0 - gi),            # input gate
+                             dc * cs[t] * gf * (1.0 - gf),         # forget gate
+                             dc * gi * (1.0 - gg * gg),            # candidate
+                             dh * tc * go * (1.0 - go)], axis=1)   # output gate
+        G["Wx"] += X[t].T @ dz
+        G["Uh"] += hs[t].T @ dz
+        G["b"] += dz.sum(axis=0)
+        dh = dz @ Uh.T
+        dc = dc * gf
+    return loss, G
