@@ -186,6 +186,28 @@ sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, const sat_pred
 sat_status sat_predict_state(sat_ctx *ctx, int32_t layer, float *S_host, int32_t h);
 
 /* ---------------------------------------------------------------------------------------
+ * sat_pred_grad — objective of the embedding predictor of cached layer `layer` and its gradient with respect to the
+ * predictor's parameters (Eq. "predictor loss" with the squared Euclidean norm; Eq. "mini-batch training" through
+ * row_weight; Algorithm 1 "Embedding predictor update": omega <- omega - eta_2 grad, e.g. with sat_sgd_step per array).
+ *   input   the temporal graph: the min(n_valid, tau) valid snapshots of the layer (oldest first);
+ *   target  the embeddings pushed in the RUNNING epoch (the ring's write buffer): call it after every partition's
+ *           sat_cache_update for this layer and before sat_cache_commit;
+ *   Hhat_u  as in sat_predict (LSTM -> S, graph convolution on S, skip connection), recomputed here with the
+ *           intermediate gate values kept for the backward pass;
+ *   L = (1/M) sum_m sum_{u in B_m} w_u * 1/2 |Hhat_u^(m) - target_u|^2,   w_u = 1/b_m, or row_weight[u] when given
+ *       (1/|batch| on the rows of a sampled batch, 0 elsewhere);
+ *   gradient: through the output layer (Wg, bg), the transposed graph convolution and back through time in the LSTM.
+ * params      DEVICE arrays as for sat_predict (version is ignored: nothing is reused from earlier calls)
+ * row_weight  DEVICE [sum_m b_m] (halo rows of all partitions, concatenated in partition order) or NULL
+ * g_Wx [d x 4h], g_Uh [h x 4h], g_b [4h], g_Wg [h x d], g_bg [d]   DEVICE, dense row-major, overwritten
+ * loss_host   HOST, may be NULL; when given the call synchronises the stream
+ * Scratch (owned by the context, kept): about k * |C| * 6h + sum_m b_m * (d + 2h) floats.
+ * Errors: SAT_ESTATE without a cache, SAT_EINVAL for null / misaligned arrays or h not a multiple of 4.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_pred_grad(sat_ctx *ctx, int32_t layer, const sat_pred_params *params, const float *row_weight, float *g_Wx,
+                         float *g_Uh, float *g_b, float *g_Wg, float *g_bg, double *loss_host);
+
+/* ---------------------------------------------------------------------------------------
  * sat_layer_fwd — local GCN layer forward (Appendix, forward of SAT):
  *     AGG = P_in h_in + P_out h_halo ;  Z = AGG W + bias ;  h_out = ReLU(Z) or Z.
  *   h_in   DEVICE [n_m x ld_in]   in-subgraph embeddings H_in^(l-1, m), rows in I_m order

@@ -59,7 +59,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad",
 ]
 
 
@@ -294,6 +294,15 @@ def sat_dense_tn(ctx, A, Bm, out):
     assert out.is_contiguous()
     _check(ctx, _lib.sat_dense_tn(ctx, C.c_int64(A.shape[0]), C.c_int32(A.shape[1]), C.c_int32(Bm.shape[1]), _dev(A), C.c_int32(_ld(A)),
                                   _dev(Bm), C.c_int32(_ld(Bm)), _dev(out)))
+
+
+def sat_pred_grad(ctx, layer: int, params, row_weight, g_Wx, g_Uh, g_b, g_Wg, g_bg, want_loss: bool = False):
+    """Gradient of the predictor objective of cached layer `layer` into the CUDA fp32 arrays g_* (dense, shapes of the
+    parameters); row_weight: CUDA fp32 [sum_m b_m] or None.  Returns the loss when want_loss (synchronises), else None."""
+    loss = C.c_double(0.0)
+    _check(ctx, _lib.sat_pred_grad(ctx, C.c_int32(layer), C.byref(params), _dev(row_weight), _dev(g_Wx), _dev(g_Uh), _dev(g_b),
+                                   _dev(g_Wg), _dev(g_bg), C.byref(loss) if want_loss else None))
+    return float(loss.value) if want_loss else None
 
 
 def sat_staleness(ctx, part: int, h_fresh, h_used_halo, sq_sum):

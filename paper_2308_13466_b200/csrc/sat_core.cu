@@ -178,6 +178,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_wsplit);
     sat_free_buf(ctx->buf_wsplit2);
     sat_free_buf(ctx->buf_bias);
+    sat_free_buf(ctx->buf_pred_train);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;
@@ -215,7 +216,7 @@ extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
 // per-family device timing
 // =====================================================================================
 static const char *k_family_names[SATK_COUNT] = {"spmm_fwd", "spmm_bwd", "spmm_hrow", "gemm_nn", "gemm_nt", "gemm_tn",
-                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side", "codec"};
+                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side", "codec", "pred_train"};
 
 static void prof_clear(sat_ctx *ctx)
 {

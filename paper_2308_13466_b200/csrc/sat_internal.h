@@ -46,7 +46,7 @@ struct CacheLayer {
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
-    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_CODEC, SATK_COUNT
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_CODEC, SATK_PRED_TRAIN, SATK_COUNT
 };
 
 struct ProfRec {
@@ -119,7 +119,7 @@ struct sat_ctx {
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2, buf_bias;
+        buf_wsplit, buf_wsplit2, buf_bias, buf_pred_train;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);

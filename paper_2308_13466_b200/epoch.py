@@ -106,10 +106,43 @@ class SatEpoch:
             B.sat_layer_bwd(ctx, m, l, g, W[l - 1], self.gW[l - 1], self.gb[l - 1], flags, g_in, None)
             g = g_in
 
-    def step(self, W, b, pred, lr: float | None = None):
-        """All partitions per launch.  W, b: lists of CUDA tensors; pred: list of sat_pred_params or None."""
+    def pred_update(self, pred, lr: float, max_steps: int = 1, min_gain: float | None = None, row_weight=None):
+        """Algorithm 1 "Embedding predictor update", to be called after the pushes of an epoch and before the commit:
+        up to max_steps gradient steps omega <- omega - lr grad L_Pred per cached layer, on the parameter tensors behind the
+        sat_pred_params; the parameter version (when one is used) is bumped.  min_gain switches early stopping on: the
+        steps of a layer end when a step lowered the loss by less than that fraction (this reads the loss back every
+        step).  row_weight: per cached layer a CUDA fp32 [sum_m b_m] of mini-batch weights, or None.
+        Returns the losses seen, per cached layer (empty lists without early stopping)."""
+        seen = []
+        for l in range(1, self.L):
+            p = pred[l - 1]
+            losses = []
+            if p is None:
+                seen.append(losses)
+                continue
+            if not hasattr(p, "_grads"):
+                p._grads = tuple(torch.zeros_like(t) for t in p._keep)
+            rw = None if row_weight is None else row_weight[l - 1]
+            for _ in range(max_steps):
+                loss = B.sat_pred_grad(self.ctx, l, p, rw, *p._grads, want_loss=min_gain is not None)
+                if min_gain is not None:
+                    losses.append(loss)
+                    if len(losses) > 1 and losses[-1] > (1.0 - min_gain) * losses[-2]:
+                        break
+                for t, g in zip(p._keep, p._grads):
+                    B.sat_sgd_step(self.ctx, t, g, lr)
+                if p.version:
+                    p.version += 1
+            seen.append(losses)
+        return seen
+
+    def step(self, W, b, pred, lr: float | None = None, pred_lr: float | None = None):
+        """All partitions per launch.  W, b: lists of CUDA tensors; pred: list of sat_pred_params or None.
+        pred_lr: also run one predictor update (pred_update) before the ring is committed."""
         self.loss_sum.zero_()
         self._forward_backward(B.SAT_ALL_PARTS, W, b, pred, 0, 0)
+        if pred_lr is not None and pred is not None:
+            self.pred_update(pred, pred_lr)
         B.sat_cache_commit(self.ctx)
         if lr is not None:
             for l in range(self.L):
