@@ -39,6 +39,7 @@ NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 683.6e6, "gemm_side": 304.4
 
 # predictor update period Delta-T of Algorithm 1 emulated by the run (epochs between two parameter-version bumps)
 PRED_PERIOD = 10
+PRED_LR = 0.01
 
 # L2 -> SM streaming rate measured on this box with a TMA-only kernel (operand tiles resident in L2), in GB/s
 L2_STREAM_GBS = 9700.0
@@ -354,6 +355,33 @@ def run_ours(args, wl):
     if not np.isfinite(e2e_loss) or not (0.5 * abs(loss) <= abs(e2e_loss) <= 2.0 * abs(loss)):
         raise RuntimeError(f"end-to-end path returned loss {e2e_loss}, device-resident path {loss}")
 
+    # ---- predictor update of Algorithm 1 (not part of the epoch metric: the epochs above only see its effect, the bumped
+    #      parameter version): one gradient step on the predictor objective per cached layer, between the pushes of an
+    #      epoch and the commit ----
+    pred_update = None
+    if rank == 0 and wl.L > 1:
+        ep.loss_sum.zero_()
+        ep._forward_backward(B.SAT_ALL_PARTS, W, b, preds, 0, 0)
+        first = ep.pred_update(preds, PRED_LR, max_steps=2, min_gain=0.0)      # warm-up (scratch allocation); reads the losses back
+        B.sat_profile_enable(ep.ctx, True)
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_upd = 3
+        l0 = B.sat_launch_count(ep.ctx)
+        p0.record(stream)
+        for _ in range(n_upd):
+            ep.pred_update(preds, PRED_LR)
+        p1.record(stream)
+        stream.synchronize()
+        upd_launches = (B.sat_launch_count(ep.ctx) - l0) // n_upd
+        upd_fam = {k: v["ms"] / n_upd for k, v in B.sat_profile_read(ep.ctx).items() if v["calls"]}
+        B.sat_profile_enable(ep.ctx, False)
+        B.sat_cache_commit(ep.ctx)
+        upd_ms = p0.elapsed_time(p1) / n_upd
+        pred_update = dict(what="sat_pred_grad + SGD step on the five parameter arrays, for each of the cached layers "
+                                "(forward with kept gates, loss against the pushed embeddings, back-propagation through time)",
+                           ms=upd_ms, launches=int(upd_launches), period_epochs=PRED_PERIOD, ms_per_epoch_amortised=upd_ms / PRED_PERIOD,
+                           loss_first_two_steps=[[float(x) for x in ls] for ls in first], kernel_families_ms=upd_fam)
+
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None
     if rank == 0 and wl.L > 1:
@@ -424,7 +452,7 @@ def run_ours(args, wl):
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
                     e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                              loss=e2e_loss, pipelined="inputs of step i+1 copied on a second stream while step i computes"),
-                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, codec=codec, kernel_families=families,
+                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, codec=codec, kernel_families=families,
                     loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
                     multi_gpu="replicas only" if world > 1 else None)
         print(json.dumps(line), flush=True)

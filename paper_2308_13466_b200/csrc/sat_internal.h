@@ -198,7 +198,7 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
 
 // SpMM family (sat_spmm.cu)
 //   out[row] = dinv[row] * sum_e dinv[col_e] * src(col_e), over all entries of the row (inner_only = 0)
-//   or over its inner prefix (inner_only = 1).  `in_base` / `halo_base` are the virtual bases of the
+//   or over its inner prefix (inner_only = 1), or over its halo suffix (inner_only = 2; in_base is not read).  `in_base` / `halo_base` are the virtual bases of the
 //   partition-major inner matrix and of the concatenated halo matrix (already offset for a single
 //   partition); `out_base` likewise.
 // omask (or null): bit mask [rows x omask_words] indexed like out_base; output components whose bit is 0 are written as 0

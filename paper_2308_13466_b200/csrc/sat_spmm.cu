@@ -53,9 +53,11 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
     const int32_t row = item_row[item];
     const int32_t k = item - first_item[row];
     const int64_t rb = lrowptr[row];
-    const int64_t re = inner_only ? rb + inner_cnt[row] : lrowptr[row + 1];
-    const int64_t e0 = rb + (int64_t)k * SAT_SPMM_CHUNK;
+    // inner_only: 0 = all entries, 1 = the inner prefix of the row, 2 = its halo suffix
+    const int64_t re = inner_only == 1 ? rb + inner_cnt[row] : lrowptr[row + 1];
+    int64_t e0 = rb + (int64_t)k * SAT_SPMM_CHUNK;
     const int64_t e1 = (e0 + SAT_SPMM_CHUNK < re) ? e0 + SAT_SPMM_CHUNK : re;
+    if (inner_only == 2 && e0 < rb + inner_cnt[row]) e0 = rb + inner_cnt[row];
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -147,8 +149,9 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     if (v.n_items == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
     // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once
-    const double n_src = inner_only ? (double)v.n_rows : (double)v.n_rows + (double)v.n_halo;
-    const double n_ent = (double)(inner_only ? v.lnnz - v.hnnz : v.lnnz);  // the backward reads the inner prefix of every row
+    const double n_src = inner_only == 1 ? (double)v.n_rows : inner_only == 2 ? (double)v.n_halo : (double)v.n_rows + (double)v.n_halo;
+    // the backward reads the inner prefix of every row, the transposed predictor convolution the halo suffix
+    const double n_ent = (double)(inner_only == 1 ? v.lnnz - v.hnnz : inner_only == 2 ? v.hnnz : v.lnnz);
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
                    4.0 * n_ent + 12.0 * v.n_rows + 4.0 * n_src + 4.0 * d * (n_src + v.n_rows), 2.0 * n_ent * d);
     float *partial = nullptr;
