@@ -317,15 +317,48 @@ class EpochResult:
     S_slots: object = None  # slots for which S was computed (None = all)
 
 
+class GradHistory:
+    """Gradient-side history (Appendix, back-propagation of SAT): for every layer j = 2..L the matrix
+    Q^(j) = sum_m P_out^(m)T D^(m, j) over the |C| boundary nodes, D = G o sigma'(Z) being the layer's pre-activation
+    gradient.  Row v holds what the partitions that use v as a halo node sent back for it.  `read[j-2]` is the snapshot
+    of the previous epoch (None before the first commit), `write[j-2]` collects the running epoch."""
+
+    def __init__(self, n_slots: int, widths):
+        self.n_slots, self.widths = n_slots, list(widths)        # widths[j-2] = d_j
+        self.read = [None] * len(self.widths)
+        self.write = [np.zeros((n_slots, w), dtype=np.float64) for w in self.widths]
+
+    def commit(self):
+        self.read = [w.astype(np.float32) for w in self.write]
+        self.write = [np.zeros((self.n_slots, w), dtype=np.float64) for w in self.widths]
+
+
+def halo_pre_gradient(P: Partitioning, m: int, dtil, D) -> np.ndarray:
+    """(P_out^T D)[u] = sum_{v in V_m, v ~ u} p_uv D[v] for the halo nodes u of partition m (float64)."""
+    dt = np.asarray(dtil, dtype=np.float64)
+    halo = P.halo_gid[m]
+    counts = np.diff(P.hrow_ptr[m]).astype(np.int64)
+    rows = np.repeat(np.arange(halo.shape[0], dtype=np.int64), counts)
+    loc = P.hrow_col[m].astype(np.int64)
+    p = 1.0 / np.sqrt(dt[halo[rows]] * dt[P.inner_gid[m][loc]])
+    out = np.zeros((halo.shape[0], D.shape[1]))
+    np.add.at(out, rows, p[:, None] * np.asarray(D, dtype=np.float64)[loc])
+    return out
+
+
 def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, loss_kind: str,
-              order=None, keep: bool = True, want_halo_grad: bool = False, parts=None, masks=None) -> EpochResult:
+              order=None, keep: bool = True, want_halo_grad: bool = False, parts=None, masks=None,
+              grad_hist: GradHistory = None) -> EpochResult:
     """pull (predict) -> forward -> push, per layer; loss; backward; commit the ring.
 
     pred: list (one entry per cached layer) of dict(Wx, Uh, b, Wg, bg) or None for the
     identity predictor (plain historical embeddings).  `parts` restricts the epoch to a
     subset of partitions (then the ring is not committed).  `masks[m][l-1]`, when given,
     replaces [Z^(l) > 0] in the backward of partition m (the derivative of ReLU where Z is
-    zero up to rounding is a tie: either sign decision is a correct result)."""
+    zero up to rounding is a tie: either sign decision is a correct result).
+    grad_hist switches the stale-gradient term of the Appendix's back-propagation on:
+    G_H^(t, l-1) = P_in^T D^(t, l) W^(l)T + [Q^(t-1, l) W^(l)T on the boundary rows], and this epoch's P_out^T D^(t, l) is
+    collected for the next one."""
     L = len(W)
     n = P.n
     ms = list(range(P.M)) if parts is None else list(parts)
@@ -382,6 +415,14 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
                 mask = np.ascontiguousarray(masks[m][l - 1], dtype=np.uint8)
             G_in, G_halo = layer_bwd(P, m, dtil, G, mask, rec["AGG"][l - 1], W[l - 1], G_W[l - 1], G_b[l - 1],
                                      want_in=(l > 1), want_halo=want_halo_grad)
+            if grad_hist is not None and l >= 2:
+                D = np.asarray(G, dtype=np.float64) * (1.0 if mask is None else mask)
+                grad_hist.write[l - 2][P.halo_slot[m]] += halo_pre_gradient(P, m, dtil, D)
+                if grad_hist.read[l - 2] is not None:
+                    stale = grad_hist.read[l - 2][P.push_slot[m]].astype(np.float64) @ np.asarray(W[l - 1], dtype=np.float64).T
+                    G_in = G_in.astype(np.float64)
+                    G_in[P.push_local[m]] += stale
+                    G_in = G_in.astype(np.float32)
             g_ins[l - 1] = G_in
             g_halos[l - 1] = G_halo
             G = G_in
@@ -392,6 +433,8 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
         per_part[m] = rec
     if parts is None:
         cache.commit()
+        if grad_hist is not None:
+            grad_hist.commit()
     return EpochResult(loss=total_loss, G_W=G_W, G_b=G_b, per_part=per_part, S=S, S_slots=sel)
 
 
