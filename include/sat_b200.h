@@ -238,6 +238,16 @@ sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in
  *                                        h_in (no-op when layer - 1 has no ReLU or has not run): saves the separate
  *                                        masking pass over the activations' gradient
  *               SAT_BWD_G_OUT_MASKED (4) g_out is such a pre-masked gradient (D of this layer): the mask is not applied again
+ *               SAT_BWD_GRAD_HISTORY (8) the stale-gradient term of SAT's back-propagation (Appendix):
+ *                                        G_H^(t, l-1) = P_in^T D^(t, l) W^T + P_out^T D^(t-1, l) W^T.  For layer >= 2 the call
+ *                                        (a) adds (P_out^T D)[u] of the selected partitions' halo nodes u to the running
+ *                                        epoch's history Q^(l) [|C| x d_out] at the cache slot of u, and (b) when a
+ *                                        committed history exists and g_in is wanted, adds Q_prev^(l)[slot(v)] W^T (with
+ *                                        this call's W) to g_in for the boundary rows v, under the same mask as g_in.
+ *                                        sat_cache_commit turns the running history into the committed one.  The history
+ *                                        buffers (2 x |C| x d_out floats per layer) are allocated on first use and dropped
+ *                                        on re-partitioning.  Partitions add to the history in call order (all partitions
+ *                                        of a SAT_ALL_PARTS call in index order).
  *   g_in   DEVICE [n_m x ld_gin] or NULL (layer 1);  g_halo DEVICE [b_m x ld_gh] or NULL
  * Requires the matching sat_layer_fwd to have run (SAT_ESTATE otherwise).  Results are
  * bit-reproducible from run to run (no floating-point atomics).
@@ -245,6 +255,7 @@ sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in
 #define SAT_BWD_ACCUMULATE 1
 #define SAT_BWD_MASK_G_IN 2
 #define SAT_BWD_G_OUT_MASKED 4
+#define SAT_BWD_GRAD_HISTORY 8
 sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g,
                          const float *W, float *g_W, float *g_b, int accumulate,
                          float *g_in, int32_t ld_gin, float *g_halo, int32_t ld_gh);
@@ -260,6 +271,14 @@ sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float 
  * ------------------------------------------------------------------------------------- */
 sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer, const float *h_out, int32_t ld);
 sat_status sat_cache_commit(sat_ctx *ctx);
+
+/* Gradient-side history of layer `layer` >= 2 (see SAT_BWD_GRAD_HISTORY), for checkpoints and tests.
+ * sat_grad_history_read: copies the committed history (which = 0; SAT_ESTATE before the first commit) or the running
+ * epoch's (which = 1) to HOST memory, dense [|C| x d_out].
+ * sat_grad_history_write: makes in_host (HOST, dense [|C| x width]) the committed history and clears the running one;
+ * in_host = NULL clears both and marks the committed one absent. */
+sat_status sat_grad_history_read(sat_ctx *ctx, int32_t layer, int which, float *out_host);
+sat_status sat_grad_history_write(sat_ctx *ctx, int32_t layer, int32_t width, const float *in_host);
 /* Ring bookkeeping: index of the write buffer in [0, tau] and number of valid snapshots. */
 sat_status sat_cache_state(sat_ctx *ctx, int32_t *write_idx, int32_t *n_valid);
 /* Copies snapshot `age` (0 = newest committed, ..., n_valid-1 = oldest; -1 = the write

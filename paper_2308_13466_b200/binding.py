@@ -21,7 +21,7 @@ SAT_ALL_PARTS = -1
 SAT_PART_GIVEN, SAT_PART_CONTIG_BLOCKS = 0, 1
 SAT_ACT_NONE, SAT_ACT_RELU = 0, 1
 SAT_LOSS_SOFTMAX_CE, SAT_LOSS_SIGMOID_BCE = 0, 1
-SAT_BWD_ACCUMULATE, SAT_BWD_MASK_G_IN, SAT_BWD_G_OUT_MASKED = 1, 2, 4
+SAT_BWD_ACCUMULATE, SAT_BWD_MASK_G_IN, SAT_BWD_G_OUT_MASKED, SAT_BWD_GRAD_HISTORY = 1, 2, 4, 8
 SAT_ROWS_INNER, SAT_ROWS_HALO = 0, 1
 SAT_CACHE_ZERO, SAT_CACHE_COPY = 0, 1
 
@@ -59,7 +59,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write",
 ]
 
 
@@ -303,6 +303,22 @@ def sat_pred_grad(ctx, layer: int, params, row_weight, g_Wx, g_Uh, g_b, g_Wg, g_
     _check(ctx, _lib.sat_pred_grad(ctx, C.c_int32(layer), C.byref(params), _dev(row_weight), _dev(g_Wx), _dev(g_Uh), _dev(g_b),
                                    _dev(g_Wg), _dev(g_bg), C.byref(loss) if want_loss else None))
     return float(loss.value) if want_loss else None
+
+
+def sat_grad_history_read(ctx, layer: int, which: int, n_slots: int, width: int) -> np.ndarray:
+    """Committed (which = 0) or running (which = 1) gradient-side history of layer `layer` as a host array [n_slots, width]."""
+    out = np.empty((n_slots, width), np.float32)
+    _check(ctx, _lib.sat_grad_history_read(ctx, C.c_int32(layer), C.c_int(which), out.ctypes.data_as(C.c_void_p)))
+    return out
+
+
+def sat_grad_history_write(ctx, layer: int, width: int, hist):
+    """hist: host array [n_slots, width] that becomes the committed history, or None to clear it."""
+    if hist is None:
+        _check(ctx, _lib.sat_grad_history_write(ctx, C.c_int32(layer), C.c_int32(width), None))
+        return
+    hist = np.ascontiguousarray(hist, dtype=np.float32)
+    _check(ctx, _lib.sat_grad_history_write(ctx, C.c_int32(layer), C.c_int32(width), hist.ctypes.data_as(C.c_void_p)))
 
 
 def sat_staleness(ctx, part: int, h_fresh, h_used_halo, sq_sum):

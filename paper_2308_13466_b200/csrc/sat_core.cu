@@ -147,6 +147,8 @@ static void free_layers(sat_ctx *ctx)
         dev_free(&ctx->layers[i].agg);
         dev_free(&ctx->layers[i].mask);
         ctx->layers[i] = LayerState();
+        dev_free(&ctx->ghist[i].buf);
+        ctx->ghist[i] = GradHist();
     }
 }
 
@@ -179,6 +181,9 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_wsplit2);
     sat_free_buf(ctx->buf_bias);
     sat_free_buf(ctx->buf_pred_train);
+    sat_free_buf(ctx->buf_ghist_halo);
+    sat_free_buf(ctx->buf_ghist_rows);
+    sat_free_buf(ctx->buf_ghist_out);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;

@@ -43,6 +43,15 @@ struct CacheLayer {
     std::vector<uint64_t> proj_tag;
 };
 
+// Gradient-side history of one layer j >= 2 (Appendix, back-propagation of SAT): Q^(j) = sum_m P_out^(m)T D^(m, j) over the
+// boundary nodes, two buffers [n_slots x ld]: buf + read_idx * plane is the previous epoch's, the other one collects the
+// running epoch (zeroed at commit).
+struct GradHist {
+    float *buf = nullptr;
+    int32_t width = 0, ld = 0, read_idx = 0;
+    bool has_read = false;
+};
+
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
@@ -115,11 +124,12 @@ struct sat_ctx {
 
     // ---- layers ----
     LayerState layers[SAT_MAX_LAYERS + 1];
+    GradHist ghist[SAT_MAX_LAYERS + 1];
 
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2, buf_bias, buf_pred_train;
+        buf_wsplit, buf_wsplit2, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
@@ -212,6 +222,10 @@ sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d
                       float *out, int32_t ld_out);
 sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d,
                        const float *src_base, int32_t ld_src, float *dst, int32_t ld_dst);
+// dst[dst_row[i]] += src[src_row ? src_row[i] : i] (o mask bits of the destination row, when given); the dst_row[i] of one
+// call must be distinct
+sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
+                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words);
 
 // GEMM family (sat_gemm.cu)
 // C[m x n] = A[m x k] B[k x n] (+ bias) with optional ReLU, sign-mask output, row-gathered residual add.

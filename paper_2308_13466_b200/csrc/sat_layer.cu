@@ -118,6 +118,53 @@ extern "C" sat_status sat_cache_commit(sat_ctx *ctx)
     ctx->write_idx = (ctx->write_idx + 1) % (ctx->tau + 1);
     ctx->n_valid = ctx->n_valid + 1 < ctx->tau ? ctx->n_valid + 1 : ctx->tau;
     for (int i = 0; i < ctx->n_cached; ++i) ctx->cache[i].S_valid = false;
+    // gradient-side history: what the epoch collected becomes readable, the other buffer starts the next epoch at zero
+    for (int l = 0; l <= SAT_MAX_LAYERS; ++l) {
+        GradHist &GH = ctx->ghist[l];
+        if (!GH.buf) continue;
+        const size_t plane = (size_t)ctx->n_slots * GH.ld;
+        GH.read_idx = 1 - GH.read_idx;
+        GH.has_read = true;
+        SAT_CUDA(ctx, cudaMemsetAsync(GH.buf + (size_t)(1 - GH.read_idx) * plane, 0, plane * sizeof(float), ctx->stream));
+    }
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_grad_history_read(sat_ctx *ctx, int32_t layer, int which, float *out_host)
+{
+    CHECK_CTX(ctx);
+    if (layer < 2 || layer > SAT_MAX_LAYERS || !out_host || (which != 0 && which != 1))
+        return sat_fail(ctx, SAT_EINVAL, "sat_grad_history_read: layer must be in [2, %d], which 0 or 1, output non-null", SAT_MAX_LAYERS);
+    GradHist &GH = ctx->ghist[layer];
+    if (!GH.buf || (which == 0 && !GH.has_read)) return sat_fail(ctx, SAT_ESTATE, "sat_grad_history_read: no such history for layer %d", layer);
+    const size_t plane = (size_t)ctx->n_slots * GH.ld;
+    const float *src = GH.buf + (size_t)(which == 0 ? GH.read_idx : 1 - GH.read_idx) * plane;
+    SAT_CUDA(ctx, cudaMemcpy2DAsync(out_host, (size_t)GH.width * 4, src, (size_t)GH.ld * 4, (size_t)GH.width * 4, (size_t)ctx->n_slots,
+                                    cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_grad_history_write(sat_ctx *ctx, int32_t layer, int32_t width, const float *in_host)
+{
+    CHECK_CTX(ctx);
+    if (!ctx->part_ok) return sat_fail(ctx, SAT_ESTATE, "sat_grad_history_write: call sat_partition first");
+    if (layer < 2 || layer > SAT_MAX_LAYERS || width <= 0) return sat_fail(ctx, SAT_EINVAL, "sat_grad_history_write: bad layer or width");
+    GradHist &GH = ctx->ghist[layer];
+    const int32_t ld_q = round_up4(width);
+    const size_t plane = (size_t)ctx->n_slots * ld_q;
+    if (!GH.buf || GH.width != width) {
+        SAT_TRY(dev_realloc(ctx, &GH.buf, (int64_t)(2 * plane > 0 ? 2 * plane : 1)));
+        GH.width = width;
+        GH.ld = ld_q;
+        GH.read_idx = 0;
+    }
+    SAT_CUDA(ctx, cudaMemsetAsync(GH.buf, 0, 2 * plane * sizeof(float), ctx->stream));
+    GH.has_read = in_host != nullptr;
+    if (in_host && ctx->n_slots > 0)
+        SAT_CUDA(ctx, cudaMemcpy2DAsync(GH.buf + (size_t)GH.read_idx * plane, (size_t)ld_q * 4, in_host, (size_t)width * 4, (size_t)width * 4,
+                                        (size_t)ctx->n_slots, cudaMemcpyHostToDevice, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     return SAT_OK;
 }
 
@@ -502,7 +549,9 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     if (g_halo && v.n_halo > 0 && (!ok_ld(ld_gh, d_in) || !aligned16(g_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: misaligned g_halo or bad ld_gh");
     const int flags = accumulate;
     accumulate = flags & SAT_BWD_ACCUMULATE;
-    if (flags & ~(SAT_BWD_ACCUMULATE | SAT_BWD_MASK_G_IN | SAT_BWD_G_OUT_MASKED)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: unknown flag bits");
+    if (flags & ~(SAT_BWD_ACCUMULATE | SAT_BWD_MASK_G_IN | SAT_BWD_G_OUT_MASKED | SAT_BWD_GRAD_HISTORY))
+        return sat_fail(ctx, SAT_EINVAL, "sat_layer_bwd: unknown flag bits");
+    const bool hist = (flags & SAT_BWD_GRAD_HISTORY) && layer >= 2 && ctx->n_slots > 0;
     const uint32_t *mask = (L.act == SAT_ACT_RELU && !(flags & SAT_BWD_G_OUT_MASKED)) ? L.mask + (int64_t)v.row0 * L.mask_words : nullptr;
     // ReLU mask of the layer below, applied to g_in on request (indexed by partition-major row like g_in)
     const uint32_t *mask_in = nullptr;
@@ -524,7 +573,7 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     const bool tc_x = want_dx && !g_halo && sat_use_tc(d_in, d_out);
     const float *D = g_out;  // D = g_out o [Z > 0]: materialised once for the tensor-core contractions
     int32_t ld_d = ld_g;
-    if (tc_w || tc_x) {
+    if (tc_w || tc_x || (hist && mask)) {
         float *dm = nullptr;
         if (mask) {
             ld_d = round_up4(d_out);
@@ -538,6 +587,31 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     if (tc_w && d_out <= 64) SAT_TRY(sat_gemm_tn_narrow(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
     else if (tc_w) SAT_TRY(sat_gemm_tc_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, D, ld_d, g_W, d_out, accumulate));
     else SAT_TRY(sat_gemm_tn(ctx, v.n_rows, d_in, d_out, agg, L.ld_in, g_out, ld_g, mask, L.mask_words, g_W, d_out, g_b, accumulate));
+    // gradient-side history, this epoch's contribution: Q_write[slot(u)] += (P_out^T D)[u] for the halo nodes u of the
+    // selected partitions, one partition after the other (the halo slots of one partition are distinct)
+    GradHist &GH = ctx->ghist[layer];
+    if (hist) {
+        const int32_t ld_q = round_up4(d_out);
+        const size_t plane = (size_t)ctx->n_slots * ld_q;
+        if (!GH.buf || GH.width != d_out) {
+            SAT_TRY(dev_realloc(ctx, &GH.buf, (int64_t)(2 * plane)));
+            SAT_CUDA(ctx, cudaMemsetAsync(GH.buf, 0, 2 * plane * sizeof(float), ctx->stream));
+            GH.width = d_out;
+            GH.ld = ld_q;
+            GH.read_idx = 0;
+            GH.has_read = false;
+        }
+        if (v.n_halo > 0 && v.n_rows > 0) {
+            SAT_TRY(sat_ensure(ctx, ctx->buf_ghist_halo, (size_t)v.n_halo * ld_q * sizeof(float)));
+            float *qh = (float *)ctx->buf_ghist_halo.p;
+            SAT_TRY(sat_spmm_hrow(ctx, v, d_out, D - (int64_t)v.row0 * ld_d, ld_d, 0, nullptr, qh - v.halo0 * (int64_t)ld_q, ld_q));
+            float *qw = GH.buf + (size_t)(1 - GH.read_idx) * plane;
+            for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m) {
+                const int64_t h0 = ctx->h_halo_off[m], cnt = ctx->h_halo_off[m + 1] - h0;
+                SAT_TRY(sat_scatter_add(ctx, nullptr, ctx->halo_slot + h0, cnt, d_out, qh + (h0 - v.halo0) * ld_q, ld_q, qw, ld_q, nullptr, 0));
+            }
+        }
+    }
     if (!want_dx) return SAT_OK;
     // G_AGG = D W^T
     const int32_t ld_ga = round_up4(d_in);
@@ -556,6 +630,27 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
     const float *ga_base = gagg - (int64_t)v.row0 * ld_ga;
     // G_in = P_in^T G_AGG: the inner block of P is symmetric, so P_in^T = P_in (inner prefix of every local row)
     if (g_in) SAT_TRY(sat_spmm(ctx, v, 1, d_in, ga_base, ld_ga, nullptr, 0, g_in - (int64_t)v.row0 * ld_gin, ld_gin, mask_in, mask_in_words));
+    // gradient-side history, the stale term: G_in[v] += (Q_read[slot(v)] W^T) o mask for the boundary rows v of the selection
+    if (hist && GH.has_read && g_in && v.n_push > 0) {
+        const size_t plane = (size_t)ctx->n_slots * GH.ld;
+        const float *qr = GH.buf + (size_t)GH.read_idx * plane;
+        SAT_TRY(sat_ensure(ctx, ctx->buf_ghist_rows, (size_t)v.n_push * GH.ld * sizeof(float)));
+        SAT_TRY(sat_ensure(ctx, ctx->buf_ghist_out, (size_t)v.n_push * ld_ga * sizeof(float)));
+        float *rows = (float *)ctx->buf_ghist_rows.p, *stale = (float *)ctx->buf_ghist_out.p;
+        SAT_TRY(sat_gather(ctx, ctx->push_slot + v.push0, v.n_push, d_out, qr, GH.ld, rows, GH.ld));
+        if (sat_use_tc(d_in, d_out)) {
+            TcWeights Wp;
+            SAT_TRY(sat_tc_weights(ctx, W, d_out, d_out, nullptr, 0, 0, d_in, 0, ctx->buf_wsplit, &Wp));
+            TcEpilogueHost eh;
+            eh.C = stale;
+            eh.ldc = ld_ga;
+            SAT_TRY(sat_gemm_tc(ctx, v.n_push, d_in, rows, GH.ld, d_out, nullptr, 0, 0, Wp, eh, SATK_GEMM_NT));
+        } else {
+            SAT_TRY(sat_gemm_nt(ctx, v.n_push, d_in, d_out, rows, GH.ld, nullptr, 0, W, d_out, stale, ld_ga));
+        }
+        SAT_TRY(sat_scatter_add(ctx, nullptr, ctx->push_row + v.push0, v.n_push, d_in, stale, ld_ga, g_in - (int64_t)v.row0 * ld_gin, ld_gin,
+                                mask_in, mask_in_words));
+    }
     // G_halo = P_out^T G_AGG over the halo-row CSR
     if (g_halo) SAT_TRY(sat_spmm_hrow(ctx, v, d_in, ga_base, ld_ga, 0, nullptr, g_halo - v.halo0 * (int64_t)ld_gh, ld_gh));
     return SAT_OK;

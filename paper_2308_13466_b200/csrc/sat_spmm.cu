@@ -376,3 +376,35 @@ sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
+
+__global__ void k_scatter_add_rows(const int32_t *__restrict__ src_row, const int32_t *__restrict__ dst_row, int64_t count, int32_t d4,
+                                   const float *__restrict__ src_base, int64_t ld_src, float *__restrict__ dst, int64_t ld_dst,
+                                   const uint32_t *__restrict__ mask, int32_t mask_words)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= count) return;
+    float4 x = ld4(src_base + (src_row ? (int64_t)src_row[i] : i) * ld_src + 4 * c);
+    const int64_t r = dst_row[i];
+    if (mask) mask4(x, mask, r * mask_words, c);
+    float4 *o = reinterpret_cast<float4 *>(dst + r * ld_dst + 4 * c);
+    float4 y = *o;
+    y.x += x.x;
+    y.y += x.y;
+    y.z += x.z;
+    y.w += x.w;
+    *o = y;
+}
+
+sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
+                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words)
+{
+    if (count == 0) return SAT_OK;
+    const int32_t d4 = (d + 3) / 4;
+    ProfScope prof(ctx, SATK_SCATTER, (12.0 * d + 8.0) * (double)count, 0.0);
+    k_scatter_add_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(src_row, dst_row, count, d4, src_base, ld_src, dst, ld_dst, mask,
+                                                                                   mask_words);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}

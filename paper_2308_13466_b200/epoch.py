@@ -81,7 +81,7 @@ class SatEpoch:
         return t[self.inner_off[m]:self.inner_off[m + 1]]
 
     # ---- one epoch ----------------------------------------------------------------
-    def _forward_backward(self, m: int, W, b, pred, accumulate: int, reuse_state: int):
+    def _forward_backward(self, m: int, W, b, pred, accumulate: int, reuse_state: int, grad_history: bool = False):
         ctx, L = self.ctx, self.L
         h_in = self.rows(self.X_in, m)
         for l in range(1, L + 1):
@@ -103,6 +103,8 @@ class SatEpoch:
             g_in = self.rows(self.G[l - 1], m) if l > 1 else None
             # the gradient handed down is written already multiplied by the ReLU mask of the layer below (no separate pass)
             flags = accumulate | (B.SAT_BWD_MASK_G_IN if l > 1 else 0) | (B.SAT_BWD_G_OUT_MASKED if l < L else 0)
+            if grad_history and l > 1:
+                flags |= B.SAT_BWD_GRAD_HISTORY      # stale-gradient term of the Appendix's back-propagation
             B.sat_layer_bwd(ctx, m, l, g, W[l - 1], self.gW[l - 1], self.gb[l - 1], flags, g_in, None)
             g = g_in
 
@@ -136,11 +138,12 @@ class SatEpoch:
             seen.append(losses)
         return seen
 
-    def step(self, W, b, pred, lr: float | None = None, pred_lr: float | None = None):
+    def step(self, W, b, pred, lr: float | None = None, pred_lr: float | None = None, grad_history: bool = False):
         """All partitions per launch.  W, b: lists of CUDA tensors; pred: list of sat_pred_params or None.
-        pred_lr: also run one predictor update (pred_update) before the ring is committed."""
+        pred_lr: also run one predictor update (pred_update) before the ring is committed.
+        grad_history: back-propagate with the stale-gradient term (gradient-side history of the previous epoch)."""
         self.loss_sum.zero_()
-        self._forward_backward(B.SAT_ALL_PARTS, W, b, pred, 0, 0)
+        self._forward_backward(B.SAT_ALL_PARTS, W, b, pred, 0, 0, grad_history)
         if pred_lr is not None and pred is not None:
             self.pred_update(pred, pred_lr)
         B.sat_cache_commit(self.ctx)
@@ -149,11 +152,11 @@ class SatEpoch:
                 B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
                 B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
 
-    def step_per_partition(self, W, b, pred, order=None, lr: float | None = None):
+    def step_per_partition(self, W, b, pred, order=None, lr: float | None = None, grad_history: bool = False):
         """Same epoch, one partition at a time (the LSTM state table is computed by the first call of every layer)."""
         self.loss_sum.zero_()
         for i, m in enumerate(order if order is not None else range(self.M)):
-            self._forward_backward(m, W, b, pred, 0 if i == 0 else 1, 0 if i == 0 else 1)
+            self._forward_backward(m, W, b, pred, 0 if i == 0 else 1, 0 if i == 0 else 1, grad_history)
         B.sat_cache_commit(self.ctx)
         if lr is not None:
             for l in range(self.L):
