@@ -382,6 +382,25 @@ def run_ours(args, wl):
                            ms=upd_ms, launches=int(upd_launches), period_epochs=PRED_PERIOD, ms_per_epoch_amortised=upd_ms / PRED_PERIOD,
                            loss_first_two_steps=[[float(x) for x in ls] for ls in first], kernel_families_ms=upd_fam)
 
+    # ---- epochs with the gradient-side history (stale-gradient term of the Appendix's back-propagation; not part of the
+    #      epoch metric) ----
+    grad_history = None
+    if rank == 0 and wl.L > 1:
+        for _ in range(2):
+            ep.step(W, b, preds, lr, grad_history=True)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_gh = 5
+        l0 = B.sat_launch_count(ep.ctx)
+        g0.record(stream)
+        for _ in range(n_gh):
+            ep.step(W, b, preds, lr, grad_history=True)
+        g1.record(stream)
+        stream.synchronize()
+        grad_history = dict(what="same epoch with SAT_BWD_GRAD_HISTORY on the layers >= 2: halo-row SpMM of D, per-partition adds "
+                                 "into the history, gather + W^T contraction + add of the stale term on the boundary rows",
+                            ms_per_epoch=g0.elapsed_time(g1) / n_gh, launches_per_epoch=int((B.sat_launch_count(ep.ctx) - l0) // n_gh),
+                            history_bytes=int(sum(2 * ep.n_slots * ((d + 3) & ~3) * 4 for d in wl.dims[2:])))
+
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None
     if rank == 0 and wl.L > 1:
@@ -452,7 +471,7 @@ def run_ours(args, wl):
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
                     e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                              loss=e2e_loss, pipelined="inputs of step i+1 copied on a second stream while step i computes"),
-                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, codec=codec, kernel_families=families,
+                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, grad_history=grad_history, codec=codec, kernel_families=families,
                     loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
                     multi_gpu="replicas only" if world > 1 else None)
         print(json.dumps(line), flush=True)
