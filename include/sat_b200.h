@@ -156,8 +156,9 @@ sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, const int32_t *
  * version: 0 = no promise.  A non-zero version promises that the VALUES of Wx and b are the same as in every earlier
  * call that passed the same version for this cached layer (the paper updates the predictor only every Delta-T epochs,
  * Algorithm 1 "Embedding predictor update"; bump the version after each update).  The library then keeps the input
- * projection x Wx + b of every cached snapshot it has already seen and computes it only for new snapshots — the result
- * is the same LSTM, one of tau input projections per epoch instead of tau.  Costs (tau+1) * |C| * 4h * 4 bytes per
+ * projection x Wx + b of every new snapshot and reuses it in the following epochs — the result is the same LSTM, one of
+ * tau input projections per epoch instead of tau.  After a version bump the older snapshots are not re-projected: their
+ * steps contract over [x | s] as without a version, until they have left the window.  Costs (tau+1) * |C| * 4h * 4 bytes per
  * cached layer. */
 typedef struct sat_pred_params {
     const float *Wx, *Uh, *b, *Wg, *bg;
@@ -396,11 +397,15 @@ sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
  * paper has no counterpart).  sat_profile_enable(1) clears the records and starts bracketing every family's
  * launches with an event pair; sat_profile_enable(0) stops.  sat_profile_read waits for the stream and returns,
  * for family f in [0, sat_profile_families()), its name, number of bracketed calls, total milliseconds and the
- * algorithmic bytes / flops those calls moved / performed (each operand read once, each result written once). */
+ * algorithmic bytes / flops those calls moved / performed (each operand read once, each result written once).
+ * Every bracketed call costs two event records on the stream (of the order of a microsecond of device time each);
+ * sat_profile_select restricts the bracketing to the families whose bit (1 << family) is set in family_mask (default: all),
+ * so that a timed run can carry the events of one family only. */
 enum { SAT_PROF_SPMM_FWD = 0, SAT_PROF_SPMM_BWD, SAT_PROF_SPMM_HROW, SAT_PROF_GEMM_NN, SAT_PROF_GEMM_NT,
        SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS, SAT_PROF_MASK };
 int32_t sat_profile_families(void);
 sat_status sat_profile_enable(sat_ctx *ctx, int enable);
+sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask);
 sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int64_t *calls, double *ms, double *bytes,
                             double *flops);
 

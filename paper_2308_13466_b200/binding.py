@@ -58,7 +58,7 @@ EXPORTS = [
     "sat_part_sizes", "sat_part_lists", "sat_slot_map", "sat_gather_rows", "sat_cache_init", "sat_predict",
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
-    "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_read",
+    "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
     "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write",
 ]
 
@@ -379,6 +379,23 @@ def sat_profile_families() -> int:
 
 def sat_profile_enable(ctx, enable: bool):
     _check(ctx, _lib.sat_profile_enable(ctx, C.c_int(1 if enable else 0)))
+
+
+def sat_profile_select(ctx, names=None):
+    """Restrict the per-family event bracketing to the named families (None = all of them)."""
+    mask = (1 << 64) - 1
+    if names is not None:
+        order = []
+        for f in range(sat_profile_families()):
+            name = C.c_char_p()
+            calls = C.c_int64()
+            ms, by, fl = C.c_double(), C.c_double(), C.c_double()
+            _check(ctx, _lib.sat_profile_read(ctx, C.c_int32(f), C.byref(name), C.byref(calls), C.byref(ms), C.byref(by), C.byref(fl)))
+            order.append(name.value.decode())
+        mask = 0
+        for n in names:
+            mask |= 1 << order.index(n)
+    _check(ctx, _lib.sat_profile_select(ctx, C.c_uint64(mask)))
 
 
 def sat_profile_read(ctx) -> dict:

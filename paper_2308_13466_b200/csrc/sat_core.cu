@@ -179,6 +179,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_dmask);
     sat_free_buf(ctx->buf_wsplit);
     sat_free_buf(ctx->buf_wsplit2);
+    sat_free_buf(ctx->buf_wsplit3);
     sat_free_buf(ctx->buf_bias);
     sat_free_buf(ctx->buf_pred_train);
     sat_free_buf(ctx->buf_ghist_halo);
@@ -242,6 +243,13 @@ extern "C" sat_status sat_profile_enable(sat_ctx *ctx, int enable)
         prof_clear(ctx);
     }
     ctx->prof_on = enable != 0;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask)
+{
+    if (!ctx) return SAT_EINVAL;
+    ctx->prof_mask = family_mask;
     return SAT_OK;
 }
 

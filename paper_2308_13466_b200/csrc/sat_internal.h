@@ -66,6 +66,7 @@ struct ProfRec {
 
 struct sat_ctx {
     bool prof_on = false;
+    uint64_t prof_mask = ~0ull;  // families that are bracketed while prof_on
     std::vector<ProfRec> prof;
     int device = 0;
     cudaStream_t stream = nullptr;
@@ -129,7 +130,7 @@ struct sat_ctx {
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out;
+        buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
@@ -162,7 +163,7 @@ struct ProfScope {
     sat_ctx *ctx;
     ProfRec rec;
     bool on;
-    ProfScope(sat_ctx *c, int family, double bytes, double flops) : ctx(c), on(c->prof_on)
+    ProfScope(sat_ctx *c, int family, double bytes, double flops) : ctx(c), on(c->prof_on && ((c->prof_mask >> family) & 1ull))
     {
         if (!on) return;
         rec.family = family;

@@ -291,8 +291,11 @@ __global__ void k_lstm_cell_first(const float *__restrict__ proj, int64_t rows, 
     s[t] = go * tanh_fast(cn);
 }
 
-// LSTM with cached input projections (parameter version promised by the caller): only ring buffers whose projection is
-// missing or was made with another version are projected; the recurrence then contracts over h only.
+// LSTM with cached input projections (parameter version promised by the caller).  A snapshot whose projection x Wx + b is
+// cached runs its step as a contraction over h only, with the projection added in the epilogue.  A missing projection is
+// computed (and kept) only for the newest snapshot, which has tau - 1 further epochs of use ahead; an older snapshot
+// without one (after a version bump) runs its step as the contraction over [x | s] instead, which costs less than
+// projecting it for the one or two epochs it has left.
 static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p, int32_t k, float *cell)
 {
     const int32_t h = p->h, d = c->width;
@@ -303,40 +306,50 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
         c->proj_h = h;
         c->proj_tag.assign(ctx->tau + 1, 0);
     }
-    TcWeights Wp;
-    bool packed = false;
-    for (int32_t t = 0; t < k; ++t) {
-        const int32_t idx = ring_index(ctx, k - 1 - t);
-        if (c->proj_tag[idx] == p->version) continue;
-        if (!packed) {
-            SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
-            packed = true;
-        }
+    TcWeights Wp, Wxu, Up;   // Wx alone, [Wx ; Uh], Uh alone (all gate-interleaved)
+    bool have_wp = false, have_wxu = false, have_up = false;
+    const int32_t newest = ring_index(ctx, 0);
+    if (c->proj_tag[newest] != p->version) {
+        SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
+        have_wp = true;
         TcEpilogueHost eh;
-        eh.C = c->proj + (int64_t)idx * plane;
+        eh.C = c->proj + (int64_t)newest * plane;
         eh.ldc = 4 * h;
         eh.bias = p->b;
         eh.pack_gate_h = h;
-        SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
-        c->proj_tag[idx] = p->version;
+        SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, newest), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+        c->proj_tag[newest] = p->version;
     }
-    TcWeights Up;
-    if (k > 1) SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit2, &Up, h));
     for (int32_t t = 0; t < k; ++t) {
-        const float *pr = c->proj + (int64_t)ring_index(ctx, k - 1 - t) * plane;  // oldest first
-        if (t == 0) {
+        const int32_t idx = ring_index(ctx, k - 1 - t);  // oldest first
+        const bool cached = c->proj_tag[idx] == p->version;
+        const float *pr = c->proj + (int64_t)idx * plane;
+        TcEpilogueHost eh;
+        eh.C = c->S;
+        eh.ldc = h;
+        eh.lstm_h = h;
+        eh.lstm_c = cell;
+        if (cached && t == 0) {
             ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 6.0, 0.0);
             k_lstm_cell_first<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(pr, rows, h, cell, c->S);
             SAT_LAUNCHED(ctx);
-        } else {
-            TcEpilogueHost eh;
-            eh.C = c->S;
-            eh.ldc = h;
-            eh.lstm_h = h;
-            eh.lstm_c = cell;
+        } else if (cached) {
+            if (!have_up) SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit2, &Up, h));
+            have_up = true;
             eh.addend = pr;
             eh.ld_addend = 4 * h;
             SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
+        } else if (t == 0) {
+            if (!have_wp) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
+            have_wp = true;
+            eh.bias = p->b;
+            eh.lstm_first = 1;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+        } else {
+            if (!have_wxu) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit3, &Wxu, h));
+            have_wxu = true;
+            eh.bias = p->b;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, c->S, h, h, Wxu, eh, SATK_GEMM_NN));
         }
     }
     c->S_valid = true;

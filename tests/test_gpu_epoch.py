@@ -160,11 +160,16 @@ def test_cached_input_projections_over_a_wrapping_ring(B):
     bd = [dev(x) for x in wl.b]
     n_epochs = 2 * (wl.tau + 1) + 1
     outs = {}
-    for version in (0, 9):
-        preds = pred_to_device(wl.pred, B, version)
+    for version in (0, 9, "bump"):
+        preds = pred_to_device(wl.pred, B, 9 if version == "bump" else version)
         ep, P, dtil, perm = _setup(B, wl)
         try:
-            for _ in range(n_epochs):
+            for t in range(n_epochs):
+                if version == "bump" and t == wl.tau + 2:
+                    # same values under a new version: the cached projections are dropped; the epochs that follow mix steps
+                    # with a cached projection (new snapshots) and steps that contract over [x | s] (older snapshots)
+                    for pp in preds:
+                        pp.version = 10
                 ep.step(Wd, bd, preds)
             torch.cuda.synchronize()
             # the LSTM state of the ring as the next epoch would see it (the commit dropped the one the epochs used)
@@ -181,7 +186,7 @@ def test_cached_input_projections_over_a_wrapping_ring(B):
     cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
     for _ in range(n_epochs):
         res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=False)
-    for version in (0, 9):
+    for version in (0, 9, "bump"):
         o = outs[version]
         assert o["state"] == (cache.write_idx, cache.n_valid)
         for l in range(1, wl.L):
