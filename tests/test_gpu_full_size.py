@@ -81,6 +81,88 @@ def test_medium_full_size_epochs(B):
         ep.close()
 
 
+def test_medium_full_size_predictor_gradient(B):
+    """sat_pred_grad at the benchmark's size on a ring of real embeddings: tau epochs on the device fill the ring, the
+    forward of one more epoch fills the write buffer; the oracle gets both through the export and computes the objective
+    and the gradient of every predictor array in float64."""
+    import torch
+    from paper_2308_13466_b200.epoch import SatEpoch
+    wl = make_workload("medium")
+    part = orc.contig_blocks(wl.n, wl.M)
+    dtil, _ = orc.degrees(wl.rowptr)
+    P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+    ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss)
+    try:
+        perm = np.concatenate(P.inner_gid)
+        ep.set_inputs(dev2d(wl.X), dev(wl.labels[perm]))
+        Wd = [dev(w) for w in wl.W]
+        bd = [dev(x) for x in wl.b]
+        preds = pred_to_device(wl.pred, B, 1)
+        for _ in range(wl.tau):
+            ep.step(Wd, bd, preds, 0.05)
+        ep.loss_sum.zero_()
+        ep._forward_backward(B.SAT_ALL_PARTS, Wd, bd, preds, 0, 0)
+        write_idx, n_valid = B.sat_cache_state(ep.ctx)
+        assert n_valid == wl.tau
+        names = ("Wx", "Uh", "b", "Wg", "bg")
+        for l in range(1, wl.L):
+            ring = B.sat_cache_export(ep.ctx, l, wl.tau, P.n_slots, wl.dims[l])
+            snaps = [ring[(write_idx - 1 - a) % (wl.tau + 1)] for a in range(n_valid - 1, -1, -1)]
+            pr = wl.pred[l - 1]
+            want_loss, want = orc.pred_loss_grad(P, dtil, snaps, ring[write_idx], pr["Wx"], pr["Uh"], pr["b"], pr["Wg"], pr["bg"])
+            g = tuple(torch.full_like(t, float("nan")) for t in preds[l - 1]._keep)
+            loss = B.sat_pred_grad(ep.ctx, l, preds[l - 1], None, *g, want_loss=True)
+            assert abs(loss - want_loss) <= 1e-5 * abs(want_loss), (l, loss, want_loss)
+            for a, t in zip(names, g):
+                assert_close(t.cpu().numpy(), want[a], f"full-size predictor gradient, layer {l}: G_{a}")
+            del ring, snaps
+    finally:
+        ep.close()
+
+
+def test_medium_full_size_gradient_history(B):
+    """Two epochs with the gradient-side history at the benchmark's size, from an empty ring: the second one back-propagates
+    with the stale term."""
+    import torch
+    from paper_2308_13466_b200.epoch import SatEpoch
+    wl = make_workload("medium")
+    part = orc.contig_blocks(wl.n, wl.M)
+    dtil, _ = orc.degrees(wl.rowptr)
+    P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+    ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss)
+    try:
+        perm = np.concatenate(P.inner_gid)
+        ep.set_inputs(dev2d(wl.X), dev(wl.labels[perm]))
+        Wd = [dev(w) for w in wl.W]
+        bd = [dev(x) for x in wl.b]
+        preds = pred_to_device(wl.pred, B)
+        cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
+        hist = orc.GradHistory(P.n_slots, wl.dims[2:])
+        for t in (1, 2):
+            before, hist_before = copy.deepcopy(cache), copy.deepcopy(hist)
+            res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=True, grad_hist=hist)
+            ep.step(Wd, bd, preds, grad_history=True)
+            torch.cuda.synchronize()
+            H_gpu = [None] + [ep.H[l].cpu().numpy() for l in range(1, wl.L + 1)]
+            masks, redo = relu_tie_masks(res, P, H_gpu, ep.inner_off, wl.L)
+            if redo:
+                del res
+                cache, hist = before, hist_before
+                res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=False, masks=masks, grad_hist=hist)
+            for l in range(wl.L):
+                assert_close(ep.gW[l].cpu().numpy(), res.G_W[l], f"epoch {t} G_W{l + 1} with the gradient history")
+                assert_close(ep.gb[l].cpu().numpy(), res.G_b[l], f"epoch {t} G_b{l + 1} with the gradient history")
+            for j in range(2, wl.L + 1):
+                got = B.sat_grad_history_read(ep.ctx, j, 0, P.n_slots, wl.dims[j])
+                assert_close(got, hist.read[j - 2], f"epoch {t} history of layer {j}")
+                B.sat_grad_history_write(ep.ctx, j, wl.dims[j], hist.read[j - 2])
+            for l in range(1, wl.L):
+                B.sat_cache_import(ep.ctx, l, cache.buf[l - 1])
+            del res
+    finally:
+        ep.close()
+
+
 @pytest.mark.parametrize("name", ["dense", "large", "multilabel"])
 def test_big_workloads_sampled(B, name):
     import torch
