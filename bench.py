@@ -311,8 +311,10 @@ def run_ours(args, wl):
         stream.synchronize()
         return u0.elapsed_time(u1) / max(args.steps, 1)
 
-    ms_cached = side_epochs(1 << 40)
-    ms_uncached = side_epochs(0)
+    ms_cached = None if args.epochs_only else side_epochs(1 << 40)
+    ms_uncached = None if args.epochs_only else side_epochs(0)
+    for pp in preds:
+        pp.version = 1 + epoch_no[0] // PRED_PERIOD
 
     # ---- end to end: host buffers in, host results out, every step ----
     hX = torch.from_numpy(np.ascontiguousarray(wl.X)).pin_memory()
@@ -382,7 +384,7 @@ def run_ours(args, wl):
     # ---- predictor update of Algorithm 1 (not part of the epoch metric): one gradient step on the predictor objective per
     #      cached layer, between the pushes of an epoch and the commit ----
     pred_update = None
-    if rank == 0 and wl.L > 1:
+    if rank == 0 and wl.L > 1 and not args.epochs_only:
         ep.loss_sum.zero_()
         ep._forward_backward(B.SAT_ALL_PARTS, W, b, preds, 0, 0)
         first = ep.pred_update(preds, PRED_LR, max_steps=2, min_gain=0.0)      # warm-up (scratch allocation); reads the losses back
@@ -408,7 +410,7 @@ def run_ours(args, wl):
     # ---- epochs with the gradient-side history (stale-gradient term of the Appendix's back-propagation; not part of the
     #      epoch metric) ----
     grad_history = None
-    if rank == 0 and wl.L > 1:
+    if rank == 0 and wl.L > 1 and not args.epochs_only:
         for _ in range(2):
             ep.step(W, b, preds, lr, grad_history=True)
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -426,7 +428,7 @@ def run_ours(args, wl):
 
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None
-    if rank == 0 and wl.L > 1:
+    if rank == 0 and wl.L > 1 and not args.epochs_only:
         prec = 3
         B.sat_cache_requantise(ep.ctx, 1, 1, prec)          # warm-up (scratch allocation)
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -513,6 +515,8 @@ def main():
     ap.add_argument("--workload", default="medium")
     ap.add_argument("--shrink", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--epochs-only", action="store_true",
+                    help="skip the side measurements (predictor never updated / unversioned, predictor update, gradient history, codec)")
     args = ap.parse_args()
     from sat_synth import make_workload
     if args.impl == "reference" and int(os.environ.get("RANK", "0")) != 0:

@@ -267,6 +267,59 @@ void orc_lstm(int32_t n_sel, const int32_t *slots_sel, int32_t n_slots, int32_t 
 }
 
 /* ------------------------------------------------------------------------------------
+ * O-4b  GRU in place of the LSTM (Section "Embedding Predictor" names GRU-GCN as a variant of the RNN-GNN
+ * predictor; the paper gives no equations, so this is the standard gated recurrent unit):
+ *     r = sigm(x W_r + s U_r + b_r)   z = sigm(x W_z + s U_z + b_z)
+ *     n = tanh(x W_n + b_n + r o (s U_n + b_hn))
+ *     s = (1 - z) o n + z o s
+ * W_x = [W_r | W_z | W_n] is [d x 3h], U_h likewise [h x 3h], b = [b_r | b_z | b_n | b_hn] has 4h entries.
+ * Same calling convention as orc_lstm.
+ * ---------------------------------------------------------------------------------- */
+void orc_gru(int32_t n_sel, const int32_t *slots_sel, int32_t n_slots, int32_t k,
+             const float *const *snaps, int64_t ld, int32_t d, int32_t h,
+             const float *Wx /* [d x 3h] */, const float *Uh /* [h x 3h] */, const float *b /* [4h] */,
+             float *S /* [n_slots x h] */)
+{
+    int32_t count = slots_sel ? n_sel : n_slots;
+#pragma omp parallel
+    {
+        double *ax = (double *)malloc(sizeof(double) * 3 * (size_t)h);
+        double *ah = (double *)malloc(sizeof(double) * 3 * (size_t)h);
+        double *s = (double *)malloc(sizeof(double) * (size_t)h);
+#pragma omp for schedule(dynamic, 16)
+        for (int32_t idx = 0; idx < count; ++idx) {
+            int32_t w = slots_sel ? slots_sel[idx] : idx;
+            for (int32_t j = 0; j < h; ++j) s[j] = 0.0;
+            for (int32_t t = 0; t < k; ++t) {
+                const float *x = snaps[t] + (int64_t)w * ld;
+                for (int32_t j = 0; j < 3 * h; ++j) ax[j] = ah[j] = 0.0;
+                for (int32_t q = 0; q < d; ++q) {
+                    double xv = (double)x[q];
+                    const float *wr = Wx + (int64_t)q * 3 * h;
+                    for (int32_t j = 0; j < 3 * h; ++j) ax[j] += xv * (double)wr[j];
+                }
+                for (int32_t q = 0; q < h; ++q) {
+                    double sv = s[q];
+                    const float *ur = Uh + (int64_t)q * 3 * h;
+                    for (int32_t j = 0; j < 3 * h; ++j) ah[j] += sv * (double)ur[j];
+                }
+                for (int32_t j = 0; j < h; ++j) {
+                    double r = sigm(ax[j] + ah[j] + (double)b[j]);
+                    double z = sigm(ax[h + j] + ah[h + j] + (double)b[h + j]);
+                    double n = tanh(ax[2 * h + j] + (double)b[2 * h + j] + r * (ah[2 * h + j] + (double)b[3 * h + j]));
+                    ax[j] = (1.0 - z) * n + z * s[j];   /* new state, kept aside until every unit has read the old one */
+                }
+                for (int32_t j = 0; j < h; ++j) s[j] = ax[j];
+            }
+            for (int32_t j = 0; j < h; ++j) S[(int64_t)w * h + j] = (float)s[j];
+        }
+        free(ax);
+        free(ah);
+        free(s);
+    }
+}
+
+/* ------------------------------------------------------------------------------------
  * O-5  Graph convolution on the final LSTM state plus skip connection, for the halo
  * rows of partition m (Section "Embedding Predictor": dH = GCN(S, A) on the 1-hop
  * extended subgraph; the prediction corrects the newest cached embedding):

@@ -223,6 +223,24 @@ def lstm_state(snaps, d: int, h: int, Wx, Uh, b, n_slots: int, slots_sel=None) -
     return S
 
 
+def gru_state(snaps, d: int, h: int, Wx, Uh, b, n_slots: int, slots_sel=None) -> np.ndarray:
+    """Final GRU hidden state S [n_slots, h] over the snapshots (oldest first): Wx [d, 3h] and Uh [h, 3h] in gate order
+    (r, z, n), b [4h] = (b_r, b_z, b_n, b_hn)."""
+    k = len(snaps)
+    S = np.zeros((n_slots, h), dtype=np.float32)
+    if k == 0:
+        return S
+    snaps = [_f32(s) for s in snaps]
+    ld = snaps[0].shape[1]
+    arr = (C.c_void_p * k)(*[s.ctypes.data for s in snaps])
+    Wx, Uh, b = _f32(Wx), _f32(Uh), _f32(b)
+    assert Wx.shape == (d, 3 * h) and Uh.shape == (h, 3 * h) and b.shape == (4 * h,)
+    sel = None if slots_sel is None else np.ascontiguousarray(slots_sel, dtype=np.int32)
+    lib().orc_gru(C.c_int32(0 if sel is None else sel.shape[0]), _p(sel), C.c_int32(n_slots), C.c_int32(k),
+                  arr, C.c_int64(ld), C.c_int32(d), C.c_int32(h), _p(Wx), _p(Uh), _p(b), _p(S))
+    return S
+
+
 def predict_halo(P: Partitioning, m: int, dtil, S, newest, Wg, bg, rows_sel=None) -> np.ndarray:
     """Predicted halo embeddings of partition m: newest snapshot + GCN(S) (skip connection)."""
     h, d = Wg.shape
@@ -377,7 +395,8 @@ def run_epoch(P: Partitioning, dtil, cache: CacheRing, X, labels, W, b, pred, lo
             S.append(None)
         else:
             h, d = pr["Wg"].shape
-            S.append(lstm_state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots, slots_sel=sel))
+            state = gru_state if pr.get("cell", "lstm") == "gru" else lstm_state
+            S.append(state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots, slots_sel=sel))
     G_W = [np.zeros(w.shape, dtype=np.float64) for w in W]
     G_b = [np.zeros(w.shape[1], dtype=np.float64) for w in W]
     total_loss = 0.0

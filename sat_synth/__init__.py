@@ -7,7 +7,7 @@ sides can consume it without sharing any of their own code.
 """
 from .graphs import sbm_graph, rmat_graph, bfs_relabel, csr_from_undirected_pairs
 from .tensors import normal_features, uniform_labels, bernoulli_labels, glorot_uniform, stream_rng
-from .workloads import WORKLOADS, Workload, make_workload
+from .workloads import WORKLOADS, Workload, as_gru, make_workload
 
 __all__ = [
     "sbm_graph", "rmat_graph", "bfs_relabel", "csr_from_undirected_pairs",

@@ -139,3 +139,17 @@ def make_workload(name: str, seed: int = 0, shrink: int = 1, with_dense: bool = 
             h=h,
         ))
     return wl
+
+
+def as_gru(pred):
+    """GRU-shaped parameters cut out of LSTM-shaped ones (a generator of inputs, no arithmetic): the first 3h gate columns
+    of Wx and Uh become (r, z, n); the 4h bias entries become (b_r, b_z, b_n, b_hn)."""
+    out = []
+    for p in pred:
+        h = int(p["h"])
+        q = dict(p)
+        q["Wx"] = np.ascontiguousarray(p["Wx"][:, :3 * h])
+        q["Uh"] = np.ascontiguousarray(p["Uh"][:, :3 * h])
+        q["cell"] = "gru"
+        out.append(q)
+    return out

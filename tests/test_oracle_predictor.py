@@ -132,3 +132,51 @@ def test_cache_ring_window():
         assert vals == [float(x) for x in range(max(1, t - tau + 1), t + 1)]   # a snapshot leaves after tau commits
         assert ring.n_valid == min(t, tau)
         assert ring.write_idx == t % (tau + 1)
+
+
+@pytest.mark.parametrize("k,d,h", [(1, 5, 3), (4, 9, 6), (7, 16, 8)])
+def test_gru_against_library_cell(k, d, h):
+    """Same weights through torch.nn.GRU in float64 (gate order r, z, n; the hidden-side bias only on the candidate)."""
+    rng = np.random.default_rng(k * 10 + d)
+    n = 9
+    snaps = [rng.standard_normal((n, d)).astype(np.float32) for _ in range(k)]
+    Wx = (rng.standard_normal((d, 3 * h)) * 0.4).astype(np.float32)
+    Uh = (rng.standard_normal((h, 3 * h)) * 0.4).astype(np.float32)
+    b = (rng.standard_normal(4 * h) * 0.3).astype(np.float32)
+    S = orc.gru_state(snaps, d, h, Wx, Uh, b, n)
+    gru = torch.nn.GRU(d, h, batch_first=False).double()
+    with torch.no_grad():
+        gru.weight_ih_l0.copy_(torch.tensor(Wx.T, dtype=torch.float64))
+        gru.weight_hh_l0.copy_(torch.tensor(Uh.T, dtype=torch.float64))
+        gru.bias_ih_l0.copy_(torch.tensor(b[:3 * h], dtype=torch.float64))
+        bh = np.zeros(3 * h)
+        bh[2 * h:] = b[3 * h:]
+        gru.bias_hh_l0.copy_(torch.tensor(bh, dtype=torch.float64))
+        _, hn = gru(torch.tensor(np.stack(snaps), dtype=torch.float64))
+    np.testing.assert_allclose(S, hn[0].numpy(), atol=1e-6)
+    sel = np.array([4, 1], dtype=np.int32)
+    S2 = orc.gru_state(snaps, d, h, Wx, Uh, b, n, slots_sel=sel)
+    assert np.array_equal(S2[sel], S[sel])
+
+
+def test_gru_degenerate_cases():
+    rng = np.random.default_rng(1)
+    n, d, h = 5, 4, 3
+    snaps = [rng.standard_normal((n, d)).astype(np.float32) for _ in range(3)]
+    z = lambda *s: np.zeros(s, dtype=np.float32)
+    # all-zero parameters: z = 1/2, n = 0 -> the state halves from zero: stays zero; no snapshot: zero state
+    assert np.all(orc.gru_state(snaps, d, h, z(d, 3 * h), z(h, 3 * h), z(4 * h), n) == 0)
+    assert np.all(orc.gru_state([], d, h, z(d, 3 * h), z(h, 3 * h), z(4 * h), n) == 0)
+    # one step from the zero state: s = (1 - sigm(a_z)) tanh(a_n + sigm(a_r) b_hn)
+    Wx = (rng.standard_normal((d, 3 * h)) * 0.5).astype(np.float32)
+    Uh = (rng.standard_normal((h, 3 * h)) * 0.5).astype(np.float32)
+    b = (rng.standard_normal(4 * h) * 0.5).astype(np.float32)
+    S = orc.gru_state(snaps[:1], d, h, Wx, Uh, b, n)
+    a = snaps[0].astype(np.float64) @ Wx.astype(np.float64) + b[:3 * h]
+    sig = lambda t: 1 / (1 + np.exp(-t))
+    want = (1 - sig(a[:, h:2 * h])) * np.tanh(a[:, 2 * h:] + sig(a[:, :h]) * b[3 * h:])
+    np.testing.assert_allclose(S, want, atol=1e-7)
+    # a saturated update gate (b_z large) freezes the state: it stays at its initial zero whatever the inputs
+    b2 = b.copy()
+    b2[h:2 * h] = 40.0
+    assert np.abs(orc.gru_state(snaps, d, h, Wx, Uh, b2, n)).max() < 1e-12
