@@ -163,8 +163,17 @@ sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, const int32_t *
 typedef struct sat_pred_params {
     const float *Wx, *Uh, *b, *Wg, *bg;
     int32_t h;
+    int32_t cell;      /* SAT_CELL_LSTM (0) or SAT_CELL_GRU (1) */
     uint64_t version;
 } sat_pred_params;
+/* cell = SAT_CELL_GRU selects the GRU-GCN variant of the RNN-GNN predictor (Section "Embedding Predictor" names it; the
+ * standard gated recurrent unit): Wx [d x 3h] and Uh [h x 3h] in gate order (r, z, n), b [4h] = (b_r, b_z, b_n, b_hn),
+ *     r = sigm(x W_r + s U_r + b_r), z = sigm(x W_z + s U_z + b_z), n = tanh(x W_n + b_n + r o (s U_n + b_hn)),
+ *     s = (1 - z) o n + z o s.
+ * The graph convolution and the skip connection are the same.  version is ignored for the GRU (no projections are kept),
+ * and sat_pred_grad supports the LSTM only (SAT_EINVAL otherwise). */
+#define SAT_CELL_LSTM 0
+#define SAT_CELL_GRU 1
 
 /* ---------------------------------------------------------------------------------------
  * sat_predict — predicted out-of-subgraph embeddings Hhat_out^(l, m) = g_omega over the

@@ -36,7 +36,10 @@ class SatError(RuntimeError):
 
 class sat_pred_params(C.Structure):
     _fields_ = [("Wx", C.c_void_p), ("Uh", C.c_void_p), ("b", C.c_void_p), ("Wg", C.c_void_p), ("bg", C.c_void_p),
-                ("h", C.c_int32), ("version", C.c_uint64)]
+                ("h", C.c_int32), ("cell", C.c_int32), ("version", C.c_uint64)]
+
+
+SAT_CELL_LSTM, SAT_CELL_GRU = 0, 1
 
 
 def _load():
@@ -190,11 +193,14 @@ def sat_cache_init(ctx, widths, tau: int, mode: int = SAT_CACHE_ZERO, init=None)
     _check(ctx, _lib.sat_cache_init(ctx, C.c_int32(n), w, C.c_int32(tau), C.c_int(mode), arr))
 
 
-def make_pred_params(Wx, Uh, b, Wg, bg, h: int, version: int = 0) -> sat_pred_params:
-    """version != 0 promises that the values of Wx and b stay the same for as long as the same version is passed."""
+def make_pred_params(Wx, Uh, b, Wg, bg, h: int, version: int = 0, cell: int = 0) -> sat_pred_params:
+    """version != 0 promises that the values of Wx and b stay the same for as long as the same version is passed.
+    cell: SAT_CELL_LSTM (Wx [d, 4h], Uh [h, 4h], b [4h]) or SAT_CELL_GRU (Wx [d, 3h], Uh [h, 3h], b [4h])."""
     for t in (Wx, Uh, b, Wg, bg):
         assert t.is_cuda and t.is_contiguous()
-    p = sat_pred_params(Wx.data_ptr(), Uh.data_ptr(), b.data_ptr(), Wg.data_ptr(), bg.data_ptr(), h, version)
+    gates = 3 if cell == SAT_CELL_GRU else 4
+    assert Wx.shape[1] == gates * h and tuple(Uh.shape) == (h, gates * h) and b.numel() == 4 * h
+    p = sat_pred_params(Wx.data_ptr(), Uh.data_ptr(), b.data_ptr(), Wg.data_ptr(), bg.data_ptr(), h, cell, version)
     p._keep = (Wx, Uh, b, Wg, bg)
     return p
 

@@ -356,8 +356,87 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
     return SAT_OK;
 }
 
+// GRU cell on the two pre-activation matrices gx = x Wx + (b_r | b_z | b_n) and gh = s Uh (null at the first step, where the
+// state is zero), gate blocks r | z | n:  n = tanh(gx_n + r (gh_n + b_hn)),  s = (1 - z) n + z s.
+__global__ void k_gru_cell(const float *__restrict__ gx, const float *__restrict__ gh, const float *__restrict__ b_hn, int64_t rows, int32_t h,
+                           float *__restrict__ s)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= rows * h) return;
+    const int64_t r0 = t / h;
+    const int j = (int)(t - r0 * h);
+    const float *ax = gx + r0 * 3 * (int64_t)h;
+    float hr = 0.f, hz = 0.f, hn = 0.f, sp = 0.f;
+    if (gh) {
+        const float *ah = gh + r0 * 3 * (int64_t)h;
+        hr = ah[j];
+        hz = ah[h + j];
+        hn = ah[2 * h + j];
+        sp = s[t];
+    }
+    const float r = 1.f / (1.f + expf(-(ax[j] + hr)));
+    const float z = 1.f / (1.f + expf(-(ax[h + j] + hz)));
+    const float n = tanhf(ax[2 * h + j] + r * (hn + b_hn[j]));
+    s[t] = (1.f - z) * n + z * sp;
+}
+
+// GRU-GCN variant: two plain contractions per step (input side with the bias, hidden side) and the cell kernel
+static sat_status run_gru(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p)
+{
+    const int32_t h = p->h, d = c->width;
+    const int64_t rows = ctx->n_slots;
+    if (!c->S || c->S_h != h) {
+        SAT_TRY(dev_realloc(ctx, &c->S, rows * h));
+        c->S_h = h;
+    }
+    const int32_t k = ctx->n_valid < ctx->tau ? ctx->n_valid : ctx->tau;
+    if (k == 0 || rows == 0) {
+        SAT_CUDA(ctx, cudaMemsetAsync(c->S, 0, (size_t)(rows > 0 ? rows : 1) * h * sizeof(float), ctx->stream));
+        c->S_valid = true;
+        return SAT_OK;
+    }
+    const int64_t plane = rows * 3 * h;
+    SAT_TRY(sat_ensure(ctx, ctx->buf_lstm_w, (size_t)2 * plane * sizeof(float)));
+    float *gx = (float *)ctx->buf_lstm_w.p, *gh = gx + plane;
+    const bool tc_x = sat_use_tc(3 * h, d), tc_h = sat_use_tc(3 * h, h);
+    TcWeights Wxp, Uhp;
+    if (tc_x) SAT_TRY(sat_tc_weights(ctx, p->Wx, 3 * h, d, nullptr, 0, 0, 3 * h, 1, ctx->buf_wsplit, &Wxp));
+    if (tc_h && k > 1) SAT_TRY(sat_tc_weights(ctx, p->Uh, 3 * h, h, nullptr, 0, 0, 3 * h, 1, ctx->buf_wsplit2, &Uhp));
+    for (int32_t t = 0; t < k; ++t) {
+        const float *x = ring_buf(ctx, c, ring_index(ctx, k - 1 - t));  // oldest first
+        if (tc_x) {
+            TcEpilogueHost eh;
+            eh.C = gx;
+            eh.ldc = 3 * h;
+            eh.bias = p->b;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 3 * h, x, c->ld, d, nullptr, 0, 0, Wxp, eh, SATK_GEMM_NN));
+        } else {
+            GemmEpilogue ep;
+            ep.bias = p->b;
+            SAT_TRY(sat_gemm_nn(ctx, rows, 3 * h, d, x, c->ld, p->Wx, 3 * h, gx, 3 * h, ep));
+        }
+        if (t > 0) {
+            if (tc_h) {
+                TcEpilogueHost eh;
+                eh.C = gh;
+                eh.ldc = 3 * h;
+                SAT_TRY(sat_gemm_tc(ctx, rows, 3 * h, c->S, h, h, nullptr, 0, 0, Uhp, eh, SATK_GEMM_SIDE));
+            } else {
+                GemmEpilogue ep;
+                SAT_TRY(sat_gemm_nn(ctx, rows, 3 * h, h, c->S, h, p->Uh, 3 * h, gh, 3 * h, ep));
+            }
+        }
+        ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 8.0, 0.0);
+        k_gru_cell<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(gx, t > 0 ? gh : nullptr, p->b + 3 * h, rows, h, c->S);
+        SAT_LAUNCHED(ctx);
+    }
+    c->S_valid = true;
+    return SAT_OK;
+}
+
 static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p)
 {
+    if (p->cell == SAT_CELL_GRU) return run_gru(ctx, c, p);
     const int32_t h = p->h, d = c->width;
     const int64_t rows = ctx->n_slots;
     if (!c->S || c->S_h != h) {
@@ -436,6 +515,7 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
     }
     if (params->h <= 0 || !params->Wx || !params->Uh || !params->b || !params->Wg || !params->bg)
         return sat_fail(ctx, SAT_EINVAL, "sat_predict: incomplete predictor parameters");
+    if (params->cell != SAT_CELL_LSTM && params->cell != SAT_CELL_GRU) return sat_fail(ctx, SAT_EINVAL, "sat_predict: unknown recurrent cell %d", params->cell);
     if (reuse_state) {
         if (!c->S_valid || c->S_h != params->h) return sat_fail(ctx, SAT_ESTATE, "sat_predict: no LSTM state table to reuse for layer %d", layer);
     } else {

@@ -292,6 +292,7 @@ extern "C" sat_status sat_pred_grad(sat_ctx *ctx, int32_t layer, const sat_pred_
     CacheLayer *c = &ctx->cache[layer - 1];
     if (!params || params->h <= 0 || (params->h & 3) || !params->Wx || !params->Uh || !params->b || !params->Wg || !params->bg)
         return sat_fail(ctx, SAT_EINVAL, "sat_pred_grad: incomplete predictor parameters or h not a multiple of 4");
+    if (params->cell != SAT_CELL_LSTM) return sat_fail(ctx, SAT_EINVAL, "sat_pred_grad: only the LSTM predictor is differentiated");
     if (params->h > 1024 || c->width > 1536) return sat_fail(ctx, SAT_EINVAL, "sat_pred_grad: supports h <= 1024 and cached widths <= 1536");
     if (!g_Wx || !g_Uh || !g_b || !g_Wg || !g_bg) return sat_fail(ctx, SAT_EINVAL, "sat_pred_grad: null gradient array");
     if (!aligned16(g_Wx) || !aligned16(g_Uh) || !aligned16(g_Wg)) return sat_fail(ctx, SAT_EINVAL, "sat_pred_grad: misaligned gradient array");

@@ -56,7 +56,8 @@ def pred_to_device(pred_list, B, version: int = 0):
         h = int(p["Wg"].shape[0])
         out.append(B.make_pred_params(dev(p["Wx"].astype(np.float32)), dev(p["Uh"].astype(np.float32)),
                                       dev(p["b"].astype(np.float32)), dev(p["Wg"].astype(np.float32)),
-                                      dev(p["bg"].astype(np.float32)), h, version))
+                                      dev(p["bg"].astype(np.float32)), h, version,
+                                      B.SAT_CELL_GRU if p.get("cell", "lstm") == "gru" else B.SAT_CELL_LSTM))
     return out
 
 

@@ -40,10 +40,17 @@ def _gather_H(res, P, l):
     ("medium", 16, {"h": 256}, 0),     # wide predictor: 4h = 1024 gate columns, cell update as a kernel of its own
     # widths that are no multiple of a tile / k-block / 8, non-zero biases in the layers and the predictor; with and
     # without cached input projections (the oracle keeps no such state)
-    ("odd", 1, {}, 0), ("odd", 1, {}, 3), ("odd", 1, {"h": 20}, 0), ("odd", 1, {"h": 20}, 3), ("odd", 1, {"h": 32}, 3)])
+    ("odd", 1, {}, 0), ("odd", 1, {}, 3), ("odd", 1, {"h": 20}, 0), ("odd", 1, {"h": 20}, 3), ("odd", 1, {"h": 32}, 3),
+    # GRU-GCN variant of the predictor
+    ("tiny", 1, {"cell": "gru"}, 0), ("medium", 16, {"cell": "gru"}, 0), ("odd", 1, {"cell": "gru"}, 0), ("odd", 1, {"cell": "gru", "h": 20}, 5)])
 def test_epochs_from_synchronised_state(B, name, shrink, over, version):
     import torch
+    over = dict(over)
+    cell = over.pop("cell", "lstm")
     wl = make_workload(name, shrink=shrink, **over)
+    if cell == "gru":
+        from sat_synth import as_gru
+        wl.pred = as_gru(wl.pred)
     ep, P, dtil, perm = _setup(B, wl)
     try:
         cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
