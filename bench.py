@@ -431,10 +431,16 @@ def run_ours(args, wl):
             ep.step(W, b, preds, lr, grad_history=True)
         g1.record(stream)
         stream.synchronize()
+        B.sat_profile_enable(ep.ctx, True)      # a second, bracketed pass for the per-family split
+        for _ in range(n_gh):
+            ep.step(W, b, preds, lr, grad_history=True)
+        gh_fam = {k: v["ms"] / n_gh for k, v in B.sat_profile_read(ep.ctx).items() if v["calls"]}
+        B.sat_profile_enable(ep.ctx, False)
         grad_history = dict(what="same epoch with SAT_BWD_GRAD_HISTORY on the layers >= 2: halo-row SpMM of D, per-partition adds "
                                  "into the history, gather + W^T contraction + add of the stale term on the boundary rows",
                             ms_per_epoch=g0.elapsed_time(g1) / n_gh, launches_per_epoch=int((B.sat_launch_count(ep.ctx) - l0) // n_gh),
-                            history_bytes=int(sum(2 * ep.n_slots * ((d + 3) & ~3) * 4 for d in wl.dims[2:])))
+                            history_bytes=int(sum(2 * ep.n_slots * ((d + 3) & ~3) * 4 for d in wl.dims[2:])),
+                            kernel_families_ms=gh_fam)
 
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None

@@ -106,6 +106,8 @@ struct sat_ctx {
     int32_t *hrow_slot = nullptr; // [nnz_cut] its cache slot
     float *hrow_w = nullptr;      // [nnz_cut] its dinv (the entry's weight up to the row's own dinv)
     int64_t nnz_cut = 0;
+    int64_t *hs_ptr = nullptr;    // [n_slots+1] halo positions by cache slot (built on first use): slot s is the halo node at
+    int32_t *hs_pos = nullptr;    // [nb]        positions hs_pos[hs_ptr[s] .. hs_ptr[s+1]), in ascending partition order
     int32_t *hlong = nullptr;     // [n_hlong] halo positions of the halo rows longer than SAT_HROW_LONG
     int32_t n_hlong = 0;
     std::vector<int32_t> h_hlong_off;
@@ -223,6 +225,9 @@ sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d
                       float *out, int32_t ld_out);
 sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d,
                        const float *src_base, int32_t ld_src, float *dst, int32_t ld_dst);
+// out[s] (+)= scale_s * sum over the halo positions p of cache slot s, in ascending partition order, of src[p]; scale_s = p_ss
+// (the self-loop weight of the node behind the slot) when self_scale, else 1.  One writer per slot: no atomics, fixed order.
+sat_status sat_sum_by_slot(sat_ctx *ctx, int32_t d, const float *src, int32_t ld_src, int self_scale, int add, float *out, int32_t ld_out);
 // dst[dst_row[i]] += src[src_row ? src_row[i] : i] (o mask bits of the destination row, when given); the dst_row[i] of one
 // call must be distinct
 sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,

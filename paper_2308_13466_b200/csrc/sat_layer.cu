@@ -699,9 +699,12 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
             float *qh = (float *)ctx->buf_ghist_halo.p;
             SAT_TRY(sat_spmm_hrow(ctx, v, d_out, D - (int64_t)v.row0 * ld_d, ld_d, 0, nullptr, qh - v.halo0 * (int64_t)ld_q, ld_q));
             float *qw = GH.buf + (size_t)(1 - GH.read_idx) * plane;
-            for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m) {
-                const int64_t h0 = ctx->h_halo_off[m], cnt = ctx->h_halo_off[m + 1] - h0;
-                SAT_TRY(sat_scatter_add(ctx, nullptr, ctx->halo_slot + h0, cnt, d_out, qh + (h0 - v.halo0) * ld_q, ld_q, qw, ld_q, nullptr, 0));
+            if (part == SAT_ALL_PARTS) {
+                // all copies of every boundary node are in qh: one gather-sum per slot, copies taken in partition order
+                SAT_TRY(sat_sum_by_slot(ctx, d_out, qh, ld_q, 0, 1, qw, ld_q));
+            } else {
+                const int64_t h0 = ctx->h_halo_off[part], cnt = ctx->h_halo_off[part + 1] - h0;
+                SAT_TRY(sat_scatter_add(ctx, nullptr, ctx->halo_slot + h0, cnt, d_out, qh, ld_q, qw, ld_q, nullptr, 0));
             }
         }
     }

@@ -222,32 +222,9 @@ __global__ void __launch_bounds__(256) k_pt_sum(const double *__restrict__ block
 //      neighbours u of p_uv G_a[halo position of u in v's partition] — the halo suffix of v's local CSR row, i.e. the
 //      layer SpMM restricted to halo columns (rows cut into chunks like there, so hub nodes do not serialise); the rows of
 //      the boundary nodes are then copied to their cache slots, every slot exactly once;
-//  (2) self terms (this kernel): halo row u of partition m adds p_uu G_a[u] to the slot of u; the halo slots of one
-//      partition are distinct, and the partitions are launched one after the other.  16 lanes per row, float4 per lane.
+//  (2) self terms: the slot of u receives p_uu times the sum of G_a over the copies of u (its halo positions in the other
+//      partitions), taken in partition order through the halo-positions-by-slot index (sat_sum_by_slot).
 // -------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
-k_pt_gs_self(const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
-             int32_t h4, const float *__restrict__ g_a, int64_t ld_a, float *__restrict__ g_s, int64_t ld_s)
-{
-    const int lane = threadIdx.x & 15;
-    const int64_t i = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 4;
-    if (i >= n_halo) return;
-    const int64_t u = halo0 + i;
-    const float du = dinv_enc[n + u];
-    const float p = du * du;
-    float4 *dst = reinterpret_cast<float4 *>(g_s + (int64_t)halo_slot[u] * ld_s);
-    const float4 *src = reinterpret_cast<const float4 *>(g_a + u * ld_a);
-    for (int c = lane; c < h4; c += 16) {
-        float4 o = dst[c];
-        const float4 x = src[c];
-        o.x = fmaf(p, x.x, o.x);
-        o.y = fmaf(p, x.y, o.y);
-        o.z = fmaf(p, x.z, o.z);
-        o.w = fmaf(p, x.w, o.w);
-        dst[c] = o;
-    }
-}
-
 // -------------------------------------------------------------------------------------
 // host side
 // -------------------------------------------------------------------------------------
@@ -401,16 +378,7 @@ extern "C" sat_status sat_pred_grad(sat_ctx *ctx, int32_t layer, const sat_pred_
         // ---- transposed graph convolution: gradient of the final hidden state ----
         SAT_TRY(sat_spmm(ctx, v, 2, h, nullptr, 0, g_a, h, g_rows, h));
         SAT_TRY(sat_scatter(ctx, ctx->push_row, ctx->push_slot, R, h, g_rows, h, dh, h));
-        {
-            ProfScope prof(ctx, SATK_PRED_TRAIN, 0.0, 0.0);
-            for (int32_t m = 0; m < M; ++m) {
-                const int64_t h0 = ctx->h_halo_off[m], cnt = ctx->h_halo_off[m + 1] - h0;
-                if (cnt == 0) continue;
-                k_pt_gs_self<<<(unsigned)cdiv64(cnt * 16, 256), 256, 0, ctx->stream>>>(ctx->halo_slot, ctx->dinv_enc, ctx->n, h0, cnt, h / 4, g_a, h,
-                                                                                      dh, h);
-                SAT_LAUNCHED(ctx);
-            }
-        }
+        SAT_TRY(sat_sum_by_slot(ctx, h, g_a, h, 1, 1, dh, h));
         // ---- back-propagation through time ----
         for (int32_t t = k - 1; t >= 0; --t) {
             const float *x = ring_buf(ctx, c, ring_index(ctx, k - 1 - t));

@@ -408,3 +408,110 @@ sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
+
+// -------------------------------------------------------------------------------------
+// Halo positions by cache slot: the inverse of halo_slot[].  A boundary node is a halo node of every other partition it has
+// a neighbour in; reductions over "all copies of a node" (gradient-side history, transposed predictor convolution) read
+// their terms through this index, one writer per slot, in ascending partition order.
+// -------------------------------------------------------------------------------------
+__global__ void k_hs_count(const int32_t *__restrict__ halo_slot, int64_t nb, int32_t *__restrict__ cnt)
+{
+    const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p < nb) atomicAdd(cnt + halo_slot[p], 1);   // integer counts: the result does not depend on the order
+}
+
+// the halo slots of one partition are distinct, so the cursor of a slot is touched by one thread per launch; the partitions
+// are launched in ascending order
+__global__ void k_hs_fill(const int32_t *__restrict__ halo_slot, int64_t p0, int64_t count, const int64_t *__restrict__ hs_ptr,
+                          int32_t *__restrict__ cursor, int32_t *__restrict__ hs_pos)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= count) return;
+    const int32_t s = halo_slot[p0 + i];
+    const int32_t k = cursor[s];
+    cursor[s] = k + 1;
+    hs_pos[hs_ptr[s] + k] = (int32_t)(p0 + i);
+}
+
+static sat_status build_halo_by_slot(sat_ctx *ctx)
+{
+    if (ctx->hs_ptr) return SAT_OK;
+    const int64_t ns = ctx->n_slots, nb = ctx->nb;
+    int32_t *cnt = nullptr;
+    SAT_CUDA(ctx, cudaMalloc(&cnt, (size_t)(ns + 1) * sizeof(int32_t)));
+    cudaError_t e = cudaMalloc(&ctx->hs_ptr, (size_t)(ns + 1) * sizeof(int64_t));
+    if (e == cudaSuccess) e = cudaMalloc(&ctx->hs_pos, (size_t)(nb > 0 ? nb : 1) * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMemsetAsync(cnt, 0, (size_t)(ns + 1) * sizeof(int32_t), ctx->stream);
+    sat_status rc = SAT_OK;
+    if (e == cudaSuccess && nb > 0) {
+        k_hs_count<<<(unsigned)cdiv64(nb, 256), 256, 0, ctx->stream>>>(ctx->halo_slot, nb, cnt);
+        ctx->launches++;
+    }
+    if (e == cudaSuccess) rc = sat_scan_i32(ctx, cnt, ns, ctx->hs_ptr);
+    if (e == cudaSuccess && rc == SAT_OK) e = cudaMemsetAsync(cnt, 0, (size_t)(ns + 1) * sizeof(int32_t), ctx->stream);
+    for (int32_t m = 0; e == cudaSuccess && rc == SAT_OK && m < ctx->M; ++m) {
+        const int64_t p0 = ctx->h_halo_off[m], count = ctx->h_halo_off[m + 1] - p0;
+        if (count == 0) continue;
+        k_hs_fill<<<(unsigned)cdiv64(count, 256), 256, 0, ctx->stream>>>(ctx->halo_slot, p0, count, ctx->hs_ptr, cnt, ctx->hs_pos);
+        ctx->launches++;
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    cudaFree(cnt);
+    if (e != cudaSuccess || rc != SAT_OK) {
+        cudaFree(ctx->hs_ptr);
+        cudaFree(ctx->hs_pos);
+        ctx->hs_ptr = nullptr;
+        ctx->hs_pos = nullptr;
+        return rc != SAT_OK ? rc : sat_check_cuda(ctx, e, "halo positions by slot");
+    }
+    return SAT_OK;
+}
+
+__global__ void __launch_bounds__(256)
+k_sum_by_slot(const int64_t *__restrict__ hs_ptr, const int32_t *__restrict__ hs_pos, int32_t n_slots, const float *__restrict__ dinv_enc,
+              int32_t n, int32_t d4, const float *__restrict__ src, int64_t ld_src, int self_scale, int add, float *__restrict__ out, int64_t ld_out)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t s = t / d4;
+    const int c = (int)(t - s * d4);
+    if (s >= n_slots) return;
+    const int64_t b = hs_ptr[s], e = hs_ptr[s + 1];
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t i = b; i < e; ++i) {
+        const float4 x = ld4(src + (int64_t)__ldg(hs_pos + i) * ld_src + 4 * c);
+        acc.x += x.x;
+        acc.y += x.y;
+        acc.z += x.z;
+        acc.w += x.w;
+    }
+    if (self_scale && e > b) {
+        const float du = __ldg(dinv_enc + n + hs_pos[b]);
+        const float p = du * du;
+        acc.x *= p;
+        acc.y *= p;
+        acc.z *= p;
+        acc.w *= p;
+    }
+    float4 *o = reinterpret_cast<float4 *>(out + s * ld_out + 4 * c);
+    if (add) {
+        const float4 y = *o;
+        acc.x += y.x;
+        acc.y += y.y;
+        acc.z += y.z;
+        acc.w += y.w;
+    }
+    *o = acc;
+}
+
+sat_status sat_sum_by_slot(sat_ctx *ctx, int32_t d, const float *src, int32_t ld_src, int self_scale, int add, float *out, int32_t ld_out)
+{
+    if (ctx->n_slots == 0) return SAT_OK;
+    SAT_TRY(build_halo_by_slot(ctx));
+    const int32_t d4 = (d + 3) / 4;
+    ProfScope prof(ctx, SATK_SCATTER, 8.0 * (double)ctx->nb + 4.0 * d * ((double)ctx->nb + (add ? 2.0 : 1.0) * ctx->n_slots), 0.0);
+    k_sum_by_slot<<<(unsigned)cdiv64((int64_t)ctx->n_slots * d4, 256), 256, 0, ctx->stream>>>(ctx->hs_ptr, ctx->hs_pos, ctx->n_slots, ctx->dinv_enc,
+                                                                                              ctx->n, d4, src, ld_src, self_scale, add, out, ld_out);
+    SAT_LAUNCHED(ctx);
+    return SAT_OK;
+}
