@@ -411,7 +411,8 @@ sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
  * sat_profile_select restricts the bracketing to the families whose bit (1 << family) is set in family_mask (default: all),
  * so that a timed run can carry the events of one family only. */
 enum { SAT_PROF_SPMM_FWD = 0, SAT_PROF_SPMM_BWD, SAT_PROF_SPMM_HROW, SAT_PROF_GEMM_NN, SAT_PROF_GEMM_NT,
-       SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS, SAT_PROF_MASK };
+       SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS, SAT_PROF_MASK,
+       SAT_PROF_GEMM_SIDE, SAT_PROF_CODEC, SAT_PROF_PRED_TRAIN };
 int32_t sat_profile_families(void);
 sat_status sat_profile_enable(sat_ctx *ctx, int enable);
 sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask);

@@ -385,6 +385,11 @@ static sat_status run_gru(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p)
 {
     const int32_t h = p->h, d = c->width;
     const int64_t rows = ctx->n_slots;
+    if (rows == 0) {   // a single partition: nothing is cached, the state table is empty
+        c->S_h = h;
+        c->S_valid = true;
+        return SAT_OK;
+    }
     if (!c->S || c->S_h != h) {
         SAT_TRY(dev_realloc(ctx, &c->S, rows * h));
         c->S_h = h;
@@ -439,6 +444,11 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
     if (p->cell == SAT_CELL_GRU) return run_gru(ctx, c, p);
     const int32_t h = p->h, d = c->width;
     const int64_t rows = ctx->n_slots;
+    if (rows == 0) {   // a single partition: nothing is cached, the state table is empty
+        c->S_h = h;
+        c->S_valid = true;
+        return SAT_OK;
+    }
     if (!c->S || c->S_h != h) {
         SAT_TRY(dev_realloc(ctx, &c->S, rows * h));
         c->S_h = h;

@@ -148,3 +148,55 @@ def test_update_inside_running_epochs(B):
         assert np.isfinite(float(ep.loss_sum.item()))
     finally:
         ep.close()
+
+
+def test_degenerate_cases_and_argument_errors(B):
+    """One partition (no halo, no cached node): empty objective, zero gradients, history flag is a no-op.  Unsupported
+    requests are refused with a status, not run."""
+    import torch
+    from tests.gpu_util import dev2d
+    wl = make_workload("odd", M=1)
+    ep, P, dtil = _setup(B, wl)
+    try:
+        assert P.n_slots == 0 and ep.nb == 0
+        perm = np.concatenate(P.inner_gid)
+        ep.set_inputs(dev2d(wl.X), dev(wl.labels[perm]))
+        Wd = [dev(w) for w in wl.W]
+        bd = [dev(x) for x in wl.b]
+        preds = pred_to_device(wl.pred, B, 0)
+        ep.step(Wd, bd, preds, grad_history=True)
+        ep.loss_sum.zero_()
+        ep._forward_backward(B.SAT_ALL_PARTS, Wd, bd, preds, 0, 0, True)
+        loss, got = _grads(B, ep, 1, preds[0])
+        assert loss == 0.0 and all(np.all(g == 0) for g in got.values())
+        B.sat_cache_commit(ep.ctx)
+        # the single-partition epoch equals the oracle's unpartitioned epoch
+        res = orc.run_epoch(P, dtil, orc.CacheRing(0, wl.dims[1:-1], wl.tau), wl.X, wl.labels, wl.W, wl.b, None, wl.loss)
+        torch.cuda.synchronize()
+        for l in range(wl.L):
+            assert_close(ep.gW[l].cpu().numpy(), res.G_W[l], f"single partition G_W{l + 1}")
+    finally:
+        ep.close()
+    wl = make_workload("tiny")
+    ep, P, dtil = _setup(B, wl)
+    try:
+        from sat_synth import as_gru
+        gru = pred_to_device(as_gru(wl.pred), B, 0)
+        g = tuple(torch.zeros_like(t) for t in gru[0]._keep)
+        with pytest.raises(B.SatError) as e:
+            B.sat_pred_grad(ep.ctx, 1, gru[0], None, *g)          # only the LSTM predictor is differentiated
+        assert e.value.status == B.SAT_EINVAL
+        lstm = pred_to_device(wl.pred, B, 0)
+        g = tuple(torch.zeros_like(t) for t in lstm[0]._keep)
+        with pytest.raises(B.SatError) as e:
+            B.sat_pred_grad(ep.ctx, wl.L, lstm[0], None, *g)      # not a cached layer
+        assert e.value.status == B.SAT_EINVAL
+        with pytest.raises(B.SatError) as e:
+            B.sat_grad_history_read(ep.ctx, 2, 0, P.n_slots, wl.dims[2])   # nothing committed yet
+        assert e.value.status == B.SAT_ESTATE
+        # a context stays usable after refused calls
+        B.sat_pred_grad(ep.ctx, 1, lstm[0], None, *g)
+        torch.cuda.synchronize()
+        assert all(bool(torch.isfinite(t).all()) for t in g)
+    finally:
+        ep.close()
