@@ -255,3 +255,68 @@ def test_staleness_of_historical_and_predicted_halos(B):
         assert float(sq.item()) == 0.0
     finally:
         ep.close()
+
+
+@pytest.mark.parametrize("over,empty_part", [
+    ({"dims": [50, 70, 38, 7], "h": 20}, False),     # cached widths that are no multiple of 4 (padded row strides)
+    ({"tau": 1}, False),                               # a window of one snapshot
+    ({"M": 5}, True),                                  # a partition without nodes
+    ({"M": 2, "h": 4, "dims": [50, 6, 5, 3]}, False),  # widths below the tensor-core threshold everywhere
+])
+def test_odd_shapes_and_degenerate_partitions(B, over, empty_part):
+    import torch
+    wl = make_workload("odd", **over)
+    if empty_part:
+        rng = np.random.default_rng(3)
+        wl.part_given = rng.choice(np.array([0, 1, 3, 4], dtype=np.int32), size=wl.n)     # nobody lands in partition 2
+    ep, P, dtil, perm = _setup(B, wl)
+    try:
+        if empty_part:
+            assert P.inner_gid[2].shape[0] == 0
+        cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
+        hist = orc.GradHistory(P.n_slots, wl.dims[2:])
+        Wd = [dev(w) for w in wl.W]
+        bd = [dev(x) for x in wl.b]
+        for version, use_hist in ((0, False), (7, True)):
+            preds = pred_to_device(wl.pred, B, version)
+            for t in range(wl.tau + 2):
+                before, hist_before = copy.deepcopy(cache), copy.deepcopy(hist)
+                res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, grad_hist=hist if use_hist else None)
+                ep.step(Wd, bd, preds, grad_history=use_hist)
+                torch.cuda.synchronize()
+                H_gpu = [None] + [ep.H[l].cpu().numpy() for l in range(1, wl.L + 1)]
+                masks, redo = relu_tie_masks(res, P, H_gpu, ep.inner_off, wl.L)
+                if redo:
+                    cache, hist = before, hist_before
+                    res = orc.run_epoch(P, dtil, cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, masks=masks,
+                                        grad_hist=hist if use_hist else None)
+                for l in range(1, wl.L + 1):
+                    assert_close(H_gpu[l], _gather_H(res, P, l), f"{over} epoch {t} H^{l}")
+                for l in range(wl.L):
+                    assert_close(ep.gW[l].cpu().numpy(), res.G_W[l], f"{over} epoch {t} G_W{l + 1}")
+                    assert_close(ep.gb[l].cpu().numpy(), res.G_b[l], f"{over} epoch {t} G_b{l + 1}")
+                for l in range(1, wl.L):
+                    B.sat_cache_import(ep.ctx, l, cache.buf[l - 1])
+                if use_hist:
+                    for j in range(2, wl.L + 1):
+                        B.sat_grad_history_write(ep.ctx, j, wl.dims[j], hist.read[j - 2])
+            # the predictor gradient on the same shapes
+            if version == 0:
+                ep.loss_sum.zero_()
+                ep._forward_backward(B.SAT_ALL_PARTS, Wd, bd, preds, 0, 0)
+                write_idx, n_valid = B.sat_cache_state(ep.ctx)
+                for l in range(1, wl.L):
+                    ring = B.sat_cache_export(ep.ctx, l, wl.tau, P.n_slots, wl.dims[l])
+                    snaps = [ring[(write_idx - 1 - a) % (wl.tau + 1)] for a in range(n_valid - 1, -1, -1)]
+                    pr = wl.pred[l - 1]
+                    want_loss, want = orc.pred_loss_grad(P, dtil, snaps, ring[write_idx], pr["Wx"], pr["Uh"], pr["b"], pr["Wg"], pr["bg"])
+                    g = tuple(torch.full_like(x, float("nan")) for x in preds[l - 1]._keep)
+                    loss = B.sat_pred_grad(ep.ctx, l, preds[l - 1], None, *g, want_loss=True)
+                    assert abs(loss - want_loss) <= 1e-5 * abs(want_loss)
+                    for a, x in zip(("Wx", "Uh", "b", "Wg", "bg"), g):
+                        assert_close(x.cpu().numpy(), want[a], f"{over} predictor gradient layer {l}: G_{a}")
+                for l in range(1, wl.L):
+                    B.sat_cache_import(ep.ctx, l, cache.buf[l - 1])
+                B.sat_cache_set_state(ep.ctx, cache.write_idx, cache.n_valid)
+    finally:
+        ep.close()
