@@ -163,7 +163,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     if (d4 <= 4) launch_items<4, 1>(ARGS);
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);
-    else if (d4 <= 32) launch_items<16, 2>(ARGS);
+    else if (d4 <= 32) launch_items<8, 4>(ARGS);
     else if (d4 <= 64) launch_items<32, 2>(ARGS);
     else if (d4 <= 96) launch_items<32, 3>(ARGS);
     else if (d4 <= 128) launch_items<32, 4>(ARGS);
