@@ -350,9 +350,11 @@ k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, con
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    float acc0[NT], acc1[NT];
+    // accumulators as pairs: the packed FMA of sm_100 (two IEEE-rounded fp32 FMAs per instruction, same results as fmaf)
+    // halves the issue slots of the inner loop, which is bound by FMA issue
+    float2 acc0[NT / 2], acc1[NT / 2];
 #pragma unroll
-    for (int j = 0; j < NT; ++j) acc0[j] = acc1[j] = 0.f;
+    for (int j = 0; j < NT / 2; ++j) acc0[j] = acc1[j] = make_float2(0.f, 0.f);
     int s = 0;
     load_stage(0, r_begin);
     for (int64_t r0 = r_begin; r0 < r_end; r0 += TNN_STAGE, s ^= 1) {
@@ -367,17 +369,15 @@ k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, con
 #pragma unroll 2
         for (int rr = 0; rr < TNN_STAGE; ++rr) {
             const float a0 = As[rr * 256 + threadIdx.x], a1 = As[rr * 256 + 128 + threadIdx.x];
+            const float2 a0p = make_float2(a0, a0), a1p = make_float2(a1, a1);
 #pragma unroll
             for (int j4 = 0; j4 < NT; j4 += 4) {
                 const float4 b = *reinterpret_cast<const float4 *>(Bs + rr * NT + j4);
-                acc0[j4] = fmaf(a0, b.x, acc0[j4]);
-                acc0[j4 + 1] = fmaf(a0, b.y, acc0[j4 + 1]);
-                acc0[j4 + 2] = fmaf(a0, b.z, acc0[j4 + 2]);
-                acc0[j4 + 3] = fmaf(a0, b.w, acc0[j4 + 3]);
-                acc1[j4] = fmaf(a1, b.x, acc1[j4]);
-                acc1[j4 + 1] = fmaf(a1, b.y, acc1[j4 + 1]);
-                acc1[j4 + 2] = fmaf(a1, b.z, acc1[j4 + 2]);
-                acc1[j4 + 3] = fmaf(a1, b.w, acc1[j4 + 3]);
+                const float2 blo = make_float2(b.x, b.y), bhi = make_float2(b.z, b.w);
+                acc0[j4 / 2] = __ffma2_rn(a0p, blo, acc0[j4 / 2]);
+                acc0[j4 / 2 + 1] = __ffma2_rn(a0p, bhi, acc0[j4 / 2 + 1]);
+                acc1[j4 / 2] = __ffma2_rn(a1p, blo, acc1[j4 / 2]);
+                acc1[j4 / 2 + 1] = __ffma2_rn(a1p, bhi, acc1[j4 / 2 + 1]);
             }
         }
         __syncthreads();  // the stage is refilled two iterations later
@@ -386,13 +386,13 @@ k_gemm_tn_narrow(int64_t rows, int64_t rows_per_block, int32_t m, int32_t n, con
         float *o = part + ((int64_t)blockIdx.x * m + col0) * n;
 #pragma unroll
         for (int j = 0; j < NT; ++j)
-            if (j < n) o[j] = acc0[j];
+            if (j < n) o[j] = (j & 1) ? acc0[j / 2].y : acc0[j / 2].x;
     }
     if (col1 < m) {
         float *o = part + ((int64_t)blockIdx.x * m + col1) * n;
 #pragma unroll
         for (int j = 0; j < NT; ++j)
-            if (j < n) o[j] = acc1[j];
+            if (j < n) o[j] = (j & 1) ? acc1[j / 2].y : acc1[j / 2].x;
     }
 }
 
