@@ -119,6 +119,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->lenc);
     dev_free(&ctx->inner_cnt);
     dev_free(&ctx->dinv_enc);
+    dev_free(&ctx->lw);
     dev_free(&ctx->hrow_ptr);
     dev_free(&ctx->hrow_pos);
     dev_free(&ctx->hrow_slot);
@@ -680,6 +681,12 @@ __global__ void k_dinv_enc(const float *__restrict__ dinv, const int32_t *__rest
     else if (i < n + nb) out[i] = dinv[halo_gid[i - n]];
 }
 
+__global__ void k_entry_weights(const int32_t *__restrict__ lenc, const float *__restrict__ dinv_enc, int64_t lnnz, float *__restrict__ lw)
+{
+    int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e < lnnz) lw[e] = dinv_enc[lenc[e]];
+}
+
 // partition of each halo entry: largest m with halo_off[m] <= j
 __device__ __forceinline__ int32_t find_part(const int64_t *off, int32_t M, int64_t j)
 {
@@ -941,6 +948,9 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
     for (int m = 0; m <= M; ++m) P_TRY(copy_i64(ctx, ctx->lrowptr + ctx->h_inner_off[m], &ctx->h_lnnz_off[m]));
     P_TRY(dev_alloc(ctx, &ctx->dinv_enc, (int64_t)n + ctx->nb));
     k_dinv_enc<<<GRID1((int64_t)n + ctx->nb)>>>(ctx->dinv, ctx->perm, ctx->halo_gid, n, ctx->nb, ctx->dinv_enc);
+    P_LAUNCHED();
+    P_TRY(dev_alloc(ctx, &ctx->lw, lnnz));
+    k_entry_weights<<<GRID1(lnnz)>>>(ctx->lenc, ctx->dinv_enc, lnnz, ctx->lw);
     P_LAUNCHED();
 
     // ---- halo-row CSR ----

@@ -101,6 +101,7 @@ struct sat_ctx {
     int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
     int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
     float *dinv_enc = nullptr;    // [n + nb] dinv of the node behind each encoded column
+    float *lw = nullptr;          // [nnz+n] dinv_enc[lenc[e]] stored per entry (read with the column instead of gathered)
     int64_t *hrow_ptr = nullptr;  // [nb+1] halo-row CSR
     int32_t *hrow_pos = nullptr;  // [nnz_cut] partition-major row of the inner neighbour
     int32_t *hrow_slot = nullptr; // [nnz_cut] its cache slot

@@ -39,7 +39,7 @@ __device__ __forceinline__ unsigned group_mask(int lane_in_warp)
 template <int G, int NV>
 __global__ void __launch_bounds__(256)
 k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ inner_cnt, const int32_t *__restrict__ lenc,
-             const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
+             const float *__restrict__ lw, const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
              const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0, int inner_only, int32_t n,
              int32_t d4, const float *__restrict__ in_base, int64_t ld_in, const float *__restrict__ halo_base, int64_t ld_halo,
              float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial, const uint32_t *__restrict__ omask, int32_t omask_words)
@@ -67,7 +67,7 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
         float w = 0.f;
         if (e < e1) {
             c = __ldg(lenc + e);
-            w = __ldg(dinv_enc + c);
+            w = __ldg(lw + e);
         }
         const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
 #pragma unroll 4
@@ -138,7 +138,7 @@ static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_
                          int32_t omask_words)
 {
     dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
-    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->dinv_enc, ctx->item_row,
+    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->lw, ctx->dinv_enc, ctx->item_row,
                                                         ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
                                                         ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words);
 }
