@@ -37,7 +37,7 @@ __device__ __forceinline__ unsigned group_mask(int lane_in_warp)
 //   them in chunk order.
 // -------------------------------------------------------------------------------------
 template <int G, int NV>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, NV <= 2 ? 8 : 4)
 k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ inner_cnt, const int32_t *__restrict__ lenc,
              const float *__restrict__ lw, const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
              const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0, int inner_only, int32_t n,
