@@ -592,3 +592,73 @@ def pred_loss_grad(P: Partitioning, dtil, snaps, target, Wx, Uh, b, Wg, bg, row_
         dh = dz @ Uh.T
         dc = dc * gf
     return loss, G
+
+
+# ------------------------------------------------------------------------------------------
+# O-13  Graph-attention layer as the local layer of a partition (the paper evaluates SAT with a GAT backbone as well and
+#       gives no equations for it; this is the standard single-head graph attention layer on the 1-hop extended subgraph,
+#       with the out-of-subgraph embeddings taken from the cache / predictor exactly as for the GCN layer).  float64 numpy.
+# ------------------------------------------------------------------------------------------
+GAT_SLOPE = 0.2
+
+
+def _gat_rows(P: Partitioning, m: int):
+    counts = np.diff(P.loc_rowptr[m]).astype(np.int64)
+    rows = np.repeat(np.arange(counts.shape[0], dtype=np.int64), counts)
+    return rows, P.loc_col[m].astype(np.int64)
+
+
+def gat_fwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, bias, act: int):
+    """For inner node v of partition m, over the entries u of its local row (its neighbours inside and outside the
+    partition and v itself):
+        z_u = h_u W;  e_vu = LeakyReLU_0.2(a_dst . z_v + a_src . z_u);  alpha_vu = softmax_u(e_vu);
+        o_v = sum_u alpha_vu z_u + bias;  h'_v = ReLU(o_v) (act = 1) or o_v.
+    Returns dict(Z=[n_m + b_m, d_out] (inner rows first), alpha=[entries], O, H (fp32))."""
+    Hc = np.concatenate([np.asarray(H_in, dtype=np.float64), np.asarray(H_halo, dtype=np.float64).reshape(-1, np.asarray(H_in).shape[1])])
+    W = np.asarray(W, dtype=np.float64)
+    a_src, a_dst = np.asarray(a_src, dtype=np.float64), np.asarray(a_dst, dtype=np.float64)
+    n_in = np.asarray(H_in).shape[0]
+    Z = Hc @ W
+    s_src, s_dst = Z @ a_src, Z[:n_in] @ a_dst
+    rows, cols = _gat_rows(P, m)
+    pre = s_dst[rows] + s_src[cols]
+    e = np.where(pre > 0, pre, GAT_SLOPE * pre)
+    mx = np.full(n_in, -np.inf)
+    np.maximum.at(mx, rows, e)
+    w = np.exp(e - mx[rows])
+    den = np.zeros(n_in)
+    np.add.at(den, rows, w)
+    alpha = w / den[rows]
+    O = np.zeros((n_in, W.shape[1]))
+    np.add.at(O, rows, alpha[:, None] * Z[cols])
+    if bias is not None:
+        O = O + np.asarray(bias, dtype=np.float64)
+    H = np.maximum(O, 0.0) if act else O
+    return dict(Z=Z, alpha=alpha, pre=pre, O=O, H=H.astype(np.float32))
+
+
+def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, act: int, mask=None):
+    """Gradients of sum(G_out * h') for the layer above; the out-of-subgraph embeddings are constants of the epoch, the
+    weights act on them as on the inner rows.  Returns dict(W, a_src, a_dst, b, H_in) in float64."""
+    Hc = np.concatenate([np.asarray(H_in, dtype=np.float64), np.asarray(H_halo, dtype=np.float64).reshape(-1, np.asarray(H_in).shape[1])])
+    W = np.asarray(W, dtype=np.float64)
+    a_src, a_dst = np.asarray(a_src, dtype=np.float64), np.asarray(a_dst, dtype=np.float64)
+    n_in = np.asarray(H_in).shape[0]
+    Z, alpha, pre = fwd["Z"], fwd["alpha"], fwd["pre"]
+    rows, cols = _gat_rows(P, m)
+    D = np.asarray(G_out, dtype=np.float64)
+    if act:
+        D = D * ((fwd["O"] > 0) if mask is None else np.asarray(mask, dtype=np.float64))
+    d_alpha = np.sum(D[rows] * Z[cols], axis=1)                       # dL / d alpha_vu
+    t = np.zeros(n_in)
+    np.add.at(t, rows, alpha * d_alpha)
+    d_pre = alpha * (d_alpha - t[rows]) * np.where(pre > 0, 1.0, GAT_SLOPE)   # through softmax and LeakyReLU
+    ds_dst = np.zeros(n_in)
+    np.add.at(ds_dst, rows, d_pre)
+    ds_src = np.zeros(Z.shape[0])
+    np.add.at(ds_src, cols, d_pre)
+    dZ = np.zeros_like(Z)
+    np.add.at(dZ, cols, alpha[:, None] * D[rows])
+    dZ += ds_src[:, None] * a_src
+    dZ[:n_in] += ds_dst[:, None] * a_dst
+    return dict(W=Hc.T @ dZ, a_src=Z.T @ ds_src, a_dst=Z[:n_in].T @ ds_dst, b=D.sum(axis=0), H_in=dZ[:n_in] @ W.T)
