@@ -282,6 +282,30 @@ sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float 
 sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer, const float *h_out, int32_t ld);
 sat_status sat_cache_commit(sat_ctx *ctx);
 
+/* ---------------------------------------------------------------------------------------
+ * sat_gat_fwd / sat_gat_bwd — graph-attention layer in place of the GCN layer (the paper reports SAT with a GAT backbone as
+ * well, Table "performance comparison"; it gives no equations: this is the standard single-head graph attention layer).
+ * For inner node v of the partition, over the entries u of its local row (neighbours inside the partition, v itself, and
+ * neighbours outside, whose embeddings come from the cache / predictor exactly as for sat_layer_fwd):
+ *     z_u = h_u W ;  e_vu = LeakyReLU_0.2(a_dst . z_v + a_src . z_u) ;  alpha_vu = softmax_u(e_vu) ;
+ *     h_out_v = act( sum_u alpha_vu z_u + bias ).
+ * The GCN normalisation is not used.  W [d_in x d_out], a_src [d_out], a_dst [d_out], bias [d_out] or NULL: DEVICE, dense.
+ * sat_gat_fwd keeps z, the attention scores and the log-sum-exp of every row for sat_gat_bwd (memory: (n + sum_m b_m) *
+ * d_out floats per layer, owned by the context).  d_out <= 1024.
+ * sat_gat_bwd: g_out [n_m x ld_g] gradient w.r.t. h_out; h_out as written by sat_gat_fwd (used for the ReLU mask; may be
+ * NULL for SAT_ACT_NONE); h_in / h_halo the same inputs as in the forward call.  The halo embeddings are constants of the
+ * epoch, W acts on them as on the inner rows:  g_W [d_in x d_out], g_a_src [d_out], g_a_dst [d_out], g_b [d_out] are
+ * overwritten (accumulate = 0) or added to (accumulate = 1); g_in [n_m x ld_gin] (or NULL) = gradient w.r.t. h_in.
+ * Results are bit-reproducible (no floating-point atomics).  SAT_ESTATE without the matching forward call.
+ * ------------------------------------------------------------------------------------- */
+sat_status sat_gat_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in, int32_t d_out, const float *h_in, int32_t ld_in,
+                       const float *h_halo, int32_t ld_halo, const float *W, const float *a_src, const float *a_dst,
+                       const float *bias, int act, float *h_out, int32_t ld_out);
+sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g, const float *h_out, int32_t ld_out,
+                       const float *h_in, int32_t ld_in, const float *h_halo, int32_t ld_halo, int32_t d_in, const float *W,
+                       const float *a_src, const float *a_dst, float *g_W, float *g_a_src, float *g_a_dst, float *g_b,
+                       int accumulate, float *g_in, int32_t ld_gin);
+
 /* Gradient-side history of layer `layer` >= 2 (see SAT_BWD_GRAD_HISTORY), for checkpoints and tests.
  * sat_grad_history_read: copies the committed history (which = 0; SAT_ESTATE before the first commit) or the running
  * epoch's (which = 1) to HOST memory, dense [|C| x d_out].
@@ -412,7 +436,7 @@ sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
  * so that a timed run can carry the events of one family only. */
 enum { SAT_PROF_SPMM_FWD = 0, SAT_PROF_SPMM_BWD, SAT_PROF_SPMM_HROW, SAT_PROF_GEMM_NN, SAT_PROF_GEMM_NT,
        SAT_PROF_GEMM_TN, SAT_PROF_LSTM_CELL, SAT_PROF_GATHER, SAT_PROF_SCATTER, SAT_PROF_LOSS, SAT_PROF_MASK,
-       SAT_PROF_GEMM_SIDE, SAT_PROF_CODEC, SAT_PROF_PRED_TRAIN };
+       SAT_PROF_GEMM_SIDE, SAT_PROF_CODEC, SAT_PROF_PRED_TRAIN, SAT_PROF_GAT };
 int32_t sat_profile_families(void);
 sat_status sat_profile_enable(sat_ctx *ctx, int enable);
 sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask);

@@ -62,7 +62,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd",
 ]
 
 
@@ -325,6 +325,24 @@ def sat_grad_history_write(ctx, layer: int, width: int, hist):
         return
     hist = np.ascontiguousarray(hist, dtype=np.float32)
     _check(ctx, _lib.sat_grad_history_write(ctx, C.c_int32(layer), C.c_int32(width), hist.ctypes.data_as(C.c_void_p)))
+
+
+def sat_gat_fwd(ctx, part: int, layer: int, h_in, h_halo, W, a_src, a_dst, bias, act: int, h_out):
+    """Graph-attention layer forward; all arguments CUDA fp32 tensors (2-D ones with row strides that are multiples of 4)."""
+    d_in, d_out = int(W.shape[0]), int(W.shape[1])
+    assert W.is_contiguous() and a_src.is_contiguous() and a_dst.is_contiguous() and (bias is None or bias.is_contiguous())
+    _check(ctx, _lib.sat_gat_fwd(ctx, C.c_int32(part), C.c_int32(layer), C.c_int32(d_in), C.c_int32(d_out), _dev(h_in), C.c_int32(_ld(h_in)),
+                                 _dev(h_halo), C.c_int32(_ld(h_halo) if h_halo is not None and h_halo.shape[0] else d_in + (-d_in) % 4),
+                                 _dev(W), _dev(a_src), _dev(a_dst), _dev(bias), C.c_int(act), _dev(h_out), C.c_int32(_ld(h_out))))
+
+
+def sat_gat_bwd(ctx, part: int, layer: int, g_out, h_out, h_in, h_halo, W, a_src, a_dst, g_W, g_a_src, g_a_dst, g_b, accumulate: int, g_in):
+    d_in = int(W.shape[0])
+    _check(ctx, _lib.sat_gat_bwd(ctx, C.c_int32(part), C.c_int32(layer), _dev(g_out), C.c_int32(_ld(g_out)), _dev(h_out),
+                                 C.c_int32(_ld(h_out) if h_out is not None else 0), _dev(h_in), C.c_int32(_ld(h_in)), _dev(h_halo),
+                                 C.c_int32(_ld(h_halo) if h_halo is not None and h_halo.shape[0] else d_in + (-d_in) % 4), C.c_int32(d_in),
+                                 _dev(W), _dev(a_src), _dev(a_dst), _dev(g_W), _dev(g_a_src), _dev(g_a_dst), _dev(g_b), C.c_int(accumulate),
+                                 _dev(g_in), C.c_int32(_ld(g_in) if g_in is not None else 0)))
 
 
 def sat_staleness(ctx, part: int, h_fresh, h_used_halo, sq_sum):

@@ -152,6 +152,11 @@ static void free_layers(sat_ctx *ctx)
         ctx->layers[i] = LayerState();
         dev_free(&ctx->ghist[i].buf);
         ctx->ghist[i] = GradHist();
+        sat_free_buf(ctx->gat[i].z_in);
+        sat_free_buf(ctx->gat[i].z_halo);
+        sat_free_buf(ctx->gat[i].scal);
+        ctx->gat[i].d_out = 0;
+        ctx->gat[i].valid.clear();
     }
 }
 
@@ -188,6 +193,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_ghist_halo);
     sat_free_buf(ctx->buf_ghist_rows);
     sat_free_buf(ctx->buf_ghist_out);
+    sat_free_buf(ctx->buf_gat);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;
@@ -225,7 +231,7 @@ extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
 // per-family device timing
 // =====================================================================================
 static const char *k_family_names[SATK_COUNT] = {"spmm_fwd", "spmm_bwd", "spmm_hrow", "gemm_nn", "gemm_nt", "gemm_tn",
-                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side", "codec", "pred_train"};
+                                                 "lstm_cell", "gather", "scatter", "loss", "mask", "gemm_side", "codec", "pred_train", "gat"};
 
 static void prof_clear(sat_ctx *ctx)
 {

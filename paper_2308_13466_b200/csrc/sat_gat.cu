@@ -1,0 +1,506 @@
+// Graph-attention layer as the local layer of a partition (the paper also evaluates SAT with a GAT backbone; the layer
+// itself is the standard single-head graph attention layer).  For inner node v, over the entries u of its local CSR row
+// (neighbours inside the partition, v itself, neighbours outside = halo rows with cached / predicted embeddings):
+//     z_u = h_u W;  e_vu = LeakyReLU_0.2(a_dst . z_v + a_src . z_u);  alpha_vu = softmax_u(e_vu);
+//     o_v = sum_u alpha_vu z_u + bias;  h'_v = ReLU(o_v) or o_v.
+// Backward with the halo embeddings constant (their z still depends on W):
+//     D = g o [o > 0];  dalpha_vu = D_v . z_u;  t_v = sum_u alpha_vu dalpha_vu;
+//     dpre_vu = alpha_vu (dalpha_vu - t_v) LeakyReLU'(pre_vu);  ds_dst[v] = sum_u dpre_vu;  ds_src[u] = sum_v dpre_vu;
+//     dZ_u = sum_v alpha_vu D_v + ds_src[u] a_src (+ ds_dst[u] a_dst for inner u);
+//     G_W = H^T dZ over inner and halo rows;  G_a_src = Z^T ds_src;  G_a_dst = Z_in^T ds_dst;  G_b = 1^T D;  G_in = dZ_in W^T.
+// The sums over v for a fixed u run over the inner prefix of u's own row (the inner block is symmetric) or over the
+// halo-row CSR; alpha_vu is recomputed from the per-row scalars (s_dst[v], log-sum-exp of row v), so no per-edge array
+// is stored.  One warp per row / node; every sum has a single writer and a fixed order.  A first, untuned build: rows of
+// hub nodes are walked by one warp.
+#include "sat_internal.h"
+
+#define CHECK_CTX(ctx)                                                                             \
+    do {                                                                                           \
+        if (!(ctx)) return SAT_EINVAL;                                                             \
+        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
+        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
+    } while (0)
+
+#define GAT_SLOPE 0.2f
+#define GAT_MAX_NV 8   /* float4 per lane: widths up to 1024 */
+
+static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+static bool ok_ld(int32_t ld, int32_t d) { return ld >= d && (ld & 3) == 0; }
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
+__device__ __forceinline__ float warp_max(float x)
+{
+    for (int o = 16; o > 0; o >>= 1) x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, o));
+    return x;
+}
+__device__ __forceinline__ float4 ldz(const float *row, int c4, int d)
+{
+    // the padding columns of the last vector of a row are not data: read them as zero
+    float4 x = *reinterpret_cast<const float4 *>(row + 4 * c4);
+    if (4 * c4 + 3 >= d) {
+        if (4 * c4 + 1 >= d) x.y = 0.f;
+        if (4 * c4 + 2 >= d) x.z = 0.f;
+        x.w = 0.f;
+    }
+    return x;
+}
+__device__ __forceinline__ float dot4(const float4 &a, const float4 &b) { return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w))); }
+__device__ __forceinline__ float lrelu(float x) { return x > 0.f ? x : GAT_SLOPE * x; }
+
+// s_src[r] = a_src . z_r, s_dst[r] = a_dst . z_r (when asked for); one warp per row
+__global__ void __launch_bounds__(256)
+k_gat_scores(const float *__restrict__ z, int64_t ld, int64_t rows, int32_t d, const float *__restrict__ a_src, const float *__restrict__ a_dst,
+             float *__restrict__ s_src, float *__restrict__ s_dst)
+{
+    const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (r >= rows) return;
+    float ps = 0.f, pd = 0.f;
+    for (int c = lane; c < d; c += 32) {
+        const float x = z[r * ld + c];
+        ps = fmaf(x, a_src[c], ps);
+        if (a_dst) pd = fmaf(x, a_dst[c], pd);
+    }
+    ps = warp_sum(ps);
+    pd = warp_sum(pd);
+    if (lane == 0) {
+        s_src[r] = ps;
+        if (a_dst) s_dst[r] = pd;
+    }
+}
+
+// forward: one warp per inner row.  Sweep 1 (lanes over entries): row maximum and log-sum-exp.  Sweep 2: the weighted sum,
+// entries in order, lanes owning float4 column slices.
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
+          const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
+          const float *__restrict__ s_halo, const float *__restrict__ s_dst, int32_t d, const float *__restrict__ bias, int relu,
+          float *__restrict__ lse, float *__restrict__ out_base, int64_t ld_out)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_rows) return;
+    const int32_t row = row0 + (int32_t)w;
+    const int64_t e0 = lrowptr[row], e1 = lrowptr[row + 1];
+    const float sd = s_dst[row];
+    float mx = -INFINITY;
+    for (int64_t e = e0 + lane; e < e1; e += 32) {
+        const int32_t c = lenc[e];
+        mx = fmaxf(mx, lrelu(sd + (c < n ? s_in[c] : s_halo[c - n])));
+    }
+    mx = warp_max(mx);
+    float den = 0.f;
+    for (int64_t e = e0 + lane; e < e1; e += 32) {
+        const int32_t c = lenc[e];
+        den += expf(lrelu(sd + (c < n ? s_in[c] : s_halo[c - n])) - mx);
+    }
+    den = warp_sum(den);
+    const float l = mx + logf(den);
+    if (lane == 0) lse[row] = l;
+    const int d4 = (d + 3) >> 2;
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t eb = e0; eb < e1; eb += 32) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float a = 0.f;
+        if (e < e1) {
+            c = lenc[e];
+            a = expf(lrelu(sd + (c < n ? s_in[c] : s_halo[c - n])) - l);
+        }
+        const int cnt = (e1 - eb) < 32 ? (int)(e1 - eb) : 32;
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t cj = __shfl_sync(0xffffffffu, c, j);
+            const float aj = __shfl_sync(0xffffffffu, a, j);
+            const float *src = cj < n ? z_in + (int64_t)cj * ld_z : z_halo + (int64_t)(cj - n) * ld_z;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c4 = lane + 32 * v;
+                if (c4 < d4) {
+                    const float4 x = *reinterpret_cast<const float4 *>(src + 4 * c4);
+                    acc[v].x = fmaf(aj, x.x, acc[v].x);
+                    acc[v].y = fmaf(aj, x.y, acc[v].y);
+                    acc[v].z = fmaf(aj, x.z, acc[v].z);
+                    acc[v].w = fmaf(aj, x.w, acc[v].w);
+                }
+            }
+        }
+    }
+    float *o = out_base + (int64_t)row * ld_out;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        if (c4 < d4) {
+            float4 r = acc[v];
+            if (bias) {
+                const int c = 4 * c4;
+                r.x += bias[c];
+                if (c + 1 < d) r.y += bias[c + 1];
+                if (c + 2 < d) r.z += bias[c + 2];
+                if (c + 3 < d) r.w += bias[c + 3];
+            }
+            if (relu) {
+                r.x = fmaxf(r.x, 0.f);
+                r.y = fmaxf(r.y, 0.f);
+                r.z = fmaxf(r.z, 0.f);
+                r.w = fmaxf(r.w, 0.f);
+            }
+            *reinterpret_cast<float4 *>(o + 4 * c4) = r;
+        }
+    }
+}
+
+// D = g o [h_out > 0] (ReLU layer) or g
+__global__ void k_gat_dmask(const float *__restrict__ g, int64_t ld_g, const float *__restrict__ h_out, int64_t ld_h, int64_t rows, int32_t d,
+                            float *__restrict__ D, int64_t ld_d)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t r = t / d;
+    const int c = (int)(t - r * d);
+    if (r >= rows) return;
+    const float x = g[r * ld_g + c];
+    D[r * ld_d + c] = (!h_out || h_out[r * ld_h + c] > 0.f) ? x : 0.f;
+}
+
+// backward, row side: one warp per inner row v keeps D_v in registers and walks the entries u of the row:
+//   t_v = sum alpha dalpha,  ds_dst[v] = sum alpha slope dalpha - t_v sum alpha slope
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_bwd_rows(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
+               const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
+               const float *__restrict__ s_halo, const float *__restrict__ s_dst, const float *__restrict__ lse, int32_t d,
+               const float *__restrict__ D, int64_t ld_d, float *__restrict__ t_out, float *__restrict__ ds_dst)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_rows) return;
+    const int32_t row = row0 + (int32_t)w;
+    const int d4 = (d + 3) >> 2;
+    float4 dv[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        dv[v] = c4 < d4 ? ldz(D + (int64_t)row * ld_d, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t e0 = lrowptr[row], e1 = lrowptr[row + 1];
+    const float sd = s_dst[row], l = lse[row];
+    float a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int64_t e = e0; e < e1; ++e) {
+        const int32_t c = lenc[e];
+        const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
+        const float alpha = expf(lrelu(pre) - l);
+        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+        const float *src = c < n ? z_in + (int64_t)c * ld_z : z_halo + (int64_t)(c - n) * ld_z;
+        float p = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) p += dot4(dv[v], ldz(src, c4, d));
+        }
+        const float da = warp_sum(p);
+        a1 = fmaf(alpha, da, a1);
+        a2 = fmaf(alpha * slope, da, a2);
+        a3 = fmaf(alpha, slope, a3);
+    }
+    if (lane == 0) {
+        t_out[row] = a1;
+        ds_dst[row] = a2 - a1 * a3;
+    }
+}
+
+// backward, column side: one warp per node u keeps z_u in registers and walks the rows v that have u as an entry:
+//   HALO = 0: u is inner row `row0 + w`, the v are the inner prefix of its own row (symmetric block, self entry included);
+//   HALO = 1: u is halo position `halo0 + w`, the v are its halo-row CSR entries.
+//   dZ_u = sum_v alpha_vu D_v + ds_src[u] a_src (+ ds_dst[u] a_dst),  ds_src[u] = sum_v alpha_vu (D_v . z_u - t_v) slope_vu
+template <int NV, int HALO>
+__global__ void __launch_bounds__(256)
+k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx, const int32_t *__restrict__ inner_cnt, int64_t u0, int64_t n_u,
+               const float *__restrict__ z_u_base, int64_t ld_z, const float *__restrict__ s_u, const float *__restrict__ s_dst,
+               const float *__restrict__ lse, const float *__restrict__ t_in, const float *__restrict__ ds_dst, int32_t d,
+               const float *__restrict__ D, int64_t ld_d, const float *__restrict__ a_src, const float *__restrict__ a_dst,
+               float *__restrict__ dz_base, float *__restrict__ ds_src)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_u) return;
+    const int64_t u = u0 + w;
+    const int d4 = (d + 3) >> 2;
+    float4 zu[NV], acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        zu[v] = c4 < d4 ? ldz(z_u_base + u * ld_z, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t e0 = ptr[u], e1 = HALO ? ptr[u + 1] : e0 + inner_cnt[u];
+    const float su = s_u[u];
+    float dss = 0.f;
+    for (int64_t e = e0; e < e1; ++e) {
+        const int32_t v_row = idx[e];
+        const float pre = s_dst[v_row] + su;
+        const float alpha = expf(lrelu(pre) - lse[v_row]);
+        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+        const float *dr = D + (int64_t)v_row * ld_d;
+        float p = 0.f;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) {
+                const float4 x = ldz(dr, c4, d);
+                p += dot4(x, zu[v]);
+                acc[v].x = fmaf(alpha, x.x, acc[v].x);
+                acc[v].y = fmaf(alpha, x.y, acc[v].y);
+                acc[v].z = fmaf(alpha, x.z, acc[v].z);
+                acc[v].w = fmaf(alpha, x.w, acc[v].w);
+            }
+        }
+        const float da = warp_sum(p);
+        dss = fmaf(alpha * slope, da - t_in[v_row], dss);
+    }
+    const float dsd = HALO ? 0.f : ds_dst[u];
+    float *o = dz_base + u * ld_z;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        if (c4 < d4) {
+            const int c = 4 * c4;
+            float4 r = acc[v];
+            r.x += dss * a_src[c] + (HALO ? 0.f : dsd * a_dst[c]);
+            if (c + 1 < d) r.y += dss * a_src[c + 1] + (HALO ? 0.f : dsd * a_dst[c + 1]);
+            if (c + 2 < d) r.z += dss * a_src[c + 2] + (HALO ? 0.f : dsd * a_dst[c + 2]);
+            if (c + 3 < d) r.w += dss * a_src[c + 3] + (HALO ? 0.f : dsd * a_dst[c + 3]);
+            if (c + 1 >= d) r.y = 0.f;
+            if (c + 2 >= d) r.z = 0.f;
+            if (c + 3 >= d) r.w = 0.f;
+            *reinterpret_cast<float4 *>(o + 4 * c4) = r;
+        }
+    }
+    if (lane == 0) ds_src[u] = dss;
+}
+
+// part[b][c] = sum over the rows r of block b, in order, of w[r] x[r][c]
+#define GAT_WSUM_ROWS 256
+__global__ void __launch_bounds__(256)
+k_gat_wcolsum(const float *__restrict__ x, int64_t ld, int64_t rows, int32_t d, const float *__restrict__ wgt, float *__restrict__ part)
+{
+    const int64_t r0 = (int64_t)blockIdx.x * GAT_WSUM_ROWS;
+    const int64_t r1 = r0 + GAT_WSUM_ROWS < rows ? r0 + GAT_WSUM_ROWS : rows;
+    for (int c = threadIdx.x; c < d; c += 256) {
+        float s = 0.f;
+        for (int64_t r = r0; r < r1; ++r) s = fmaf(wgt[r], x[r * ld + c], s);
+        part[(int64_t)blockIdx.x * d + c] = s;
+    }
+}
+
+// -------------------------------------------------------------------------------------
+// host side
+// -------------------------------------------------------------------------------------
+static sat_status gat_nn(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W, float *C, int32_t ldc)
+{
+    if (m == 0) return SAT_OK;
+    if (sat_use_tc(n, k)) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, n, k, nullptr, 0, 0, n, 1, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = C;
+        eh.ldc = ldc;
+        return sat_gemm_tc(ctx, m, n, A, lda, k, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN);
+    }
+    GemmEpilogue ep;
+    return sat_gemm_nn(ctx, m, n, k, A, lda, W, n, C, ldc, ep);
+}
+
+static sat_status gat_nt(sat_ctx *ctx, int64_t m, int32_t n, int32_t k, const float *A, int32_t lda, const float *W, float *C, int32_t ldc)
+{
+    if (m == 0) return SAT_OK;
+    if (sat_use_tc(n, k)) {
+        TcWeights Wp;
+        SAT_TRY(sat_tc_weights(ctx, W, k, k, nullptr, 0, 0, n, 0, ctx->buf_wsplit, &Wp));
+        TcEpilogueHost eh;
+        eh.C = C;
+        eh.ldc = ldc;
+        return sat_gemm_tc(ctx, m, n, A, lda, k, nullptr, 0, 0, Wp, eh, SATK_GEMM_NT);
+    }
+    return sat_gemm_nt(ctx, m, n, k, A, lda, nullptr, 0, W, k, C, ldc);
+}
+
+static sat_status gat_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const float *A, int32_t lda, const float *B, int32_t ldb, float *C,
+                         int accumulate)
+{
+    if (rows == 0) {
+        if (!accumulate) SAT_CUDA(ctx, cudaMemsetAsync(C, 0, (size_t)m * n * sizeof(float), ctx->stream));
+        return SAT_OK;
+    }
+    if (sat_use_tc(n, m) && rows >= 256) {
+        if (n <= 64) return sat_gemm_tn_narrow(ctx, rows, m, n, A, lda, B, ldb, C, n, accumulate);
+        return sat_gemm_tc_tn(ctx, rows, m, n, A, lda, B, ldb, C, n, accumulate);
+    }
+    return sat_gemm_tn(ctx, rows, m, n, A, lda, B, ldb, nullptr, 0, C, n, nullptr, accumulate);
+}
+
+// out[c] (+)= sum_r w[r] x[r][c]
+static sat_status gat_wcolsum(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, const float *w, float *out, int accumulate)
+{
+    if (rows == 0) {
+        if (!accumulate) SAT_CUDA(ctx, cudaMemsetAsync(out, 0, (size_t)d * sizeof(float), ctx->stream));
+        return SAT_OK;
+    }
+    const int64_t blocks = cdiv64(rows, GAT_WSUM_ROWS);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_colsum, (size_t)blocks * d * sizeof(float)));
+    k_gat_wcolsum<<<(unsigned)blocks, 256, 0, ctx->stream>>>(x, ld, rows, d, w, (float *)ctx->buf_colsum.p);
+    SAT_LAUNCHED(ctx);
+    return sat_splitk_reduce(ctx, (const float *)ctx->buf_colsum.p, d, (int32_t)blocks, accumulate, out, d, d);
+}
+
+#define GAT_DISPATCH(NVV, CALL)            \
+    do {                                   \
+        if ((NVV) <= 1) { CALL(1); }       \
+        else if ((NVV) <= 2) { CALL(2); }  \
+        else if ((NVV) <= 4) { CALL(4); }  \
+        else { CALL(8); }                  \
+    } while (0)
+
+extern "C" sat_status sat_gat_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in, int32_t d_out, const float *h_in, int32_t ld_in,
+                                  const float *h_halo, int32_t ld_halo, const float *W, const float *a_src, const float *a_dst,
+                                  const float *bias, int act, float *h_out, int32_t ld_out)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_gat_fwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    if (d_in <= 0 || d_out <= 0 || d_out > 128 * GAT_MAX_NV || !W || !a_src || !a_dst) return sat_fail(ctx, SAT_EINVAL, "sat_gat_fwd: bad widths or null parameters");
+    if (act != SAT_ACT_NONE && act != SAT_ACT_RELU) return sat_fail(ctx, SAT_EINVAL, "sat_gat_fwd: unknown activation");
+    if (v.n_rows > 0 && (!h_in || !h_out || !ok_ld(ld_in, d_in) || !ok_ld(ld_out, d_out) || !aligned16(h_in) || !aligned16(h_out)))
+        return sat_fail(ctx, SAT_EINVAL, "sat_gat_fwd: null / misaligned h_in / h_out or bad leading dimension");
+    if (v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_gat_fwd: null / misaligned h_halo");
+    GatState &G = ctx->gat[layer];
+    const int32_t ld_z = round_up4(d_out);
+    const int64_t n = ctx->n, nb = ctx->nb;
+    if (G.d_out != d_out || G.valid.size() != (size_t)ctx->M) {
+        // buffers over all rows / halo positions of the graph (any partition may be called); zeroed once so that the padding
+        // columns of the z rows, which no kernel writes, read as zero
+        SAT_TRY(sat_ensure(ctx, G.z_in, (size_t)(n > 0 ? n : 1) * ld_z * sizeof(float)));
+        SAT_TRY(sat_ensure(ctx, G.z_halo, (size_t)(nb > 0 ? nb : 1) * ld_z * sizeof(float)));
+        SAT_TRY(sat_ensure(ctx, G.scal, (size_t)(3 * (n > 0 ? n : 1) + (nb > 0 ? nb : 1)) * sizeof(float)));
+        SAT_CUDA(ctx, cudaMemsetAsync(G.z_in.p, 0, G.z_in.bytes, ctx->stream));
+        SAT_CUDA(ctx, cudaMemsetAsync(G.z_halo.p, 0, G.z_halo.bytes, ctx->stream));
+        G.d_out = d_out;
+        G.valid.assign(ctx->M, 0);
+    }
+    G.relu = act == SAT_ACT_RELU;
+    float *z_in = (float *)G.z_in.p, *z_halo = (float *)G.z_halo.p;
+    float *s_in = (float *)G.scal.p, *s_dst = s_in + n, *lse = s_dst + n, *s_halo = lse + n;
+    SAT_TRY(gat_nn(ctx, v.n_rows, d_out, d_in, h_in, ld_in, W, z_in + (int64_t)v.row0 * ld_z, ld_z));
+    SAT_TRY(gat_nn(ctx, v.n_halo, d_out, d_in, h_halo, ld_halo, W, z_halo + v.halo0 * ld_z, ld_z));
+    ProfScope prof(ctx, SATK_GAT, 0.0, 0.0);
+    if (v.n_rows > 0) {
+        k_gat_scores<<<(unsigned)cdiv64((int64_t)v.n_rows * 32, 256), 256, 0, ctx->stream>>>(z_in + (int64_t)v.row0 * ld_z, ld_z, v.n_rows, d_out, a_src, a_dst,
+                                                                                           s_in + v.row0, s_dst + v.row0);
+        SAT_LAUNCHED(ctx);
+    }
+    if (v.n_halo > 0) {
+        k_gat_scores<<<(unsigned)cdiv64(v.n_halo * 32, 256), 256, 0, ctx->stream>>>(z_halo + v.halo0 * ld_z, ld_z, v.n_halo, d_out, a_src, nullptr,
+                                                                                  s_halo + v.halo0, nullptr);
+        SAT_LAUNCHED(ctx);
+    }
+    if (v.n_rows > 0) {
+        const int nv = ((d_out + 3) / 4 + 31) / 32;
+        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
+#define CALL(NV)                                                                                                                              \
+    k_gat_fwd<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->n, v.row0, v.n_rows, z_in, z_halo, ld_z, s_in, s_halo, s_dst, d_out, \
+                                                 bias, G.relu, lse, h_out - (int64_t)v.row0 * ld_out, ld_out)
+        GAT_DISPATCH(nv, CALL);
+#undef CALL
+        SAT_LAUNCHED(ctx);
+    }
+    for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m) G.valid[m] = 1;
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g, const float *h_out, int32_t ld_out,
+                                  const float *h_in, int32_t ld_in, const float *h_halo, int32_t ld_halo, int32_t d_in, const float *W,
+                                  const float *a_src, const float *a_dst, float *g_W, float *g_a_src, float *g_a_dst, float *g_b,
+                                  int accumulate, float *g_in, int32_t ld_gin)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    GatState &G = ctx->gat[layer];
+    if (G.d_out <= 0 || G.valid.size() != (size_t)ctx->M) return sat_fail(ctx, SAT_ESTATE, "sat_gat_bwd: sat_gat_fwd has not run for layer %d", layer);
+    for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m)
+        if (!G.valid[m]) return sat_fail(ctx, SAT_ESTATE, "sat_gat_bwd: sat_gat_fwd has not run for partition %d of layer %d", m, layer);
+    const int32_t d_out = G.d_out, ld_z = round_up4(d_out);
+    if (d_in <= 0 || !W || !a_src || !a_dst || !g_W || !g_a_src || !g_a_dst || !g_b) return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: null parameter or gradient array");
+    if (accumulate != 0 && accumulate != 1) return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: accumulate must be 0 or 1");
+    if (v.n_rows > 0 && (!g_out || !h_in || !ok_ld(ld_g, d_out) || !ok_ld(ld_in, d_in) || !aligned16(g_out) || !aligned16(h_in) ||
+                         (G.relu && (!h_out || !ok_ld(ld_out, d_out)))))
+        return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: null / misaligned g_out / h_in / h_out or bad leading dimension");
+    if (v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo))) return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: null / misaligned h_halo");
+    if (g_in && v.n_rows > 0 && (!ok_ld(ld_gin, d_in) || !aligned16(g_in))) return sat_fail(ctx, SAT_EINVAL, "sat_gat_bwd: misaligned g_in or bad ld_gin");
+    const int64_t n = ctx->n, nb = ctx->nb;
+    float *z_in = (float *)G.z_in.p, *z_halo = (float *)G.z_halo.p;
+    float *s_in = (float *)G.scal.p, *s_dst = s_in + n, *lse = s_dst + n, *s_halo = lse + n;
+    // scratch of the call: D, dZ (inner rows of the selection, halo rows of the selection), t, ds_dst, ds_src
+    const size_t f_rows = (size_t)(v.n_rows > 0 ? v.n_rows : 1), f_halo = (size_t)(v.n_halo > 0 ? v.n_halo : 1);
+    SAT_TRY(sat_ensure(ctx, ctx->buf_gat, ((2 * f_rows + f_halo) * ld_z + 3 * f_rows + f_halo + 64) * sizeof(float)));
+    float *D = (float *)ctx->buf_gat.p, *dz_in = D + f_rows * ld_z, *dz_halo = dz_in + f_rows * ld_z;
+    float *t = dz_halo + f_halo * ld_z, *ds_dst = t + f_rows, *ds_in = ds_dst + f_rows, *ds_halo = ds_in + f_rows;
+    // virtual bases indexed by partition-major row / global halo position
+    const float *Db = D - (int64_t)v.row0 * ld_z;
+    float *dz_in_b = dz_in - (int64_t)v.row0 * ld_z, *dz_halo_b = dz_halo - v.halo0 * ld_z;
+    float *t_b = t - v.row0, *ds_dst_b = ds_dst - v.row0, *ds_in_b = ds_in - v.row0, *ds_halo_b = ds_halo - v.halo0;
+    const int nv = ((d_out + 3) / 4 + 31) / 32;
+    if (v.n_rows > 0) {
+        SAT_CUDA(ctx, cudaMemsetAsync(D, 0, f_rows * ld_z * sizeof(float), ctx->stream));   // padding columns of D read as zero
+        {
+            ProfScope prof(ctx, SATK_GAT, 0.0, 0.0);
+            k_gat_dmask<<<(unsigned)cdiv64((int64_t)v.n_rows * d_out, 256), 256, 0, ctx->stream>>>(g_out, ld_g, G.relu ? h_out : nullptr, ld_out, v.n_rows, d_out,
+                                                                                                 D, ld_z);
+            SAT_LAUNCHED(ctx);
+        }
+        SAT_TRY(sat_mask_rows(ctx, D, ld_z, v.n_rows, d_out, nullptr, 0, nullptr, 0, g_b, accumulate));
+        ProfScope prof(ctx, SATK_GAT, 0.0, 0.0);
+        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
+#define CALL(NV)                                                                                                                                  \
+    k_gat_bwd_rows<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->n, v.row0, v.n_rows, z_in, z_halo, ld_z, s_in, s_halo, s_dst, lse, \
+                                                      d_out, Db, ld_z, t_b, ds_dst_b)
+        GAT_DISPATCH(nv, CALL);
+#undef CALL
+        SAT_LAUNCHED(ctx);
+#define CALL(NV)                                                                                                                                    \
+    k_gat_bwd_cols<NV, 0><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->inner_cnt, v.row0, v.n_rows, z_in, ld_z, s_in, s_dst, lse, t_b, \
+                                                         ds_dst_b, d_out, Db, ld_z, a_src, a_dst, dz_in_b, ds_in_b)
+        GAT_DISPATCH(nv, CALL);
+#undef CALL
+        SAT_LAUNCHED(ctx);
+    } else if (!accumulate) {
+        SAT_CUDA(ctx, cudaMemsetAsync(g_b, 0, (size_t)d_out * sizeof(float), ctx->stream));
+    }
+    if (v.n_halo > 0 && v.n_rows > 0) {
+        ProfScope prof(ctx, SATK_GAT, 0.0, 0.0);
+        const unsigned grid = (unsigned)cdiv64(v.n_halo * 32, 256);
+#define CALL(NV)                                                                                                                                   \
+    k_gat_bwd_cols<NV, 1><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, nullptr, v.halo0, v.n_halo, z_halo, ld_z, s_halo, s_dst, lse, \
+                                                         t_b, nullptr, d_out, Db, ld_z, a_src, a_dst, dz_halo_b, ds_halo_b)
+        GAT_DISPATCH(nv, CALL);
+#undef CALL
+        SAT_LAUNCHED(ctx);
+    }
+    const int64_t halo_rows = v.n_rows > 0 ? v.n_halo : 0;
+    // parameter gradients
+    SAT_TRY(gat_tn(ctx, v.n_rows, d_in, d_out, h_in, ld_in, dz_in, ld_z, g_W, accumulate));
+    if (halo_rows > 0) SAT_TRY(gat_tn(ctx, halo_rows, d_in, d_out, h_halo, ld_halo, dz_halo, ld_z, g_W, 1));
+    SAT_TRY(gat_wcolsum(ctx, z_in + (int64_t)v.row0 * ld_z, ld_z, v.n_rows, d_out, ds_in, g_a_src, accumulate));
+    if (halo_rows > 0) SAT_TRY(gat_wcolsum(ctx, z_halo + v.halo0 * ld_z, ld_z, halo_rows, d_out, ds_halo, g_a_src, 1));
+    SAT_TRY(gat_wcolsum(ctx, z_in + (int64_t)v.row0 * ld_z, ld_z, v.n_rows, d_out, ds_dst, g_a_dst, accumulate));
+    // input gradient of the inner rows
+    if (g_in && v.n_rows > 0) SAT_TRY(gat_nt(ctx, v.n_rows, d_in, d_out, dz_in, ld_z, W, g_in, ld_gin));
+    return SAT_OK;
+}

@@ -52,10 +52,19 @@ struct GradHist {
     bool has_read = false;
 };
 
+// Saved forward state of a graph-attention layer: z = h W for all inner rows and halo positions of the graph, the attention
+// scores s_src (inner, halo), s_dst and the log-sum-exp of every inner row (scal = [s_in | s_dst | lse | s_halo]).
+struct GatState {
+    DevBuf z_in, z_halo, scal;
+    int32_t d_out = 0;
+    int relu = 0;
+    std::vector<uint8_t> valid;
+};
+
 // kernel families for the optional per-family device timing (sat_profile_*)
 enum {
     SATK_SPMM_FWD = 0, SATK_SPMM_BWD, SATK_SPMM_HROW, SATK_GEMM_NN, SATK_GEMM_NT, SATK_GEMM_TN, SATK_LSTM_CELL,
-    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_CODEC, SATK_PRED_TRAIN, SATK_COUNT
+    SATK_GATHER, SATK_SCATTER, SATK_LOSS, SATK_SPLIT, SATK_GEMM_SIDE, SATK_CODEC, SATK_PRED_TRAIN, SATK_GAT, SATK_COUNT
 };
 
 struct ProfRec {
@@ -129,11 +138,12 @@ struct sat_ctx {
     // ---- layers ----
     LayerState layers[SAT_MAX_LAYERS + 1];
     GradHist ghist[SAT_MAX_LAYERS + 1];
+    GatState gat[SAT_MAX_LAYERS + 1];
 
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out;
+        buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out, buf_gat;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
