@@ -662,3 +662,66 @@ def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, 
     dZ += ds_src[:, None] * a_src
     dZ[:n_in] += ds_dst[:, None] * a_dst
     return dict(W=Hc.T @ dZ, a_src=Z.T @ ds_src, a_dst=Z[:n_in].T @ ds_dst, b=D.sum(axis=0), H_in=dZ[:n_in] @ W.T)
+
+
+def run_epoch_gat(P: Partitioning, dtil, cache: CacheRing, X, labels, params, pred, loss_kind: str, masks=None):
+    """One SAT epoch with graph-attention layers in place of the GCN layers (Algorithm 1 unchanged around them): for every
+    partition and layer pull (features for layer 1, predicted / historical embeddings of the cached layer otherwise),
+    gat_fwd, push; loss; gat_bwd down the layers with the pulled embeddings held constant; commit.
+    params: per layer dict(W, a_src, a_dst, b).  Returns dict(loss, grads=[per layer dict(W, a_src, a_dst, b)], H=[per
+    partition [H^(1..L)]], O=[per partition [pre-activation outputs]], logit_margin=[per layer: the smallest |attention
+    logit before the LeakyReLU| relative to their rms: where it is at rounding level the slope of that logit is a tie])."""
+    L = len(params)
+    n = P.n
+    S = []
+    for l in range(1, L):
+        pr = pred[l - 1] if pred is not None else None
+        if pr is None:
+            S.append(None)
+        else:
+            h, d = pr["Wg"].shape
+            state = gru_state if pr.get("cell", "lstm") == "gru" else lstm_state
+            S.append(state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots))
+    grads = [dict(W=np.zeros(p["W"].shape), a_src=np.zeros(p["a_src"].shape), a_dst=np.zeros(p["a_dst"].shape), b=np.zeros(p["b"].shape))
+             for p in params]
+    total, Hs, Os = 0.0, [None] * P.M, [None] * P.M
+    margin = [np.inf] * L        # per layer: smallest |pre-activation of an attention logit| relative to their rms
+    for m in range(P.M):
+        inner, halo = P.inner_gid[m], P.halo_gid[m]
+        H_in = _f32(X[inner])
+        ins, halos, fws = [], [], []
+        for l in range(1, L + 1):
+            if l == 1:
+                H_halo = _f32(X[halo])
+            else:
+                pr = pred[l - 2] if pred is not None else None
+                d_prev = params[l - 1]["W"].shape[0]
+                if pr is None:
+                    H_halo = historical_halo(P, m, cache.newest(l - 1), d_prev)
+                else:
+                    H_halo = predict_halo(P, m, dtil, S[l - 2], cache.newest(l - 1), pr["Wg"], pr["bg"])
+            p = params[l - 1]
+            f = gat_fwd(P, m, H_in, H_halo, _f32(p["W"]), _f32(p["a_src"]), _f32(p["a_dst"]), _f32(p["b"]), 1 if l < L else 0)
+            if f["pre"].size:
+                margin[l - 1] = min(margin[l - 1], float(np.min(np.abs(f["pre"])) / max(np.sqrt(np.mean(f["pre"] ** 2)), 1e-300)))
+            if l < L:
+                cache.push(l, P.push_slot[m], f["H"][P.push_local[m]])
+            ins.append(H_in)
+            halos.append(H_halo)
+            fws.append(f)
+            H_in = f["H"]
+        val, G = loss_grad(loss_kind, fws[-1]["H"], labels[inner], 1.0 / n)
+        total += val
+        for l in range(L, 0, -1):
+            p = params[l - 1]
+            mk = None
+            if masks is not None and masks[m] is not None and l < L and masks[m][l - 1] is not None:
+                mk = masks[m][l - 1]
+            g = gat_bwd(P, m, ins[l - 1], halos[l - 1], _f32(p["W"]), _f32(p["a_src"]), _f32(p["a_dst"]), fws[l - 1], G, 1 if l < L else 0, mask=mk)
+            for k in ("W", "a_src", "a_dst", "b"):
+                grads[l - 1][k] += g[k]
+            G = g["H_in"].astype(np.float32)
+        Hs[m] = [f["H"] for f in fws]
+        Os[m] = [f["O"] for f in fws]
+    cache.commit()
+    return dict(loss=total, grads=grads, H=Hs, O=Os, logit_margin=margin)

@@ -50,6 +50,16 @@ __device__ __forceinline__ float4 ldz(const float *row, int c4, int d)
 }
 __device__ __forceinline__ float dot4(const float4 &a, const float4 &b) { return fmaf(a.x, b.x, fmaf(a.y, b.y, fmaf(a.z, b.z, a.w * b.w))); }
 __device__ __forceinline__ float lrelu(float x) { return x > 0.f ? x : GAT_SLOPE * x; }
+// D_v . z_u feeds differences (dalpha - t_v) that cancel most of their size: the products are summed in double
+__device__ __forceinline__ double ddot4(const float4 &a, const float4 &b)
+{
+    return (double)a.x * (double)b.x + (double)a.y * (double)b.y + (double)a.z * (double)b.z + (double)a.w * (double)b.w;
+}
+__device__ __forceinline__ double warp_sum_d(double x)
+{
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    return x;
+}
 
 // s_src[r] = a_src . z_r, s_dst[r] = a_dst . z_r (when asked for); one warp per row
 __global__ void __launch_bounds__(256)
@@ -169,13 +179,13 @@ __global__ void k_gat_dmask(const float *__restrict__ g, int64_t ld_g, const flo
 }
 
 // backward, row side: one warp per inner row v keeps D_v in registers and walks the entries u of the row:
-//   t_v = sum alpha dalpha,  ds_dst[v] = sum alpha slope dalpha - t_v sum alpha slope
+//   t_v = sum alpha dalpha,  ds_dst[v] = sum alpha slope dalpha - t_v sum alpha slope   (alpha renormalised, see below)
 template <int NV>
 __global__ void __launch_bounds__(256)
 k_gat_bwd_rows(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
                const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
                const float *__restrict__ s_halo, const float *__restrict__ s_dst, const float *__restrict__ lse, int32_t d,
-               const float *__restrict__ D, int64_t ld_d, float *__restrict__ t_out, float *__restrict__ ds_dst)
+               const float *__restrict__ D, int64_t ld_d, double *__restrict__ t_out, float *__restrict__ ds_dst)
 {
     const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -190,27 +200,32 @@ k_gat_bwd_rows(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ 
     }
     const int64_t e0 = lrowptr[row], e1 = lrowptr[row + 1];
     const float sd = s_dst[row], l = lse[row];
-    float a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    // ds_dst = a2 - a1 a3 subtracts sums of the same size (it is exactly zero when every entry has the same LeakyReLU slope):
+    // the three sums are kept in double so that the difference keeps its digits
+    // the fp32 weights alpha = exp(e - lse) of a row sum to 1 + eps (rounding of lse), and ds_dst would inherit -eps t_v, which
+    // is not small against its true value; a0 = sum alpha renormalises them
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
     for (int64_t e = e0; e < e1; ++e) {
         const int32_t c = lenc[e];
         const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
         const float alpha = expf(lrelu(pre) - l);
         const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
         const float *src = c < n ? z_in + (int64_t)c * ld_z : z_halo + (int64_t)(c - n) * ld_z;
-        float p = 0.f;
+        double p = 0.0;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int c4 = lane + 32 * v;
-            if (c4 < d4) p += dot4(dv[v], ldz(src, c4, d));
+            if (c4 < d4) p += ddot4(dv[v], ldz(src, c4, d));
         }
-        const float da = warp_sum(p);
-        a1 = fmaf(alpha, da, a1);
-        a2 = fmaf(alpha * slope, da, a2);
-        a3 = fmaf(alpha, slope, a3);
+        const double da = warp_sum_d(p);
+        a0 += (double)alpha;
+        a1 += (double)alpha * da;
+        a2 += (double)(alpha * slope) * da;
+        a3 += (double)alpha * (double)slope;
     }
     if (lane == 0) {
-        t_out[row] = a1;
-        ds_dst[row] = a2 - a1 * a3;
+        t_out[row] = a1 / a0;
+        ds_dst[row] = (float)(a2 / a0 - (a1 / a0) * (a3 / a0));
     }
 }
 
@@ -222,7 +237,7 @@ template <int NV, int HALO>
 __global__ void __launch_bounds__(256)
 k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx, const int32_t *__restrict__ inner_cnt, int64_t u0, int64_t n_u,
                const float *__restrict__ z_u_base, int64_t ld_z, const float *__restrict__ s_u, const float *__restrict__ s_dst,
-               const float *__restrict__ lse, const float *__restrict__ t_in, const float *__restrict__ ds_dst, int32_t d,
+               const float *__restrict__ lse, const double *__restrict__ t_in, const float *__restrict__ ds_dst, int32_t d,
                const float *__restrict__ D, int64_t ld_d, const float *__restrict__ a_src, const float *__restrict__ a_dst,
                float *__restrict__ dz_base, float *__restrict__ ds_src)
 {
@@ -240,30 +255,31 @@ k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
     }
     const int64_t e0 = ptr[u], e1 = HALO ? ptr[u + 1] : e0 + inner_cnt[u];
     const float su = s_u[u];
-    float dss = 0.f;
+    double dss = 0.0;
     for (int64_t e = e0; e < e1; ++e) {
         const int32_t v_row = idx[e];
         const float pre = s_dst[v_row] + su;
         const float alpha = expf(lrelu(pre) - lse[v_row]);
         const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
         const float *dr = D + (int64_t)v_row * ld_d;
-        float p = 0.f;
+        double p = 0.0;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int c4 = lane + 32 * v;
             if (c4 < d4) {
                 const float4 x = ldz(dr, c4, d);
-                p += dot4(x, zu[v]);
+                p += ddot4(x, zu[v]);
                 acc[v].x = fmaf(alpha, x.x, acc[v].x);
                 acc[v].y = fmaf(alpha, x.y, acc[v].y);
                 acc[v].z = fmaf(alpha, x.z, acc[v].z);
                 acc[v].w = fmaf(alpha, x.w, acc[v].w);
             }
         }
-        const float da = warp_sum(p);
-        dss = fmaf(alpha * slope, da - t_in[v_row], dss);
+        const double da = warp_sum_d(p);
+        dss += (double)(alpha * slope) * (da - t_in[v_row]);
     }
     const float dsd = HALO ? 0.f : ds_dst[u];
+    const float dssf = (float)dss;
     float *o = dz_base + u * ld_z;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
@@ -271,17 +287,17 @@ k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
         if (c4 < d4) {
             const int c = 4 * c4;
             float4 r = acc[v];
-            r.x += dss * a_src[c] + (HALO ? 0.f : dsd * a_dst[c]);
-            if (c + 1 < d) r.y += dss * a_src[c + 1] + (HALO ? 0.f : dsd * a_dst[c + 1]);
-            if (c + 2 < d) r.z += dss * a_src[c + 2] + (HALO ? 0.f : dsd * a_dst[c + 2]);
-            if (c + 3 < d) r.w += dss * a_src[c + 3] + (HALO ? 0.f : dsd * a_dst[c + 3]);
+            r.x += dssf * a_src[c] + (HALO ? 0.f : dsd * a_dst[c]);
+            if (c + 1 < d) r.y += dssf * a_src[c + 1] + (HALO ? 0.f : dsd * a_dst[c + 1]);
+            if (c + 2 < d) r.z += dssf * a_src[c + 2] + (HALO ? 0.f : dsd * a_dst[c + 2]);
+            if (c + 3 < d) r.w += dssf * a_src[c + 3] + (HALO ? 0.f : dsd * a_dst[c + 3]);
             if (c + 1 >= d) r.y = 0.f;
             if (c + 2 >= d) r.z = 0.f;
             if (c + 3 >= d) r.w = 0.f;
             *reinterpret_cast<float4 *>(o + 4 * c4) = r;
         }
     }
-    if (lane == 0) ds_src[u] = dss;
+    if (lane == 0) ds_src[u] = dssf;
 }
 
 // part[b][c] = sum over the rows r of block b, in order, of w[r] x[r][c]
@@ -449,13 +465,16 @@ extern "C" sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, con
     float *s_in = (float *)G.scal.p, *s_dst = s_in + n, *lse = s_dst + n, *s_halo = lse + n;
     // scratch of the call: D, dZ (inner rows of the selection, halo rows of the selection), t, ds_dst, ds_src
     const size_t f_rows = (size_t)(v.n_rows > 0 ? v.n_rows : 1), f_halo = (size_t)(v.n_halo > 0 ? v.n_halo : 1);
-    SAT_TRY(sat_ensure(ctx, ctx->buf_gat, ((2 * f_rows + f_halo) * ld_z + 3 * f_rows + f_halo + 64) * sizeof(float)));
-    float *D = (float *)ctx->buf_gat.p, *dz_in = D + f_rows * ld_z, *dz_halo = dz_in + f_rows * ld_z;
-    float *t = dz_halo + f_halo * ld_z, *ds_dst = t + f_rows, *ds_in = ds_dst + f_rows, *ds_halo = ds_in + f_rows;
+    const size_t t_floats = (2 * f_rows + 3) & ~(size_t)3;                  // the doubles first, then 16-byte aligned rows
+    SAT_TRY(sat_ensure(ctx, ctx->buf_gat, (t_floats + (2 * f_rows + f_halo) * ld_z + 2 * f_rows + f_halo + 64) * sizeof(float)));
+    double *t = (double *)ctx->buf_gat.p;
+    float *D = (float *)ctx->buf_gat.p + t_floats, *dz_in = D + f_rows * ld_z, *dz_halo = dz_in + f_rows * ld_z;
+    float *ds_dst = dz_halo + f_halo * ld_z, *ds_in = ds_dst + f_rows, *ds_halo = ds_in + f_rows;
     // virtual bases indexed by partition-major row / global halo position
     const float *Db = D - (int64_t)v.row0 * ld_z;
     float *dz_in_b = dz_in - (int64_t)v.row0 * ld_z, *dz_halo_b = dz_halo - v.halo0 * ld_z;
-    float *t_b = t - v.row0, *ds_dst_b = ds_dst - v.row0, *ds_in_b = ds_in - v.row0, *ds_halo_b = ds_halo - v.halo0;
+    double *t_b = t - v.row0;
+    float *ds_dst_b = ds_dst - v.row0, *ds_in_b = ds_in - v.row0, *ds_halo_b = ds_halo - v.halo0;
     const int nv = ((d_out + 3) / 4 + 31) / 32;
     if (v.n_rows > 0) {
         SAT_CUDA(ctx, cudaMemsetAsync(D, 0, f_rows * ld_z * sizeof(float), ctx->stream));   // padding columns of D read as zero

@@ -162,3 +162,43 @@ class SatEpoch:
             for l in range(self.L):
                 B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
                 B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
+
+    # ---- graph-attention backbone ---------------------------------------------------
+    def step_gat(self, params, pred, lr: float | None = None):
+        """One SAT epoch with graph-attention layers in place of the GCN layers, all partitions per launch: the pull / predict,
+        push, loss and commit calls are the same; sat_gat_fwd / sat_gat_bwd take the place of sat_layer_fwd / sat_layer_bwd.
+        params: per layer dict(W, a_src, a_dst, b) of CUDA tensors.  The gradients land in self.gat_grads (same keys)."""
+        ctx, L, m = self.ctx, self.L, B.SAT_ALL_PARTS
+        dev = self.device
+        if not hasattr(self, "gat_grads"):
+            self.gat_grads = [{k: torch.zeros_like(v) for k, v in p.items()} for p in params]
+            self.gat_halo = [_buf(self.nb, self.dims[l], dev) for l in range(L)]       # the pulled embeddings are needed again in the backward
+        self.loss_sum.zero_()
+        h_in = self.X_in
+        ins = []
+        for l in range(1, L + 1):
+            hv = self.gat_halo[l - 1]
+            if l == 1:
+                B.sat_gather_rows(ctx, m, B.SAT_ROWS_HALO, self.X, hv)
+            else:
+                B.sat_predict(ctx, l - 1, m, pred[l - 2] if pred is not None else None, 0, hv)
+            p = params[l - 1]
+            B.sat_gat_fwd(ctx, m, l, h_in, hv, p["W"], p["a_src"], p["a_dst"], p["b"], B.SAT_ACT_RELU if l < L else B.SAT_ACT_NONE, self.H[l])
+            if l < L:
+                B.sat_cache_update(ctx, m, l, self.H[l])
+            ins.append(h_in)
+            h_in = self.H[l]
+        kind = B.SAT_LOSS_SOFTMAX_CE if self.loss == "ce" else B.SAT_LOSS_SIGMOID_BCE
+        g = self.G[L]
+        B.sat_loss_grad(ctx, m, kind, self.H[L], self.labels, self.loss_sum, g)
+        for l in range(L, 0, -1):
+            p, gr = params[l - 1], self.gat_grads[l - 1]
+            g_in = self.G[l - 1] if l > 1 else None
+            B.sat_gat_bwd(ctx, m, l, g, self.H[l], ins[l - 1], self.gat_halo[l - 1], p["W"], p["a_src"], p["a_dst"], gr["W"], gr["a_src"], gr["a_dst"],
+                          gr["b"], 0, g_in)
+            g = g_in
+        B.sat_cache_commit(ctx)
+        if lr is not None:
+            for p, gr in zip(params, self.gat_grads):
+                for k in p:
+                    B.sat_sgd_step(ctx, p[k], gr[k], lr)
