@@ -442,6 +442,34 @@ def run_ours(args, wl):
                             history_bytes=int(sum(2 * ep.n_slots * ((d + 3) & ~3) * 4 for d in wl.dims[2:])),
                             kernel_families_ms=gh_fam)
 
+    # ---- the same workload with graph-attention layers in place of the GCN layers (not part of the epoch metric; a first,
+    #      untuned build of that backbone) ----
+    gat = None
+    if rank == 0 and wl.L > 1 and not args.epochs_only:
+        grng = np.random.default_rng(5)
+        gparams = []
+        for l in range(wl.L):
+            d_i, d_o = wl.dims[l], wl.dims[l + 1]
+            gparams.append(dict(W=up((grng.standard_normal((d_i, d_o)) / np.sqrt(d_i)).astype(np.float32)),
+                                a_src=up((grng.standard_normal(d_o) * 0.3).astype(np.float32)),
+                                a_dst=up((grng.standard_normal(d_o) * 0.3).astype(np.float32)),
+                                b=up(np.zeros(d_o, dtype=np.float32))))
+        for _ in range(2):
+            ep.step_gat(gparams, preds, lr)
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_ga = 5
+        l0 = B.sat_launch_count(ep.ctx)
+        a0.record(stream)
+        for _ in range(n_ga):
+            ep.step_gat(gparams, preds, lr)
+        a1.record(stream)
+        stream.synchronize()
+        gat_ms = a0.elapsed_time(a1) / n_ga
+        gat = dict(what="SAT epoch with single-head graph-attention layers (sat_gat_fwd / sat_gat_bwd) instead of GCN layers, same "
+                        "pull / predict / push / loss / commit calls",
+                   ms_per_epoch=gat_ms, edges_per_s=wl.nnz / (gat_ms * 1e-3), launches_per_epoch=int((B.sat_launch_count(ep.ctx) - l0) // n_ga),
+                   loss=float(ep.loss_sum.item()))
+
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None
     if rank == 0 and wl.L > 1 and not args.epochs_only:
@@ -513,7 +541,7 @@ def run_ours(args, wl):
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
                     e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                              loss=e2e_loss, pipelined="inputs of step i+1 copied on a second stream while step i computes; the host reads the results of step i while step i+1 is queued"),
-                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, grad_history=grad_history, codec=codec, kernel_families=families,
+                    gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, grad_history=grad_history, gat=gat, codec=codec, kernel_families=families,
                     loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
                     multi_gpu="replicas only" if world > 1 else None)
         print(json.dumps(line), flush=True)
