@@ -194,6 +194,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     sat_free_buf(ctx->buf_ghist_rows);
     sat_free_buf(ctx->buf_ghist_out);
     sat_free_buf(ctx->buf_gat);
+    sat_free_buf(ctx->buf_gat_items);
     if (ctx->d_flag) cudaFree(ctx->d_flag);
     if (ctx->h_flag) cudaFreeHost(ctx->h_flag);
     delete ctx;

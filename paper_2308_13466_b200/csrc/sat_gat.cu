@@ -10,8 +10,9 @@
 //     G_W = H^T dZ over inner and halo rows;  G_a_src = Z^T ds_src;  G_a_dst = Z_in^T ds_dst;  G_b = 1^T D;  G_in = dZ_in W^T.
 // The sums over v for a fixed u run over the inner prefix of u's own row (the inner block is symmetric) or over the
 // halo-row CSR; alpha_vu is recomputed from the per-row scalars (s_dst[v], log-sum-exp of row v), so no per-edge array
-// is stored.  One warp per row / node; every sum has a single writer and a fixed order.  A first, untuned build: rows of
-// hub nodes are walked by one warp.
+// is stored.  One warp per work item of the SpMM (a row, or a 256-entry chunk of a long row), per-item partial sums added in
+// item order by small combine kernels: every sum has a single writer and a fixed order.  The halo-node side of the backward
+// still walks a halo row with one warp.
 #include "sat_internal.h"
 
 #define CHECK_CTX(ctx)                                                                             \
@@ -83,14 +84,12 @@ k_gat_scores(const float *__restrict__ z, int64_t ld, int64_t rows, int32_t d, c
     }
 }
 
-// forward: one warp per inner row.  Sweep 1 (lanes over entries): row maximum and log-sum-exp.  Sweep 2: the weighted sum,
-// entries in order, lanes owning float4 column slices.
-template <int NV>
+// forward over work items: k_gat_lse (a warp per row, lanes over the entries) gives the log-sum-exp of every row; then one warp
+// per item accumulates its chunk of the weighted sum.  Rows of a single item are finished here (bias, ReLU); items of
+// longer rows write their partial sum to `partial` (row index item_mslot) and k_gat_fwd_fixup adds them in item order.
 __global__ void __launch_bounds__(256)
-k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
-          const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
-          const float *__restrict__ s_halo, const float *__restrict__ s_dst, int32_t d, const float *__restrict__ bias, int relu,
-          float *__restrict__ lse, float *__restrict__ out_base, int64_t ld_out)
+k_gat_lse(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
+          const float *__restrict__ s_in, const float *__restrict__ s_halo, const float *__restrict__ s_dst, float *__restrict__ lse)
 {
     const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
@@ -110,8 +109,26 @@ k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc,
         den += expf(lrelu(sd + (c < n ? s_in[c] : s_halo[c - n])) - mx);
     }
     den = warp_sum(den);
-    const float l = mx + logf(den);
-    if (lane == 0) lse[row] = l;
+    if (lane == 0) lse[row] = mx + logf(den);
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_fwd_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, const int32_t *__restrict__ item_row,
+                const int32_t *__restrict__ first_item, const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0,
+                int32_t n, const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
+                const float *__restrict__ s_halo, const float *__restrict__ s_dst, const float *__restrict__ lse, int32_t d,
+                const float *__restrict__ bias, int relu, float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_items) return;
+    const int32_t item = item0 + (int32_t)w;
+    const int32_t row = item_row[item];
+    const int64_t re = lrowptr[row + 1];
+    const int64_t e0 = lrowptr[row] + (int64_t)(item - first_item[row]) * SAT_SPMM_CHUNK;
+    const int64_t e1 = e0 + SAT_SPMM_CHUNK < re ? e0 + SAT_SPMM_CHUNK : re;
+    const float sd = s_dst[row], l = lse[row];
     const int d4 = (d + 3) >> 2;
     float4 acc[NV];
 #pragma unroll
@@ -125,6 +142,7 @@ k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc,
             a = expf(lrelu(sd + (c < n ? s_in[c] : s_halo[c - n])) - l);
         }
         const int cnt = (e1 - eb) < 32 ? (int)(e1 - eb) : 32;
+#pragma unroll 4
         for (int j = 0; j < cnt; ++j) {
             const int32_t cj = __shfl_sync(0xffffffffu, c, j);
             const float aj = __shfl_sync(0xffffffffu, a, j);
@@ -142,14 +160,24 @@ k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc,
             }
         }
     }
+    const int32_t ms = item_mslot[item];
+    if (ms >= 0) {
+        float *o = partial + (int64_t)(ms - mitem0) * ld_z;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) *reinterpret_cast<float4 *>(o + 4 * c4) = acc[v];
+        }
+        return;
+    }
     float *o = out_base + (int64_t)row * ld_out;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
         const int c4 = lane + 32 * v;
         if (c4 < d4) {
             float4 r = acc[v];
+            const int c = 4 * c4;
             if (bias) {
-                const int c = 4 * c4;
                 r.x += bias[c];
                 if (c + 1 < d) r.y += bias[c + 1];
                 if (c + 2 < d) r.z += bias[c + 2];
@@ -166,6 +194,43 @@ k_gat_fwd(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc,
     }
 }
 
+// rows cut into several items: add the partial sums in item order, then bias and activation
+__global__ void k_gat_fwd_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, int32_t n_mrows, const int32_t *__restrict__ first_item,
+                                const int32_t *__restrict__ item_mslot, int32_t mitem0, int32_t d, const float *__restrict__ partial, int64_t ld_z,
+                                const float *__restrict__ bias, int relu, float *__restrict__ out_base, int64_t ld_out)
+{
+    const int d4 = (d + 3) >> 2;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c4 = (int)(t - i * d4);
+    if (i >= n_mrows) return;
+    const int32_t row = mrows[mrow0 + i];
+    const int32_t it0 = first_item[row], it1 = first_item[row + 1];
+    const int32_t ms0 = item_mslot[it0] - mitem0;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int32_t q = 0; q < it1 - it0; ++q) {
+        const float4 x = *reinterpret_cast<const float4 *>(partial + (int64_t)(ms0 + q) * ld_z + 4 * c4);
+        r.x += x.x;
+        r.y += x.y;
+        r.z += x.z;
+        r.w += x.w;
+    }
+    const int c = 4 * c4;
+    if (bias) {
+        r.x += bias[c];
+        if (c + 1 < d) r.y += bias[c + 1];
+        if (c + 2 < d) r.z += bias[c + 2];
+        if (c + 3 < d) r.w += bias[c + 3];
+    }
+    if (relu) {
+        r.x = fmaxf(r.x, 0.f);
+        r.y = fmaxf(r.y, 0.f);
+        r.z = fmaxf(r.z, 0.f);
+        r.w = fmaxf(r.w, 0.f);
+    }
+    *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c4) = r;
+}
+
 // D = g o [h_out > 0] (ReLU layer) or g
 __global__ void k_gat_dmask(const float *__restrict__ g, int64_t ld_g, const float *__restrict__ h_out, int64_t ld_h, int64_t rows, int32_t d,
                             float *__restrict__ D, int64_t ld_d)
@@ -176,57 +241,6 @@ __global__ void k_gat_dmask(const float *__restrict__ g, int64_t ld_g, const flo
     if (r >= rows) return;
     const float x = g[r * ld_g + c];
     D[r * ld_d + c] = (!h_out || h_out[r * ld_h + c] > 0.f) ? x : 0.f;
-}
-
-// backward, row side: one warp per inner row v keeps D_v in registers and walks the entries u of the row:
-//   t_v = sum alpha dalpha,  ds_dst[v] = sum alpha slope dalpha - t_v sum alpha slope   (alpha renormalised, see below)
-template <int NV>
-__global__ void __launch_bounds__(256)
-k_gat_bwd_rows(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t n, int32_t row0, int32_t n_rows,
-               const float *__restrict__ z_in, const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in,
-               const float *__restrict__ s_halo, const float *__restrict__ s_dst, const float *__restrict__ lse, int32_t d,
-               const float *__restrict__ D, int64_t ld_d, double *__restrict__ t_out, float *__restrict__ ds_dst)
-{
-    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int lane = threadIdx.x & 31;
-    if (w >= n_rows) return;
-    const int32_t row = row0 + (int32_t)w;
-    const int d4 = (d + 3) >> 2;
-    float4 dv[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int c4 = lane + 32 * v;
-        dv[v] = c4 < d4 ? ldz(D + (int64_t)row * ld_d, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    const int64_t e0 = lrowptr[row], e1 = lrowptr[row + 1];
-    const float sd = s_dst[row], l = lse[row];
-    // ds_dst = a2 - a1 a3 subtracts sums of the same size (it is exactly zero when every entry has the same LeakyReLU slope):
-    // the three sums are kept in double so that the difference keeps its digits
-    // the fp32 weights alpha = exp(e - lse) of a row sum to 1 + eps (rounding of lse), and ds_dst would inherit -eps t_v, which
-    // is not small against its true value; a0 = sum alpha renormalises them
-    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    for (int64_t e = e0; e < e1; ++e) {
-        const int32_t c = lenc[e];
-        const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
-        const float alpha = expf(lrelu(pre) - l);
-        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
-        const float *src = c < n ? z_in + (int64_t)c * ld_z : z_halo + (int64_t)(c - n) * ld_z;
-        double p = 0.0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c4 = lane + 32 * v;
-            if (c4 < d4) p += ddot4(dv[v], ldz(src, c4, d));
-        }
-        const double da = warp_sum_d(p);
-        a0 += (double)alpha;
-        a1 += (double)alpha * da;
-        a2 += (double)(alpha * slope) * da;
-        a3 += (double)alpha * (double)slope;
-    }
-    if (lane == 0) {
-        t_out[row] = a1 / a0;
-        ds_dst[row] = (float)(a2 / a0 - (a1 / a0) * (a3 / a0));
-    }
 }
 
 // backward, column side: one warp per node u keeps z_u in registers and walks the rows v that have u as an entry:
@@ -298,6 +312,170 @@ k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
         }
     }
     if (lane == 0) ds_src[u] = dssf;
+}
+
+// -------------------------------------------------------------------------------------
+// The same two sweeps over the SpMM's work items (rows cut into chunks of SAT_SPMM_CHUNK entries), one warp per item, so
+// that a hub row is walked by many warps; the per-item partial sums are added per row in item order by the combine kernels.
+// -------------------------------------------------------------------------------------
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_bwd_rows_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, const int32_t *__restrict__ item_row,
+                     const int32_t *__restrict__ first_item, int32_t item0, int32_t n_items, int32_t n, const float *__restrict__ z_in,
+                     const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_in, const float *__restrict__ s_halo,
+                     const float *__restrict__ s_dst, const float *__restrict__ lse, int32_t d, const float *__restrict__ D, int64_t ld_d,
+                     double *__restrict__ part4)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_items) return;
+    const int32_t item = item0 + (int32_t)w;
+    const int32_t row = item_row[item];
+    const int d4 = (d + 3) >> 2;
+    float4 dv[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        dv[v] = c4 < d4 ? ldz(D + (int64_t)row * ld_d, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t re = lrowptr[row + 1];
+    const int64_t e0 = lrowptr[row] + (int64_t)(item - first_item[row]) * SAT_SPMM_CHUNK;
+    const int64_t e1 = e0 + SAT_SPMM_CHUNK < re ? e0 + SAT_SPMM_CHUNK : re;
+    const float sd = s_dst[row], l = lse[row];
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    for (int64_t e = e0; e < e1; ++e) {
+        const int32_t c = lenc[e];
+        const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
+        const float alpha = expf(lrelu(pre) - l);
+        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+        const float *src = c < n ? z_in + (int64_t)c * ld_z : z_halo + (int64_t)(c - n) * ld_z;
+        double p = 0.0;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) p += ddot4(dv[v], ldz(src, c4, d));
+        }
+        const double da = warp_sum_d(p);
+        a0 += (double)alpha;
+        a1 += (double)alpha * da;
+        a2 += (double)(alpha * slope) * da;
+        a3 += (double)alpha * (double)slope;
+    }
+    if (lane == 0) {
+        double *o = part4 + 4 * w;
+        o[0] = a0;
+        o[1] = a1;
+        o[2] = a2;
+        o[3] = a3;
+    }
+}
+
+__global__ void k_gat_rows_combine(const int32_t *__restrict__ first_item, int32_t item0, int32_t row0, int32_t n_rows,
+                                   const double *__restrict__ part4, double *__restrict__ t_out, float *__restrict__ ds_dst)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_rows) return;
+    const int32_t row = row0 + (int32_t)i;
+    double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
+    for (int32_t it = first_item[row]; it < first_item[row + 1]; ++it) {
+        const double *p = part4 + 4 * (int64_t)(it - item0);
+        a0 += p[0];
+        a1 += p[1];
+        a2 += p[2];
+        a3 += p[3];
+    }
+    t_out[row] = a1 / a0;
+    ds_dst[row] = (float)(a2 / a0 - (a1 / a0) * (a3 / a0));
+}
+
+// column side for the inner nodes: the item's entries that lie in the inner prefix of the row of u
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_bwd_cols_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, const int32_t *__restrict__ inner_cnt,
+                     const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item, int32_t item0, int32_t n_items,
+                     const float *__restrict__ z_in, int64_t ld_z, const float *__restrict__ s_in, const float *__restrict__ s_dst,
+                     const float *__restrict__ lse, const double *__restrict__ t_in, int32_t d, const float *__restrict__ D, int64_t ld_d,
+                     float *__restrict__ pdz, double *__restrict__ pdss)
+{
+    const int64_t w = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (w >= n_items) return;
+    const int32_t item = item0 + (int32_t)w;
+    const int32_t u = item_row[item];
+    const int d4 = (d + 3) >> 2;
+    float4 zu[NV], acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        zu[v] = c4 < d4 ? ldz(z_in + (int64_t)u * ld_z, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t rb = lrowptr[u], re = rb + inner_cnt[u];
+    const int64_t e0 = rb + (int64_t)(item - first_item[u]) * SAT_SPMM_CHUNK;
+    const int64_t e1 = e0 + SAT_SPMM_CHUNK < re ? e0 + SAT_SPMM_CHUNK : re;
+    const float su = s_in[u];
+    double dss = 0.0;
+    for (int64_t e = e0; e < e1; ++e) {
+        const int32_t v_row = lenc[e];
+        const float pre = s_dst[v_row] + su;
+        const float alpha = expf(lrelu(pre) - lse[v_row]);
+        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+        const float *dr = D + (int64_t)v_row * ld_d;
+        double p = 0.0;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) {
+                const float4 x = ldz(dr, c4, d);
+                p += ddot4(x, zu[v]);
+                acc[v].x = fmaf(alpha, x.x, acc[v].x);
+                acc[v].y = fmaf(alpha, x.y, acc[v].y);
+                acc[v].z = fmaf(alpha, x.z, acc[v].z);
+                acc[v].w = fmaf(alpha, x.w, acc[v].w);
+            }
+        }
+        const double da = warp_sum_d(p);
+        dss += (double)(alpha * slope) * (da - t_in[v_row]);
+    }
+    float *o = pdz + w * ld_z;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        if (c4 < d4) *reinterpret_cast<float4 *>(o + 4 * c4) = acc[v];
+    }
+    if (lane == 0) pdss[w] = dss;
+}
+
+// dZ_u = sum of the item partials in item order + ds_src[u] a_src + ds_dst[u] a_dst; one thread per (row, float4 column)
+__global__ void k_gat_cols_combine(const int32_t *__restrict__ first_item, int32_t item0, int32_t row0, int32_t n_rows, int32_t d,
+                                   const float *__restrict__ pdz, int64_t ld_z, const double *__restrict__ pdss, const float *__restrict__ ds_dst,
+                                   const float *__restrict__ a_src, const float *__restrict__ a_dst, float *__restrict__ dz_base,
+                                   float *__restrict__ ds_src)
+{
+    const int d4 = (d + 3) >> 2;
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c4 = (int)(t - i * d4);
+    if (i >= n_rows) return;
+    const int32_t u = row0 + (int32_t)i;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    double dss = 0.0;
+    for (int32_t it = first_item[u]; it < first_item[u + 1]; ++it) {
+        const float4 x = *reinterpret_cast<const float4 *>(pdz + (int64_t)(it - item0) * ld_z + 4 * c4);
+        r.x += x.x;
+        r.y += x.y;
+        r.z += x.z;
+        r.w += x.w;
+        dss += pdss[it - item0];
+    }
+    const float s1 = (float)dss, s2 = ds_dst[u];
+    const int c = 4 * c4;
+    r.x += s1 * a_src[c] + s2 * a_dst[c];
+    r.y = c + 1 < d ? r.y + s1 * a_src[c + 1] + s2 * a_dst[c + 1] : 0.f;
+    r.z = c + 2 < d ? r.z + s1 * a_src[c + 2] + s2 * a_dst[c + 2] : 0.f;
+    r.w = c + 3 < d ? r.w + s1 * a_src[c + 3] + s2 * a_dst[c + 3] : 0.f;
+    *reinterpret_cast<float4 *>(dz_base + (int64_t)u * ld_z + 4 * c4) = r;
+    if (c4 == 0) ds_src[u] = s1;
 }
 
 // part[b][c] = sum over the rows r of block b, in order, of w[r] x[r][c]
@@ -427,13 +605,28 @@ extern "C" sat_status sat_gat_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int
     }
     if (v.n_rows > 0) {
         const int nv = ((d_out + 3) / 4 + 31) / 32;
-        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
-#define CALL(NV)                                                                                                                              \
-    k_gat_fwd<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->n, v.row0, v.n_rows, z_in, z_halo, ld_z, s_in, s_halo, s_dst, d_out, \
-                                                 bias, G.relu, lse, h_out - (int64_t)v.row0 * ld_out, ld_out)
+        float *partial = nullptr;
+        if (v.n_mitems > 0) {
+            SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * ld_z * sizeof(float)));
+            partial = (float *)ctx->buf_partial.p;
+        }
+        k_gat_lse<<<(unsigned)cdiv64((int64_t)v.n_rows * 32, 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->n, v.row0, v.n_rows, s_in, s_halo,
+                                                                                        s_dst, lse);
+        SAT_LAUNCHED(ctx);
+        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_items * 32, 256);
+        float *out_base = h_out - (int64_t)v.row0 * ld_out;
+#define CALL(NV)                                                                                                                                    \
+    k_gat_fwd_items<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->item_row, ctx->first_item, ctx->item_mslot, v.item0, v.n_items,    \
+                                                       v.mitem0, ctx->n, z_in, z_halo, ld_z, s_in, s_halo, s_dst, lse, d_out, bias, G.relu, out_base, \
+                                                       ld_out, partial)
         GAT_DISPATCH(nv, CALL);
 #undef CALL
         SAT_LAUNCHED(ctx);
+        if (v.n_mrows > 0) {
+            k_gat_fwd_fixup<<<(unsigned)cdiv64((int64_t)v.n_mrows * ((d_out + 3) / 4), 256), 256, 0, ctx->stream>>>(
+                ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, d_out, partial, ld_z, bias, G.relu, out_base, ld_out);
+            SAT_LAUNCHED(ctx);
+        }
     }
     for (int m = (part == SAT_ALL_PARTS ? 0 : part); m < (part == SAT_ALL_PARTS ? ctx->M : part + 1); ++m) G.valid[m] = 1;
     return SAT_OK;
@@ -485,19 +678,29 @@ extern "C" sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, con
             SAT_LAUNCHED(ctx);
         }
         SAT_TRY(sat_mask_rows(ctx, D, ld_z, v.n_rows, d_out, nullptr, 0, nullptr, 0, g_b, accumulate));
+        // per-item partial sums: 4 doubles for the row side, a dZ row and a double for the column side
+        const size_t n_it = (size_t)v.n_items;
+        SAT_TRY(sat_ensure(ctx, ctx->buf_gat_items, (5 * n_it * 2 + n_it * ld_z + 64) * sizeof(float)));
+        double *part4 = (double *)ctx->buf_gat_items.p, *pdss = part4 + 4 * n_it;
+        float *pdz = (float *)(pdss + n_it + (n_it & 1));   // 16-byte aligned rows after an even number of doubles
         ProfScope prof(ctx, SATK_GAT, 0.0, 0.0);
-        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_rows * 32, 256);
-#define CALL(NV)                                                                                                                                  \
-    k_gat_bwd_rows<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->n, v.row0, v.n_rows, z_in, z_halo, ld_z, s_in, s_halo, s_dst, lse, \
-                                                      d_out, Db, ld_z, t_b, ds_dst_b)
+        const unsigned grid = (unsigned)cdiv64((int64_t)v.n_items * 32, 256);
+#define CALL(NV)                                                                                                                                 \
+    k_gat_bwd_rows_items<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->item_row, ctx->first_item, v.item0, v.n_items, ctx->n, z_in, \
+                                                            z_halo, ld_z, s_in, s_halo, s_dst, lse, d_out, Db, ld_z, part4)
         GAT_DISPATCH(nv, CALL);
 #undef CALL
         SAT_LAUNCHED(ctx);
-#define CALL(NV)                                                                                                                                    \
-    k_gat_bwd_cols<NV, 0><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->inner_cnt, v.row0, v.n_rows, z_in, ld_z, s_in, s_dst, lse, t_b, \
-                                                         ds_dst_b, d_out, Db, ld_z, a_src, a_dst, dz_in_b, ds_in_b)
+        k_gat_rows_combine<<<(unsigned)cdiv64(v.n_rows, 256), 256, 0, ctx->stream>>>(ctx->first_item, v.item0, v.row0, v.n_rows, part4, t_b, ds_dst_b);
+        SAT_LAUNCHED(ctx);
+#define CALL(NV)                                                                                                                                  \
+    k_gat_bwd_cols_items<NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, ctx->inner_cnt, ctx->item_row, ctx->first_item, v.item0, v.n_items, \
+                                                            z_in, ld_z, s_in, s_dst, lse, t_b, d_out, Db, ld_z, pdz, pdss)
         GAT_DISPATCH(nv, CALL);
 #undef CALL
+        SAT_LAUNCHED(ctx);
+        k_gat_cols_combine<<<(unsigned)cdiv64((int64_t)v.n_rows * ((d_out + 3) / 4), 256), 256, 0, ctx->stream>>>(
+            ctx->first_item, v.item0, v.row0, v.n_rows, d_out, pdz, ld_z, pdss, ds_dst_b, a_src, a_dst, dz_in_b, ds_in_b);
         SAT_LAUNCHED(ctx);
     } else if (!accumulate) {
         SAT_CUDA(ctx, cudaMemsetAsync(g_b, 0, (size_t)d_out * sizeof(float), ctx->stream));

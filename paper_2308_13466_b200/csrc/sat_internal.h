@@ -143,7 +143,7 @@ struct sat_ctx {
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
-        buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out, buf_gat;
+        buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out, buf_gat, buf_gat_items;
 };
 
 sat_status sat_fail(sat_ctx *ctx, sat_status code, const char *fmt, ...);
