@@ -268,6 +268,7 @@ k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
         acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
     const int64_t e0 = ptr[u], e1 = HALO ? ptr[u + 1] : e0 + inner_cnt[u];
+    if (HALO && e1 - e0 > SAT_HROW_LONG) return;   // long halo rows: k_gat_bwd_cols_long, a thread block each
     const float su = s_u[u];
     double dss = 0.0;
     for (int64_t e = e0; e < e1; ++e) {
@@ -476,6 +477,84 @@ __global__ void k_gat_cols_combine(const int32_t *__restrict__ first_item, int32
     r.w = c + 3 < d ? r.w + s1 * a_src[c + 3] + s2 * a_dst[c + 3] : 0.f;
     *reinterpret_cast<float4 *>(dz_base + (int64_t)u * ld_z + 4 * c4) = r;
     if (c4 == 0) ds_src[u] = s1;
+}
+
+// column side for the halo rows with more than SAT_HROW_LONG entries (hub nodes seen from another partition): one thread
+// block per row, its 8 warps taking the entries round-robin; the warps' partial sums are added in warp order.
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_gat_bwd_cols_long(const int32_t *__restrict__ hlong, int32_t hlong0, const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
+                    const float *__restrict__ z_halo, int64_t ld_z, const float *__restrict__ s_halo, const float *__restrict__ s_dst,
+                    const float *__restrict__ lse, const double *__restrict__ t_in, int32_t d, const float *__restrict__ D, int64_t ld_d,
+                    const float *__restrict__ a_src, float *__restrict__ dz_base, float *__restrict__ ds_src)
+{
+    __shared__ float4 red[8][NV][32];
+    __shared__ double red_s[8];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t u = hlong[hlong0 + blockIdx.x];
+    const int d4 = (d + 3) >> 2;
+    float4 zu[NV], acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        zu[v] = c4 < d4 ? ldz(z_halo + u * ld_z, c4, d) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int64_t e0 = ptr[u], e1 = ptr[u + 1];
+    const float su = s_halo[u];
+    double dss = 0.0;
+    for (int64_t e = e0 + warp; e < e1; e += 8) {
+        const int32_t v_row = idx[e];
+        const float pre = s_dst[v_row] + su;
+        const float alpha = expf(lrelu(pre) - lse[v_row]);
+        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+        const float *dr = D + (int64_t)v_row * ld_d;
+        double p = 0.0;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int c4 = lane + 32 * v;
+            if (c4 < d4) {
+                const float4 x = ldz(dr, c4, d);
+                p += ddot4(x, zu[v]);
+                acc[v].x = fmaf(alpha, x.x, acc[v].x);
+                acc[v].y = fmaf(alpha, x.y, acc[v].y);
+                acc[v].z = fmaf(alpha, x.z, acc[v].z);
+                acc[v].w = fmaf(alpha, x.w, acc[v].w);
+            }
+        }
+        const double da = warp_sum_d(p);
+        dss += (double)(alpha * slope) * (da - t_in[v_row]);
+    }
+#pragma unroll
+    for (int v = 0; v < NV; ++v) red[warp][v][lane] = acc[v];
+    if (lane == 0) red_s[warp] = dss;
+    __syncthreads();
+    if (warp != 0) return;
+    double tot = 0.0;
+    for (int q = 0; q < 8; ++q) tot += red_s[q];
+    const float s1 = (float)tot;
+    float *o = dz_base + u * ld_z;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) {
+        const int c4 = lane + 32 * v;
+        if (c4 < d4) {
+            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int q = 0; q < 8; ++q) {
+                const float4 x = red[q][v][lane];
+                r.x += x.x;
+                r.y += x.y;
+                r.z += x.z;
+                r.w += x.w;
+            }
+            const int c = 4 * c4;
+            r.x += s1 * a_src[c];
+            r.y = c + 1 < d ? r.y + s1 * a_src[c + 1] : 0.f;
+            r.z = c + 2 < d ? r.z + s1 * a_src[c + 2] : 0.f;
+            r.w = c + 3 < d ? r.w + s1 * a_src[c + 3] : 0.f;
+            *reinterpret_cast<float4 *>(o + 4 * c4) = r;
+        }
+    }
+    if (lane == 0) ds_src[u] = s1;
 }
 
 // part[b][c] = sum over the rows r of block b, in order, of w[r] x[r][c]
@@ -714,6 +793,14 @@ extern "C" sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, con
         GAT_DISPATCH(nv, CALL);
 #undef CALL
         SAT_LAUNCHED(ctx);
+        if (v.n_hlong > 0) {
+#define CALL(NV)                                                                                                                                  \
+    k_gat_bwd_cols_long<NV><<<(unsigned)v.n_hlong, 256, 0, ctx->stream>>>(ctx->hlong, v.hlong0, ctx->hrow_ptr, ctx->hrow_pos, z_halo, ld_z, s_halo, s_dst, \
+                                                                          lse, t_b, d_out, Db, ld_z, a_src, dz_halo_b, ds_halo_b)
+            GAT_DISPATCH(nv, CALL);
+#undef CALL
+            SAT_LAUNCHED(ctx);
+        }
     }
     const int64_t halo_rows = v.n_rows > 0 ? v.n_halo : 0;
     // parameter gradients
