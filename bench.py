@@ -35,7 +35,7 @@ if ROOT not in sys.path:
 # workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
 # gemm_nn: 302 MB = the 256-wide layer transform; gemm_side: 304 MB = the LSTM recurrence step (profiles/k_gemm_tc_k_medium.md);
 # spmm_fwd: 684 MB = the d = 256 launch (profiles/k_spmm_items_medium.md).
-NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 683.6e6, "gemm_side": 304.4e6}
+NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 757.9e6, "gemm_side": 304.4e6}
 
 # predictor update period Delta-T of Algorithm 1 followed by the run (epochs between two parameter-version bumps)
 PRED_PERIOD = 10
