@@ -15,18 +15,9 @@
 // still walks a halo row with one warp.
 #include "sat_internal.h"
 
-#define CHECK_CTX(ctx)                                                                             \
-    do {                                                                                           \
-        if (!(ctx)) return SAT_EINVAL;                                                             \
-        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
-        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
-    } while (0)
-
 #define GAT_SLOPE 0.2f
 #define GAT_MAX_NV 8   /* float4 per lane: widths up to 1024 */
 
-static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
-static bool ok_ld(int32_t ld, int32_t d) { return ld >= d && (ld & 3) == 0; }
 
 __device__ __forceinline__ float warp_sum(float x)
 {

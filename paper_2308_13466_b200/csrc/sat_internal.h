@@ -196,6 +196,21 @@ struct ProfScope {
     }
 };
 
+// entry-point prologue: a usable context on its device
+#define CHECK_CTX(ctx)                                                                             \
+    do {                                                                                           \
+        if (!(ctx)) return SAT_EINVAL;                                                             \
+        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
+        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
+    } while (0)
+
+// argument checks of the entry points: 16-byte aligned base, leading dimension >= width and a multiple of 4 floats
+static inline bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+static inline bool ok_ld(int32_t ld, int32_t d) { return ld >= d && (ld & 3) == 0; }
+// ring buffer `age` epochs back from the newest committed snapshot (age 0), and its base address
+static inline int32_t ring_index(const sat_ctx *ctx, int32_t age) { return ((ctx->write_idx - 1 - age) % (ctx->tau + 1) + (ctx->tau + 1)) % (ctx->tau + 1); }
+static inline float *ring_buf(const sat_ctx *ctx, const CacheLayer *c, int32_t idx) { return c->buf + (size_t)idx * ctx->n_slots * c->ld; }
+
 static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline int32_t round_up4(int32_t x) { return (x + 3) & ~3; }
 

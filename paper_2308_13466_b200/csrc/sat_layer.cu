@@ -4,15 +4,6 @@
 
 #include "sat_internal.h"
 
-#define CHECK_CTX(ctx)                                                                             \
-    do {                                                                                           \
-        if (!(ctx)) return SAT_EINVAL;                                                             \
-        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
-        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
-    } while (0)
-
-static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
-static bool ok_ld(int32_t ld, int32_t d) { return ld >= d && (ld & 3) == 0; }
 
 template <typename T>
 static sat_status dev_realloc(sat_ctx *ctx, T **p, int64_t count)
@@ -93,8 +84,6 @@ static sat_status cache_layer(sat_ctx *ctx, int32_t layer, CacheLayer **c, const
 }
 
 // buffer index of the snapshot of a given age (0 = newest committed)
-static int32_t ring_index(const sat_ctx *ctx, int32_t age) { return ((ctx->write_idx - 1 - age) % (ctx->tau + 1) + (ctx->tau + 1)) % (ctx->tau + 1); }
-static float *ring_buf(const sat_ctx *ctx, const CacheLayer *c, int32_t idx) { return c->buf + (size_t)idx * ctx->n_slots * c->ld; }
 
 extern "C" sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer, const float *h_out, int32_t ld)
 {

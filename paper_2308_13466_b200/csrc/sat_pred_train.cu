@@ -5,16 +5,6 @@
 // GEMM kernels as the layer steps; this file holds the element-wise and sparse kernels around them.
 #include "sat_internal.h"
 
-#define CHECK_CTX(ctx)                                                                             \
-    do {                                                                                           \
-        if (!(ctx)) return SAT_EINVAL;                                                             \
-        if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
-        SAT_CUDA(ctx, cudaSetDevice((ctx)->device));                                               \
-    } while (0)
-
-static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
-static int32_t ring_index(const sat_ctx *ctx, int32_t age) { return ((ctx->write_idx - 1 - age) % (ctx->tau + 1) + (ctx->tau + 1)) % (ctx->tau + 1); }
-static float *ring_buf(const sat_ctx *ctx, const CacheLayer *c, int32_t idx) { return c->buf + (size_t)idx * ctx->n_slots * c->ld; }
 
 // -------------------------------------------------------------------------------------
 // LSTM cell kernels.  A thread owns four consecutive hidden units of a row (one 16-byte access per gate block and state
