@@ -153,12 +153,13 @@ sat_status sat_cache_init(sat_ctx *ctx, int32_t n_cached_layers, const int32_t *
 /* Predictor parameters g_omega (Section "Embedding Predictor": LSTM + GCN), all DEVICE,
  * dense row-major without padding: Wx [d x 4h], Uh [h x 4h], b [4h] (gate order i, f, g, o),
  * Wg [h x d], bg [d].  d = width of the cached layer.
- * version: 0 = no promise.  A non-zero version promises that the VALUES of Wx and b are the same as in every earlier
+ * version: 0 = no promise.  A non-zero version promises that the VALUES of all five arrays are the same as in every earlier
  * call that passed the same version for this cached layer (the paper updates the predictor only every Delta-T epochs,
  * Algorithm 1 "Embedding predictor update"; bump the version after each update).  The library then keeps the input
  * projection x Wx + b of every new snapshot and reuses it in the following epochs — the result is the same LSTM, one of
  * tau input projections per epoch instead of tau.  After a version bump the older snapshots are not re-projected: their
- * steps contract over [x | s] as without a version, until they have left the window.  Costs (tau+1) * |C| * 4h * 4 bytes per
+ * steps contract over [x | s] as without a version, until they have left the window.  The library also keeps its packed
+ * copies of the weights and biases (a few hundred KB per cached layer) for as long as the version stays the same.  Costs (tau+1) * |C| * 4h * 4 bytes per
  * cached layer. */
 typedef struct sat_pred_params {
     const float *Wx, *Uh, *b, *Wg, *bg;

@@ -194,7 +194,7 @@ def sat_cache_init(ctx, widths, tau: int, mode: int = SAT_CACHE_ZERO, init=None)
 
 
 def make_pred_params(Wx, Uh, b, Wg, bg, h: int, version: int = 0, cell: int = 0) -> sat_pred_params:
-    """version != 0 promises that the values of Wx and b stay the same for as long as the same version is passed.
+    """version != 0 promises that the values of all five arrays stay the same for as long as the same version is passed.
     cell: SAT_CELL_LSTM (Wx [d, 4h], Uh [h, 4h], b [4h]) or SAT_CELL_GRU (Wx [d, 3h], Uh [h, 3h], b [4h])."""
     for t in (Wx, Uh, b, Wg, bg):
         assert t.is_cuda and t.is_contiguous()

@@ -138,6 +138,11 @@ static void free_cache(sat_ctx *ctx)
         dev_free(&ctx->cache[i].buf);
         dev_free(&ctx->cache[i].S);
         dev_free(&ctx->cache[i].proj);
+        sat_free_buf(ctx->cache[i].pk_wx);
+        sat_free_buf(ctx->cache[i].pk_uh);
+        sat_free_buf(ctx->cache[i].pk_wg);
+        sat_free_buf(ctx->cache[i].pk_b);
+        sat_free_buf(ctx->cache[i].pk_bg);
         ctx->cache[i] = CacheLayer();
     }
     ctx->cache_ok = false;

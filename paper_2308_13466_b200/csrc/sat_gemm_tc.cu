@@ -978,6 +978,21 @@ sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1,
     return SAT_OK;
 }
 
+// the description of planes that an earlier sat_tc_weights call (single source, k terms, n outputs) left in `buf`
+sat_status sat_tc_weights_layout(int32_t k, int32_t n, const DevBuf &buf, TcWeights *out)
+{
+    const int32_t k_pad = (k + TC_BK - 1) / TC_BK * TC_BK;
+    const int32_t bn = tile_n_for(n);
+    const int32_t n_pad = (n + bn - 1) / bn * bn;
+    const size_t plane = ((size_t)n_pad * k_pad * sizeof(float) + 255) & ~(size_t)255;
+    if (!buf.p || buf.bytes < 2 * plane) return SAT_ESTATE;
+    out->hi = (float *)buf.p;
+    out->lo = (float *)((char *)buf.p + plane);
+    out->ld = k_pad;
+    out->n_pad = n_pad;
+    return SAT_OK;
+}
+
 static bool g_attr_mn = false;
 #define TC_SMEM_BUDGET (100 * 1024)
 
@@ -1037,11 +1052,14 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     ep.bias = nullptr;
     if (eh.bias) {  // zero-padded copy so that the epilogue can read whole 128-bit vectors
         const size_t padded = (size_t)cdiv64(n, bn) * bn;
-        SAT_TRY(sat_ensure(ctx, ctx->buf_bias, padded * sizeof(float)));
-        k_pack_bias<<<(unsigned)cdiv64(padded, 256), 256, 0, ctx->stream>>>(eh.bias, n, (int32_t)padded, eh.lstm_h > 0 ? eh.lstm_h : eh.pack_gate_h,
-                                                                            (float *)ctx->buf_bias.p);
-        SAT_LAUNCHED(ctx);
-        ep.bias = (const float *)ctx->buf_bias.p;
+        DevBuf &home = eh.bias_home ? *eh.bias_home : ctx->buf_bias;
+        if (!(eh.bias_home && eh.bias_ready && home.bytes >= padded * sizeof(float))) {
+            SAT_TRY(sat_ensure(ctx, home, padded * sizeof(float)));
+            k_pack_bias<<<(unsigned)cdiv64(padded, 256), 256, 0, ctx->stream>>>(eh.bias, n, (int32_t)padded, eh.lstm_h > 0 ? eh.lstm_h : eh.pack_gate_h,
+                                                                                (float *)home.p);
+            SAT_LAUNCHED(ctx);
+        }
+        ep.bias = (const float *)home.p;
     }
     ep.lstm_h = eh.lstm_h;
     ep.lstm_first = eh.lstm_first;

@@ -41,6 +41,11 @@ struct CacheLayer {
     float *proj = nullptr;
     int32_t proj_h = 0;
     std::vector<uint64_t> proj_tag;
+    // packed (TF32 hi / lo planes, padded) copies of the predictor's weights and biases, reused while the caller's
+    // parameter version stays the same: input weights Wx, recurrent weights Uh, output weights Wg, gate bias b, output bias bg
+    DevBuf pk_wx, pk_uh, pk_wg, pk_b, pk_bg;
+    uint64_t tag_wx = 0, tag_uh = 0, tag_wg = 0, tag_b = 0, tag_bg = 0;
+    int32_t pk_h = 0;
 };
 
 // Gradient-side history of one layer j >= 2 (Appendix, back-propagation of SAT): Q^(j) = sum_m P_out^(m)T D^(m, j) over the
@@ -340,6 +345,10 @@ struct TcEpilogueHost {
     const float *addend = nullptr;     // dense [m x ld_addend], added to the accumulators before the LSTM cell (row-aligned)
     int32_t ld_addend = 0;
     int32_t pack_gate_h = 0;           // > 0: the bias is interleaved like weights packed with gate_h (without the LSTM epilogue)
+    // optional home of the padded bias copy (default: a scratch buffer of the context, repacked by every call); with
+    // bias_ready the copy in *bias_home is current and is used as it is
+    DevBuf *bias_home = nullptr;
+    bool bias_ready = false;
 };
 // tensor-core path on / off for a contraction with n outputs and k terms (SAT_NO_TC=1 in the environment forces the CUDA cores)
 bool sat_use_tc(int32_t n, int32_t k);
@@ -351,6 +360,7 @@ sat_status sat_mask_rows(sat_ctx *ctx, const float *src, int32_t ld, int64_t row
 // of hidden unit j (what the fused LSTM epilogue expects)
 sat_status sat_tc_weights(sat_ctx *ctx, const float *W, int32_t ldw, int32_t k1, const float *W2, int32_t ldw2, int32_t k2, int32_t n,
                           int transpose, DevBuf &buf, TcWeights *out, int32_t gate_h = 0);
+sat_status sat_tc_weights_layout(int32_t k, int32_t n, const DevBuf &buf, TcWeights *out);
 // C[m x n] = [A | A2] B^T (+ epilogue)
 sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32_t lda, int32_t k1, const float *A2, int32_t lda2, int32_t k2,
                        const TcWeights &Bw, const TcEpilogueHost &eh, int family);

@@ -297,15 +297,33 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
     }
     TcWeights Wp, Wxu, Up;   // Wx alone, [Wx ; Uh], Uh alone (all gate-interleaved)
     bool have_wp = false, have_wxu = false, have_up = false;
+    if (c->pk_h != h) {      // another predictor width: nothing packed fits
+        c->tag_wx = c->tag_uh = c->tag_wg = c->tag_b = c->tag_bg = 0;
+        c->pk_h = h;
+    }
+    // the packed weight planes live in the cache layer and are made once per parameter version
+    auto pack_wx = [&]() -> sat_status {
+        if (have_wp) return SAT_OK;
+        if (c->tag_wx == p->version) {
+            SAT_TRY(sat_tc_weights_layout(d, 4 * h, c->pk_wx, &Wp));
+        } else {
+            SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, c->pk_wx, &Wp, h));
+            c->tag_wx = p->version;
+        }
+        have_wp = true;
+        return SAT_OK;
+    };
     const int32_t newest = ring_index(ctx, 0);
     if (c->proj_tag[newest] != p->version) {
-        SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
-        have_wp = true;
+        SAT_TRY(pack_wx());
         TcEpilogueHost eh;
         eh.C = c->proj + (int64_t)newest * plane;
         eh.ldc = 4 * h;
         eh.bias = p->b;
         eh.pack_gate_h = h;
+        eh.bias_home = &c->pk_b;
+        eh.bias_ready = c->tag_b == p->version;
+        c->tag_b = p->version;
         SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, newest), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
         c->proj_tag[newest] = p->version;
     }
@@ -323,14 +341,20 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
             k_lstm_cell_first<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(pr, rows, h, cell, c->S);
             SAT_LAUNCHED(ctx);
         } else if (cached) {
-            if (!have_up) SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit2, &Up, h));
+            if (!have_up) {
+                if (c->tag_uh == p->version) {
+                    SAT_TRY(sat_tc_weights_layout(h, 4 * h, c->pk_uh, &Up));
+                } else {
+                    SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, c->pk_uh, &Up, h));
+                    c->tag_uh = p->version;
+                }
+            }
             have_up = true;
             eh.addend = pr;
             eh.ld_addend = 4 * h;
             SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
         } else if (t == 0) {
-            if (!have_wp) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, nullptr, 0, 0, 4 * h, 1, ctx->buf_wsplit, &Wp, h));
-            have_wp = true;
+            SAT_TRY(pack_wx());
             eh.bias = p->b;
             eh.lstm_first = 1;
             SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
@@ -531,8 +555,24 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
     SAT_TRY(sat_spmm_hrow(ctx, v, h, c->S, h, 1, c->S, a - v.halo0 * ld_a, ld_a));
     if (sat_use_tc(d, h)) {
         TcWeights Wg;
-        SAT_TRY(sat_tc_weights(ctx, params->Wg, d, h, nullptr, 0, 0, d, 1, ctx->buf_wsplit, &Wg));
         TcEpilogueHost eh;
+        if (params->version != 0 && params->cell == SAT_CELL_LSTM) {   // packed output weights and bias kept per parameter version
+            if (c->pk_h != h) {
+                c->tag_wx = c->tag_uh = c->tag_wg = c->tag_b = c->tag_bg = 0;
+                c->pk_h = h;
+            }
+            if (c->tag_wg == params->version) {
+                SAT_TRY(sat_tc_weights_layout(h, d, c->pk_wg, &Wg));
+            } else {
+                SAT_TRY(sat_tc_weights(ctx, params->Wg, d, h, nullptr, 0, 0, d, 1, c->pk_wg, &Wg));
+                c->tag_wg = params->version;
+            }
+            eh.bias_home = &c->pk_bg;
+            eh.bias_ready = c->tag_bg == params->version;
+            c->tag_bg = params->version;
+        } else {
+            SAT_TRY(sat_tc_weights(ctx, params->Wg, d, h, nullptr, 0, 0, d, 1, ctx->buf_wsplit, &Wg));
+        }
         eh.C = halo_out;
         eh.ldc = ld_out;
         eh.bias = params->bg;
