@@ -340,6 +340,9 @@ sat_status sat_cache_set_state(sat_ctx *ctx, int32_t write_idx, int32_t n_valid)
 sat_status sat_loss_grad(sat_ctx *ctx, int32_t part, int kind, int32_t n_classes, const float *z, int32_t ld_z,
                          const void *labels, double *loss_sum, float *g, int32_t ld_g);
 sat_status sat_sgd_step(sat_ctx *ctx, int64_t count, float *w, const float *g, float lr);
+/* The same step on n_arrays arrays at once: counts[i] floats of w[i] and g[i] (HOST arrays of sizes and of DEVICE pointers);
+ * one launch per 16 arrays. */
+sat_status sat_sgd_steps(sat_ctx *ctx, int32_t n_arrays, const int64_t *counts, float *const *w, const float *const *g, float lr);
 
 /* ---------------------------------------------------------------------------------------
  * The dense contractions of the layer step on caller tensors (all DEVICE fp32; the paper has no counterpart:

@@ -60,7 +60,7 @@ EXPORTS = [
     "sat_create", "sat_destroy", "sat_last_error", "sat_sync_status", "sat_graph_load", "sat_graph_dinv", "sat_partition",
     "sat_part_sizes", "sat_part_lists", "sat_slot_map", "sat_gather_rows", "sat_cache_init", "sat_predict",
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
-    "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step",
+    "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step", "sat_sgd_steps",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
     "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd",
 ]
@@ -274,6 +274,16 @@ def sat_loss_grad(ctx, part: int, kind: int, z, labels, loss_sum, g):
     """labels: int32 [n] (CE) or uint8 [n, C] (BCE) CUDA tensor; loss_sum: float64 CUDA scalar tensor or None."""
     _check(ctx, _lib.sat_loss_grad(ctx, C.c_int32(part), C.c_int(kind), C.c_int32(z.shape[1]), _dev(z), C.c_int32(_ld(z)),
                                    _dev(labels), _dev(loss_sum), _dev(g), C.c_int32(_ld(g))))
+
+
+def sat_sgd_steps(ctx, ws, gs, lr: float):
+    """w <- w - lr g for a list of (contiguous CUDA fp32) parameter tensors and their gradients, in one launch per 16."""
+    n = len(ws)
+    assert n == len(gs) and all(w.is_contiguous() and g.is_contiguous() and w.numel() == g.numel() for w, g in zip(ws, gs))
+    counts = (C.c_int64 * n)(*[int(w.numel()) for w in ws])
+    wp = (C.c_void_p * n)(*[w.data_ptr() for w in ws])
+    gp = (C.c_void_p * n)(*[g.data_ptr() for g in gs])
+    _check(ctx, _lib.sat_sgd_steps(ctx, C.c_int32(n), counts, wp, gp, C.c_float(lr)))
 
 
 def sat_sgd_step(ctx, w, g, lr: float):

@@ -1060,3 +1060,46 @@ extern "C" sat_status sat_sgd_step(sat_ctx *ctx, int64_t count, float *w, const 
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
+
+// the same step on up to SAT_SGD_MAX arrays in one launch (the parameter arrays of a model are many and small)
+#define SAT_SGD_MAX 16
+struct SgdBatch {
+    float *w[SAT_SGD_MAX];
+    const float *g[SAT_SGD_MAX];
+    int64_t end[SAT_SGD_MAX];   // running totals of the element counts
+    int32_t n;
+};
+
+__global__ void k_sgd_many(SgdBatch b, float lr)
+{
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= b.end[b.n - 1]) return;
+    int t = 0;
+    while (i >= b.end[t]) ++t;
+    const int64_t j = i - (t ? b.end[t - 1] : 0);
+    b.w[t][j] = b.w[t][j] - lr * b.g[t][j];
+}
+
+extern "C" sat_status sat_sgd_steps(sat_ctx *ctx, int32_t n_arrays, const int64_t *counts, float *const *w, const float *const *g, float lr)
+{
+    CHECK_CTX(ctx);
+    if (n_arrays < 0 || (n_arrays > 0 && (!counts || !w || !g))) return sat_fail(ctx, SAT_EINVAL, "sat_sgd_steps: null argument");
+    for (int32_t a0 = 0; a0 < n_arrays; a0 += SAT_SGD_MAX) {
+        SgdBatch b;
+        b.n = 0;
+        int64_t total = 0;
+        for (int32_t a = a0; a < n_arrays && a < a0 + SAT_SGD_MAX; ++a) {
+            if (counts[a] < 0 || (counts[a] > 0 && (!w[a] || !g[a]))) return sat_fail(ctx, SAT_EINVAL, "sat_sgd_steps: null tensor %d", a);
+            if (counts[a] == 0) continue;
+            total += counts[a];
+            b.w[b.n] = w[a];
+            b.g[b.n] = g[a];
+            b.end[b.n] = total;
+            ++b.n;
+        }
+        if (b.n == 0) continue;
+        k_sgd_many<<<(unsigned)cdiv64(total, 256), 256, 0, ctx->stream>>>(b, lr);
+        SAT_LAUNCHED(ctx);
+    }
+    return SAT_OK;
+}

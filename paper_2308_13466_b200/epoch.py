@@ -131,8 +131,7 @@ class SatEpoch:
                     losses.append(loss)
                     if len(losses) > 1 and losses[-1] > (1.0 - min_gain) * losses[-2]:
                         break
-                for t, g in zip(p._keep, p._grads):
-                    B.sat_sgd_step(self.ctx, t, g, lr)
+                B.sat_sgd_steps(self.ctx, list(p._keep), list(p._grads), lr)
                 if p.version:
                     p.version += 1
             seen.append(losses)
@@ -148,9 +147,7 @@ class SatEpoch:
             self.pred_update(pred, pred_lr)
         B.sat_cache_commit(self.ctx)
         if lr is not None:
-            for l in range(self.L):
-                B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
-                B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
+            B.sat_sgd_steps(self.ctx, list(W) + list(b), list(self.gW) + list(self.gb), lr)
 
     def step_per_partition(self, W, b, pred, order=None, lr: float | None = None, grad_history: bool = False):
         """Same epoch, one partition at a time (the LSTM state table is computed by the first call of every layer)."""
@@ -159,9 +156,7 @@ class SatEpoch:
             self._forward_backward(m, W, b, pred, 0 if i == 0 else 1, 0 if i == 0 else 1, grad_history)
         B.sat_cache_commit(self.ctx)
         if lr is not None:
-            for l in range(self.L):
-                B.sat_sgd_step(self.ctx, W[l], self.gW[l], lr)
-                B.sat_sgd_step(self.ctx, b[l], self.gb[l], lr)
+            B.sat_sgd_steps(self.ctx, list(W) + list(b), list(self.gW) + list(self.gb), lr)
 
     # ---- graph-attention backbone ---------------------------------------------------
     def step_gat(self, params, pred, lr: float | None = None):
@@ -199,6 +194,5 @@ class SatEpoch:
             g = g_in
         B.sat_cache_commit(ctx)
         if lr is not None:
-            for p, gr in zip(params, self.gat_grads):
-                for k in p:
-                    B.sat_sgd_step(ctx, p[k], gr[k], lr)
+            keys = [(l, k) for l, p in enumerate(params) for k in p]
+            B.sat_sgd_steps(ctx, [params[l][k] for l, k in keys], [self.gat_grads[l][k] for l, k in keys], lr)

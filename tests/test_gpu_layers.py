@@ -281,3 +281,29 @@ def test_shrunk_workloads_every_call(B, name, shrink, parts):
         print(name, {k: f"{v:.2e}" for k, v in worst.items()})
     finally:
         case.close()
+
+
+def test_parameter_step_on_many_arrays(B):
+    """sat_sgd_steps on a list of arrays (more than one launch's worth, one of them empty) equals sat_sgd_step array by array."""
+    import torch
+    ctx = B.sat_create(0, torch.cuda.current_stream().cuda_stream)
+    try:
+        rng = np.random.default_rng(2)
+        shapes = [(7,), (128, 256), (0,), (1,), (40,), (256, 40)] + [(3 + i,) for i in range(14)]
+        ws = [dev(rng.standard_normal(s).astype(np.float32)) for s in shapes]
+        gs = [dev(rng.standard_normal(s).astype(np.float32)) for s in shapes]
+        one = [w.clone() for w in ws]
+        for w, g in zip(one, gs):
+            B.sat_sgd_step(ctx, w, g, 0.37)
+        B.sat_sgd_steps(ctx, ws, gs, 0.37)
+        torch.cuda.synchronize()
+        for a, b_ in zip(ws, one):
+            assert torch.equal(a, b_)
+        # and the step itself: w - lr g
+        w0 = rng.standard_normal((5, 9)).astype(np.float32)
+        g0 = rng.standard_normal((5, 9)).astype(np.float32)
+        wd = dev(w0)
+        B.sat_sgd_steps(ctx, [wd], [dev(g0)], 0.25)
+        assert_close(wd.cpu().numpy(), w0.astype(np.float64) - 0.25 * g0.astype(np.float64), "w - lr g", 1e-6)
+    finally:
+        B.sat_destroy(ctx)
