@@ -54,6 +54,11 @@ enum { SAT_HOST = 0, SAT_DEVICE = 1 };                   /* where an index array
 enum { SAT_ALL_PARTS = -1 };
 enum { SAT_PART_GIVEN = 0, SAT_PART_CONTIG_BLOCKS = 1 }; /* sat_partition methods                */
 enum { SAT_ACT_NONE = 0, SAT_ACT_RELU = 1 };
+/* Flag for the `act` argument of sat_layer_fwd (act = SAT_ACT_* | SAT_FWD_PUSH): the rows of h_out that belong to boundary
+ * nodes are also written into the write buffer of cached layer `layer`, exactly what sat_cache_update(part, layer, h_out)
+ * does afterwards (Algorithm 1 "Push"), from the epilogue of the layer transform instead of a second pass over h_out.
+ * Needs sat_cache_init with that layer cached at width d_out (SAT_ESTATE / SAT_EINVAL otherwise). */
+#define SAT_FWD_PUSH 0x100
 enum { SAT_LOSS_SOFTMAX_CE = 0, SAT_LOSS_SIGMOID_BCE = 1 };
 enum { SAT_ROWS_INNER = 0, SAT_ROWS_HALO = 1 };          /* sat_gather_rows                      */
 enum { SAT_CACHE_ZERO = 0, SAT_CACHE_COPY = 1 };         /* sat_cache_init                       */

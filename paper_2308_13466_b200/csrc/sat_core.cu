@@ -113,6 +113,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->slot);
     dev_free(&ctx->push_row);
     dev_free(&ctx->push_slot);
+    dev_free(&ctx->row_slot);
     dev_free(&ctx->hs_ptr);
     dev_free(&ctx->hs_pos);
     dev_free(&ctx->lrowptr);

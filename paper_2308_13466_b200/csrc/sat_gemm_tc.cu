@@ -235,6 +235,9 @@ struct TcEpilogue {
     float *lstm_c;       // cell state in the blocked layout of sat_cell_offset
     const float *addend; // [M x ld_addend] added to the gate pre-activations (cached input projection), or null
     int64_t ld_addend;
+    float *push_dst;     // (EPI_PUSH) row i is also written to push_dst + push_slot[i] * ld_push when push_slot[i] >= 0
+    const int32_t *push_slot;
+    int64_t ld_push;
 };
 
 struct TcShared {
@@ -267,7 +270,7 @@ struct TcShared {
 // LSTM input projection) keep a ring of 32 x 32 side tiles per epilogue warp in shared memory, filled by cp.async ahead of
 // the consumer: one chunk in flight per warp left the loads latency-bound at ~2 TB/s.  Those variants contract over a
 // small K (the predictor width), so they give up main-loop stages for the ring.
-enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3 };
+enum { EPI_PLAIN = 0, EPI_RESID = 1, EPI_LSTM = 2, EPI_LSTM_ADD = 3, EPI_PUSH = 4 };   // EPI_PUSH = EPI_PLAIN + a second copy of the rows that have a cache slot
 template <int EPI> struct TckCfg { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = epi_warps * 4096; };
 template <> struct TckCfg<EPI_RESID> { static constexpr int stages = 2, ring = 1, conv_warps = 2, epi_warps = 12, out_bytes = epi_warps * 4096; };
 template <> struct TckCfg<EPI_LSTM> { static constexpr int stages = 4, ring = 0, conv_warps = 6, epi_warps = 8, out_bytes = 0; };
@@ -510,6 +513,11 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             const int64_t row = m0 + q * 32 + lane;
             const bool row_ok = row < M;
             float *crow = ep.C + row * ep.ldc;
+            float *prow = nullptr;   // (EPI_PUSH) this row's home in the cache ring, if it has one
+            if (EPI == EPI_PUSH && row_ok) {
+                const int32_t ps = __ldg(ep.push_slot + row);
+                if (ps >= 0) prow = ep.push_dst + (int64_t)ps * ep.ld_push;
+            }
             float4 side[8], cside[2];
             // previous cell state of the next chunk, fetched one chunk ahead (two 128-bit loads per thread)
             auto load_cell = [&](int c0) {
@@ -609,13 +617,26 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         r[4 * j + 2] = __float_as_uint(__uint_as_float(r[4 * j + 2]) + b4.z);
                         r[4 * j + 3] = __float_as_uint(__uint_as_float(r[4 * j + 3]) + b4.w);
                     }
-                    if (EPI == EPI_PLAIN && ep.mask_out) {
+                    if ((EPI == EPI_PLAIN || EPI == EPI_PUSH) && ep.mask_out) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) bits |= (__uint_as_float(r[j]) > 0.f ? 1u : 0u) << j;
                     }
                     if (ep.relu) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(fmaxf(__uint_as_float(r[j]), 0.f));
+                    }
+                }
+                if (EPI == EPI_PUSH && prow) {   // one full 128-byte line per thread and chunk
+#pragma unroll
+                    for (int j4 = 0; j4 < 32; j4 += 4) {
+                        const int32_t colb = n0 + c0 + j4;
+                        if (colb + 3 < N) {
+                            *reinterpret_cast<uint4 *>(prow + colb) = make_uint4(r[j4], r[j4 + 1], r[j4 + 2], r[j4 + 3]);
+                        } else {
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+                                if (colb + jj < N) prow[colb + jj] = __uint_as_float(r[j4 + jj]);
+                        }
                     }
                 }
                 if (use_tma_store) {
@@ -643,7 +664,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                         }
                     }
                 }
-                if (EPI == EPI_PLAIN && ep.mask_out && row_ok) {
+                if ((EPI == EPI_PLAIN || EPI == EPI_PUSH) && ep.mask_out && row_ok) {
                     const int32_t word = (n0 + c0) >> 5;
                     if (word < ep.mask_words) ep.mask_out[row * ep.mask_words + word] = bits;
                 }
@@ -1061,6 +1082,11 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
         }
         ep.bias = (const float *)home.p;
     }
+    ep.push_dst = eh.push_dst;
+    ep.push_slot = eh.push_slot;
+    ep.ld_push = eh.ld_push;
+    if (eh.push_dst && (eh.lstm_h > 0 || eh.resid_idx || !eh.push_slot || (eh.ld_push & 3) || (((uintptr_t)eh.push_dst) & 15u)))
+        return sat_fail(ctx, SAT_EINVAL, "push epilogue needs a slot map, an aligned destination and the plain epilogue");
     ep.lstm_h = eh.lstm_h;
     ep.lstm_first = eh.lstm_first;
     ep.lstm_c = eh.lstm_c;
@@ -1089,6 +1115,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     L.stage_bytes = stage_bytes;
     if (ep.lstm_h > 0) return ep.addend ? launch_tck<EPI_LSTM_ADD>(ctx, L, ep) : launch_tck<EPI_LSTM>(ctx, L, ep);
     if (ep.resid_idx) return launch_tck<EPI_RESID>(ctx, L, ep);
+    if (ep.push_dst) return launch_tck<EPI_PUSH>(ctx, L, ep);
     return launch_tck<EPI_PLAIN>(ctx, L, ep);
 }
 

@@ -111,6 +111,7 @@ struct sat_ctx {
     int64_t nb = 0;               // sum_m b_m
     int32_t *push_row = nullptr;  // [n_slots] partition-major row index of every boundary node
     int32_t *push_slot = nullptr; // [n_slots]
+    int32_t *row_slot = nullptr;  // [n] cache slot of every partition-major row, -1 for interior nodes (built on first use)
     int64_t *lrowptr = nullptr;   // [n+1] local CSR, rows partition-major
     int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
     int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
@@ -345,6 +346,11 @@ struct TcEpilogueHost {
     const float *addend = nullptr;     // dense [m x ld_addend], added to the accumulators before the LSTM cell (row-aligned)
     int32_t ld_addend = 0;
     int32_t pack_gate_h = 0;           // > 0: the bias is interleaved like weights packed with gate_h (without the LSTM epilogue)
+    // second destination of the rows that have a cache slot (the push of Algorithm 1 fused into the layer transform):
+    // row i also goes to push_dst + push_slot[i] * ld_push when push_slot[i] >= 0
+    float *push_dst = nullptr;
+    const int32_t *push_slot = nullptr;
+    int32_t ld_push = 0;
     // optional home of the padded bias copy (default: a scratch buffer of the context, repacked by every call); with
     // bias_ready the copy in *bias_home is current and is used as it is
     DevBuf *bias_home = nullptr;

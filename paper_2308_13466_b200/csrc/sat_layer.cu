@@ -608,6 +608,12 @@ extern "C" sat_status sat_predict_state(sat_ctx *ctx, int32_t layer, float *S_ho
 // =====================================================================================
 // sat_layer_fwd / sat_layer_bwd
 // =====================================================================================
+__global__ void k_row_slot(const int32_t *__restrict__ perm, const int32_t *__restrict__ slot, int32_t n, int32_t *__restrict__ row_slot)
+{
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < n) row_slot[r] = slot[perm[r]];
+}
+
 extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int32_t d_in, int32_t d_out, const float *h_in,
                                     int32_t ld_in, const float *h_halo, int32_t ld_halo, const float *W, const float *bias, int act,
                                     float *h_out, int32_t ld_out)
@@ -616,7 +622,14 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     PartView v;
     SAT_TRY(sat_part_view(ctx, part, &v));
     if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    const bool push = (act & SAT_FWD_PUSH) != 0;
+    act &= ~SAT_FWD_PUSH;
     if (d_in <= 0 || d_out <= 0 || !W || (act != SAT_ACT_NONE && act != SAT_ACT_RELU)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: bad dims / W / act");
+    CacheLayer *pc = nullptr;
+    if (push) {
+        SAT_TRY(cache_layer(ctx, layer, &pc, "sat_layer_fwd"));
+        if (pc->width != d_out) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: cached layer %d has width %d, not %d", layer, pc->width, d_out);
+    }
     if (v.n_rows > 0 && (!h_in || !h_out || !ok_ld(ld_in, d_in) || !ok_ld(ld_out, d_out) || !aligned16(h_in) || !aligned16(h_out)))
         return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: null / misaligned h_in / h_out or bad leading dimension");
     if (v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo)))
@@ -649,6 +662,17 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
         eh.relu = act == SAT_ACT_RELU;
         eh.mask_out = mask_out;
         eh.mask_words = words;
+        if (push && ctx->n_slots > 0) {   // the boundary rows go to the ring's write buffer from the epilogue
+            if (!ctx->row_slot) {
+                SAT_TRY(dev_realloc(ctx, &ctx->row_slot, (int64_t)ctx->n));
+                k_row_slot<<<(unsigned)cdiv64(ctx->n, 256), 256, 0, ctx->stream>>>(ctx->perm, ctx->slot, ctx->n, ctx->row_slot);
+                SAT_LAUNCHED(ctx);
+            }
+            eh.push_dst = ring_buf(ctx, pc, ctx->write_idx);
+            eh.push_slot = ctx->row_slot + v.row0;
+            eh.ld_push = pc->ld;
+            if (!pc->proj_tag.empty()) pc->proj_tag[ctx->write_idx] = 0;
+        }
         SAT_TRY(sat_gemm_tc(ctx, v.n_rows, d_out, agg, ld_agg, d_in, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
     } else {
         GemmEpilogue ep;
@@ -660,6 +684,8 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     }
     if (part == SAT_ALL_PARTS) L.valid.assign(ctx->M, 1);
     else L.valid[part] = 1;
+    // widths the tensor-core path does not take: the push as its own step
+    if (push && !sat_use_tc(d_out, d_in)) return sat_cache_update(ctx, part, layer, h_out, ld_out);
     return SAT_OK;
 }
 

@@ -92,9 +92,8 @@ class SatEpoch:
             else:
                 B.sat_predict(ctx, l - 1, m, pred[l - 2] if pred is not None else None, reuse_state, hv)  # pull predicted
             h_out = self.rows(self.H[l], m)
-            B.sat_layer_fwd(ctx, m, l, h_in, hv, W[l - 1], b[l - 1], B.SAT_ACT_RELU if l < L else B.SAT_ACT_NONE, h_out)
-            if l < L:
-                B.sat_cache_update(ctx, m, l, h_out)                                    # push
+            # forward; for the cached layers the push of the boundary rows rides on the transform's epilogue
+            B.sat_layer_fwd(ctx, m, l, h_in, hv, W[l - 1], b[l - 1], (B.SAT_ACT_RELU | B.SAT_FWD_PUSH) if l < L else B.SAT_ACT_NONE, h_out)
             h_in = h_out
         kind = B.SAT_LOSS_SOFTMAX_CE if self.loss == "ce" else B.SAT_LOSS_SIGMOID_BCE
         g = self.rows(self.G[L], m)
