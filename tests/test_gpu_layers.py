@@ -307,3 +307,44 @@ def test_parameter_step_on_many_arrays(B):
         assert_close(wd.cpu().numpy(), w0.astype(np.float64) - 0.25 * g0.astype(np.float64), "w - lr g", 1e-6)
     finally:
         B.sat_destroy(ctx)
+
+
+@pytest.mark.parametrize("name,shrink", [("medium", 16), ("odd", 1)])
+def test_push_from_the_layer_transform_equals_the_separate_push(B, name, shrink):
+    """SAT_FWD_PUSH: the ring's write buffer after sat_layer_fwd(..., act | SAT_FWD_PUSH) is bit-identical to the one after
+    sat_layer_fwd + sat_cache_update, all partitions per launch and partition by partition, and h_out is the same."""
+    import torch
+    from paper_2308_13466_b200.epoch import SatEpoch
+    wl = make_workload(name, shrink=shrink)
+    part = wl.part_given if wl.part_given is not None else orc.contig_blocks(wl.n, wl.M)
+    P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+    perm = np.concatenate(P.inner_gid)
+    halo_all = np.concatenate(P.halo_gid)
+    inner_off = np.concatenate([[0], np.cumsum([g.shape[0] for g in P.inner_gid])])
+    halo_off = np.concatenate([[0], np.cumsum([g.shape[0] for g in P.halo_gid])])
+    h_in, h_halo = dev2d(wl.X[perm]), dev2d(wl.X[halo_all])
+    Wd, bd = dev(wl.W[0]), dev(wl.b[0])
+    d_out = wl.dims[1]
+    rings, outs = [], []
+    for mode in ("separate", "fused", "fused-per-partition"):
+        ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss, part_given=wl.part_given)
+        try:
+            h_out = empty2d(wl.n, d_out)
+            if mode == "separate":
+                B.sat_layer_fwd(ep.ctx, B.SAT_ALL_PARTS, 1, h_in, h_halo, Wd, bd, B.SAT_ACT_RELU, h_out)
+                B.sat_cache_update(ep.ctx, B.SAT_ALL_PARTS, 1, h_out)
+            elif mode == "fused":
+                B.sat_layer_fwd(ep.ctx, B.SAT_ALL_PARTS, 1, h_in, h_halo, Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_PUSH, h_out)
+            else:
+                for m in range(P.M):
+                    r0, r1, q0, q1 = inner_off[m], inner_off[m + 1], halo_off[m], halo_off[m + 1]
+                    B.sat_layer_fwd(ep.ctx, m, 1, h_in[r0:r1], h_halo[q0:q1], Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_PUSH, h_out[r0:r1])
+            B.sat_cache_commit(ep.ctx)
+            torch.cuda.synchronize()
+            rings.append(B.sat_cache_read(ep.ctx, 1, 0, P.n_slots, d_out))
+            outs.append(h_out.cpu().numpy().copy())
+        finally:
+            ep.close()
+    assert np.abs(rings[0]).max() > 0
+    for r, o in zip(rings[1:], outs[1:]):
+        assert np.array_equal(r, rings[0]) and np.array_equal(o, outs[0])
