@@ -381,7 +381,8 @@ sat_status sat_dense_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, const 
  * SAT_EINVAL and a message naming the limit — use sat_dense_tn then.  Fewer splits fit for larger m * n, so very tall
  * inputs run slower here than through sat_dense_tn.
  * Set-up: the first call on each device looks up the device address of the array (once per device, kept for the
- * process); make that first call outside any stream capture.
+ * process); make that first call outside any stream capture, and do not reset the device (cudaDeviceReset) afterwards:
+ * the kept address belongs to the device's primary context.
  * Sharing: all calls on a device use the same array.  It keeps whatever the previous call left; nothing has to be
  * cleared because each call overwrites every partial block it later reads.  Two calls that overlap on the GPU (different
  * streams, or concurrent threads) race on the array: serialise them.
@@ -417,8 +418,10 @@ sat_status sat_staleness(sat_ctx *ctx, int32_t part, int32_t d, const float *h_f
  *   sat_codec_plan    sizes: writes row_offsets (DEVICE int64 [rows + 1], exclusive prefix sums of the row sizes) and
  *                     returns the total in *total_bytes (HOST); synchronises the context's stream
  *   sat_codec_encode  writes the bytes (DEVICE uint8, capacity >= the planned total) for the same x / precision
- *   sat_codec_decode  inverse; rows whose bytes do not hold exactly d values raise the device status word
- *                     (sat_sync_status returns SAT_EDATA) and are left partly written
+ *   sat_codec_decode  inverse; `in` holds in_bytes bytes.  Rows whose bytes do not hold exactly d values, and rows whose
+ *                     offsets do not lie inside [0, in_bytes] in ascending order (such a row is skipped: nothing outside
+ *                     the buffer is read), raise the device status word (sat_sync_status returns SAT_EDATA); a row with
+ *                     malformed bytes is left partly written
  *   sat_cache_requantise  stores the committed snapshot `age` (0 = newest) of cached layer `layer` the way a compressed
  *                     ring would hold it: encode + decode in place (context scratch); *bytes (HOST, nullable) = size
  *                     of the encoded snapshot.  Cached input projections of that snapshot are dropped.
@@ -428,7 +431,7 @@ sat_status sat_codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows
                           int64_t *row_offsets, int64_t *total_bytes);
 sat_status sat_codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
                             const int64_t *row_offsets, uint8_t *out, int64_t out_capacity);
-sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d,
+sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, int64_t in_bytes, const int64_t *row_offsets, int64_t rows, int32_t d,
                             int32_t precision, float *x, int32_t ld);
 sat_status sat_cache_requantise(sat_ctx *ctx, int32_t layer, int32_t age, int32_t precision, int64_t *bytes);
 

@@ -379,7 +379,7 @@ def sat_codec_encode(ctx, x, precision: int, row_offsets, out):
 
 def sat_codec_decode(ctx, data, row_offsets, precision: int, x):
     """Decodes rows into x (CUDA fp32 [rows, d]); malformed rows surface as SAT_EDATA from sat_sync_status."""
-    _check(ctx, _lib.sat_codec_decode(ctx, _dev(data), _dev(row_offsets), C.c_int64(x.shape[0]), C.c_int32(x.shape[1]), C.c_int32(precision),
+    _check(ctx, _lib.sat_codec_decode(ctx, _dev(data), C.c_int64(data.numel()), _dev(row_offsets), C.c_int64(x.shape[0]), C.c_int32(x.shape[1]), C.c_int32(precision),
                                       _dev(x), C.c_int32(_ld(x))))
 
 

@@ -28,10 +28,16 @@ def _stale(out: str) -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
+LAST_ACTION = None   # "compiled" or "reused": what the most recent build() call did
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
+    global LAST_ACTION
     out = lib_path()
     if not force and not _stale(out):
+        LAST_ACTION = "reused"
         return out
+    LAST_ACTION = "compiled"
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     objdir = os.path.join(_HERE, "build")
     os.makedirs(objdir, exist_ok=True)

@@ -83,17 +83,22 @@ k_codec_encode(const float *__restrict__ x, int64_t ld, int64_t rows, int32_t d,
 // lanes' delta sums go through one 64-bit warp prefix sum per window, and the element index of a value is the number of
 // terminators before it (one 32-bit prefix sum per window).
 __global__ void __launch_bounds__(256)
-k_codec_decode(const uint8_t *__restrict__ in, const int64_t *__restrict__ offsets, int64_t rows, int32_t d, double scale,
+k_codec_decode(const uint8_t *__restrict__ in, int64_t in_bytes, const int64_t *__restrict__ offsets, int64_t rows, int32_t d, double scale,
                float *__restrict__ x, int64_t ld, int *__restrict__ status)
 {
     const int64_t r = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (r >= rows) return;
     const int64_t b0 = offsets[r], b1 = offsets[r + 1];
+    // an offset pair that does not lie inside the byte buffer is a malformed row: flagged and skipped, never dereferenced
+    if (b0 < 0 || b1 > in_bytes || b1 < b0) {
+        if (lane == 0) atomicOr(status, 2);
+        return;
+    }
     float *row = x + r * ld;
     int64_t q_run = 0;
     int32_t elem_base = 0;
-    bool bad = b1 < b0;
+    bool bad = false;
     for (int64_t pos = b0; pos < b1; pos += 128) {
         const int64_t p0 = pos + 4 * lane;
         uint32_t c[4];
@@ -198,7 +203,7 @@ static sat_status codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t r
 extern "C" sat_status sat_codec_plan(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
                                      int64_t *row_offsets, int64_t *total_bytes)
 {
-    if (!ctx) return SAT_EINVAL;
+    CHECK_CTX(ctx);
     SAT_TRY(codec_check(ctx, "sat_codec_plan", x, ld, rows, d, precision));
     if (!row_offsets || !total_bytes) return sat_fail(ctx, SAT_EINVAL, "sat_codec_plan: null row_offsets / total_bytes");
     return codec_plan(ctx, x, ld, rows, d, precision, row_offsets, total_bytes);
@@ -217,7 +222,7 @@ static sat_status codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t
 extern "C" sat_status sat_codec_encode(sat_ctx *ctx, const float *x, int32_t ld, int64_t rows, int32_t d, int32_t precision,
                                        const int64_t *row_offsets, uint8_t *out, int64_t out_capacity)
 {
-    if (!ctx) return SAT_EINVAL;
+    CHECK_CTX(ctx);
     SAT_TRY(codec_check(ctx, "sat_codec_encode", x, ld, rows, d, precision));
     if (!row_offsets || out_capacity < 0 || (rows > 0 && !out)) return sat_fail(ctx, SAT_EINVAL, "sat_codec_encode: null row_offsets / out");
     int64_t total = 0;
@@ -228,24 +233,24 @@ extern "C" sat_status sat_codec_encode(sat_ctx *ctx, const float *x, int32_t ld,
     return codec_encode(ctx, x, ld, rows, d, precision, row_offsets, out, total);
 }
 
-static sat_status codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d, int32_t precision,
-                               float *x, int32_t ld, double bytes_in)
+static sat_status codec_decode(sat_ctx *ctx, const uint8_t *in, int64_t in_bytes, const int64_t *row_offsets, int64_t rows, int32_t d,
+                               int32_t precision, float *x, int32_t ld)
 {
     if (rows == 0) return SAT_OK;
-    ProfScope prof(ctx, SATK_CODEC, 4.0 * (double)rows * d + 8.0 * (double)rows + bytes_in, 0.0);
-    k_codec_decode<<<(unsigned)cdiv64(rows * 32, 256), 256, 0, ctx->stream>>>(in, row_offsets, rows, d, codec_scale(precision), x, ld,
+    ProfScope prof(ctx, SATK_CODEC, 4.0 * (double)rows * d + 8.0 * (double)rows + (double)in_bytes, 0.0);
+    k_codec_decode<<<(unsigned)cdiv64(rows * 32, 256), 256, 0, ctx->stream>>>(in, in_bytes, row_offsets, rows, d, codec_scale(precision), x, ld,
                                                                              ctx->d_flag + 1);
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
 
-extern "C" sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, const int64_t *row_offsets, int64_t rows, int32_t d,
+extern "C" sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, int64_t in_bytes, const int64_t *row_offsets, int64_t rows, int32_t d,
                                        int32_t precision, float *x, int32_t ld)
 {
-    if (!ctx) return SAT_EINVAL;
+    CHECK_CTX(ctx);
     SAT_TRY(codec_check(ctx, "sat_codec_decode", x, ld, rows, d, precision));
-    if (!row_offsets || (rows > 0 && !in)) return sat_fail(ctx, SAT_EINVAL, "sat_codec_decode: null row_offsets / in");
-    return codec_decode(ctx, in, row_offsets, rows, d, precision, x, ld, 0.0);
+    if (!row_offsets || in_bytes < 0 || (rows > 0 && in_bytes > 0 && !in)) return sat_fail(ctx, SAT_EINVAL, "sat_codec_decode: null row_offsets / in, or negative in_bytes");
+    return codec_decode(ctx, in, in_bytes, row_offsets, rows, d, precision, x, ld);
 }
 
 // encode + decode of one matrix in place through context scratch (what a compressed ring would hand back)
@@ -258,7 +263,7 @@ sat_status sat_codec_roundtrip(sat_ctx *ctx, float *x, int32_t ld, int64_t rows,
     SAT_TRY(sat_ensure(ctx, ctx->buf_codec_bytes, (size_t)(total > 0 ? total : 1)));
     uint8_t *data = (uint8_t *)ctx->buf_codec_bytes.p;
     SAT_TRY(codec_encode(ctx, x, ld, rows, d, precision, offsets, data, total));
-    SAT_TRY(codec_decode(ctx, data, offsets, rows, d, precision, x, ld, (double)total));
+    SAT_TRY(codec_decode(ctx, data, total, offsets, rows, d, precision, x, ld));
     if (bytes) *bytes = total;
     return SAT_OK;
 }

@@ -451,32 +451,68 @@ extern "C" sat_status sat_graph_load(sat_ctx *ctx, int32_t n, int64_t nnz, const
     if (nnz + (int64_t)n >= ((int64_t)1 << 31) * 8) return sat_fail(ctx, SAT_EINVAL, "sat_graph_load: graph too large");
     if (ptr_space != SAT_HOST && ptr_space != SAT_DEVICE) return sat_fail(ctx, SAT_EINVAL, "sat_graph_load: bad ptr_space");
     SAT_CUDA(ctx, cudaSetDevice(ctx->device));
+    // The new graph is copied and validated in buffers of its own; the context's graph, partition, cache and layer state
+    // are replaced only once it has passed, so a rejected graph leaves the context as it was.
+    int64_t *t_rowptr = nullptr;
+    int32_t *t_col = nullptr;
+    float *t_dinv = nullptr;
+    auto drop = [&]() {
+        dev_free(&t_rowptr);
+        dev_free(&t_col);
+        dev_free(&t_dinv);
+    };
+    sat_status rc = dev_alloc(ctx, &t_rowptr, (int64_t)n + 1);
+    if (rc == SAT_OK) rc = dev_alloc(ctx, &t_col, nnz);
+    if (rc == SAT_OK) rc = dev_alloc(ctx, &t_dinv, n);
+    if (rc != SAT_OK) {
+        drop();
+        return rc;
+    }
+    cudaMemcpyKind kind = ptr_space == SAT_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    cudaError_t e = cudaMemcpyAsync(t_rowptr, rowptr, sizeof(int64_t) * ((size_t)n + 1), kind, ctx->stream);
+    if (e == cudaSuccess && nnz) e = cudaMemcpyAsync(t_col, col, sizeof(int32_t) * (size_t)nnz, kind, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), ctx->stream);
+    if (e != cudaSuccess) {
+        drop();
+        return sat_check_cuda(ctx, e, "sat_graph_load: copy of the graph arrays");
+    }
+    int flag = 0;
+    k_check_rowptr<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(t_rowptr, n, nnz, ctx->d_flag);
+    ctx->launches++;
+    rc = read_flag(ctx, &flag);
+    if (rc == SAT_OK && flag) rc = sat_fail(ctx, SAT_EDATA, "sat_graph_load: rowptr is not a monotone offset array ending at nnz");
+    if (rc == SAT_OK) {
+        k_check_cols<<<(unsigned)cdiv64((int64_t)n * 32, 256), 256, 0, ctx->stream>>>(t_rowptr, t_col, n, ctx->d_flag);
+        ctx->launches++;
+        rc = read_flag(ctx, &flag);
+        if (rc == SAT_OK && flag)
+            rc = sat_fail(ctx, SAT_EDATA, "sat_graph_load: malformed graph:%s%s%s%s",
+                          (flag & BAD_COL_RANGE) ? " column out of range;" : "",
+                          (flag & BAD_COL_ORDER) ? " columns unsorted or duplicated;" : "",
+                          (flag & BAD_SELF_LOOP) ? " self-loop stored;" : "", (flag & BAD_ASYM) ? " not symmetric;" : "");
+    }
+    if (rc == SAT_OK) {
+        k_dinv<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(t_rowptr, n, t_dinv);
+        ctx->launches++;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) rc = sat_check_cuda(ctx, e, "kernel launch");
+    }
+    if (rc != SAT_OK) {
+        cudaStreamSynchronize(ctx->stream);
+        drop();
+        return rc;
+    }
+    // accepted: the old graph and everything derived from it go
     ctx->graph_ok = false;
     free_partition(ctx);
     free_cache(ctx);
     free_layers(ctx);
-    SAT_TRY(dev_alloc(ctx, &ctx->rowptr, (int64_t)n + 1));
-    SAT_TRY(dev_alloc(ctx, &ctx->col, nnz));
-    SAT_TRY(dev_alloc(ctx, &ctx->dinv, n));
-    cudaMemcpyKind kind = ptr_space == SAT_HOST ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
-    SAT_CUDA(ctx, cudaMemcpyAsync(ctx->rowptr, rowptr, sizeof(int64_t) * ((size_t)n + 1), kind, ctx->stream));
-    if (nnz) SAT_CUDA(ctx, cudaMemcpyAsync(ctx->col, col, sizeof(int32_t) * (size_t)nnz, kind, ctx->stream));
-    SAT_CUDA(ctx, cudaMemsetAsync(ctx->d_flag, 0, sizeof(int), ctx->stream));
-    k_check_rowptr<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(ctx->rowptr, n, nnz, ctx->d_flag);
-    SAT_LAUNCHED(ctx);
-    int flag = 0;
-    SAT_TRY(read_flag(ctx, &flag));
-    if (flag) return sat_fail(ctx, SAT_EDATA, "sat_graph_load: rowptr is not a monotone offset array ending at nnz");
-    k_check_cols<<<(unsigned)cdiv64((int64_t)n * 32, 256), 256, 0, ctx->stream>>>(ctx->rowptr, ctx->col, n, ctx->d_flag);
-    SAT_LAUNCHED(ctx);
-    SAT_TRY(read_flag(ctx, &flag));
-    if (flag)
-        return sat_fail(ctx, SAT_EDATA, "sat_graph_load: malformed graph:%s%s%s%s",
-                        (flag & BAD_COL_RANGE) ? " column out of range;" : "",
-                        (flag & BAD_COL_ORDER) ? " columns unsorted or duplicated;" : "",
-                        (flag & BAD_SELF_LOOP) ? " self-loop stored;" : "", (flag & BAD_ASYM) ? " not symmetric;" : "");
-    k_dinv<<<(unsigned)cdiv64(n, 256), 256, 0, ctx->stream>>>(ctx->rowptr, n, ctx->dinv);
-    SAT_LAUNCHED(ctx);
+    dev_free(&ctx->rowptr);
+    dev_free(&ctx->col);
+    dev_free(&ctx->dinv);
+    ctx->rowptr = t_rowptr;
+    ctx->col = t_col;
+    ctx->dinv = t_dinv;
     ctx->n = n;
     ctx->nnz = nnz;
     ctx->graph_ok = true;

@@ -400,11 +400,11 @@ template <int NT>
 static sat_status launch_tn_narrow(sat_ctx *ctx, dim3 grid, int64_t rows, int64_t rpb, int32_t m, int32_t n, const float *A, int32_t lda,
                                    const float *B, int32_t ldb, float *part)
 {
-    static bool attr_set = false;
+    static PerDeviceOnce attr_set;
     const size_t smem = 2 * (size_t)(TNN_STAGE * 256 + TNN_STAGE * NT) * sizeof(float);
-    if (!attr_set) {
+    if (attr_set.need(ctx->device)) {
         SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tn_narrow<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_set = true;
+        attr_set.mark(ctx->device);
     }
     k_gemm_tn_narrow<NT><<<grid, 128, smem, ctx->stream>>>(rows, rpb, m, n, A, lda, B, ldb, part);
     SAT_LAUNCHED(ctx);
@@ -482,7 +482,9 @@ extern "C" sat_status sat_dense_tn_static(void *cuda_stream, int64_t rows, int32
     float *scratch = nullptr;
     {
         // one-time set-up per device: `sat_static_scratch` named in host code is only a handle, the kernels need the
-        // address the symbol has on the current device
+        // address the symbol has on the current device.  The address is kept for the life of the process, so the device's
+        // primary context must not be reset (cudaDeviceReset) while this library is in use: the kept address would
+        // then point into a context that no longer exists.
         std::lock_guard<std::mutex> lock(g_static_mutex);
         if (!g_static_ptr[dev]) {
             float *p = nullptr;

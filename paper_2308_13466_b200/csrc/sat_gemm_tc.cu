@@ -1014,7 +1014,7 @@ sat_status sat_tc_weights_layout(int32_t k, int32_t n, const DevBuf &buf, TcWeig
     return SAT_OK;
 }
 
-static bool g_attr_mn = false;
+static PerDeviceOnce g_attr_mn;
 #define TC_SMEM_BUDGET (100 * 1024)
 
 struct TckLaunch {
@@ -1030,13 +1030,13 @@ struct TckLaunch {
 template <int EPI>
 static sat_status launch_tck(sat_ctx *ctx, const TckLaunch &L, const TcEpilogue &ep)
 {
-    static bool attr_set = false;
+    static PerDeviceOnce attr_set;
     const size_t smem = (size_t)TckCfg<EPI>::stages * L.stage_bytes + TckCfg<EPI>::out_bytes + (size_t)TckCfg<EPI>::epi_warps * TckCfg<EPI>::ring * 4096 +
                         sizeof(TcShared) + 1024;
     if (smem > 227 * 1024) return sat_fail(ctx, SAT_EINVAL, "tensor-core GEMM: shared-memory layout of %zu bytes does not fit", smem);
-    if (!attr_set) {
+    if (attr_set.need(ctx->device)) {
         SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_k<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr_set = true;
+        attr_set.mark(ctx->device);
     }
     k_gemm_tc_k<EPI><<<L.grid, TCK_THREADS, smem, ctx->stream>>>(L.mA, L.mA2, L.mB, L.mBlo, L.mC, L.use_tma_store, L.m, L.n, L.nkb1, L.nkb2, L.bn, L.n_tiles_n,
                                                                 L.n_tiles, ep, ctx->d_flag + 1);
@@ -1144,9 +1144,9 @@ sat_status sat_gemm_tc_tn(sat_ctx *ctx, int64_t rows, int32_t m, int32_t n, cons
     CUtensorMap mA, mB;
     SAT_TRY(make_map(ctx, &mA, A, m, rows, lda, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B));
     SAT_TRY(make_map(ctx, &mB, B, n, rows, ldb, 32, TC_BK, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B));
-    if (!g_attr_mn) {
+    if (g_attr_mn.need(ctx->device)) {
         SAT_CUDA(ctx, cudaFuncSetAttribute(k_gemm_tc_mn, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
-        g_attr_mn = true;
+        g_attr_mn.mark(ctx->device);
     }
     dim3 grid((unsigned)cdiv64(m, TC_BM), (unsigned)cdiv64(n, bn), (unsigned)splits);
     k_gemm_tc_mn<<<grid, TC_THREADS, smem, ctx->stream>>>(mA, mB, m, n, rps, bn, stages, tmem_cols_for(bn), part, ctx->d_flag + 1);

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -218,6 +219,17 @@ static inline int32_t ring_index(const sat_ctx *ctx, int32_t age) { return ((ctx
 static inline float *ring_buf(const sat_ctx *ctx, const CacheLayer *c, int32_t idx) { return c->buf + (size_t)idx * ctx->n_slots * c->ld; }
 
 static inline int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// One-time per-device set-up of a kernel (cudaFuncSetAttribute applies to the current device only): a bit per device
+// ordinal; devices beyond 63 simply repeat the (idempotent) set-up on every launch.
+struct PerDeviceOnce {
+    std::atomic<uint64_t> done{0};
+    bool need(int dev) const { return dev < 0 || dev >= 64 || !((done.load(std::memory_order_acquire) >> dev) & 1ull); }
+    void mark(int dev)
+    {
+        if (dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+    }
+};
 static inline int32_t round_up4(int32_t x) { return (x + 3) & ~3; }
 
 // ---- device-side helpers implemented in the .cu files ----

@@ -539,6 +539,8 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
     if (params->h <= 0 || !params->Wx || !params->Uh || !params->b || !params->Wg || !params->bg)
         return sat_fail(ctx, SAT_EINVAL, "sat_predict: incomplete predictor parameters");
     if (params->cell != SAT_CELL_LSTM && params->cell != SAT_CELL_GRU) return sat_fail(ctx, SAT_EINVAL, "sat_predict: unknown recurrent cell %d", params->cell);
+    // the state table S uses ld = h, and its rows must be 16-byte aligned; checked before any state is touched
+    if (params->h & 3) return sat_fail(ctx, SAT_EINVAL, "sat_predict: predictor width h must be a multiple of 4");
     if (reuse_state) {
         if (!c->S_valid || c->S_h != params->h) return sat_fail(ctx, SAT_ESTATE, "sat_predict: no LSTM state table to reuse for layer %d", layer);
     } else {
@@ -550,8 +552,6 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
     SAT_TRY(sat_ensure(ctx, ctx->buf_pred_a, (size_t)v.n_halo * ld_a * sizeof(float)));
     float *a = (float *)ctx->buf_pred_a.p;
     // graph convolution on the LSTM state: a_u = p_uu S_u + sum_{v in N(u) cap V_m} p_uv S_v
-    // (h is a multiple of 4 or the S rows are not 16-byte aligned: the S table uses ld = h, so require h % 4 == 0)
-    if (h & 3) return sat_fail(ctx, SAT_EINVAL, "sat_predict: predictor width h must be a multiple of 4");
     SAT_TRY(sat_spmm_hrow(ctx, v, h, c->S, h, 1, c->S, a - v.halo0 * ld_a, ld_a));
     if (sat_use_tc(d, h)) {
         TcWeights Wg;

@@ -109,6 +109,15 @@ def test_malformed_rows_raise_edata_and_leave_the_context_usable(B, ctx):
     B.sat_codec_decode(ctx, data_g, off_g, 1, wrong_d)    # one value too many per row
     with pytest.raises(B.SatError):
         B.sat_sync_status(ctx)
+    # an offset table that does not match the byte buffer (past its end, negative, descending): the rows are flagged
+    # and skipped, nothing outside the buffer is read
+    for r, val in ((2, total + 4096), (0, -8), (1, total + 1)):
+        off_bad = off_g.clone()
+        off_bad[r] = val
+        B.sat_codec_decode(ctx, data_g, off_bad, 1, back)
+        with pytest.raises(B.SatError) as ei:
+            B.sat_sync_status(ctx)
+        assert ei.value.status == B.SAT_EDATA
     B.sat_codec_decode(ctx, data_g, off_g, 1, back)       # and the context still works
     B.sat_sync_status(ctx)
     assert np.array_equal(back.cpu().numpy(), orc.codec_decode(data_g.cpu().numpy(), off_g.cpu().numpy(), 6, 1))

@@ -146,6 +146,13 @@ def test_malformed_inputs_are_rejected(B):
         expect(B.SAT_ESTATE, lambda: B.sat_layer_bwd(ctx, 0, 1, g, W, W.clone(), None, 0))   # backward before forward
         odd = torch.zeros((3, 5), device="cuda")[:, :4]
         expect(B.SAT_EINVAL, lambda: B.sat_layer_fwd(ctx, 0, 1, odd, odd, W, None, 0, g))    # ld not a multiple of 4
+        # a rejected graph leaves the loaded graph, its partition and the cache as they were
+        before = B.sat_part_lists(ctx, 1)
+        expect(B.SAT_EDATA, lambda: B.sat_graph_load(ctx, rowptr, c2))
+        expect(B.SAT_EDATA, lambda: B.sat_graph_load(ctx, bad, col))
+        after = B.sat_part_lists(ctx, 1)
+        assert all(np.array_equal(before[k], after[k]) for k in before)
+        assert B.sat_cache_state(ctx) == (0, 0)
         B.sat_sync_status(ctx)
     finally:
         B.sat_destroy(ctx)

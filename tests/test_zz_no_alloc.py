@@ -33,10 +33,16 @@ def test_static_scratch_variant_matches_regular_entry_point_twice():
             # and both agree with the plain definition
             ref = (A.double().T @ Bm.double()).cpu().numpy()
             assert_close(got.cpu().numpy(), ref, "static-scratch A^T B vs definition", TOL)
-            # same call again: identical bits (fixed split sizes, fixed summation order)
+            # same call again: identical bits (fixed split sizes, fixed summation order) — and the property in the name: the
+            # device's free memory, as the driver reports it, is the same before and after the call (the first call above
+            # has already loaded the kernels and looked up the array's address; `again` is allocated before the reading)
             again = torch.empty_like(got)
+            torch.cuda.synchronize()
+            free_before = torch.cuda.mem_get_info()[0]
             B.sat_dense_tn_static(stream, A, Bm, again)
             torch.cuda.synchronize()
+            free_after = torch.cuda.mem_get_info()[0]
+            assert free_after == free_before, f"device free memory changed across the call: {free_before} -> {free_after}"
             assert torch.equal(got, again)
         # a shape beyond the built-in scratch is refused with a message, and nothing is launched
         A = torch.zeros(4, 2048, device="cuda")
