@@ -96,3 +96,102 @@ def test_uniform_attention_closed_form():
         f = orc.gat_fwd(P, m, H[inner], H[halo], W, np.zeros_like(a_src), np.zeros_like(a_dst), None, 0)
         want = np.stack([(H[adj[v]] @ W).mean(axis=0) for v in inner])
         np.testing.assert_allclose(f["O"], want, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------------
+# the epoch sequencing around the attention layers (run_epoch_gat): which cached layer feeds which layer, the push, the
+# loss weighting, the hand-down of the gradient
+# ------------------------------------------------------------------------------------------
+def _epoch_case(seed, n, M, dims, p=0.14):
+    rng = np.random.default_rng(seed)
+    rowptr, col = random_graph(rng, n, p)
+    part = rng.integers(0, M, size=n).astype(np.int32)
+    P = orc.build_partition(rowptr, col, part, M)
+    dtil, _ = orc.degrees(rowptr)
+    X = rng.standard_normal((n, dims[0])).astype(np.float32)
+    y = rng.integers(0, dims[-1], size=n).astype(np.int32)
+    params = []
+    for l in range(len(dims) - 1):
+        params.append(dict(W=(rng.standard_normal((dims[l], dims[l + 1])) * 0.6).astype(np.float32),
+                           a_src=(rng.standard_normal(dims[l + 1]) * 0.7).astype(np.float32),
+                           a_dst=(rng.standard_normal(dims[l + 1]) * 0.7).astype(np.float32),
+                           b=(rng.standard_normal(dims[l + 1]) * 0.2).astype(np.float32)))
+    adj = np.eye(n, dtype=bool)
+    for v in range(n):
+        adj[v, col[rowptr[v]:rowptr[v + 1]]] = True
+    return rowptr, col, P, dtil, X, y, params, adj
+
+
+def _dense_model(adj, X, y, params):
+    """The unpartitioned multi-layer attention network in torch (float64) with the mean cross-entropy loss; returns
+    (loss, per-layer outputs, per-layer parameter gradients)."""
+    t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64), requires_grad=True)
+    tp = [{k: t(v) for k, v in p.items()} for p in params]
+    H = torch.tensor(np.asarray(X, dtype=np.float64))
+    outs = []
+    L = len(params)
+    for l, p in enumerate(tp):
+        H = _dense_gat(torch.tensor(adj), H, p["W"], p["a_src"], p["a_dst"], p["b"], 1 if l < L - 1 else 0)
+        outs.append(H)
+    loss = torch.nn.functional.cross_entropy(H, torch.tensor(y, dtype=torch.long), reduction="mean")
+    loss.backward()
+    grads = [{k: v.grad.numpy() for k, v in p.items()} for p in tp]
+    return float(loss.detach()), [o.detach().numpy() for o in outs], grads
+
+
+@pytest.mark.parametrize("seed,dims", [(11, [5, 4, 6, 3]), (12, [4, 7, 3])])
+def test_attention_epoch_on_one_partition_is_the_dense_network(seed, dims):
+    """M = 1: no out-of-subgraph nodes, so the epoch is plain full-graph training — loss and every parameter gradient of
+    every layer equal autograd's on the dense multi-layer model."""
+    rowptr, col, P, dtil, X, y, params, adj = _epoch_case(seed, 26, 1, dims)
+    cache = orc.CacheRing(P.n_slots, dims[1:-1], 2)
+    res = orc.run_epoch_gat(P, dtil, cache, X, y, params, None, "ce")
+    want_loss, outs, grads = _dense_model(adj, X, y, params)
+    assert abs(res["loss"] - want_loss) <= 2e-6 * abs(want_loss)
+    for l in range(len(params)):
+        np.testing.assert_allclose(res["H"][0][l], outs[l], atol=5e-6)
+        for k in ("W", "a_src", "a_dst", "b"):
+            # the oracle rounds the activations it hands from layer to layer to fp32 (as the device path stores them)
+            np.testing.assert_allclose(res["grads"][l][k], grads[l][k], atol=3e-6, err_msg=f"layer {l + 1} G_{k}")
+    assert cache.n_valid == 1
+
+
+@pytest.mark.parametrize("with_predictor", [False, True])
+def test_attention_epoch_with_exact_cache_is_the_full_graph_forward(with_predictor):
+    """M > 1 with the ring holding the exact embeddings of every cached layer (different widths per layer, so a wrong
+    layer index cannot go unnoticed): every layer's output equals the dense full-graph network; the last layer's
+    parameter gradients too (its inputs are exact and nothing below it is differentiated through the halo); what the
+    epoch pushed is again the exact embedding of the boundary nodes.  With a predictor whose output weights are zero
+    the prediction is the newest snapshot, so the same holds through the LSTM / graph-convolution path."""
+    dims = [5, 4, 6, 3]
+    rowptr, col, P, dtil, X, y, params, adj = _epoch_case(21, 30, 3, dims)
+    want_loss, outs, grads = _dense_model(adj, X, y, params)
+    Cn = np.nonzero(P.slot >= 0)[0]
+    cache = orc.CacheRing(P.n_slots, dims[1:-1], 3)
+    for l in range(1, len(dims) - 1):
+        cache.push(l, P.slot[Cn], outs[l - 1][Cn].astype(np.float32))
+    cache.commit()
+    pred = None
+    if with_predictor:
+        rng = np.random.default_rng(5)
+        pred = []
+        for l in range(1, len(dims) - 1):
+            d, h = dims[l], 4
+            pred.append(dict(Wx=rng.standard_normal((d, 4 * h)).astype(np.float32), Uh=rng.standard_normal((h, 4 * h)).astype(np.float32),
+                             b=rng.standard_normal(4 * h).astype(np.float32), Wg=np.zeros((h, d), dtype=np.float32),
+                             bg=np.zeros(d, dtype=np.float32)))
+    res = orc.run_epoch_gat(P, dtil, cache, X, y, params, pred, "ce")
+    L = len(params)
+    for l in range(L):
+        got = np.zeros_like(outs[l])
+        for m in range(P.M):
+            got[P.inner_gid[m]] = res["H"][m][l]
+        np.testing.assert_allclose(got, outs[l], atol=1e-5, err_msg=f"H^{l + 1}")
+    assert abs(res["loss"] - want_loss) <= 1e-5 * abs(want_loss)
+    for k in ("W", "a_src", "a_dst", "b"):
+        np.testing.assert_allclose(res["grads"][L - 1][k], grads[L - 1][k], atol=1e-5, err_msg=f"last layer G_{k}")
+    # the lower layers' gradients miss the paths through the halo copies, so they differ from the full graph's
+    assert np.max(np.abs(res["grads"][0]["W"] - grads[0]["W"])) > 1e-4
+    for l in range(1, L):
+        np.testing.assert_allclose(cache.newest(l)[P.slot[Cn]], outs[l - 1][Cn], atol=1e-5)
+    assert cache.n_valid == 2

@@ -305,3 +305,60 @@ def test_staleness_norm_closed_forms():
         if halo.shape[0] > 1:
             rolled = np.roll(H[halo], 1, axis=0)
             assert orc.staleness(P, m, H, rolled) > 0.0
+
+
+def test_epoch_restricted_to_some_partitions_equals_the_full_epoch():
+    """run_epoch(parts=...) computes the recurrent state only for the cache slots the selected partitions read; what it
+    returns for them (predicted halo, every layer output, the gradients handed down, the state rows) must be the
+    bits of the unrestricted epoch, and it must not commit the ring."""
+    rng = np.random.default_rng(31)
+    n, M, dims, tau, h = 60, 4, [6, 5, 7, 3], 3, 4
+    rowptr, col = random_graph(rng, n, 0.1)
+    dtil, _ = orc.degrees(rowptr)
+    part = rng.integers(0, M, size=n).astype(np.int32)
+    P = orc.build_partition(rowptr, col, part, M)
+    X = rng.standard_normal((n, dims[0])).astype(np.float32)
+    y = rng.integers(0, dims[-1], size=n).astype(np.int32)
+    W = [rng.standard_normal((dims[i], dims[i + 1])).astype(np.float32) * 0.5 for i in range(3)]
+    b = [rng.standard_normal(dims[i + 1]).astype(np.float32) * 0.1 for i in range(3)]
+    pred = []
+    for l in (1, 2):
+        d = dims[l]
+        pred.append(dict(Wx=rng.standard_normal((d, 4 * h)).astype(np.float32) * 0.4, Uh=rng.standard_normal((h, 4 * h)).astype(np.float32) * 0.4,
+                         b=rng.standard_normal(4 * h).astype(np.float32) * 0.1, Wg=rng.standard_normal((h, d)).astype(np.float32) * 0.4,
+                         bg=rng.standard_normal(d).astype(np.float32) * 0.1))
+
+    def filled_ring():
+        r = np.random.default_rng(77)
+        c = orc.CacheRing(P.n_slots, dims[1:-1], tau)
+        for _ in range(2):
+            for l in (1, 2):
+                c.push(l, np.arange(P.n_slots), r.standard_normal((P.n_slots, dims[l])).astype(np.float32))
+            c.commit()
+        return c
+
+    full = orc.run_epoch(P, dtil, filled_ring(), X, y, W, b, pred, "ce")
+    sel = [2, 0]
+    ring = filled_ring()
+    some = orc.run_epoch(P, dtil, ring, X, y, W, b, pred, "ce", parts=sel)
+    assert ring.n_valid == 2 and ring.write_idx == 2          # not committed
+    assert some.S_slots is not None and some.S_slots.shape[0] < P.n_slots
+    for l in range(2):
+        assert np.array_equal(some.S[l][some.S_slots], full.S[l][some.S_slots])
+    for m in range(M):
+        if m not in sel:
+            assert some.per_part[m] is None
+            continue
+        for key in ("H", "halo", "Z", "AGG"):
+            for got, want in zip(some.per_part[m][key], full.per_part[m][key]):
+                assert np.array_equal(got, want), (m, key)
+        for got, want in zip(some.per_part[m]["G_in"][1:], full.per_part[m]["G_in"][1:]):
+            assert np.array_equal(got, want)
+    # the gradients it returns are the sum over the selected partitions only
+    only = [np.zeros_like(g) for g in full.G_W]
+    for m in sel:
+        one = orc.run_epoch(P, dtil, filled_ring(), X, y, W, b, pred, "ce", parts=[m])
+        for l in range(3):
+            only[l] += one.G_W[l]
+    for l in range(3):
+        np.testing.assert_allclose(some.G_W[l], only[l], rtol=1e-12, atol=1e-15)
