@@ -312,6 +312,12 @@ sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g
                        const float *a_src, const float *a_dst, float *g_W, float *g_a_src, float *g_a_dst, float *g_b,
                        int accumulate, float *g_in, int32_t ld_gin);
 
+/* The attention scores sat_gat_fwd kept for layer `layer` (all partitions must have run), copied to HOST memory (any pointer may
+ * be NULL): s_src of the inner rows (a_src . z_u, fp32 [n], partition-major rows), s_dst (a_dst . z_v, fp32 [n]) and s_src of
+ * the halo positions (fp32 [sum_m b_m]).  The logit of entry (v, u) before the LeakyReLU is the fp32 sum s_dst[v] + s_src[u],
+ * which is what decides its slope in sat_gat_bwd.  For tests and diagnostics (the paper has no counterpart).  Synchronises. */
+sat_status sat_gat_scores(sat_ctx *ctx, int32_t layer, float *s_src_inner_host, float *s_dst_host, float *s_src_halo_host);
+
 /* Gradient-side history of layer `layer` >= 2 (see SAT_BWD_GRAD_HISTORY), for checkpoints and tests.
  * sat_grad_history_read: copies the committed history (which = 0; SAT_ESTATE before the first commit) or the running
  * epoch's (which = 1) to HOST memory, dense [|C| x d_out].

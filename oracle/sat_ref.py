@@ -637,9 +637,11 @@ def gat_fwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, bias, act: i
     return dict(Z=Z, alpha=alpha, pre=pre, O=O, H=H.astype(np.float32))
 
 
-def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, act: int, mask=None):
+def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, act: int, mask=None, positive=None):
     """Gradients of sum(G_out * h') for the layer above; the out-of-subgraph embeddings are constants of the epoch, the
-    weights act on them as on the inner rows.  Returns dict(W, a_src, a_dst, b, H_in) in float64."""
+    weights act on them as on the inner rows.  Returns dict(W, a_src, a_dst, b, H_in) in float64.
+    `positive` (bool per entry of the local rows), when given, replaces [pre > 0] as the LeakyReLU's slope decision:
+    where a logit is zero up to rounding either slope is a correct result (as `mask` does for the ReLU)."""
     Hc = np.concatenate([np.asarray(H_in, dtype=np.float64), np.asarray(H_halo, dtype=np.float64).reshape(-1, np.asarray(H_in).shape[1])])
     W = np.asarray(W, dtype=np.float64)
     a_src, a_dst = np.asarray(a_src, dtype=np.float64), np.asarray(a_dst, dtype=np.float64)
@@ -652,7 +654,8 @@ def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, 
     d_alpha = np.sum(D[rows] * Z[cols], axis=1)                       # dL / d alpha_vu
     t = np.zeros(n_in)
     np.add.at(t, rows, alpha * d_alpha)
-    d_pre = alpha * (d_alpha - t[rows]) * np.where(pre > 0, 1.0, GAT_SLOPE)   # through softmax and LeakyReLU
+    pos = (pre > 0) if positive is None else np.asarray(positive, dtype=bool)
+    d_pre = alpha * (d_alpha - t[rows]) * np.where(pos, 1.0, GAT_SLOPE)        # through softmax and LeakyReLU
     ds_dst = np.zeros(n_in)
     np.add.at(ds_dst, rows, d_pre)
     ds_src = np.zeros(Z.shape[0])
@@ -664,13 +667,15 @@ def gat_bwd(P: Partitioning, m: int, H_in, H_halo, W, a_src, a_dst, fwd, G_out, 
     return dict(W=Hc.T @ dZ, a_src=Z.T @ ds_src, a_dst=Z[:n_in].T @ ds_dst, b=D.sum(axis=0), H_in=dZ[:n_in] @ W.T)
 
 
-def run_epoch_gat(P: Partitioning, dtil, cache: CacheRing, X, labels, params, pred, loss_kind: str, masks=None):
+def run_epoch_gat(P: Partitioning, dtil, cache: CacheRing, X, labels, params, pred, loss_kind: str, masks=None, positive=None):
     """One SAT epoch with graph-attention layers in place of the GCN layers (Algorithm 1 unchanged around them): for every
     partition and layer pull (features for layer 1, predicted / historical embeddings of the cached layer otherwise),
     gat_fwd, push; loss; gat_bwd down the layers with the pulled embeddings held constant; commit.
     params: per layer dict(W, a_src, a_dst, b).  Returns dict(loss, grads=[per layer dict(W, a_src, a_dst, b)], H=[per
-    partition [H^(1..L)]], O=[per partition [pre-activation outputs]], logit_margin=[per layer: the smallest |attention
-    logit before the LeakyReLU| relative to their rms: where it is at rounding level the slope of that logit is a tie])."""
+    partition [H^(1..L)]], O=[per partition [pre-activation outputs]], pre=[per partition [per layer: the attention logits
+    before the LeakyReLU, one per entry of the local rows]], logit_margin=[per layer: the smallest |logit| relative to
+    their rms: where it is at rounding level the slope of that logit is a tie]).  masks[m][l-1] / positive[m][l-1] replace
+    the ReLU / LeakyReLU sign decisions of partition m, layer l in the backward pass."""
     L = len(params)
     n = P.n
     S = []
@@ -684,7 +689,7 @@ def run_epoch_gat(P: Partitioning, dtil, cache: CacheRing, X, labels, params, pr
             S.append(state(cache.snapshots(l), d, h, pr["Wx"], pr["Uh"], pr["b"], P.n_slots))
     grads = [dict(W=np.zeros(p["W"].shape), a_src=np.zeros(p["a_src"].shape), a_dst=np.zeros(p["a_dst"].shape), b=np.zeros(p["b"].shape))
              for p in params]
-    total, Hs, Os = 0.0, [None] * P.M, [None] * P.M
+    total, Hs, Os, Pres = 0.0, [None] * P.M, [None] * P.M, [None] * P.M
     margin = [np.inf] * L        # per layer: smallest |pre-activation of an attention logit| relative to their rms
     for m in range(P.M):
         inner, halo = P.inner_gid[m], P.halo_gid[m]
@@ -717,11 +722,16 @@ def run_epoch_gat(P: Partitioning, dtil, cache: CacheRing, X, labels, params, pr
             mk = None
             if masks is not None and masks[m] is not None and l < L and masks[m][l - 1] is not None:
                 mk = masks[m][l - 1]
-            g = gat_bwd(P, m, ins[l - 1], halos[l - 1], _f32(p["W"]), _f32(p["a_src"]), _f32(p["a_dst"]), fws[l - 1], G, 1 if l < L else 0, mask=mk)
+            ps = None
+            if positive is not None and positive[m] is not None and positive[m][l - 1] is not None:
+                ps = positive[m][l - 1]
+            g = gat_bwd(P, m, ins[l - 1], halos[l - 1], _f32(p["W"]), _f32(p["a_src"]), _f32(p["a_dst"]), fws[l - 1], G, 1 if l < L else 0, mask=mk,
+                        positive=ps)
             for k in ("W", "a_src", "a_dst", "b"):
                 grads[l - 1][k] += g[k]
             G = g["H_in"].astype(np.float32)
         Hs[m] = [f["H"] for f in fws]
         Os[m] = [f["O"] for f in fws]
+        Pres[m] = [f["pre"] for f in fws]
     cache.commit()
-    return dict(loss=total, grads=grads, H=Hs, O=Os, logit_margin=margin)
+    return dict(loss=total, grads=grads, H=Hs, O=Os, pre=Pres, logit_margin=margin)

@@ -63,7 +63,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step", "sat_sgd_steps",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores",
 ]
 
 
@@ -354,6 +354,16 @@ def sat_gat_bwd(ctx, part: int, layer: int, g_out, h_out, h_in, h_halo, W, a_src
                                  C.c_int32(_ld(h_halo) if h_halo is not None and h_halo.shape[0] else d_in + (-d_in) % 4), C.c_int32(d_in),
                                  _dev(W), _dev(a_src), _dev(a_dst), _dev(g_W), _dev(g_a_src), _dev(g_a_dst), _dev(g_b), C.c_int(accumulate),
                                  _dev(g_in), C.c_int32(_ld(g_in) if g_in is not None else 0)))
+
+
+def sat_gat_scores(ctx, layer: int, n: int, nb: int):
+    """(s_src of the inner rows [n], s_dst [n], s_src of the halo positions [nb]) kept by sat_gat_fwd for `layer`."""
+    s_in = np.empty(n, dtype=np.float32)
+    s_dst = np.empty(n, dtype=np.float32)
+    s_halo = np.empty(max(nb, 1), dtype=np.float32)
+    _check(ctx, _lib.sat_gat_scores(ctx, C.c_int32(layer), s_in.ctypes.data_as(C.c_void_p), s_dst.ctypes.data_as(C.c_void_p),
+                                    s_halo.ctypes.data_as(C.c_void_p)))
+    return s_in, s_dst, s_halo[:nb]
 
 
 def sat_staleness(ctx, part: int, h_fresh, h_used_halo, sq_sum):

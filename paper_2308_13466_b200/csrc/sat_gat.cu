@@ -702,6 +702,24 @@ extern "C" sat_status sat_gat_fwd(sat_ctx *ctx, int32_t part, int32_t layer, int
     return SAT_OK;
 }
 
+// the attention scores kept by the forward call, for checkpoints and tests
+extern "C" sat_status sat_gat_scores(sat_ctx *ctx, int32_t layer, float *s_src_inner_host, float *s_dst_host, float *s_src_halo_host)
+{
+    CHECK_CTX(ctx);
+    if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_gat_scores: layer must be in [1, %d]", SAT_MAX_LAYERS);
+    GatState &G = ctx->gat[layer];
+    if (G.d_out <= 0 || G.valid.size() != (size_t)ctx->M) return sat_fail(ctx, SAT_ESTATE, "sat_gat_scores: sat_gat_fwd has not run for layer %d", layer);
+    for (int m = 0; m < ctx->M; ++m)
+        if (!G.valid[m]) return sat_fail(ctx, SAT_ESTATE, "sat_gat_scores: sat_gat_fwd has not run for partition %d of layer %d", m, layer);
+    const int64_t n = ctx->n, nb = ctx->nb;
+    const float *s_in = (const float *)G.scal.p, *s_dst = s_in + n, *s_halo = s_dst + 2 * n;
+    if (s_src_inner_host) SAT_CUDA(ctx, cudaMemcpyAsync(s_src_inner_host, s_in, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    if (s_dst_host) SAT_CUDA(ctx, cudaMemcpyAsync(s_dst_host, s_dst, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    if (s_src_halo_host && nb > 0) SAT_CUDA(ctx, cudaMemcpyAsync(s_src_halo_host, s_halo, (size_t)nb * sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
 extern "C" sat_status sat_gat_bwd(sat_ctx *ctx, int32_t part, int32_t layer, const float *g_out, int32_t ld_g, const float *h_out, int32_t ld_out,
                                   const float *h_in, int32_t ld_in, const float *h_halo, int32_t ld_halo, int32_t d_in, const float *W,
                                   const float *a_src, const float *a_dst, float *g_W, float *g_a_src, float *g_a_dst, float *g_b,

@@ -44,3 +44,29 @@ def glorot_uniform(seed: int, fan_in: int, fan_out: int, tag: str) -> np.ndarray
     a = np.sqrt(6.0 / (fan_in + fan_out))
     rng = stream_rng(seed, tag)
     return ((rng.random((fan_in, fan_out)) * 2.0 - 1.0) * a).astype(np.float32)
+
+
+# ------------------------------------------------------------------------------------------
+# Embedding-like rows that are a function of (seed, tag, row id): any subset of the rows of a very large matrix can be
+# produced without producing the matrix (full-size parity tests hand the whole matrix to one side and sampled rows to the
+# other).  Rows are picked from a seeded table of non-negative values (what ReLU outputs look like), so this is pure
+# indexing: no arithmetic of the method.
+# ------------------------------------------------------------------------------------------
+_TABLE_ROWS = 8191
+
+
+def embedding_table(seed: int, d: int, tag: str = "embedding-table", signed: bool = False) -> np.ndarray:
+    """[8191, d] fp32: |N(0, 1)| / 2 with about a third of the entries set to zero (signed=True: N(0, 1) / 2, dense)."""
+    rng = stream_rng(seed, f"{tag}:{d}:{int(signed)}")
+    t = rng.standard_normal((_TABLE_ROWS, d), dtype=np.float32) * np.float32(0.5)
+    if signed:
+        return t
+    t = np.abs(t)
+    t[rng.random((_TABLE_ROWS, d), dtype=np.float32) < np.float32(0.33)] = 0.0
+    return t
+
+
+def table_rows(table: np.ndarray, ids, salt: int = 0) -> np.ndarray:
+    """Rows of the virtual matrix M[i] = table[(i * 7919 + salt * 104729) mod 8191] for the given row ids i."""
+    ids = np.asarray(ids, dtype=np.int64)
+    return table[(ids * 7919 + int(salt) * 104729) % _TABLE_ROWS]

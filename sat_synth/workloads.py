@@ -112,6 +112,8 @@ def make_workload(name: str, seed: int = 0, shrink: int = 1, with_dense: bool = 
             kw["n_samples"] = cfg["n_samples"] // shrink
         else:
             kw["n_unique_undirected"] = cfg["n_unique"] // shrink
+        if "attach_isolated" in cfg:          # False keeps the nodes R-MAT leaves without an edge (degenerate-case tests)
+            kw["attach_isolated"] = bool(cfg["attach_isolated"])
         rowptr, col = rmat_graph(seed, scale, n, **kw)
         rowptr, col, _ = bfs_relabel(rowptr, col)
     dims = list(cfg["dims"])

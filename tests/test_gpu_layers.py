@@ -283,6 +283,83 @@ def test_shrunk_workloads_every_call(B, name, shrink, parts):
         case.close()
 
 
+def test_isolated_inner_nodes_every_call(B):
+    """Nodes without any edge (row of P = the self-loop alone, p_vv = 1): the generator normally gives every such node an
+    edge; here it does not, and a random assignment spreads the ~1,800 isolated nodes of the graph over all partitions.
+    Every call of the layer step against the oracle, as for the other workloads."""
+    wl = make_workload("odd", attach_isolated=False)
+    deg = np.diff(wl.rowptr)
+    assert int((deg == 0).sum()) > 1000
+    wl.part_given = np.random.default_rng(3).integers(0, wl.M, size=wl.n).astype(np.int32)
+    for m in range(wl.M):
+        assert int(((deg == 0) & (wl.part_given == m)).sum()) > 100
+    case = Case(B, wl, 2)
+    try:
+        worst = _check_calls(B, case, list(range(wl.M)))
+        print("isolated", {k: f"{v:.2e}" for k, v in worst.items()})
+        # an isolated node's layer-1 output is its own feature row through the transform: AGG_v = x_v
+        m = 0
+        inner = case.P.inner_gid[m]
+        iso = np.nonzero(deg[inner] == 0)[0][:64]
+        h_out = empty2d(inner.shape[0], wl.dims[1])
+        B.sat_layer_fwd(case.ctx, m, 1, dev2d(wl.X[inner]), dev2d(wl.X[case.P.halo_gid[m]]), dev(wl.W[0]), dev(wl.b[0]), B.SAT_ACT_NONE, h_out)
+        want = wl.X[inner][iso].astype(np.float64) @ wl.W[0].astype(np.float64) + wl.b[0]
+        assert_close(h_out.cpu().numpy()[iso], want, "isolated rows: x_v W + b")
+    finally:
+        case.close()
+
+
+def test_cache_init_from_a_given_snapshot(B):
+    """SAT_CACHE_COPY: the caller's matrices become the single valid snapshot of every cached layer (ring state (1, 1)),
+    visible to the identity predictor, to the LSTM predictor (one-snapshot window) and to the export; the source is copied,
+    not kept."""
+    import torch
+    wl = make_workload("odd")
+    part = orc.contig_blocks(wl.n, wl.M)
+    dtil, _ = orc.degrees(wl.rowptr)
+    P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+    rng = np.random.default_rng(8)
+    init = [np.abs(rng.standard_normal((P.n_slots, d))).astype(np.float32) for d in wl.dims[1:-1]]
+    cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
+    for l, a in enumerate(init, start=1):
+        cache.push(l, np.arange(P.n_slots), a)
+    cache.commit()
+    ctx = B.sat_create(0, 0)
+    try:
+        B.sat_graph_load(ctx, wl.rowptr, wl.col)
+        B.sat_partition(ctx, wl.M, B.SAT_PART_CONTIG_BLOCKS)
+        init_d = [dev2d(a) for a in init]
+        B.sat_cache_init(ctx, wl.dims[1:-1], wl.tau, B.SAT_CACHE_COPY, init_d)
+        for t in init_d:
+            t.fill_(float("nan"))                      # the library must have copied
+        torch.cuda.synchronize()
+        assert B.sat_cache_state(ctx) == (1, 1)
+        preds = pred_to_device(wl.pred, B)
+        for l in range(1, wl.L):
+            assert np.array_equal(B.sat_cache_read(ctx, l, 0, P.n_slots, wl.dims[l]), init[l - 1])
+            S = orc.lstm_state(cache.snapshots(l), wl.dims[l], wl.pred[l - 1]["Wg"].shape[0], wl.pred[l - 1]["Wx"], wl.pred[l - 1]["Uh"],
+                               wl.pred[l - 1]["b"], P.n_slots)
+            for m in range(wl.M):
+                out = empty2d(P.halo_gid[m].shape[0], wl.dims[l])
+                B.sat_predict(ctx, l, m, None, 0, out)
+                assert np.array_equal(out.cpu().numpy(), init[l - 1][P.halo_slot[m]])
+                B.sat_predict(ctx, l, m, preds[l - 1], 0, out)
+                want = orc.predict_halo(P, m, dtil, S, cache.newest(l), wl.pred[l - 1]["Wg"], wl.pred[l - 1]["bg"])
+                assert_close(out.cpu().numpy(), want, f"prediction from the given snapshot, layer {l} partition {m}")
+        # the rest of the ring is zero and the next commit makes the write buffer the second snapshot
+        ring = B.sat_cache_export(ctx, 1, wl.tau, P.n_slots, wl.dims[1])
+        assert np.array_equal(ring[0], init[0]) and not ring[1:].any()
+        B.sat_cache_commit(ctx)
+        assert B.sat_cache_state(ctx) == (2, 2)
+        # argument errors: a missing matrix
+        with pytest.raises(B.SatError) as ei:
+            B.sat_cache_init(ctx, wl.dims[1:-1], wl.tau, B.SAT_CACHE_COPY, None)
+        assert ei.value.status == B.SAT_EINVAL
+        B.sat_sync_status(ctx)
+    finally:
+        B.sat_destroy(ctx)
+
+
 def test_parameter_step_on_many_arrays(B):
     """sat_sgd_steps on a list of arrays (more than one launch's worth, one of them empty) equals sat_sgd_step array by array."""
     import torch

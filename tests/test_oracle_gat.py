@@ -195,3 +195,31 @@ def test_attention_epoch_with_exact_cache_is_the_full_graph_forward(with_predict
     for l in range(1, L):
         np.testing.assert_allclose(cache.newest(l)[P.slot[Cn]], outs[l - 1][Cn], atol=1e-5)
     assert cache.n_valid == 2
+
+
+def test_slope_override_of_the_backward():
+    """gat_bwd(positive=...) replaces the LeakyReLU's sign decision entry by entry: the oracle's own decision gives the
+    same bits, and flipping one entry changes the logit's gradient by exactly the ratio of the two slopes."""
+    rowptr, col, P, H, W, a_src, a_dst, bias, G, adj = _case(13, M=2)
+    m = 0
+    inner, halo = P.inner_gid[m], P.halo_gid[m]
+    f = orc.gat_fwd(P, m, H[inner], H[halo], W, a_src, a_dst, bias, 1)
+    g0 = orc.gat_bwd(P, m, H[inner], H[halo], W, a_src, a_dst, f, G[inner], 1)
+    g1 = orc.gat_bwd(P, m, H[inner], H[halo], W, a_src, a_dst, f, G[inner], 1, positive=f["pre"] > 0)
+    for k in g0:
+        assert np.array_equal(g0[k], g1[k])
+    pos = f["pre"] > 0
+    e = int(np.argmax(np.abs(f["pre"])))       # one entry, decided the other way
+    flipped = pos.copy()
+    flipped[e] = ~flipped[e]
+    g2 = orc.gat_bwd(P, m, H[inner], H[halo], W, a_src, a_dst, f, G[inner], 1, positive=flipped)
+    # only the path through that logit changes: G_a_dst changes by (new slope - old slope) * alpha (d_alpha - t) * z_v
+    rows, cols = orc._gat_rows(P, m)
+    Z, alpha = f["Z"], f["alpha"]
+    D = G[inner] * (f["O"] > 0)
+    d_alpha = np.sum(D[rows] * Z[cols], axis=1)
+    t = np.zeros(inner.shape[0])
+    np.add.at(t, rows, alpha * d_alpha)
+    base = alpha[e] * (d_alpha[e] - t[rows[e]])
+    delta = ((1.0 if flipped[e] else orc.GAT_SLOPE) - (1.0 if pos[e] else orc.GAT_SLOPE)) * base
+    np.testing.assert_allclose(g2["a_dst"] - g0["a_dst"], delta * Z[rows[e]], atol=1e-12)
