@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the SAT epoch step on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload medium]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload large]
 
 A step is one steady-state SAT epoch over all partitions of the workload: layer-1 halo
 pull, predictor (LSTM over the cached snapshots + graph convolution + skip) for every
@@ -9,11 +9,14 @@ cached layer, every layer forward (SpMM + transform), cache push, loss seed, eve
 backward, ring commit and the SGD step.  metric = edges/s = nnz(A + I) / epoch time.
 Prints ONE JSON line on rank 0.
 
+The default workload is the largest of the five configurations that fits one GPU
+("large": 2.45 M nodes, 128 M entries of A + I, 32 partitions); the others are selectable.
 --impl reference times the CPU oracle (as it stands) on the host cores instead, on a
 bounded sample of the same workload per step.
-With N > 1 (torchrun, one rank per GPU) every rank runs an independent replica of the
-workload (the path of this build does not shard across GPUs; there is no collective on
-the data path); the value is the aggregate over ranks, timed as the max over ranks.
+With N > 1 every rank runs an independent replica of the workload (the path of this build
+does not shard across GPUs; there is no collective on the data path); the value is the
+aggregate over ranks, timed as the max over ranks.  Started as plain `python bench.py
+--gpus N` it launches the N ranks itself (torch.distributed.run on 127.0.0.1).
 """
 from __future__ import annotations
 
@@ -31,18 +34,25 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel on the benchmark
-# workload, from the committed ncu summary under profiles/ (None until a capture exists for the family).
-# gemm_nn: 302 MB = the 256-wide layer transform; gemm_side: 304 MB = the LSTM recurrence step (profiles/k_gemm_tc_k_medium.md);
-# spmm_fwd: 684 MB = the d = 256 launch (profiles/k_spmm_items_medium.md).
-NCU_TRAFFIC_BYTES = {"gemm_nn": 301.8e6, "spmm_fwd": 757.9e6, "gemm_side": 304.4e6}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel comes from the committed ncu
+# summaries under profiles/: a line of the form
+#     traffic_bytes_per_launch[<workload>/<family>] = <bytes>
+# in any profiles/*.md is picked up; no such line for the workload that runs means "traffic": null in the JSON line.
+def ncu_traffic(workload: str, family: str):
+    import glob
+    import re
+    pat = re.compile(r"traffic_bytes_per_launch\[" + re.escape(workload) + "/" + re.escape(family) + r"\]\s*=\s*([0-9.eE+]+)")
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "*.md"))):
+        with open(path) as f:
+            m = pat.search(f.read())
+        if m:
+            return float(m.group(1)), os.path.basename(path)
+    return None, None
+
 
 # predictor update period Delta-T of Algorithm 1 followed by the run (epochs between two parameter-version bumps)
 PRED_PERIOD = 10
 PRED_LR = 0.01
-
-# L2 -> SM streaming rate measured on this box with a TMA-only kernel (operand tiles resident in L2), in GB/s
-L2_STREAM_GBS = 9700.0
 
 # The contractions run on the tensor cores in TF32 (two-term split: three TF32 MMAs per product term).  The box's
 # measured tensor peak is a bf16 figure; TF32 is taken as measured bf16 x the nominal ratio 1.1 / 2.25 PFLOP/s.
@@ -112,49 +122,74 @@ class ClockSampler:
 # ------------------------------------------------------------------------------------------
 # CPU oracle leg (cpu_baseline of the default run, and the whole of --impl reference)
 # ------------------------------------------------------------------------------------------
-class OracleSample:
-    """The oracle on a bounded sample of the workload: `k` partitions per step (all their layers, forward and
-    backward, plus the LSTM for the cached nodes they read), from a full ring (tau snapshots of synthetic
-    non-negative embeddings — the work does not depend on the values)."""
+# one step of the CPU legs handles at most this many entries of A + I (a whole partition of the smaller workloads)
+ORACLE_SAMPLE_ENTRIES = 1_200_000
 
-    def __init__(self, wl):
+
+class OracleSample:
+    """The oracle on a bounded sample of the workload.  The unit of a sample is a `block`: a whole partition when a
+    partition has at most ORACLE_SAMPLE_ENTRIES entries of A + I; otherwise every partition's contiguous id range is cut
+    into `cut` equal ranges and the oracle runs one of them as a partition of that finer contiguous partitioning (all layers
+    forward and backward plus the LSTM for the cached nodes the block reads: its out-of-block neighbours are its halo).
+    The ring is full: tau snapshots of seeded non-negative embeddings, materialised only for the cache slots the
+    sampled blocks read — the work does not depend on the values."""
+
+    def __init__(self, wl, n_blocks: int):
         from oracle import sat_ref as orc
+        from sat_synth import embedding_table, table_rows
         self.orc, self.wl = orc, wl
-        part = wl.part_given if wl.part_given is not None else orc.contig_blocks(wl.n, wl.M)
+        per_part = wl.nnz / wl.M
+        self.cut = 1 if wl.part_given is not None else max(1, int(np.ceil(per_part / ORACLE_SAMPLE_ENTRIES)))
+        self.M = wl.M * self.cut
+        part = wl.part_given if wl.part_given is not None else orc.contig_blocks(wl.n, self.M)
+        # the sampled blocks: evenly spread over the id range
+        n_blocks = min(n_blocks, self.M)
+        self.blocks = [int(i * self.M // n_blocks) for i in range(n_blocks)]
         self.dtil, _ = orc.degrees(wl.rowptr)
-        self.P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
-        self.cache = orc.CacheRing(self.P.n_slots, wl.dims[1:-1], wl.tau)
-        rng = np.random.default_rng(0)
-        for buf in self.cache.buf:
-            buf[:] = np.abs(rng.standard_normal(buf.shape, dtype=np.float32))
+        self.P = orc.build_partition(wl.rowptr, wl.col, part, self.M, only_parts=self.blocks)
+        self.cache = orc.CacheRing(self.P.n_slots, wl.dims[1:-1], wl.tau)     # zero pages: nothing is touched yet
+        need = [self.P.halo_slot[m] for m in self.blocks] + [self.P.slot[self.P.inner_gid[m][self.P.hrow_col[m]]] for m in self.blocks]
+        slots = np.unique(np.concatenate(need)) if need else np.empty(0, dtype=np.int64)
+        for li, buf in enumerate(self.cache.buf):
+            table = embedding_table(wl.seed, wl.dims[1 + li])
+            for s in range(buf.shape[0]):
+                buf[s][slots] = table_rows(table, slots, 1 + s + 100 * li)
         self.cache.n_valid = wl.tau
         self.cores = orc.num_threads()
 
-    def run(self, parts):
+    def describe(self) -> str:
+        wl = self.wl
+        unit = (f"1 of {wl.M} partitions" if self.cut == 1 else
+                f"1 of {self.M} contiguous id blocks (each of the {wl.M} partitions cut into {self.cut}; the block runs as a partition of that "
+                f"finer partitioning, its out-of-block neighbours being its halo)")
+        return (f"{unit} of the {wl.name} workload, all layers fwd+bwd+predictor incl. the LSTM for the cached nodes the block reads; "
+                f"ring full (tau={wl.tau})")
+
+    def run(self, blocks):
         wl = self.wl
         t0 = time.perf_counter()
-        self.orc.run_epoch(self.P, self.dtil, self.cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=True, parts=parts)
+        self.orc.run_epoch(self.P, self.dtil, self.cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss, keep=True, parts=blocks)
         dt = time.perf_counter() - t0
-        edges = sum(int(self.P.loc_rowptr[m][-1]) for m in parts)
+        edges = sum(int(self.P.loc_rowptr[m][-1]) for m in blocks)
         return edges, dt
 
 
 def run_reference(args, wl):
-    """--impl reference: the oracle, one partition per step (rotating), W warm-up steps then K timed steps."""
+    """--impl reference: the oracle, one block per step (rotating over the sampled blocks), W warm-up steps then K timed steps."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    smp = OracleSample(wl)
+    smp = OracleSample(wl, args.warmup + args.steps)
+    nb = len(smp.blocks)
     for i in range(args.warmup):
-        smp.run([i % wl.M])
+        smp.run([smp.blocks[i % nb]])
     edges, secs = 0, 0.0
     for i in range(args.steps):
-        e, t = smp.run([(args.warmup + i) % wl.M])
+        e, t = smp.run([smp.blocks[(args.warmup + i) % nb]])
         edges += e
         secs += t
     value = edges / secs
-    sample = (f"per step: 1 of {wl.M} partitions (rotating) of the {wl.name} workload, all layers fwd+bwd+predictor "
-              f"incl. the LSTM for the cached nodes that partition reads; ring full (tau={wl.tau})")
+    sample = "per step: " + smp.describe()
     line = dict(impl="reference", metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s",
                 n_gpus=0, steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * secs / max(args.steps, 1), higher_is_better=True,
                 scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
@@ -420,7 +455,7 @@ def run_ours(args, wl):
     # ---- epochs with the gradient-side history (stale-gradient term of the Appendix's back-propagation; not part of the
     #      epoch metric) ----
     grad_history = None
-    if rank == 0 and wl.L > 1 and not args.epochs_only:
+    if rank == 0 and wl.L > 1 and args.extras:
         for _ in range(2):
             ep.step(W, b, preds, lr, grad_history=True)
         g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -445,7 +480,7 @@ def run_ours(args, wl):
     # ---- the same workload with graph-attention layers in place of the GCN layers (not part of the epoch metric; a first,
     #      untuned build of that backbone) ----
     gat = None
-    if rank == 0 and wl.L > 1 and not args.epochs_only:
+    if rank == 0 and wl.L > 1 and args.extras:
         grng = np.random.default_rng(5)
         gparams = []
         for l in range(wl.L):
@@ -472,7 +507,7 @@ def run_ours(args, wl):
 
     # ---- embedding codec on a ring snapshot (not part of the epoch metric; run last because it rewrites the snapshot) ----
     codec = None
-    if rank == 0 and wl.L > 1 and not args.epochs_only:
+    if rank == 0 and wl.L > 1 and args.extras:
         prec = 3
         B.sat_cache_requantise(ep.ctx, 1, 1, prec)          # warm-up (scratch allocation)
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -496,36 +531,39 @@ def run_ours(args, wl):
         fam = top_family
         rec = prof_top[fam]     # measured inside the timed region
         per_launch_ms = rec["ms"] / max(rec["calls"], 1)
+        traffic, traffic_src = ncu_traffic(wl.name if args.shrink == 1 else f"{wl.name}/{args.shrink}", fam)
         if fam.startswith("gemm") and fam != "gemm_side":   # gemm_side: K = h contractions with a streamed side operand (HBM-bound)
-            tfl = TF32_MMAS_PER_TERM * rec["flops"] / (rec["ms"] * 1e-3) / 1e12
+            tfl_alg = rec["flops"] / (rec["ms"] * 1e-3) / 1e12
+            tfl = TF32_MMAS_PER_TERM * tfl_alg
             peak = peaks["bf16"] * TF32_OVER_BF16
             roofline = dict(kernel=fam, bound="tensor", achieved=tfl, peak=peak, unit="TFLOP/s", frac=tfl / peak,
-                            traffic=NCU_TRAFFIC_BYTES.get(fam),
-                            achieved_note="TF32 tensor flops issued = 3 x the algorithmic 2mnk (two-term TF32 split)",
+                            achieved_2mnk=tfl_alg, frac_2mnk=tfl_alg / peak,
+                            achieved_note="achieved / frac count the TF32 tensor flops issued = 3 x the method's 2mnk (two-term TF32 split, the "
+                                          "price of the 1e-4 tolerance): the tensor pipe's utilisation; achieved_2mnk / frac_2mnk count the method's own flops",
                             peak_source=f"{peaks['source']} sustained bf16 {peaks['bf16']:.0f} TFLOP/s x nominal TF32/bf16 ratio {TF32_OVER_BF16:.3f}")
         else:
             gbs = rec["bytes"] / (rec["ms"] * 1e-3) / 1e9
             roofline = dict(kernel=fam, bound="hbm", achieved=gbs, peak=peaks["hbm"], unit="GB/s", frac=gbs / peaks["hbm"],
-                            traffic=NCU_TRAFFIC_BYTES.get(fam), peak_source=f"{peaks['source']} HBM copy bandwidth")
-        roofline.update(launches=rec["calls"], ms_per_launch=per_launch_ms, share_of_step=rec["ms"] / ms)
+                            peak_source=f"{peaks['source']} HBM copy bandwidth")
+        roofline.update(traffic=traffic, traffic_source=(f"profiles/{traffic_src}" if traffic_src else
+                                                         "no ncu capture of this kernel on this workload is committed"),
+                        launches=rec["calls"], ms_per_launch=per_launch_ms, share_of_step=rec["ms"] / ms)
         if fam.startswith("spmm") and rec["flops"] > 0:
-            # the SpMM reads every neighbour row once per edge: that stream comes out of L2, not HBM (hit rate 63 % in the ncu
-            # capture), and its rate, not the HBM fraction above, is what bounds the kernel
-            gather = rec["flops"] / 2.0 * 4.0 / (rec["ms"] * 1e-3) / 1e9
-            roofline["l2_gather"] = dict(achieved=gather, unit="GB/s", reference=L2_STREAM_GBS, frac=gather / L2_STREAM_GBS,
-                                         reference_source="L2 -> SM rate of a pure TMA streaming kernel on this box (DESIGN.md section 8)")
+            # the SpMM reads one neighbour row per entry: that stream comes mostly out of L2, not HBM; its rate is reported
+            # beside the HBM figure (no roof is claimed for it)
+            roofline["gather_gbs"] = rec["flops"] / 2.0 * 4.0 / (rec["ms"] * 1e-3) / 1e9
         families = {k: dict(calls=v["calls"], ms_per_step=v["ms"] / args.steps,
                             gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else 0.0,
+                            hbm_frac=(v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm"]) if v["ms"] > 0 else 0.0,
                             tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else 0.0)
                     for k, v in prof.items() if v["calls"]}
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            smp = OracleSample(wl)
-            k = max(1, wl.M // 2)
-            edges, secs = smp.run(list(range(k)))
+            k = 4
+            smp = OracleSample(wl, k)
+            edges, secs = smp.run(list(smp.blocks))
             cpu = dict(value=edges / secs, unit="edges/s", cores=smp.cores, kind="oracle", seconds=secs,
-                       sample=f"partitions 0..{k - 1} of {wl.M} of the {wl.name} workload (all layers fwd+bwd+predictor, "
-                              f"LSTM for the cached nodes they read), ring full; {edges} edges")
+                       sample=f"{len(smp.blocks)} x " + smp.describe() + f"; {edges} edges")
         # whole-epoch view: algorithmic bytes of every kernel family over the epoch time, against the HBM copy rate; the
         # SpMM families also as the gather rate they sustain from L2 (entries x row bytes / time), which is what bounds them
         alg_bytes = sum(v["bytes"] for v in prof.values()) / args.steps
@@ -550,18 +588,38 @@ def run_ours(args, wl):
         dist.destroy_process_group()
 
 
+def launch_ranks(n: int) -> int:
+    """`python bench.py --gpus N` outside a launcher: start the N ranks on this node and hand back their exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="medium")
+    ap.add_argument("--workload", default="large", choices=["tiny", "medium", "dense", "large", "multilabel", "odd"])
     ap.add_argument("--shrink", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--epochs-only", action="store_true",
-                    help="skip the side measurements (predictor never updated / unversioned, predictor update, gradient history, codec)")
+                    help="skip the side measurements (predictor never updated / unversioned, predictor update)")
+    ap.add_argument("--extras", action="store_true",
+                    help="also time the parts outside the epoch metric: gradient-side history, graph-attention backbone, embedding codec")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus > 1 and "RANK" not in os.environ:
+        sys.exit(launch_ranks(args.gpus))
+    if world != args.gpus:
+        ap.error(f"--gpus {args.gpus} but the launcher started {world} rank(s)")
     from sat_synth import make_workload
     if args.impl == "reference" and int(os.environ.get("RANK", "0")) != 0:
         return

@@ -316,7 +316,11 @@ sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float
 {
     if (v.n_halo == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
-    ProfScope prof(ctx, SATK_SPMM_HROW, 0.0, 0.0);
+    // algorithmic bytes: column + weight per entry, row offsets / slot / dinv per halo row, every source row once (the
+    // boundary rows of the selection, plus the halo nodes' own rows for the self term), every output row once
+    const double n_src = (double)v.n_push + (self_src ? (double)v.n_halo : 0.0);
+    ProfScope prof(ctx, SATK_SPMM_HROW, 8.0 * (double)v.hnnz + 12.0 * (double)v.n_halo + 4.0 * d * (n_src + (double)v.n_halo),
+                   2.0 * d * ((double)v.hnnz + (self_src ? (double)v.n_halo : 0.0)));
 #define ARGS ctx, v, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out
     if (d4 <= 4) launch_hrow<4, 1>(ARGS);
     else if (d4 <= 8) launch_hrow<8, 1>(ARGS);
