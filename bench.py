@@ -330,6 +330,11 @@ def run_ours(args, wl):
     B.sat_profile_enable(ep.ctx, False)
     B.sat_profile_select(ep.ctx, None)
     loss = float(ep.loss_sum.item())
+    # what the L2 -> SM path delivers on this GPU right now (64 MiB buffer resident in L2): contiguous stream, and random
+    # rows of the hidden width with the SpMM's access shape
+    l2_row = int(max(wl.dims[1:-1])) if wl.L > 1 else int(wl.dims[0])
+    l2_row = min(1024, (l2_row + 3) & ~3)
+    l2_stream_gbs, l2_gather_gbs = B.sat_profile_l2_rates(ep.ctx, l2_row)
     # for reference, outside the headline and without any profiling events: the same epochs (a) with a predictor that is
     # never updated (one version throughout: all tau - 1 older projections cached) and (b) with no version promise (nothing
     # kept between epochs: every epoch runs all steps from the raw ring, K = d + h in the recurrence)
@@ -551,7 +556,12 @@ def run_ours(args, wl):
         if fam.startswith("spmm") and rec["flops"] > 0:
             # the SpMM reads one neighbour row per entry: that stream comes mostly out of L2, not HBM; its rate is reported
             # beside the HBM figure (no roof is claimed for it)
-            roofline["gather_gbs"] = rec["flops"] / 2.0 * 4.0 / (rec["ms"] * 1e-3) / 1e9
+            gather = rec["flops"] / 2.0 * 4.0 / (rec["ms"] * 1e-3) / 1e9
+            roofline["l2_gather"] = dict(
+                achieved=gather, unit="GB/s", reference=l2_gather_gbs, reference_stream=l2_stream_gbs, ratio=gather / l2_gather_gbs,
+                what="neighbour-row bytes gathered per second (entries x row bytes / time) against the rate at which this GPU "
+                     f"delivers random {l2_row}-float rows (reference) and a contiguous stream (reference_stream) out of an L2-resident "
+                     "64 MiB buffer, both measured in this run (sat_profile_l2_rates); a ratio above 1 means rows served from L1 / shared memory")
         families = {k: dict(calls=v["calls"], ms_per_step=v["ms"] / args.steps,
                             gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else 0.0,
                             hbm_frac=(v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm"]) if v["ms"] > 0 else 0.0,
@@ -565,7 +575,7 @@ def run_ours(args, wl):
             cpu = dict(value=edges / secs, unit="edges/s", cores=smp.cores, kind="oracle", seconds=secs,
                        sample=f"{len(smp.blocks)} x " + smp.describe() + f"; {edges} edges")
         # whole-epoch view: algorithmic bytes of every kernel family over the epoch time, against the HBM copy rate; the
-        # SpMM families also as the gather rate they sustain from L2 (entries x row bytes / time), which is what bounds them
+        # SpMM families also as the gather rate they sustain (entries x row bytes / time)
         alg_bytes = sum(v["bytes"] for v in prof.values()) / args.steps
         epoch = dict(ms_median=float(np.median(step_ms)), ms_min=float(min(step_ms)), ms_max=float(max(step_ms)),
                      ms_with_events_on_every_family=ms_profiled,
@@ -573,7 +583,8 @@ def run_ours(args, wl):
                      edge_passes_per_s=world * wl.nnz * 2 * wl.L / (ms_per_step * 1e-3),
                      algorithmic_bytes=alg_bytes, hbm_frac=alg_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm"],
                      spmm_gather_gbs={k: (prof[k]["flops"] / 2.0 * 4.0) / (prof[k]["ms"] * 1e-3) / 1e9
-                                      for k in ("spmm_fwd", "spmm_bwd") if prof.get(k, {}).get("ms", 0) > 0})
+                                      for k in ("spmm_fwd", "spmm_bwd", "spmm_hrow") if prof.get(k, {}).get("ms", 0) > 0},
+                     l2_stream_gbs=l2_stream_gbs, l2_random_row_gbs=l2_gather_gbs, l2_row_floats=l2_row)
         line = dict(metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s", n_gpus=world,
                     steps=args.steps, warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),

@@ -461,6 +461,13 @@ sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask);
 sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int64_t *calls, double *ms, double *bytes,
                             double *flops);
 
+/* What the L2 -> SM path of the GPU delivers, measured now (measurement aid; the paper has no counterpart): a 64 MiB buffer,
+ * resident in L2, read (a) as a contiguous stream by all SMs and (b) as rows of `row_floats` floats (a multiple of 4, at most
+ * 1024) in pseudo-random order with the access shape of the SpMM kernels.  Both in GB/s (HOST outputs, either may be NULL).
+ * Allocates and frees its buffer; synchronises the stream.  The SpMM's neighbour-row gather comes mostly out of L2, so
+ * these are the rates to hold its gather rate against — measured in the same run, on the same GPU, at the same clocks. */
+sat_status sat_profile_l2_rates(sat_ctx *ctx, int32_t row_floats, double *stream_gbs, double *gather_gbs);
+
 #ifdef __cplusplus
 }
 #endif

@@ -63,7 +63,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step", "sat_sgd_steps",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores", "sat_profile_l2_rates",
 ]
 
 
@@ -416,6 +416,13 @@ def sat_launch_count(ctx) -> int:
     c = C.c_int64()
     _check(ctx, _lib.sat_launch_count(ctx, C.byref(c)))
     return c.value
+
+
+def sat_profile_l2_rates(ctx, row_floats: int):
+    """(stream GB/s, random-row gather GB/s) out of an L2-resident 64 MiB buffer, measured now."""
+    a, b = C.c_double(), C.c_double()
+    _check(ctx, _lib.sat_profile_l2_rates(ctx, C.c_int32(row_floats), C.byref(a), C.byref(b)))
+    return float(a.value), float(b.value)
 
 
 def sat_profile_families() -> int:

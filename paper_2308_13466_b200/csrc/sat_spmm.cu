@@ -519,3 +519,117 @@ sat_status sat_sum_by_slot(sat_ctx *ctx, int32_t d, const float *src, int32_t ld
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
+
+
+// -------------------------------------------------------------------------------------
+// Measurement aid: what the L2 -> SM path of this GPU delivers, measured in the run that quotes it.
+//   stream: every thread block reads a contiguous 128-bit-per-lane stream of a buffer that fits in L2;
+//   gather: one warp per item reads `row_floats`-wide rows of that buffer in a seeded pseudo-random order with the
+//           access shape of the SpMM (lanes own 128-bit column slices, several rows in flight), accumulating them.
+// Results are kept live through a predicated store that never fires for finite data.
+// -------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+k_l2_stream(const float4 *__restrict__ buf, int64_t n_vec, int reps, float *__restrict__ sink)
+{
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int r = 0; r < reps; ++r) {
+        int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+        for (; i + 3 * stride < n_vec; i += 4 * stride) {
+            const float4 a = __ldg(buf + i), b = __ldg(buf + i + stride), c = __ldg(buf + i + 2 * stride), d = __ldg(buf + i + 3 * stride);
+            acc.x += a.x + b.x + c.x + d.x;
+            acc.y += a.y + b.y + c.y + d.y;
+            acc.z += a.z + b.z + c.z + d.z;
+            acc.w += a.w + b.w + c.w + d.w;
+        }
+        for (; i < n_vec; i += stride) {
+            const float4 a = __ldg(buf + i);
+            acc.x += a.x; acc.y += a.y; acc.z += a.z; acc.w += a.w;
+        }
+    }
+    if (acc.x + acc.y + acc.z + acc.w == 12345.678f) sink[0] = acc.x;   // never true for the zero-filled buffer
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256, NV <= 2 ? 8 : 4)
+k_l2_gather(const float *__restrict__ buf, int64_t n_rows, int32_t d4, int64_t n_items, int per_item, float *__restrict__ sink)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t item = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (item >= n_items) return;
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint64_t state = 0x9E3779B97F4A7C15ull * (uint64_t)(item + 1);
+    for (int e = 0; e < per_item; e += 4) {
+        int64_t r[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            state = state * 6364136223846793005ull + 1442695040888963407ull;   // the same sequence in every lane of the warp
+            r[u] = (int64_t)((state >> 20) % (uint64_t)n_rows);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const float *src = buf + r[u] * (4 * (int64_t)d4);
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = lane + 32 * v;
+                if (idx < d4) fma4(acc[v], 0.5f, ld4(src + 4 * idx));
+            }
+        }
+    }
+    float t = 0.f;
+#pragma unroll
+    for (int v = 0; v < NV; ++v) t += acc[v].x + acc[v].y + acc[v].z + acc[v].w;
+    if (t == 12345.678f) sink[0] = t;
+}
+
+extern "C" sat_status sat_profile_l2_rates(sat_ctx *ctx, int32_t row_floats, double *stream_gbs, double *gather_gbs)
+{
+    CHECK_CTX(ctx);
+    if (row_floats < 4 || row_floats > 1024 || (row_floats & 3)) return sat_fail(ctx, SAT_EINVAL, "sat_profile_l2_rates: row width must be a multiple of 4 in [4, 1024]");
+    const size_t bytes = (size_t)64 << 20;                        // well inside the 126 MB L2
+    const int32_t d4 = row_floats / 4;
+    const int64_t n_rows = (int64_t)(bytes / ((size_t)row_floats * 4));
+    float *buf = nullptr, *sink = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    cudaError_t e = cudaMalloc((void **)&buf, bytes);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&sink, 256);
+    if (e == cudaSuccess) e = cudaMemsetAsync(buf, 0, bytes, ctx->stream);
+    if (e == cudaSuccess) e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    float ms_stream = 0.f, ms_gather = 0.f;
+    const int reps = 8, per_item = 64;
+    const int64_t n_items = (int64_t)1 << 20;                      // 64 rows each: 64 Mi row reads per launch
+    if (e == cudaSuccess) {
+        const int64_t n_vec = (int64_t)(bytes / 16);
+        for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {  // first pass warms the L2 and the instruction cache
+            cudaEventRecord(e0, ctx->stream);
+            k_l2_stream<<<148 * 8, 256, 0, ctx->stream>>>((const float4 *)buf, n_vec, reps, sink);
+            cudaEventRecord(e1, ctx->stream);
+            ctx->launches++;
+            e = cudaEventSynchronize(e1);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms_stream, e0, e1);
+        }
+        for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
+            cudaEventRecord(e0, ctx->stream);
+            const unsigned grid = (unsigned)cdiv64(n_items * 32, 256);
+            if (d4 <= 32) k_l2_gather<1><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
+            else if (d4 <= 64) k_l2_gather<2><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
+            else if (d4 <= 128) k_l2_gather<4><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
+            else k_l2_gather<8><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
+            cudaEventRecord(e1, ctx->stream);
+            ctx->launches++;
+            e = cudaEventSynchronize(e1);
+            if (e == cudaSuccess) e = cudaEventElapsedTime(&ms_gather, e0, e1);
+        }
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(buf);
+    cudaFree(sink);
+    if (e != cudaSuccess) return sat_check_cuda(ctx, e, "sat_profile_l2_rates");
+    if (stream_gbs) *stream_gbs = (double)bytes * reps / (ms_stream * 1e-3) / 1e9;
+    if (gather_gbs) *gather_gbs = (double)n_items * per_item * row_floats * 4.0 / (ms_gather * 1e-3) / 1e9;
+    return SAT_OK;
+}
