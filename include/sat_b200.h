@@ -52,7 +52,7 @@ enum {
 
 enum { SAT_HOST = 0, SAT_DEVICE = 1 };                   /* where an index array lives           */
 enum { SAT_ALL_PARTS = -1 };
-enum { SAT_PART_GIVEN = 0, SAT_PART_CONTIG_BLOCKS = 1 }; /* sat_partition methods                */
+enum { SAT_PART_GIVEN = 0, SAT_PART_CONTIG_BLOCKS = 1, SAT_PART_BFS_BLOCKS = 2 }; /* sat_partition methods */
 enum { SAT_ACT_NONE = 0, SAT_ACT_RELU = 1 };
 /* Flag for the `act` argument of sat_layer_fwd (act = SAT_ACT_* | SAT_FWD_PUSH): the rows of h_out that belong to boundary
  * nodes are also written into the write buffer of cached layer `layer`, exactly what sat_cache_update(part, layer, h_out)
@@ -112,9 +112,12 @@ sat_status sat_graph_dinv(sat_ctx *ctx, float *dinv_host);
  *   C = sorted union of all B_m = the nodes the cache stores; slot[v] = rank of v in C or -1
  *   push list of m: local ids (ascending) and slots of the inner nodes of m that are in C.
  * Methods: SAT_PART_GIVEN uses part_of_node (int32 [n], values in [0, M), HOST or DEVICE
- * per `ptr_space`); SAT_PART_CONTIG_BLOCKS ignores it and uses part[v] = floor(v*M/n)
- * (the paper partitions with METIS, which is a third-party tool and not part of this
- * library: pass its output through SAT_PART_GIVEN).
+ * per `ptr_space`); SAT_PART_CONTIG_BLOCKS ignores it and uses part[v] = floor(v*M/n);
+ * SAT_PART_BFS_BLOCKS ignores it too: rank[v] = position of v in a breadth-first traversal (FIFO queue, start at node 0,
+ * neighbours in ascending id, restart at the smallest unvisited id when the queue is empty) and part[v] =
+ * floor(rank[v]*M/n); the graph is not relabelled.  That traversal runs on the host over a copy of the graph (set-up work).
+ * (The paper partitions with METIS, which is a third-party tool and not part of this
+ * library: pass its output through SAT_PART_GIVEN.)
  * All structures are integer and are built on the device; this call synchronises.
  * ------------------------------------------------------------------------------------- */
 sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const int32_t *part_of_node, int ptr_space);

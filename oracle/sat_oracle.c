@@ -504,3 +504,32 @@ int64_t orc_codec_decode(int64_t rows, int32_t d, const uint8_t *in, const int64
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------
+ * O-2 (partitioner)  Breadth-first visit order with a plain first-in first-out queue: start at node 0, neighbours of the
+ * node taken off the queue are visited in ascending id (the CSR rows are sorted), and when the queue runs empty the
+ * traversal restarts at the smallest unvisited id.  rank[v] = position of v in the visit order.  The partitioner built on
+ * it cuts that order into M equal blocks (Algorithm 1, "Partitioning the raw graph": any non-overlapping partition will do).
+ * ------------------------------------------------------------------------------------ */
+void orc_bfs_rank(int32_t n, const int64_t *rowptr, const int32_t *col, int32_t *rank)
+{
+    int32_t *queue = (int32_t *)malloc(sizeof(int32_t) * (size_t)(n > 0 ? n : 1));
+    for (int32_t v = 0; v < n; ++v) rank[v] = -1;
+    int32_t head = 0, tail = 0, visited = 0;
+    for (int32_t start = 0; start < n; ++start) {
+        if (rank[start] >= 0) continue;
+        rank[start] = visited++;
+        queue[tail++] = start;
+        while (head < tail) {
+            int32_t u = queue[head++];
+            for (int64_t e = rowptr[u]; e < rowptr[u + 1]; ++e) {
+                int32_t w = col[e];
+                if (rank[w] < 0) {
+                    rank[w] = visited++;
+                    queue[tail++] = w;
+                }
+            }
+        }
+    }
+    free(queue);
+}

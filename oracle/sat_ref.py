@@ -71,6 +71,23 @@ def contig_blocks(n: int, M: int) -> np.ndarray:
     return (np.arange(n, dtype=np.int64) * M // n).astype(np.int32)
 
 
+def bfs_rank(rowptr: np.ndarray, col: np.ndarray) -> np.ndarray:
+    """rank[v] = position of v in the breadth-first visit order (FIFO queue from node 0, neighbours ascending, restart at
+    the smallest unvisited id)."""
+    n = rowptr.shape[0] - 1
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    col = np.ascontiguousarray(col, dtype=np.int32)
+    rank = np.empty(n, dtype=np.int32)
+    lib().orc_bfs_rank(C.c_int32(n), _p(rowptr), _p(col), _p(rank))
+    return rank
+
+
+def bfs_blocks(rowptr: np.ndarray, col: np.ndarray, M: int) -> np.ndarray:
+    """Breadth-first block partition: part[v] = floor(rank[v] * M / n); the graph is not relabelled."""
+    n = rowptr.shape[0] - 1
+    return (bfs_rank(rowptr, col).astype(np.int64) * M // n).astype(np.int32)
+
+
 @dataclass
 class Partitioning:
     n: int

@@ -18,7 +18,7 @@ from .build import lib_path
 SAT_OK, SAT_EINVAL, SAT_ESTATE, SAT_ENOMEM, SAT_ECUDA, SAT_EDATA = 0, -1, -2, -3, -4, -5
 SAT_HOST, SAT_DEVICE = 0, 1
 SAT_ALL_PARTS = -1
-SAT_PART_GIVEN, SAT_PART_CONTIG_BLOCKS = 0, 1
+SAT_PART_GIVEN, SAT_PART_CONTIG_BLOCKS, SAT_PART_BFS_BLOCKS = 0, 1, 2
 SAT_ACT_NONE, SAT_ACT_RELU = 0, 1
 SAT_LOSS_SOFTMAX_CE, SAT_LOSS_SIGMOID_BCE = 0, 1
 SAT_BWD_ACCUMULATE, SAT_BWD_MASK_G_IN, SAT_BWD_G_OUT_MASKED, SAT_BWD_GRAD_HISTORY = 1, 2, 4, 8

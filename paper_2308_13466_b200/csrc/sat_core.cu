@@ -1,5 +1,7 @@
 // Context, graph load and partition construction of the sat_b200 library.
 // All graph structures are integer and are built by the kernels below on the device.
+#include <new>
+
 #include "sat_internal.h"
 
 // =====================================================================================
@@ -842,13 +844,60 @@ static sat_status copy_i64(sat_ctx *ctx, const int64_t *dev, int64_t *host)
 #define GRID1(count) (unsigned)cdiv64((count) > 0 ? (count) : 1, 256), 256, 0, ctx->stream
 #define GRIDW(count) (unsigned)cdiv64(((count) > 0 ? (int64_t)(count) : 1) * 32, 256), 256, 0, ctx->stream
 
+// SAT_PART_BFS_BLOCKS: breadth-first visit order of the loaded graph (first-in first-out queue, start at node 0, the
+// neighbours of a node taken in ascending id, restart at the smallest unvisited id when the queue runs empty);
+// part[v] = floor(rank[v] * M / n).  The visit order of a FIFO traversal is inherently sequential, and this is set-up work
+// done once per graph: it runs on the host over a copy of the CSR arrays, and only part[] goes back to the device.
+static sat_status bfs_block_partition(sat_ctx *ctx, int32_t M, int32_t *part_dev)
+{
+    const int32_t n = ctx->n;
+    const int64_t nnz = ctx->nnz;
+    std::vector<int64_t> rp;
+    std::vector<int32_t> cl, order, part;
+    std::vector<uint8_t> seen;
+    try {
+        rp.resize((size_t)n + 1);
+        cl.resize((size_t)(nnz > 0 ? nnz : 1));
+        order.reserve((size_t)n);
+        part.resize((size_t)n);
+        seen.assign((size_t)n, 0);
+    } catch (const std::bad_alloc &) {
+        return sat_fail(ctx, SAT_ENOMEM, "sat_partition: host memory for the breadth-first ordering");
+    }
+    SAT_CUDA(ctx, cudaMemcpyAsync(rp.data(), ctx->rowptr, sizeof(int64_t) * ((size_t)n + 1), cudaMemcpyDeviceToHost, ctx->stream));
+    if (nnz) SAT_CUDA(ctx, cudaMemcpyAsync(cl.data(), ctx->col, sizeof(int32_t) * (size_t)nnz, cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    int32_t next_start = 0;
+    size_t head = 0;
+    while ((int32_t)order.size() < n) {
+        while (seen[next_start]) ++next_start;
+        seen[next_start] = 1;
+        order.push_back(next_start);
+        while (head < order.size()) {
+            const int32_t u = order[head++];
+            for (int64_t e = rp[u]; e < rp[u + 1]; ++e) {
+                const int32_t w = cl[e];
+                if (!seen[w]) {
+                    seen[w] = 1;
+                    order.push_back(w);
+                }
+            }
+        }
+    }
+    for (int32_t r = 0; r < n; ++r) part[order[r]] = (int32_t)(((int64_t)r * M) / n);
+    SAT_CUDA(ctx, cudaMemcpyAsync(part_dev, part.data(), sizeof(int32_t) * (size_t)n, cudaMemcpyHostToDevice, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
 extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const int32_t *part_of_node, int ptr_space)
 {
     if (!ctx) return SAT_EINVAL;
     if (ctx->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error");
     if (!ctx->graph_ok) return sat_fail(ctx, SAT_ESTATE, "sat_partition: call sat_graph_load first");
     if (M <= 0 || M > SAT_MAX_PARTS || M > ctx->n) return sat_fail(ctx, SAT_EINVAL, "sat_partition: M must be in [1, min(n, %d)]", SAT_MAX_PARTS);
-    if (method != SAT_PART_GIVEN && method != SAT_PART_CONTIG_BLOCKS) return sat_fail(ctx, SAT_EINVAL, "sat_partition: unknown method");
+    if (method != SAT_PART_GIVEN && method != SAT_PART_CONTIG_BLOCKS && method != SAT_PART_BFS_BLOCKS)
+        return sat_fail(ctx, SAT_EINVAL, "sat_partition: unknown method");
     if (method == SAT_PART_GIVEN && (!part_of_node || (ptr_space != SAT_HOST && ptr_space != SAT_DEVICE)))
         return sat_fail(ctx, SAT_EINVAL, "sat_partition: SAT_PART_GIVEN needs part_of_node and a valid ptr_space");
     SAT_CUDA(ctx, cudaSetDevice(ctx->device));
@@ -871,6 +920,8 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
         int flag = 0;
         SAT_TRY(read_flag(ctx, &flag));
         if (flag) return sat_fail(ctx, SAT_EINVAL, "sat_partition: part_of_node has a value outside [0, M)");
+    } else if (method == SAT_PART_BFS_BLOCKS) {
+        SAT_TRY(bfs_block_partition(ctx, M, ctx->part));
     } else {
         k_part_contig<<<GRID1(n)>>>(n, M, ctx->part);
         SAT_LAUNCHED(ctx);

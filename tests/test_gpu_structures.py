@@ -91,6 +91,36 @@ def test_workload_partitions(B, name, shrink):
         B.sat_destroy(ctx)
 
 
+@pytest.mark.parametrize("case", ["five", "random-disconnected", "edgeless", "rmat"])
+def test_bfs_block_partitioner(B, five_node, case):
+    """SAT_PART_BFS_BLOCKS: breadth-first order inside the library (FIFO from node 0, neighbours ascending, restarts at the
+    smallest unvisited id), cut into M blocks; the graph keeps its ids, so the blocks are scattered id sets.  part[] and
+    every derived structure against the oracle's own traversal."""
+    from sat_synth import rmat_graph
+    if case == "five":
+        rowptr, col = csr_from_edges(5, five_node["edges"])
+        M = 2
+    elif case == "random-disconnected":
+        rowptr, col = random_graph(np.random.default_rng(11), 400, 0.004)
+        M = 5
+    elif case == "edgeless":
+        rowptr, col = random_graph(np.random.default_rng(12), 50, 0.0)
+        M = 3
+    else:
+        rowptr, col = rmat_graph(4, 15, 21_000, n_samples=150_000)       # seeded id permutation, no relabelling
+        M = 8
+    part = orc.bfs_blocks(rowptr, col, M)
+    ctx = B.sat_create(0, 0)
+    try:
+        B.sat_graph_load(ctx, rowptr, col)
+        B.sat_partition(ctx, M, B.SAT_PART_BFS_BLOCKS)
+        _compare_partition(B, ctx, rowptr, col, part, M)
+        if case == "five":
+            assert part.tolist() == five_node["part"]
+    finally:
+        B.sat_destroy(ctx)
+
+
 def test_device_resident_inputs(B):
     import torch
     wl = make_workload("tiny", with_dense=False)

@@ -91,3 +91,60 @@ def test_contig_blocks():
     assert part[0] == 0 and part[-1] == 31 and np.all(np.diff(part) >= 0)
     cnt = np.bincount(part)
     assert cnt.max() - cnt.min() <= 1
+
+
+# ------------------------------------------------------------------------------------------
+# breadth-first block partitioner
+# ------------------------------------------------------------------------------------------
+def test_bfs_blocks_five_node(five_node):
+    """Hand-worked: from node 0 the queue visits 0, 1, then 1's unvisited neighbours 2, 3 in ascending id, then 4: the visit
+    order is the id order, and two blocks of it are the example's partition (0, 0, 0, 1, 1)."""
+    from tests.dense_pins import csr_from_edges
+    rowptr, col = csr_from_edges(5, five_node["edges"])
+    assert orc.bfs_rank(rowptr, col).tolist() == [0, 1, 2, 3, 4]
+    assert orc.bfs_blocks(rowptr, col, 2).tolist() == five_node["part"]
+    # a star seen from a leaf: 0 - 3, 3 - {1, 2, 4}: visit order 0, 3, 1, 2, 4
+    rowptr, col = csr_from_edges(5, [[0, 3], [3, 1], [3, 2], [3, 4]])
+    assert orc.bfs_rank(rowptr, col).tolist() == [0, 2, 3, 1, 4]
+
+
+def _queue_bfs(rowptr, col):
+    from collections import deque
+    n = rowptr.shape[0] - 1
+    rank = [-1] * n
+    k = 0
+    for s in range(n):
+        if rank[s] >= 0:
+            continue
+        rank[s] = k
+        k += 1
+        q = deque([s])
+        while q:
+            u = q.popleft()
+            for w in sorted(col[rowptr[u]:rowptr[u + 1]].tolist()):
+                if rank[w] < 0:
+                    rank[w] = k
+                    k += 1
+                    q.append(w)
+    return rank
+
+
+@pytest.mark.parametrize("seed,n,p", [(0, 40, 0.08), (1, 60, 0.02), (2, 25, 0.0), (3, 80, 0.05)])
+def test_bfs_rank_against_a_queue_and_the_library_traversal(seed, n, p):
+    """Random graphs, most of them disconnected (restarts at the smallest unvisited id): a deque written out in Python; on the
+    component of node 0, scipy's breadth-first order (which also walks the sorted CSR rows); and the invariants of a
+    breadth-first order (a bijection; every non-root node has a neighbour with a smaller rank inside its component)."""
+    import scipy.sparse as sp
+    from scipy.sparse.csgraph import breadth_first_order
+    from tests.dense_pins import random_graph
+    rng = np.random.default_rng(seed)
+    rowptr, col = random_graph(rng, n, p)
+    rank = orc.bfs_rank(rowptr, col)
+    assert rank.tolist() == _queue_bfs(rowptr, col)
+    assert sorted(rank.tolist()) == list(range(n))
+    A = sp.csr_matrix((np.ones(col.shape[0], dtype=np.int8), col, rowptr), shape=(n, n))
+    first = breadth_first_order(A, 0, directed=False, return_predecessors=False)
+    assert rank[first].tolist() == list(range(first.shape[0]))
+    part = orc.bfs_blocks(rowptr, col, 4)
+    assert np.array_equal(part, (rank.astype(np.int64) * 4 // n).astype(np.int32))
+    assert np.bincount(part, minlength=4).max() - np.bincount(part, minlength=4).min() <= 1
