@@ -444,6 +444,16 @@ sat_status sat_codec_decode(sat_ctx *ctx, const uint8_t *in, int64_t in_bytes, c
                             int32_t precision, float *x, int32_t ld);
 sat_status sat_cache_requantise(sat_ctx *ctx, int32_t layer, int32_t age, int32_t precision, int64_t *bytes);
 
+/* Bounds-checking debug build (libsat_b200_dbg.so: the same sources compiled with -DSAT_DEBUG_BOUNDS; the paper has no
+ * counterpart).  Every index the graph kernels (SpMM, halo-row products, row gather / scatter, per-slot sums) load from an
+ * index array is compared with the extent of the matrix it addresses; an index outside it raises a bit of the device status
+ * word — sat_sync_status then returns SAT_EDATA once, the context stays usable — and is replaced by a valid index before use, so
+ * nothing outside the matrix is touched: no trap, no device assert.  It stands in for a memory checker on these kernels.
+ * sat_debug_poke_index overwrites entry `pos` of an internal index array (which = 0: encoded column ids of the local CSR,
+ * length nnz(A+I); 1: cache slots of the halo positions, length sum_m b_m) and returns the old value (HOST, nullable), so
+ * that a test can show the checks at work; in the regular build it changes nothing and returns SAT_ESTATE. */
+sat_status sat_debug_poke_index(sat_ctx *ctx, int which, int64_t pos, int32_t value, int32_t *old_value);
+
 /* Number of kernels this context has launched since creation (all entry points). */
 sat_status sat_launch_count(sat_ctx *ctx, int64_t *count);
 

@@ -44,7 +44,8 @@ SAT_CELL_LSTM, SAT_CELL_GRU = 0, 1
 
 
 def _load():
-    path = lib_path()
+    # SAT_B200_DEBUG=1 selects the bounds-checking build of the same sources (libsat_b200_dbg.so)
+    path = lib_path(debug=os.environ.get("SAT_B200_DEBUG", "0") == "1")
     if not os.path.exists(path):
         raise ImportError(f"{path} is missing: build it with `python -m paper_2308_13466_b200.build` "
                           "(there is no fallback implementation)")
@@ -63,7 +64,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step", "sat_sgd_steps",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores", "sat_profile_l2_rates",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores", "sat_profile_l2_rates", "sat_debug_poke_index",
 ]
 
 
@@ -416,6 +417,13 @@ def sat_launch_count(ctx) -> int:
     c = C.c_int64()
     _check(ctx, _lib.sat_launch_count(ctx, C.byref(c)))
     return c.value
+
+
+def sat_debug_poke_index(ctx, which: int, pos: int, value: int) -> int:
+    """Debug build only: overwrite one entry of an internal index array; returns the old value."""
+    old = C.c_int32(0)
+    _check(ctx, _lib.sat_debug_poke_index(ctx, C.c_int(which), C.c_int64(pos), C.c_int32(value), C.byref(old)))
+    return int(old.value)
 
 
 def sat_profile_l2_rates(ctx, row_floats: int):

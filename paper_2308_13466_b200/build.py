@@ -12,8 +12,11 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
               "-Xcompiler", "-fPIC"]
 
 
-def lib_path() -> str:
-    return os.path.join(_HERE, LIB_NAME)
+DEBUG_LIB_NAME = "libsat_b200_dbg.so"   # the same sources with -DSAT_DEBUG_BOUNDS (index checks in the graph kernels)
+
+
+def lib_path(debug: bool = False) -> str:
+    return os.path.join(_HERE, DEBUG_LIB_NAME if debug else LIB_NAME)
 
 
 def sources():
@@ -31,22 +34,25 @@ def _stale(out: str) -> bool:
 LAST_ACTION = None   # "compiled" or "reused": what the most recent build() call did
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compiles the library when it is older than a source file; debug=True builds the bounds-checking variant."""
     global LAST_ACTION
-    out = lib_path()
+    out = lib_path(debug)
     if not force and not _stale(out):
-        LAST_ACTION = "reused"
+        if not debug:
+            LAST_ACTION = "reused"
         return out
-    LAST_ACTION = "compiled"
+    if not debug:
+        LAST_ACTION = "compiled"
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    objdir = os.path.join(_HERE, "build")
+    objdir = os.path.join(_HERE, "build", "dbg" if debug else "rel")
     os.makedirs(objdir, exist_ok=True)
     objs = []
     procs = []
     for src in sources():
         obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        cmd = [nvcc, *NVCC_FLAGS, "-c", src, "-o", obj]
+        cmd = [nvcc, *NVCC_FLAGS, *(["-DSAT_DEBUG_BOUNDS"] if debug else []), "-c", src, "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas=-v")
         procs.append((cmd, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
@@ -57,11 +63,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         if p.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd) + "\n" + (log or ""))
     tmp = out + f".tmp{os.getpid()}"
-    cmd = [nvcc, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"]
+    cmd = [nvcc, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a", "-ldl"]
     subprocess.run(cmd, check=True)
     os.replace(tmp, out)
     return out
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -222,11 +222,34 @@ extern "C" sat_status sat_sync_status(sat_ctx *ctx)
         ctx->cuda_failed = true;
         return sat_fail(ctx, SAT_ECUDA, "a tensor-core kernel gave up waiting on a barrier (status %d)", *ctx->h_flag);
     }
+    if (*ctx->h_flag & 4) {  // debug build only: an index outside its matrix was met (and replaced by 0); reported once
+        SAT_CUDA(ctx, cudaMemsetAsync(ctx->d_flag + 1, 0, sizeof(int), ctx->stream));
+        return sat_fail(ctx, SAT_EDATA, "bounds check of the debug build: a graph kernel loaded an index outside the matrix it addresses");
+    }
     if (*ctx->h_flag & 2) {  // malformed codec input: reported once, the context stays usable
         SAT_CUDA(ctx, cudaMemsetAsync(ctx->d_flag + 1, 0, sizeof(int), ctx->stream));
         return sat_fail(ctx, SAT_EDATA, "sat_codec_decode: a row does not hold exactly d well-formed values");
     }
     return SAT_OK;
+}
+
+// Debug build only: overwrite one entry of an internal index array, so that a test can show the bounds checks at work.
+extern "C" sat_status sat_debug_poke_index(sat_ctx *ctx, int which, int64_t pos, int32_t value, int32_t *old_value)
+{
+    CHECK_CTX(ctx);
+#if SAT_DBG
+    if (!ctx->part_ok) return sat_fail(ctx, SAT_ESTATE, "sat_debug_poke_index: call sat_partition first");
+    int32_t *arr = which == 0 ? ctx->lenc : which == 1 ? ctx->halo_slot : nullptr;
+    const int64_t len = which == 0 ? ctx->nnz + ctx->n : ctx->nb;
+    if (!arr || pos < 0 || pos >= len) return sat_fail(ctx, SAT_EINVAL, "sat_debug_poke_index: unknown array or position outside it");
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (old_value) SAT_CUDA(ctx, cudaMemcpy(old_value, arr + pos, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    SAT_CUDA(ctx, cudaMemcpy(arr + pos, &value, sizeof(int32_t), cudaMemcpyHostToDevice));
+    return SAT_OK;
+#else
+    (void)which; (void)pos; (void)value; (void)old_value;
+    return sat_fail(ctx, SAT_ESTATE, "sat_debug_poke_index: only in the bounds-checking debug build of the library");
+#endif
 }
 
 extern "C" sat_status sat_launch_count(sat_ctx *ctx, int64_t *count)
@@ -447,6 +470,7 @@ __global__ void k_dinv(const int64_t *__restrict__ rowptr, int32_t n, float *__r
 extern "C" sat_status sat_graph_load(sat_ctx *ctx, int32_t n, int64_t nnz, const int64_t *rowptr, const int32_t *col,
                                      int ptr_space)
 {
+    SatRange sat_range__(__func__);
     if (!ctx) return SAT_EINVAL;
     if (ctx->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error");
     if (n <= 0 || nnz < 0 || !rowptr || (nnz > 0 && !col)) return sat_fail(ctx, SAT_EINVAL, "sat_graph_load: bad n / nnz / null array");
@@ -892,6 +916,7 @@ static sat_status bfs_block_partition(sat_ctx *ctx, int32_t M, int32_t *part_dev
 
 extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const int32_t *part_of_node, int ptr_space)
 {
+    SatRange sat_range__(__func__);
     if (!ctx) return SAT_EINVAL;
     if (ctx->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error");
     if (!ctx->graph_ok) return sat_fail(ctx, SAT_ESTATE, "sat_partition: call sat_graph_load first");

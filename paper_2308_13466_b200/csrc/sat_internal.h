@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include <atomic>
@@ -16,6 +17,43 @@
 #define SAT_MAX_PARTS 4096
 #define SAT_SPMM_CHUNK 256 /* edges per SpMM work item */
 #define SAT_HROW_LONG 256  /* halo rows with more entries than this get a whole thread block */
+
+// Debug build (-DSAT_DEBUG_BOUNDS, libsat_b200_dbg.so): every index the graph kernels load from an index array (column ids,
+// row lists, cache slots) is checked against the extent of the matrix it addresses; an index outside it raises bit 4 of
+// the device status word (reported by sat_sync_status as SAT_EDATA) and is replaced by the first valid index, so the access that
+// follows stays inside the matrix: no trap, no assert, the context stays usable.  The stand-in for a memory checker on these kernels.
+#ifdef SAT_DEBUG_BOUNDS
+#define SAT_DBG 1
+#ifdef __CUDACC__
+__device__ __forceinline__ int64_t sat_bound(int64_t i, int64_t lo, int64_t hi, int *status)
+{
+    if (i < lo || i >= hi) {
+        atomicOr(status, 4);
+        return lo;    // a row that exists (the kernels are not launched on empty matrices)
+    }
+    return i;
+}
+#endif
+#define SAT_IDX(i, lo, hi, status) sat_bound((i), (lo), (hi), (status))
+#else
+#define SAT_DBG 0
+#define SAT_IDX(i, lo, hi, status) (i)
+#endif
+// valid row indices [lo, hi) of a matrix as a kernel addresses it (a per-partition view starts above 0)
+struct DbgRange {
+    int64_t lo, hi;
+};
+// index ranges handed to the graph kernels for those checks (unused, and optimised away, in the regular build)
+struct DbgLimits {
+    int64_t src_lo, src_hi;     // rows of the first source matrix (inner rows / cache slots / generic source)
+    int64_t halo_lo, halo_hi;   // rows of the halo source matrix
+    int64_t out_lo, out_hi;     // rows of the output
+    int *status;                // device status word
+};
+static inline DbgLimits dbg_limits(DbgRange src, DbgRange halo, DbgRange out, int *status)
+{
+    return DbgLimits{src.lo, src.hi, halo.lo, halo.hi, out.lo, out.hi, status};
+}
 
 // A growable device buffer owned by the context.
 struct DevBuf {
@@ -203,8 +241,18 @@ struct ProfScope {
     }
 };
 
-// entry-point prologue: a usable context on its device
+// NVTX range around an entry point (named after the function): shows the library's calls on a profiler's timeline; costs
+// a few nanoseconds when no tool is attached
+struct SatRange {
+    explicit SatRange(const char *name) { nvtxRangePushA(name); }
+    ~SatRange() { nvtxRangePop(); }
+    SatRange(const SatRange &) = delete;
+    SatRange &operator=(const SatRange &) = delete;
+};
+
+// entry-point prologue: an NVTX range for the call, and a usable context on its device
 #define CHECK_CTX(ctx)                                                                             \
+    SatRange sat_range__(__func__);                                                                \
     do {                                                                                           \
         if (!(ctx)) return SAT_EINVAL;                                                             \
         if ((ctx)->cuda_failed) return sat_fail(ctx, SAT_ECUDA, "context has a sticky CUDA error"); \
@@ -265,17 +313,22 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
 //   halo-row products: out[j] = sum_{e in hrow(j)} dinv[halo j] dinv[inner e] * src[pos_e]   (+ self term if self_src)
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src,
                          int by_slot, const float *self_src, float *out_base, int32_t ld_out);
+// src_rows / dst_rows: valid row indices of the source / destination matrices, used by the debug build's index checks
+// (SAT_ANY_ROW: unknown, not checked)
+static const DbgRange SAT_ANY_ROW = {INT64_MIN, INT64_MAX};
 sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d, const float *src, int32_t ld_src,
-                      float *out, int32_t ld_out);
+                      float *out, int32_t ld_out, DbgRange src_rows = SAT_ANY_ROW);
 sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d,
-                       const float *src_base, int32_t ld_src, float *dst, int32_t ld_dst);
+                       const float *src_base, int32_t ld_src, float *dst, int32_t ld_dst, DbgRange src_rows = SAT_ANY_ROW,
+                       DbgRange dst_rows = SAT_ANY_ROW);
 // out[s] (+)= scale_s * sum over the halo positions p of cache slot s, in ascending partition order, of src[p]; scale_s = p_ss
 // (the self-loop weight of the node behind the slot) when self_scale, else 1.  One writer per slot: no atomics, fixed order.
 sat_status sat_sum_by_slot(sat_ctx *ctx, int32_t d, const float *src, int32_t ld_src, int self_scale, int add, float *out, int32_t ld_out);
 // dst[dst_row[i]] += src[src_row ? src_row[i] : i] (o mask bits of the destination row, when given); the dst_row[i] of one
 // call must be distinct
 sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
-                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words);
+                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words, DbgRange src_rows = SAT_ANY_ROW,
+                           DbgRange dst_rows = SAT_ANY_ROW);
 
 // GEMM family (sat_gemm.cu)
 // C[m x n] = A[m x k] B[k x n] (+ bias) with optional ReLU, sign-mask output, row-gathered residual add.

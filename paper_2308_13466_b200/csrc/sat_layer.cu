@@ -32,7 +32,7 @@ extern "C" sat_status sat_gather_rows(sat_ctx *ctx, int32_t part, int which, con
     if (!x || !out || d <= 0 || !ok_ld(ld_x, d) || !ok_ld(ld_out, d) || !aligned16(x) || !aligned16(out))
         return sat_fail(ctx, SAT_EINVAL, "sat_gather_rows: null / misaligned tensor or bad leading dimension");
     const int32_t *idx = which == SAT_ROWS_INNER ? ctx->perm + v.row0 : ctx->halo_gid + v.halo0;
-    return sat_gather(ctx, idx, count, d, x, ld_x, out, ld_out);
+    return sat_gather(ctx, idx, count, d, x, ld_x, out, ld_out, DbgRange{0, ctx->n});
 }
 
 // =====================================================================================
@@ -97,7 +97,7 @@ extern "C" sat_status sat_cache_update(sat_ctx *ctx, int32_t part, int32_t layer
     if (!c->proj_tag.empty()) c->proj_tag[ctx->write_idx] = 0;  // the buffer changes: its cached input projection is stale
     const float *src_base = h_out - (int64_t)v.row0 * ld;
     return sat_scatter(ctx, ctx->push_row + v.push0, ctx->push_slot + v.push0, v.n_push, c->width, src_base, ld,
-                       ring_buf(ctx, c, ctx->write_idx), c->ld);
+                       ring_buf(ctx, c, ctx->write_idx), c->ld, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{0, ctx->n_slots});
 }
 
 extern "C" sat_status sat_cache_commit(sat_ctx *ctx)
@@ -534,7 +534,7 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
             SAT_CUDA(ctx, cudaMemset2DAsync(halo_out, (size_t)ld_out * 4, 0, (size_t)d * 4, (size_t)v.n_halo, ctx->stream));
             return SAT_OK;
         }
-        return sat_gather(ctx, ctx->halo_slot + v.halo0, v.n_halo, d, newest, c->ld, halo_out, ld_out);
+        return sat_gather(ctx, ctx->halo_slot + v.halo0, v.n_halo, d, newest, c->ld, halo_out, ld_out, DbgRange{0, ctx->n_slots});
     }
     if (params->h <= 0 || !params->Wx || !params->Uh || !params->b || !params->Wg || !params->bg)
         return sat_fail(ctx, SAT_EINVAL, "sat_predict: incomplete predictor parameters");
@@ -798,7 +798,7 @@ extern "C" sat_status sat_layer_bwd(sat_ctx *ctx, int32_t part, int32_t layer, c
         SAT_TRY(sat_ensure(ctx, ctx->buf_ghist_rows, (size_t)v.n_push * GH.ld * sizeof(float)));
         SAT_TRY(sat_ensure(ctx, ctx->buf_ghist_out, (size_t)v.n_push * ld_ga * sizeof(float)));
         float *rows = (float *)ctx->buf_ghist_rows.p, *stale = (float *)ctx->buf_ghist_out.p;
-        SAT_TRY(sat_gather(ctx, ctx->push_slot + v.push0, v.n_push, d_out, qr, GH.ld, rows, GH.ld));
+        SAT_TRY(sat_gather(ctx, ctx->push_slot + v.push0, v.n_push, d_out, qr, GH.ld, rows, GH.ld, DbgRange{0, ctx->n_slots}));
         if (sat_use_tc(d_in, d_out)) {
             TcWeights Wp;
             SAT_TRY(sat_tc_weights(ctx, W, d_out, d_out, nullptr, 0, 0, d_in, 0, ctx->buf_wsplit, &Wp));

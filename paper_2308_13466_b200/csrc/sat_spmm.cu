@@ -44,7 +44,8 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
              const float *__restrict__ lw, const float *__restrict__ dinv_enc, const int32_t *__restrict__ item_row, const int32_t *__restrict__ first_item,
              const int32_t *__restrict__ item_mslot, int32_t item0, int32_t n_items, int32_t mitem0, int inner_only, int32_t n,
              int32_t d4, const float *__restrict__ in_base, int64_t ld_in, const float *__restrict__ halo_base, int64_t ld_halo,
-             float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial, const uint32_t *__restrict__ omask, int32_t omask_words)
+             float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial, const uint32_t *__restrict__ omask, int32_t omask_words,
+             DbgLimits dbg)
 {
     const int lane = threadIdx.x & (G - 1);
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
@@ -52,7 +53,7 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
     const unsigned mask = group_mask<G>(threadIdx.x & 31);
     const int col0 = blockIdx.y * (G * NV);  // first float4 column of this block column
     const int32_t item = item0 + (int32_t)gid;
-    const int32_t row = item_row[item];
+    const int32_t row = (int32_t)SAT_IDX(item_row[item], dbg.out_lo, dbg.out_hi, dbg.status);
     const int32_t k = item - first_item[row];
     const int64_t rb = lrowptr[row];
     // inner_only: 0 = all entries, 1 = the inner prefix of the row, 2 = its halo suffix
@@ -76,7 +77,8 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
         for (int j = 0; j < cnt; ++j) {
             const int32_t cj = __shfl_sync(mask, c, j, G);
             const float wj = __shfl_sync(mask, w, j, G);
-            const float *src = cj < n ? in_base + (int64_t)cj * ld_in : halo_base + (int64_t)(cj - n) * ld_halo;
+            const float *src = cj < n ? in_base + SAT_IDX((int64_t)cj, dbg.src_lo, dbg.src_hi, dbg.status) * ld_in
+                                      : halo_base + SAT_IDX((int64_t)(cj - n), dbg.halo_lo, dbg.halo_hi, dbg.status) * ld_halo;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
                 const int idx = col0 + lane + v * G;
@@ -111,13 +113,13 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
 __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, int32_t n_mrows, const int32_t *__restrict__ first_item,
                              const int32_t *__restrict__ item_mslot, int32_t mitem0, const float *__restrict__ dinv_enc, int32_t d4,
                              const float *__restrict__ partial, float *__restrict__ out_base, int64_t ld_out,
-                             const uint32_t *__restrict__ omask, int32_t omask_words)
+                             const uint32_t *__restrict__ omask, int32_t omask_words, DbgLimits dbg)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / d4;
     const int c = (int)(t - i * d4);
     if (i >= n_mrows) return;
-    const int32_t row = mrows[mrow0 + i];
+    const int32_t row = (int32_t)SAT_IDX(mrows[mrow0 + i], dbg.out_lo, dbg.out_hi, dbg.status);
     const int32_t it0 = first_item[row], it1 = first_item[row + 1];
     const int32_t ms0 = item_mslot[it0] - mitem0;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -142,7 +144,8 @@ static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_
     dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
     k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->lw, ctx->dinv_enc, ctx->item_row,
                                                         ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
-                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words);
+                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words,
+                                                        dbg_limits(DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo}, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
 }
 
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
@@ -187,7 +190,8 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     SAT_LAUNCHED(ctx);
     if (v.n_mrows > 0) {
         k_spmm_fixup<<<(unsigned)cdiv64((int64_t)v.n_mrows * d4, 256), 256, 0, ctx->stream>>>(
-            ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, ctx->dinv_enc, d4, partial, out_base, ld_out, omask, omask_words);
+            ctx->mrows, v.mrow0, v.n_mrows, ctx->first_item, ctx->item_mslot, v.mitem0, ctx->dinv_enc, d4, partial, out_base, ld_out, omask, omask_words,
+            dbg_limits(DbgRange{0, 0}, DbgRange{0, 0}, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
         SAT_LAUNCHED(ctx);
     }
     return SAT_OK;
@@ -210,7 +214,7 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
                                                 const int32_t *__restrict__ halo_slot,
                                                 const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4,
                                                 const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
-                                                float *__restrict__ out_base, int64_t ld_out)
+                                                float *__restrict__ out_base, int64_t ld_out, const DbgLimits &dbg)
 {
     constexpr int NG = 256 / G;
     __shared__ float4 red[NG][G * NV];
@@ -223,7 +227,7 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
     const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
     for (int64_t e = e0 + grp; e < e1; e += NG) {
         const float w = __ldg(hrow_w + e);
-        const int32_t c = by_slot ? __ldg(hrow_slot + e) : __ldg(hrow_pos + e);
+        const int32_t c = (int32_t)SAT_IDX(by_slot ? __ldg(hrow_slot + e) : __ldg(hrow_pos + e), dbg.src_lo, dbg.src_hi, dbg.status);
         const float *src = src_base + (int64_t)c * ld_src;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
@@ -240,7 +244,7 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
             const int idx = col0 + lane + v * G;
             if (idx >= d4) continue;
             float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (self_src) fma4(a, du, ld4(self_src + (int64_t)halo_slot[j] * ld_src + 4 * idx));
+            if (self_src) fma4(a, du, ld4(self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * idx));
             for (int g = 0; g < NG; ++g) {
                 const float4 x = red[g][lane + v * G];
                 a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
@@ -255,11 +259,11 @@ __global__ void __launch_bounds__(256)
 k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
             const float *__restrict__ hrow_w, const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
             int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
-            float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong)
+            float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong, DbgLimits dbg)
 {
     if ((int32_t)blockIdx.x < n_hlong) {
-        hrow_long_block<G, NV>(hlong[hlong0 + blockIdx.x], hrow_ptr, hrow_pos, hrow_slot, hrow_w, halo_slot, dinv_enc, n, by_slot, d4, src_base, ld_src,
-                               self_src, out_base, ld_out);
+        hrow_long_block<G, NV>(SAT_IDX((int64_t)hlong[hlong0 + blockIdx.x], dbg.halo_lo, dbg.halo_hi, dbg.status), hrow_ptr, hrow_pos, hrow_slot, hrow_w, halo_slot,
+                               dinv_enc, n, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out, dbg);
         return;
     }
     const int lane = threadIdx.x & (G - 1);
@@ -272,7 +276,7 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     if (self_src) {
-        const float *src = self_src + (int64_t)halo_slot[j] * ld_src;
+        const float *src = self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int idx = col0 + lane + v * G;
@@ -291,7 +295,7 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             const bool ok = e + u < e1;
-            c[u] = ok ? __ldg(ecol + e + u) : -1;
+            c[u] = ok ? (int32_t)SAT_IDX(__ldg(ecol + e + u), dbg.src_lo, dbg.src_hi, dbg.status) : -1;
             w[u] = ok ? __ldg(hrow_w + e + u) : 0.f;
         }
 #pragma unroll
@@ -321,7 +325,8 @@ static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4
     dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hlong), (unsigned)cdiv64(d4, G * NV));
     k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->hrow_w, ctx->halo_slot, ctx->dinv_enc, ctx->n,
                                                        v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out,
-                                                       ctx->hlong, (int32_t)v.hlong0, (int32_t)v.n_hlong);
+                                                       ctx->hlong, (int32_t)v.hlong0, (int32_t)v.n_hlong,
+                                                       dbg_limits(by_slot ? DbgRange{0, ctx->n_slots} : DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo}, DbgRange{v.halo0, v.halo0 + v.n_halo}, ctx->d_flag + 1));
 }
 
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src, int by_slot,
@@ -351,59 +356,61 @@ sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float
 // row gather / scatter (pull of raw features, push into the cache, identity predictor)
 // -------------------------------------------------------------------------------------
 __global__ void k_gather_rows(const int32_t *__restrict__ idx, int64_t count, int32_t d4, const float *__restrict__ src, int64_t ld_src,
-                              float *__restrict__ out, int64_t ld_out)
+                              float *__restrict__ out, int64_t ld_out, DbgLimits dbg)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / d4;
     const int c = (int)(t - i * d4);
     if (i >= count) return;
-    const float4 x = ld4(src + (int64_t)idx[i] * ld_src + 4 * c);
+    const float4 x = ld4(src + SAT_IDX((int64_t)idx[i], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * c);
     *reinterpret_cast<float4 *>(out + i * ld_out + 4 * c) = x;
 }
 
 sat_status sat_gather(sat_ctx *ctx, const int32_t *idx, int64_t count, int32_t d, const float *src, int32_t ld_src, float *out,
-                      int32_t ld_out)
+                      int32_t ld_out, DbgRange src_rows)
 {
     if (count == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
     ProfScope prof(ctx, SATK_GATHER, (8.0 * d + 4.0) * (double)count, 0.0);
-    k_gather_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(idx, count, d4, src, ld_src, out, ld_out);
+    k_gather_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(idx, count, d4, src, ld_src, out, ld_out,
+                                                                              dbg_limits(src_rows, DbgRange{0, 0}, DbgRange{0, count}, ctx->d_flag + 1));
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
 
 __global__ void k_scatter_rows(const int32_t *__restrict__ src_row, const int32_t *__restrict__ dst_row, int64_t count, int32_t d4,
-                               const float *__restrict__ src_base, int64_t ld_src, float *__restrict__ dst, int64_t ld_dst)
+                               const float *__restrict__ src_base, int64_t ld_src, float *__restrict__ dst, int64_t ld_dst, DbgLimits dbg)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / d4;
     const int c = (int)(t - i * d4);
     if (i >= count) return;
-    const float4 x = ld4(src_base + (int64_t)src_row[i] * ld_src + 4 * c);
-    *reinterpret_cast<float4 *>(dst + (int64_t)dst_row[i] * ld_dst + 4 * c) = x;
+    const float4 x = ld4(src_base + SAT_IDX((int64_t)src_row[i], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * c);
+    *reinterpret_cast<float4 *>(dst + SAT_IDX((int64_t)dst_row[i], dbg.out_lo, dbg.out_hi, dbg.status) * ld_dst + 4 * c) = x;
 }
 
 sat_status sat_scatter(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
-                       int32_t ld_src, float *dst, int32_t ld_dst)
+                       int32_t ld_src, float *dst, int32_t ld_dst, DbgRange src_rows, DbgRange dst_rows)
 {
     if (count == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
     ProfScope prof(ctx, SATK_SCATTER, (8.0 * d + 8.0) * (double)count, 0.0);
-    k_scatter_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(src_row, dst_row, count, d4, src_base, ld_src, dst, ld_dst);
+    k_scatter_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(src_row, dst_row, count, d4, src_base, ld_src, dst, ld_dst,
+                                                                               dbg_limits(src_rows, DbgRange{0, 0}, dst_rows, ctx->d_flag + 1));
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
 
 __global__ void k_scatter_add_rows(const int32_t *__restrict__ src_row, const int32_t *__restrict__ dst_row, int64_t count, int32_t d4,
                                    const float *__restrict__ src_base, int64_t ld_src, float *__restrict__ dst, int64_t ld_dst,
-                                   const uint32_t *__restrict__ mask, int32_t mask_words)
+                                   const uint32_t *__restrict__ mask, int32_t mask_words, DbgLimits dbg)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t i = t / d4;
     const int c = (int)(t - i * d4);
     if (i >= count) return;
-    float4 x = ld4(src_base + (src_row ? (int64_t)src_row[i] : i) * ld_src + 4 * c);
-    const int64_t r = dst_row[i];
+    float4 x = ld4(src_base + (src_row ? SAT_IDX((int64_t)src_row[i], dbg.src_lo, dbg.src_hi, dbg.status) : i) * ld_src + 4 * c);
+    const int64_t r = SAT_IDX((int64_t)dst_row[i], dbg.out_lo, dbg.out_hi, dbg.status);
     if (mask) mask4(x, mask, r * mask_words, c);
     float4 *o = reinterpret_cast<float4 *>(dst + r * ld_dst + 4 * c);
     float4 y = *o;
@@ -415,13 +422,13 @@ __global__ void k_scatter_add_rows(const int32_t *__restrict__ src_row, const in
 }
 
 sat_status sat_scatter_add(sat_ctx *ctx, const int32_t *src_row, const int32_t *dst_row, int64_t count, int32_t d, const float *src_base,
-                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words)
+                           int32_t ld_src, float *dst, int32_t ld_dst, const uint32_t *mask, int32_t mask_words, DbgRange src_rows, DbgRange dst_rows)
 {
     if (count == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
     ProfScope prof(ctx, SATK_SCATTER, (12.0 * d + 8.0) * (double)count, 0.0);
     k_scatter_add_rows<<<(unsigned)cdiv64(count * d4, 256), 256, 0, ctx->stream>>>(src_row, dst_row, count, d4, src_base, ld_src, dst, ld_dst, mask,
-                                                                                   mask_words);
+                                                                                   mask_words, dbg_limits(src_rows, DbgRange{0, 0}, dst_rows, ctx->d_flag + 1));
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
@@ -487,7 +494,8 @@ static sat_status build_halo_by_slot(sat_ctx *ctx)
 
 __global__ void __launch_bounds__(256)
 k_sum_by_slot(const int64_t *__restrict__ hs_ptr, const int32_t *__restrict__ hs_pos, int32_t n_slots, const float *__restrict__ dinv_enc,
-              int32_t n, int32_t d4, const float *__restrict__ src, int64_t ld_src, int self_scale, int add, float *__restrict__ out, int64_t ld_out)
+              int32_t n, int32_t d4, const float *__restrict__ src, int64_t ld_src, int self_scale, int add, float *__restrict__ out, int64_t ld_out,
+              DbgLimits dbg)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t s = t / d4;
@@ -496,7 +504,7 @@ k_sum_by_slot(const int64_t *__restrict__ hs_ptr, const int32_t *__restrict__ hs
     const int64_t b = hs_ptr[s], e = hs_ptr[s + 1];
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int64_t i = b; i < e; ++i) {
-        const float4 x = ld4(src + (int64_t)__ldg(hs_pos + i) * ld_src + 4 * c);
+        const float4 x = ld4(src + SAT_IDX((int64_t)__ldg(hs_pos + i), dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * c);
         acc.x += x.x;
         acc.y += x.y;
         acc.z += x.z;
@@ -528,7 +536,8 @@ sat_status sat_sum_by_slot(sat_ctx *ctx, int32_t d, const float *src, int32_t ld
     const int32_t d4 = (d + 3) / 4;
     ProfScope prof(ctx, SATK_SCATTER, 8.0 * (double)ctx->nb + 4.0 * d * ((double)ctx->nb + (add ? 2.0 : 1.0) * ctx->n_slots), 0.0);
     k_sum_by_slot<<<(unsigned)cdiv64((int64_t)ctx->n_slots * d4, 256), 256, 0, ctx->stream>>>(ctx->hs_ptr, ctx->hs_pos, ctx->n_slots, ctx->dinv_enc,
-                                                                                              ctx->n, d4, src, ld_src, self_scale, add, out, ld_out);
+                                                                                              ctx->n, d4, src, ld_src, self_scale, add, out, ld_out,
+                                                                                              dbg_limits(DbgRange{0, ctx->nb}, DbgRange{0, 0}, DbgRange{0, ctx->n_slots}, ctx->d_flag + 1));
     SAT_LAUNCHED(ctx);
     return SAT_OK;
 }
