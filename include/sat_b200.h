@@ -59,6 +59,11 @@ enum { SAT_ACT_NONE = 0, SAT_ACT_RELU = 1 };
  * does afterwards (Algorithm 1 "Push"), from the epilogue of the layer transform instead of a second pass over h_out.
  * Needs sat_cache_init with that layer cached at width d_out (SAT_ESTATE / SAT_EINVAL otherwise). */
 #define SAT_FWD_PUSH 0x100
+/* Flag for the `act` argument of sat_layer_fwd: h_halo is not the [b_m x ld_halo] matrix of the partition's halo rows but a
+ * matrix over ALL n nodes in global id order ([n x ld_halo], e.g. the raw feature matrix for layer 1, whose out-of-subgraph
+ * rows are exact and need no cache: Eq. "mini-batch" with h^(0) = x); the layer reads the halo nodes' rows from it directly,
+ * which saves the sat_gather_rows pull and its [sum_m b_m x d] copy.  Same result, bit for bit, as the gathered call. */
+#define SAT_FWD_HALO_GLOBAL 0x200
 enum { SAT_LOSS_SOFTMAX_CE = 0, SAT_LOSS_SIGMOID_BCE = 1 };
 enum { SAT_ROWS_INNER = 0, SAT_ROWS_HALO = 1 };          /* sat_gather_rows                      */
 enum { SAT_CACHE_ZERO = 0, SAT_CACHE_COPY = 1 };         /* sat_cache_init                       */

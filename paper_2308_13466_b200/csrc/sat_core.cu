@@ -120,6 +120,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->hs_pos);
     dev_free(&ctx->lrowptr);
     dev_free(&ctx->lenc);
+    dev_free(&ctx->lenc_gid);
     dev_free(&ctx->inner_cnt);
     dev_free(&ctx->dinv_enc);
     dev_free(&ctx->lw);
@@ -128,6 +129,9 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->hrow_slot);
     dev_free(&ctx->hrow_w);
     dev_free(&ctx->hlong);
+    dev_free(&ctx->hchunk_first);
+    dev_free(&ctx->hchunk_row);
+    ctx->n_hchunks = 0;
     dev_free(&ctx->first_item);
     dev_free(&ctx->item_row);
     dev_free(&ctx->item_mslot);
@@ -181,6 +185,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     dev_free(&ctx->col);
     dev_free(&ctx->dinv);
     sat_free_buf(ctx->buf_partial);
+    sat_free_buf(ctx->buf_hpartial);
     sat_free_buf(ctx->buf_gagg);
     sat_free_buf(ctx->buf_splitk);
     sat_free_buf(ctx->buf_lstm_c);
@@ -817,6 +822,23 @@ __global__ void k_hlong_fill(const int32_t *__restrict__ flag, const int64_t *__
     if (j < nb && flag[j]) out[off[j]] = (int32_t)j;
 }
 
+// chunks of the long halo rows
+__global__ void k_hchunk_count(const int32_t *__restrict__ hlong, const int64_t *__restrict__ hrow_ptr, int32_t n_hlong, int32_t *__restrict__ nch)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_hlong) {
+        const int64_t j = hlong[i];
+        nch[i] = (int32_t)((hrow_ptr[j + 1] - hrow_ptr[j] + SAT_HROW_CHUNK - 1) / SAT_HROW_CHUNK);
+    }
+}
+
+__global__ void k_hchunk_fill(const int64_t *__restrict__ first, int32_t n_hlong, int32_t *__restrict__ chunk_row)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_hlong)
+        for (int64_t c = first[i]; c < first[i + 1]; ++c) chunk_row[c] = (int32_t)i;
+}
+
 __global__ void k_chunks(const int64_t *__restrict__ lrowptr, int32_t n, int32_t *__restrict__ nch)
 {
     int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -1143,6 +1165,35 @@ extern "C" sat_status sat_partition(sat_ctx *ctx, int32_t M, int method, const i
         dev_free(&t_ho);
         if (e != cudaSuccess) P_TRY(sat_check_cuda(ctx, e, "long halo rows"));
         P_TRY(rc);
+        // ... and are cut into chunks of SAT_HROW_CHUNK entries
+        ctx->h_hchunk_off.assign(M + 1, 0);
+        ctx->n_hchunks = 0;
+        if (ctx->n_hlong > 0) {
+            int32_t *t_nch = nullptr;
+            P_TRY(dev_alloc(ctx, &t_nch, ctx->n_hlong + 1));
+            rc = dev_alloc(ctx, &ctx->hchunk_first, (int64_t)ctx->n_hlong + 2);
+            if (rc == SAT_OK) {
+                k_hchunk_count<<<GRID1(ctx->n_hlong)>>>(ctx->hlong, ctx->hrow_ptr, ctx->n_hlong, t_nch);
+                ctx->launches++;
+                rc = sat_scan_i32(ctx, t_nch, ctx->n_hlong, ctx->hchunk_first);
+            }
+            std::vector<int64_t> off_c((size_t)M + 1, 0);
+            for (int m = 0; m <= M && rc == SAT_OK; ++m) rc = copy_i64(ctx, ctx->hchunk_first + ctx->h_hlong_off[m], &off_c[m]);
+            e = cudaStreamSynchronize(st);
+            if (rc == SAT_OK && e == cudaSuccess) {
+                for (int m = 0; m <= M; ++m) ctx->h_hchunk_off[m] = (int32_t)off_c[m];
+                ctx->n_hchunks = (int32_t)off_c[M];
+                rc = dev_alloc(ctx, &ctx->hchunk_row, ctx->n_hchunks);
+            }
+            if (rc == SAT_OK && e == cudaSuccess) {
+                k_hchunk_fill<<<GRID1(ctx->n_hlong)>>>(ctx->hchunk_first, ctx->n_hlong, ctx->hchunk_row);
+                ctx->launches++;
+                e = cudaStreamSynchronize(st);
+            }
+            dev_free(&t_nch);
+            if (e != cudaSuccess) P_TRY(sat_check_cuda(ctx, e, "chunks of the long halo rows"));
+            P_TRY(rc);
+        }
     }
 
     // ---- SpMM work items ----
@@ -1225,6 +1276,8 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v)
     v->hnnz = ctx->h_hrow_off.empty() ? 0 : ctx->h_hrow_off[b] - ctx->h_hrow_off[a];
     v->hlong0 = ctx->h_hlong_off[a];
     v->n_hlong = ctx->h_hlong_off[b] - v->hlong0;
+    v->hchunk0 = ctx->h_hchunk_off.empty() ? 0 : ctx->h_hchunk_off[a];
+    v->n_hchunks = ctx->h_hchunk_off.empty() ? 0 : ctx->h_hchunk_off[b] - v->hchunk0;
     return SAT_OK;
 }
 

@@ -16,7 +16,8 @@
 #define SAT_MAX_LAYERS 16
 #define SAT_MAX_PARTS 4096
 #define SAT_SPMM_CHUNK 256 /* edges per SpMM work item */
-#define SAT_HROW_LONG 256  /* halo rows with more entries than this get a whole thread block */
+#define SAT_HROW_LONG 256  /* halo rows with more entries than this are cut into chunks, a thread block per chunk */
+#define SAT_HROW_CHUNK 2048 /* entries per chunk of a long halo row */
 
 // Debug build (-DSAT_DEBUG_BOUNDS, libsat_b200_dbg.so): every index the graph kernels load from an index array (column ids,
 // row lists, cache slots) is checked against the extent of the matrix it addresses; an index outside it raises bit 4 of
@@ -153,6 +154,7 @@ struct sat_ctx {
     int32_t *row_slot = nullptr;  // [n] cache slot of every partition-major row, -1 for interior nodes (built on first use)
     int64_t *lrowptr = nullptr;   // [n+1] local CSR, rows partition-major
     int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
+    int32_t *lenc_gid = nullptr;  // [nnz+n] the same with halo columns as n + global node id (built on first use: SAT_FWD_HALO_GLOBAL)
     int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
     float *dinv_enc = nullptr;    // [n + nb] dinv of the node behind each encoded column
     float *lw = nullptr;          // [nnz+n] dinv_enc[lenc[e]] stored per entry (read with the column instead of gathered)
@@ -166,6 +168,11 @@ struct sat_ctx {
     int32_t *hlong = nullptr;     // [n_hlong] halo positions of the halo rows longer than SAT_HROW_LONG
     int32_t n_hlong = 0;
     std::vector<int32_t> h_hlong_off;
+    // the long halo rows cut into chunks of SAT_HROW_CHUNK entries (a hub next to most of a partition has tens of thousands)
+    int64_t *hchunk_first = nullptr; // [n_hlong+1] first chunk of every long row
+    int32_t *hchunk_row = nullptr;   // [n_hchunks] index into hlong[] of the row a chunk belongs to
+    int32_t n_hchunks = 0;
+    std::vector<int32_t> h_hchunk_off;  // [M+1] first chunk of every partition
     // SpMM work items (rows cut into chunks of SAT_SPMM_CHUNK edges)
     int32_t *first_item = nullptr; // [n+1]
     int32_t *item_row = nullptr;   // [n_items]
@@ -187,6 +194,7 @@ struct sat_ctx {
 
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
+    DevBuf buf_hpartial;
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
         buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out, buf_gat, buf_gat_items;
 };
@@ -296,6 +304,7 @@ struct PartView {
     int32_t mitem0, n_mitems; // partial-sum rows
     int32_t push0, n_push;
     int32_t hlong0, n_hlong;  // long halo rows
+    int32_t hchunk0, n_hchunks; // their chunks
     int64_t lnnz;             // local non-zeros (entries of A + I) of the selected rows
     int64_t hnnz;             // of which entries with a halo column (= entries of the halo-row CSR)
 };
@@ -307,9 +316,10 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
 //   partition-major inner matrix and of the concatenated halo matrix (already offset for a single
 //   partition); `out_base` likewise.
 // omask (or null): bit mask [rows x omask_words] indexed like out_base; output components whose bit is 0 are written as 0
+// halo_global: the halo columns address a matrix over all n nodes in global id order (halo_base = its first row)
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
                     const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask = nullptr,
-                    int32_t omask_words = 0);
+                    int32_t omask_words = 0, bool halo_global = false);
 //   halo-row products: out[j] = sum_{e in hrow(j)} dinv[halo j] dinv[inner e] * src[pos_e]   (+ self term if self_src)
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src,
                          int by_slot, const float *self_src, float *out_base, int32_t ld_out);

@@ -327,42 +327,52 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
         SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, newest), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
         c->proj_tag[newest] = p->version;
     }
-    for (int32_t t = 0; t < k; ++t) {
-        const int32_t idx = ring_index(ctx, k - 1 - t);  // oldest first
-        const bool cached = c->proj_tag[idx] == p->version;
-        const float *pr = c->proj + (int64_t)idx * plane;
-        TcEpilogueHost eh;
-        eh.C = c->S;
-        eh.ldc = h;
-        eh.lstm_h = h;
-        eh.lstm_c = cell;
-        if (cached && t == 0) {
-            ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 6.0, 0.0);
-            k_lstm_cell_first<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(pr, rows, h, cell, c->S);
-            SAT_LAUNCHED(ctx);
-        } else if (cached) {
-            if (!have_up) {
-                if (c->tag_uh == p->version) {
-                    SAT_TRY(sat_tc_weights_layout(h, 4 * h, c->pk_uh, &Up));
-                } else {
-                    SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, c->pk_uh, &Up, h));
-                    c->tag_uh = p->version;
+    // The recurrence is row-wise: a block of rows can run all of its steps before the next block starts.  With blocks small
+    // enough for their state (s and c) to stay in L2 between two steps, only the cached projections stream from HBM.
+    const char *chunk_env = getenv("SAT_LSTM_CHUNK");
+    const int64_t chunk = chunk_env ? (atoll(chunk_env) + 127) / 128 * 128 : 0;   // rows per block (multiple of the row tile); 0: all rows at once
+    for (int64_t r0 = 0; r0 < rows; r0 += (chunk > 0 ? chunk : rows)) {
+        const int64_t cnt = chunk > 0 && r0 + chunk < rows ? chunk : rows - r0;
+        float *S_blk = c->S + r0 * h;
+        float *cell_blk = cell + sat_cell_offset(r0, 0, h);
+        for (int32_t t = 0; t < k; ++t) {
+            const int32_t idx = ring_index(ctx, k - 1 - t);  // oldest first
+            const bool cached = c->proj_tag[idx] == p->version;
+            const float *pr = c->proj + (int64_t)idx * plane + r0 * 4 * h;
+            const float *x_blk = ring_buf(ctx, c, idx) + r0 * c->ld;
+            TcEpilogueHost eh;
+            eh.C = S_blk;
+            eh.ldc = h;
+            eh.lstm_h = h;
+            eh.lstm_c = cell_blk;
+            if (cached && t == 0) {
+                ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)cnt * h * 6.0, 0.0);
+                k_lstm_cell_first<<<(unsigned)cdiv64(cnt * h, 256), 256, 0, ctx->stream>>>(pr, cnt, h, cell_blk, S_blk);
+                SAT_LAUNCHED(ctx);
+            } else if (cached) {
+                if (!have_up) {
+                    if (c->tag_uh == p->version) {
+                        SAT_TRY(sat_tc_weights_layout(h, 4 * h, c->pk_uh, &Up));
+                    } else {
+                        SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, c->pk_uh, &Up, h));
+                        c->tag_uh = p->version;
+                    }
                 }
+                have_up = true;
+                eh.addend = pr;
+                eh.ld_addend = 4 * h;
+                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, S_blk, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
+            } else if (t == 0) {
+                SAT_TRY(pack_wx());
+                eh.bias = p->b;
+                eh.lstm_first = 1;
+                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, x_blk, c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+            } else {
+                if (!have_wxu) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit3, &Wxu, h));
+                have_wxu = true;
+                eh.bias = p->b;
+                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, x_blk, c->ld, d, S_blk, h, h, Wxu, eh, SATK_GEMM_NN));
             }
-            have_up = true;
-            eh.addend = pr;
-            eh.ld_addend = 4 * h;
-            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
-        } else if (t == 0) {
-            SAT_TRY(pack_wx());
-            eh.bias = p->b;
-            eh.lstm_first = 1;
-            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
-        } else {
-            if (!have_wxu) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit3, &Wxu, h));
-            have_wxu = true;
-            eh.bias = p->b;
-            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, c->S, h, h, Wxu, eh, SATK_GEMM_NN));
         }
     }
     c->S_valid = true;
@@ -623,7 +633,8 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     SAT_TRY(sat_part_view(ctx, part, &v));
     if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
     const bool push = (act & SAT_FWD_PUSH) != 0;
-    act &= ~SAT_FWD_PUSH;
+    const bool halo_global = (act & SAT_FWD_HALO_GLOBAL) != 0;
+    act &= ~(SAT_FWD_PUSH | SAT_FWD_HALO_GLOBAL);
     if (d_in <= 0 || d_out <= 0 || !W || (act != SAT_ACT_NONE && act != SAT_ACT_RELU)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: bad dims / W / act");
     CacheLayer *pc = nullptr;
     if (push) {
@@ -648,8 +659,9 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     L.act = act;
     if (v.n_rows == 0) return SAT_OK;
     const float *in_base = h_in - (int64_t)v.row0 * ld_in;
-    const float *halo_base = h_halo ? h_halo - v.halo0 * (int64_t)ld_halo : nullptr;
-    SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg));
+    // the halo source is the concatenated halo matrix (addressed from its virtual first row) or a matrix over all nodes
+    const float *halo_base = !h_halo ? nullptr : halo_global ? h_halo : h_halo - v.halo0 * (int64_t)ld_halo;
+    SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg, nullptr, 0, halo_global));
     uint32_t *mask_out = act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * words : nullptr;
     const float *agg = L.agg + (int64_t)v.row0 * ld_agg;
     if (sat_use_tc(d_out, d_in)) {

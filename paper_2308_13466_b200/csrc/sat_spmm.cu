@@ -139,22 +139,48 @@ __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, i
 template <int G, int NV>
 static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d4, const float *in_base, int32_t ld_in,
                          const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial, const uint32_t *omask,
-                         int32_t omask_words)
+                         int32_t omask_words, const int32_t *cols, DbgRange halo_range)
 {
     dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
-    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, ctx->lenc, ctx->lw, ctx->dinv_enc, ctx->item_row,
+    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, cols, ctx->lw, ctx->dinv_enc, ctx->item_row,
                                                         ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
                                                         ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words,
-                                                        dbg_limits(DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo}, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
+                                                        dbg_limits(DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, halo_range,
+                                                                  DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
+}
+
+// halo columns as global node ids (for a halo source that is a matrix over all nodes)
+__global__ void k_cols_by_gid(const int32_t *__restrict__ lenc, const int32_t *__restrict__ halo_gid, int64_t count, int32_t n,
+                              int32_t *__restrict__ out)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    const int32_t c = lenc[e];
+    out[e] = c < n ? c : n + halo_gid[c - n];
 }
 
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
-                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask, int32_t omask_words)
+                    const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask, int32_t omask_words,
+                    bool halo_global)
 {
     if (v.n_items == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
-    // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once
-    const double n_src = inner_only == 1 ? (double)v.n_rows : inner_only == 2 ? (double)v.n_halo : (double)v.n_rows + (double)v.n_halo;
+    const int32_t *cols = ctx->lenc;
+    DbgRange halo_range{v.halo0, v.halo0 + v.n_halo};
+    if (halo_global) {
+        if (!ctx->lenc_gid) {
+            const int64_t lnnz = ctx->nnz + ctx->n;
+            SAT_CUDA(ctx, cudaMalloc((void **)&ctx->lenc_gid, (size_t)lnnz * sizeof(int32_t)));
+            k_cols_by_gid<<<(unsigned)cdiv64(lnnz, 256), 256, 0, ctx->stream>>>(ctx->lenc, ctx->halo_gid, lnnz, ctx->n, ctx->lenc_gid);
+            SAT_LAUNCHED(ctx);
+        }
+        cols = ctx->lenc_gid;
+        halo_range = DbgRange{0, ctx->n};
+    }
+    // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once (a halo source over
+    // all nodes holds at most n distinct rows)
+    const double n_halo_src = halo_global && v.n_halo > ctx->n ? (double)ctx->n : (double)v.n_halo;
+    const double n_src = inner_only == 1 ? (double)v.n_rows : inner_only == 2 ? n_halo_src : (double)v.n_rows + n_halo_src;
     // the backward reads the inner prefix of every row, the transposed predictor convolution the halo suffix
     const double n_ent = (double)(inner_only == 1 ? v.lnnz - v.hnnz : inner_only == 2 ? v.hnnz : v.lnnz);
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
@@ -164,7 +190,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
         SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * d4 * 16));
         partial = (float *)ctx->buf_partial.p;
     }
-#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words
+#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words, cols, halo_range
     // experiment switch: SAT_SPMM_CFG = 100 * lanes + vectors per lane selects the lane-group shape (column slices run as grid.y)
     const char *cfg_env = getenv("SAT_SPMM_CFG");
     const int cfg = cfg_env ? atoi(cfg_env) : 0;
@@ -205,26 +231,29 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
 // Used for the predictor's graph convolution on the LSTM state (self term, by slot) and for
 // the optional halo gradient P_out^T G_AGG (no self term, by row).
 // -------------------------------------------------------------------------------------
-// One thread block per long halo row (the first blocks of the grid, so that they start first and the short rows fill the
-// other SMs meanwhile): the 256 / G lane groups take the entries round-robin, their partial sums are added
-// in group order through shared memory (fixed order: reproducible), group 0 adds the self term and stores.
+// One thread block per chunk of SAT_HROW_CHUNK entries of a long halo row (the first blocks of the grid, so that they start
+// first and the short rows fill the other SMs meanwhile): the 256 / G lane groups take the chunk's entries round-robin, their
+// partial sums are added in group order through shared memory (fixed order: reproducible) and written, un-scaled and
+// without the self term, to the chunk's row of `partial`; k_hrow_long_fixup adds the chunks of a row in chunk order.
 template <int G, int NV>
-__device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos,
-                                                const int32_t *__restrict__ hrow_slot, const float *__restrict__ hrow_w,
-                                                const int32_t *__restrict__ halo_slot,
-                                                const float *__restrict__ dinv_enc, int32_t n, int by_slot, int32_t d4,
-                                                const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
-                                                float *__restrict__ out_base, int64_t ld_out, const DbgLimits &dbg)
+__device__ __forceinline__ void hrow_chunk_block(int32_t chunk, const int32_t *__restrict__ hlong, const int64_t *__restrict__ hchunk_first,
+                                                 const int32_t *__restrict__ hchunk_row, int32_t hchunk0, const int64_t *__restrict__ hrow_ptr,
+                                                 const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
+                                                 const float *__restrict__ hrow_w, int by_slot, int32_t d4, const float *__restrict__ src_base,
+                                                 int64_t ld_src, float *__restrict__ partial, const DbgLimits &dbg)
 {
     constexpr int NG = 256 / G;
     __shared__ float4 red[NG][G * NV];
     const int lane = threadIdx.x & (G - 1), grp = threadIdx.x / G;
     const int col0 = blockIdx.y * (G * NV);
-    const float du = __ldg(dinv_enc + n + j);
+    const int32_t li = hchunk_row[chunk];
+    const int64_t j = SAT_IDX((int64_t)hlong[li], dbg.halo_lo, dbg.halo_hi, dbg.status);
+    const int64_t k = chunk - hchunk_first[li];
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+    const int64_t e0 = hrow_ptr[j] + k * SAT_HROW_CHUNK;
+    const int64_t e1 = e0 + SAT_HROW_CHUNK < hrow_ptr[j + 1] ? e0 + SAT_HROW_CHUNK : hrow_ptr[j + 1];
     for (int64_t e = e0 + grp; e < e1; e += NG) {
         const float w = __ldg(hrow_w + e);
         const int32_t c = (int32_t)SAT_IDX(by_slot ? __ldg(hrow_slot + e) : __ldg(hrow_pos + e), dbg.src_lo, dbg.src_hi, dbg.status);
@@ -239,19 +268,40 @@ __device__ __forceinline__ void hrow_long_block(int64_t j, const int64_t *__rest
     for (int v = 0; v < NV; ++v) red[grp][lane + v * G] = acc[v];
     __syncthreads();
     if (grp == 0) {
+        float *o = partial + (int64_t)(chunk - hchunk0) * (4 * (int64_t)d4);
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int idx = col0 + lane + v * G;
             if (idx >= d4) continue;
             float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (self_src) fma4(a, du, ld4(self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * idx));
             for (int g = 0; g < NG; ++g) {
                 const float4 x = red[g][lane + v * G];
                 a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
             }
-            *reinterpret_cast<float4 *>(out_base + j * ld_out + 4 * idx) = make_float4(du * a.x, du * a.y, du * a.z, du * a.w);
+            *reinterpret_cast<float4 *>(o + 4 * idx) = a;
         }
     }
+}
+
+// long halo rows: out[j] = dinv[u_j] * ( [self] dinv[u_j] * self_src[halo_slot_j] + sum over the row's chunks, in chunk order )
+__global__ void k_hrow_long_fixup(const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong, const int64_t *__restrict__ hchunk_first,
+                                  int32_t hchunk0, const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n,
+                                  int32_t d4, const float *__restrict__ partial, const float *__restrict__ self_src, int64_t ld_src,
+                                  float *__restrict__ out_base, int64_t ld_out, DbgLimits dbg)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= n_hlong) return;
+    const int64_t j = SAT_IDX((int64_t)hlong[hlong0 + i], dbg.halo_lo, dbg.halo_hi, dbg.status);
+    const float du = __ldg(dinv_enc + n + j);
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (self_src) fma4(a, du, ld4(self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src + 4 * c));
+    for (int64_t q = hchunk_first[hlong0 + i]; q < hchunk_first[hlong0 + i + 1]; ++q) {
+        const float4 x = *reinterpret_cast<const float4 *>(partial + ((q - hchunk0) * d4 + c) * 4);
+        a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
+    }
+    *reinterpret_cast<float4 *>(out_base + j * ld_out + 4 * c) = make_float4(du * a.x, du * a.y, du * a.z, du * a.w);
 }
 
 template <int G, int NV>
@@ -259,15 +309,16 @@ __global__ void __launch_bounds__(256)
 k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hrow_pos, const int32_t *__restrict__ hrow_slot,
             const float *__restrict__ hrow_w, const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
             int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
-            float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, int32_t hlong0, int32_t n_hlong, DbgLimits dbg)
+            float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, const int64_t *__restrict__ hchunk_first,
+            const int32_t *__restrict__ hchunk_row, int32_t hchunk0, int32_t n_hchunks, float *__restrict__ hpartial, DbgLimits dbg)
 {
-    if ((int32_t)blockIdx.x < n_hlong) {
-        hrow_long_block<G, NV>(SAT_IDX((int64_t)hlong[hlong0 + blockIdx.x], dbg.halo_lo, dbg.halo_hi, dbg.status), hrow_ptr, hrow_pos, hrow_slot, hrow_w, halo_slot,
-                               dinv_enc, n, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out, dbg);
+    if ((int32_t)blockIdx.x < n_hchunks) {
+        hrow_chunk_block<G, NV>(hchunk0 + (int32_t)blockIdx.x, hlong, hchunk_first, hchunk_row, hchunk0, hrow_ptr, hrow_pos, hrow_slot, hrow_w, by_slot,
+                                d4, src_base, ld_src, hpartial, dbg);
         return;
     }
     const int lane = threadIdx.x & (G - 1);
-    const int64_t gid = ((int64_t)(blockIdx.x - n_hlong) * blockDim.x + threadIdx.x) / G;
+    const int64_t gid = ((int64_t)(blockIdx.x - n_hchunks) * blockDim.x + threadIdx.x) / G;
     if (gid >= n_halo) return;
     const int col0 = blockIdx.y * (G * NV);
     const int64_t j = halo0 + gid;
@@ -284,7 +335,7 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
         }
     }
     const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
-    if (e1 - e0 > SAT_HROW_LONG) return;  // handled by a block of its own (hrow_long_block)
+    if (e1 - e0 > SAT_HROW_LONG) return;  // cut into chunks, a block each (hrow_chunk_block), combined by k_hrow_long_fixup
     // Halo rows are short (a handful of cut edges): every lane reads the entry's column and weight itself (one broadcast
     // transaction per group) instead of sharing them through shuffles, four entries in flight; entries in order, so the
     // sum has the same order as the long-row path's per-group partial sums.
@@ -320,12 +371,12 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
 
 template <int G, int NV>
 static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4, const float *src_base, int32_t ld_src,
-                        const float *self_src, float *out_base, int32_t ld_out)
+                        const float *self_src, float *out_base, int32_t ld_out, float *hpartial)
 {
-    dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hlong), (unsigned)cdiv64(d4, G * NV));
+    dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hchunks), (unsigned)cdiv64(d4, G * NV));
     k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->hrow_w, ctx->halo_slot, ctx->dinv_enc, ctx->n,
                                                        v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out,
-                                                       ctx->hlong, (int32_t)v.hlong0, (int32_t)v.n_hlong,
+                                                       ctx->hlong, ctx->hchunk_first, ctx->hchunk_row, v.hchunk0, v.n_hchunks, hpartial,
                                                        dbg_limits(by_slot ? DbgRange{0, ctx->n_slots} : DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo}, DbgRange{v.halo0, v.halo0 + v.n_halo}, ctx->d_flag + 1));
 }
 
@@ -339,7 +390,12 @@ sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float
     const double n_src = (double)v.n_push + (self_src ? (double)v.n_halo : 0.0);
     ProfScope prof(ctx, SATK_SPMM_HROW, 8.0 * (double)v.hnnz + 12.0 * (double)v.n_halo + 4.0 * d * (n_src + (double)v.n_halo),
                    2.0 * d * ((double)v.hnnz + (self_src ? (double)v.n_halo : 0.0)));
-#define ARGS ctx, v, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out
+    float *hpartial = nullptr;
+    if (v.n_hchunks > 0) {
+        SAT_TRY(sat_ensure(ctx, ctx->buf_hpartial, (size_t)v.n_hchunks * d4 * 16));
+        hpartial = (float *)ctx->buf_hpartial.p;
+    }
+#define ARGS ctx, v, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out, hpartial
     if (d4 <= 4) launch_hrow<4, 1>(ARGS);
     else if (d4 <= 8) launch_hrow<8, 1>(ARGS);
     else if (d4 <= 16) launch_hrow<16, 1>(ARGS);
@@ -349,6 +405,14 @@ sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float
     else launch_hrow<32, 8>(ARGS);
 #undef ARGS
     SAT_LAUNCHED(ctx);
+    if (v.n_hlong > 0) {
+        k_hrow_long_fixup<<<(unsigned)cdiv64((int64_t)v.n_hlong * d4, 256), 256, 0, ctx->stream>>>(
+            ctx->hlong, v.hlong0, v.n_hlong, ctx->hchunk_first, v.hchunk0, ctx->halo_slot, ctx->dinv_enc, ctx->n, d4, hpartial, self_src, ld_src,
+            out_base, ld_out,
+            dbg_limits(by_slot ? DbgRange{0, ctx->n_slots} : DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo},
+                       DbgRange{v.halo0, v.halo0 + v.n_halo}, ctx->d_flag + 1));
+        SAT_LAUNCHED(ctx);
+    }
     return SAT_OK;
 }
 
@@ -574,7 +638,7 @@ k_l2_stream(const float4 *__restrict__ buf, int64_t n_vec, int reps, float *__re
 
 template <int NV>
 __global__ void __launch_bounds__(256, NV <= 2 ? 8 : 4)
-k_l2_gather(const float *__restrict__ buf, int64_t n_rows, int32_t d4, int64_t n_items, int per_item, float *__restrict__ sink)
+k_l2_gather(const float *__restrict__ buf, uint32_t row_mask, int32_t d4, int64_t n_items, int per_item, float *__restrict__ sink)
 {
     const int lane = threadIdx.x & 31;
     const int64_t item = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -588,7 +652,7 @@ k_l2_gather(const float *__restrict__ buf, int64_t n_rows, int32_t d4, int64_t n
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             state = state * 6364136223846793005ull + 1442695040888963407ull;   // the same sequence in every lane of the warp
-            r[u] = (int64_t)((state >> 20) % (uint64_t)n_rows);
+            r[u] = (int64_t)((uint32_t)(state >> 24) & row_mask);   // the row count is a power of two
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
@@ -612,7 +676,8 @@ extern "C" sat_status sat_profile_l2_rates(sat_ctx *ctx, int32_t row_floats, dou
     if (row_floats < 4 || row_floats > 1024 || (row_floats & 3)) return sat_fail(ctx, SAT_EINVAL, "sat_profile_l2_rates: row width must be a multiple of 4 in [4, 1024]");
     const size_t bytes = (size_t)64 << 20;                        // well inside the 126 MB L2
     const int32_t d4 = row_floats / 4;
-    const int64_t n_rows = (int64_t)(bytes / ((size_t)row_floats * 4));
+    int64_t n_rows = 1;                                           // the largest power of two of rows that fits the buffer
+    while (2 * n_rows * (int64_t)row_floats * 4 <= (int64_t)bytes) n_rows *= 2;
     float *buf = nullptr, *sink = nullptr;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
     cudaError_t e = cudaMalloc((void **)&buf, bytes);
@@ -636,10 +701,10 @@ extern "C" sat_status sat_profile_l2_rates(sat_ctx *ctx, int32_t row_floats, dou
         for (int pass = 0; pass < 2 && e == cudaSuccess; ++pass) {
             cudaEventRecord(e0, ctx->stream);
             const unsigned grid = (unsigned)cdiv64(n_items * 32, 256);
-            if (d4 <= 32) k_l2_gather<1><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
-            else if (d4 <= 64) k_l2_gather<2><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
-            else if (d4 <= 128) k_l2_gather<4><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
-            else k_l2_gather<8><<<grid, 256, 0, ctx->stream>>>(buf, n_rows, d4, n_items, per_item, sink);
+            if (d4 <= 32) k_l2_gather<1><<<grid, 256, 0, ctx->stream>>>(buf, (uint32_t)(n_rows - 1), d4, n_items, per_item, sink);
+            else if (d4 <= 64) k_l2_gather<2><<<grid, 256, 0, ctx->stream>>>(buf, (uint32_t)(n_rows - 1), d4, n_items, per_item, sink);
+            else if (d4 <= 128) k_l2_gather<4><<<grid, 256, 0, ctx->stream>>>(buf, (uint32_t)(n_rows - 1), d4, n_items, per_item, sink);
+            else k_l2_gather<8><<<grid, 256, 0, ctx->stream>>>(buf, (uint32_t)(n_rows - 1), d4, n_items, per_item, sink);
             cudaEventRecord(e1, ctx->stream);
             ctx->launches++;
             e = cudaEventSynchronize(e1);

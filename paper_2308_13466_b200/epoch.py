@@ -49,7 +49,7 @@ class SatEpoch:
         dev = self.device
         self.H = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # H[l], l = 1..L (partition-major rows)
         self.G = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # gradient w.r.t. H[l]
-        self.halo = _buf(self.nb, max(self.dims[:-1]), dev)                       # halo input of the running layer
+        self.halo = _buf(self.nb, max(self.dims[1:-1] or [1]), dev)               # predicted halo input of the running layer (layers >= 2)
         self.X_in = _buf(self.n, self.dims[0], dev)
         self.gW = [torch.zeros((self.dims[l], self.dims[l + 1]), dtype=torch.float32, device=dev) for l in range(self.L)]
         self.gb = [torch.zeros(self.dims[l + 1], dtype=torch.float32, device=dev) for l in range(self.L)]
@@ -86,14 +86,18 @@ class SatEpoch:
         h_in = self.rows(self.X_in, m)
         for l in range(1, L + 1):
             d_in = self.dims[l - 1]
-            hv = self.halo_view(d_in, m)
+            act = (B.SAT_ACT_RELU | B.SAT_FWD_PUSH) if l < L else B.SAT_ACT_NONE
             if l == 1:
-                B.sat_gather_rows(ctx, m, B.SAT_ROWS_HALO, self.X, hv)                 # pull raw features
+                # pull of layer 1: the out-of-subgraph rows are raw features, exact; the layer reads them from the feature
+                # matrix itself (global id order) instead of a gathered copy
+                hv = self.X
+                act |= B.SAT_FWD_HALO_GLOBAL
             else:
+                hv = self.halo_view(d_in, m)
                 B.sat_predict(ctx, l - 1, m, pred[l - 2] if pred is not None else None, reuse_state, hv)  # pull predicted
             h_out = self.rows(self.H[l], m)
             # forward; for the cached layers the push of the boundary rows rides on the transform's epilogue
-            B.sat_layer_fwd(ctx, m, l, h_in, hv, W[l - 1], b[l - 1], (B.SAT_ACT_RELU | B.SAT_FWD_PUSH) if l < L else B.SAT_ACT_NONE, h_out)
+            B.sat_layer_fwd(ctx, m, l, h_in, hv, W[l - 1], b[l - 1], act, h_out)
             h_in = h_out
         kind = B.SAT_LOSS_SOFTMAX_CE if self.loss == "ce" else B.SAT_LOSS_SIGMOID_BCE
         g = self.rows(self.G[L], m)

@@ -360,6 +360,53 @@ def test_cache_init_from_a_given_snapshot(B):
         B.sat_destroy(ctx)
 
 
+@pytest.mark.parametrize("name,shrink", [("medium", 16), ("odd", 1)])
+def test_halo_rows_read_from_the_global_feature_matrix(B, name, shrink):
+    """SAT_FWD_HALO_GLOBAL: layer 1 with h_halo = the feature matrix over all nodes gives the bits of the call on the gathered
+    halo rows (same entries, same order, same values), per partition and for all partitions at once, and the backward that
+    follows is the same."""
+    import torch
+    wl = make_workload(name, shrink=shrink)
+    part = orc.contig_blocks(wl.n, wl.M)
+    P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
+    perm = np.concatenate(P.inner_gid)
+    halo_all = np.concatenate(P.halo_gid)
+    inner_off = np.concatenate([[0], np.cumsum([g.shape[0] for g in P.inner_gid])])
+    halo_off = np.concatenate([[0], np.cumsum([g.shape[0] for g in P.halo_gid])])
+    ctx = B.sat_create(0, 0)
+    try:
+        B.sat_graph_load(ctx, wl.rowptr, wl.col)
+        B.sat_partition(ctx, wl.M, B.SAT_PART_CONTIG_BLOCKS)
+        Xd = dev2d(wl.X)
+        h_in, h_halo = dev2d(wl.X[perm]), dev2d(wl.X[halo_all])
+        Wd, bd = dev(wl.W[0]), dev(wl.b[0])
+        d1 = wl.dims[1]
+        G = dev2d((np.random.default_rng(4).standard_normal((wl.n, d1)) / wl.n).astype(np.float32))
+        outs, grads = [], []
+        for mode in ("gathered", "global", "global-per-partition"):
+            h_out = empty2d(wl.n, d1)
+            if mode == "gathered":
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, h_halo, Wd, bd, B.SAT_ACT_RELU, h_out)
+            elif mode == "global":
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, Xd, Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_HALO_GLOBAL, h_out)
+            else:
+                for m in range(P.M):
+                    r0, r1 = inner_off[m], inner_off[m + 1]
+                    B.sat_layer_fwd(ctx, m, 1, h_in[r0:r1], Xd, Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_HALO_GLOBAL, h_out[r0:r1])
+            gW = torch.full_like(Wd, float("nan"))
+            gb = torch.full_like(bd, float("nan"))
+            B.sat_layer_bwd(ctx, B.SAT_ALL_PARTS, 1, G, Wd, gW, gb, 0, None, None)
+            torch.cuda.synchronize()
+            outs.append(h_out.cpu().numpy().copy())
+            grads.append(gW.cpu().numpy().copy())
+        assert np.abs(outs[0]).max() > 0
+        for o, g in zip(outs[1:], grads[1:]):
+            assert np.array_equal(o, outs[0]) and np.array_equal(g, grads[0])
+        B.sat_sync_status(ctx)
+    finally:
+        B.sat_destroy(ctx)
+
+
 def test_parameter_step_on_many_arrays(B):
     """sat_sgd_steps on a list of arrays (more than one launch's worth, one of them empty) equals sat_sgd_step array by array."""
     import torch
