@@ -225,6 +225,52 @@ def whole_job_value(total_ms, steps, units_per_rank_step, world):
     return ms_per_step, world * units_per_rank_step / (ms_per_step * 1e-3)
 
 
+def side_workload(name: str, steps: int, peaks):
+    """A short device-resident run of another configuration (ring filled, `steps` timed epochs with the per-family events
+    on): epoch time, edges/s and the SpMM / whole-epoch fractions, for the side table of the JSON line."""
+    import torch
+    import paper_2308_13466_b200.binding as B
+    from paper_2308_13466_b200.epoch import SatEpoch
+    from sat_synth import make_workload
+    wl = make_workload(name)
+    dev = torch.device("cuda", torch.cuda.current_device())
+    up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss, part_given=wl.part_given, device=dev.index)
+    try:
+        perm = np.concatenate([B.sat_part_lists(ep.ctx, m)["inner_gid"] for m in range(wl.M)])
+        X = torch.zeros((wl.n, (wl.dims[0] + 3) & ~3), dtype=torch.float32, device=dev)[:, :wl.dims[0]]
+        X.copy_(torch.from_numpy(wl.X))
+        ep.set_inputs(X, up(wl.labels[perm]))
+        W, b = [up(w) for w in wl.W], [up(x) for x in wl.b]
+        preds = [B.make_pred_params(up(p["Wx"]), up(p["Uh"]), up(p["b"]), up(p["Wg"]), up(p["bg"]), int(p["h"]), 1) for p in wl.pred]
+        for _ in range(wl.tau + 3):
+            ep.step(W, b, preds, 0.01)
+        stream = torch.cuda.current_stream(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            ep.step(W, b, preds, 0.01)
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        B.sat_profile_enable(ep.ctx, True)
+        for _ in range(steps):
+            ep.step(W, b, preds, 0.01)
+        prof = B.sat_profile_read(ep.ctx)
+        B.sat_profile_enable(ep.ctx, False)
+        fam = {k: dict(ms_per_step=v["ms"] / steps, hbm_frac=v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm"])
+               for k, v in prof.items() if v["calls"] and v["ms"] > 0}
+        alg = sum(v["bytes"] for v in prof.values()) / steps
+        return dict(workload=workload_config(wl)["workload"], steps=steps, ms_per_step=ms, edges_per_s=wl.nnz / (ms * 1e-3),
+                    epoch_hbm_frac=alg / (ms * 1e-3) / 1e9 / peaks["hbm"],
+                    spmm_fwd=dict(ms_per_step=fam.get("spmm_fwd", {}).get("ms_per_step"), hbm_frac=fam.get("spmm_fwd", {}).get("hbm_frac"),
+                                  gather_gbs=(prof["spmm_fwd"]["flops"] / 2.0 * 4.0 / (prof["spmm_fwd"]["ms"] * 1e-3) / 1e9) if prof.get("spmm_fwd", {}).get("ms") else None),
+                    largest_families_ms={k: round(v["ms_per_step"], 3) for k, v in sorted(fam.items(), key=lambda kv: -kv[1]["ms_per_step"])[:5]},
+                    halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n)
+    finally:
+        ep.close()
+
+
 # ------------------------------------------------------------------------------------------
 def run_ours(args, wl):
     import torch
@@ -585,16 +631,29 @@ def run_ours(args, wl):
                      spmm_gather_gbs={k: (prof[k]["flops"] / 2.0 * 4.0) / (prof[k]["ms"] * 1e-3) / 1e9
                                       for k in ("spmm_fwd", "spmm_bwd", "spmm_hrow") if prof.get(k, {}).get("ms", 0) > 0},
                      l2_stream_gbs=l2_stream_gbs, l2_random_row_gbs=l2_gather_gbs, l2_row_floats=l2_row)
+        # the other configurations, briefly (device-resident epochs only; the headline above is the workload named in `config`)
+        others = {}
+        if world == 1 and args.others:
+            ep.close()
+            del X_dev, X_dev2, W, b, preds, in_bufs, w_bufs, hX
+            torch.cuda.empty_cache()
+            for name in [x for x in args.others.split(",") if x and x != wl.name]:
+                try:
+                    others[name] = side_workload(name, 5, peaks)
+                except Exception as exc:      # a side table must not cost the headline line
+                    others[name] = dict(error=f"{type(exc).__name__}: {exc}"[:300])
+                torch.cuda.empty_cache()
         line = dict(metric="SAT epoch edges/s (fwd+bwd+predictor, P partitions)", value=value, unit="edges/s", n_gpus=world,
                     steps=args.steps, warmup=args.warmup, ms_per_step=ms_per_step, higher_is_better=True, scaling="weak",
                     vs_baseline=None, dtype="f32", data="synthetic", config=workload_config(wl),
                     e2e=dict(value=e2e_value, unit="edges/s", h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h, steps=e2e_steps,
                              loss=e2e_loss, pipelined="inputs of step i+1 copied on a second stream while step i computes; the host reads the results of step i while step i+1 is queued"),
                     gpu_launches=int(launches), clocks=clocks, roofline=roofline, cpu_baseline=cpu, epoch=epoch, pred_update=pred_update, grad_history=grad_history, gat=gat, codec=codec, kernel_families=families,
-                    loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n,
+                    loss=loss, halo_rows=int(ep.nb), boundary_fraction=ep.n_slots / wl.n, other_workloads=others,
                     multi_gpu="replicas only" if world > 1 else None)
         print(json.dumps(line), flush=True)
-    ep.close()
+    if ep.ctx is not None:
+        ep.close()
     if dist is not None:
         dist.destroy_process_group()
 
@@ -621,6 +680,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--epochs-only", action="store_true",
                     help="skip the side measurements (predictor never updated / unversioned, predictor update)")
+    ap.add_argument("--others", default="medium,multilabel,tiny",
+                    help="comma-separated other configurations to run briefly for the side table of the line ('' = none; dense takes minutes to generate)")
     ap.add_argument("--extras", action="store_true",
                     help="also time the parts outside the epoch metric: gradient-side history, graph-attention backbone, embedding codec")
     args = ap.parse_args()

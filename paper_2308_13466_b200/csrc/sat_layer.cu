@@ -327,52 +327,44 @@ static sat_status run_lstm_cached(sat_ctx *ctx, CacheLayer *c, const sat_pred_pa
         SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, newest), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
         c->proj_tag[newest] = p->version;
     }
-    // The recurrence is row-wise: a block of rows can run all of its steps before the next block starts.  With blocks small
-    // enough for their state (s and c) to stay in L2 between two steps, only the cached projections stream from HBM.
-    const char *chunk_env = getenv("SAT_LSTM_CHUNK");
-    const int64_t chunk = chunk_env ? (atoll(chunk_env) + 127) / 128 * 128 : 0;   // rows per block (multiple of the row tile); 0: all rows at once
-    for (int64_t r0 = 0; r0 < rows; r0 += (chunk > 0 ? chunk : rows)) {
-        const int64_t cnt = chunk > 0 && r0 + chunk < rows ? chunk : rows - r0;
-        float *S_blk = c->S + r0 * h;
-        float *cell_blk = cell + sat_cell_offset(r0, 0, h);
-        for (int32_t t = 0; t < k; ++t) {
-            const int32_t idx = ring_index(ctx, k - 1 - t);  // oldest first
-            const bool cached = c->proj_tag[idx] == p->version;
-            const float *pr = c->proj + (int64_t)idx * plane + r0 * 4 * h;
-            const float *x_blk = ring_buf(ctx, c, idx) + r0 * c->ld;
-            TcEpilogueHost eh;
-            eh.C = S_blk;
-            eh.ldc = h;
-            eh.lstm_h = h;
-            eh.lstm_c = cell_blk;
-            if (cached && t == 0) {
-                ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)cnt * h * 6.0, 0.0);
-                k_lstm_cell_first<<<(unsigned)cdiv64(cnt * h, 256), 256, 0, ctx->stream>>>(pr, cnt, h, cell_blk, S_blk);
-                SAT_LAUNCHED(ctx);
-            } else if (cached) {
-                if (!have_up) {
-                    if (c->tag_uh == p->version) {
-                        SAT_TRY(sat_tc_weights_layout(h, 4 * h, c->pk_uh, &Up));
-                    } else {
-                        SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, c->pk_uh, &Up, h));
-                        c->tag_uh = p->version;
-                    }
+    // (Running the steps row block by row block, so that a block's state stays in L2 between two steps, was measured and
+    // was slower: the smaller launches cost more than the state traffic they save.)
+    for (int32_t t = 0; t < k; ++t) {
+        const int32_t idx = ring_index(ctx, k - 1 - t);  // oldest first
+        const bool cached = c->proj_tag[idx] == p->version;
+        const float *pr = c->proj + (int64_t)idx * plane;
+        TcEpilogueHost eh;
+        eh.C = c->S;
+        eh.ldc = h;
+        eh.lstm_h = h;
+        eh.lstm_c = cell;
+        if (cached && t == 0) {
+            ProfScope prof(ctx, SATK_LSTM_CELL, 4.0 * (double)rows * h * 6.0, 0.0);
+            k_lstm_cell_first<<<(unsigned)cdiv64(rows * h, 256), 256, 0, ctx->stream>>>(pr, rows, h, cell, c->S);
+            SAT_LAUNCHED(ctx);
+        } else if (cached) {
+            if (!have_up) {
+                if (c->tag_uh == p->version) {
+                    SAT_TRY(sat_tc_weights_layout(h, 4 * h, c->pk_uh, &Up));
+                } else {
+                    SAT_TRY(sat_tc_weights(ctx, p->Uh, 4 * h, h, nullptr, 0, 0, 4 * h, 1, c->pk_uh, &Up, h));
+                    c->tag_uh = p->version;
                 }
-                have_up = true;
-                eh.addend = pr;
-                eh.ld_addend = 4 * h;
-                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, S_blk, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
-            } else if (t == 0) {
-                SAT_TRY(pack_wx());
-                eh.bias = p->b;
-                eh.lstm_first = 1;
-                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, x_blk, c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
-            } else {
-                if (!have_wxu) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit3, &Wxu, h));
-                have_wxu = true;
-                eh.bias = p->b;
-                SAT_TRY(sat_gemm_tc(ctx, cnt, 4 * h, x_blk, c->ld, d, S_blk, h, h, Wxu, eh, SATK_GEMM_NN));
             }
+            have_up = true;
+            eh.addend = pr;
+            eh.ld_addend = 4 * h;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, c->S, h, h, nullptr, 0, 0, Up, eh, SATK_GEMM_SIDE));
+        } else if (t == 0) {
+            SAT_TRY(pack_wx());
+            eh.bias = p->b;
+            eh.lstm_first = 1;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, nullptr, 0, 0, Wp, eh, SATK_GEMM_NN));
+        } else {
+            if (!have_wxu) SAT_TRY(sat_tc_weights(ctx, p->Wx, 4 * h, d, p->Uh, 4 * h, h, 4 * h, 1, ctx->buf_wsplit3, &Wxu, h));
+            have_wxu = true;
+            eh.bias = p->b;
+            SAT_TRY(sat_gemm_tc(ctx, rows, 4 * h, ring_buf(ctx, c, idx), c->ld, d, c->S, h, h, Wxu, eh, SATK_GEMM_NN));
         }
     }
     c->S_valid = true;

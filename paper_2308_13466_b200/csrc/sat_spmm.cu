@@ -2,8 +2,6 @@
 // row gather and row scatter.  All of them are bandwidth-bound: every feature row is moved
 // with 128-bit loads, one group of lanes per work item, warp shuffles broadcast the column
 // ids, and nothing is accumulated with floating-point atomics (results are reproducible).
-#include <cstdlib>
-
 #include "sat_internal.h"
 
 __device__ __forceinline__ float4 ld4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
@@ -191,17 +189,6 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
         partial = (float *)ctx->buf_partial.p;
     }
 #define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words, cols, halo_range
-    // experiment switch: SAT_SPMM_CFG = 100 * lanes + vectors per lane selects the lane-group shape (column slices run as grid.y)
-    const char *cfg_env = getenv("SAT_SPMM_CFG");
-    const int cfg = cfg_env ? atoi(cfg_env) : 0;
-    if (cfg == 1601) launch_items<16, 1>(ARGS);
-    else if (cfg == 802) launch_items<8, 2>(ARGS);
-    else if (cfg == 3201) launch_items<32, 1>(ARGS);
-    else if (cfg == 1602) launch_items<16, 2>(ARGS);
-    else if (cfg == 801) launch_items<8, 1>(ARGS);
-    else if (cfg == 3202) launch_items<32, 2>(ARGS);
-    else if (cfg == 804) launch_items<8, 4>(ARGS);
-    else
     if (d4 <= 4) launch_items<4, 1>(ARGS);
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);

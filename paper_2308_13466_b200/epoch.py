@@ -58,9 +58,13 @@ class SatEpoch:
         self.labels = None
 
     def close(self):
+        """Destroys the context and drops the activation / gradient buffers (sizes and offsets stay readable)."""
         if self.ctx is not None:
             B.sat_destroy(self.ctx)
             self.ctx = None
+        self.H = self.G = self.halo = self.X_in = self.X = self.labels = None
+        if hasattr(self, "gat_halo"):
+            self.gat_halo = None
 
     # ---- inputs -------------------------------------------------------------------
     def set_inputs(self, X: torch.Tensor, labels_perm: torch.Tensor):
