@@ -45,6 +45,8 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
              float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial, const uint32_t *__restrict__ omask, int32_t omask_words,
              DbgLimits dbg)
 {
+    // (Several consecutive work items per lane group — fewer, longer-lived blocks — were measured: neutral on the large
+    // workload, 40 % slower on the medium one, where the chunks of a hub row then land in one warp.)
     const int lane = threadIdx.x & (G - 1);
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
     if (gid >= n_items) return;
@@ -297,7 +299,7 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
             const float *__restrict__ hrow_w, const int32_t *__restrict__ halo_slot, const float *__restrict__ dinv_enc, int32_t n, int64_t halo0, int64_t n_halo,
             int by_slot, int32_t d4, const float *__restrict__ src_base, int64_t ld_src, const float *__restrict__ self_src,
             float *__restrict__ out_base, int64_t ld_out, const int32_t *__restrict__ hlong, const int64_t *__restrict__ hchunk_first,
-            const int32_t *__restrict__ hchunk_row, int32_t hchunk0, int32_t n_hchunks, float *__restrict__ hpartial, DbgLimits dbg)
+            const int32_t *__restrict__ hchunk_row, int32_t hchunk0, int32_t n_hchunks, float *__restrict__ hpartial, int32_t ipg, DbgLimits dbg)
 {
     if ((int32_t)blockIdx.x < n_hchunks) {
         hrow_chunk_block<G, NV>(hchunk0 + (int32_t)blockIdx.x, hlong, hchunk_first, hchunk_row, hchunk0, hrow_ptr, hrow_pos, hrow_slot, hrow_w, by_slot,
@@ -306,53 +308,59 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
     }
     const int lane = threadIdx.x & (G - 1);
     const int64_t gid = ((int64_t)(blockIdx.x - n_hchunks) * blockDim.x + threadIdx.x) / G;
-    if (gid >= n_halo) return;
     const int col0 = blockIdx.y * (G * NV);
-    const int64_t j = halo0 + gid;
-    const float du = __ldg(dinv_enc + n + j);
-    float4 acc[NV];
-#pragma unroll
-    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (self_src) {
-        const float *src = self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int idx = col0 + lane + v * G;
-            if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
-        }
-    }
-    const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
-    if (e1 - e0 > SAT_HROW_LONG) return;  // cut into chunks, a block each (hrow_chunk_block), combined by k_hrow_long_fixup
-    // Halo rows are short (a handful of cut edges): every lane reads the entry's column and weight itself (one broadcast
-    // transaction per group) instead of sharing them through shuffles, four entries in flight; entries in order, so the
-    // sum has the same order as the long-row path's per-group partial sums.
+    // a lane group walks `ipg` consecutive halo rows (fewer, longer-lived blocks; the header loads of a row overlap the
+    // gathers of the one before)
+    const int64_t g0 = gid * ipg;
+    if (g0 >= n_halo) return;
+    const int64_t g1 = g0 + ipg < n_halo ? g0 + ipg : n_halo;
     const int32_t *__restrict__ ecol = by_slot ? hrow_slot : hrow_pos;
-    for (int64_t e = e0; e < e1; e += 4) {
-        int32_t c[4];
-        float w[4];
+    for (int64_t g = g0; g < g1; ++g) {
+        const int64_t j = halo0 + g;
+        const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
+        if (e1 - e0 > SAT_HROW_LONG) continue;  // cut into chunks, a block each (hrow_chunk_block), combined by k_hrow_long_fixup
+        const float du = __ldg(dinv_enc + n + j);
+        float4 acc[NV];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const bool ok = e + u < e1;
-            c[u] = ok ? (int32_t)SAT_IDX(__ldg(ecol + e + u), dbg.src_lo, dbg.src_hi, dbg.status) : -1;
-            w[u] = ok ? __ldg(hrow_w + e + u) : 0.f;
+        for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (self_src) {
+            const float *src = self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
+            }
         }
+        // Halo rows are short (a handful of cut edges): every lane reads the entry's column and weight itself (one broadcast
+        // transaction per group) instead of sharing them through shuffles, four entries in flight; entries in order, so the
+        // sum has the same order as the long-row path's per-group partial sums.
+        for (int64_t e = e0; e < e1; e += 4) {
+            int32_t c[4];
+            float w[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const bool ok = e + u < e1;
+                c[u] = ok ? (int32_t)SAT_IDX(__ldg(ecol + e + u), dbg.src_lo, dbg.src_hi, dbg.status) : -1;
+                w[u] = ok ? __ldg(hrow_w + e + u) : 0.f;
+            }
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx >= d4) continue;
+                float4 x[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) x[u] = c[u] >= 0 ? ld4(src_base + (int64_t)c[u] * ld_src + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (c[u] >= 0) fma4(acc[v], w[u], x[u]);
+            }
+        }
+        float *o = out_base + j * ld_out;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
             const int idx = col0 + lane + v * G;
-            if (idx >= d4) continue;
-            float4 x[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) x[u] = c[u] >= 0 ? ld4(src_base + (int64_t)c[u] * ld_src + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (c[u] >= 0) fma4(acc[v], w[u], x[u]);
+            if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(du * acc[v].x, du * acc[v].y, du * acc[v].z, du * acc[v].w);
         }
-    }
-    float *o = out_base + j * ld_out;
-#pragma unroll
-    for (int v = 0; v < NV; ++v) {
-        const int idx = col0 + lane + v * G;
-        if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = make_float4(du * acc[v].x, du * acc[v].y, du * acc[v].z, du * acc[v].w);
     }
 }
 
@@ -360,10 +368,14 @@ template <int G, int NV>
 static void launch_hrow(sat_ctx *ctx, const PartView &v, int by_slot, int32_t d4, const float *src_base, int32_t ld_src,
                         const float *self_src, float *out_base, int32_t ld_out, float *hpartial)
 {
-    dim3 grid((unsigned)(cdiv64(v.n_halo * G, 256) + v.n_hchunks), (unsigned)cdiv64(d4, G * NV));
+    // rows per lane group: launches of millions of halo rows (hundreds of thousands of short-lived blocks at one row per
+    // group) run 18 % faster at four rows per group; smaller launches need every block they can get (measured: 263 k rows
+    // are 25 % slower at four)
+    const int32_t ipg = v.n_halo >= ((int64_t)4 << 20) ? 4 : v.n_halo >= ((int64_t)2 << 20) ? 2 : 1;
+    dim3 grid((unsigned)(cdiv64(cdiv64(v.n_halo, ipg) * G, 256) + v.n_hchunks), (unsigned)cdiv64(d4, G * NV));
     k_spmm_hrow<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->hrow_ptr, ctx->hrow_pos, ctx->hrow_slot, ctx->hrow_w, ctx->halo_slot, ctx->dinv_enc, ctx->n,
                                                        v.halo0, v.n_halo, by_slot, d4, src_base, ld_src, self_src, out_base, ld_out,
-                                                       ctx->hlong, ctx->hchunk_first, ctx->hchunk_row, v.hchunk0, v.n_hchunks, hpartial,
+                                                       ctx->hlong, ctx->hchunk_first, ctx->hchunk_row, v.hchunk0, v.n_hchunks, hpartial, ipg,
                                                        dbg_limits(by_slot ? DbgRange{0, ctx->n_slots} : DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, DbgRange{v.halo0, v.halo0 + v.n_halo}, DbgRange{v.halo0, v.halo0 + v.n_halo}, ctx->d_flag + 1));
 }
 
