@@ -201,7 +201,8 @@ def run_reference(args, wl):
 
 def workload_config(wl):
     return dict(workload=f"{wl.name}: {wl.n} nodes, nnz(A+I)={wl.nnz}, GCN {'-'.join(map(str, wl.dims))}, "
-                         f"{wl.M} partitions (contiguous id blocks after BFS relabel), predictor history {wl.tau}, h={wl.pred[0]['h'] if wl.pred else 0}",
+                         f"{wl.M} partitions ({'the blocks of the stochastic block model' if wl.part_given is not None else 'contiguous id blocks after BFS relabel'}), "
+                         f"predictor history {wl.tau}, h={wl.pred[0]['h'] if wl.pred else 0}",
                 nodes=wl.n, nnz=wl.nnz, partitions=wl.M, tau=wl.tau,
                 predictor_update_period=f"{PRED_PERIOD} epochs (Algorithm 1's Delta-T): the predictor's parameter version is bumped every "
                                         f"{PRED_PERIOD}th epoch, which drops the cached LSTM input projections; the timed epochs contain "

@@ -514,9 +514,19 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             const bool row_ok = row < M;
             float *crow = ep.C + row * ep.ldc;
             float *prow = nullptr;   // (EPI_PUSH) this row's home in the cache ring, if it has one
-            if (EPI == EPI_PUSH && row_ok) {
+            // (EPI_PUSH with the staged store) the push goes out of the staging tile, four rows of 128 bytes per warp
+            // instruction: lane L writes 16-byte piece L & 7 of rows (L >> 3) + 4 i, so it needs those rows' ring rows
+            int32_t ps8[8];
+            if (EPI == EPI_PUSH && !use_tma_store && row_ok) {
                 const int32_t ps = __ldg(ep.push_slot + row);
                 if (ps >= 0) prow = ep.push_dst + (int64_t)ps * ep.ld_push;
+            }
+            if (EPI == EPI_PUSH && use_tma_store) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int64_t rr = m0 + q * 32 + (lane >> 3) + 4 * i;
+                    ps8[i] = rr < M ? __ldg(ep.push_slot + rr) : -1;
+                }
             }
             float4 side[8], cside[2];
             // previous cell state of the next chunk, fetched one chunk ahead (two 128-bit loads per thread)
@@ -651,6 +661,26 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) tma_store_2d(&mapC, obuf, n0 + c0, (int32_t)(m0 + q * 32));
+                    if (EPI == EPI_PUSH) {
+                        // the boundary rows also go to the cache ring, read back from the staged block: every instruction
+                        // writes whole 128-byte row segments (the per-thread form touches 32 different lines per instruction)
+                        const int piece = lane & 7;
+                        const int32_t colb = n0 + c0 + 4 * piece;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            if (ps8[i] < 0 || colb >= N) continue;
+                            float *pr = ep.push_dst + (int64_t)ps8[i] * ep.ld_push;
+                            const int rr = (lane >> 3) + 4 * i;
+                            const uint4 x = *reinterpret_cast<const uint4 *>(obuf + rr * 128 + ((piece ^ (rr & 7)) << 4));
+                            if (colb + 3 < N) {
+                                *reinterpret_cast<uint4 *>(pr + colb) = x;
+                            } else {
+                                pr[colb] = __uint_as_float(x.x);
+                                if (colb + 1 < N) pr[colb + 1] = __uint_as_float(x.y);
+                                if (colb + 2 < N) pr[colb + 2] = __uint_as_float(x.z);
+                            }
+                        }
+                    }
                 } else if (row_ok) {
 #pragma unroll
                     for (int j4 = 0; j4 < 32; j4 += 4) {

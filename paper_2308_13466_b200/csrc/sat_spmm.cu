@@ -195,7 +195,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);
     else if (d4 <= 32) launch_items<8, 4>(ARGS);
-    else if (d4 <= 64) launch_items<32, 2>(ARGS);
+    else if (d4 <= 64) launch_items<32, 2>(ARGS);   // compiled for 8 resident blocks per SM (32 registers): 6 / 5 / 4 blocks (40-44 registers, no spills) measured 3 / 12 / 11 % slower
     else if (d4 <= 96) launch_items<32, 3>(ARGS);
     else if (d4 <= 128) launch_items<32, 4>(ARGS);
     else if (d4 <= 160) launch_items<32, 5>(ARGS);
