@@ -64,6 +64,8 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // (Computing the row addresses in float4 units with 32 x 32 -> 64-bit multiplies saves instructions but costs registers:
+    // at the 32 registers this kernel is compiled for it spills, and was 10 % slower on every workload.)
     for (int64_t eb = e0; eb < e1; eb += G) {
         const int64_t e = eb + lane;
         int32_t c = 0;
@@ -243,14 +245,16 @@ __device__ __forceinline__ void hrow_chunk_block(int32_t chunk, const int32_t *_
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     const int64_t e0 = hrow_ptr[j] + k * SAT_HROW_CHUNK;
     const int64_t e1 = e0 + SAT_HROW_CHUNK < hrow_ptr[j + 1] ? e0 + SAT_HROW_CHUNK : hrow_ptr[j + 1];
+    const float4 *src4 = reinterpret_cast<const float4 *>(src_base) + (col0 + lane);
+    const uint32_t lds4 = (uint32_t)(ld_src >> 2);
+    const int32_t *__restrict__ ecol = by_slot ? hrow_slot : hrow_pos;
     for (int64_t e = e0 + grp; e < e1; e += NG) {
         const float w = __ldg(hrow_w + e);
-        const int32_t c = (int32_t)SAT_IDX(by_slot ? __ldg(hrow_slot + e) : __ldg(hrow_pos + e), dbg.src_lo, dbg.src_hi, dbg.status);
-        const float *src = src_base + (int64_t)c * ld_src;
+        const int32_t c = (int32_t)SAT_IDX(__ldg(ecol + e), dbg.src_lo, dbg.src_hi, dbg.status);
+        const float4 *src = src4 + (uint64_t)(uint32_t)c * lds4;
 #pragma unroll
         for (int v = 0; v < NV; ++v) {
-            const int idx = col0 + lane + v * G;
-            if (idx < d4) fma4(acc[v], w, ld4(src + 4 * idx));
+            if (col0 + lane + v * G < d4) fma4(acc[v], w, __ldg(src + v * G));
         }
     }
 #pragma unroll
@@ -315,6 +319,10 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
     if (g0 >= n_halo) return;
     const int64_t g1 = g0 + ipg < n_halo ? g0 + ipg : n_halo;
     const int32_t *__restrict__ ecol = by_slot ? hrow_slot : hrow_pos;
+    // row addresses in float4 units: one 32 x 32 -> 64-bit multiply per gathered row
+    const float4 *src4 = reinterpret_cast<const float4 *>(src_base) + (col0 + lane);
+    const float4 *self4 = reinterpret_cast<const float4 *>(self_src) + (col0 + lane);
+    const uint32_t lds4 = (uint32_t)(ld_src >> 2);
     for (int64_t g = g0; g < g1; ++g) {
         const int64_t j = halo0 + g;
         const int64_t e0 = hrow_ptr[j], e1 = hrow_ptr[j + 1];
@@ -324,11 +332,10 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
 #pragma unroll
         for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (self_src) {
-            const float *src = self_src + SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * ld_src;
+            const float4 *src = self4 + (uint64_t)(uint32_t)SAT_IDX((int64_t)halo_slot[j], dbg.src_lo, dbg.src_hi, dbg.status) * lds4;
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                const int idx = col0 + lane + v * G;
-                if (idx < d4) fma4(acc[v], du, ld4(src + 4 * idx));
+                if (col0 + lane + v * G < d4) fma4(acc[v], du, __ldg(src + v * G));
             }
         }
         // Halo rows are short (a handful of cut edges): every lane reads the entry's column and weight itself (one broadcast
@@ -345,11 +352,11 @@ k_spmm_hrow(const int64_t *__restrict__ hrow_ptr, const int32_t *__restrict__ hr
             }
 #pragma unroll
             for (int v = 0; v < NV; ++v) {
-                const int idx = col0 + lane + v * G;
-                if (idx >= d4) continue;
+                if (col0 + lane + v * G >= d4) continue;
                 float4 x[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) x[u] = c[u] >= 0 ? ld4(src_base + (int64_t)c[u] * ld_src + 4 * idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int u = 0; u < 4; ++u)
+                    x[u] = c[u] >= 0 ? __ldg(src4 + (uint64_t)(uint32_t)c[u] * lds4 + v * G) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
                     if (c[u] >= 0) fma4(acc[v], w[u], x[u]);
