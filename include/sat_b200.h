@@ -64,6 +64,11 @@ enum { SAT_ACT_NONE = 0, SAT_ACT_RELU = 1 };
  * rows are exact and need no cache: Eq. "mini-batch" with h^(0) = x); the layer reads the halo nodes' rows from it directly,
  * which saves the sat_gather_rows pull and its [sum_m b_m x d] copy.  Same result, bit for bit, as the gathered call. */
 #define SAT_FWD_HALO_GLOBAL 0x200
+/* ... and SAT_FWD_INPUT_GLOBAL: h_in too is that matrix over all n nodes in global id order ([n x ld_in]; h_halo is ignored
+ * and may be NULL): the in-subgraph rows are read through the partition's inner list, the out-of-subgraph rows through its
+ * halo list.  For layer 1 the caller then needs neither the partition-major copy of the features nor the halo pull.  Same
+ * result, bit for bit, as the call on gathered rows. */
+#define SAT_FWD_INPUT_GLOBAL 0x400
 enum { SAT_LOSS_SOFTMAX_CE = 0, SAT_LOSS_SIGMOID_BCE = 1 };
 enum { SAT_ROWS_INNER = 0, SAT_ROWS_HALO = 1 };          /* sat_gather_rows                      */
 enum { SAT_CACHE_ZERO = 0, SAT_CACHE_COPY = 1 };         /* sat_cache_init                       */

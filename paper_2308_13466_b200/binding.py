@@ -24,6 +24,7 @@ SAT_LOSS_SOFTMAX_CE, SAT_LOSS_SIGMOID_BCE = 0, 1
 SAT_BWD_ACCUMULATE, SAT_BWD_MASK_G_IN, SAT_BWD_G_OUT_MASKED, SAT_BWD_GRAD_HISTORY = 1, 2, 4, 8
 SAT_FWD_PUSH = 0x100
 SAT_FWD_HALO_GLOBAL = 0x200
+SAT_FWD_INPUT_GLOBAL = 0x400
 SAT_ROWS_INNER, SAT_ROWS_HALO = 0, 1
 SAT_CACHE_ZERO, SAT_CACHE_COPY = 0, 1
 

@@ -121,6 +121,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->lrowptr);
     dev_free(&ctx->lenc);
     dev_free(&ctx->lenc_gid);
+    dev_free(&ctx->lenc_all_gid);
     dev_free(&ctx->inner_cnt);
     dev_free(&ctx->dinv_enc);
     dev_free(&ctx->lw);

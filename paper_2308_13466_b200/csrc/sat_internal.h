@@ -155,6 +155,7 @@ struct sat_ctx {
     int64_t *lrowptr = nullptr;   // [n+1] local CSR, rows partition-major
     int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
     int32_t *lenc_gid = nullptr;  // [nnz+n] the same with halo columns as n + global node id (built on first use: SAT_FWD_HALO_GLOBAL)
+    int32_t *lenc_all_gid = nullptr; // [nnz+n] every column as a global node id (built on first use: SAT_FWD_INPUT_GLOBAL)
     int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
     float *dinv_enc = nullptr;    // [n + nb] dinv of the node behind each encoded column
     float *lw = nullptr;          // [nnz+n] dinv_enc[lenc[e]] stored per entry (read with the column instead of gathered)
@@ -316,10 +317,11 @@ sat_status sat_part_view(sat_ctx *ctx, int32_t part, PartView *v);
 //   partition-major inner matrix and of the concatenated halo matrix (already offset for a single
 //   partition); `out_base` likewise.
 // omask (or null): bit mask [rows x omask_words] indexed like out_base; output components whose bit is 0 are written as 0
-// halo_global: the halo columns address a matrix over all n nodes in global id order (halo_base = its first row)
+// halo_global: the halo columns address a matrix over all n nodes in global id order (halo_base = its first row);
+// in_global: inner and halo columns both address such a matrix (in_base = its first row; halo_base is not used)
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
                     const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask = nullptr,
-                    int32_t omask_words = 0, bool halo_global = false);
+                    int32_t omask_words = 0, bool halo_global = false, bool in_global = false);
 //   halo-row products: out[j] = sum_{e in hrow(j)} dinv[halo j] dinv[inner e] * src[pos_e]   (+ self term if self_src)
 sat_status sat_spmm_hrow(sat_ctx *ctx, const PartView &v, int32_t d, const float *src_base, int32_t ld_src,
                          int by_slot, const float *self_src, float *out_base, int32_t ld_out);

@@ -625,8 +625,9 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     SAT_TRY(sat_part_view(ctx, part, &v));
     if (layer < 1 || layer > SAT_MAX_LAYERS) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: layer must be in [1, %d]", SAT_MAX_LAYERS);
     const bool push = (act & SAT_FWD_PUSH) != 0;
-    const bool halo_global = (act & SAT_FWD_HALO_GLOBAL) != 0;
-    act &= ~(SAT_FWD_PUSH | SAT_FWD_HALO_GLOBAL);
+    const bool in_global = (act & SAT_FWD_INPUT_GLOBAL) != 0;
+    const bool halo_global = in_global || (act & SAT_FWD_HALO_GLOBAL) != 0;
+    act &= ~(SAT_FWD_PUSH | SAT_FWD_HALO_GLOBAL | SAT_FWD_INPUT_GLOBAL);
     if (d_in <= 0 || d_out <= 0 || !W || (act != SAT_ACT_NONE && act != SAT_ACT_RELU)) return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: bad dims / W / act");
     CacheLayer *pc = nullptr;
     if (push) {
@@ -635,7 +636,7 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     }
     if (v.n_rows > 0 && (!h_in || !h_out || !ok_ld(ld_in, d_in) || !ok_ld(ld_out, d_out) || !aligned16(h_in) || !aligned16(h_out)))
         return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: null / misaligned h_in / h_out or bad leading dimension");
-    if (v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo)))
+    if (!in_global && v.n_halo > 0 && (!h_halo || !ok_ld(ld_halo, d_in) || !aligned16(h_halo)))
         return sat_fail(ctx, SAT_EINVAL, "sat_layer_fwd: null / misaligned h_halo or bad ld_halo");
     LayerState &L = ctx->layers[layer];
     const int32_t ld_agg = round_up4(d_in), words = (d_out + 31) / 32;
@@ -650,10 +651,11 @@ extern "C" sat_status sat_layer_fwd(sat_ctx *ctx, int32_t part, int32_t layer, i
     }
     L.act = act;
     if (v.n_rows == 0) return SAT_OK;
-    const float *in_base = h_in - (int64_t)v.row0 * ld_in;
-    // the halo source is the concatenated halo matrix (addressed from its virtual first row) or a matrix over all nodes
-    const float *halo_base = !h_halo ? nullptr : halo_global ? h_halo : h_halo - v.halo0 * (int64_t)ld_halo;
-    SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg, nullptr, 0, halo_global));
+    // the inner source is the partition-major matrix (addressed from its virtual first row) or, like the halo source, a matrix
+    // over all nodes; the halo source is the concatenated halo matrix (virtual first row) or a matrix over all nodes
+    const float *in_base = in_global ? h_in : h_in - (int64_t)v.row0 * ld_in;
+    const float *halo_base = in_global || !h_halo ? nullptr : halo_global ? h_halo : h_halo - v.halo0 * (int64_t)ld_halo;
+    SAT_TRY(sat_spmm(ctx, v, 0, d_in, in_base, ld_in, halo_base, ld_halo, L.agg, ld_agg, nullptr, 0, halo_global, in_global));
     uint32_t *mask_out = act == SAT_ACT_RELU ? L.mask + (int64_t)v.row0 * words : nullptr;
     const float *agg = L.agg + (int64_t)v.row0 * ld_agg;
     if (sat_use_tc(d_out, d_in)) {

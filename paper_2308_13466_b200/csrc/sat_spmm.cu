@@ -64,8 +64,11 @@ k_spmm_items(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ in
     float4 acc[NV];
 #pragma unroll
     for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
-    // (Computing the row addresses in float4 units with 32 x 32 -> 64-bit multiplies saves instructions but costs registers:
-    // at the 32 registers this kernel is compiled for it spills, and was 10 % slower on every workload.)
+    // (Cheaper row addressing was measured twice and was slower both times: 32 x 32 -> 64-bit multiplies in float4 units for the
+    // two matrices, and a single-matrix form — one multiply-add, no select — for launches whose columns all index one matrix
+    // (inner-only, halo-only, a halo matrix right behind the inner one, both read from a matrix over all nodes).  Either way
+    // the kernel executes a third fewer instructions and runs 4-10 % slower on every workload: it is bound by memory
+    // latency and DRAM, not by instruction issue, and at 32 registers the leaner loop spills more.)
     for (int64_t eb = e0; eb < e1; eb += G) {
         const int64_t e = eb + lane;
         int32_t c = 0;
@@ -141,14 +144,13 @@ __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, i
 template <int G, int NV>
 static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d4, const float *in_base, int32_t ld_in,
                          const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial, const uint32_t *omask,
-                         int32_t omask_words, const int32_t *cols, DbgRange halo_range)
+                         int32_t omask_words, const int32_t *cols, DbgRange halo_range, DbgRange src_range)
 {
     dim3 grid((unsigned)cdiv64((int64_t)v.n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
-    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, cols, ctx->lw, ctx->dinv_enc, ctx->item_row,
-                                                        ctx->first_item, ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only,
-                                                        ctx->n, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words,
-                                                        dbg_limits(DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, halo_range,
-                                                                  DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
+    k_spmm_items<G, NV><<<grid, 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->inner_cnt, cols, ctx->lw, ctx->dinv_enc, ctx->item_row, ctx->first_item,
+                                                        ctx->item_mslot, v.item0, v.n_items, v.mitem0, inner_only, ctx->n, d4, in_base, ld_in, halo_base,
+                                                        ld_halo, out_base, ld_out, partial, omask, omask_words,
+                                                        dbg_limits(src_range, halo_range, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
 }
 
 // halo columns as global node ids (for a halo source that is a matrix over all nodes)
@@ -161,15 +163,39 @@ __global__ void k_cols_by_gid(const int32_t *__restrict__ lenc, const int32_t *_
     out[e] = c < n ? c : n + halo_gid[c - n];
 }
 
+// all columns as global node ids (inner columns through the partition-major order, halo columns through the halo list)
+__global__ void k_cols_all_gid(const int32_t *__restrict__ lenc, const int32_t *__restrict__ perm, const int32_t *__restrict__ halo_gid,
+                               int64_t count, int32_t n, int32_t *__restrict__ out)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= count) return;
+    const int32_t c = lenc[e];
+    out[e] = c < n ? perm[c] : halo_gid[c - n];
+}
+
 sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, const float *in_base, int32_t ld_in,
                     const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, const uint32_t *omask, int32_t omask_words,
-                    bool halo_global)
+                    bool halo_global, bool in_global)
 {
     if (v.n_items == 0) return SAT_OK;
     const int32_t d4 = (d + 3) / 4;
     const int32_t *cols = ctx->lenc;
     DbgRange halo_range{v.halo0, v.halo0 + v.n_halo};
-    if (halo_global) {
+    DbgRange src_range{v.row0, (int64_t)v.row0 + v.n_rows};
+    if (in_global) {
+        // inner and halo rows both come from one matrix over all nodes (`in_base`, global id order): every column becomes a
+        // node id (all below n, so the kernel takes its inner branch for each of them)
+        if (!ctx->lenc_all_gid) {
+            const int64_t lnnz = ctx->nnz + ctx->n;
+            SAT_CUDA(ctx, cudaMalloc((void **)&ctx->lenc_all_gid, (size_t)lnnz * sizeof(int32_t)));
+            k_cols_all_gid<<<(unsigned)cdiv64(lnnz, 256), 256, 0, ctx->stream>>>(ctx->lenc, ctx->perm, ctx->halo_gid, lnnz, ctx->n, ctx->lenc_all_gid);
+            SAT_LAUNCHED(ctx);
+        }
+        cols = ctx->lenc_all_gid;
+        src_range = DbgRange{0, ctx->n};
+        halo_range = DbgRange{0, 0};
+    }
+    if (!in_global && halo_global) {
         if (!ctx->lenc_gid) {
             const int64_t lnnz = ctx->nnz + ctx->n;
             SAT_CUDA(ctx, cudaMalloc((void **)&ctx->lenc_gid, (size_t)lnnz * sizeof(int32_t)));
@@ -182,7 +208,8 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     // algorithmic bytes: column ids + row offsets + dinv, every source row once, every output row once (a halo source over
     // all nodes holds at most n distinct rows)
     const double n_halo_src = halo_global && v.n_halo > ctx->n ? (double)ctx->n : (double)v.n_halo;
-    const double n_src = inner_only == 1 ? (double)v.n_rows : inner_only == 2 ? n_halo_src : (double)v.n_rows + n_halo_src;
+    double n_src = inner_only == 1 ? (double)v.n_rows : inner_only == 2 ? n_halo_src : (double)v.n_rows + n_halo_src;
+    if (in_global && n_src > ctx->n) n_src = ctx->n;
     // the backward reads the inner prefix of every row, the transposed predictor convolution the halo suffix
     const double n_ent = (double)(inner_only == 1 ? v.lnnz - v.hnnz : inner_only == 2 ? v.hnnz : v.lnnz);
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
@@ -192,7 +219,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
         SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * d4 * 16));
         partial = (float *)ctx->buf_partial.p;
     }
-#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words, cols, halo_range
+#define ARGS ctx, v, inner_only, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words, cols, halo_range, src_range
     if (d4 <= 4) launch_items<4, 1>(ARGS);
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);

@@ -50,7 +50,7 @@ class SatEpoch:
         self.H = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # H[l], l = 1..L (partition-major rows)
         self.G = [None] + [_buf(self.n, d, dev) for d in self.dims[1:]]          # gradient w.r.t. H[l]
         self.halo = _buf(self.nb, max(self.dims[1:-1] or [1]), dev)               # predicted halo input of the running layer (layers >= 2)
-        self.X_in = _buf(self.n, self.dims[0], dev)
+        self.X_in = None                                                          # partition-major copy of the features (made on demand)
         self.gW = [torch.zeros((self.dims[l], self.dims[l + 1]), dtype=torch.float32, device=dev) for l in range(self.L)]
         self.gb = [torch.zeros(self.dims[l + 1], dtype=torch.float32, device=dev) for l in range(self.L)]
         self.loss_sum = torch.zeros(1, dtype=torch.float64, device=dev)
@@ -72,9 +72,19 @@ class SatEpoch:
         labels_perm: labels in partition-major row order (int32 [n] or uint8 [n, C])."""
         self.X = X
         self.labels = labels_perm
-        B.sat_gather_rows(self.ctx, B.SAT_ALL_PARTS, B.SAT_ROWS_INNER, X, self.X_in)
+        self.X_in = None
 
-    def halo_view(self, d: int, m: int = B.SAT_ALL_PARTS):
+    def inner_features(self) -> torch.Tensor:
+        """The features of the inner nodes in partition-major row order (a gathered copy, made when first asked for: the
+        GCN layer step reads the feature matrix itself)."""
+        if self.X_in is None:
+            self.X_in = _buf(self.n, self.dims[0], self.device)
+            B.sat_gather_rows(self.ctx, B.SAT_ALL_PARTS, B.SAT_ROWS_INNER, self.X, self.X_in)
+        return self.X_in
+
+    def halo_view(self, l: int, m: int = B.SAT_ALL_PARTS):
+        """Halo rows of the input of GNN layer l + 1 (predicted embeddings of cached layer l), all partitions or one."""
+        d = self.dims[l]
         if m == B.SAT_ALL_PARTS:
             return self.halo[:, :d]
         return self.halo[self.halo_off[m]:self.halo_off[m + 1], :d]
@@ -87,17 +97,16 @@ class SatEpoch:
     # ---- one epoch ----------------------------------------------------------------
     def _forward_backward(self, m: int, W, b, pred, accumulate: int, reuse_state: int, grad_history: bool = False):
         ctx, L = self.ctx, self.L
-        h_in = self.rows(self.X_in, m)
+        h_in = None
         for l in range(1, L + 1):
-            d_in = self.dims[l - 1]
             act = (B.SAT_ACT_RELU | B.SAT_FWD_PUSH) if l < L else B.SAT_ACT_NONE
             if l == 1:
-                # pull of layer 1: the out-of-subgraph rows are raw features, exact; the layer reads them from the feature
-                # matrix itself (global id order) instead of a gathered copy
-                hv = self.X
-                act |= B.SAT_FWD_HALO_GLOBAL
+                # layer 1: in- and out-of-subgraph rows are raw features, exact; the layer reads both from the feature matrix
+                # itself (global id order) through the partition's inner and halo lists: no gathered copies, no pull
+                h_in, hv = self.X, None
+                act |= B.SAT_FWD_INPUT_GLOBAL
             else:
-                hv = self.halo_view(d_in, m)
+                hv = self.halo_view(l - 1, m)
                 B.sat_predict(ctx, l - 1, m, pred[l - 2] if pred is not None else None, reuse_state, hv)  # pull predicted
             h_out = self.rows(self.H[l], m)
             # forward; for the cached layers the push of the boundary rows rides on the transform's epilogue
@@ -176,7 +185,7 @@ class SatEpoch:
             self.gat_grads = [{k: torch.zeros_like(v) for k, v in p.items()} for p in params]
             self.gat_halo = [_buf(self.nb, self.dims[l], dev) for l in range(L)]       # the pulled embeddings are needed again in the backward
         self.loss_sum.zero_()
-        h_in = self.X_in
+        h_in = self.inner_features()
         ins = []
         for l in range(1, L + 1):
             hv = self.gat_halo[l - 1]

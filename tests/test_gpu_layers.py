@@ -360,14 +360,16 @@ def test_cache_init_from_a_given_snapshot(B):
         B.sat_destroy(ctx)
 
 
-@pytest.mark.parametrize("name,shrink", [("medium", 16), ("odd", 1)])
-def test_halo_rows_read_from_the_global_feature_matrix(B, name, shrink):
-    """SAT_FWD_HALO_GLOBAL: layer 1 with h_halo = the feature matrix over all nodes gives the bits of the call on the gathered
-    halo rows (same entries, same order, same values), per partition and for all partitions at once, and the backward that
-    follows is the same."""
+@pytest.mark.parametrize("name,shrink,given", [("medium", 16, False), ("odd", 1, False), ("odd", 1, True)])
+def test_rows_read_from_the_global_feature_matrix(B, name, shrink, given):
+    """SAT_FWD_HALO_GLOBAL (h_halo = the feature matrix over all nodes) and SAT_FWD_INPUT_GLOBAL (h_in too): layer 1 gives the
+    bits of the call on gathered rows (same entries, same order, same values), per partition and for all partitions at once,
+    with contiguous blocks and with a scattered assignment (where the partition-major order is not the id order), and the
+    backward that follows is the same.  So is a layer whose halo matrix starts right behind its inner matrix in one buffer
+    against the same layer on two separate matrices (where the operands live must not matter)."""
     import torch
     wl = make_workload(name, shrink=shrink)
-    part = orc.contig_blocks(wl.n, wl.M)
+    part = np.random.default_rng(6).integers(0, wl.M, size=wl.n).astype(np.int32) if given else orc.contig_blocks(wl.n, wl.M)
     P = orc.build_partition(wl.rowptr, wl.col, part, wl.M)
     perm = np.concatenate(P.inner_gid)
     halo_all = np.concatenate(P.halo_gid)
@@ -376,23 +378,42 @@ def test_halo_rows_read_from_the_global_feature_matrix(B, name, shrink):
     ctx = B.sat_create(0, 0)
     try:
         B.sat_graph_load(ctx, wl.rowptr, wl.col)
-        B.sat_partition(ctx, wl.M, B.SAT_PART_CONTIG_BLOCKS)
+        if given:
+            B.sat_partition(ctx, wl.M, B.SAT_PART_GIVEN, part)
+        else:
+            B.sat_partition(ctx, wl.M, B.SAT_PART_CONTIG_BLOCKS)
         Xd = dev2d(wl.X)
         h_in, h_halo = dev2d(wl.X[perm]), dev2d(wl.X[halo_all])
         Wd, bd = dev(wl.W[0]), dev(wl.b[0])
-        d1 = wl.dims[1]
+        d0, d1 = wl.dims[0], wl.dims[1]
         G = dev2d((np.random.default_rng(4).standard_normal((wl.n, d1)) / wl.n).astype(np.float32))
+        # one buffer holding the inner rows and, right behind them, the halo rows
+        nb = halo_all.shape[0]
+        both = torch.zeros((wl.n + nb, (d0 + 3) & ~3), dtype=torch.float32, device="cuda")[:, :d0]
+        both[:wl.n].copy_(h_in)
+        both[wl.n:].copy_(h_halo)
         outs, grads = [], []
-        for mode in ("gathered", "global", "global-per-partition"):
+        for mode in ("gathered", "halo-global", "halo-global-per-partition", "input-global", "input-global-per-partition",
+                     "one-buffer", "one-buffer-per-partition"):
             h_out = empty2d(wl.n, d1)
+            relu = B.SAT_ACT_RELU
             if mode == "gathered":
-                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, h_halo, Wd, bd, B.SAT_ACT_RELU, h_out)
-            elif mode == "global":
-                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, Xd, Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_HALO_GLOBAL, h_out)
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, h_halo, Wd, bd, relu, h_out)
+            elif mode == "halo-global":
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, h_in, Xd, Wd, bd, relu | B.SAT_FWD_HALO_GLOBAL, h_out)
+            elif mode == "input-global":
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, Xd, None, Wd, bd, relu | B.SAT_FWD_INPUT_GLOBAL, h_out)
+            elif mode == "one-buffer":
+                B.sat_layer_fwd(ctx, B.SAT_ALL_PARTS, 1, both[:wl.n], both[wl.n:], Wd, bd, relu, h_out)
             else:
                 for m in range(P.M):
-                    r0, r1 = inner_off[m], inner_off[m + 1]
-                    B.sat_layer_fwd(ctx, m, 1, h_in[r0:r1], Xd, Wd, bd, B.SAT_ACT_RELU | B.SAT_FWD_HALO_GLOBAL, h_out[r0:r1])
+                    r0, r1, q0, q1 = inner_off[m], inner_off[m + 1], halo_off[m], halo_off[m + 1]
+                    if mode == "halo-global-per-partition":
+                        B.sat_layer_fwd(ctx, m, 1, h_in[r0:r1], Xd, Wd, bd, relu | B.SAT_FWD_HALO_GLOBAL, h_out[r0:r1])
+                    elif mode == "input-global-per-partition":
+                        B.sat_layer_fwd(ctx, m, 1, Xd, None, Wd, bd, relu | B.SAT_FWD_INPUT_GLOBAL, h_out[r0:r1])
+                    else:
+                        B.sat_layer_fwd(ctx, m, 1, both[r0:r1], both[wl.n + q0:wl.n + q1], Wd, bd, relu, h_out[r0:r1])
             gW = torch.full_like(Wd, float("nan"))
             gb = torch.full_like(bd, float("nan"))
             B.sat_layer_bwd(ctx, B.SAT_ALL_PARTS, 1, G, Wd, gW, gb, 0, None, None)
