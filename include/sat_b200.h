@@ -484,6 +484,19 @@ sat_status sat_profile_select(sat_ctx *ctx, uint64_t family_mask);
 sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int64_t *calls, double *ms, double *bytes,
                             double *flops);
 
+/* How the forward aggregation (the `P_in H_in + P_out Hhat` product of sat_layer_fwd; Appendix, forward of SAT) at width `d`
+ * walks partition `part` (or SAT_ALL_PARTS).  Where a partition's source rows (inner + out-of-subgraph) are several times
+ * the L2 and its rows are long, the library walks it once per block of sources instead of once, row by row: a row then
+ * contributes one partial sum per block it has entries in, added in block order afterwards (fixed order: reproducible, and
+ * the same whether the partition is run alone or with all others).  HOST outputs, each may be NULL: `n_blocks` = source
+ * blocks of the most finely cut partition (1 = plain row-by-row walk), `n_items` = work items of the launch,
+ * `n_partial_rows` = partial-sum rows of width d it writes and re-reads.  The cut is chosen per width (blocks of 64 MiB of
+ * source rows, for partitions above 192 MiB whose rows meet a block with 8 or more entries on average); the environment
+ * variable SAT_SPMM_SRC_BLOCK="<block bytes>[,<from bytes>[,<entries>]]" overrides the three figures for the process
+ * ("0" = never).  Builds the work list on first use (device memory, freed with the partition); synchronises the stream.
+ * Errors: SAT_ESTATE without a partition, SAT_EINVAL for a bad `part` or d < 1. */
+sat_status sat_spmm_plan(sat_ctx *ctx, int32_t part, int32_t d, int32_t *n_blocks, int64_t *n_items, int64_t *n_partial_rows);
+
 /* What the L2 -> SM path of the GPU delivers, measured now (measurement aid; the paper has no counterpart): a 64 MiB buffer,
  * resident in L2, read (a) as a contiguous stream by all SMs and (b) as rows of `row_floats` floats (a multiple of 4, at most
  * 1024) in pseudo-random order with the access shape of the SpMM kernels.  Both in GB/s (HOST outputs, either may be NULL).

@@ -66,7 +66,7 @@ EXPORTS = [
     "sat_predict_state", "sat_layer_fwd", "sat_layer_bwd", "sat_cache_update", "sat_cache_commit", "sat_cache_state",
     "sat_cache_read", "sat_cache_export", "sat_cache_import", "sat_cache_set_state", "sat_loss_grad", "sat_sgd_step", "sat_sgd_steps",
     "sat_dense_nn", "sat_dense_nt", "sat_dense_tn", "sat_dense_tn_static", "sat_launch_count", "sat_profile_families", "sat_profile_enable", "sat_profile_select", "sat_profile_read",
-    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores", "sat_profile_l2_rates", "sat_debug_poke_index",
+    "sat_codec_plan", "sat_codec_encode", "sat_codec_decode", "sat_cache_requantise", "sat_staleness", "sat_pred_grad", "sat_grad_history_read", "sat_grad_history_write", "sat_gat_fwd", "sat_gat_bwd", "sat_gat_scores", "sat_profile_l2_rates", "sat_debug_poke_index", "sat_spmm_plan",
 ]
 
 
@@ -433,6 +433,13 @@ def sat_profile_l2_rates(ctx, row_floats: int):
     a, b = C.c_double(), C.c_double()
     _check(ctx, _lib.sat_profile_l2_rates(ctx, C.c_int32(row_floats), C.byref(a), C.byref(b)))
     return float(a.value), float(b.value)
+
+
+def sat_spmm_plan(ctx, part: int, d: int):
+    """(source blocks, work items, partial-sum rows) of the forward aggregation at width d for `part`."""
+    nb, ni, ns = C.c_int32(), C.c_int64(), C.c_int64()
+    _check(ctx, _lib.sat_spmm_plan(ctx, C.c_int32(part), C.c_int32(d), C.byref(nb), C.byref(ni), C.byref(ns)))
+    return int(nb.value), int(ni.value), int(ns.value)
 
 
 def sat_profile_families() -> int:

@@ -122,6 +122,13 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->lenc);
     dev_free(&ctx->lenc_gid);
     dev_free(&ctx->lenc_all_gid);
+    for (SrcBlockedItems &sb : ctx->src_blocked) {
+        dev_free(&sb.item);
+        dev_free(&sb.slot0);
+        dev_free(&sb.tot);
+        dev_free(&sb.mrows);
+    }
+    ctx->src_blocked.clear();
     dev_free(&ctx->inner_cnt);
     dev_free(&ctx->dinv_enc);
     dev_free(&ctx->lw);
@@ -187,6 +194,7 @@ extern "C" sat_status sat_destroy(sat_ctx *ctx)
     dev_free(&ctx->dinv);
     sat_free_buf(ctx->buf_partial);
     sat_free_buf(ctx->buf_hpartial);
+    sat_free_buf(ctx->buf_sbpartial);
     sat_free_buf(ctx->buf_gagg);
     sat_free_buf(ctx->buf_splitk);
     sat_free_buf(ctx->buf_lstm_c);

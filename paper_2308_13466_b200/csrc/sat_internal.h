@@ -118,6 +118,23 @@ struct ProfRec {
     double bytes, flops;
 };
 
+// Forward SpMM work list in source-block-major order (sat_spmm.cu).  The sources of a partition (its inner rows, then its
+// halo rows) are cut into blocks of at most `block_rows` rows; the entries of every local-CSR row are sorted by source, so a
+// row meets each block in one contiguous run of entries.  An item is such a run (cut further at SAT_SPMM_CHUNK entries);
+// within a partition items are ordered by block, then by row, so that the rows gathered at any one time come from one or
+// two blocks.  Rows with more than one item add their partial sums in item order (k_spmm_sb_fixup).
+struct SrcBlockedItems {
+    int64_t block_rows = 0, fit_rows = 0, min_run = 0;  // key
+    int32_t n_items = 0, n_mrows = 0;
+    int64_t n_slots = 0;
+    int4 *item = nullptr;      // {row, partial slot or -1, first entry: low 32 bits, first entry: high 16 bits | entries << 16}
+    int32_t *slot0 = nullptr;  // [n] first partial slot of a row with several items
+    int32_t *tot = nullptr;    // [n] items of the row
+    int32_t *mrows = nullptr;  // [n_mrows] rows with several items
+    std::vector<int32_t> h_item_off, h_mrow_off;  // [M+1] per partition
+    std::vector<int64_t> h_slot_off;              // [M+1]
+};
+
 struct sat_ctx {
     bool prof_on = false;
     uint64_t prof_mask = ~0ull;  // families that are bracketed while prof_on
@@ -156,6 +173,7 @@ struct sat_ctx {
     int32_t *lenc = nullptr;      // [nnz+n] encoded column: < n: partition-major row of an inner node; >= n: n + halo position
     int32_t *lenc_gid = nullptr;  // [nnz+n] the same with halo columns as n + global node id (built on first use: SAT_FWD_HALO_GLOBAL)
     int32_t *lenc_all_gid = nullptr; // [nnz+n] every column as a global node id (built on first use: SAT_FWD_INPUT_GLOBAL)
+    std::vector<SrcBlockedItems> src_blocked;  // source-blocked forward work lists, one per block size (built on first use)
     int32_t *inner_cnt = nullptr; // [n] number of inner entries (incl. self-loop) at the front of each row
     float *dinv_enc = nullptr;    // [n + nb] dinv of the node behind each encoded column
     float *lw = nullptr;          // [nnz+n] dinv_enc[lenc[e]] stored per entry (read with the column instead of gathered)
@@ -195,7 +213,7 @@ struct sat_ctx {
 
     // ---- scratch ----
     DevBuf buf_codec_sizes, buf_codec_off, buf_codec_bytes;  // embedding codec scratch
-    DevBuf buf_hpartial;
+    DevBuf buf_hpartial, buf_sbpartial;
     DevBuf buf_partial, buf_gagg, buf_splitk, buf_lstm_c, buf_lstm_s, buf_lstm_w, buf_pred_a, buf_misc, buf_colsum, buf_dmask,
         buf_wsplit, buf_wsplit2, buf_wsplit3, buf_bias, buf_pred_train, buf_ghist_halo, buf_ghist_rows, buf_ghist_out, buf_gat, buf_gat_items;
 };

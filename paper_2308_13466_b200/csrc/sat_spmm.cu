@@ -4,6 +4,9 @@
 // ids, and nothing is accumulated with floating-point atomics (results are reproducible).
 #include "sat_internal.h"
 
+#include <algorithm>
+#include <cstdlib>
+
 __device__ __forceinline__ float4 ld4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 __device__ __forceinline__ void fma4(float4 &a, float w, const float4 &x)
 {
@@ -141,6 +144,359 @@ __global__ void k_spmm_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, i
     *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c) = r;
 }
 
+// -------------------------------------------------------------------------------------
+// Source-blocked forward SpMM.  When the sources of a partition (inner + halo rows) are several times the L2, a row-major
+// walk re-reads most of them from DRAM: every source row is used by ~10-20 rows spread over the whole partition and is
+// evicted between two uses.  The blocked work list walks the partition once per block of sources instead (the entries of a
+// row are sorted by source, so a row meets a block in one contiguous run); the rows gathered at any one time then belong to
+// one or two blocks, which the L2 holds.  The price is one partial sum per (row, block) and the pass that adds them.
+// -------------------------------------------------------------------------------------
+__device__ __forceinline__ int64_t lower_bound_col(const int32_t *__restrict__ lenc, int64_t lo, int64_t hi, int64_t key)
+{
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)lenc[mid] < key) lo = mid + 1;
+        else hi = mid;
+    }
+    return lo;
+}
+
+// encoded column of source p of a partition whose sources are [n_rows inner rows from row0 ; halo rows from halo0]
+__device__ __forceinline__ int64_t sb_source_col(int64_t p, int32_t row0, int32_t n_rows, int32_t n, int64_t halo0)
+{
+    return p < n_rows ? (int64_t)row0 + p : (int64_t)n + halo0 + (p - n_rows);
+}
+
+// entries [lo, hi) of `row` whose source falls into block j
+__device__ __forceinline__ void sb_run(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row, int32_t j,
+                                       int32_t n_blocks, int64_t block_rows, int32_t row0, int32_t n_rows, int32_t n, int64_t halo0,
+                                       int64_t *lo, int64_t *hi)
+{
+    const int64_t rb = lrowptr[row], re = lrowptr[row + 1];
+    *lo = j == 0 ? rb : lower_bound_col(lenc, rb, re, sb_source_col((int64_t)j * block_rows, row0, n_rows, n, halo0));
+    *hi = j == n_blocks - 1 ? re : lower_bound_col(lenc, *lo, re, sb_source_col((int64_t)(j + 1) * block_rows, row0, n_rows, n, halo0));
+}
+
+// count[j * n_rows + r] = items of row row0 + r in block j
+__global__ void k_sb_count(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
+                           int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t *__restrict__ count)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (int64_t)n_rows * n_blocks) return;
+    const int32_t j = (int32_t)(t / n_rows), r = (int32_t)(t - (int64_t)j * n_rows);
+    int64_t lo, hi;
+    sb_run(lrowptr, lenc, row0 + r, j, n_blocks, block_rows, row0, n_rows, n, halo0, &lo, &hi);
+    count[t] = (int32_t)((hi - lo + SAT_SPMM_CHUNK - 1) / SAT_SPMM_CHUNK);
+}
+
+__global__ void k_sb_row_totals(const int32_t *__restrict__ count, int32_t row0, int32_t n_rows, int32_t n_blocks, int32_t *__restrict__ tot,
+                                int32_t *__restrict__ slots, int32_t *__restrict__ multi)
+{
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n_rows) return;
+    int32_t s = 0;
+    for (int32_t j = 0; j < n_blocks; ++j) s += count[(int64_t)j * n_rows + r];
+    tot[row0 + r] = s;
+    slots[row0 + r] = s > 1 ? s : 0;
+    multi[row0 + r] = s > 1 ? 1 : 0;
+}
+
+__global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
+                          int64_t halo0, int32_t n_blocks, int64_t block_rows, const int32_t *__restrict__ count,
+                          const int64_t *__restrict__ item_off, const int32_t *__restrict__ tot, const int64_t *__restrict__ slot_off,
+                          int4 *__restrict__ item)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (int64_t)n_rows * n_blocks) return;
+    const int32_t j = (int32_t)(t / n_rows), r = (int32_t)(t - (int64_t)j * n_rows);
+    const int32_t c = count[t];
+    if (c == 0) return;
+    const int32_t row = row0 + r;
+    int64_t lo, hi;
+    sb_run(lrowptr, lenc, row, j, n_blocks, block_rows, row0, n_rows, n, halo0, &lo, &hi);
+    int32_t before = 0;
+    for (int32_t q = 0; q < j; ++q) before += count[(int64_t)q * n_rows + r];
+    const bool multi = tot[row] > 1;
+    for (int32_t q = 0; q < c; ++q) {
+        const int64_t e0 = lo + (int64_t)q * SAT_SPMM_CHUNK;
+        const int32_t len = (int32_t)((hi - e0) < SAT_SPMM_CHUNK ? (hi - e0) : SAT_SPMM_CHUNK);
+        item[item_off[t] + q] = make_int4(row, multi ? (int32_t)(slot_off[row] + before + q) : -1, (int32_t)(uint32_t)(e0 & 0xffffffffll),
+                                          (int32_t)((e0 >> 32) & 0xffff) | (len << 16));
+    }
+}
+
+__global__ void k_sb_rows(const int64_t *__restrict__ slot_off, const int32_t *__restrict__ multi, const int64_t *__restrict__ mrow_off,
+                          int32_t n, int32_t *__restrict__ slot0, int32_t *__restrict__ mrows)
+{
+    const int64_t r = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (r >= n) return;
+    slot0[r] = (int32_t)slot_off[r];
+    if (multi[r]) mrows[mrow_off[r]] = (int32_t)r;
+}
+
+static sat_status sb_read_i64(sat_ctx *ctx, const int64_t *d, int64_t *h)
+{
+    SAT_CUDA(ctx, cudaMemcpyAsync(h, d, sizeof(int64_t), cudaMemcpyDeviceToHost, ctx->stream));
+    SAT_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return SAT_OK;
+}
+
+// partitions whose sources fit `fit_rows` rows keep one block (their items are then the row chunks of the plain list)
+static int64_t sb_blocks_of(const sat_ctx *ctx, int m, int64_t block_rows, int64_t fit_rows, int64_t min_run)
+{
+    const int64_t rows = ctx->h_inner_off[m + 1] - ctx->h_inner_off[m];
+    const int64_t T = rows + (ctx->h_halo_off[m + 1] - ctx->h_halo_off[m]);
+    if (T <= fit_rows || rows == 0) return 1;
+    int64_t B = cdiv64(T, block_rows);
+    if (B > 4096) B = 4096;
+    // blocking pays where a row meets a block with a run of entries long enough to carry the extra partial sum
+    const int64_t entries = ctx->h_lnnz_off[m + 1] - ctx->h_lnnz_off[m];
+    return entries / (rows * B) >= min_run ? B : 1;
+}
+
+static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, int64_t min_run, SrcBlockedItems **out)
+{
+    for (SrcBlockedItems &sb : ctx->src_blocked)
+        if (sb.block_rows == block_rows && sb.min_run == min_run && sb.fit_rows == fit_rows) {
+            *out = &sb;
+            return SAT_OK;
+        }
+    const int32_t M = ctx->M, n = ctx->n;
+    std::vector<int32_t> nb((size_t)M);
+    std::vector<int64_t> br((size_t)M), cbase((size_t)M + 1, 0);
+    for (int m = 0; m < M; ++m) {
+        const int64_t rows = ctx->h_inner_off[m + 1] - ctx->h_inner_off[m];
+        const int64_t T = rows + (ctx->h_halo_off[m + 1] - ctx->h_halo_off[m]);
+        const int64_t B = sb_blocks_of(ctx, m, block_rows, fit_rows, min_run);
+        nb[m] = (int32_t)B;
+        br[m] = cdiv64(T > 0 ? T : 1, B);  // equal blocks
+        cbase[m + 1] = cbase[m] + rows * B;
+    }
+    const int64_t total = cbase[M];
+    int32_t *count = nullptr, *slots = nullptr, *multi = nullptr;
+    int64_t *item_off = nullptr, *slot_off = nullptr, *mrow_off = nullptr;
+    SrcBlockedItems sb;
+    sb.block_rows = block_rows;
+    sb.min_run = min_run;
+    sb.fit_rows = fit_rows;
+    auto cleanup = [&](bool all) {
+        cudaFree(count); cudaFree(slots); cudaFree(multi); cudaFree(item_off); cudaFree(slot_off); cudaFree(mrow_off);
+        if (all) { cudaFree(sb.item); cudaFree(sb.slot0); cudaFree(sb.tot); cudaFree(sb.mrows); }
+    };
+#define SB_TRY(expr)                       \
+    do {                                   \
+        sat_status s_ = (expr);            \
+        if (s_ != SAT_OK) {                \
+            cleanup(true);                 \
+            return s_;                     \
+        }                                  \
+    } while (0)
+#define SB_CUDA(call)                                                     \
+    do {                                                                  \
+        cudaError_t e_ = (call);                                          \
+        if (e_ != cudaSuccess) {                                          \
+            cleanup(true);                                                \
+            return sat_check_cuda(ctx, e_, #call);                        \
+        }                                                                 \
+    } while (0)
+    SB_CUDA(cudaMalloc((void **)&count, (size_t)(total + 1) * sizeof(int32_t)));
+    SB_CUDA(cudaMalloc((void **)&item_off, (size_t)(total + 2) * sizeof(int64_t)));
+    SB_CUDA(cudaMalloc((void **)&slots, (size_t)(n + 1) * sizeof(int32_t)));
+    SB_CUDA(cudaMalloc((void **)&multi, (size_t)(n + 1) * sizeof(int32_t)));
+    SB_CUDA(cudaMalloc((void **)&slot_off, (size_t)(n + 2) * sizeof(int64_t)));
+    SB_CUDA(cudaMalloc((void **)&mrow_off, (size_t)(n + 2) * sizeof(int64_t)));
+    SB_CUDA(cudaMalloc((void **)&sb.slot0, (size_t)(n + 1) * sizeof(int32_t)));
+    SB_CUDA(cudaMalloc((void **)&sb.tot, (size_t)(n + 1) * sizeof(int32_t)));
+    for (int m = 0; m < M; ++m) {
+        const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
+        if (rows == 0) continue;
+        k_sb_count<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
+                                                                                         nb[m], br[m], count + cbase[m]);
+        k_sb_row_totals<<<(unsigned)cdiv64(rows, 256), 256, 0, ctx->stream>>>(count + cbase[m], row0, rows, nb[m], sb.tot, slots, multi);
+    }
+    SAT_LAUNCHED(ctx);
+    SB_TRY(sat_scan_i32(ctx, count, total, item_off));
+    SB_TRY(sat_scan_i32(ctx, slots, n, slot_off));
+    SB_TRY(sat_scan_i32(ctx, multi, n, mrow_off));
+    int64_t n_items = 0, n_mrows = 0;
+    SB_TRY(sb_read_i64(ctx, item_off + total, &n_items));
+    SB_TRY(sb_read_i64(ctx, slot_off + n, &sb.n_slots));
+    SB_TRY(sb_read_i64(ctx, mrow_off + n, &n_mrows));
+    if (n_items >= ((int64_t)1 << 31) || sb.n_slots >= ((int64_t)1 << 31)) {
+        cleanup(true);
+        return sat_fail(ctx, SAT_EINVAL, "sat_spmm: too many source-blocked work items");
+    }
+    sb.n_items = (int32_t)n_items;
+    sb.n_mrows = (int32_t)n_mrows;
+    SB_CUDA(cudaMalloc((void **)&sb.item, (size_t)(n_items > 0 ? n_items : 1) * sizeof(int4)));
+    SB_CUDA(cudaMalloc((void **)&sb.mrows, (size_t)(n_mrows > 0 ? n_mrows : 1) * sizeof(int32_t)));
+    for (int m = 0; m < M; ++m) {
+        const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
+        if (rows == 0) continue;
+        k_sb_fill<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
+                                                                                        nb[m], br[m], count + cbase[m], item_off + cbase[m], sb.tot,
+                                                                                        slot_off, sb.item);
+    }
+    k_sb_rows<<<(unsigned)cdiv64(n > 0 ? n : 1, 256), 256, 0, ctx->stream>>>(slot_off, multi, mrow_off, n, sb.slot0, sb.mrows);
+    SAT_LAUNCHED(ctx);
+    sb.h_item_off.assign((size_t)M + 1, 0);
+    sb.h_mrow_off.assign((size_t)M + 1, 0);
+    sb.h_slot_off.assign((size_t)M + 1, 0);
+    for (int m = 0; m <= M; ++m) {
+        int64_t a = 0, b = 0, c = 0;
+        SB_TRY(sb_read_i64(ctx, item_off + cbase[m], &a));
+        SB_TRY(sb_read_i64(ctx, slot_off + ctx->h_inner_off[m], &b));
+        SB_TRY(sb_read_i64(ctx, mrow_off + ctx->h_inner_off[m], &c));
+        sb.h_item_off[m] = (int32_t)a;
+        sb.h_slot_off[m] = b;
+        sb.h_mrow_off[m] = (int32_t)c;
+    }
+    SB_CUDA(cudaStreamSynchronize(ctx->stream));
+#undef SB_TRY
+#undef SB_CUDA
+    cleanup(false);
+    ctx->src_blocked.push_back(std::move(sb));
+    *out = &ctx->src_blocked.back();
+    return SAT_OK;
+}
+
+// Source blocking is used for partitions whose sources exceed `fit` bytes and whose rows meet a block with a run of at least
+// `min_run` entries on average.  Defaults: blocks of 64 MiB, partitions from 192 MiB, runs from 8 entries; the environment
+// variable SAT_SPMM_SRC_BLOCK = "<block bytes>[,<fit bytes>[,<min run>]]" overrides them for a process (0 = never blocked).
+struct SbConfig {
+    int64_t block_rows, fit_rows, min_run;
+};
+static SbConfig sb_config(int32_t d4)
+{
+    int64_t block_bytes = (int64_t)64 << 20, fit_bytes = (int64_t)192 << 20, min_run = 8;
+    if (const char *e = getenv("SAT_SPMM_SRC_BLOCK")) {
+        char *end = nullptr;
+        block_bytes = strtoll(e, &end, 10);
+        fit_bytes = 3 * block_bytes;
+        if (end && *end == ',') fit_bytes = strtoll(end + 1, &end, 10);
+        if (end && *end == ',') min_run = strtoll(end + 1, &end, 10);
+    }
+    SbConfig c{0, 0, min_run};
+    if (block_bytes > 0) {
+        c.block_rows = std::max<int64_t>(64, block_bytes / ((int64_t)d4 * 16) / 64 * 64);
+        c.fit_rows = fit_bytes / ((int64_t)d4 * 16);
+    }
+    return c;
+}
+
+// partitions [a, b) of a view that covers whole partitions; true when at least one of them is source-blocked
+static bool sb_view_blocked(const sat_ctx *ctx, const PartView &v, const SbConfig &cfg, int *a, int *b)
+{
+    if (cfg.block_rows <= 0) return false;
+    *a = (int)(std::lower_bound(ctx->h_inner_off.begin(), ctx->h_inner_off.end(), v.row0) - ctx->h_inner_off.begin());
+    *b = (int)(std::lower_bound(ctx->h_inner_off.begin(), ctx->h_inner_off.end(), v.row0 + v.n_rows) - ctx->h_inner_off.begin());
+    if (*b > ctx->M || *a > *b || ctx->h_inner_off[*a] != v.row0 || ctx->h_inner_off[*b] != v.row0 + v.n_rows) return false;
+    for (int m = *a; m < *b; ++m)
+        if (sb_blocks_of(ctx, m, cfg.block_rows, cfg.fit_rows, cfg.min_run) > 1) return true;
+    return false;
+}
+
+template <int G, int NV>
+__global__ void __launch_bounds__(256, NV <= 2 ? 8 : 4)
+k_spmm_sb(const int4 *__restrict__ items, int32_t item0, int32_t n_items, int64_t slot_base, const int32_t *__restrict__ lenc,
+          const float *__restrict__ lw, const float *__restrict__ dinv_enc, int32_t n, int32_t d4, const float *__restrict__ in_base, int64_t ld_in,
+          const float *__restrict__ halo_base, int64_t ld_halo, float *__restrict__ out_base, int64_t ld_out, float *__restrict__ partial,
+          const uint32_t *__restrict__ omask, int32_t omask_words, DbgLimits dbg)
+{
+    const int lane = threadIdx.x & (G - 1);
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;
+    if (gid >= n_items) return;
+    const unsigned mask = group_mask<G>(threadIdx.x & 31);
+    const int col0 = blockIdx.y * (G * NV);
+    const int4 it = __ldg(items + item0 + gid);
+    const int32_t row = (int32_t)SAT_IDX(it.x, dbg.out_lo, dbg.out_hi, dbg.status);
+    const int64_t e0 = (int64_t)(uint32_t)it.z | ((int64_t)(it.w & 0xffff) << 32);
+    const int64_t e1 = e0 + (it.w >> 16);
+    float4 acc[NV];
+#pragma unroll
+    for (int v = 0; v < NV; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t eb = e0; eb < e1; eb += G) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float w = 0.f;
+        if (e < e1) {
+            c = __ldg(lenc + e);
+            w = __ldg(lw + e);
+        }
+        const int cnt = (e1 - eb) < G ? (int)(e1 - eb) : G;
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t cj = __shfl_sync(mask, c, j, G);
+            const float wj = __shfl_sync(mask, w, j, G);
+            const float *src = cj < n ? in_base + SAT_IDX((int64_t)cj, dbg.src_lo, dbg.src_hi, dbg.status) * ld_in
+                                      : halo_base + SAT_IDX((int64_t)(cj - n), dbg.halo_lo, dbg.halo_hi, dbg.status) * ld_halo;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int idx = col0 + lane + v * G;
+                if (idx < d4) fma4(acc[v], wj, ld4(src + 4 * idx));
+            }
+        }
+    }
+    if (it.y < 0) {
+        const float s = __ldg(dinv_enc + row);
+        float *o = out_base + (int64_t)row * ld_out;
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) {
+                float4 r = make_float4(s * acc[v].x, s * acc[v].y, s * acc[v].z, s * acc[v].w);
+                if (omask) mask4(r, omask, (int64_t)row * omask_words, idx);
+                *reinterpret_cast<float4 *>(o + 4 * idx) = r;
+            }
+        }
+    } else {
+        float *o = partial + ((int64_t)it.y - slot_base) * (4 * (int64_t)d4);
+#pragma unroll
+        for (int v = 0; v < NV; ++v) {
+            const int idx = col0 + lane + v * G;
+            if (idx < d4) *reinterpret_cast<float4 *>(o + 4 * idx) = acc[v];
+        }
+    }
+}
+
+// rows with several source-blocked items: add the partial sums in item order (block by block), scale, store
+__global__ void k_spmm_sb_fixup(const int32_t *__restrict__ mrows, int32_t mrow0, int32_t n_mrows, const int32_t *__restrict__ slot0,
+                                const int32_t *__restrict__ tot, int64_t slot_base, const float *__restrict__ dinv_enc, int32_t d4,
+                                const float *__restrict__ partial, float *__restrict__ out_base, int64_t ld_out,
+                                const uint32_t *__restrict__ omask, int32_t omask_words, DbgLimits dbg)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d4;
+    const int c = (int)(t - i * d4);
+    if (i >= n_mrows) return;
+    const int32_t row = (int32_t)SAT_IDX(mrows[mrow0 + i], dbg.out_lo, dbg.out_hi, dbg.status);
+    const int64_t s0 = (int64_t)slot0[row] - slot_base;
+    const int32_t cnt = tot[row];
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int32_t q = 0; q < cnt; ++q) {
+        const float4 x = *reinterpret_cast<const float4 *>(partial + ((s0 + q) * d4 + c) * 4);
+        a.x += x.x;
+        a.y += x.y;
+        a.z += x.z;
+        a.w += x.w;
+    }
+    const float s = dinv_enc[row];
+    float4 r = make_float4(s * a.x, s * a.y, s * a.z, s * a.w);
+    if (omask) mask4(r, omask, (int64_t)row * omask_words, c);
+    *reinterpret_cast<float4 *>(out_base + (int64_t)row * ld_out + 4 * c) = r;
+}
+
+template <int G, int NV>
+static void launch_sb(sat_ctx *ctx, const PartView &v, const SrcBlockedItems &sb, int32_t item0, int32_t n_items, int64_t slot_base, int32_t d4,
+                      const float *in_base, int32_t ld_in, const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial,
+                      const uint32_t *omask, int32_t omask_words, const int32_t *cols, DbgRange halo_range, DbgRange src_range)
+{
+    dim3 grid((unsigned)cdiv64((int64_t)n_items * G, 256), (unsigned)cdiv64(d4, G * NV));
+    k_spmm_sb<G, NV><<<grid, 256, 0, ctx->stream>>>(sb.item, item0, n_items, slot_base, cols, ctx->lw, ctx->dinv_enc, ctx->n, d4, in_base, ld_in,
+                                                     halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words,
+                                                     dbg_limits(src_range, halo_range, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
+}
+
 template <int G, int NV>
 static void launch_items(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d4, const float *in_base, int32_t ld_in,
                          const float *halo_base, int32_t ld_halo, float *out_base, int32_t ld_out, float *partial, const uint32_t *omask,
@@ -214,6 +570,44 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     const double n_ent = (double)(inner_only == 1 ? v.lnnz - v.hnnz : inner_only == 2 ? v.hnnz : v.lnnz);
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
                    4.0 * n_ent + 12.0 * v.n_rows + 4.0 * n_src + 4.0 * d * (n_src + v.n_rows), 2.0 * n_ent * d);
+    if (inner_only == 0) {
+        const SbConfig cfg = sb_config(d4);
+        int a = 0, b = 0;
+        const bool blocked = sb_view_blocked(ctx, v, cfg, &a, &b);
+        const int64_t block_rows = cfg.block_rows, fit_rows = cfg.fit_rows, min_run = cfg.min_run;
+        if (blocked) {
+            SrcBlockedItems *sb = nullptr;
+            SAT_TRY(sb_build(ctx, block_rows, fit_rows, min_run, &sb));
+            const int32_t item0 = sb->h_item_off[a], n_items = sb->h_item_off[b] - item0;
+            const int32_t mrow0 = sb->h_mrow_off[a], n_mrows = sb->h_mrow_off[b] - mrow0;
+            const int64_t slot_base = sb->h_slot_off[a], n_slots = sb->h_slot_off[b] - slot_base;
+            float *partial = nullptr;
+            if (n_slots > 0) {
+                SAT_TRY(sat_ensure(ctx, ctx->buf_sbpartial, (size_t)n_slots * d4 * 16));
+                partial = (float *)ctx->buf_sbpartial.p;
+            }
+#define ARGS ctx, v, *sb, item0, n_items, slot_base, d4, in_base, ld_in, halo_base, ld_halo, out_base, ld_out, partial, omask, omask_words, cols, halo_range, src_range
+            if (d4 <= 4) launch_sb<4, 1>(ARGS);
+            else if (d4 <= 8) launch_sb<8, 1>(ARGS);
+            else if (d4 <= 16) launch_sb<16, 1>(ARGS);
+            else if (d4 <= 32) launch_sb<8, 4>(ARGS);
+            else if (d4 <= 64) launch_sb<32, 2>(ARGS);
+            else if (d4 <= 96) launch_sb<32, 3>(ARGS);
+            else if (d4 <= 128) launch_sb<32, 4>(ARGS);
+            else if (d4 <= 160) launch_sb<32, 5>(ARGS);
+            else if (d4 <= 192) launch_sb<32, 6>(ARGS);
+            else launch_sb<32, 8>(ARGS);
+#undef ARGS
+            SAT_LAUNCHED(ctx);
+            if (n_mrows > 0) {
+                k_spmm_sb_fixup<<<(unsigned)cdiv64((int64_t)n_mrows * d4, 256), 256, 0, ctx->stream>>>(
+                    sb->mrows, mrow0, n_mrows, sb->slot0, sb->tot, slot_base, ctx->dinv_enc, d4, partial, out_base, ld_out, omask, omask_words,
+                    dbg_limits(DbgRange{0, 0}, DbgRange{0, 0}, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
+                SAT_LAUNCHED(ctx);
+            }
+            return SAT_OK;
+        }
+    }
     float *partial = nullptr;
     if (v.n_mitems > 0) {
         SAT_TRY(sat_ensure(ctx, ctx->buf_partial, (size_t)v.n_mitems * d4 * 16));
@@ -238,6 +632,29 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
             dbg_limits(DbgRange{0, 0}, DbgRange{0, 0}, DbgRange{v.row0, (int64_t)v.row0 + v.n_rows}, ctx->d_flag + 1));
         SAT_LAUNCHED(ctx);
     }
+    return SAT_OK;
+}
+
+extern "C" sat_status sat_spmm_plan(sat_ctx *ctx, int32_t part, int32_t d, int32_t *n_blocks, int64_t *n_items, int64_t *n_partial_rows)
+{
+    CHECK_CTX(ctx);
+    PartView v;
+    SAT_TRY(sat_part_view(ctx, part, &v));
+    if (d < 1) return sat_fail(ctx, SAT_EINVAL, "sat_spmm_plan: d = %d", d);
+    const SbConfig cfg = sb_config((d + 3) / 4);
+    int a = 0, b = 0;
+    int32_t nb = 1;
+    int64_t items = v.n_items, slots = v.n_mitems;
+    if (sb_view_blocked(ctx, v, cfg, &a, &b)) {
+        SrcBlockedItems *sb = nullptr;
+        SAT_TRY(sb_build(ctx, cfg.block_rows, cfg.fit_rows, cfg.min_run, &sb));
+        for (int m = a; m < b; ++m) nb = std::max<int32_t>(nb, (int32_t)sb_blocks_of(ctx, m, cfg.block_rows, cfg.fit_rows, cfg.min_run));
+        items = sb->h_item_off[b] - sb->h_item_off[a];
+        slots = sb->h_slot_off[b] - sb->h_slot_off[a];
+    }
+    if (n_blocks) *n_blocks = nb;
+    if (n_items) *n_items = items;
+    if (n_partial_rows) *n_partial_rows = slots;
     return SAT_OK;
 }
 

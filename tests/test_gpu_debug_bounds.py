@@ -34,6 +34,8 @@ def _child():
     cache = orc.CacheRing(P.n_slots, wl.dims[1:-1], wl.tau)
     ep = SatEpoch(wl.rowptr, wl.col, wl.M, wl.dims, wl.tau, wl.loss, part_given=wl.part_given)
     try:
+        if os.environ.get("SAT_TEST_EXPECT_BLOCKED"):
+            assert B.sat_spmm_plan(ep.ctx, B.SAT_ALL_PARTS, wl.dims[1])[0] > 1
         perm = np.concatenate(P.inner_gid)
         ep.set_inputs(dev2d(wl.X), dev(wl.labels[perm]))
         W, b = [dev(w) for w in wl.W], [dev(x) for x in wl.b]
@@ -73,10 +75,18 @@ def _child():
     print("debug-bounds child ok")
 
 
-def test_bounds_checking_build_on_the_small_cases():
+@pytest.mark.parametrize("source_blocked", [False, True])
+def test_bounds_checking_build_on_the_small_cases(source_blocked):
+    """source_blocked: the forward aggregation walks its source-blocked work list (forced: blocks of a few hundred
+    rows, every partition) instead of the row-by-row one, so that kernel's index checks run too."""
     from paper_2308_13466_b200.build import build
     build(debug=True)
     env = dict(os.environ, SAT_B200_DEBUG="1")
+    if source_blocked:
+        env["SAT_SPMM_SRC_BLOCK"] = "16384,16384,0"
+        env["SAT_TEST_EXPECT_BLOCKED"] = "1"
+    else:
+        env.pop("SAT_SPMM_SRC_BLOCK", None)
     out = subprocess.run([sys.executable, os.path.abspath(__file__), "--child"], cwd=ROOT, env=env, capture_output=True, text=True, timeout=900)
     assert out.returncode == 0 and "debug-bounds child ok" in out.stdout, out.stdout[-2000:] + out.stderr[-4000:]
 
