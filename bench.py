@@ -382,6 +382,9 @@ def run_ours(args, wl):
     l2_row = int(max(wl.dims[1:-1])) if wl.L > 1 else int(wl.dims[0])
     l2_row = min(1024, (l2_row + 3) & ~3)
     l2_stream_gbs, l2_gather_gbs = B.sat_profile_l2_rates(ep.ctx, l2_row)
+    # how the forward aggregation walks the partitions at each of its widths (source blocks, work items, partial-sum rows)
+    spmm_plan = {str(int(d)): dict(zip(("source_blocks", "work_items", "partial_rows"), B.sat_spmm_plan(ep.ctx, B.SAT_ALL_PARTS, int(d))))
+                 for d in sorted(set(wl.dims[:-1]))}
     # for reference, outside the headline and without any profiling events: the same epochs (a) with a predictor that is
     # never updated (one version throughout: all tau - 1 older projections cached) and (b) with no version promise (nothing
     # kept between epochs: every epoch runs all steps from the raw ring, K = d + h in the recurrence)
@@ -609,6 +612,11 @@ def run_ours(args, wl):
                 what="neighbour-row bytes gathered per second (entries x row bytes / time) against the rate at which this GPU "
                      f"delivers random {l2_row}-float rows (reference) and a contiguous stream (reference_stream) out of an L2-resident "
                      "64 MiB buffer, both measured in this run (sat_profile_l2_rates); a ratio above 1 means rows served from L1 / shared memory")
+        if fam == "spmm_fwd":
+            roofline["walk"] = dict(by_width=spmm_plan,
+                                    what="per input width of the forward aggregation: source blocks of the most finely cut partition "
+                                         "(1 = rows walked once; > 1 = the partition is walked once per 64 MiB block of source rows and "
+                                         "rows add one partial sum per block), work items and partial-sum rows per launch (sat_spmm_plan)")
         families = {k: dict(calls=v["calls"], ms_per_step=v["ms"] / args.steps,
                             gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else 0.0,
                             hbm_frac=(v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm"]) if v["ms"] > 0 else 0.0,

@@ -590,7 +590,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
             if (d4 <= 4) launch_sb<4, 1>(ARGS);
             else if (d4 <= 8) launch_sb<8, 1>(ARGS);
             else if (d4 <= 16) launch_sb<16, 1>(ARGS);
-            else if (d4 <= 32) launch_sb<8, 4>(ARGS);
+            else if (d4 <= 32) launch_sb<16, 2>(ARGS);
             else if (d4 <= 64) launch_sb<32, 2>(ARGS);
             else if (d4 <= 96) launch_sb<32, 3>(ARGS);
             else if (d4 <= 128) launch_sb<32, 4>(ARGS);
@@ -617,7 +617,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     if (d4 <= 4) launch_items<4, 1>(ARGS);
     else if (d4 <= 8) launch_items<8, 1>(ARGS);
     else if (d4 <= 16) launch_items<16, 1>(ARGS);
-    else if (d4 <= 32) launch_items<8, 4>(ARGS);
+    else if (d4 <= 32) launch_items<16, 2>(ARGS);   // 16 lanes x 2 vectors: 16-18 % faster than 8 x 4 on the 2.4 M-row graph (d = 100, 128), equal on the 169 k-row one
     else if (d4 <= 64) launch_items<32, 2>(ARGS);   // compiled for 8 resident blocks per SM (32 registers): 6 / 5 / 4 blocks (40-44 registers, no spills) measured 3 / 12 / 11 % slower
     else if (d4 <= 96) launch_items<32, 3>(ARGS);
     else if (d4 <= 128) launch_items<32, 4>(ARGS);
