@@ -90,3 +90,60 @@ def test_blocked_and_plain_walks_agree_and_the_plan_says_which_ran(B, monkeypatc
         assert np.array_equal(again.cpu().numpy(), plain.cpu().numpy())
     finally:
         B.sat_destroy(ctx)
+
+
+@pytest.mark.parametrize("kind", ["one_partition", "an_empty_partition", "random_assignment"])
+def test_degenerate_partitionings_with_the_blocked_walk(B, monkeypatch, kind):
+    """No halo rows at all (one partition: the blocks cut the inner rows alone), a partition without any node, and a random
+    assignment (nearly every entry has a halo column): blocked and plain walks agree, and under the blocked walk the
+    all-partition launch gives the bits of the per-partition calls."""
+    wl = make_workload("odd")
+    rng = np.random.default_rng(11)
+    if kind == "one_partition":
+        M, part = 1, np.zeros(wl.n, dtype=np.int32)
+    elif kind == "an_empty_partition":
+        M = 4
+        part = rng.integers(0, 3, wl.n).astype(np.int32)
+        part[part == 2] = 3                              # partition 2 owns nothing
+    else:
+        M, part = 5, rng.integers(0, 5, wl.n).astype(np.int32)
+    d, d_out = wl.dims[1], wl.dims[2]
+    ctx = B.sat_create(0, 0)
+    try:
+        B.sat_graph_load(ctx, wl.rowptr, wl.col)
+        B.sat_partition(ctx, M, B.SAT_PART_GIVEN, part)
+        B.sat_cache_init(ctx, wl.dims[1:-1], wl.tau)
+        sizes = [B.sat_part_sizes(ctx, m) for m in range(M)]
+        n_halo = sum(s[1] for s in sizes)
+        if kind == "one_partition":
+            assert n_halo == 0
+        h_in = dev2d(rng.standard_normal((wl.n, d)).astype(np.float32))
+        h_halo = dev2d(rng.standard_normal((max(n_halo, 1), d)).astype(np.float32))
+        W, b = dev(wl.W[1]), dev(wl.b[1])
+
+        def run(part_id, rows0, rows1, halo0, halo1):
+            out = empty2d(rows1 - rows0, d_out)
+            B.sat_layer_fwd(ctx, part_id, 2, h_in[rows0:rows1], h_halo[halo0:max(halo1, halo0 + 1)] if n_halo else h_halo,
+                            W, b, B.SAT_ACT_RELU, out)
+            return out.cpu().numpy()
+
+        monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", "0")
+        plain = run(B.SAT_ALL_PARTS, 0, wl.n, 0, n_halo)
+        monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", FORCED)
+        assert B.sat_spmm_plan(ctx, B.SAT_ALL_PARTS, d)[0] > 1
+        blocked = run(B.SAT_ALL_PARTS, 0, wl.n, 0, n_halo)
+        B.sat_sync_status(ctx)
+        assert np.max(np.abs(plain.astype(np.float64) - blocked)) <= 2e-6 * np.max(np.abs(plain))
+        r0 = h0 = 0
+        for m in range(M):
+            n_m, b_m = sizes[m][0], sizes[m][1]
+            if n_m:
+                got = run(m, r0, r0 + n_m, h0, h0 + b_m)
+                assert np.array_equal(got, blocked[r0:r0 + n_m]), f"partition {m} alone"
+            else:
+                assert B.sat_spmm_plan(ctx, m, d) == (1, 0, 0)
+            r0 += n_m
+            h0 += b_m
+        B.sat_sync_status(ctx)
+    finally:
+        B.sat_destroy(ctx)
