@@ -139,6 +139,7 @@ static void free_partition(sat_ctx *ctx)
     dev_free(&ctx->hlong);
     dev_free(&ctx->hchunk_first);
     dev_free(&ctx->hchunk_row);
+    dev_free(&ctx->halo_tile_order);
     ctx->n_hchunks = 0;
     dev_free(&ctx->first_item);
     dev_free(&ctx->item_row);

@@ -238,7 +238,16 @@ struct TcEpilogue {
     float *push_dst;     // (EPI_PUSH) row i is also written to push_dst + push_slot[i] * ld_push when push_slot[i] >= 0
     const int32_t *push_slot;
     int64_t ld_push;
+    const int32_t *tile_order;  // row tile walked at position i of the schedule (null: i itself)
 };
+
+// Row tile (of TC_BM rows) of schedule position t: the persistent CTAs walk positions blockIdx.x, blockIdx.x + gridDim.x, ...;
+// a permutation lets the caller choose which row tiles run at the same time (results do not depend on it).
+__device__ __forceinline__ int64_t tck_row_tile(const TcEpilogue &ep, int64_t t, int32_t n_tiles_n)
+{
+    const int64_t rt = t / n_tiles_n;
+    return ep.tile_order ? (int64_t)__ldg(ep.tile_order + rt) : rt;
+}
 
 struct TcShared {
     uint64_t full[4];       // TMA bytes of the stage have landed
@@ -346,7 +355,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (lane == 0) {
             uint32_t it = 0;
             for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-                const int32_t m0 = (int32_t)(t / n_tiles_n) * TC_BM;
+                const int32_t m0 = (int32_t)tck_row_tile(ep, t, n_tiles_n) * TC_BM;
                 const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
                 for (int32_t kb = 0; kb < nkb; ++kb, ++it) {
                     const int s = it % STAGES;
@@ -442,13 +451,13 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
             // called when the cursor enters tile pf_t; idx_now = gathered row index for this thread's row, or -1
             pf_srow = nullptr;
             if (pf_t < n_tiles) {
-                const int64_t prow = (pf_t / n_tiles_n) * TC_BM + q * 32 + lane;
+                const int64_t prow = tck_row_tile(ep, pf_t, n_tiles_n) * TC_BM + q * 32 + lane;
                 const int32_t pn0 = (int32_t)(pf_t % n_tiles_n) * bn;
                 if (EPI == EPI_RESID) {
                     if (prow < M && idx_now >= 0) pf_srow = ep.resid + (int64_t)idx_now * ep.ld_resid + pn0;  // rows padded to 4 floats
                     pf_lim = n4 - pn0;
                     const int64_t nt = pf_t + gridDim.x;
-                    const int64_t nrow = (nt / n_tiles_n) * TC_BM + q * 32 + lane;
+                    const int64_t nrow = tck_row_tile(ep, nt, n_tiles_n) * TC_BM + q * 32 + lane;
                     pf_idx_next = (nt < n_tiles && nrow < M) ? __ldg(ep.resid_idx + nrow) : -1;
                 } else {
                     if (prow < M) pf_srow = ep.addend + prow * ep.ld_addend + pn0;
@@ -475,7 +484,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
                     }
                 } else {
                     // dense side operand: rows of the tile are ld_addend apart
-                    const int64_t prow0 = (pf_t / n_tiles_n) * TC_BM + q * 32 + (lane >> 3);
+                    const int64_t prow0 = tck_row_tile(ep, pf_t, n_tiles_n) * TC_BM + q * 32 + (lane >> 3);
                     const float *p0 = base + prow0 * ep.ld_addend + (int32_t)(pf_t % n_tiles_n) * bn + pf_c + 4 * piece;
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
@@ -497,7 +506,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
         if (RING > 0 && c_first < bn) {
             int32_t idx0 = -1;
             if (EPI == EPI_RESID && pf_t < n_tiles) {
-                const int64_t prow = (pf_t / n_tiles_n) * TC_BM + q * 32 + lane;
+                const int64_t prow = tck_row_tile(ep, pf_t, n_tiles_n) * TC_BM + q * 32 + lane;
                 if (prow < M) idx0 = __ldg(ep.resid_idx + prow);
             }
             pf_enter_tile(idx0);
@@ -507,7 +516,7 @@ k_gemm_tc_k(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CU
 
         uint32_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
-            const int64_t m0 = (t / n_tiles_n) * TC_BM;
+            const int64_t m0 = tck_row_tile(ep, t, n_tiles_n) * TC_BM;
             const int32_t n0 = (int32_t)(t % n_tiles_n) * bn;
             const uint32_t buf = lt & 1u;
             const int64_t row = m0 + q * 32 + lane;
@@ -1132,6 +1141,7 @@ sat_status sat_gemm_tc(sat_ctx *ctx, int64_t m, int32_t n, const float *A, int32
     ep.resid = eh.resid;
     ep.resid_idx = eh.resid_idx;
     ep.ld_resid = eh.ld_resid;
+    ep.tile_order = eh.tile_order;
     const int32_t n_tiles_n = (int32_t)cdiv64(n, bn);
     const int64_t n_tiles = cdiv64(m, TC_BM) * n_tiles_n;
     int sms = 148;

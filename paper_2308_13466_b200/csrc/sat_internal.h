@@ -190,6 +190,7 @@ struct sat_ctx {
     // the long halo rows cut into chunks of SAT_HROW_CHUNK entries (a hub next to most of a partition has tens of thousands)
     int64_t *hchunk_first = nullptr; // [n_hlong+1] first chunk of every long row
     int32_t *hchunk_row = nullptr;   // [n_hchunks] index into hlong[] of the row a chunk belongs to
+    int32_t *halo_tile_order = nullptr;  // [ceil(n_halo / 128)] tiles of 128 halo rows ordered by the cache slot of their first row (built on first use)
     int32_t n_hchunks = 0;
     std::vector<int32_t> h_hchunk_off;  // [M+1] first chunk of every partition
     // SpMM work items (rows cut into chunks of SAT_SPMM_CHUNK edges)
@@ -433,6 +434,9 @@ struct TcEpilogueHost {
     const float *resid = nullptr;      // C += resid[resid_idx[i]] (row gather)
     const int32_t *resid_idx = nullptr;
     int32_t ld_resid = 0;
+    // order in which the persistent kernel walks the tiles of 128 rows: [ceil(m / 128)] row-tile indices, a permutation
+    // (null: ascending).  Results do not depend on it; it decides which rows are in flight together.
+    const int32_t *tile_order = nullptr;
     // fused LSTM cell (the weights must have been packed with gate interleave): the n = 4h outputs of a row are the gate
     // pre-activations; the epilogue applies c = f c + i g, s = o tanh(c) and writes s to C [m x h] and c to lstm_c [m x h]
     int32_t lstm_h = 0;

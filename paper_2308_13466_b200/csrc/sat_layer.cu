@@ -4,6 +4,10 @@
 
 #include "sat_internal.h"
 
+#include <algorithm>
+#include <cstdlib>
+#include <vector>
+
 
 template <typename T>
 static sat_status dev_realloc(sat_ctx *ctx, T **p, int64_t count)
@@ -518,6 +522,44 @@ static sat_status run_lstm(sat_ctx *ctx, CacheLayer *c, const sat_pred_params *p
     return SAT_OK;
 }
 
+// Schedule of the predictor-output contraction over the halo rows of all partitions: tiles of 128 rows ordered by the
+// cache slot of their first row.  Every partition's halo list is sorted by node id, hence by slot, so a tile covers a
+// narrow slot range; walking the tiles of all partitions in slot order puts the (on average 3-4) halo copies of a cached
+// node in flight together, and its newest-snapshot row — the skip connection the epilogue gathers — is read from DRAM once
+// instead of once per copy.
+__global__ void k_tile_keys(const int32_t *__restrict__ halo_slot, int64_t n_halo, int64_t n_tiles, int32_t *__restrict__ keys)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < n_tiles) keys[t] = halo_slot[t * 128 < n_halo ? t * 128 : n_halo - 1];
+}
+
+static sat_status halo_tile_order(sat_ctx *ctx, int64_t n_halo, const int32_t **out)
+{
+    if (!ctx->halo_tile_order) {
+        const int64_t n_tiles = cdiv64(n_halo, 128);
+        int32_t *d = nullptr;
+        SAT_CUDA(ctx, cudaMalloc((void **)&d, (size_t)n_tiles * sizeof(int32_t)));
+        k_tile_keys<<<(unsigned)cdiv64(n_tiles, 256), 256, 0, ctx->stream>>>(ctx->halo_slot, n_halo, n_tiles, d);
+        std::vector<int32_t> keys((size_t)n_tiles), order((size_t)n_tiles);
+        cudaError_t e = cudaMemcpyAsync(keys.data(), d, (size_t)n_tiles * sizeof(int32_t), cudaMemcpyDeviceToHost, ctx->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+        if (e == cudaSuccess) {
+            for (int64_t t = 0; t < n_tiles; ++t) order[(size_t)t] = (int32_t)t;
+            std::stable_sort(order.begin(), order.end(), [&](int32_t x, int32_t y) { return keys[(size_t)x] < keys[(size_t)y]; });
+            e = cudaMemcpyAsync(d, order.data(), (size_t)n_tiles * sizeof(int32_t), cudaMemcpyHostToDevice, ctx->stream);
+        }
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+        if (e != cudaSuccess) {
+            cudaFree(d);
+            return sat_check_cuda(ctx, e, "halo_tile_order");
+        }
+        SAT_LAUNCHED(ctx);
+        ctx->halo_tile_order = d;
+    }
+    *out = ctx->halo_tile_order;
+    return SAT_OK;
+}
+
 extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, const sat_pred_params *params, int reuse_state,
                                   float *halo_out, int32_t ld_out)
 {
@@ -582,6 +624,12 @@ extern "C" sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, con
             eh.resid = newest;
             eh.resid_idx = ctx->halo_slot + v.halo0;
             eh.ld_resid = c->ld;
+            // all partitions at once and a snapshot several times the L2: walk the row tiles in slot order
+            const bool all = v.halo0 == 0 && v.n_halo == ctx->h_halo_off[ctx->M];
+            // (SAT_PRED_TILE_ORDER in the environment: 0 = never, 1 = whenever all partitions run at once)
+            const char *force = getenv("SAT_PRED_TILE_ORDER");
+            const bool pays = v.n_halo > ctx->n_slots && (size_t)ctx->n_slots * c->ld * sizeof(float) > ((size_t)128 << 20);
+            if (all && v.n_halo > 0 && (force ? atoi(force) != 0 : pays)) SAT_TRY(halo_tile_order(ctx, v.n_halo, &eh.tile_order));
         }
         return sat_gemm_tc(ctx, v.n_halo, d, a, ld_a, h, nullptr, 0, 0, Wg, eh, SATK_GEMM_SIDE);
     }

@@ -493,3 +493,31 @@ def test_push_from_the_layer_transform_equals_the_separate_push(B, name, shrink)
     assert np.abs(rings[0]).max() > 0
     for r, o in zip(rings[1:], outs[1:]):
         assert np.array_equal(r, rings[0]) and np.array_equal(o, outs[0])
+
+
+@pytest.mark.parametrize("name,shrink", [("medium", 8), ("odd", 1), ("tiny", 1)])
+def test_predictor_output_walks_its_row_tiles_in_slot_order(B, monkeypatch, name, shrink):
+    """The output contraction of sat_predict over the halo rows of all partitions may walk its tiles of 128 rows in the
+    order of their cache slots (so that the halo copies of a node read its newest snapshot row together; chosen by the
+    library when the snapshot is several times the L2, forced here): every row is computed as before, so the predicted
+    rows are bit-identical to the ascending walk, and both agree with the oracle."""
+    wl = make_workload(name, shrink=shrink)
+    case = Case(B, wl, wl.tau + 1)
+    try:
+        res = orc.run_epoch(case.P, case.dtil, case.cache, wl.X, wl.labels, wl.W, wl.b, wl.pred, wl.loss,
+                            parts=list(range(wl.M)))          # a subset run: the oracle's ring is not committed
+        preds = pred_to_device(wl.pred, B)
+        nb = sum(h.shape[0] for h in case.P.halo_gid)
+        for l in range(1, wl.L):
+            want = np.concatenate([res.per_part[m]["halo"][l] for m in range(wl.M)])
+            outs = []
+            for order in ("0", "1"):
+                monkeypatch.setenv("SAT_PRED_TILE_ORDER", order)
+                out = empty2d(nb, wl.dims[l])
+                B.sat_predict(case.ctx, l, B.SAT_ALL_PARTS, preds[l - 1], 0, out)
+                outs.append(out.cpu().numpy())
+                assert_close(outs[-1], want, f"predicted rows, layer {l}, tile order {order}")
+            assert np.array_equal(outs[0], outs[1])
+        B.sat_sync_status(case.ctx)
+    finally:
+        case.close()
