@@ -593,7 +593,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
             else if (d4 <= 8) launch_sb<8, 1>(ARGS);
             else if (d4 <= 16) launch_sb<16, 1>(ARGS);
             else if (d4 <= 32) launch_sb<16, 2>(ARGS);
-            else if (d4 <= 64) launch_sb<32, 2>(ARGS);
+            else if (d4 <= 64) launch_sb<32, 2>(ARGS);   // 8 resident blocks per SM; 6 / 5 blocks (38-40 registers, no spills, loop unrolled 4-8x): 10-20 % slower here too
             else if (d4 <= 96) launch_sb<32, 3>(ARGS);
             else if (d4 <= 128) launch_sb<32, 4>(ARGS);
             else if (d4 <= 160) launch_sb<32, 5>(ARGS);
