@@ -208,6 +208,10 @@ typedef struct sat_pred_params {
  *                this layer (caller guarantees parameters and ring are unchanged;
  *                SAT_ESTATE if there is none since the last commit).
  *   halo_out     DEVICE [b_m x ld_out] (part = SAT_ALL_PARTS: [sum_m b_m x ld_out]).
+ * Every predicted row is computed independently of the others, so the order in which the rows are worked on does not
+ * change a bit of the result; with part = SAT_ALL_PARTS and a snapshot above 128 MiB the output step walks its tiles of
+ * 128 rows in the order of their cache slots (the halo copies of a node then read its newest row together).  The
+ * environment variable SAT_PRED_TILE_ORDER=0 / 1 forces that order off / on for the process.
  * ------------------------------------------------------------------------------------- */
 sat_status sat_predict(sat_ctx *ctx, int32_t layer, int32_t part, const sat_pred_params *params, int reuse_state,
                        float *halo_out, int32_t ld_out);

@@ -147,3 +147,21 @@ def test_degenerate_partitionings_with_the_blocked_walk(B, monkeypatch, kind):
         B.sat_sync_status(ctx)
     finally:
         B.sat_destroy(ctx)
+
+
+def test_plan_query_errors(B):
+    wl = make_workload("tiny")
+    ctx = B.sat_create(0, 0)
+    try:
+        B.sat_graph_load(ctx, wl.rowptr, wl.col)
+        with pytest.raises(B.SatError) as ei:                 # no partition yet
+            B.sat_spmm_plan(ctx, B.SAT_ALL_PARTS, 16)
+        assert ei.value.status == B.SAT_ESTATE
+        B.sat_partition(ctx, wl.M, B.SAT_PART_GIVEN, wl.part_given)
+        for bad_part, bad_d in ((wl.M, 16), (-7, 16), (0, 0), (0, -4)):
+            with pytest.raises(B.SatError) as ei:
+                B.sat_spmm_plan(ctx, bad_part, bad_d)
+            assert ei.value.status == B.SAT_EINVAL
+        assert B.sat_spmm_plan(ctx, 0, 16)[0] == 1          # usable after the refusals
+    finally:
+        B.sat_destroy(ctx)
