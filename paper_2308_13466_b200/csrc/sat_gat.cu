@@ -234,6 +234,57 @@ __global__ void k_gat_dmask(const float *__restrict__ g, int64_t ld_g, const flo
     D[r * ld_d + c] = (!h_out || h_out[r * ld_h + c] > 0.f) ? x : 0.f;
 }
 
+// Column-side walk shared by the three kernels below: entries e_first, e_first + stride, ... (< e_end) of an index list of
+// rows v that hold node u.  The lanes fetch the row scalars of 32 entries at a time — one exponential per entry instead of
+// one per lane and entry — and then walk those entries together, lanes over the columns, four rows in flight.
+//   acc += alpha_vu D_v,   returns sum_v alpha_vu slope_vu (D_v . z_u - t_v), the same on every lane
+// ds_src is linear in the dot products, so every lane keeps its own share and the warp is reduced once at the end (the
+// first version reduced every dot product across the warp: ten dependent shuffles per entry).
+template <int NV>
+__device__ __forceinline__ double gat_cols_walk(const int32_t *__restrict__ idx, int64_t e_first, int64_t e_end, int64_t stride, float su,
+                                                const float *__restrict__ s_dst, const float *__restrict__ lse, const double *__restrict__ t_in,
+                                                const float *__restrict__ D, int64_t ld_d, int32_t d, int d4, int lane, const float4 (&zu)[NV],
+                                                float4 (&acc)[NV])
+{
+    double dss = 0.0, tss = 0.0;
+    for (int64_t eb = e_first; eb < e_end; eb += 32 * stride) {
+        const int64_t e = eb + lane * stride;
+        int32_t v_row = 0;
+        float al = 0.f, as = 0.f;
+        if (e < e_end) {
+            v_row = idx[e];
+            const float pre = s_dst[v_row] + su;
+            al = expf(lrelu(pre) - lse[v_row]);
+            as = al * (pre > 0.f ? 1.f : GAT_SLOPE);
+            tss += (double)as * t_in[v_row];
+        }
+        const int64_t left = (e_end - eb + stride - 1) / stride;
+        const int cnt = left < 32 ? (int)left : 32;
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t vj = __shfl_sync(0xffffffffu, v_row, j);
+            const float aj = __shfl_sync(0xffffffffu, al, j);
+            const float asj = __shfl_sync(0xffffffffu, as, j);
+            const float *dr = D + (int64_t)vj * ld_d;
+            double p = 0.0;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c4 = lane + 32 * v;
+                if (c4 < d4) {
+                    const float4 x = ldz(dr, c4, d);
+                    p += ddot4(x, zu[v]);
+                    acc[v].x = fmaf(aj, x.x, acc[v].x);
+                    acc[v].y = fmaf(aj, x.y, acc[v].y);
+                    acc[v].z = fmaf(aj, x.z, acc[v].z);
+                    acc[v].w = fmaf(aj, x.w, acc[v].w);
+                }
+            }
+            dss += (double)asj * p;
+        }
+    }
+    return warp_sum_d(dss) - warp_sum_d(tss);
+}
+
 // backward, column side: one warp per node u keeps z_u in registers and walks the rows v that have u as an entry:
 //   HALO = 0: u is inner row `row0 + w`, the v are the inner prefix of its own row (symmetric block, self entry included);
 //   HALO = 1: u is halo position `halo0 + w`, the v are its halo-row CSR entries.
@@ -261,29 +312,7 @@ k_gat_bwd_cols(const int64_t *__restrict__ ptr, const int32_t *__restrict__ idx,
     const int64_t e0 = ptr[u], e1 = HALO ? ptr[u + 1] : e0 + inner_cnt[u];
     if (HALO && e1 - e0 > SAT_HROW_LONG) return;   // long halo rows: k_gat_bwd_cols_long, a thread block each
     const float su = s_u[u];
-    double dss = 0.0;
-    for (int64_t e = e0; e < e1; ++e) {
-        const int32_t v_row = idx[e];
-        const float pre = s_dst[v_row] + su;
-        const float alpha = expf(lrelu(pre) - lse[v_row]);
-        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
-        const float *dr = D + (int64_t)v_row * ld_d;
-        double p = 0.0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c4 = lane + 32 * v;
-            if (c4 < d4) {
-                const float4 x = ldz(dr, c4, d);
-                p += ddot4(x, zu[v]);
-                acc[v].x = fmaf(alpha, x.x, acc[v].x);
-                acc[v].y = fmaf(alpha, x.y, acc[v].y);
-                acc[v].z = fmaf(alpha, x.z, acc[v].z);
-                acc[v].w = fmaf(alpha, x.w, acc[v].w);
-            }
-        }
-        const double da = warp_sum_d(p);
-        dss += (double)(alpha * slope) * (da - t_in[v_row]);
-    }
+    const double dss = gat_cols_walk<NV>(idx, e0, e1, 1, su, s_dst, lse, t_in, D, ld_d, d, d4, lane, zu, acc);
     const float dsd = HALO ? 0.f : ds_dst[u];
     const float dssf = (float)dss;
     float *o = dz_base + u * ld_z;
@@ -334,25 +363,44 @@ k_gat_bwd_rows_items(const int64_t *__restrict__ lrowptr, const int32_t *__restr
     const int64_t e0 = lrowptr[row] + (int64_t)(item - first_item[row]) * SAT_SPMM_CHUNK;
     const int64_t e1 = e0 + SAT_SPMM_CHUNK < re ? e0 + SAT_SPMM_CHUNK : re;
     const float sd = s_dst[row], l = lse[row];
+    // the lanes fetch the scalars of 32 entries at a time (one exponential per entry), then the warp walks those entries
+    // together; t_v and ds_dst are linear in the dot products D_v . z_u, so the lanes keep their shares and the warp is reduced
+    // once per item
     double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
-    for (int64_t e = e0; e < e1; ++e) {
-        const int32_t c = lenc[e];
-        const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
-        const float alpha = expf(lrelu(pre) - l);
-        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
-        const float *src = c < n ? z_in + (int64_t)c * ld_z : z_halo + (int64_t)(c - n) * ld_z;
-        double p = 0.0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c4 = lane + 32 * v;
-            if (c4 < d4) p += ddot4(dv[v], ldz(src, c4, d));
+    for (int64_t eb = e0; eb < e1; eb += 32) {
+        const int64_t e = eb + lane;
+        int32_t c = 0;
+        float al = 0.f, as = 0.f;
+        if (e < e1) {
+            c = lenc[e];
+            const float pre = sd + (c < n ? s_in[c] : s_halo[c - n]);
+            const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
+            al = expf(lrelu(pre) - l);
+            as = al * slope;
+            a0 += (double)al;
+            a3 += (double)al * (double)slope;
         }
-        const double da = warp_sum_d(p);
-        a0 += (double)alpha;
-        a1 += (double)alpha * da;
-        a2 += (double)(alpha * slope) * da;
-        a3 += (double)alpha * (double)slope;
+        const int cnt = (e1 - eb) < 32 ? (int)(e1 - eb) : 32;
+#pragma unroll 4
+        for (int j = 0; j < cnt; ++j) {
+            const int32_t cj = __shfl_sync(0xffffffffu, c, j);
+            const float aj = __shfl_sync(0xffffffffu, al, j);
+            const float asj = __shfl_sync(0xffffffffu, as, j);
+            const float *src = cj < n ? z_in + (int64_t)cj * ld_z : z_halo + (int64_t)(cj - n) * ld_z;
+            double p = 0.0;
+#pragma unroll
+            for (int v = 0; v < NV; ++v) {
+                const int c4 = lane + 32 * v;
+                if (c4 < d4) p += ddot4(dv[v], ldz(src, c4, d));
+            }
+            a1 += (double)aj * p;
+            a2 += (double)asj * p;
+        }
     }
+    a0 = warp_sum_d(a0);
+    a1 = warp_sum_d(a1);
+    a2 = warp_sum_d(a2);
+    a3 = warp_sum_d(a3);
     if (lane == 0) {
         double *o = part4 + 4 * w;
         o[0] = a0;
@@ -406,29 +454,7 @@ k_gat_bwd_cols_items(const int64_t *__restrict__ lrowptr, const int32_t *__restr
     const int64_t e0 = rb + (int64_t)(item - first_item[u]) * SAT_SPMM_CHUNK;
     const int64_t e1 = e0 + SAT_SPMM_CHUNK < re ? e0 + SAT_SPMM_CHUNK : re;
     const float su = s_in[u];
-    double dss = 0.0;
-    for (int64_t e = e0; e < e1; ++e) {
-        const int32_t v_row = lenc[e];
-        const float pre = s_dst[v_row] + su;
-        const float alpha = expf(lrelu(pre) - lse[v_row]);
-        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
-        const float *dr = D + (int64_t)v_row * ld_d;
-        double p = 0.0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c4 = lane + 32 * v;
-            if (c4 < d4) {
-                const float4 x = ldz(dr, c4, d);
-                p += ddot4(x, zu[v]);
-                acc[v].x = fmaf(alpha, x.x, acc[v].x);
-                acc[v].y = fmaf(alpha, x.y, acc[v].y);
-                acc[v].z = fmaf(alpha, x.z, acc[v].z);
-                acc[v].w = fmaf(alpha, x.w, acc[v].w);
-            }
-        }
-        const double da = warp_sum_d(p);
-        dss += (double)(alpha * slope) * (da - t_in[v_row]);
-    }
+    const double dss = gat_cols_walk<NV>(lenc, e0, e1, 1, su, s_dst, lse, t_in, D, ld_d, d, d4, lane, zu, acc);
     float *o = pdz + w * ld_z;
 #pragma unroll
     for (int v = 0; v < NV; ++v) {
@@ -493,29 +519,7 @@ k_gat_bwd_cols_long(const int32_t *__restrict__ hlong, int32_t hlong0, const int
     }
     const int64_t e0 = ptr[u], e1 = ptr[u + 1];
     const float su = s_halo[u];
-    double dss = 0.0;
-    for (int64_t e = e0 + warp; e < e1; e += 8) {
-        const int32_t v_row = idx[e];
-        const float pre = s_dst[v_row] + su;
-        const float alpha = expf(lrelu(pre) - lse[v_row]);
-        const float slope = pre > 0.f ? 1.f : GAT_SLOPE;
-        const float *dr = D + (int64_t)v_row * ld_d;
-        double p = 0.0;
-#pragma unroll
-        for (int v = 0; v < NV; ++v) {
-            const int c4 = lane + 32 * v;
-            if (c4 < d4) {
-                const float4 x = ldz(dr, c4, d);
-                p += ddot4(x, zu[v]);
-                acc[v].x = fmaf(alpha, x.x, acc[v].x);
-                acc[v].y = fmaf(alpha, x.y, acc[v].y);
-                acc[v].z = fmaf(alpha, x.z, acc[v].z);
-                acc[v].w = fmaf(alpha, x.w, acc[v].w);
-            }
-        }
-        const double da = warp_sum_d(p);
-        dss += (double)(alpha * slope) * (da - t_in[v_row]);
-    }
+    const double dss = gat_cols_walk<NV>(idx, e0 + warp, e1, 8, su, s_dst, lse, t_in, D, ld_d, d, d4, lane, zu, acc);
 #pragma unroll
     for (int v = 0; v < NV; ++v) red[warp][v][lane] = acc[v];
     if (lane == 0) red_s[warp] = dss;
