@@ -495,9 +495,10 @@ sat_status sat_profile_read(sat_ctx *ctx, int32_t family, const char **name, int
  * the same whether the partition is run alone or with all others).  HOST outputs, each may be NULL: `n_blocks` = source
  * blocks of the most finely cut partition (1 = plain row-by-row walk), `n_items` = work items of the launch,
  * `n_partial_rows` = partial-sum rows of width d it writes and re-reads.  The cut is chosen per width (blocks of 64 MiB of
- * source rows, for partitions above 192 MiB whose rows meet a block with 8 or more entries on average); the environment
- * variable SAT_SPMM_SRC_BLOCK="<block bytes>[,<from bytes>[,<entries>]]" overrides the three figures for the process
- * ("0" = never).  Builds the work list on first use (device memory, freed with the partition); synchronises the stream.
+ * source rows, for partitions above 192 MiB whose rows meet a block with 8 or more entries on average; inside such a
+ * partition a short row is walked in groups of consecutive blocks, at least 32 entries per group, so that it leaves few
+ * partial sums); the environment variable SAT_SPMM_SRC_BLOCK="<block bytes>[,<from bytes>[,<entries>[,<entries per row
+ * group>]]]" overrides the four figures for the process ("0" = never).  Builds the work list on first use (device memory, freed with the partition); synchronises the stream.
  * Errors: SAT_ESTATE without a partition, SAT_EINVAL for a bad `part` or d < 1. */
 sat_status sat_spmm_plan(sat_ctx *ctx, int32_t part, int32_t d, int32_t *n_blocks, int64_t *n_items, int64_t *n_partial_rows);
 

@@ -167,25 +167,36 @@ __device__ __forceinline__ int64_t sb_source_col(int64_t p, int32_t row0, int32_
     return p < n_rows ? (int64_t)row0 + p : (int64_t)n + halo0 + (p - n_rows);
 }
 
-// entries [lo, hi) of `row` whose source falls into block j
+// The run of entries [lo, hi) of `row` that is walked with block j, or an empty run.  A row of `len` entries is cut into
+// G = min(blocks, len / min_run) groups of consecutive blocks (a short row would otherwise leave a partial sum per block for
+// a handful of entries each): group g covers blocks [ceil(g B / G), ceil((g + 1) B / G)) and its run is walked with the
+// first of them.
 __device__ __forceinline__ void sb_run(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row, int32_t j,
-                                       int32_t n_blocks, int64_t block_rows, int32_t row0, int32_t n_rows, int32_t n, int64_t halo0,
-                                       int64_t *lo, int64_t *hi)
+                                       int32_t n_blocks, int64_t block_rows, int32_t min_run, int32_t row0, int32_t n_rows, int32_t n,
+                                       int64_t halo0, int64_t *lo, int64_t *hi)
 {
     const int64_t rb = lrowptr[row], re = lrowptr[row + 1];
+    int64_t G = min_run > 0 ? (re - rb) / min_run : n_blocks;
+    G = G < 1 ? 1 : G > n_blocks ? n_blocks : G;
+    const int64_t g = (int64_t)j * G / n_blocks;
+    const int64_t j_first = (g * n_blocks + G - 1) / G, j_next = ((g + 1) * n_blocks + G - 1) / G;
+    if (j != j_first) {
+        *lo = *hi = rb;
+        return;
+    }
     *lo = j == 0 ? rb : lower_bound_col(lenc, rb, re, sb_source_col((int64_t)j * block_rows, row0, n_rows, n, halo0));
-    *hi = j == n_blocks - 1 ? re : lower_bound_col(lenc, *lo, re, sb_source_col((int64_t)(j + 1) * block_rows, row0, n_rows, n, halo0));
+    *hi = j_next >= n_blocks ? re : lower_bound_col(lenc, *lo, re, sb_source_col(j_next * block_rows, row0, n_rows, n, halo0));
 }
 
 // count[j * n_rows + r] = items of row row0 + r in block j
 __global__ void k_sb_count(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
-                           int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t *__restrict__ count)
+                           int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, int32_t *__restrict__ count)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= (int64_t)n_rows * n_blocks) return;
     const int32_t j = (int32_t)(t / n_rows), r = (int32_t)(t - (int64_t)j * n_rows);
     int64_t lo, hi;
-    sb_run(lrowptr, lenc, row0 + r, j, n_blocks, block_rows, row0, n_rows, n, halo0, &lo, &hi);
+    sb_run(lrowptr, lenc, row0 + r, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
     count[t] = (int32_t)((hi - lo + SAT_SPMM_CHUNK - 1) / SAT_SPMM_CHUNK);
 }
 
@@ -202,7 +213,7 @@ __global__ void k_sb_row_totals(const int32_t *__restrict__ count, int32_t row0,
 }
 
 __global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
-                          int64_t halo0, int32_t n_blocks, int64_t block_rows, const int32_t *__restrict__ count,
+                          int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, const int32_t *__restrict__ count,
                           const int64_t *__restrict__ item_off, const int32_t *__restrict__ tot, const int64_t *__restrict__ slot_off,
                           int4 *__restrict__ item)
 {
@@ -213,7 +224,7 @@ __global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__
     if (c == 0) return;
     const int32_t row = row0 + r;
     int64_t lo, hi;
-    sb_run(lrowptr, lenc, row, j, n_blocks, block_rows, row0, n_rows, n, halo0, &lo, &hi);
+    sb_run(lrowptr, lenc, row, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
     int32_t before = 0;
     for (int32_t q = 0; q < j; ++q) before += count[(int64_t)q * n_rows + r];
     const bool multi = tot[row] > 1;
@@ -254,10 +265,10 @@ static int64_t sb_blocks_of(const sat_ctx *ctx, int m, int64_t block_rows, int64
     return entries / (rows * B) >= min_run ? B : 1;
 }
 
-static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, int64_t min_run, SrcBlockedItems **out)
+static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, int64_t min_run, int64_t row_run, SrcBlockedItems **out)
 {
     for (SrcBlockedItems &sb : ctx->src_blocked)
-        if (sb.block_rows == block_rows && sb.min_run == min_run && sb.fit_rows == fit_rows) {
+        if (sb.block_rows == block_rows && sb.min_run == min_run && sb.fit_rows == fit_rows && sb.row_run == row_run) {
             *out = &sb;
             return SAT_OK;
         }
@@ -273,12 +284,14 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
         cbase[m + 1] = cbase[m] + rows * B;
     }
     const int64_t total = cbase[M];
+    const int32_t row_min_run = (int32_t)(row_run < 0 ? 0 : row_run > (1 << 20) ? (1 << 20) : row_run);   // per-row grouping of blocks (sb_run)
     int32_t *count = nullptr, *slots = nullptr, *multi = nullptr;
     int64_t *item_off = nullptr, *slot_off = nullptr, *mrow_off = nullptr;
     SrcBlockedItems sb;
     sb.block_rows = block_rows;
     sb.min_run = min_run;
     sb.fit_rows = fit_rows;
+    sb.row_run = row_run;
     auto cleanup = [&](bool all) {
         cudaFree(count); cudaFree(slots); cudaFree(multi); cudaFree(item_off); cudaFree(slot_off); cudaFree(mrow_off);
         if (all) { cudaFree(sb.item); cudaFree(sb.slot0); cudaFree(sb.tot); cudaFree(sb.mrows); }
@@ -311,7 +324,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
         const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
         if (rows == 0) continue;
         k_sb_count<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
-                                                                                         nb[m], br[m], count + cbase[m]);
+                                                                                         nb[m], br[m], row_min_run, count + cbase[m]);
         k_sb_row_totals<<<(unsigned)cdiv64(rows, 256), 256, 0, ctx->stream>>>(count + cbase[m], row0, rows, nb[m], sb.tot, slots, multi);
     }
     SAT_LAUNCHED(ctx);
@@ -334,7 +347,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
         const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
         if (rows == 0) continue;
         k_sb_fill<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
-                                                                                        nb[m], br[m], count + cbase[m], item_off + cbase[m], sb.tot,
+                                                                                        nb[m], br[m], row_min_run, count + cbase[m], item_off + cbase[m], sb.tot,
                                                                                         slot_off, sb.item);
     }
     k_sb_rows<<<(unsigned)cdiv64(n > 0 ? n : 1, 256), 256, 0, ctx->stream>>>(slot_off, multi, mrow_off, n, sb.slot0, sb.mrows);
@@ -361,22 +374,27 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
 }
 
 // Source blocking is used for partitions whose sources exceed `fit` bytes and whose rows meet a block with a run of at least
-// `min_run` entries on average.  Defaults: blocks of 64 MiB, partitions from 192 MiB, runs from 8 entries; the environment
-// variable SAT_SPMM_SRC_BLOCK = "<block bytes>[,<fit bytes>[,<min run>]]" overrides them for a process (0 = never blocked).
+// `min_run` entries on average; inside such a partition a row of `len` entries is cut into at most len / row_run groups of
+// blocks (sb_run).  Defaults: blocks of 64 MiB; partitions from 192 MiB whose rows meet a block with 8 entries on average;
+// row groups of at least 32 entries (measured on the 2.4 M-row graph: 0 / 8 / 16 / 32 / 64 entries give 6.47 / 6.26 / 6.11 /
+// 6.06 / 6.13 ms per d = 100 launch; work items 4.39 M -> 3.53 M, partial-sum rows 2.37 M -> 1.30 M).  The environment variable SAT_SPMM_SRC_BLOCK = "<block bytes>[,<fit bytes>[,<min run>[,<row run>]]]" overrides them for a
+// process (block bytes 0 = never blocked; row run 0 = every row cut at every block).
 struct SbConfig {
-    int64_t block_rows, fit_rows, min_run;
+    int64_t block_rows, fit_rows, min_run, row_run;
 };
 static SbConfig sb_config(int32_t d4)
 {
-    int64_t block_bytes = (int64_t)64 << 20, fit_bytes = (int64_t)192 << 20, min_run = 8;
+    int64_t block_bytes = (int64_t)64 << 20, fit_bytes = (int64_t)192 << 20, min_run = 8, row_run = 32;
     if (const char *e = getenv("SAT_SPMM_SRC_BLOCK")) {
         char *end = nullptr;
         block_bytes = strtoll(e, &end, 10);
         fit_bytes = 3 * block_bytes;
         if (end && *end == ',') fit_bytes = strtoll(end + 1, &end, 10);
         if (end && *end == ',') min_run = strtoll(end + 1, &end, 10);
+        row_run = min_run;
+        if (end && *end == ',') row_run = strtoll(end + 1, &end, 10);
     }
-    SbConfig c{0, 0, min_run};
+    SbConfig c{0, 0, min_run, row_run};
     if (block_bytes > 0) {
         c.block_rows = std::max<int64_t>(64, block_bytes / ((int64_t)d4 * 16) / 64 * 64);
         c.fit_rows = fit_bytes / ((int64_t)d4 * 16);
@@ -579,7 +597,7 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
         const int64_t block_rows = cfg.block_rows, fit_rows = cfg.fit_rows, min_run = cfg.min_run;
         if (blocked) {
             SrcBlockedItems *sb = nullptr;
-            SAT_TRY(sb_build(ctx, block_rows, fit_rows, min_run, &sb));
+            SAT_TRY(sb_build(ctx, block_rows, fit_rows, min_run, cfg.row_run, &sb));
             const int32_t item0 = sb->h_item_off[a], n_items = sb->h_item_off[b] - item0;
             const int32_t mrow0 = sb->h_mrow_off[a], n_mrows = sb->h_mrow_off[b] - mrow0;
             const int64_t slot_base = sb->h_slot_off[a], n_slots = sb->h_slot_off[b] - slot_base;
@@ -649,7 +667,7 @@ extern "C" sat_status sat_spmm_plan(sat_ctx *ctx, int32_t part, int32_t d, int32
     int64_t items = v.n_items, slots = v.n_mitems;
     if (sb_view_blocked(ctx, v, cfg, &a, &b)) {
         SrcBlockedItems *sb = nullptr;
-        SAT_TRY(sb_build(ctx, cfg.block_rows, cfg.fit_rows, cfg.min_run, &sb));
+        SAT_TRY(sb_build(ctx, cfg.block_rows, cfg.fit_rows, cfg.min_run, cfg.row_run, &sb));
         for (int m = a; m < b; ++m) nb = std::max<int32_t>(nb, (int32_t)sb_blocks_of(ctx, m, cfg.block_rows, cfg.fit_rows, cfg.min_run));
         items = sb->h_item_off[b] - sb->h_item_off[a];
         slots = sb->h_slot_off[b] - sb->h_slot_off[a];

@@ -16,6 +16,7 @@ from tests.gpu_util import dev, dev2d, empty2d
 pytestmark = pytest.mark.gpu
 
 FORCED = "16384,16384,0"     # blocks of 16 KiB of source rows (at least 64 rows), every partition, runs of any length
+GROUPED = "16384,16384,0,6"  # the same cut, rows of fewer than 6 entries per block walked in groups of blocks (len / 6 groups)
 
 
 @pytest.fixture(scope="module")
@@ -30,8 +31,9 @@ def B():
     ("dense", 64, [0, 9], 2),     # rows of thousands of entries: runs longer than one 256-entry chunk inside a block
     ("odd", 1, [0, 2], 2),        # ragged widths 50 / 72 / 40
 ])
-def test_every_call_with_the_blocked_walk(B, monkeypatch, name, shrink, parts, warm):
-    monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", FORCED)
+@pytest.mark.parametrize("cut", [FORCED, GROUPED])
+def test_every_call_with_the_blocked_walk(B, monkeypatch, name, shrink, parts, warm, cut):
+    monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", cut)
     wl = make_workload(name, shrink=shrink)
     case = TL.Case(B, wl, warm)
     try:
@@ -92,6 +94,14 @@ def test_blocked_and_plain_walks_agree_and_the_plan_says_which_ran(B, monkeypatc
         B.sat_destroy(ctx)
 
 
+def B_items_forced(B, ctx, d, monkeypatch):
+    """Work items of the all-partition launch with every row cut at every block (the environment is left on GROUPED)."""
+    monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", FORCED)
+    n_items = B.sat_spmm_plan(ctx, B.SAT_ALL_PARTS, d)[1]
+    monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", GROUPED)
+    return n_items
+
+
 @pytest.mark.parametrize("kind", ["one_partition", "an_empty_partition", "random_assignment"])
 def test_degenerate_partitionings_with_the_blocked_walk(B, monkeypatch, kind):
     """No halo rows at all (one partition: the blocks cut the inner rows alone), a partition without any node, and a random
@@ -134,6 +144,12 @@ def test_degenerate_partitionings_with_the_blocked_walk(B, monkeypatch, kind):
         blocked = run(B.SAT_ALL_PARTS, 0, wl.n, 0, n_halo)
         B.sat_sync_status(ctx)
         assert np.max(np.abs(plain.astype(np.float64) - blocked)) <= 2e-6 * np.max(np.abs(plain))
+        monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", GROUPED)          # fewer, longer runs for the short rows: same sums again
+        plan_g = B.sat_spmm_plan(ctx, B.SAT_ALL_PARTS, d)
+        assert plan_g[0] > 1 and plan_g[1] < B_items_forced(B, ctx, d, monkeypatch)
+        grouped = run(B.SAT_ALL_PARTS, 0, wl.n, 0, n_halo)
+        assert np.max(np.abs(plain.astype(np.float64) - grouped)) <= 2e-6 * np.max(np.abs(plain))
+        monkeypatch.setenv("SAT_SPMM_SRC_BLOCK", FORCED)
         r0 = h0 = 0
         for m in range(M):
             n_m, b_m = sizes[m][0], sizes[m][1]
