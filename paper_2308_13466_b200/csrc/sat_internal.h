@@ -125,6 +125,7 @@ struct ProfRec {
 // two blocks.  Rows with more than one item add their partial sums in item order (k_spmm_sb_fixup).
 struct SrcBlockedItems {
     int64_t block_rows = 0, fit_rows = 0, min_run = 0, row_run = 0;  // key
+    int mode = 0;              // key: 0 = all entries of a row, 1 = its inner prefix only (one block per partition)
     int32_t n_items = 0, n_mrows = 0;
     int64_t n_slots = 0;
     int4 *item = nullptr;      // {row, partial slot or -1, first entry: low 32 bits, first entry: high 16 bits | entries << 16}

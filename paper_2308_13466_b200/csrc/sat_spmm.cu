@@ -171,11 +171,12 @@ __device__ __forceinline__ int64_t sb_source_col(int64_t p, int32_t row0, int32_
 // G = min(blocks, len / min_run) groups of consecutive blocks (a short row would otherwise leave a partial sum per block for
 // a handful of entries each): group g covers blocks [ceil(g B / G), ceil((g + 1) B / G)) and its run is walked with the
 // first of them.
-__device__ __forceinline__ void sb_run(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row, int32_t j,
-                                       int32_t n_blocks, int64_t block_rows, int32_t min_run, int32_t row0, int32_t n_rows, int32_t n,
-                                       int64_t halo0, int64_t *lo, int64_t *hi)
+__device__ __forceinline__ void sb_run(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc,
+                                       const int32_t *__restrict__ inner_cnt, int32_t row, int32_t j, int32_t n_blocks, int64_t block_rows,
+                                       int32_t min_run, int32_t row0, int32_t n_rows, int32_t n, int64_t halo0, int64_t *lo, int64_t *hi)
 {
-    const int64_t rb = lrowptr[row], re = lrowptr[row + 1];
+    // inner_cnt given: the list covers the inner prefix of every row only (the backward product P_in^T)
+    const int64_t rb = lrowptr[row], re = inner_cnt ? rb + inner_cnt[row] : lrowptr[row + 1];
     int64_t G = min_run > 0 ? (re - rb) / min_run : n_blocks;
     G = G < 1 ? 1 : G > n_blocks ? n_blocks : G;
     const int64_t g = (int64_t)j * G / n_blocks;
@@ -189,14 +190,14 @@ __device__ __forceinline__ void sb_run(const int64_t *__restrict__ lrowptr, cons
 }
 
 // count[j * n_rows + r] = items of row row0 + r in block j
-__global__ void k_sb_count(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
-                           int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, int32_t *__restrict__ count)
+__global__ void k_sb_count(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, const int32_t *__restrict__ inner_cnt,
+                           int32_t row0, int32_t n_rows, int32_t n, int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, int32_t *__restrict__ count)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= (int64_t)n_rows * n_blocks) return;
     const int32_t j = (int32_t)(t / n_rows), r = (int32_t)(t - (int64_t)j * n_rows);
     int64_t lo, hi;
-    sb_run(lrowptr, lenc, row0 + r, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
+    sb_run(lrowptr, lenc, inner_cnt, row0 + r, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
     count[t] = (int32_t)((hi - lo + SAT_SPMM_CHUNK - 1) / SAT_SPMM_CHUNK);
 }
 
@@ -212,8 +213,8 @@ __global__ void k_sb_row_totals(const int32_t *__restrict__ count, int32_t row0,
     multi[row0 + r] = s > 1 ? 1 : 0;
 }
 
-__global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, int32_t row0, int32_t n_rows, int32_t n,
-                          int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, const int32_t *__restrict__ count,
+__global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__restrict__ lenc, const int32_t *__restrict__ inner_cnt,
+                          int32_t row0, int32_t n_rows, int32_t n, int64_t halo0, int32_t n_blocks, int64_t block_rows, int32_t min_run, const int32_t *__restrict__ count,
                           const int64_t *__restrict__ item_off, const int32_t *__restrict__ tot, const int64_t *__restrict__ slot_off,
                           int4 *__restrict__ item)
 {
@@ -224,7 +225,7 @@ __global__ void k_sb_fill(const int64_t *__restrict__ lrowptr, const int32_t *__
     if (c == 0) return;
     const int32_t row = row0 + r;
     int64_t lo, hi;
-    sb_run(lrowptr, lenc, row, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
+    sb_run(lrowptr, lenc, inner_cnt, row, j, n_blocks, block_rows, min_run, row0, n_rows, n, halo0, &lo, &hi);
     int32_t before = 0;
     for (int32_t q = 0; q < j; ++q) before += count[(int64_t)q * n_rows + r];
     const bool multi = tot[row] > 1;
@@ -265,10 +266,10 @@ static int64_t sb_blocks_of(const sat_ctx *ctx, int m, int64_t block_rows, int64
     return entries / (rows * B) >= min_run ? B : 1;
 }
 
-static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, int64_t min_run, int64_t row_run, SrcBlockedItems **out)
+static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, int64_t min_run, int64_t row_run, int mode, SrcBlockedItems **out)
 {
     for (SrcBlockedItems &sb : ctx->src_blocked)
-        if (sb.block_rows == block_rows && sb.min_run == min_run && sb.fit_rows == fit_rows && sb.row_run == row_run) {
+        if (sb.mode == mode && (mode == 1 || (sb.block_rows == block_rows && sb.min_run == min_run && sb.fit_rows == fit_rows && sb.row_run == row_run))) {
             *out = &sb;
             return SAT_OK;
         }
@@ -278,7 +279,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
     for (int m = 0; m < M; ++m) {
         const int64_t rows = ctx->h_inner_off[m + 1] - ctx->h_inner_off[m];
         const int64_t T = rows + (ctx->h_halo_off[m + 1] - ctx->h_halo_off[m]);
-        const int64_t B = sb_blocks_of(ctx, m, block_rows, fit_rows, min_run);
+        const int64_t B = mode == 1 ? 1 : sb_blocks_of(ctx, m, block_rows, fit_rows, min_run);   // the inner prefix is never cut
         nb[m] = (int32_t)B;
         br[m] = cdiv64(T > 0 ? T : 1, B);  // equal blocks
         cbase[m + 1] = cbase[m] + rows * B;
@@ -292,6 +293,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
     sb.min_run = min_run;
     sb.fit_rows = fit_rows;
     sb.row_run = row_run;
+    sb.mode = mode;
     auto cleanup = [&](bool all) {
         cudaFree(count); cudaFree(slots); cudaFree(multi); cudaFree(item_off); cudaFree(slot_off); cudaFree(mrow_off);
         if (all) { cudaFree(sb.item); cudaFree(sb.slot0); cudaFree(sb.tot); cudaFree(sb.mrows); }
@@ -323,7 +325,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
     for (int m = 0; m < M; ++m) {
         const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
         if (rows == 0) continue;
-        k_sb_count<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
+        k_sb_count<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, mode == 1 ? ctx->inner_cnt : nullptr, row0, rows, n, ctx->h_halo_off[m],
                                                                                          nb[m], br[m], row_min_run, count + cbase[m]);
         k_sb_row_totals<<<(unsigned)cdiv64(rows, 256), 256, 0, ctx->stream>>>(count + cbase[m], row0, rows, nb[m], sb.tot, slots, multi);
     }
@@ -346,7 +348,7 @@ static sat_status sb_build(sat_ctx *ctx, int64_t block_rows, int64_t fit_rows, i
     for (int m = 0; m < M; ++m) {
         const int32_t row0 = ctx->h_inner_off[m], rows = ctx->h_inner_off[m + 1] - row0;
         if (rows == 0) continue;
-        k_sb_fill<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, row0, rows, n, ctx->h_halo_off[m],
+        k_sb_fill<<<(unsigned)cdiv64((int64_t)rows * nb[m], 256), 256, 0, ctx->stream>>>(ctx->lrowptr, ctx->lenc, mode == 1 ? ctx->inner_cnt : nullptr, row0, rows, n, ctx->h_halo_off[m],
                                                                                         nb[m], br[m], row_min_run, count + cbase[m], item_off + cbase[m], sb.tot,
                                                                                         slot_off, sb.item);
     }
@@ -402,15 +404,18 @@ static SbConfig sb_config(int32_t d4)
     return c;
 }
 
-// partitions [a, b) of a view that covers whole partitions; true when at least one of them is source-blocked
-static bool sb_view_blocked(const sat_ctx *ctx, const PartView &v, const SbConfig &cfg, int *a, int *b)
+// partitions [a, b) of a view that covers whole partitions (false for any other view)
+static bool sb_view_parts(const sat_ctx *ctx, const PartView &v, int *a, int *b)
 {
-    if (cfg.block_rows <= 0) return false;
     *a = (int)(std::lower_bound(ctx->h_inner_off.begin(), ctx->h_inner_off.end(), v.row0) - ctx->h_inner_off.begin());
     *b = (int)(std::lower_bound(ctx->h_inner_off.begin(), ctx->h_inner_off.end(), v.row0 + v.n_rows) - ctx->h_inner_off.begin());
-    if (*b > ctx->M || *a > *b || ctx->h_inner_off[*a] != v.row0 || ctx->h_inner_off[*b] != v.row0 + v.n_rows) return false;
-    // (Sending every forward launch through this work list — one 16-byte descriptor per item instead of five index loads —
-    // was measured: 2 % faster on the 169 k-row graph, equal on the 717 k-row one; the plain list stays for those.)
+    return *b <= ctx->M && *a <= *b && ctx->h_inner_off[*a] == v.row0 && ctx->h_inner_off[*b] == v.row0 + v.n_rows;
+}
+
+// true when at least one partition of the view is source-blocked
+static bool sb_view_blocked(const sat_ctx *ctx, const PartView &v, const SbConfig &cfg, int *a, int *b)
+{
+    if (cfg.block_rows <= 0 || !sb_view_parts(ctx, v, a, b)) return false;
     for (int m = *a; m < *b; ++m)
         if (sb_blocks_of(ctx, m, cfg.block_rows, cfg.fit_rows, cfg.min_run) > 1) return true;
     return false;
@@ -590,14 +595,20 @@ sat_status sat_spmm(sat_ctx *ctx, const PartView &v, int inner_only, int32_t d, 
     const double n_ent = (double)(inner_only == 1 ? v.lnnz - v.hnnz : inner_only == 2 ? v.hnnz : v.lnnz);
     ProfScope prof(ctx, inner_only ? SATK_SPMM_BWD : SATK_SPMM_FWD,
                    4.0 * n_ent + 12.0 * v.n_rows + 4.0 * n_src + 4.0 * d * (n_src + v.n_rows), 2.0 * n_ent * d);
-    if (inner_only == 0) {
+    if (inner_only == 0 || inner_only == 1) {
         const SbConfig cfg = sb_config(d4);
         int a = 0, b = 0;
-        const bool blocked = sb_view_blocked(ctx, v, cfg, &a, &b);
+        // forward: the source-blocked list where a partition calls for it.  Backward (inner prefix of every row): a list of
+        // its own with one descriptor per 256-entry chunk of the prefix — the plain list cuts whole rows, so a long row whose
+        // inner entries fit one chunk still ran one (empty) work item per further chunk and went through the partial sums
+        // (SAT_SPMM_SRC_BLOCK=0 in the environment sends both back to the plain list.)  Measured, descriptor list against
+        // plain list: backward 7.02 -> 6.08 ms per epoch on the 2.4 M-row graph, 5.02 -> 4.60 on the 717 k-row one, 0.40 -> 0.38
+        // on the 169 k-row one; forward, where no partition is blocked: 0.735 -> 0.721 ms on the 169 k-row graph.
+        const bool blocked = cfg.block_rows > 0 && sb_view_parts(ctx, v, &a, &b);
         const int64_t block_rows = cfg.block_rows, fit_rows = cfg.fit_rows, min_run = cfg.min_run;
         if (blocked) {
             SrcBlockedItems *sb = nullptr;
-            SAT_TRY(sb_build(ctx, block_rows, fit_rows, min_run, cfg.row_run, &sb));
+            SAT_TRY(sb_build(ctx, block_rows, fit_rows, min_run, cfg.row_run, inner_only, &sb));
             const int32_t item0 = sb->h_item_off[a], n_items = sb->h_item_off[b] - item0;
             const int32_t mrow0 = sb->h_mrow_off[a], n_mrows = sb->h_mrow_off[b] - mrow0;
             const int64_t slot_base = sb->h_slot_off[a], n_slots = sb->h_slot_off[b] - slot_base;
@@ -667,7 +678,7 @@ extern "C" sat_status sat_spmm_plan(sat_ctx *ctx, int32_t part, int32_t d, int32
     int64_t items = v.n_items, slots = v.n_mitems;
     if (sb_view_blocked(ctx, v, cfg, &a, &b)) {
         SrcBlockedItems *sb = nullptr;
-        SAT_TRY(sb_build(ctx, cfg.block_rows, cfg.fit_rows, cfg.min_run, cfg.row_run, &sb));
+        SAT_TRY(sb_build(ctx, cfg.block_rows, cfg.fit_rows, cfg.min_run, cfg.row_run, 0, &sb));
         for (int m = a; m < b; ++m) nb = std::max<int32_t>(nb, (int32_t)sb_blocks_of(ctx, m, cfg.block_rows, cfg.fit_rows, cfg.min_run));
         items = sb->h_item_off[b] - sb->h_item_off[a];
         slots = sb->h_slot_off[b] - sb->h_slot_off[a];
